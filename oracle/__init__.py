@@ -1,0 +1,116 @@
+"""ctypes loader for the CPU oracle (``bi_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  Importers: ``tests/``, the smoke check and the
+benchmark's CPU-baseline leg.  The CUDA package never imports this module, and
+this module imports nothing from the CUDA package.
+
+``build()`` compiles the C file with gcc next to it; ``run()`` marshals numpy
+arrays into the C entry point.  No arithmetic of the method lives here.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "bi_oracle.c")
+_LIB = os.path.join(_HERE, "libbi_oracle.so")
+_lib = None
+
+ALGOS = {"filter": 0, "vmp": 1, "mmp": 2}
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle shared library if it is missing or stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True, capture_output=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.bi_ref_run.restype = ctypes.c_int
+        lib.bi_ref_max_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def max_threads() -> int:
+    return int(_load().bi_ref_max_threads())
+
+
+def _ptr_array(arrs):
+    arr_t = ctypes.c_void_p * max(len(arrs), 1)
+    return arr_t(*[a.ctypes.data for a in arrs])
+
+
+def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G: int,
+        A, B, D, obs: np.ndarray, act: Optional[np.ndarray], K: int, *,
+        q_init: Optional[np.ndarray] = None, threads: int = 0, round32: bool = False):
+    """Run ``algo`` ('filter' | 'vmp' | 'mmp') and return ``(q, logq, argmax)``.
+
+    ``obs`` is ``[N, T, M]`` int32, ``act`` ``[N, T-1, F]`` int32 (ignored when
+    T == 1); ``q`` and ``logq`` come back as float64 ``[N, T, S]``, ``argmax`` as
+    int32 ``[N, T, F]``.
+    """
+    lib = _load()
+    n = np.ascontiguousarray(n, dtype=np.int32)
+    m = np.ascontiguousarray(m, dtype=np.int32)
+    U = np.ascontiguousarray(U, dtype=np.int32)
+    F, M = len(n), len(m)
+    dep_len = np.ascontiguousarray([len(d) for d in dep], dtype=np.int32)
+    dep_flat = np.ascontiguousarray([f for d in dep for f in d] or [0], dtype=np.int32)
+    A = [np.ascontiguousarray(a, dtype=np.float32) for a in A]
+    B = [np.ascontiguousarray(b, dtype=np.float32) for b in B]
+    D = [np.ascontiguousarray(d, dtype=np.float32) for d in D]
+    obs = np.ascontiguousarray(obs, dtype=np.int32)
+    N, T = int(obs.shape[0]), int(obs.shape[1])
+    assert obs.shape == (N, T, M)
+    if T > 1:
+        act = np.ascontiguousarray(act, dtype=np.int32)
+        assert act.shape == (N, T - 1, F)
+        act_p = act.ctypes.data
+    else:
+        act_p = None
+    S = int(n.sum())
+    for i, a in enumerate(A):
+        assert a.shape == (G, int(m[i])) + tuple(int(n[f]) for f in dep[i]), (i, a.shape)
+    for f in range(F):
+        assert B[f].shape == (G, int(n[f]), int(n[f]), int(U[f])), (f, B[f].shape)
+        assert D[f].shape == (G, int(n[f]))
+    q = np.empty((N, T, S), dtype=np.float64)
+    lq = np.empty((N, T, S), dtype=np.float64)
+    am = np.empty((N, T, F), dtype=np.int32)
+    if q_init is not None:
+        q_init = np.ascontiguousarray(q_init, dtype=np.float64)
+        assert q_init.shape == (N, T, S)
+    Ap, Bp, Dp = _ptr_array(A), _ptr_array(B), _ptr_array(D)
+    rc = lib.bi_ref_run(
+        ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),
+        ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),
+        ctypes.c_void_p(dep_len.ctypes.data), ctypes.c_void_p(dep_flat.ctypes.data),
+        ctypes.c_void_p(U.ctypes.data), ctypes.c_int(G), Ap, Bp, Dp,
+        ctypes.c_int(N), ctypes.c_int(T), ctypes.c_void_p(obs.ctypes.data),
+        ctypes.c_void_p(act_p), ctypes.c_int(K),
+        ctypes.c_void_p(q_init.ctypes.data if q_init is not None else None),
+        ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(lq.ctypes.data),
+        ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads), ctypes.c_int(int(round32)))
+    if rc != 0:
+        raise ValueError(f"bi_ref_run rejected its arguments (code {rc})")
+    return q, lq, am
+
+
+def run_workload(w, algo: Optional[str] = None, **kw):
+    """Convenience: run on an object with the workload generator's field names."""
+    return run(algo or w.algo, w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, w.obs, w.act, w.K, **kw)

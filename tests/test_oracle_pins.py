@@ -1,0 +1,315 @@
+"""Pins for the CPU oracle: closed forms, brute-force enumeration, invariants.
+
+The oracle is the yardstick for the CUDA path, so it is checked here against
+things that are not itself: hand-derived fixtures, the textbook HMM forward
+recursion, enumeration of every joint trajectory of tiny models (the model's
+definition, Section III-B, and the generic coordinate update, Section III-A),
+and metamorphic properties (the paper's claim that padding / regrouping never
+changes results).
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from biwl import make_config, make_model, sample_streams
+from bruteforce import TinyModel, hmm_forward
+from conftest import read_golden
+
+
+def tiny(seed, n, m, dep, U, T, *, sparsity=0.0, d_alpha=1.0, N=1):
+    rng = np.random.default_rng(seed)
+    A, B, D = make_model(rng, n, m, dep, U, 1, sparsity=sparsity, d_alpha=d_alpha)
+    obs, act = sample_streams(rng, n, m, dep, U, 1, A, B, D, N, T)
+    return dict(n=n, m=m, dep=dep, U=U, G=1, A=A, B=B, D=D, obs=obs, act=act)
+
+
+def run(algo, w, K, **kw):
+    return oracle.run(algo, w["n"], w["m"], w["dep"], w["U"], w["G"], w["A"], w["B"], w["D"],
+                      w["obs"], w["act"], K, **kw)
+
+
+def tm(w, a=0):
+    return TinyModel(w["n"], w["m"], w["dep"], w["U"], w["A"], w["B"], w["D"], w["obs"][a], w["act"][a])
+
+
+# ---- P1: single factor filtering is exact Bayes --------------------------------
+
+def test_golden_two_state_hmm(golden_dir):
+    g = read_golden(os.path.join(golden_dir, "hmm_two_state.txt"))
+    A = [g["A"].reshape(1, 2, 2).astype(np.float32)]
+    B = [g["B"].reshape(1, 2, 2, 1).astype(np.float32)]
+    D = [g["D"].reshape(1, 2).astype(np.float32)]
+    obs = g["obs"].astype(np.int32).reshape(1, 2, 1)
+    act = np.zeros((1, 1, 1), np.int32)
+    for K in (1, 2, 7):
+        q, lq, am = oracle.run("filter", [2], [2], [[0]], [1], 1, A, B, D, obs, act, K)
+        np.testing.assert_allclose(q[0, 0], g["q1"], atol=2e-7)
+        np.testing.assert_allclose(q[0, 1], g["q2"], atol=2e-7)
+        np.testing.assert_allclose(np.exp(lq), q, atol=1e-14)
+        assert am.tolist() == [[[0], [1]]]
+
+
+def test_golden_state_independent_transition(golden_dir):
+    g = read_golden(os.path.join(golden_dir, "state_independent_transition.txt"))
+    A = [g["A"].reshape(1, 2, 2).astype(np.float32)]
+    B = [np.repeat(g["pi"].reshape(1, 2, 1, 1), 2, axis=2).astype(np.float32)]
+    D = [g["D"].reshape(1, 2).astype(np.float32)]
+    obs = g["obs"].astype(np.int32).reshape(1, 3, 1)
+    act = np.zeros((1, 2, 1), np.int32)
+    for K in (1, 3):
+        qv, _, _ = oracle.run("vmp", [2], [2], [[0]], [1], 1, A, B, D, obs, act, K)
+        qm, _, _ = oracle.run("mmp", [2], [2], [[0]], [1], 1, A, B, D, obs, act, K)
+        for q, key in ((qv, "q_vmp"), (qm, "q_mmp")):
+            np.testing.assert_allclose(q[0, 0], g["q_first"], atol=2e-7)
+            np.testing.assert_allclose(q[0, 1], g[key], atol=2e-7)
+            np.testing.assert_allclose(q[0, 2], g[key], atol=2e-7)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_single_factor_filter_is_forward_recursion(seed):
+    w = tiny(seed, [5], [4], [[0]], [3], T=8, N=3)
+    for K in (1, 4):
+        q, lq, am = run("filter", w, K)
+        for a in range(3):
+            ref = hmm_forward(w["A"][0][0], w["B"][0][0], w["D"][0][0], w["obs"][a, :, 0], w["act"][a, :, 0])
+            np.testing.assert_allclose(q[a], ref, atol=1e-12)
+            np.testing.assert_allclose(lq[a], np.log(ref), atol=1e-10)
+            assert (am[a, :, 0] == ref.argmax(axis=1)).all()
+
+
+def test_single_factor_filter_matches_enumeration():
+    w = tiny(5, [3], [3], [[0]], [2], T=4)
+    q, _, _ = run("filter", w, 2)
+    np.testing.assert_allclose(q[0], tm(w).exact_filter_marginals(), atol=1e-12)
+
+
+# ---- P2: every modality on one factor -> factors decouple ------------------------
+
+def test_decoupled_factors_are_exact_and_independent_of_K():
+    w = tiny(7, [3, 2], [3, 2, 2], [[0], [1], [0]], [2, 1], T=3)
+    exact = tm(w).exact_filter_marginals()
+    for K in (1, 5):
+        q, _, _ = run("filter", w, K)
+        np.testing.assert_allclose(q[0], exact, atol=1e-12)
+
+
+# ---- P3: the update is the coordinate optimum of Section III-A --------------------
+
+@pytest.mark.parametrize("seed,sparsity", [(11, 0.0), (12, 0.5)])
+def test_vmp_update_is_enumerated_coordinate_optimum(seed, sparsity):
+    w = tiny(seed, [2, 3], [2, 3], [[0, 1], [1, 0]], [2, 1], T=3, sparsity=sparsity)
+    model = tm(w)
+    rng = np.random.default_rng(seed)
+    S = 5
+    q0 = np.concatenate([rng.dirichlet(np.ones(2), size=3), rng.dirichlet(np.ones(3), size=3)], axis=1)
+    q1, _, _ = run("vmp", w, 1, q_init=q0[None])
+    for t in range(3):
+        for f in range(2):
+            want = model.coordinate_optimum(q0, t, f)
+            got = q1[0, t, model.off[f]:model.off[f + 1]]
+            np.testing.assert_allclose(got, want, atol=1e-12)
+    assert q1.shape == (1, 3, S)
+
+
+def test_filter_step_is_enumerated_coordinate_optimum():
+    # One filtering step is the T = 1 problem whose initial-state prior is the
+    # predictive prior; with T = 1 the prior is D.
+    w = tiny(21, [3, 2, 2], [3, 2], [[0, 1, 2], [2, 0]], [1, 1, 1], T=1)
+    model = tm(w)
+    rng = np.random.default_rng(3)
+    q0 = np.concatenate([rng.dirichlet(np.ones(k), size=1) for k in (3, 2, 2)], axis=1)
+    q1, _, _ = run("filter", w, 1, q_init=q0[None])
+    for f in range(3):
+        np.testing.assert_allclose(q1[0, 0, model.off[f]:model.off[f + 1]],
+                                   model.coordinate_optimum(q0, 0, f), atol=1e-12)
+
+
+def test_filter_recursion_uses_predictive_prior():
+    # Step 2 of the filter equals a fresh one-step problem whose D is B_u q_1.
+    w = tiny(22, [3, 2], [3, 2], [[0, 1], [1]], [2, 2], T=2)
+    q, _, _ = run("filter", w, 6)
+    D2 = []
+    for f, (lo, hi) in enumerate([(0, 3), (3, 5)]):
+        Bu = w["B"][f][0][:, :, w["act"][0, 0, f]].astype(np.float64)
+        D2.append((Bu @ q[0, 0, lo:hi]).astype(np.float32)[None])
+    w2 = dict(w, D=D2, obs=w["obs"][:, 1:], act=w["act"][:, :0])
+    q2, _, _ = run("filter", w2, 6)
+    np.testing.assert_allclose(q2[0, 0], q[0, 1], atol=5e-7)
+
+
+def test_free_energy_never_increases_under_coordinate_updates():
+    w = tiny(31, [2, 2], [2, 2], [[0, 1], [0]], [2, 2], T=3)
+    model = tm(w)
+    rng = np.random.default_rng(0)
+    q = np.concatenate([rng.dirichlet(np.ones(2), size=3), rng.dirichlet(np.ones(2), size=3)], axis=1)
+    f_prev = model.free_energy(q)
+    assert f_prev >= -model.ln_evidence() - 1e-12
+    for sweep in range(3):
+        for t, f in itertools.product(range(3), range(2)):
+            upd, _, _ = run("vmp", w, 1, q_init=q[None])
+            cand = q.copy()
+            cand[t, model.off[f]:model.off[f + 1]] = upd[0, t, model.off[f]:model.off[f + 1]]
+            f_new = model.free_energy(cand)
+            assert f_new <= f_prev + 1e-12
+            # the coordinate minimiser beats random alternatives at that coordinate
+            for _ in range(5):
+                alt = q.copy()
+                alt[t, model.off[f]:model.off[f + 1]] = rng.dirichlet(np.ones(2))
+                assert model.free_energy(alt) >= f_new - 1e-12
+            q, f_prev = cand, f_new
+    assert f_prev >= -model.ln_evidence() - 1e-12
+
+
+def test_jacobi_schedule_composes():
+    # K iterations from a start equal K single iterations chained: every
+    # coordinate of iteration k+1 reads iteration k only.
+    w = tiny(41, [3, 2], [2, 3], [[0, 1], [1]], [2, 1], T=4, N=2)
+    for algo in ("vmp", "mmp"):
+        q3, _, _ = run(algo, w, 3)
+        q = None
+        for _ in range(3):
+            q, _, _ = run(algo, w, 1, q_init=q)
+        np.testing.assert_allclose(q, q3, atol=1e-14)
+
+
+# ---- P4: window edge conventions ------------------------------------------------
+
+def test_single_step_window_equals_filter_step():
+    w = tiny(51, [4, 3], [3, 4], [[0, 1], [1, 0]], [2, 2], T=1, N=4)
+    qf, lf, af = run("filter", w, 5)
+    for algo in ("vmp", "mmp"):
+        q, lq, am = run(algo, w, 5)
+        np.testing.assert_allclose(q, qf, atol=1e-12)
+        np.testing.assert_allclose(lq, lf, atol=1e-12)
+        assert (am == af).all()
+
+
+# ---- P8: normalisation ------------------------------------------------------------
+
+@pytest.mark.parametrize("algo", ["filter", "vmp", "mmp"])
+def test_beliefs_are_distributions(algo):
+    w = make_config(1)
+    q, lq, am = oracle.run_workload(w, algo)
+    assert (q >= 0).all()
+    off = np.concatenate([[0], np.cumsum(w.n)])
+    for f in range(w.F):
+        blk = q[..., off[f]:off[f + 1]]
+        np.testing.assert_allclose(blk.sum(-1), 1.0, atol=1e-12)
+        assert (blk.argmax(-1) == am[..., f]).all()
+    np.testing.assert_allclose(np.exp(lq), q, atol=1e-12)
+
+
+# ---- metamorphic properties ---------------------------------------------------------
+
+def _base(seed=61, T=4, N=3):
+    return tiny(seed, [3, 4, 2], [3, 2, 4], [[0, 1], [1, 2], [2, 0, 1]], [2, 3, 1], T=T, N=N, sparsity=0.5)
+
+
+@pytest.mark.parametrize("algo", ["filter", "vmp", "mmp"])
+def test_modality_permutation(algo):
+    w = _base()
+    q, _, _ = run(algo, w, 4)
+    perm = [2, 0, 1]
+    w2 = dict(w, m=[w["m"][i] for i in perm], dep=[w["dep"][i] for i in perm],
+              A=[w["A"][i] for i in perm], obs=w["obs"][:, :, perm])
+    q2, _, _ = run(algo, w2, 4)
+    np.testing.assert_allclose(q2, q, atol=1e-12)
+
+
+@pytest.mark.parametrize("algo", ["filter", "vmp", "mmp"])
+def test_state_relabelling(algo):
+    w = _base()
+    q, _, _ = run(algo, w, 4)
+    p = np.array([2, 0, 3, 1])  # new label j holds old state p[j] of factor 1
+    A = [np.ascontiguousarray(np.take(w["A"][0], p, axis=3)),
+         np.ascontiguousarray(np.take(w["A"][1], p, axis=2)),
+         np.ascontiguousarray(np.take(w["A"][2], p, axis=4))]
+    B = list(w["B"])
+    B[1] = np.ascontiguousarray(w["B"][1][:, p][:, :, p])
+    D = list(w["D"])
+    D[1] = np.ascontiguousarray(w["D"][1][:, p])
+    q2, _, _ = run(algo, dict(w, A=A, B=B, D=D), 4)
+    want = q.copy()
+    want[..., 3:7] = q[..., 3:7][..., p]
+    np.testing.assert_allclose(q2, want, atol=1e-12)
+
+
+@pytest.mark.parametrize("algo", ["filter", "vmp", "mmp"])
+def test_uninformative_modality_and_dependency_superset(algo):
+    w = _base()
+    q, _, _ = run(algo, w, 4)
+    N, T = w["obs"].shape[:2]
+    # a modality whose A does not depend on the outcome
+    const = np.full((1, 3, 4), 1.0 / 3.0, np.float32)
+    w2 = dict(w, m=w["m"] + [3], dep=w["dep"] + [[1]], A=w["A"] + [const],
+              obs=np.concatenate([w["obs"], np.ones((N, T, 1), np.int32)], axis=2))
+    q2, _, _ = run(algo, w2, 4)
+    np.testing.assert_allclose(q2, q, atol=1e-12)
+    # modality 1 (deps [1,2]) declared on the superset [1,2,0], A replicated along the new axis
+    rep = np.ascontiguousarray(np.repeat(w["A"][1][..., None], 3, axis=-1))
+    dep = [w["dep"][0], [1, 2, 0], w["dep"][2]]
+    q3, _, _ = run(algo, dict(w, dep=dep, A=[w["A"][0], rep, w["A"][2]]), 4)
+    np.testing.assert_allclose(q3, q, atol=1e-12)
+
+
+@pytest.mark.parametrize("algo", ["filter", "vmp", "mmp"])
+def test_unobserved_and_singleton_factors(algo):
+    w = _base()
+    q, _, _ = run(algo, w, 4)
+    N, T = w["obs"].shape[:2]
+    rng = np.random.default_rng(9)
+    # add a factor with one state and a factor no modality depends on
+    Bx = rng.dirichlet(np.ones(3), size=(3, 2)).transpose(2, 0, 1)[None].astype(np.float32)  # [1,3,3,2]
+    Dx = rng.dirichlet(np.ones(3))[None].astype(np.float32)
+    act_x = rng.integers(0, 2, size=(N, T - 1, 1)).astype(np.int32)
+    w2 = dict(w, n=w["n"] + [1, 3], U=w["U"] + [1, 2],
+              B=w["B"] + [np.ones((1, 1, 1, 1), np.float32), Bx],
+              D=w["D"] + [np.ones((1, 1), np.float32), Dx],
+              act=np.concatenate([w["act"], np.zeros((N, T - 1, 1), np.int32), act_x], axis=2))
+    q2, _, _ = run(algo, w2, 4)
+    np.testing.assert_allclose(q2[..., :9], q, atol=1e-12)
+    np.testing.assert_allclose(q2[..., 9], 1.0, atol=1e-15)
+    if algo == "filter":
+        # the unobserved factor just follows its transition recursion
+        for a in range(N):
+            p = Dx[0].astype(np.float64)
+            for t in range(T):
+                if t > 0:
+                    p = Bx[0][:, :, act_x[a, t - 1, 0]].astype(np.float64) @ p
+                np.testing.assert_allclose(q2[a, t, 10:], p / p.sum(), atol=1e-12)
+
+
+@pytest.mark.parametrize("algo", ["filter", "vmp", "mmp"])
+def test_shared_vs_replicated_model_and_batch_independence(algo):
+    w = _base(N=4)
+    q, _, am = run(algo, w, 3)
+    rep = dict(w, G=4, A=[np.repeat(a, 4, axis=0) for a in w["A"]],
+               B=[np.repeat(b, 4, axis=0) for b in w["B"]], D=[np.repeat(d, 4, axis=0) for d in w["D"]])
+    q2, _, am2 = run(algo, rep, 3)
+    assert np.array_equal(q2, q) and np.array_equal(am2, am)
+    sub = dict(w, obs=w["obs"][[2]], act=w["act"][[2]])
+    q3, _, _ = run(algo, sub, 3)
+    assert np.array_equal(q3[0], q[2])
+
+
+def test_threads_do_not_change_results():
+    w = make_config(1)
+    a = oracle.run_workload(w, threads=1)
+    b = oracle.run_workload(w, threads=4)
+    assert all(np.array_equal(x, y) for x, y in zip(a, b))
+
+
+def test_zero_probabilities_use_the_clamped_log():
+    # A with exact zeros: an observed outcome that is impossible under a state
+    # drives that state's belief to (numerically) zero but stays finite.
+    A = [np.array([[[1.0, 0.5], [0.0, 0.5]]], np.float32)]
+    B = [np.eye(2, dtype=np.float32).reshape(1, 2, 2, 1)]
+    D = [np.array([[0.5, 0.5]], np.float32)]
+    q, lq, _ = oracle.run("filter", [2], [2], [[0]], [1], 1, A, B, D,
+                          np.array([[[1]]], np.int32), None, 2)
+    want = np.array([1e-16, 0.5]) / (1e-16 + 0.5)
+    np.testing.assert_allclose(q[0, 0], want, rtol=1e-12)
+    assert np.isfinite(lq).all()
