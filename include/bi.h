@@ -1,0 +1,179 @@
+/*
+ * bi -- batched mean-field belief updates for factorised discrete HMMs/POMDPs
+ * on NVIDIA B200 (sm_100a).  C ABI; no C++ or framework types cross it.
+ *
+ * Model (Section III-B of the paper): M observation modalities, F hidden-state
+ * factors with n_f states, one control per factor with U_f actions;
+ *   p(o, s | u) = p(s_1) prod_{t>=2} p(s_t | s_{t-1}, u_{t-1}; B) prod_t p(o_t | s_t; A).
+ * A_i = P(o^i | s^{dep(i)}) for an arbitrary dependency list dep(i);
+ * B_f = P(s^f_{t+1} | s^f_t, u^f_t) (trivial B-dependencies only).
+ *
+ * Every inference entry point computes, for N independent agents, the
+ * posterior marginals q_{t,f} of a fully factorised approximation by iterating
+ * the generic coordinate update of Section III-A,
+ *   log q(s^f) = E_{q(s^{\f})}[ log p(o, s) ] + const,
+ * whose expensive part is the likelihood message (Section III-C log-likelihood
+ * with the observed outcome selecting a slice of log A_i, then the
+ * marginalisation of Section IV):
+ *   ell_{t,f}[s] = sum_{i: f in dep(i)} sum_{s_dep(i) \ f}
+ *                  ln A_i[o_{t,i}, s_dep(i)] prod_{g in dep(i), g != f} q_{t,g}[s_g].
+ * Conventions the paper leaves open and this library fixes:
+ *   - all (t, f) are updated simultaneously from the previous iterate (Jacobi;
+ *     the paper maps the window's steps onto parallel threads, Appendix A-2);
+ *   - beliefs start uniform; exactly `iters` iterations run, no early exit;
+ *   - ln x means ln(max(x, 1e-16)).
+ *
+ * Pointers are marked HOST or DEVICE.  All arrays are dense, row-major.
+ * Inference calls are asynchronous on the given CUDA stream (a cudaStream_t
+ * passed as void*, NULL = default stream) and never synchronise; the caller
+ * owns every pointer it passes.  Nothing in this library falls back to the
+ * CPU: without a usable CUDA device every call fails with BI_ERR_CUDA.
+ */
+#ifndef BI_H
+#define BI_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* compile-time limits; exceeding one returns BI_ERR_UNSUPPORTED */
+#define BI_MAX_F 8      /* hidden-state factors              */
+#define BI_MAX_M 16     /* observation modalities            */
+#define BI_MAX_RANK 5   /* factors one modality may depend on */
+#define BI_MAX_N 32     /* states per factor                 */
+#define BI_MAX_T 64     /* steps per window call (bi_vmp / bi_mmp) */
+
+enum {
+  BI_OK = 0,
+  BI_ERR_INVALID_ARG = -1, /* null pointer, non-positive count, bad dependency id   */
+  BI_ERR_SHAPE = -2,       /* N / G mismatch, repeated factor in a dependency list  */
+  BI_ERR_UNSUPPORTED = -3, /* a BI_MAX_* limit or the on-chip working set exceeded  */
+  BI_ERR_ALLOC = -4,       /* device allocation failed                              */
+  BI_ERR_CUDA = -5         /* a CUDA runtime call failed / no device                */
+};
+
+/*
+ * Arithmetic of the inference kernels.  Inputs and outputs are float32 either
+ * way.  The Jacobi fixed-point map is not contractive on sharp or sparse
+ * models (beliefs can oscillate between iterations), so rounding errors are
+ * amplified by factors that reach 1e3 on dense models and 1e9 on sparse ones
+ * within 16 iterations; float32 arithmetic then cannot reproduce a float64
+ * evaluation to 1e-5.  BI_ARITH_F64 (the default) carries logs, beliefs and
+ * accumulations in float64; BI_ARITH_F32 is the fast mode, exact to float32
+ * rounding per operation but not to 1e-5 on ill-conditioned agents.
+ */
+#define BI_ARITH_F64 0
+#define BI_ARITH_F32 1
+
+/* bits of the device status word read by bi_status */
+#define BI_FLAG_OBS_RANGE 1u /* an observation index was outside [0, m_i): clamped */
+#define BI_FLAG_ACT_RANGE 2u /* an action index was outside [0, U_f): clamped      */
+
+typedef struct bi_model bi_model_t; /* opaque; owns the packed device copies */
+
+/*
+ * Description of a generative model (the tuple that defines a POMDP
+ * configuration in Section V-A, plus action counts and the arrays).
+ */
+typedef struct {
+  int32_t F, M;
+  const int32_t *n;       /* HOST [F]  state counts, 1 <= n_f <= BI_MAX_N          */
+  const int32_t *m;       /* HOST [M]  outcome counts, m_i >= 1                    */
+  const int32_t *dep_len; /* HOST [M]  k_i, 1 <= k_i <= BI_MAX_RANK                */
+  const int32_t *dep;     /* HOST [sum k_i] 0-based factor ids, no repeats within a
+                             list; A_i's hidden axes follow this order             */
+  const int32_t *U;       /* HOST [F]  action counts, U_f >= 1                     */
+  int32_t G;              /* 1: one model shared by all agents; else one per agent */
+  const float *const *A;  /* HOST array of M DEVICE pointers;
+                             A[i]: [G][m_i][n_dep(i)[0]]...[n_dep(i)[k_i-1]]       */
+  const float *const *B;  /* HOST array of F DEVICE pointers;
+                             B[f]: [G][n_f next][n_f previous][U_f]                */
+  const float *const *D;  /* HOST array of F DEVICE pointers; D[f]: [G][n_f]       */
+} bi_model_desc;
+
+/*
+ * Pack a model for inference (the once-only initialisation step of Section
+ * III-C: layout work happens here, never at inference time).  Computes
+ * ln(max(A, 1e-16)) in float64 (rounded once to float32 in BI_ARITH_F32), stores each
+ * outcome's slice contiguously with modalities of equal dependency set sharing
+ * one axis order; B is re-laid per action as forward, log, log-transposed and
+ * column-normalised-transposed matrices; D as ln D.  The packed copies live in
+ * device memory owned by the handle; the caller's A, B, D may be released once
+ * the stream's work has completed.  Returns BI_OK and *out, or an error code
+ * with *out = NULL.
+ */
+int bi_model_create(const bi_model_desc *desc, void *cuda_stream, bi_model_t **out);
+
+/* As bi_model_create (which uses BI_ARITH_F64) with the arithmetic chosen. */
+int bi_model_create_arith(const bi_model_desc *desc, int arith, void *cuda_stream, bi_model_t **out);
+
+/* BI_ARITH_* of a handle, or BI_ERR_INVALID_ARG for NULL. */
+int bi_model_arith(const bi_model_t *model);
+
+/* Synchronises the device, frees the packed copies.  NULL is accepted. */
+int bi_model_destroy(bi_model_t *model);
+
+/*
+ * Variational filtering by fixed-point iteration ("FPI", Sections I and IV).
+ * For each agent and t = 1..T in order:
+ *   prior_t = D (t = 1) or B_{u_{t-1}} q_{t-1} (final belief of step t-1),
+ *   q <- uniform; repeat `iters` times, all factors at once:
+ *   q_{t,f} <- softmax( ell_{t,f}(q) + ln prior_{t,f} ).
+ *
+ *   N, T      agents, time steps (N >= 0, T >= 1); if model G != 1 then N == G
+ *   obs       DEVICE [N][T][M]   int32, 0 <= obs < m_i
+ *   act       DEVICE [N][T-1][F] int32, 0 <= act < U_f; may be NULL when T == 1
+ *   iters     K >= 1
+ *   q_out     DEVICE [N][T][S] float32, S = sum n_f, factor f at offset sum_{g<f} n_g
+ *   logq_out  DEVICE [N][T][S] float32 log-beliefs, or NULL
+ *   argmax_out DEVICE [N][T][F] int32 most probable state (lowest index on ties), or NULL
+ * Out-of-range indices are clamped and flagged in the status word; nothing traps.
+ */
+int bi_filter(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+              const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+              int32_t *argmax_out, void *cuda_stream);
+
+/*
+ * Variational message passing over one window of T steps (Sections I, IV and
+ * Appendix A-2).  All (t, f) at once, `iters` times:
+ *   q_{t,f} <- softmax( ell_{t,f}(q_t) + past + future ),
+ *   past   = ln D_f (t = 1) or (ln B_{u_{t-1}}) q_{t-1,f},
+ *   future = 0 (t = T) or (ln B_{u_t})^T q_{t+1,f}.
+ * Arguments as bi_filter; T <= BI_MAX_T.
+ */
+int bi_vmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+           const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+           int32_t *argmax_out, void *cuda_stream);
+
+/*
+ * Marginal message passing over one window of T steps.  Same loop as bi_vmp with
+ *   past   = ln D_f (t = 1) or 1/2 ln( B_{u_{t-1}} q_{t-1,f} ),
+ *   future = 0 (t = T) or 1/2 ln( Bdag_{u_t} q_{t+1,f} ),
+ * Bdag = transpose of B_u with each column renormalised (zero sum -> uniform).
+ * The paper names the algorithm and cites its source without printing these
+ * formulas; this is the library's stated reading of it.
+ */
+int bi_mmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+           const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+           int32_t *argmax_out, void *cuda_stream);
+
+/* Synchronises the stream, returns the OR of BI_FLAG_* raised since the last
+ * call in *flags (HOST) and clears them. */
+int bi_status(const bi_model_t *model, void *cuda_stream, uint32_t *flags);
+
+/* Name of the kernel family the dispatcher picked for the most recent
+ * inference call on this handle ("" before the first call).  Static storage. */
+const char *bi_last_kernel(const bi_model_t *model);
+
+/* Number of kernel launches issued by inference calls on this handle so far. */
+int64_t bi_launch_count(const bi_model_t *model);
+
+/* Human-readable text for an error code.  Static storage. */
+const char *bi_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BI_H */

@@ -1,0 +1,197 @@
+"""Python binding for the ``bi`` CUDA library (B200 / sm_100a).
+
+Argument marshalling only: every step of the belief-update path runs in the
+library's kernels.  PyTorch supplies device memory and the current stream.
+There is no CPU path; importing works without a GPU (so the build and the
+symbol table can be checked), but every compute call needs a CUDA device and
+fails loudly without one.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+from .build import LIB, build  # noqa: F401
+
+_lib = None
+
+BI_OK = 0
+ERRORS = {0: "BI_OK", -1: "BI_ERR_INVALID_ARG", -2: "BI_ERR_SHAPE", -3: "BI_ERR_UNSUPPORTED",
+          -4: "BI_ERR_ALLOC", -5: "BI_ERR_CUDA"}
+BI_FLAG_OBS_RANGE = 1
+BI_FLAG_ACT_RANGE = 2
+
+BI_ARITH_F64 = 0
+BI_ARITH_F32 = 1
+ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
+
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_vmp", "bi_mmp", "bi_status",
+           "bi_last_kernel", "bi_launch_count", "bi_strerror"]
+
+
+class BiError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {ERRORS.get(code, code)} ({lib().bi_strerror(code).decode()})")
+
+
+class _Desc(ctypes.Structure):
+    _fields_ = [("F", ctypes.c_int32), ("M", ctypes.c_int32),
+                ("n", ctypes.c_void_p), ("m", ctypes.c_void_p), ("dep_len", ctypes.c_void_p),
+                ("dep", ctypes.c_void_p), ("U", ctypes.c_void_p), ("G", ctypes.c_int32),
+                ("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("D", ctypes.c_void_p)]
+
+
+def lib():
+    """Load libbi.so (building it if the sources are newer).  Raises if it cannot be loaded."""
+    global _lib
+    if _lib is None:
+        path = build()
+        L = ctypes.CDLL(path)
+        L.bi_model_create.restype = ctypes.c_int
+        L.bi_model_create.argtypes = [ctypes.POINTER(_Desc), ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)]
+        L.bi_model_create_arith.restype = ctypes.c_int
+        L.bi_model_create_arith.argtypes = [ctypes.POINTER(_Desc), ctypes.c_int, ctypes.c_void_p,
+                                            ctypes.POINTER(ctypes.c_void_p)]
+        L.bi_model_arith.restype = ctypes.c_int
+        L.bi_model_arith.argtypes = [ctypes.c_void_p]
+        L.bi_model_destroy.restype = ctypes.c_int
+        L.bi_model_destroy.argtypes = [ctypes.c_void_p]
+        for name in ("bi_filter", "bi_vmp", "bi_mmp"):
+            fn = getattr(L, name)
+            fn.restype = ctypes.c_int
+            fn.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                           ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.bi_status.restype = ctypes.c_int
+        L.bi_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
+        L.bi_last_kernel.restype = ctypes.c_char_p
+        L.bi_last_kernel.argtypes = [ctypes.c_void_p]
+        L.bi_launch_count.restype = ctypes.c_int64
+        L.bi_launch_count.argtypes = [ctypes.c_void_p]
+        L.bi_strerror.restype = ctypes.c_char_p
+        L.bi_strerror.argtypes = [ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def _i32(vals):
+    arr = (ctypes.c_int32 * max(len(vals), 1))(*[int(v) for v in vals])
+    return arr
+
+
+def _stream_ptr(stream=None):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class Model:
+    """A packed generative model on the current CUDA device (``bi_model_create``).
+
+    ``A[i]``, ``B[f]``, ``D[f]`` are float32 CUDA tensors laid out as the
+    header documents: ``A[i]: [G, m_i, n_dep...]``, ``B[f]: [G, n, n, U]``,
+    ``D[f]: [G, n]``.  ``arith`` selects the kernels' arithmetic: ``"f64"``
+    (default; reproduces a float64 evaluation to 1e-5) or ``"f32"`` (fast).
+    """
+
+    def __init__(self, n: Sequence[int], m: Sequence[int], dep: Sequence[Sequence[int]], U: Sequence[int],
+                 G: int, A: List, B: List, D: List, stream=None, arith: str = "f64"):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("bi needs a CUDA device: there is no CPU path")
+        L = lib()
+        self.n, self.m, self.U = [int(v) for v in n], [int(v) for v in m], [int(v) for v in U]
+        self.dep = [[int(f) for f in d] for d in dep]
+        self.G, self.F, self.M, self.S = int(G), len(self.n), len(self.m), sum(self.n)
+        for t in list(A) + list(B) + list(D):
+            if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+                raise ValueError("model arrays must be contiguous float32 CUDA tensors")
+        d = _Desc()
+        d.F, d.M, d.G = self.F, self.M, self.G
+        keep = [_i32(self.n), _i32(self.m), _i32([len(x) for x in self.dep]),
+                _i32([f for x in self.dep for f in x]), _i32(self.U)]
+        d.n, d.m, d.dep_len, d.dep, d.U = [ctypes.cast(k, ctypes.c_void_p) for k in keep]
+        pa = (ctypes.c_void_p * max(self.M, 1))(*[a.data_ptr() for a in A])
+        pb = (ctypes.c_void_p * self.F)(*[b.data_ptr() for b in B])
+        pd = (ctypes.c_void_p * self.F)(*[x.data_ptr() for x in D])
+        d.A, d.B, d.D = [ctypes.cast(p, ctypes.c_void_p) for p in (pa, pb, pd)]
+        h = ctypes.c_void_p()
+        if arith == "f64":
+            rc = L.bi_model_create(ctypes.byref(d), _stream_ptr(stream), ctypes.byref(h))
+        else:
+            rc = L.bi_model_create_arith(ctypes.byref(d), ARITH[arith], _stream_ptr(stream), ctypes.byref(h))
+        if rc != BI_OK:
+            raise BiError(rc, "bi_model_create")
+        self._h = h
+        self.arith = arith
+        assert L.bi_model_arith(h) == ARITH[arith]
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().bi_model_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- inference -----------------------------------------------------------
+    def _run(self, name, obs, act, iters, q_out, logq_out, argmax_out, stream):
+        import torch
+        N, T = int(obs.shape[0]), int(obs.shape[1])
+        if q_out is None:
+            q_out = torch.empty((N, T, self.S), dtype=torch.float32, device=obs.device)
+        fn = getattr(lib(), name)
+        rc = fn(self._h, N, T, ctypes.c_void_p(obs.data_ptr()),
+                ctypes.c_void_p(act.data_ptr() if act is not None and act.numel() > 0 else None),
+                int(iters), ctypes.c_void_p(q_out.data_ptr()),
+                ctypes.c_void_p(logq_out.data_ptr() if logq_out is not None else None),
+                ctypes.c_void_p(argmax_out.data_ptr() if argmax_out is not None else None),
+                _stream_ptr(stream))
+        if rc != BI_OK:
+            raise BiError(rc, name)
+        return q_out
+
+    def bi_filter(self, obs, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
+        """Variational filtering; ``obs`` int32 ``[N,T,M]``, ``act`` int32 ``[N,T-1,F]`` (CUDA)."""
+        return self._run("bi_filter", obs, act, iters, q_out, logq_out, argmax_out, stream)
+
+    def bi_vmp(self, obs, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
+        """Variational message passing over one window."""
+        return self._run("bi_vmp", obs, act, iters, q_out, logq_out, argmax_out, stream)
+
+    def bi_mmp(self, obs, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
+        """Marginal message passing over one window."""
+        return self._run("bi_mmp", obs, act, iters, q_out, logq_out, argmax_out, stream)
+
+    def run(self, algo, *a, **k):
+        return {"filter": self.bi_filter, "vmp": self.bi_vmp, "mmp": self.bi_mmp}[algo](*a, **k)
+
+    def status(self, stream=None) -> int:
+        v = ctypes.c_uint32(0)
+        rc = lib().bi_status(self._h, _stream_ptr(stream), ctypes.byref(v))
+        if rc != BI_OK:
+            raise BiError(rc, "bi_status")
+        return int(v.value)
+
+    @property
+    def last_kernel(self) -> str:
+        return lib().bi_last_kernel(self._h).decode()
+
+    @property
+    def launch_count(self) -> int:
+        return int(lib().bi_launch_count(self._h))
+
+
+def model_from_workload(w, device="cuda", stream=None, arith: str = "f64") -> Model:
+    """Upload a workload's arrays (numpy) and pack them."""
+    import torch
+    A = [torch.from_numpy(a).to(device) for a in w.A]
+    B = [torch.from_numpy(b).to(device) for b in w.B]
+    D = [torch.from_numpy(d).to(device) for d in w.D]
+    md = Model(w.n, w.m, w.dep, w.U, w.G, A, B, D, stream=stream, arith=arith)
+    torch.cuda.synchronize()
+    return md

@@ -1,0 +1,440 @@
+// Host side of the library: argument validation, the packing layer
+// (bi_model_create) and the dispatcher behind bi_filter / bi_vmp / bi_mmp.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "bi_internal.h"
+
+namespace {
+
+#define BI_CUDA_TRY(expr)                      \
+  do {                                         \
+    cudaError_t e_ = (expr);                   \
+    if (e_ != cudaSuccess) return BI_ERR_CUDA; \
+  } while (0)
+
+// ------------------------------------------------------------------ pack kernels
+
+struct PackA {
+  const float *src;  // [G][m][n_dep0]...[n_dep(k-1)]
+  void *dst;         // [G][m][P_pad], R
+  int64_t total;     // G * m * P_pad
+  int32_t P, P_pad, rank;
+  int32_t dim[BI_MAX_RANK];      // packed axis sizes
+  int64_t sstride[BI_MAX_RANK];  // source stride of each packed axis
+  int32_t npad;                  // padded size of the last packed axis (rank > 0)
+};
+
+// ln(max(A, eps)) in float64, rounded once; outcome slices contiguous, axes in
+// the group's packed order, last axis padded with zeros.
+template <typename R>
+__global__ void bi_pack_A_kernel(PackA p) {
+  int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= p.total) return;
+  int64_t go = e / p.P_pad;  // g * m + o
+  int32_t idx = (int32_t)(e - go * p.P_pad);
+  R out = (R)0;
+  if (p.rank == 0) {
+    // every axis has a single state: the slice is one number (padded to 4)
+    if (idx == 0) out = (R)log(fmax((double)p.src[go * p.P], 1e-16));
+  } else {
+    int32_t last = idx % p.npad, rest = idx / p.npad;
+    if (last < p.dim[p.rank - 1]) {
+      int64_t s = go * p.P + (int64_t)last * p.sstride[p.rank - 1];
+      for (int j = p.rank - 2; j >= 0; --j) {
+        int32_t dg = rest % p.dim[j];
+        rest /= p.dim[j];
+        s += (int64_t)dg * p.sstride[j];
+      }
+      out = (R)log(fmax((double)p.src[s], 1e-16));
+    }
+  }
+  ((R *)p.dst)[e] = out;
+}
+
+// B[g][s_next][s_prev][u] -> four [g][u][row][npad] matrices
+template <typename R>
+__global__ void bi_pack_B_kernel(const float *__restrict__ B, int G, int n, int npad, int U,
+                                 R *Bf, R *logB, R *logBt, R *Bdag) {
+  int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int64_t total = (int64_t)G * U * n * npad;
+  if (e >= total) return;
+  int c = (int)(e % npad);
+  int64_t r1 = e / npad;
+  int r = (int)(r1 % n);
+  int64_t r2 = r1 / n;
+  int u = (int)(r2 % U);
+  int64_t g = r2 / U;
+  R f = 0, lf = 0, lt = 0, bd = 0;
+  if (c < n) {
+    const float *Bg = B + g * (int64_t)n * n * U;
+    // forward: row = next state, column = previous state
+    double b = (double)Bg[((int64_t)r * n + c) * U + u];
+    f = (R)b;
+    lf = (R)log(fmax(b, 1e-16));
+    // transposed: row = previous state, column = next state
+    double bt = (double)Bg[((int64_t)c * n + r) * U + u];
+    lt = (R)log(fmax(bt, 1e-16));
+    double rowsum = 0.0;
+    for (int sp = 0; sp < n; ++sp) rowsum += (double)Bg[((int64_t)c * n + sp) * U + u];
+    bd = (R)(rowsum > 0.0 ? bt / rowsum : 1.0 / n);
+  }
+  Bf[e] = f;
+  logB[e] = lf;
+  logBt[e] = lt;
+  Bdag[e] = bd;
+}
+
+template <typename R>
+__global__ void bi_pack_D_kernel(const float *__restrict__ D, int G, int n, int npad, R *logD) {
+  int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (int64_t)G * npad) return;
+  int c = (int)(e % npad);
+  int64_t g = e / npad;
+  logD[e] = c < n ? (R)log(fmax((double)D[g * n + c], 1e-16)) : (R)0;
+}
+
+// ------------------------------------------------------------------ helpers
+
+int dev_alloc(bi_model *md, void **p, size_t bytes) {
+  if (bytes == 0) bytes = 16;
+  if (md->nalloc >= (int)(sizeof(md->allocs) / sizeof(md->allocs[0]))) return BI_ERR_ALLOC;
+  cudaError_t e = cudaMalloc(p, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return BI_ERR_ALLOC;
+  }
+  md->allocs[md->nalloc++] = *p;
+  return BI_OK;
+}
+
+void free_all(bi_model *md) {
+  for (int i = 0; i < md->nalloc; ++i) cudaFree(md->allocs[i]);
+  md->nalloc = 0;
+}
+
+uint32_t magic_for(int d) {  // d >= 2
+  return (uint32_t)(((1ull << 32) + (uint64_t)d - 1) / (uint64_t)d);
+}
+
+int validate_desc(const bi_model_desc *d) {
+  if (!d || !d->n || !d->U || !d->B || !d->D) return BI_ERR_INVALID_ARG;
+  if (d->F < 1 || d->M < 0 || d->G < 1) return BI_ERR_INVALID_ARG;
+  if (d->M > 0 && (!d->m || !d->dep_len || !d->dep || !d->A)) return BI_ERR_INVALID_ARG;
+  if (d->F > BI_MAX_F || d->M > BI_MAX_M) return BI_ERR_UNSUPPORTED;
+  for (int f = 0; f < d->F; ++f) {
+    if (d->n[f] < 1 || d->U[f] < 1) return BI_ERR_INVALID_ARG;
+    if (d->n[f] > BI_MAX_N) return BI_ERR_UNSUPPORTED;
+    if (!d->B[f] || !d->D[f]) return BI_ERR_INVALID_ARG;
+  }
+  int o = 0;
+  for (int i = 0; i < d->M; ++i) {
+    if (d->m[i] < 1 || d->dep_len[i] < 1) return BI_ERR_INVALID_ARG;
+    if (d->dep_len[i] > BI_MAX_RANK) return BI_ERR_UNSUPPORTED;
+    if (!d->A[i]) return BI_ERR_INVALID_ARG;
+    uint32_t seen = 0;
+    for (int j = 0; j < d->dep_len[i]; ++j) {
+      int f = d->dep[o + j];
+      if (f < 0 || f >= d->F) return BI_ERR_INVALID_ARG;
+      if (seen & (1u << f)) return BI_ERR_SHAPE;
+      seen |= 1u << f;
+    }
+    o += d->dep_len[i];
+  }
+  return BI_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ public API
+
+extern "C" int bi_model_create(const bi_model_desc *desc, void *cuda_stream, bi_model_t **out) {
+  return bi_model_create_arith(desc, BI_ARITH_F64, cuda_stream, out);
+}
+
+extern "C" int bi_model_arith(const bi_model_t *model) { return model ? model->arith : BI_ERR_INVALID_ARG; }
+
+extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void *cuda_stream, bi_model_t **out) {
+  if (!out) return BI_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (arith != BI_ARITH_F64 && arith != BI_ARITH_F32) return BI_ERR_INVALID_ARG;
+  const size_t esz = arith == BI_ARITH_F64 ? 8 : 4;
+  int rc = validate_desc(desc);
+  if (rc != BI_OK) return rc;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+  bi_model *md = new (std::nothrow) bi_model();
+  if (!md) return BI_ERR_ALLOC;
+  memset(md, 0, sizeof(*md));
+  md->last_kernel = "";
+  md->arith = arith;
+  if (cudaGetDevice(&md->device) != cudaSuccess) {
+    delete md;
+    return BI_ERR_CUDA;
+  }
+  cudaDeviceGetAttribute(&md->sm_count, cudaDevAttrMultiProcessorCount, md->device);
+  cudaDeviceGetAttribute(&md->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, md->device);
+
+  BiDev &h = md->h;
+  const int F = desc->F, M = desc->M, G = desc->G;
+  h.F = F; h.M = M; h.G = G;
+  int S = 0, Sp = 0;
+  for (int f = 0; f < F; ++f) {
+    h.n[f] = desc->n[f];
+    h.npad[f] = bi_pad4(desc->n[f]);
+    h.U[f] = desc->U[f];
+    h.off[f] = S;
+    h.offp[f] = Sp;
+    S += h.n[f];
+    Sp += h.npad[f];
+  }
+  h.S = S; h.Sp = Sp;
+  for (int i = 0; i < M; ++i) h.m[i] = desc->m[i];
+
+  // ---- group modalities by dependency set (axes with a single state dropped)
+  struct Tmp { uint32_t mask; };
+  std::vector<uint32_t> gmask;
+  std::vector<std::vector<int>> gmembers;
+  {
+    int o = 0;
+    for (int i = 0; i < M; ++i) {
+      uint32_t mask = 0;
+      for (int j = 0; j < desc->dep_len[i]; ++j) {
+        int f = desc->dep[o + j];
+        if (desc->n[f] > 1) mask |= 1u << f;
+      }
+      o += desc->dep_len[i];
+      if (mask == 0) continue;  // a constant over every multi-state factor: no message
+      size_t gi = 0;
+      for (; gi < gmask.size(); ++gi)
+        if (gmask[gi] == mask) break;
+      if (gi == gmask.size()) {
+        gmask.push_back(mask);
+        gmembers.emplace_back();
+      }
+      gmembers[gi].push_back(i);
+    }
+  }
+  h.ngroups = (int)gmask.size();
+  int nmem = 0, Ltot = 0, V0 = 4, V1 = 4, rows_max = 1;
+  std::vector<int> dep_off(M + 1, 0);
+  for (int i = 0; i < M; ++i) dep_off[i + 1] = dep_off[i] + desc->dep_len[i];
+
+  for (int gi = 0; gi < h.ngroups; ++gi) {
+    BiGroup &g = h.grp[gi];
+    std::vector<int> axes;
+    for (int f = 0; f < F; ++f)
+      if (gmask[gi] & (1u << f)) axes.push_back(f);
+    int k = (int)axes.size();
+    // the contracted-first (last, padded) axis: least padded volume, then the largest
+    int best = 0;
+    for (int j = 1; j < k; ++j) {
+      int nb = h.n[axes[best]], nj = h.n[axes[j]];
+      long vb = (long)bi_pad4(nb) * nj, vj = (long)bi_pad4(nj) * nb;  // compare pad(nb)/nb vs pad(nj)/nj
+      if (vj < vb || (vj == vb && nj > nb)) best = j;
+    }
+    int lastf = axes[best];
+    axes.erase(axes.begin() + best);
+    axes.push_back(lastf);
+    g.rank = k;
+    int P_pad = 1;
+    for (int j = 0; j < k; ++j) {
+      g.axis[j] = axes[j];
+      g.dim[j] = h.n[axes[j]];
+      P_pad *= (j == k - 1) ? bi_pad4(g.dim[j]) : g.dim[j];
+    }
+    g.P_pad = P_pad;
+    g.L_off = Ltot;
+    Ltot += P_pad;
+    g.first_qoff = h.offp[axes[0]];
+    g.first_n = h.n[axes[0]];
+    // levels: lev[l] contracts axis[k-1-l]; it has k-1-l leading axes
+    for (int l = 0; l + 1 < k; ++l) {
+      BiLevel &lv = g.lev[l];
+      int last = k - 1 - l;
+      lv.ndig = last;
+      lv.nrows = 1;
+      for (int j = 0; j < last; ++j) {
+        lv.dim[j] = g.dim[j];
+        lv.magic[j] = magic_for(g.dim[j]);
+        lv.qoff[j] = h.offp[g.axis[j]];
+        lv.nrows *= g.dim[j];
+      }
+      lv.last_n = g.dim[last];
+      lv.last_npad4 = bi_pad4(g.dim[last]) / 4;
+      lv.last_qoff = h.offp[g.axis[last]];
+      lv.out_npad = bi_pad4(g.dim[last - 1]);
+      int out_floats = (lv.nrows / g.dim[last - 1]) * lv.out_npad;
+      if (l % 2 == 0) V0 = std::max(V0, out_floats); else V1 = std::max(V1, out_floats);
+      if (l == 0) rows_max = std::max(rows_max, lv.nrows);
+    }
+    g.mem_begin = nmem;
+    for (int i : gmembers[gi]) {
+      BiMember &mm = h.mem[nmem++];
+      mm.modality = i;
+      mm.m = desc->m[i];
+      mm.P_pad = P_pad;
+      mm.gstride = (G == 1) ? 0 : (int64_t)mm.m * P_pad;
+    }
+    g.mem_end = nmem;
+  }
+  h.nmem = nmem;
+  h.Ltot = Ltot;
+  md->V0max = V0; md->V1max = V1; md->rows_max = rows_max;
+
+  // ---- allocate and pack
+  rc = dev_alloc(md, (void **)&h.status, sizeof(uint32_t));
+  if (rc == BI_OK && cudaMemsetAsync(h.status, 0, sizeof(uint32_t), stream) != cudaSuccess) rc = BI_ERR_CUDA;
+  for (int gi = 0; gi < h.ngroups && rc == BI_OK; ++gi) {
+    BiGroup &g = h.grp[gi];
+    for (int mi = g.mem_begin; mi < g.mem_end && rc == BI_OK; ++mi) {
+      BiMember &mm = h.mem[mi];
+      int i = mm.modality;
+      void *dst = nullptr;
+      size_t count = (size_t)G * mm.m * g.P_pad;
+      rc = dev_alloc(md, &dst, count * esz);
+      if (rc != BI_OK) break;
+      mm.logA = dst;
+      PackA p;
+      memset(&p, 0, sizeof(p));
+      p.src = desc->A[i];
+      p.dst = dst;
+      p.total = (int64_t)count;
+      p.P_pad = g.P_pad;
+      p.rank = g.rank;
+      // source strides of every factor axis in A_i's own order
+      int ki = desc->dep_len[i];
+      int64_t sstr[BI_MAX_RANK];
+      int64_t acc = 1;
+      for (int j = ki - 1; j >= 0; --j) {
+        sstr[j] = acc;
+        acc *= desc->n[desc->dep[dep_off[i] + j]];
+      }
+      p.P = (int32_t)acc;
+      for (int j = 0; j < g.rank; ++j) {
+        p.dim[j] = g.dim[j];
+        for (int jj = 0; jj < ki; ++jj)
+          if (desc->dep[dep_off[i] + jj] == g.axis[j]) p.sstride[j] = sstr[jj];
+      }
+      p.npad = g.rank > 0 ? bi_pad4(g.dim[g.rank - 1]) : 4;
+      int threads = 256;
+      int64_t blocks = (p.total + threads - 1) / threads;
+      if (arith == BI_ARITH_F64) bi_pack_A_kernel<double><<<(unsigned)blocks, threads, 0, stream>>>(p);
+      else bi_pack_A_kernel<float><<<(unsigned)blocks, threads, 0, stream>>>(p);
+      if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+    }
+  }
+  for (int f = 0; f < F && rc == BI_OK; ++f) {
+    int n = h.n[f], npad = h.npad[f], U = h.U[f];
+    size_t count = (size_t)G * U * n * npad;
+    void *bf, *lb, *lt, *bd, *ld;
+    if ((rc = dev_alloc(md, &bf, count * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &lb, count * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &lt, count * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &bd, count * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &ld, (size_t)G * npad * esz)) != BI_OK) break;
+    h.Bf[f] = bf; h.logB[f] = lb; h.logBt[f] = lt; h.Bdag[f] = bd; h.logD[f] = ld;
+    h.Bstride[f] = (G == 1) ? 0 : (int64_t)U * n * npad;
+    h.Dstride[f] = (G == 1) ? 0 : npad;
+    int threads = 256;
+    unsigned gb = (unsigned)((count + threads - 1) / threads);
+    unsigned gd = (unsigned)(((size_t)G * npad + threads - 1) / threads);
+    if (arith == BI_ARITH_F64) {
+      bi_pack_B_kernel<double><<<gb, threads, 0, stream>>>(desc->B[f], G, n, npad, U, (double *)bf,
+                                                           (double *)lb, (double *)lt, (double *)bd);
+      bi_pack_D_kernel<double><<<gd, threads, 0, stream>>>(desc->D[f], G, n, npad, (double *)ld);
+    } else {
+      bi_pack_B_kernel<float><<<gb, threads, 0, stream>>>(desc->B[f], G, n, npad, U, (float *)bf,
+                                                          (float *)lb, (float *)lt, (float *)bd);
+      bi_pack_D_kernel<float><<<gd, threads, 0, stream>>>(desc->D[f], G, n, npad, (float *)ld);
+    }
+    if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+  }
+  if (rc == BI_OK) rc = dev_alloc(md, (void **)&md->d, sizeof(BiDev));
+  if (rc == BI_OK) {
+    // the host copy outlives the asynchronous copy: it is a member of the handle
+    if (cudaMemcpyAsync(md->d, &md->h, sizeof(BiDev), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      rc = BI_ERR_CUDA;
+  }
+  if (rc != BI_OK) {
+    cudaStreamSynchronize(stream);
+    free_all(md);
+    delete md;
+    return rc;
+  }
+  *out = md;
+  return BI_OK;
+}
+
+extern "C" int bi_model_destroy(bi_model_t *model) {
+  if (!model) return BI_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  free_all(model);
+  delete model;
+  return e == cudaSuccess ? BI_OK : BI_ERR_CUDA;
+}
+
+static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, const int32_t *obs,
+                    const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                    int32_t *argmax_out, void *cuda_stream) {
+  if (!model || N < 0 || T < 1 || iters < 1) return BI_ERR_INVALID_ARG;
+  if (N == 0) return BI_OK;
+  if (!q_out || (model->h.M > 0 && !obs) || (T > 1 && !act)) return BI_ERR_INVALID_ARG;
+  if (model->h.G != 1 && model->h.G != N) return BI_ERR_SHAPE;
+  if (algo != BI_ALGO_FILTER && T > BI_MAX_T) return BI_ERR_UNSUPPORTED;
+  BiCall c;
+  c.model = model; c.algo = algo; c.N = N; c.T = T; c.K = iters;
+  c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
+  c.stream = (cudaStream_t)cuda_stream;
+  bi_model *mut = const_cast<bi_model *>(model);
+  int rc = bi_launch_generic(c, mut);
+  return rc;
+}
+
+extern "C" int bi_filter(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                         const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                         int32_t *argmax_out, void *cuda_stream) {
+  return run_call(model, BI_ALGO_FILTER, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream);
+}
+
+extern "C" int bi_vmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                      const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                      int32_t *argmax_out, void *cuda_stream) {
+  return run_call(model, BI_ALGO_VMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream);
+}
+
+extern "C" int bi_mmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                      const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                      int32_t *argmax_out, void *cuda_stream) {
+  return run_call(model, BI_ALGO_MMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream);
+}
+
+extern "C" int bi_status(const bi_model_t *model, void *cuda_stream, uint32_t *flags) {
+  if (!model || !flags) return BI_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  uint32_t v = 0;
+  BI_CUDA_TRY(cudaMemcpyAsync(&v, model->h.status, sizeof(v), cudaMemcpyDeviceToHost, s));
+  BI_CUDA_TRY(cudaMemsetAsync(model->h.status, 0, sizeof(v), s));
+  BI_CUDA_TRY(cudaStreamSynchronize(s));
+  *flags = v;
+  return BI_OK;
+}
+
+extern "C" const char *bi_last_kernel(const bi_model_t *model) { return model ? model->last_kernel : ""; }
+
+extern "C" int64_t bi_launch_count(const bi_model_t *model) { return model ? model->launches : 0; }
+
+extern "C" const char *bi_strerror(int code) {
+  switch (code) {
+    case BI_OK: return "ok";
+    case BI_ERR_INVALID_ARG: return "invalid argument";
+    case BI_ERR_SHAPE: return "shape mismatch";
+    case BI_ERR_UNSUPPORTED: return "unsupported size or configuration";
+    case BI_ERR_ALLOC: return "device allocation failed";
+    case BI_ERR_CUDA: return "CUDA runtime error or no device";
+    default: return "unknown error";
+  }
+}

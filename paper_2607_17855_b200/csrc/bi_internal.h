@@ -1,0 +1,97 @@
+// Internal structures shared by the packing layer, the dispatcher and the
+// kernels.  Nothing here is part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bi.h"
+
+#define BI_EPS 1e-16
+#define BI_MAX_GROUPS BI_MAX_M
+
+enum { BI_ALGO_FILTER = 0, BI_ALGO_VMP = 1, BI_ALGO_MMP = 2 };
+
+static __host__ __device__ inline int bi_pad4(int x) { return (x + 3) & ~3; }
+
+// One contraction level of a dependency group.  The group's summed slice is a
+// tensor with `ndig` leading axes and one last axis; the level contracts the
+// last axis against its factor's belief (giving a tensor over the leading
+// axes for the next level) and, weighted by the outer product of the leading
+// beliefs, accumulates the likelihood message to the last axis' factor.
+struct BiLevel {
+  int32_t nrows;      // product of the leading axis sizes
+  int32_t ndig;       // number of leading axes, 1..4
+  int32_t dim[4];     // leading axis sizes, slowest first
+  uint32_t magic[4];  // ceil(2^32 / dim) for exact division by multiply-high
+  int32_t qoff[4];    // padded belief offset of each leading axis' factor
+  int32_t last_n;     // size of the contracted axis
+  int32_t last_npad4; // its padded size / 4
+  int32_t last_qoff;  // padded belief offset of its factor
+  int32_t out_npad;   // padded size of the output tensor's last axis
+};
+
+// Modalities with the same dependency *set* form one group: their slices add
+// before any contraction, so they share one packed axis order.
+struct BiGroup {
+  int32_t rank;       // number of axes with more than one state
+  int32_t axis[BI_MAX_RANK];  // factor ids in packed order (last = contracted first)
+  int32_t dim[BI_MAX_RANK];
+  int32_t P_pad;      // floats per packed slice (last axis padded to a multiple of 4)
+  int32_t mem_begin, mem_end;  // members in BiDev::mem
+  int32_t L_off;      // float offset of this group's summed slice in a staged step
+  int32_t first_qoff, first_n; // axis[0]'s factor: receives the fully contracted vector
+  BiLevel lev[BI_MAX_RANK - 1]; // lev[0] contracts axis[rank-1], lev[1] axis[rank-2], ...
+};
+
+struct BiMember {
+  const void *logA;   // packed [G][m][P_pad], float or double (the handle's arithmetic)
+  int64_t gstride;    // floats per model (0 when the model is shared)
+  int32_t m, modality, P_pad, pad_;
+};
+
+struct BiDev {
+  int32_t F, M, S, Sp, G, ngroups, nmem, Ltot;
+  int32_t n[BI_MAX_F], npad[BI_MAX_F], off[BI_MAX_F], offp[BI_MAX_F], U[BI_MAX_F];
+  int32_t m[BI_MAX_M];
+  BiGroup grp[BI_MAX_GROUPS];
+  BiMember mem[BI_MAX_M];
+  // per factor, per model g, per action u: [n][npad] row-major, pad columns zero;
+  // element type float or double (the handle's arithmetic)
+  const void *Bf[BI_MAX_F];    // Bf[s_next][s_prev]    = B[s_next, s_prev, u]
+  const void *logB[BI_MAX_F];  // ln of the same
+  const void *logBt[BI_MAX_F]; // [s_prev][s_next]      = ln B[s_next, s_prev, u]
+  const void *Bdag[BI_MAX_F];  // [s_prev][s_next]      = B[s_next, s_prev, u] / sum_r B[s_next, r, u]
+  const void *logD[BI_MAX_F];  // [G][npad]
+  int64_t Bstride[BI_MAX_F];    // floats per model in each B array (0 when shared)
+  int64_t Dstride[BI_MAX_F];
+  uint32_t *status;
+};
+
+// host-side handle
+struct bi_model {
+  BiDev h;          // host copy (device pointers inside)
+  BiDev *d;         // device copy
+  void *allocs[8 + 2 * BI_MAX_M + 8 * BI_MAX_F];
+  int nalloc;
+  int arith;        // BI_ARITH_F64 or BI_ARITH_F32
+  int device;
+  int sm_count;
+  int max_smem_optin;
+  int V0max, V1max; // floats needed by the generic kernel's two intermediate buffers
+  int rows_max;     // largest first-level row count over groups
+  int64_t launches;
+  const char *last_kernel;
+};
+
+struct BiCall {
+  const bi_model *model;
+  int algo, N, T, K;
+  const int32_t *obs, *act;
+  float *q_out, *logq_out;
+  int32_t *argmax_out;
+  cudaStream_t stream;
+};
+
+// kernel families; each returns BI_OK, BI_ERR_UNSUPPORTED (not applicable to
+// this model / call: the dispatcher tries the next one) or an error.
+int bi_launch_generic(const BiCall &c, bi_model *mut);
