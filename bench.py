@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark: batched belief updates per second on B200.
+
+A step is one pass of the whole hot path over one batch: one ``bi_filter``
+call on the headline workload (4096 agents sharing one model, F = 3 factors
+[8, 8, 6], M = 3 modalities, T = 50 steps, K = 16 iterations), inputs resident
+in HBM.  A belief update is one softmax update of one factor of one agent at
+one step in one iteration, so a step performs N*T*F*K of them.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+prints one JSON line.  With ``--impl reference`` the CPU oracle is timed
+instead (rank 0 only), each step on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "belief_updates_per_sec"
+UNIT = "updates/s"
+HEADLINE = 2  # configuration the metric is quoted on
+
+# Nominal ALU peaks derived from the unit counts: 148 SMs x lanes x 2 flops x 1.965 GHz.
+FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12   # 37.2
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # 74.4
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def algorithmic_flops(w) -> float:
+    """4 * P flops (2 P multiply-adds) per dependency group with >= 2 factors,
+    per agent, step and iteration (all leave-one-out messages of the group)."""
+    groups = {}
+    for d in w.dep:
+        key = tuple(sorted(f for f in d if w.n[f] > 1))
+        if len(key) >= 2:
+            p = 1
+            for f in key:
+                p *= int(w.n[f])
+            groups[key] = p
+    return 4.0 * sum(groups.values()) * w.N * w.T * w.K
+
+
+def algorithmic_bytes(w, elem_bytes: int) -> float:
+    """Each needed slice log A_i[o_{t,i}] read once per (agent, step) plus the
+    index inputs and belief outputs."""
+    slices = 0
+    for d in w.dep:
+        p = 1
+        for f in d:
+            p *= int(w.n[f])
+        slices += p
+    io = w.obs.nbytes + w.act.nbytes + w.N * w.T * w.S * 4
+    if w.G == 1:
+        model = sum(a.size for a in w.A) * elem_bytes  # shared: read once
+        return float(io + model)
+    return float(w.N * w.T * slices * elem_bytes + io)
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while timing runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def time_steps(fn, steps, warmup, flush, torch):
+    """Device time of ``steps`` calls of fn, L2 flushed before each; returns seconds per step list."""
+    for _ in range(warmup):
+        flush.zero_()
+        fn()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(steps):
+        flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        times.append(a.elapsed_time(b) * 1e-3)
+    return times
+
+
+def bench_config(torch, bi, w, algo, arith, steps, warmup, flush):
+    md = bi.model_from_workload(w, arith=arith)
+    obs = torch.from_numpy(w.obs).cuda()
+    act = torch.from_numpy(w.act).cuda() if w.act.size else None
+    q = torch.empty((w.N, w.T, w.S), dtype=torch.float32, device="cuda")
+    l0 = md.launch_count
+    times = time_steps(lambda: md.run(algo, obs, act, w.K, q_out=q), steps, warmup, flush, torch)
+    launches = (md.launch_count - l0) // (steps + warmup)
+    assert md.status() == 0
+    res = {"seconds": sum(times) / len(times), "best": min(times), "kernel": md.last_kernel,
+           "launches_per_step": launches, "model": md, "obs": obs, "act": act, "q": q}
+    return res
+
+
+def reference_arm(args, rank, world):
+    """The CPU oracle, as it stands, on the GPU machine's host cores."""
+    if rank != 0:
+        return
+    import oracle
+    from biwl import make_config
+    w = make_config(HEADLINE)
+    sample_agents = 128
+    sub = w.take_agents(range(sample_agents))
+    cores = oracle.max_threads()
+    for _ in range(args.warmup):
+        oracle.run_workload(sub.take_agents(range(8)))
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.run_workload(sub)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = sub.updates / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"config {HEADLINE}: filtering, shared model n=[8,8,6] m=[16,8,8], T=50, K=16; "
+                               f"each step = the first {sample_agents} of 4096 agents"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{sample_agents} agents x 50 steps x 16 iterations per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--arith", default="f64", choices=["f64", "f32"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads and the CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        reference_arm(args, rank, world)
+        return
+
+    import numpy as np
+    import torch
+    import paper_2607_17855_b200 as bi
+    from biwl import make_config
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # agents are independent: each rank runs its own full-size batch (weak scaling),
+    # drawn from its own seed; there is no collective on the data path
+    w = make_config(HEADLINE, seed=1000 + HEADLINE + 7919 * rank)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
+
+    sampler = ClockSampler(local_rank)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    head = bench_config(torch, bi, w, "filter", args.arith, args.steps, args.warmup, flush)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    sec = head["seconds"]
+    if dist is not None:
+        t = torch.tensor([sec], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+    value = w.updates * world / sec
+
+    # ---- end to end: pinned host inputs -> device -> bi_filter -> host beliefs
+    md, q = head["model"], head["q"]
+    h_obs = torch.from_numpy(w.obs).pin_memory()
+    h_act = torch.from_numpy(w.act).pin_memory()
+    h_q = torch.empty(q.shape, dtype=torch.float32).pin_memory()
+    d_obs, d_act = head["obs"], head["act"]
+
+    def e2e_step():
+        d_obs.copy_(h_obs, non_blocking=True)
+        d_act.copy_(h_act, non_blocking=True)
+        md.bi_filter(d_obs, d_act, w.K, q_out=q)
+        h_q.copy_(q, non_blocking=True)
+
+    e2e_times = time_steps(e2e_step, max(3, args.steps // 2), 3, flush, torch)
+    e2e_sec = sum(e2e_times) / len(e2e_times)
+    if dist is not None:
+        t = torch.tensor([e2e_sec], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_sec = float(t.item())
+    e2e = {"value": w.updates * world / e2e_sec, "unit": UNIT,
+           "h2d_bytes_per_step": int(w.obs.nbytes + w.act.nbytes), "d2h_bytes_per_step": int(q.numel() * 4)}
+
+    flops = algorithmic_flops(w)
+    peak = FP64_PEAK_TFLOPS if args.arith == "f64" else FP32_PEAK_TFLOPS
+    achieved = flops / head["seconds"] / 1e12
+    roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "kernel": head["kernel"],
+                "peak_source": f"derived: 148 SMs x {64 if args.arith == 'f64' else 128} lanes x 2 x 1.965 GHz"}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        with open(prof) as fh:
+            roofline["traffic"] = json.load(fh).get(head["kernel"])
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": args.arith, "data": "synthetic",
+        "config": {"workload": "config 2: variational filtering, 4096 agents sharing one model, "
+                               "n=[8,8,6], m=[16,8,8], T=50, K=16",
+                   "updates_per_step": w.updates, "l2": "flushed with a 256 MiB write before every timed step",
+                   "agents_per_gpu": w.N},
+        "e2e": e2e, "gpu_launches": head["launches_per_step"] * args.steps, "clocks": clocks,
+        "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1 and not args.no_extras:
+        hbm_peak, hbm_src = measured_peaks()
+        others = {}
+        # the float32-arithmetic mode on the same workload
+        alt = "f32" if args.arith == "f64" else "f64"
+        r = bench_config(torch, bi, w, "filter", alt, max(3, args.steps // 2), 3, flush)
+        others[f"config2_filter_{alt}"] = {"value": w.updates / r["seconds"], "unit": UNIT,
+                                           "ms_per_step": r["seconds"] * 1e3, "kernel": r["kernel"]}
+        for c, algo in ((3, "vmp"), (4, "mmp")):
+            wc = make_config(c)
+            r = bench_config(torch, bi, wc, algo, args.arith, max(3, args.steps // 2), 3, flush)
+            entry = {"value": wc.updates / r["seconds"], "unit": UNIT, "ms_per_step": r["seconds"] * 1e3,
+                     "kernel": r["kernel"], "alu_tflops": algorithmic_flops(wc) / r["seconds"] / 1e12}
+            if wc.G != 1:
+                gbs = algorithmic_bytes(wc, 8 if args.arith == "f64" else 4) / r["seconds"] / 1e9
+                entry["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s",
+                                     "frac": gbs / hbm_peak, "peak_source": hbm_src}
+            others[f"config{c}_{algo}_{args.arith}"] = entry
+            del r
+        line["others"] = others
+        # ---- the oracle on this machine's host cores, on a bounded sample of the workload
+        import oracle
+        sample = 1024
+        sub = w.take_agents(range(sample))
+        t0 = time.perf_counter()
+        oracle.run_workload(sub)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": sub.updates / dt, "unit": UNIT, "cores": oracle.max_threads(),
+                                "kind": "oracle", "sample": f"first {sample} of 4096 agents, all 50 steps, "
+                                                            f"16 iterations ({dt:.1f} s wall)"}
+    elif rank == 0:
+        line["cpu_baseline"] = None
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

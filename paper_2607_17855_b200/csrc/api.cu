@@ -229,12 +229,12 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
     for (int f = 0; f < F; ++f)
       if (gmask[gi] & (1u << f)) axes.push_back(f);
     int k = (int)axes.size();
-    // the contracted-first (last, padded) axis: least padded volume, then the largest
+    // the contracted-first (last, padded) axis: least padding, then the smallest
     int best = 0;
     for (int j = 1; j < k; ++j) {
       int nb = h.n[axes[best]], nj = h.n[axes[j]];
       long vb = (long)bi_pad4(nb) * nj, vj = (long)bi_pad4(nj) * nb;  // compare pad(nb)/nb vs pad(nj)/nj
-      if (vj < vb || (vj == vb && nj > nb)) best = j;
+      if (vj < vb || (vj == vb && nj < nb)) best = j;
     }
     int lastf = axes[best];
     axes.erase(axes.begin() + best);
@@ -390,7 +390,8 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
   c.stream = (cudaStream_t)cuda_stream;
   bi_model *mut = const_cast<bi_model *>(model);
-  int rc = bi_launch_generic(c, mut);
+  int rc = bi_launch_tile3(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;
 }
 

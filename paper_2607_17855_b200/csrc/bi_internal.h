@@ -95,3 +95,4 @@ struct BiCall {
 // kernel families; each returns BI_OK, BI_ERR_UNSUPPORTED (not applicable to
 // this model / call: the dispatcher tries the next one) or an error.
 int bi_launch_generic(const BiCall &c, bi_model *mut);
+int bi_launch_tile3(const BiCall &c, bi_model *mut);

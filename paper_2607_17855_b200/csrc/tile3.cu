@@ -1,0 +1,219 @@
+// Register-tile kernels for single-group rank-3 models (every modality depends
+// on the same three factors and the model has exactly those factors).
+// Filtering: a few lanes per agent, the step recursion and the iteration loop
+// inside one launch, the summed slice of the current step held in registers.
+#include "bi_internal.h"
+#include "tile3.cuh"
+
+namespace {
+
+struct Tile3Params {
+  const void *logA[BI_MAX_M];
+  int64_t gstride[BI_MAX_M];
+  int32_t modality[BI_MAX_M], mcount[BI_MAX_M];
+  int32_t nmem, P_pad;
+  int32_t fac[3];   // factor ids of the axes a, b, c
+  int32_t off[3];   // offsets of those factors in an output belief vector
+  int32_t np[3];    // padded row length of their transition matrices
+  int32_t U[3];
+  const void *Bf[3], *logB[3], *logBt[3], *Bdag[3], *logD[3];
+  int64_t Bstride[3], Dstride[3];
+  int32_t N, T, K, M, S, G;
+  const int32_t *obs, *act;
+  float *q_out, *logq_out;
+  int32_t *argmax_out;
+  uint32_t *status;
+};
+
+template <typename R>
+__device__ __forceinline__ R row_dot(const R *__restrict__ row, const R *q, int n) {
+  R p = (R)0;
+  for (int r = 0; r < n; ++r) p = fma(__ldg(row + r), q[r], p);
+  return p;
+}
+
+template <typename R, int NA, int NB, int NC, int SB>
+__global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p) {
+  using TT = Tile3<R, NA, NB, NC, SB>;
+  constexpr int LPU = TT::LPU, UPW = TT::UPW, NBL = TT::NBL, NCP = TT::NCP, NAP = TT::NAP;
+  __shared__ __align__(16) R sm_e[UPW][NB + NCP];      // gathered e_b, e_c of the current iterate
+  __shared__ __align__(16) R sm_q[UPW][NA + NB + NC];  // final beliefs of the previous step
+
+  const int lane = threadIdx.x;
+  const int unit = lane / LPU;
+  int agent = blockIdx.x * UPW + unit;
+  const bool live = agent < p.N;
+  if (!live) agent = p.N - 1;  // keeps every shuffle warp-uniform; its stores are suppressed
+  const int g = p.G == 1 ? 0 : agent;
+
+  TT t3;
+  t3.init_lane(lane);
+  const int a = t3.a, bi = t3.bi, ci = t3.ci;
+  const bool a_ok = t3.a_ok, b_ok = (a >> TT::SHB) < NBL, c_ok = ci < NC;
+  const int bsafe = b_ok ? bi : 0, csafe = c_ok ? ci : 0, asafe = a_ok ? a : 0;
+  R *se = sm_e[unit], *sq = sm_q[unit];
+  for (int i = t3.u; i < NB + NCP; i += LPU) se[i] = (R)0;
+  __syncwarp();
+
+  const size_t out_base = (size_t)agent * p.T;
+  for (int t = 0; t < p.T; ++t) {
+    // ---- the step's summed slice: one gather of every modality's observed slice
+    const R *slice[BI_MAX_M];
+    for (int mi = 0; mi < p.nmem; ++mi) {
+      int o = clamp_flag(__ldg(p.obs + (out_base + t) * p.M + p.modality[mi]), p.mcount[mi], p.status,
+                         BI_FLAG_OBS_RANGE);
+      slice[mi] = (const R *)p.logA[mi] + (size_t)g * p.gstride[mi] + (size_t)o * p.P_pad;
+    }
+    t3.load_slices(slice, p.nmem);
+
+    // ---- ln prior of the logits this lane owns: D, or B_u times the previous step's belief
+    R lpa, lpb, lpc;
+    if (t == 0) {
+      lpa = __ldg((const R *)p.logD[0] + (size_t)g * p.Dstride[0] + asafe);
+      lpb = __ldg((const R *)p.logD[1] + (size_t)g * p.Dstride[1] + bsafe);
+      lpc = __ldg((const R *)p.logD[2] + (size_t)g * p.Dstride[2] + csafe);
+    } else {
+      const int32_t *ac = p.act + ((size_t)agent * (p.T - 1) + (t - 1)) * 3;
+      int ua = clamp_flag(__ldg(ac + p.fac[0]), p.U[0], p.status, BI_FLAG_ACT_RANGE);
+      int ub = clamp_flag(__ldg(ac + p.fac[1]), p.U[1], p.status, BI_FLAG_ACT_RANGE);
+      int uc = clamp_flag(__ldg(ac + p.fac[2]), p.U[2], p.status, BI_FLAG_ACT_RANGE);
+      const R *ra = (const R *)p.Bf[0] + (size_t)g * p.Bstride[0] + ((size_t)ua * NA + asafe) * p.np[0];
+      const R *rb = (const R *)p.Bf[1] + (size_t)g * p.Bstride[1] + ((size_t)ub * NB + bsafe) * p.np[1];
+      const R *rc = (const R *)p.Bf[2] + (size_t)g * p.Bstride[2] + ((size_t)uc * NC + csafe) * p.np[2];
+      lpa = bi_log(bi_max(row_dot<R>(ra, sq, NA), (R)BI_EPS));
+      lpb = bi_log(bi_max(row_dot<R>(rb, sq + NA, NB), (R)BI_EPS));
+      lpc = bi_log(bi_max(row_dot<R>(rc, sq + NA + NB, NC), (R)BI_EPS));
+    }
+    __syncwarp();
+
+    t3.set_uniform();
+    R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
+    float ma = 0.f, mb = 0.f, mc = 0.f;
+    for (int k = 0; k < p.K; ++k) {
+      t3.messages(xa, xb, xc);
+      xa = a_ok ? xa + lpa : -bi_inf<R>();
+      xb = b_ok ? xb + lpb : -bi_inf<R>();
+      xc = c_ok ? xc + lpc : -bi_inf<R>();
+      ma = group_max_f<NAP, SB>((float)xa);
+      mb = group_max_f<LPU, 1>((float)xb);
+      mc = group_max_f<LPU, 1>((float)xc);
+      const R ean = a_ok ? bi_exp(xa - (R)ma) : (R)0;
+      const R ebn = b_ok ? bi_exp(xb - (R)mb) : (R)0;
+      const R ecn = c_ok ? bi_exp(xc - (R)mc) : (R)0;
+      if (t3.own_b) se[bi] = ebn;
+      if (t3.own_c) se[NB + ci] = ecn;
+      za = group_sum<R, NAP, SB>(ean);
+      __syncwarp();
+      t3.ea = ean;
+      R zbl = (R)0;
+#pragma unroll
+      for (int bl = 0; bl < NBL; ++bl) {
+        t3.eb[bl] = se[t3.bh * NBL + bl];
+        zbl += t3.eb[bl];
+      }
+      zb = group_sum<R, SB, 1>(zbl);
+      zc = (R)0;
+#pragma unroll
+      for (int c = 0; c < NCP; ++c) {
+        t3.ec[c] = se[NB + c];
+        zc += t3.ec[c];
+      }
+      rinv = bi_rcp(za * zb * zc);
+      t3.sa = rinv * za;
+      t3.sb = rinv * zb;
+      t3.sc = rinv * zc;
+      __syncwarp();
+    }
+
+    // ---- final beliefs of the step: outputs, and the next step's prior input
+    const R qa = t3.ea * (rinv * zb * zc);
+    const R qb = (b_ok ? se[bsafe] : (R)0) * (rinv * za * zc);
+    const R qc = (c_ok ? se[NB + csafe] : (R)0) * (rinv * za * zb);
+    if (t3.own_a) sq[a] = qa;
+    if (t3.own_b) sq[NA + bi] = qb;
+    if (t3.own_c) sq[NA + NB + ci] = qc;
+    float *qo = p.q_out + (out_base + t) * p.S;
+    if (live) {
+      if (t3.own_a) qo[p.off[0] + a] = (float)qa;
+      if (t3.own_b) qo[p.off[1] + bi] = (float)qb;
+      if (t3.own_c) qo[p.off[2] + ci] = (float)qc;
+      if (p.logq_out) {
+        float *lo = p.logq_out + (out_base + t) * p.S;
+        if (t3.own_a) lo[p.off[0] + a] = (float)(xa - (R)ma - bi_log(za));
+        if (t3.own_b) lo[p.off[1] + bi] = (float)(xb - (R)mb - bi_log(zb));
+        if (t3.own_c) lo[p.off[2] + ci] = (float)(xc - (R)mc - bi_log(zc));
+      }
+    }
+    if (p.argmax_out) {
+      const int ia = group_argmax<R, NAP, SB>(xa, a_ok ? a : 1 << 20);
+      const int ib = group_argmax<R, LPU, 1>(xb, b_ok ? bi : 1 << 20);
+      const int ic = group_argmax<R, LPU, 1>(xc, c_ok ? ci : 1 << 20);
+      if (live && t3.u == 0) {
+        int32_t *ao = p.argmax_out + (out_base + t) * 3;
+        ao[p.fac[0]] = ia;
+        ao[p.fac[1]] = ib;
+        ao[p.fac[2]] = ic;
+      }
+    }
+    __syncwarp();
+  }
+}
+
+template <typename R, int NA, int NB, int NC, int SB>
+int launch_filter(const Tile3Params &p, cudaStream_t stream) {
+  using TT = Tile3<R, NA, NB, NC, SB>;
+  const int grid = (p.N + TT::UPW - 1) / TT::UPW;
+  bi_tile3_filter_kernel<R, NA, NB, NC, SB><<<grid, 32, 0, stream>>>(p);
+  return cudaGetLastError() == cudaSuccess ? BI_OK : BI_ERR_CUDA;
+}
+
+template <typename R>
+int dispatch_filter(const Tile3Params &p, int na, int nb, int nc, cudaStream_t stream) {
+  if (na == 8 && nb == 6 && nc == 8) return launch_filter<R, 8, 6, 8, 1>(p, stream);
+  if (na == 16 && nb == 12 && nc == 8) return launch_filter<R, 16, 12, 8, 2>(p, stream);
+  if (na == 3 && nb == 2 && nc == 4) return launch_filter<R, 3, 2, 4, 1>(p, stream);
+  return BI_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+// Applicable when the model is one dependency group over exactly its three
+// factors and a compiled tile shape matches; BI_ERR_UNSUPPORTED otherwise.
+int bi_launch_tile3(const BiCall &c, bi_model *mut) {
+  const bi_model *md = c.model;
+  const BiDev &h = md->h;
+  if (c.algo != BI_ALGO_FILTER) return BI_ERR_UNSUPPORTED;
+  if (h.ngroups != 1 || h.F != 3 || h.grp[0].rank != 3) return BI_ERR_UNSUPPORTED;
+  const BiGroup &g = h.grp[0];
+  Tile3Params p;
+  p.nmem = g.mem_end - g.mem_begin;
+  p.P_pad = g.P_pad;
+  for (int i = 0; i < p.nmem; ++i) {
+    const BiMember &mm = h.mem[g.mem_begin + i];
+    p.logA[i] = mm.logA;
+    p.gstride[i] = mm.gstride;
+    p.modality[i] = mm.modality;
+    p.mcount[i] = mm.m;
+  }
+  for (int j = 0; j < 3; ++j) {
+    const int f = g.axis[j];
+    p.fac[j] = f;
+    p.off[j] = h.off[f];
+    p.np[j] = h.npad[f];
+    p.U[j] = h.U[f];
+    p.Bf[j] = h.Bf[f]; p.logB[j] = h.logB[f]; p.logBt[j] = h.logBt[f]; p.Bdag[j] = h.Bdag[f];
+    p.logD[j] = h.logD[f];
+    p.Bstride[j] = h.Bstride[f];
+    p.Dstride[j] = h.Dstride[f];
+  }
+  p.N = c.N; p.T = c.T; p.K = c.K; p.M = h.M; p.S = h.S; p.G = h.G;
+  p.obs = c.obs; p.act = c.act; p.q_out = c.q_out; p.logq_out = c.logq_out;
+  p.argmax_out = c.argmax_out; p.status = h.status;
+  int rc = md->arith == BI_ARITH_F64 ? dispatch_filter<double>(p, g.dim[0], g.dim[1], g.dim[2], c.stream)
+                                     : dispatch_filter<float>(p, g.dim[0], g.dim[1], g.dim[2], c.stream);
+  if (rc == BI_OK) {
+    mut->launches += 1;
+    mut->last_kernel = md->arith == BI_ARITH_F64 ? "tile3_filter_f64" : "tile3_filter_f32";
+  }
+  return rc;
+}

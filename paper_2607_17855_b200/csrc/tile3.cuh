@@ -1,0 +1,182 @@
+// Register-tile contraction core for models whose modalities all depend on the
+// same three factors (one dependency group of rank 3).
+//
+// A "unit" is one agent at one time step.  LPU = NAP * SB lanes of a warp work
+// on one unit (NAP = NA rounded up to a power of two).  The group's summed
+// slice L[a][b][c] (packed order: a slowest, c fastest and padded to NCP) lives
+// in registers: lane (a, bh) holds the NBL = NB / SB values b of its half and
+// all c.  One Jacobi sweep of the three likelihood messages (Section IV,
+// marginalisation) then needs
+//   V[b]    = sum_c L[a][b][c] e_c[c]                       in-lane
+//   ell_a   = sum_b V[b] e_b[b]                             in-lane (+ SB lanes)
+//   ell_b   = sum_a e_a V[b]                                reduce-scatter over the a lanes
+//   ell_c   = sum_a e_a sum_b e_b[b] L[a][b][c]             reduce-scatter over all lanes
+// about 2 P multiply-adds for P = NA*NB*NC.  Beliefs are carried unnormalised
+// (e = exp(x - max), z = sum e) and the three messages are rescaled by
+// 1/(z z) afterwards, so one reciprocal per sweep replaces the divisions.
+#pragma once
+#include "bi_device.cuh"
+
+template <int X> struct Pow2Ceil { static constexpr int v = X <= 1 ? 1 : 2 * Pow2Ceil<(X + 1) / 2>::v; };
+template <> struct Pow2Ceil<1> { static constexpr int v = 1; };
+template <int X> struct Log2 { static constexpr int v = 1 + Log2<X / 2>::v; };
+template <> struct Log2<1> { static constexpr int v = 0; };
+
+// Sum v[i] over the NL lanes {lane ^ (k * STR)}; afterwards v[0] holds the
+// total of element (sub >> (log2 NL - log2 PV)), where sub is the lane's index
+// within the NL lanes.  PV and NL are powers of two, PV <= NL.
+template <typename R, int PV, int NL, int STR>
+__device__ __forceinline__ R reduce_scatter(R (&v)[PV], int sub) {
+  static_assert(PV <= NL, "more values than lanes");
+  if (NL == 1) return v[0];
+#pragma unroll
+  for (int d = NL / 2, cur = PV; d >= 1; d >>= 1) {
+    const bool up = (sub & d) != 0;
+    if (cur > 1) {
+      const int half = cur / 2;
+#pragma unroll
+      for (int i = 0; i < half; ++i) {
+        R send = up ? v[i] : v[i + half];
+        R keep = up ? v[i + half] : v[i];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, d * STR);
+      }
+      cur = half;
+    } else {
+      v[0] += __shfl_xor_sync(0xffffffffu, v[0], d * STR);
+    }
+  }
+  return v[0];
+}
+
+template <typename R, int NL, int STR>
+__device__ __forceinline__ R group_sum(R v) {
+#pragma unroll
+  for (int d = NL / 2; d >= 1; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d * STR);
+  return v;
+}
+// max over the group, taken in float: any common shift close to the maximum
+// makes the softmax exact, so float precision is enough for it
+template <int NL, int STR>
+__device__ __forceinline__ float group_max_f(float v) {
+#pragma unroll
+  for (int d = NL / 2; d >= 1; d >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, d * STR));
+  return v;
+}
+// exact argmax over the group: largest x, lowest index among equals
+template <typename R, int NL, int STR>
+__device__ __forceinline__ int group_argmax(R x, int idx) {
+#pragma unroll
+  for (int d = NL / 2; d >= 1; d >>= 1) {
+    R xo = __shfl_xor_sync(0xffffffffu, x, d * STR);
+    int io = __shfl_xor_sync(0xffffffffu, idx, d * STR);
+    if (xo > x || (xo == x && io < idx)) { x = xo; idx = io; }
+  }
+  return idx;
+}
+
+// reciprocal: hardware seed refined to working precision
+__device__ __forceinline__ float bi_rcp(float x) { return 1.0f / x; }
+__device__ __forceinline__ double bi_rcp(double x) { return 1.0 / x; }
+
+template <typename R, int NA_, int NB_, int NC_, int SB_>
+struct Tile3 {
+  static constexpr int NA = NA_, NB = NB_, NC = NC_, SB = SB_;
+  static constexpr int NAP = Pow2Ceil<NA>::v;
+  static constexpr int LPU = NAP * SB;          // lanes per unit
+  static constexpr int UPW = 32 / LPU;          // units per warp
+  static constexpr int NBL = NB / SB;           // b values per lane
+  static constexpr int NCP = (NC + 3) & ~3;     // padded c
+  static constexpr int PB = Pow2Ceil<NBL>::v;   // reduce-scatter widths
+  static constexpr int PC = Pow2Ceil<NCP>::v;
+  static constexpr int SHB = Log2<NAP>::v - Log2<PB>::v;  // duplicate bits of the b owner index
+  static constexpr int SHC = Log2<LPU>::v - Log2<PC>::v;
+  static_assert(NB % SB == 0, "SB must divide NB");
+  static_assert(LPU <= 32 && PB <= NAP && PC <= LPU, "tile does not fit a warp");
+
+  // lane coordinates
+  int u, a, bh;       // lane within unit, a index, b half
+  int bi, ci;         // owned b (global index) and c after the reduce-scatters
+  bool a_ok, own_a, own_b, own_c;  // valid a; designated writer of x_a / x_b / x_c
+
+  R L[NBL][NCP];      // this lane's part of the summed slice
+  R ea, eb[NBL], ec[NCP];  // unnormalised beliefs this lane contracts with
+  R sa, sb, sc;       // message scales 1/(z_b z_c), 1/(z_a z_c), 1/(z_a z_b)
+
+  __device__ __forceinline__ void init_lane(int lane) {
+    u = lane % LPU;
+    a = u / SB;
+    bh = u % SB;
+    a_ok = a < NA;
+    const int ib = a >> SHB;
+    bi = bh * NBL + ib;
+    ci = u >> SHC;
+    own_a = a_ok && bh == 0;
+    own_b = ib < NBL && (a & ((1 << SHB) - 1)) == 0;
+    own_c = ci < NC && (u & ((1 << SHC) - 1)) == 0;
+  }
+
+  // L[b][c] = sum over the group's modalities of their observed slices
+  __device__ __forceinline__ void load_slices(const R *const *slice, int nmem) {
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl)
+#pragma unroll
+      for (int c = 0; c < NCP; ++c) L[bl][c] = (R)0;
+    if (!a_ok) return;
+    const int base = (a * NB + bh * NBL) * NCP;
+    for (int mi = 0; mi < nmem; ++mi) {
+      const R *p = slice[mi] + base;
+#pragma unroll
+      for (int bl = 0; bl < NBL; ++bl)
+#pragma unroll
+        for (int c4 = 0; c4 < NCP / 4; ++c4) {
+          Vec4<R> x = ldg4(p + bl * NCP + 4 * c4);
+          L[bl][4 * c4 + 0] += x.x; L[bl][4 * c4 + 1] += x.y;
+          L[bl][4 * c4 + 2] += x.z; L[bl][4 * c4 + 3] += x.w;
+        }
+    }
+  }
+
+  __device__ __forceinline__ void set_uniform() {
+    ea = a_ok ? (R)1 : (R)0;
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl) eb[bl] = (R)1;
+#pragma unroll
+    for (int c = 0; c < NCP; ++c) ec[c] = c < NC ? (R)1 : (R)0;
+    sa = (R)1 / (R)(NB * NC);
+    sb = (R)1 / (R)(NA * NC);
+    sc = (R)1 / (R)(NA * NB);
+  }
+
+  // the three likelihood messages for the logits this lane owns
+  __device__ __forceinline__ void messages(R &xa, R &xb, R &xc) {
+    R V[NBL];
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl) {
+      R v = (R)0;
+#pragma unroll
+      for (int c = 0; c < NCP; ++c) v = fma(L[bl][c], ec[c], v);
+      V[bl] = v;
+    }
+    R la = (R)0;
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl) la = fma(V[bl], eb[bl], la);
+    la = group_sum<R, SB, 1>(la);
+    R pb[PB], pc[PC];
+#pragma unroll
+    for (int i = 0; i < PB; ++i) pb[i] = i < NBL ? ea * V[i < NBL ? i : 0] : (R)0;
+#pragma unroll
+    for (int c = 0; c < PC; ++c) {
+      R w = (R)0;
+      if (c < NCP) {
+#pragma unroll
+        for (int bl = 0; bl < NBL; ++bl) w = fma(eb[bl], L[bl][c], w);
+      }
+      pc[c] = ea * w;
+    }
+    R lb = reduce_scatter<R, PB, NAP, SB>(pb, a);
+    R lc = reduce_scatter<R, PC, LPU, 1>(pc, u);
+    xa = la * sa;
+    xb = lb * sb;
+    xc = lc * sc;
+  }
+};

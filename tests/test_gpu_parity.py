@@ -143,3 +143,23 @@ def test_float32_arithmetic_mode(c, algo, kw):
     well = floor < 1e-7  # agents whose result barely moves under float32 rounding of the state
     assert well.any() or c == 4
     assert (err[well] <= 1e-5).all()
+
+
+# ---- the register-tile filtering kernels (single rank-3 dependency group)
+
+@pytest.mark.parametrize("arith", ["f64", "f32"])
+def test_tile_filter_shapes_and_ragged_batches(arith):
+    strict = arith == "f64"
+    # 8 lanes per agent, 4 agents per warp: a batch that does not fill the last warp
+    res = check_workload(make_config(2, N=97, T=7), "filter", arith=arith, strict=strict)
+    assert res["kernel"] == f"tile3_filter_{arith}", res
+    # 32 lanes per agent, per-agent models
+    res = check_workload(make_config(4, N=5, T=6), "filter", arith=arith, strict=strict)
+    assert res["kernel"] == f"tile3_filter_{arith}", res
+    # padded lanes: n = [4, 3, 2] packs as a = 3 (4 lanes), b = 2, c = 4
+    w = _custom(31, [4, 3, 2], [3, 5, 2], [[0, 1, 2], [2, 0, 1], [1, 2, 0]], [2, 3, 1], N=11, T=5, K=9,
+                sparsity=0.5 if strict else 0.0)
+    res = check_workload(w, "filter", arith=arith, strict=strict)
+    assert res["kernel"] == f"tile3_filter_{arith}", res
+    if not strict:
+        assert res["q_max_err"] < 1e-3
