@@ -58,7 +58,7 @@ __global__ void bi_pack_A_kernel(PackA p) {
 // B[g][s_next][s_prev][u] -> four [g][u][row][npad] matrices
 template <typename R>
 __global__ void bi_pack_B_kernel(const float *__restrict__ B, int G, int n, int npad, int U,
-                                 R *Bf, R *logB, R *logBt, R *Bdag) {
+                                 R *Bf, R *logB, R *logBt, R *Bdag, R *BfT, R *BdagT) {
   int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   int64_t total = (int64_t)G * U * n * npad;
   if (e >= total) return;
@@ -68,7 +68,7 @@ __global__ void bi_pack_B_kernel(const float *__restrict__ B, int G, int n, int 
   int64_t r2 = r1 / n;
   int u = (int)(r2 % U);
   int64_t g = r2 / U;
-  R f = 0, lf = 0, lt = 0, bd = 0;
+  R f = 0, lf = 0, lt = 0, bd = 0, ft = 0, bdt = 0;
   if (c < n) {
     const float *Bg = B + g * (int64_t)n * n * U;
     // forward: row = next state, column = previous state
@@ -81,11 +81,49 @@ __global__ void bi_pack_B_kernel(const float *__restrict__ B, int G, int n, int 
     double rowsum = 0.0;
     for (int sp = 0; sp < n; ++sp) rowsum += (double)Bg[((int64_t)c * n + sp) * U + u];
     bd = (R)(rowsum > 0.0 ? bt / rowsum : 1.0 / n);
+    ft = (R)bt;
+    // row = next state r, column = previous state c, normalised over the previous states
+    double rs2 = 0.0;
+    for (int sp = 0; sp < n; ++sp) rs2 += (double)Bg[((int64_t)r * n + sp) * U + u];
+    bdt = (R)(rs2 > 0.0 ? b / rs2 : 1.0 / n);
   }
   Bf[e] = f;
   logB[e] = lf;
   logBt[e] = lt;
   Bdag[e] = bd;
+  BfT[e] = ft;
+  BdagT[e] = bdt;
+}
+
+// Lane-interleaved slice layout of the register-tile kernels: within one
+// outcome's slice, 16-byte vector v of lane u (u = a * SB + b / NBL) sits at
+// (v * LPU + u) * VE, so one warp load instruction reads whole cache lines.
+struct PackTile {
+  const float *src;
+  void *dst;
+  int64_t total;    // G * m * P_tile
+  int32_t P, P_tile, NA, NB, NC, NCP, NAP, SB, NBL, VE;
+  int64_t sstride[3];
+};
+
+template <typename R>
+__global__ void bi_pack_tile_kernel(PackTile p) {
+  int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= p.total) return;
+  int64_t go = e / p.P_tile;
+  int32_t idx = (int32_t)(e - go * p.P_tile);
+  const int LPU = p.NAP * p.SB;
+  int within = idx % p.VE, t = idx / p.VE;
+  int u = t % LPU, v = t / LPU;
+  int j = v * p.VE + within;
+  int bl = j / p.NCP, c = j % p.NCP;
+  int a = u / p.SB, b = (u % p.SB) * p.NBL + bl;
+  R out = (R)0;
+  if (a < p.NA && c < p.NC) {
+    int64_t s = go * p.P + a * p.sstride[0] + b * p.sstride[1] + c * p.sstride[2];
+    out = (R)log(fmax((double)p.src[s], 1e-16));
+  }
+  ((R *)p.dst)[e] = out;
 }
 
 template <typename R>
@@ -285,6 +323,11 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
   h.Ltot = Ltot;
   md->V0max = V0; md->V1max = V1; md->rows_max = rows_max;
 
+  // a register-tile shape applies when the model is one rank-3 group over exactly its factors
+  md->tile_sb = 0;
+  if (h.ngroups == 1 && F == 3 && h.grp[0].rank == 3)
+    md->tile_sb = bi_tile3_shape(h.grp[0].dim[0], h.grp[0].dim[1], h.grp[0].dim[2]);
+
   // ---- allocate and pack
   rc = dev_alloc(md, (void **)&h.status, sizeof(uint32_t));
   if (rc == BI_OK && cudaMemsetAsync(h.status, 0, sizeof(uint32_t), stream) != cudaSuccess) rc = BI_ERR_CUDA;
@@ -325,17 +368,46 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
       if (arith == BI_ARITH_F64) bi_pack_A_kernel<double><<<(unsigned)blocks, threads, 0, stream>>>(p);
       else bi_pack_A_kernel<float><<<(unsigned)blocks, threads, 0, stream>>>(p);
       if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+      if (rc == BI_OK && md->tile_sb > 0) {
+        PackTile q;
+        memset(&q, 0, sizeof(q));
+        q.src = desc->A[i];
+        q.P = p.P;
+        q.NA = g.dim[0]; q.NB = g.dim[1]; q.NC = g.dim[2];
+        q.NCP = bi_pad4(q.NC);
+        q.NAP = 1;
+        while (q.NAP < q.NA) q.NAP <<= 1;
+        q.SB = md->tile_sb;
+        q.NBL = q.NB / q.SB;
+        q.VE = (int)(16 / esz);
+        q.P_tile = q.NAP * q.NB * q.NCP;
+        md->tile_P = q.P_tile;
+        for (int j = 0; j < 3; ++j) q.sstride[j] = p.sstride[j];
+        q.total = (int64_t)G * mm.m * q.P_tile;
+        void *td = nullptr;
+        rc = dev_alloc(md, &td, (size_t)q.total * esz);
+        if (rc != BI_OK) break;
+        q.dst = td;
+        mm.logA_tile = td;
+        int64_t tb = (q.total + threads - 1) / threads;
+        if (arith == BI_ARITH_F64) bi_pack_tile_kernel<double><<<(unsigned)tb, threads, 0, stream>>>(q);
+        else bi_pack_tile_kernel<float><<<(unsigned)tb, threads, 0, stream>>>(q);
+        if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+      }
     }
   }
   for (int f = 0; f < F && rc == BI_OK; ++f) {
     int n = h.n[f], npad = h.npad[f], U = h.U[f];
     size_t count = (size_t)G * U * n * npad;
-    void *bf, *lb, *lt, *bd, *ld;
+    void *bf, *lb, *lt, *bd, *ld, *bft, *bdt;
     if ((rc = dev_alloc(md, &bf, count * esz)) != BI_OK) break;
     if ((rc = dev_alloc(md, &lb, count * esz)) != BI_OK) break;
     if ((rc = dev_alloc(md, &lt, count * esz)) != BI_OK) break;
     if ((rc = dev_alloc(md, &bd, count * esz)) != BI_OK) break;
     if ((rc = dev_alloc(md, &ld, (size_t)G * npad * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &bft, count * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &bdt, count * esz)) != BI_OK) break;
+    h.BfT[f] = bft; h.BdagT[f] = bdt;
     h.Bf[f] = bf; h.logB[f] = lb; h.logBt[f] = lt; h.Bdag[f] = bd; h.logD[f] = ld;
     h.Bstride[f] = (G == 1) ? 0 : (int64_t)U * n * npad;
     h.Dstride[f] = (G == 1) ? 0 : npad;
@@ -344,11 +416,13 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
     unsigned gd = (unsigned)(((size_t)G * npad + threads - 1) / threads);
     if (arith == BI_ARITH_F64) {
       bi_pack_B_kernel<double><<<gb, threads, 0, stream>>>(desc->B[f], G, n, npad, U, (double *)bf,
-                                                           (double *)lb, (double *)lt, (double *)bd);
+                                                           (double *)lb, (double *)lt, (double *)bd,
+                                                           (double *)bft, (double *)bdt);
       bi_pack_D_kernel<double><<<gd, threads, 0, stream>>>(desc->D[f], G, n, npad, (double *)ld);
     } else {
       bi_pack_B_kernel<float><<<gb, threads, 0, stream>>>(desc->B[f], G, n, npad, U, (float *)bf,
-                                                          (float *)lb, (float *)lt, (float *)bd);
+                                                          (float *)lb, (float *)lt, (float *)bd,
+                                                          (float *)bft, (float *)bdt);
       bi_pack_D_kernel<float><<<gd, threads, 0, stream>>>(desc->D[f], G, n, npad, (float *)ld);
     }
     if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;

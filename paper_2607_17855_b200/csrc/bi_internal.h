@@ -45,6 +45,7 @@ struct BiGroup {
 
 struct BiMember {
   const void *logA;   // packed [G][m][P_pad], float or double (the handle's arithmetic)
+  const void *logA_tile;  // lane-interleaved copy [G][m][P_tile] for the register-tile kernels, or NULL
   int64_t gstride;    // floats per model (0 when the model is shared)
   int32_t m, modality, P_pad, pad_;
 };
@@ -61,6 +62,8 @@ struct BiDev {
   const void *logB[BI_MAX_F];  // ln of the same
   const void *logBt[BI_MAX_F]; // [s_prev][s_next]      = ln B[s_next, s_prev, u]
   const void *Bdag[BI_MAX_F];  // [s_prev][s_next]      = B[s_next, s_prev, u] / sum_r B[s_next, r, u]
+  const void *BfT[BI_MAX_F];   // [s_prev][s_next]      = B[s_next, s_prev, u]
+  const void *BdagT[BI_MAX_F]; // [s_next][s_prev]      = B[s_next, s_prev, u] / sum_r B[s_next, r, u]
   const void *logD[BI_MAX_F];  // [G][npad]
   int64_t Bstride[BI_MAX_F];    // floats per model in each B array (0 when shared)
   int64_t Dstride[BI_MAX_F];
@@ -71,12 +74,14 @@ struct BiDev {
 struct bi_model {
   BiDev h;          // host copy (device pointers inside)
   BiDev *d;         // device copy
-  void *allocs[8 + 2 * BI_MAX_M + 8 * BI_MAX_F];
+  void *allocs[8 + 2 * BI_MAX_M + 8 * BI_MAX_F];  // status, descriptor, 2 per modality, 7 per factor
   int nalloc;
   int arith;        // BI_ARITH_F64 or BI_ARITH_F32
   int device;
   int sm_count;
   int max_smem_optin;
+  int tile_sb;      // > 0: a register-tile shape matches; lanes along b per (agent, step)
+  int tile_P;       // elements per lane-interleaved slice
   int V0max, V1max; // floats needed by the generic kernel's two intermediate buffers
   int rows_max;     // largest first-level row count over groups
   int64_t launches;
@@ -96,3 +101,5 @@ struct BiCall {
 // this model / call: the dispatcher tries the next one) or an error.
 int bi_launch_generic(const BiCall &c, bi_model *mut);
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
+// SB of the compiled register-tile shape for packed dims (na, nb, nc), or 0
+int bi_tile3_shape(int na, int nb, int nc);

@@ -2,6 +2,7 @@
 // on the same three factors and the model has exactly those factors).
 // Filtering: a few lanes per agent, the step recursion and the iteration loop
 // inside one launch, the summed slice of the current step held in registers.
+#include <cstdlib>
 #include "bi_internal.h"
 #include "tile3.cuh"
 
@@ -11,12 +12,12 @@ struct Tile3Params {
   const void *logA[BI_MAX_M];
   int64_t gstride[BI_MAX_M];
   int32_t modality[BI_MAX_M], mcount[BI_MAX_M];
-  int32_t nmem, P_pad;
+  int32_t nmem, P_tile;
   int32_t fac[3];   // factor ids of the axes a, b, c
   int32_t off[3];   // offsets of those factors in an output belief vector
   int32_t np[3];    // padded row length of their transition matrices
   int32_t U[3];
-  const void *Bf[3], *logB[3], *logBt[3], *Bdag[3], *logD[3];
+  const void *Bf[3], *logB[3], *logBt[3], *Bdag[3], *BfT[3], *BdagT[3], *logD[3];
   int64_t Bstride[3], Dstride[3];
   int32_t N, T, K, M, S, G;
   const int32_t *obs, *act;
@@ -25,14 +26,16 @@ struct Tile3Params {
   uint32_t *status;
 };
 
-template <typename R>
-__device__ __forceinline__ R row_dot(const R *__restrict__ row, const R *q, int n) {
-  R p = (R)0;
-  for (int r = 0; r < n; ++r) p = fma(__ldg(row + r), q[r], p);
-  return p;
+// sum_r M[r][s] q[r] for this lane's s: col points at M[0][s], rows are `stride` apart
+template <typename R, int N>
+__device__ __forceinline__ R col_dot(const R *__restrict__ col, int stride, const R *q) {
+  R x[N];
+#pragma unroll
+  for (int r = 0; r < N; ++r) x[r] = __ldg(col + r * stride) * q[r];
+  return tree_sum<R, N>(x);
 }
 
-template <typename R, int NA, int NB, int NC, int SB>
+template <typename R, int NA, int NB, int NC, int SB, bool STALE>
 __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p) {
   using TT = Tile3<R, NA, NB, NC, SB>;
   constexpr int LPU = TT::LPU, UPW = TT::UPW, NBL = TT::NBL, NCP = TT::NCP, NAP = TT::NAP;
@@ -62,7 +65,7 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
     for (int mi = 0; mi < p.nmem; ++mi) {
       int o = clamp_flag(__ldg(p.obs + (out_base + t) * p.M + p.modality[mi]), p.mcount[mi], p.status,
                          BI_FLAG_OBS_RANGE);
-      slice[mi] = (const R *)p.logA[mi] + (size_t)g * p.gstride[mi] + (size_t)o * p.P_pad;
+      slice[mi] = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile;
     }
     t3.load_slices(slice, p.nmem);
 
@@ -77,26 +80,35 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       int ua = clamp_flag(__ldg(ac + p.fac[0]), p.U[0], p.status, BI_FLAG_ACT_RANGE);
       int ub = clamp_flag(__ldg(ac + p.fac[1]), p.U[1], p.status, BI_FLAG_ACT_RANGE);
       int uc = clamp_flag(__ldg(ac + p.fac[2]), p.U[2], p.status, BI_FLAG_ACT_RANGE);
-      const R *ra = (const R *)p.Bf[0] + (size_t)g * p.Bstride[0] + ((size_t)ua * NA + asafe) * p.np[0];
-      const R *rb = (const R *)p.Bf[1] + (size_t)g * p.Bstride[1] + ((size_t)ub * NB + bsafe) * p.np[1];
-      const R *rc = (const R *)p.Bf[2] + (size_t)g * p.Bstride[2] + ((size_t)uc * NC + csafe) * p.np[2];
-      lpa = bi_log(bi_max(row_dot<R>(ra, sq, NA), (R)BI_EPS));
-      lpb = bi_log(bi_max(row_dot<R>(rb, sq + NA, NB), (R)BI_EPS));
-      lpc = bi_log(bi_max(row_dot<R>(rc, sq + NA + NB, NC), (R)BI_EPS));
+      // transposed forward matrices [previous][next]: the lanes of a unit read consecutive next states
+      const R *ta = (const R *)p.BfT[0] + (size_t)g * p.Bstride[0] + (size_t)ua * NA * p.np[0] + asafe;
+      const R *tb = (const R *)p.BfT[1] + (size_t)g * p.Bstride[1] + (size_t)ub * NB * p.np[1] + bsafe;
+      const R *tc = (const R *)p.BfT[2] + (size_t)g * p.Bstride[2] + (size_t)uc * NC * p.np[2] + csafe;
+      lpa = bi_log(bi_max(col_dot<R, NA>(ta, p.np[0], sq), (R)BI_EPS));
+      lpb = bi_log(bi_max(col_dot<R, NB>(tb, p.np[1], sq + NA), (R)BI_EPS));
+      lpc = bi_log(bi_max(col_dot<R, NC>(tc, p.np[2], sq + NA + NB), (R)BI_EPS));
     }
     __syncwarp();
 
     t3.set_uniform();
     R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
-    float ma = 0.f, mb = 0.f, mc = 0.f;
+    float ma = 0.f, mb = 0.f, mc = 0.f;     // softmax shifts in use
+    float pma = 0.f, pmb = 0.f, pmc = 0.f;  // exact maxima of the previous iterate
     for (int k = 0; k < p.K; ++k) {
       t3.messages(xa, xb, xc);
       xa = a_ok ? xa + lpa : -bi_inf<R>();
       xb = b_ok ? xb + lpb : -bi_inf<R>();
       xc = c_ok ? xc + lpc : -bi_inf<R>();
-      ma = group_max_f<NAP, SB>((float)xa);
-      mb = group_max_f<LPU, 1>((float)xb);
-      mc = group_max_f<LPU, 1>((float)xc);
+      // Softmax is invariant to the shift; any shift that keeps the exponents
+      // in range is exact.  With STALE the previous iterate's maximum is used
+      // (logits move by less than the range bound between iterates), which
+      // takes the max reduction off the dependency chain.
+      const float cma = group_max_f<NAP, SB>((float)xa);
+      const float cmb = group_max_f<LPU, 1>((float)xb);
+      const float cmc = group_max_f<LPU, 1>((float)xc);
+      if (!STALE || k == 0) { ma = cma; mb = cmb; mc = cmc; }
+      else { ma = pma; mb = pmb; mc = pmc; }
+      pma = cma; pmb = cmb; pmc = cmc;
       const R ean = a_ok ? bi_exp(xa - (R)ma) : (R)0;
       const R ebn = b_ok ? bi_exp(xb - (R)mb) : (R)0;
       const R ecn = c_ok ? bi_exp(xc - (R)mc) : (R)0;
@@ -105,19 +117,12 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       za = group_sum<R, NAP, SB>(ean);
       __syncwarp();
       t3.ea = ean;
-      R zbl = (R)0;
 #pragma unroll
-      for (int bl = 0; bl < NBL; ++bl) {
-        t3.eb[bl] = se[t3.bh * NBL + bl];
-        zbl += t3.eb[bl];
-      }
-      zb = group_sum<R, SB, 1>(zbl);
-      zc = (R)0;
+      for (int bl = 0; bl < NBL; ++bl) t3.eb[bl] = se[t3.bh * NBL + bl];
 #pragma unroll
-      for (int c = 0; c < NCP; ++c) {
-        t3.ec[c] = se[NB + c];
-        zc += t3.ec[c];
-      }
+      for (int c = 0; c < NCP; ++c) t3.ec[c] = se[NB + c];
+      zb = group_sum<R, SB, 1>(tree_sum<R, NBL>(t3.eb));
+      zc = tree_sum<R, NCP>(t3.ec);
       rinv = bi_rcp(za * zb * zc);
       t3.sa = rinv * za;
       t3.sb = rinv * zb;
@@ -163,19 +168,36 @@ template <typename R, int NA, int NB, int NC, int SB>
 int launch_filter(const Tile3Params &p, cudaStream_t stream) {
   using TT = Tile3<R, NA, NB, NC, SB>;
   const int grid = (p.N + TT::UPW - 1) / TT::UPW;
-  bi_tile3_filter_kernel<R, NA, NB, NC, SB><<<grid, 32, 0, stream>>>(p);
+  // shifts may lag one iterate only where the exponent range has room for the
+  // largest possible move of a logit: float64 and at most 12 modalities
+  if (sizeof(R) == 8 && p.nmem <= 12)
+    bi_tile3_filter_kernel<R, NA, NB, NC, SB, true><<<grid, 32, 0, stream>>>(p);
+  else
+    bi_tile3_filter_kernel<R, NA, NB, NC, SB, false><<<grid, 32, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? BI_OK : BI_ERR_CUDA;
 }
 
+// compiled tile shapes: packed dims (a, b, c) and the lanes along b
+#define BI_TILE3_SHAPES(X) X(8, 6, 8, 1) X(16, 12, 8, 2) X(3, 2, 4, 1)
+
 template <typename R>
 int dispatch_filter(const Tile3Params &p, int na, int nb, int nc, cudaStream_t stream) {
-  if (na == 8 && nb == 6 && nc == 8) return launch_filter<R, 8, 6, 8, 1>(p, stream);
-  if (na == 16 && nb == 12 && nc == 8) return launch_filter<R, 16, 12, 8, 2>(p, stream);
-  if (na == 3 && nb == 2 && nc == 4) return launch_filter<R, 3, 2, 4, 1>(p, stream);
+#define X(A, B, C, S) \
+  if (na == A && nb == B && nc == C) return launch_filter<R, A, B, C, S>(p, stream);
+  BI_TILE3_SHAPES(X)
+#undef X
   return BI_ERR_UNSUPPORTED;
 }
 
 }  // namespace
+
+int bi_tile3_shape(int na, int nb, int nc) {
+#define X(A, B, C, S) \
+  if (na == A && nb == B && nc == C) return S;
+  BI_TILE3_SHAPES(X)
+#undef X
+  return 0;
+}
 
 // Applicable when the model is one dependency group over exactly its three
 // factors and a compiled tile shape matches; BI_ERR_UNSUPPORTED otherwise.
@@ -183,14 +205,14 @@ int bi_launch_tile3(const BiCall &c, bi_model *mut) {
   const bi_model *md = c.model;
   const BiDev &h = md->h;
   if (c.algo != BI_ALGO_FILTER) return BI_ERR_UNSUPPORTED;
-  if (h.ngroups != 1 || h.F != 3 || h.grp[0].rank != 3) return BI_ERR_UNSUPPORTED;
+  if (md->tile_sb <= 0) return BI_ERR_UNSUPPORTED;
   const BiGroup &g = h.grp[0];
   Tile3Params p;
   p.nmem = g.mem_end - g.mem_begin;
-  p.P_pad = g.P_pad;
+  p.P_tile = md->tile_P;
   for (int i = 0; i < p.nmem; ++i) {
     const BiMember &mm = h.mem[g.mem_begin + i];
-    p.logA[i] = mm.logA;
+    p.logA[i] = mm.logA_tile;
     p.gstride[i] = mm.gstride;
     p.modality[i] = mm.modality;
     p.mcount[i] = mm.m;
@@ -202,6 +224,7 @@ int bi_launch_tile3(const BiCall &c, bi_model *mut) {
     p.np[j] = h.npad[f];
     p.U[j] = h.U[f];
     p.Bf[j] = h.Bf[f]; p.logB[j] = h.logB[f]; p.logBt[j] = h.logBt[f]; p.Bdag[j] = h.Bdag[f];
+    p.BfT[j] = h.BfT[f]; p.BdagT[j] = h.BdagT[f];
     p.logD[j] = h.logD[f];
     p.Bstride[j] = h.Bstride[f];
     p.Dstride[j] = h.Dstride[f];

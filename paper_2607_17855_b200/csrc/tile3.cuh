@@ -74,9 +74,40 @@ __device__ __forceinline__ int group_argmax(R x, int idx) {
   return idx;
 }
 
+__device__ __forceinline__ void ldg_vec(const float *p, float (&x)[4]) {
+  float4 v = __ldg(reinterpret_cast<const float4 *>(p));
+  x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+}
+__device__ __forceinline__ void ldg_vec(const double *p, double (&x)[2]) {
+  double2 v = __ldg(reinterpret_cast<const double2 *>(p));
+  x[0] = v.x; x[1] = v.y;
+}
+
+// pairwise sum of a register array (short dependency chain)
+template <typename R, int N>
+__device__ __forceinline__ R tree_sum(const R (&v)[N]) {
+  R t[N];
+#pragma unroll
+  for (int i = 0; i < N; ++i) t[i] = v[i];
+#pragma unroll
+  for (int w = 1; w < N; w *= 2)
+#pragma unroll
+    for (int i = 0; i + w < N; i += 2 * w) t[i] += t[i + w];
+  return t[0];
+}
+
 // reciprocal: hardware seed refined to working precision
 __device__ __forceinline__ float bi_rcp(float x) { return 1.0f / x; }
-__device__ __forceinline__ double bi_rcp(double x) { return 1.0 / x; }
+__device__ __forceinline__ double bi_rcp(double x) {
+  // x is a product of sums of exponentials, each in [1, 32]: a normal number.
+  // Hardware seed (about 20 bits) and two Newton steps reach full precision.
+  double y;
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+  double e = fma(-x, y, 1.0);
+  y = fma(y, e, y);
+  e = fma(-x, y, 1.0);
+  return fma(y, e, y);
+}
 
 template <typename R, int NA_, int NB_, int NC_, int SB_>
 struct Tile3 {
@@ -115,24 +146,27 @@ struct Tile3 {
     own_c = ci < NC && (u & ((1 << SHC) - 1)) == 0;
   }
 
-  // L[b][c] = sum over the group's modalities of their observed slices
+  // L[b][c] = sum over the group's modalities of their observed slices.  The
+  // slices are stored lane-interleaved (16-byte vector v of lane u at
+  // (v * LPU + u) * VE), so each load instruction of a unit reads LPU * 16
+  // contiguous bytes.
+  static constexpr int VE = 16 / (int)sizeof(R);
+  static constexpr int NV = NBL * NCP / VE;
+  static constexpr int P_TILE = NAP * NB * NCP;
   __device__ __forceinline__ void load_slices(const R *const *slice, int nmem) {
 #pragma unroll
     for (int bl = 0; bl < NBL; ++bl)
 #pragma unroll
       for (int c = 0; c < NCP; ++c) L[bl][c] = (R)0;
-    if (!a_ok) return;
-    const int base = (a * NB + bh * NBL) * NCP;
     for (int mi = 0; mi < nmem; ++mi) {
-      const R *p = slice[mi] + base;
+      const R *p = slice[mi] + u * VE;
 #pragma unroll
-      for (int bl = 0; bl < NBL; ++bl)
+      for (int v = 0; v < NV; ++v) {
+        R x[VE];
+        ldg_vec(p + v * LPU * VE, x);
 #pragma unroll
-        for (int c4 = 0; c4 < NCP / 4; ++c4) {
-          Vec4<R> x = ldg4(p + bl * NCP + 4 * c4);
-          L[bl][4 * c4 + 0] += x.x; L[bl][4 * c4 + 1] += x.y;
-          L[bl][4 * c4 + 2] += x.z; L[bl][4 * c4 + 3] += x.w;
-        }
+        for (int i = 0; i < VE; ++i) L[(v * VE + i) / NCP][(v * VE + i) % NCP] += x[i];
+      }
     }
   }
 
@@ -149,30 +183,30 @@ struct Tile3 {
 
   // the three likelihood messages for the logits this lane owns
   __device__ __forceinline__ void messages(R &xa, R &xb, R &xc) {
-    R V[NBL];
+    // V[b] = sum_c L[b][c] e_c[c] and W[c] = sum_b e_b[b] L[b][c]: independent
+    // accumulators advance together so no multiply-add waits on the previous one
+    R V[NBL], W[NCP];
 #pragma unroll
-    for (int bl = 0; bl < NBL; ++bl) {
-      R v = (R)0;
+    for (int bl = 0; bl < NBL; ++bl) V[bl] = (R)0;
 #pragma unroll
-      for (int c = 0; c < NCP; ++c) v = fma(L[bl][c], ec[c], v);
-      V[bl] = v;
-    }
-    R la = (R)0;
+    for (int c = 0; c < NCP; ++c) W[c] = (R)0;
 #pragma unroll
-    for (int bl = 0; bl < NBL; ++bl) la = fma(V[bl], eb[bl], la);
-    la = group_sum<R, SB, 1>(la);
+    for (int c = 0; c < NCP; ++c)
+#pragma unroll
+      for (int bl = 0; bl < NBL; ++bl) V[bl] = fma(L[bl][c], ec[c], V[bl]);
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl)
+#pragma unroll
+      for (int c = 0; c < NCP; ++c) W[c] = fma(eb[bl], L[bl][c], W[c]);
+    R lav[NBL];
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl) lav[bl] = V[bl] * eb[bl];
+    R la = group_sum<R, SB, 1>(tree_sum<R, NBL>(lav));
     R pb[PB], pc[PC];
 #pragma unroll
     for (int i = 0; i < PB; ++i) pb[i] = i < NBL ? ea * V[i < NBL ? i : 0] : (R)0;
 #pragma unroll
-    for (int c = 0; c < PC; ++c) {
-      R w = (R)0;
-      if (c < NCP) {
-#pragma unroll
-        for (int bl = 0; bl < NBL; ++bl) w = fma(eb[bl], L[bl][c], w);
-      }
-      pc[c] = ea * w;
-    }
+    for (int c = 0; c < PC; ++c) pc[c] = c < NCP ? ea * W[c < NCP ? c : 0] : (R)0;
     R lb = reduce_scatter<R, PB, NAP, SB>(pb, a);
     R lc = reduce_scatter<R, PC, LPU, 1>(pc, u);
     xa = la * sa;
