@@ -465,6 +465,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   c.stream = (cudaStream_t)cuda_stream;
   bi_model *mut = const_cast<bi_model *>(model);
   int rc = bi_launch_tile3(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;
 }

@@ -101,5 +101,6 @@ struct BiCall {
 // this model / call: the dispatcher tries the next one) or an error.
 int bi_launch_generic(const BiCall &c, bi_model *mut);
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
+int bi_launch_tile3_window(const BiCall &c, bi_model *mut);
 // SB of the compiled register-tile shape for packed dims (na, nb, nc), or 0
 int bi_tile3_shape(int na, int nb, int nc);

@@ -83,6 +83,15 @@ __device__ __forceinline__ void ldg_vec(const double *p, double (&x)[2]) {
   x[0] = v.x; x[1] = v.y;
 }
 
+__device__ __forceinline__ void lds_vec(const float *p, float (&x)[4]) {
+  float4 v = *reinterpret_cast<const float4 *>(p);
+  x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+}
+__device__ __forceinline__ void lds_vec(const double *p, double (&x)[2]) {
+  double2 v = *reinterpret_cast<const double2 *>(p);
+  x[0] = v.x; x[1] = v.y;
+}
+
 // pairwise sum of a register array (short dependency chain)
 template <typename R, int N>
 __device__ __forceinline__ R tree_sum(const R (&v)[N]) {
@@ -198,6 +207,33 @@ struct Tile3 {
     for (int bl = 0; bl < NBL; ++bl)
 #pragma unroll
       for (int c = 0; c < NCP; ++c) W[c] = fma(eb[bl], L[bl][c], W[c]);
+    finish(V, W, xa, xb, xc);
+  }
+
+  // the same with the slice read from shared memory (lane-interleaved layout)
+  // instead of registers: for kernels that keep many steps' slices on chip
+  __device__ __forceinline__ void messages_smem(const R *__restrict__ Ls, R &xa, R &xb, R &xc) {
+    R V[NBL], W[NCP];
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl) V[bl] = (R)0;
+#pragma unroll
+    for (int c = 0; c < NCP; ++c) W[c] = (R)0;
+    const R *p = Ls + u * VE;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      R x[VE];
+      lds_vec(p + v * LPU * VE, x);
+#pragma unroll
+      for (int i = 0; i < VE; ++i) {
+        const int bl = (v * VE + i) / NCP, c = (v * VE + i) % NCP;
+        V[bl] = fma(x[i], ec[c], V[bl]);
+        W[c] = fma(eb[bl], x[i], W[c]);
+      }
+    }
+    finish(V, W, xa, xb, xc);
+  }
+
+  __device__ __forceinline__ void finish(R (&V)[NBL], R (&W)[NCP], R &xa, R &xb, R &xc) {
     R lav[NBL];
 #pragma unroll
     for (int bl = 0; bl < NBL; ++bl) lav[bl] = V[bl] * eb[bl];

@@ -1,0 +1,318 @@
+// Register-tile window kernels (VMP and MMP) for single-group rank-3 models.
+//
+// One thread-block cluster per agent.  Each CTA of the cluster owns a run of
+// consecutive time steps; a group of LPU lanes owns one step.  The summed
+// slices of all the CTA's steps are gathered from HBM once and stay in shared
+// memory for every iteration (re-reading them would multiply the dominant HBM
+// traffic by the iteration count).  Beliefs of neighbouring steps are exchanged
+// through shared memory, across CTAs of the cluster through distributed shared
+// memory (Appendix A-2 runs the window's steps in parallel; Section IV's
+// transition messages need the neighbours' beliefs of the previous iterate).
+#include <cooperative_groups.h>
+
+#include "bi_internal.h"
+#include "tile3.cuh"
+#include "tile3_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace {
+
+struct WindowGeom {
+  int32_t CS;       // CTAs per cluster (= per agent)
+  int32_t Tc;       // time steps per CTA
+  int32_t units;    // step slots per CTA (>= Tc; whole warps)
+  int32_t off_q, off_se;  // element offsets of the belief buffers and the gather area
+};
+
+template <typename R, int NA, int NB, int NC, int SB, int ALGO, bool STALE, bool CLUSTER>
+__global__ void __launch_bounds__(512)
+bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
+  using TT = Tile3<R, NA, NB, NC, SB>;
+  constexpr int LPU = TT::LPU, NBL = TT::NBL, NCP = TT::NCP, NAP = TT::NAP, VE = TT::VE, NV = TT::NV;
+  constexpr int PT = TT::P_TILE;
+  constexpr int SQ = (NA + NB + NC + 1) & ~1;  // beliefs of one step, padded to 16 bytes
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  R *Ls = reinterpret_cast<R *>(smem_raw);           // [units][PT] summed slices
+  R *qb = Ls + geo.off_q;                            // [2][units][SQ] normalised beliefs
+  R *seb = Ls + geo.off_se;                          // [units][NB + NCP] gathered e_b, e_c
+
+  int rank = 0;
+  if (CLUSTER) rank = (int)cg::this_cluster().block_rank();
+  const int agent = blockIdx.x / geo.CS;
+  const int g = p.G == 1 ? 0 : agent;
+  const int lane = threadIdx.x & 31;
+  const int tl = threadIdx.x / LPU;        // step slot of this lane group
+  const int t_raw = rank * geo.Tc + tl;
+  const bool live = tl < geo.Tc && t_raw < p.T;
+  const int t = live ? t_raw : p.T - 1;    // idle groups shadow the last step; their stores are suppressed
+  const int T = p.T;
+
+  TT t3;
+  t3.init_lane(lane);
+  const int a = t3.a, bi = t3.bi, ci = t3.ci;
+  const bool a_ok = t3.a_ok, b_ok = (a >> TT::SHB) < NBL, c_ok = ci < NC;
+  const int bsafe = b_ok ? bi : 0, csafe = c_ok ? ci : 0, asafe = a_ok ? a : 0;
+  R *se = seb + tl * (NB + NCP);
+  R *Lt = Ls + (size_t)tl * PT;
+  for (int i = t3.u; i < NB + NCP; i += LPU) se[i] = (R)0;
+
+  // ---- gather the step's summed slice into shared memory (one HBM read per slice)
+  {
+    const size_t ob = ((size_t)agent * T + t) * p.M;
+    R acc[NV][VE];
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+#pragma unroll
+      for (int i = 0; i < VE; ++i) acc[v][i] = (R)0;
+    for (int mi = 0; mi < p.nmem; ++mi) {
+      int o = clamp_flag(__ldg(p.obs + ob + p.modality[mi]), p.mcount[mi], p.status, BI_FLAG_OBS_RANGE);
+      const R *sl = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile + t3.u * VE;
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        R x[VE];
+        ldg_vec(sl + v * LPU * VE, x);
+#pragma unroll
+        for (int i = 0; i < VE; ++i) acc[v][i] += x[i];
+      }
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+#pragma unroll
+      for (int i = 0; i < VE; ++i) Lt[(v * LPU + t3.u) * VE + i] = acc[v][i];
+  }
+
+  // ---- transition matrices of this step's two edges, as columns for the owned states
+  // (transposed layouts: the lanes of a group read consecutive addresses)
+  const R *pa[3] = {nullptr, nullptr, nullptr}, *fu[3] = {nullptr, nullptr, nullptr};
+  R dprior[3] = {0, 0, 0};
+  {
+    const int own[3] = {asafe, bsafe, csafe};
+    const int nn[3] = {NA, NB, NC};
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      if (t == 0) {
+        dprior[j] = __ldg((const R *)p.logD[j] + (size_t)g * p.Dstride[j] + own[j]);
+      } else {
+        int u = clamp_flag(__ldg(p.act + ((size_t)agent * (T - 1) + (t - 1)) * 3 + p.fac[j]), p.U[j], p.status,
+                           BI_FLAG_ACT_RANGE);
+        const void *M = ALGO == BI_ALGO_VMP ? p.logBt[j] : p.BfT[j];  // [previous][next]
+        pa[j] = (const R *)M + (size_t)g * p.Bstride[j] + (size_t)u * nn[j] * p.np[j] + own[j];
+      }
+      if (t + 1 < T) {
+        int u = clamp_flag(__ldg(p.act + ((size_t)agent * (T - 1) + t) * 3 + p.fac[j]), p.U[j], p.status,
+                           BI_FLAG_ACT_RANGE);
+        const void *M = ALGO == BI_ALGO_VMP ? p.logB[j] : p.BdagT[j];  // [next][previous]
+        fu[j] = (const R *)M + (size_t)g * p.Bstride[j] + (size_t)u * nn[j] * p.np[j] + own[j];
+      }
+    }
+  }
+
+  // ---- belief buffers: own slots plus the neighbours' (possibly in another CTA)
+  R *q_own[2] = {qb + (size_t)tl * SQ, qb + (size_t)(geo.units + tl) * SQ};
+  const R *q_prev[2], *q_next[2];
+  {
+    const R *base_prev = qb, *base_next = qb;
+    int sl_prev = tl - 1, sl_next = tl + 1;
+    if (CLUSTER) {
+      cg::cluster_group cl = cg::this_cluster();
+      if (tl == 0 && rank > 0) { base_prev = cl.map_shared_rank(qb, rank - 1); sl_prev = geo.Tc - 1; }
+      if (tl == geo.Tc - 1 && rank + 1 < geo.CS) { base_next = cl.map_shared_rank(qb, rank + 1); sl_next = 0; }
+    }
+    if (sl_prev < 0) sl_prev = 0;                  // t == 0: never read
+    if (sl_next >= geo.units) sl_next = geo.units - 1;  // t == T - 1: never read
+    for (int b = 0; b < 2; ++b) {
+      q_prev[b] = base_prev + (size_t)(b * geo.units + sl_prev) * SQ;
+      q_next[b] = base_next + (size_t)(b * geo.units + sl_next) * SQ;
+    }
+  }
+  // uniform start
+  if (t3.own_a) q_own[0][a] = (R)1 / (R)NA;
+  if (t3.own_b) q_own[0][NA + bi] = (R)1 / (R)NB;
+  if (t3.own_c) q_own[0][NA + NB + ci] = (R)1 / (R)NC;
+  t3.set_uniform();
+  if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
+
+  R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
+  float ma = 0.f, mb = 0.f, mc = 0.f, pma = 0.f, pmb = 0.f, pmc = 0.f;
+  for (int k = 0; k < p.K; ++k) {
+    const int cur = k & 1, nxt = cur ^ 1;
+    // transition messages from the previous iterate of the neighbouring steps
+    R ta = dprior[0], tb = dprior[1], tc = dprior[2];
+    if (t > 0) {
+      R va = col_dot<R, NA>(pa[0], p.np[0], q_prev[cur]);
+      R vb = col_dot<R, NB>(pa[1], p.np[1], q_prev[cur] + NA);
+      R vc = col_dot<R, NC>(pa[2], p.np[2], q_prev[cur] + NA + NB);
+      if (ALGO == BI_ALGO_MMP) {
+        va = (R)0.5 * bi_log(bi_max(va, (R)BI_EPS));
+        vb = (R)0.5 * bi_log(bi_max(vb, (R)BI_EPS));
+        vc = (R)0.5 * bi_log(bi_max(vc, (R)BI_EPS));
+      }
+      ta = va; tb = vb; tc = vc;
+    }
+    if (t + 1 < T) {
+      R va = col_dot<R, NA>(fu[0], p.np[0], q_next[cur]);
+      R vb = col_dot<R, NB>(fu[1], p.np[1], q_next[cur] + NA);
+      R vc = col_dot<R, NC>(fu[2], p.np[2], q_next[cur] + NA + NB);
+      if (ALGO == BI_ALGO_MMP) {
+        va = (R)0.5 * bi_log(bi_max(va, (R)BI_EPS));
+        vb = (R)0.5 * bi_log(bi_max(vb, (R)BI_EPS));
+        vc = (R)0.5 * bi_log(bi_max(vc, (R)BI_EPS));
+      }
+      ta += va; tb += vb; tc += vc;
+    }
+    t3.messages_smem(Lt, xa, xb, xc);
+    xa = a_ok ? xa + ta : -bi_inf<R>();
+    xb = b_ok ? xb + tb : -bi_inf<R>();
+    xc = c_ok ? xc + tc : -bi_inf<R>();
+    const float cma = group_max_f<NAP, SB>((float)xa);
+    const float cmb = group_max_f<LPU, 1>((float)xb);
+    const float cmc = group_max_f<LPU, 1>((float)xc);
+    if (!STALE || k == 0) { ma = cma; mb = cmb; mc = cmc; }
+    else { ma = pma; mb = pmb; mc = pmc; }
+    pma = cma; pmb = cmb; pmc = cmc;
+    const R ean = a_ok ? bi_exp(xa - (R)ma) : (R)0;
+    const R ebn = b_ok ? bi_exp(xb - (R)mb) : (R)0;
+    const R ecn = c_ok ? bi_exp(xc - (R)mc) : (R)0;
+    __syncwarp();
+    if (t3.own_b) se[bi] = ebn;
+    if (t3.own_c) se[NB + ci] = ecn;
+    za = group_sum<R, NAP, SB>(ean);
+    __syncwarp();
+    t3.ea = ean;
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl) t3.eb[bl] = se[t3.bh * NBL + bl];
+#pragma unroll
+    for (int c = 0; c < NCP; ++c) t3.ec[c] = se[NB + c];
+    zb = group_sum<R, SB, 1>(tree_sum<R, NBL>(t3.eb));
+    zc = tree_sum<R, NCP>(t3.ec);
+    rinv = bi_rcp(za * zb * zc);
+    t3.sa = rinv * za;
+    t3.sb = rinv * zb;
+    t3.sc = rinv * zc;
+    // normalised beliefs for the neighbours' next iteration
+    const R qa = ean * (rinv * zb * zc), qbv = ebn * (rinv * za * zc), qc = ecn * (rinv * za * zb);
+    if (t3.own_a) q_own[nxt][a] = qa;
+    if (t3.own_b) q_own[nxt][NA + bi] = qbv;
+    if (t3.own_c) q_own[nxt][NA + NB + ci] = qc;
+    if (k == p.K - 1) {
+      const size_t ob = (size_t)agent * T + t;
+      if (live) {
+        float *qo = p.q_out + ob * p.S;
+        if (t3.own_a) qo[p.off[0] + a] = (float)qa;
+        if (t3.own_b) qo[p.off[1] + bi] = (float)qbv;
+        if (t3.own_c) qo[p.off[2] + ci] = (float)qc;
+        if (p.logq_out) {
+          float *lo = p.logq_out + ob * p.S;
+          if (t3.own_a) lo[p.off[0] + a] = (float)(xa - (R)ma - bi_log(za));
+          if (t3.own_b) lo[p.off[1] + bi] = (float)(xb - (R)mb - bi_log(zb));
+          if (t3.own_c) lo[p.off[2] + ci] = (float)(xc - (R)mc - bi_log(zc));
+        }
+      }
+      if (p.argmax_out) {
+        const int ia = group_argmax<R, NAP, SB>(xa, a_ok ? a : 1 << 20);
+        const int ib = group_argmax<R, LPU, 1>(xb, b_ok ? bi : 1 << 20);
+        const int ic = group_argmax<R, LPU, 1>(xc, c_ok ? ci : 1 << 20);
+        if (live && t3.u == 0) {
+          int32_t *ao = p.argmax_out + ob * 3;
+          ao[p.fac[0]] = ia;
+          ao[p.fac[1]] = ib;
+          ao[p.fac[2]] = ic;
+        }
+      }
+    }
+    if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
+  }
+}
+
+template <typename R, int NA, int NB, int NC, int SB, int ALGO>
+int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
+  using TT = Tile3<R, NA, NB, NC, SB>;
+  constexpr int SQ = (NA + NB + NC + 1) & ~1;
+  constexpr int UPW = TT::UPW;
+  WindowGeom geo;
+  size_t bytes = 0;
+  int threads = 0;
+  bool found = false;
+  for (int cs = 1; cs <= 8; cs *= 2) {
+    const int Tc = (p.T + cs - 1) / cs;
+    const int warps = (Tc + UPW - 1) / UPW;
+    const int units = warps * UPW;
+    size_t elems = (size_t)units * TT::P_TILE + 2 * (size_t)units * SQ + (size_t)units * (NB + TT::NCP);
+    if (warps * 32 <= 512 && elems * sizeof(R) <= (size_t)smem_budget) {
+      geo.CS = cs; geo.Tc = Tc; geo.units = units;
+      geo.off_q = units * TT::P_TILE;
+      geo.off_se = geo.off_q + 2 * units * SQ;
+      bytes = elems * sizeof(R);
+      threads = warps * 32;
+      found = true;
+      break;
+    }
+  }
+  if (!found) return BI_ERR_UNSUPPORTED;
+  const bool stale = sizeof(R) == 8 && p.nmem <= 12;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(p.N * geo.CS));
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)geo.CS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = geo.CS > 1 ? 1 : 0;
+  cudaError_t e;
+#define BI_WIN_LAUNCH(ST, CL)                                                                         \
+  do {                                                                                                \
+    auto kern = bi_tile3_window_kernel<R, NA, NB, NC, SB, ALGO, ST, CL>;                             \
+    e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, kern, p, geo);                                 \
+  } while (0)
+  if (geo.CS > 1) {
+    if (stale) BI_WIN_LAUNCH(true, true); else BI_WIN_LAUNCH(false, true);
+  } else {
+    if (stale) BI_WIN_LAUNCH(true, false); else BI_WIN_LAUNCH(false, false);
+  }
+#undef BI_WIN_LAUNCH
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return BI_ERR_CUDA;
+  }
+  return BI_OK;
+}
+
+template <typename R, int ALGO>
+int dispatch_window(const Tile3Params &p, int na, int nb, int nc, int budget, cudaStream_t stream) {
+#define X(A, B, C, S) \
+  if (na == A && nb == B && nc == C) return launch_window<R, A, B, C, S, ALGO>(p, budget, stream);
+  BI_TILE3_SHAPES(X)
+#undef X
+  return BI_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+int bi_launch_tile3_window(const BiCall &c, bi_model *mut) {
+  const bi_model *md = c.model;
+  if (c.algo == BI_ALGO_FILTER || md->tile_sb <= 0) return BI_ERR_UNSUPPORTED;
+  const BiGroup &g = md->h.grp[0];
+  Tile3Params p;
+  bi_tile3_fill_params(c, p);
+  const int budget = md->max_smem_optin - 1024;
+  int rc;
+  const bool f64 = md->arith == BI_ARITH_F64;
+  if (c.algo == BI_ALGO_VMP)
+    rc = f64 ? dispatch_window<double, BI_ALGO_VMP>(p, g.dim[0], g.dim[1], g.dim[2], budget, c.stream)
+             : dispatch_window<float, BI_ALGO_VMP>(p, g.dim[0], g.dim[1], g.dim[2], budget, c.stream);
+  else
+    rc = f64 ? dispatch_window<double, BI_ALGO_MMP>(p, g.dim[0], g.dim[1], g.dim[2], budget, c.stream)
+             : dispatch_window<float, BI_ALGO_MMP>(p, g.dim[0], g.dim[1], g.dim[2], budget, c.stream);
+  if (rc == BI_OK) {
+    mut->launches += 1;
+    mut->last_kernel = c.algo == BI_ALGO_VMP ? (f64 ? "tile3_vmp_f64" : "tile3_vmp_f32")
+                                             : (f64 ? "tile3_mmp_f64" : "tile3_mmp_f32");
+  }
+  return rc;
+}

@@ -163,3 +163,29 @@ def test_tile_filter_shapes_and_ragged_batches(arith):
     assert res["kernel"] == f"tile3_filter_{arith}", res
     if not strict:
         assert res["q_max_err"] < 1e-3
+
+
+# ---- the register-tile window kernels (VMP / MMP), incl. multi-CTA clusters
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_tile_window_kernels(algo):
+    # 8 lanes per step, 4 steps per warp; T not a multiple of 4
+    res = check_workload(make_config(2, N=9, T=11, K=7), algo)
+    assert res["kernel"] == f"tile3_{algo}_f64", res
+    # 32 lanes per step; float64 slices of 20 steps exceed one SM: two-CTA cluster
+    res = check_workload(make_config(4, N=6, T=20, K=8), algo)
+    assert res["kernel"] == f"tile3_{algo}_f64", res
+    # odd split over the cluster (T = 19 -> 10 + 9), and a window of a single step
+    res = check_workload(make_config(4, N=3, T=19, K=5), algo)
+    assert res["kernel"] == f"tile3_{algo}_f64", res
+    res = check_workload(make_config(4, N=3, T=1, K=5), algo)
+    # the longest window: four-CTA cluster
+    res = check_workload(make_config(4, N=2, T=64, K=3), algo)
+    assert res["kernel"] == f"tile3_{algo}_f64", res
+    # padded lanes
+    w = _custom(33, [4, 3, 2], [3, 5], [[0, 1, 2], [2, 0, 1]], [2, 3, 1], N=7, T=6, K=9, sparsity=0.5)
+    res = check_workload(w, algo)
+    assert res["kernel"] == f"tile3_{algo}_f64", res
+    # float32 arithmetic: single CTA holds the window
+    res = check_workload(make_config(4, N=4, T=20, K=8), algo, arith="f32", strict=False)
+    assert res["kernel"] == f"tile3_{algo}_f32", res
