@@ -9,12 +9,13 @@
 
 namespace {
 
-template <typename R, int NA, int NB, int NC, int SB, bool STALE>
+template <typename R, int NA, int NB, int NC, int SB, bool LSMEM, bool STALE>
 __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p) {
   using TT = Tile3<R, NA, NB, NC, SB>;
   constexpr int LPU = TT::LPU, UPW = TT::UPW, NBL = TT::NBL, NCP = TT::NCP, NAP = TT::NAP;
   __shared__ __align__(16) R sm_e[UPW][NB + NCP];      // gathered e_b, e_c of the current iterate
   __shared__ __align__(16) R sm_q[UPW][NA + NB + NC];  // final beliefs of the previous step
+  __shared__ __align__(16) R sm_L[LSMEM ? UPW : 1][LSMEM ? TT::P_TILE : 2];  // large tiles: the step's slice
 
   const int lane = threadIdx.x;
   const int unit = lane / LPU;
@@ -41,7 +42,8 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
                          BI_FLAG_OBS_RANGE);
       slice[mi] = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile;
     }
-    t3.load_slices(slice, p.nmem);
+    if (LSMEM) t3.load_slices_smem(slice, p.nmem, sm_L[LSMEM ? unit : 0]);
+    else t3.load_slices(slice, p.nmem);
 
     // ---- ln prior of the logits this lane owns: D, or B_u times the previous step's belief
     R lpa, lpb, lpc;
@@ -69,7 +71,8 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
     float ma = 0.f, mb = 0.f, mc = 0.f;     // softmax shifts in use
     float pma = 0.f, pmb = 0.f, pmc = 0.f;  // exact maxima of the previous iterate
     for (int k = 0; k < p.K; ++k) {
-      t3.messages(xa, xb, xc);
+      if (LSMEM) t3.messages_smem(sm_L[LSMEM ? unit : 0], xa, xb, xc);
+      else t3.messages(xa, xb, xc);
       xa = a_ok ? xa + lpa : -bi_inf<R>();
       xb = b_ok ? xb + lpb : -bi_inf<R>();
       xc = c_ok ? xc + lpc : -bi_inf<R>();
@@ -138,23 +141,23 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
   }
 }
 
-template <typename R, int NA, int NB, int NC, int SB>
+template <typename R, int NA, int NB, int NC, int SB, bool LSMEM>
 int launch_filter(const Tile3Params &p, cudaStream_t stream) {
   using TT = Tile3<R, NA, NB, NC, SB>;
   const int grid = (p.N + TT::UPW - 1) / TT::UPW;
   // shifts may lag one iterate only where the exponent range has room for the
   // largest possible move of a logit: float64 and at most 12 modalities
   if (sizeof(R) == 8 && p.nmem <= 12)
-    bi_tile3_filter_kernel<R, NA, NB, NC, SB, true><<<grid, 32, 0, stream>>>(p);
+    bi_tile3_filter_kernel<R, NA, NB, NC, SB, LSMEM, true><<<grid, 32, 0, stream>>>(p);
   else
-    bi_tile3_filter_kernel<R, NA, NB, NC, SB, false><<<grid, 32, 0, stream>>>(p);
+    bi_tile3_filter_kernel<R, NA, NB, NC, SB, LSMEM, false><<<grid, 32, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? BI_OK : BI_ERR_CUDA;
 }
 
 template <typename R>
 int dispatch_filter(const Tile3Params &p, int na, int nb, int nc, cudaStream_t stream) {
-#define X(A, B, C, S) \
-  if (na == A && nb == B && nc == C) return launch_filter<R, A, B, C, S>(p, stream);
+#define X(A, B, C, S, LS) \
+  if (na == A && nb == B && nc == C) return launch_filter<R, A, B, C, S, LS>(p, stream);
   BI_TILE3_SHAPES(X)
 #undef X
   return BI_ERR_UNSUPPORTED;
@@ -163,7 +166,7 @@ int dispatch_filter(const Tile3Params &p, int na, int nb, int nc, cudaStream_t s
 }  // namespace
 
 int bi_tile3_shape(int na, int nb, int nc) {
-#define X(A, B, C, S) \
+#define X(A, B, C, S, LS) \
   if (na == A && nb == B && nc == C) return S;
   BI_TILE3_SHAPES(X)
 #undef X

@@ -179,6 +179,31 @@ struct Tile3 {
     }
   }
 
+  // the same gather, summed into shared memory (same lane-interleaved layout)
+  __device__ __forceinline__ void load_slices_smem(const R *const *slice, int nmem, R *Lt) {
+    R acc[NV][VE];
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+#pragma unroll
+      for (int i = 0; i < VE; ++i) acc[v][i] = (R)0;
+    for (int mi = 0; mi < nmem; ++mi) {
+      const R *p = slice[mi] + u * VE;
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        R x[VE];
+        ldg_vec(p + v * LPU * VE, x);
+#pragma unroll
+        for (int i = 0; i < VE; ++i) acc[v][i] += x[i];
+      }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+#pragma unroll
+      for (int i = 0; i < VE; ++i) Lt[(v * LPU + u) * VE + i] = acc[v][i];
+    __syncwarp();
+  }
+
   __device__ __forceinline__ void set_uniform() {
     ea = a_ok ? (R)1 : (R)0;
 #pragma unroll

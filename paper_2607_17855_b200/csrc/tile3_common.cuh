@@ -4,8 +4,9 @@
 #include "bi_internal.h"
 #include "tile3.cuh"
 
-// compiled tile shapes: packed dims (a, b, c) and the lanes along b
-#define BI_TILE3_SHAPES(X) X(8, 6, 8, 1) X(16, 12, 8, 2) X(3, 2, 4, 1)
+// compiled tile shapes: packed dims (a, b, c), the lanes along b, and whether the
+// filtering kernel keeps the step's slice in shared memory (large tiles) or registers
+#define BI_TILE3_SHAPES(X) X(8, 6, 8, 1, false) X(16, 12, 8, 1, true) X(3, 2, 4, 1, false)
 
 
 struct Tile3Params {
@@ -35,6 +36,15 @@ __device__ __forceinline__ R col_dot(const R *__restrict__ col, int stride, cons
   return tree_sum<R, N>(x);
 }
 
+
+// the same for a matrix that may live in shared or global memory
+template <typename R, int N>
+__device__ __forceinline__ R col_dot_any(const R *col, int stride, const R *q) {
+  R x[N];
+#pragma unroll
+  for (int r = 0; r < N; ++r) x[r] = col[r * stride] * q[r];
+  return tree_sum<R, N>(x);
+}
 
 static inline void bi_tile3_fill_params(const BiCall &c, Tile3Params &p) {
   const bi_model *md = c.model;

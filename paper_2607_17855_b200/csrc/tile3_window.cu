@@ -5,10 +5,15 @@
 // slices of all the CTA's steps are gathered from HBM once and stay in shared
 // memory for every iteration (re-reading them would multiply the dominant HBM
 // traffic by the iteration count).  Beliefs of neighbouring steps are exchanged
-// through shared memory, across CTAs of the cluster through distributed shared
-// memory (Appendix A-2 runs the window's steps in parallel; Section IV's
-// transition messages need the neighbours' beliefs of the previous iterate).
+// through shared memory; at a CTA boundary the owning lanes also store their
+// beliefs into the neighbouring CTA's halo slot through distributed shared
+// memory, so every read in the iteration loop is a local shared-memory load
+// (Appendix A-2 runs the window's steps in parallel; Section IV's transition
+// messages need the neighbours' beliefs of the previous iterate).
 #include <cooperative_groups.h>
+
+#include <algorithm>
+#include <cstdlib>
 
 #include "bi_internal.h"
 #include "tile3.cuh"
@@ -22,8 +27,21 @@ struct WindowGeom {
   int32_t CS;       // CTAs per cluster (= per agent)
   int32_t Tc;       // time steps per CTA
   int32_t units;    // step slots per CTA (>= Tc; whole warps)
-  int32_t off_q, off_se;  // element offsets of the belief buffers and the gather area
+  int32_t off_q, off_se, off_B;  // element offsets: belief buffers, gather area, transition matrices
 };
+
+// sum_r M[r][s] q[r] with two interleaved accumulators; M and q in shared memory
+template <typename R, int N>
+__device__ __forceinline__ R col_dot_smem(const R *col, int stride, const R *q) {
+  R s0 = (R)0, s1 = (R)0;
+#pragma unroll
+  for (int r = 0; r + 1 < N; r += 2) {
+    s0 = fma(col[r * stride], q[r], s0);
+    s1 = fma(col[(r + 1) * stride], q[r + 1], s1);
+  }
+  if (N & 1) s0 = fma(col[(N - 1) * stride], q[N - 1], s0);
+  return s0 + s1;
+}
 
 template <typename R, int NA, int NB, int NC, int SB, int ALGO, bool STALE, bool CLUSTER>
 __global__ void __launch_bounds__(512)
@@ -33,9 +51,12 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   constexpr int PT = TT::P_TILE;
   constexpr int SQ = (NA + NB + NC + 1) & ~1;  // beliefs of one step, padded to 16 bytes
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  R *Ls = reinterpret_cast<R *>(smem_raw);           // [units][PT] summed slices
-  R *qb = Ls + geo.off_q;                            // [2][units][SQ] normalised beliefs
-  R *seb = Ls + geo.off_se;                          // [units][NB + NCP] gathered e_b, e_c
+  R *Ls = reinterpret_cast<R *>(smem_raw);   // [units][PT] summed slices
+  // beliefs: two buffers of (units + 2) slots; slot 0 and slot units + 1 are the
+  // halos holding the neighbouring CTAs' boundary steps
+  R *qb = Ls + geo.off_q;
+  R *seb = Ls + geo.off_se;                  // [units][NB + NCP] gathered e_b, e_c
+  R *Bs = Ls + geo.off_B;                    // this agent's transition matrices, every action
 
   int rank = 0;
   if (CLUSTER) rank = (int)cg::this_cluster().block_rank();
@@ -60,89 +81,104 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   // ---- gather the step's summed slice into shared memory (one HBM read per slice)
   {
     const size_t ob = ((size_t)agent * T + t) * p.M;
-    R acc[NV][VE];
+    constexpr int CH = NV % 12 == 0 ? 12 : (NV % 8 == 0 ? 8 : (NV % 6 == 0 ? 6 : NV));  // vectors in flight per pass
+    for (int v0 = 0; v0 < NV; v0 += CH) {
+      R acc[CH][VE];
 #pragma unroll
-    for (int v = 0; v < NV; ++v)
+      for (int v = 0; v < CH; ++v)
 #pragma unroll
-      for (int i = 0; i < VE; ++i) acc[v][i] = (R)0;
-    for (int mi = 0; mi < p.nmem; ++mi) {
-      int o = clamp_flag(__ldg(p.obs + ob + p.modality[mi]), p.mcount[mi], p.status, BI_FLAG_OBS_RANGE);
-      const R *sl = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile + t3.u * VE;
+        for (int i = 0; i < VE; ++i) acc[v][i] = (R)0;
+      for (int mi = 0; mi < p.nmem; ++mi) {
+        int o = clamp_flag(__ldg(p.obs + ob + p.modality[mi]), p.mcount[mi], p.status, BI_FLAG_OBS_RANGE);
+        const R *sl = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile +
+                      ((size_t)v0 * LPU + t3.u) * VE;
 #pragma unroll
-      for (int v = 0; v < NV; ++v) {
-        R x[VE];
-        ldg_vec(sl + v * LPU * VE, x);
+        for (int v = 0; v < CH; ++v) {
+          R x[VE];
+          ldg_vec(sl + v * LPU * VE, x);
 #pragma unroll
-        for (int i = 0; i < VE; ++i) acc[v][i] += x[i];
+          for (int i = 0; i < VE; ++i) acc[v][i] += x[i];
+        }
       }
+#pragma unroll
+      for (int v = 0; v < CH; ++v)
+#pragma unroll
+        for (int i = 0; i < VE; ++i) Lt[((v0 + v) * LPU + t3.u) * VE + i] = acc[v][i];
     }
-#pragma unroll
-    for (int v = 0; v < NV; ++v)
-#pragma unroll
-      for (int i = 0; i < VE; ++i) Lt[(v * LPU + t3.u) * VE + i] = acc[v][i];
   }
 
-  // ---- transition matrices of this step's two edges, as columns for the owned states
-  // (transposed layouts: the lanes of a group read consecutive addresses)
-  const R *pa[3] = {nullptr, nullptr, nullptr}, *fu[3] = {nullptr, nullptr, nullptr};
+  // ---- this agent's transition matrices, staged once; then the columns this
+  // lane needs for its owned states on the step's two edges.  Transposed
+  // layouts ([previous][next] for the past edge, [next][previous] for the
+  // future edge): the lanes of a group read consecutive addresses.
+  const R *pa0, *pa1, *pa2, *fu0, *fu1, *fu2;
   R dprior[3] = {0, 0, 0};
   {
     const int own[3] = {asafe, bsafe, csafe};
     const int nn[3] = {NA, NB, NC};
+    const R *pa[3], *fu[3];
+    int boff = 0;
 #pragma unroll
     for (int j = 0; j < 3; ++j) {
-      if (t == 0) {
-        dprior[j] = __ldg((const R *)p.logD[j] + (size_t)g * p.Dstride[j] + own[j]);
-      } else {
-        int u = clamp_flag(__ldg(p.act + ((size_t)agent * (T - 1) + (t - 1)) * 3 + p.fac[j]), p.U[j], p.status,
-                           BI_FLAG_ACT_RANGE);
-        const void *M = ALGO == BI_ALGO_VMP ? p.logBt[j] : p.BfT[j];  // [previous][next]
-        pa[j] = (const R *)M + (size_t)g * p.Bstride[j] + (size_t)u * nn[j] * p.np[j] + own[j];
+      const int msz = p.U[j] * nn[j] * p.np[j];
+      const R *Mp = (const R *)(ALGO == BI_ALGO_VMP ? p.logBt[j] : p.BfT[j]) + (size_t)g * p.Bstride[j];
+      const R *Mf = (const R *)(ALGO == BI_ALGO_VMP ? p.logB[j] : p.BdagT[j]) + (size_t)g * p.Bstride[j];
+      for (int i = threadIdx.x; i < msz; i += blockDim.x) {
+        Bs[boff + i] = __ldg(Mp + i);
+        Bs[boff + msz + i] = __ldg(Mf + i);
       }
-      if (t + 1 < T) {
-        int u = clamp_flag(__ldg(p.act + ((size_t)agent * (T - 1) + t) * 3 + p.fac[j]), p.U[j], p.status,
+      int up = 0, uf = 0;
+      if (t == 0) dprior[j] = __ldg((const R *)p.logD[j] + (size_t)g * p.Dstride[j] + own[j]);
+      else up = clamp_flag(__ldg(p.act + ((size_t)agent * (T - 1) + (t - 1)) * 3 + p.fac[j]), p.U[j], p.status,
                            BI_FLAG_ACT_RANGE);
-        const void *M = ALGO == BI_ALGO_VMP ? p.logB[j] : p.BdagT[j];  // [next][previous]
-        fu[j] = (const R *)M + (size_t)g * p.Bstride[j] + (size_t)u * nn[j] * p.np[j] + own[j];
-      }
+      if (t + 1 < T)
+        uf = clamp_flag(__ldg(p.act + ((size_t)agent * (T - 1) + t) * 3 + p.fac[j]), p.U[j], p.status,
+                        BI_FLAG_ACT_RANGE);
+      pa[j] = Bs + boff + up * nn[j] * p.np[j] + own[j];
+      fu[j] = Bs + boff + msz + uf * nn[j] * p.np[j] + own[j];
+      boff += 2 * msz;
     }
+    pa0 = pa[0]; pa1 = pa[1]; pa2 = pa[2];
+    fu0 = fu[0]; fu1 = fu[1]; fu2 = fu[2];
   }
 
-  // ---- belief buffers: own slots plus the neighbours' (possibly in another CTA)
-  R *q_own[2] = {qb + (size_t)tl * SQ, qb + (size_t)(geo.units + tl) * SQ};
-  const R *q_prev[2], *q_next[2];
-  {
-    const R *base_prev = qb, *base_next = qb;
-    int sl_prev = tl - 1, sl_next = tl + 1;
-    if (CLUSTER) {
-      cg::cluster_group cl = cg::this_cluster();
-      if (tl == 0 && rank > 0) { base_prev = cl.map_shared_rank(qb, rank - 1); sl_prev = geo.Tc - 1; }
-      if (tl == geo.Tc - 1 && rank + 1 < geo.CS) { base_next = cl.map_shared_rank(qb, rank + 1); sl_next = 0; }
+  // ---- belief slots: own step at slot tl + 1; neighbours at tl and tl + 2
+  const int bufsz = (geo.units + 2) * SQ;
+  R *q_cur = qb + (size_t)(tl + 1) * SQ;   // this step, buffer 0
+  R *q_nxt = q_cur + bufsz;                // this step, buffer 1
+  // remote halo slots this group also feeds (same offsets in the neighbour CTA)
+  R *r_prev_cur = nullptr, *r_prev_nxt = nullptr, *r_next_cur = nullptr, *r_next_nxt = nullptr;
+  if (CLUSTER) {
+    cg::cluster_group cl = cg::this_cluster();
+    if (live && tl == 0 && rank > 0) {
+      R *rb = cl.map_shared_rank(qb, rank - 1);
+      r_prev_cur = rb + (size_t)(geo.Tc + 1) * SQ;  // the previous CTA's "next" halo
+      r_prev_nxt = r_prev_cur + bufsz;
     }
-    if (sl_prev < 0) sl_prev = 0;                  // t == 0: never read
-    if (sl_next >= geo.units) sl_next = geo.units - 1;  // t == T - 1: never read
-    for (int b = 0; b < 2; ++b) {
-      q_prev[b] = base_prev + (size_t)(b * geo.units + sl_prev) * SQ;
-      q_next[b] = base_next + (size_t)(b * geo.units + sl_next) * SQ;
+    if (live && tl == geo.Tc - 1 && rank + 1 < geo.CS) {
+      R *rb = cl.map_shared_rank(qb, rank + 1);
+      r_next_cur = rb;                              // the next CTA's "previous" halo
+      r_next_nxt = rb + bufsz;
     }
   }
-  // uniform start
-  if (t3.own_a) q_own[0][a] = (R)1 / (R)NA;
-  if (t3.own_b) q_own[0][NA + bi] = (R)1 / (R)NB;
-  if (t3.own_c) q_own[0][NA + NB + ci] = (R)1 / (R)NC;
+  // uniform start (every slot, halos included: neighbours start uniform too)
+  for (int i = threadIdx.x; i < (geo.units + 2) * SQ; i += blockDim.x) {
+    const int s = i % SQ;
+    qb[i] = s < NA ? (R)1 / (R)NA : s < NA + NB ? (R)1 / (R)NB : s < NA + NB + NC ? (R)1 / (R)NC : (R)0;
+  }
   t3.set_uniform();
   if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
 
   R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
   float ma = 0.f, mb = 0.f, mc = 0.f, pma = 0.f, pmb = 0.f, pmc = 0.f;
   for (int k = 0; k < p.K; ++k) {
-    const int cur = k & 1, nxt = cur ^ 1;
     // transition messages from the previous iterate of the neighbouring steps
     R ta = dprior[0], tb = dprior[1], tc = dprior[2];
     if (t > 0) {
-      R va = col_dot<R, NA>(pa[0], p.np[0], q_prev[cur]);
-      R vb = col_dot<R, NB>(pa[1], p.np[1], q_prev[cur] + NA);
-      R vc = col_dot<R, NC>(pa[2], p.np[2], q_prev[cur] + NA + NB);
+      const R *qp = q_cur - SQ;
+      R va = col_dot_smem<R, NA>(pa0, p.np[0], qp);
+      R vb = col_dot_smem<R, NB>(pa1, p.np[1], qp + NA);
+      R vc = col_dot_smem<R, NC>(pa2, p.np[2], qp + NA + NB);
       if (ALGO == BI_ALGO_MMP) {
         va = (R)0.5 * bi_log(bi_max(va, (R)BI_EPS));
         vb = (R)0.5 * bi_log(bi_max(vb, (R)BI_EPS));
@@ -151,9 +187,10 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       ta = va; tb = vb; tc = vc;
     }
     if (t + 1 < T) {
-      R va = col_dot<R, NA>(fu[0], p.np[0], q_next[cur]);
-      R vb = col_dot<R, NB>(fu[1], p.np[1], q_next[cur] + NA);
-      R vc = col_dot<R, NC>(fu[2], p.np[2], q_next[cur] + NA + NB);
+      const R *qn = q_cur + SQ;
+      R va = col_dot_smem<R, NA>(fu0, p.np[0], qn);
+      R vb = col_dot_smem<R, NB>(fu1, p.np[1], qn + NA);
+      R vc = col_dot_smem<R, NC>(fu2, p.np[2], qn + NA + NB);
       if (ALGO == BI_ALGO_MMP) {
         va = (R)0.5 * bi_log(bi_max(va, (R)BI_EPS));
         vb = (R)0.5 * bi_log(bi_max(vb, (R)BI_EPS));
@@ -192,9 +229,22 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     t3.sc = rinv * zc;
     // normalised beliefs for the neighbours' next iteration
     const R qa = ean * (rinv * zb * zc), qbv = ebn * (rinv * za * zc), qc = ecn * (rinv * za * zb);
-    if (t3.own_a) q_own[nxt][a] = qa;
-    if (t3.own_b) q_own[nxt][NA + bi] = qbv;
-    if (t3.own_c) q_own[nxt][NA + NB + ci] = qc;
+    // (idle groups do not publish: the slot after a CTA's last step is a halo)
+    if (live && t3.own_a) q_nxt[a] = qa;
+    if (live && t3.own_b) q_nxt[NA + bi] = qbv;
+    if (live && t3.own_c) q_nxt[NA + NB + ci] = qc;
+    if (CLUSTER) {
+      if (r_prev_nxt) {
+        if (t3.own_a) r_prev_nxt[a] = qa;
+        if (t3.own_b) r_prev_nxt[NA + bi] = qbv;
+        if (t3.own_c) r_prev_nxt[NA + NB + ci] = qc;
+      }
+      if (r_next_nxt) {
+        if (t3.own_a) r_next_nxt[a] = qa;
+        if (t3.own_b) r_next_nxt[NA + bi] = qbv;
+        if (t3.own_c) r_next_nxt[NA + NB + ci] = qc;
+      }
+    }
     if (k == p.K - 1) {
       const size_t ob = (size_t)agent * T + t;
       if (live) {
@@ -221,6 +271,10 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
         }
       }
     }
+    // swap the belief buffers (pointers stay in registers)
+    { R *tmp = q_cur; q_cur = q_nxt; q_nxt = tmp; }
+    { R *tmp = r_prev_cur; r_prev_cur = r_prev_nxt; r_prev_nxt = tmp; }
+    { R *tmp = r_next_cur; r_next_cur = r_next_nxt; r_next_nxt = tmp; }
     if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
   }
 }
@@ -234,20 +288,48 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   size_t bytes = 0;
   int threads = 0;
   bool found = false;
+  // transition matrices (both directions, every action) are staged in shared memory
+  size_t bsz = 0;
+  {
+    const int nn[3] = {NA, NB, NC};
+    for (int j = 0; j < 3; ++j) bsz += 2 * (size_t)p.U[j] * nn[j] * p.np[j];
+  }
+  if (bsz * sizeof(R) > 48 * 1024) return BI_ERR_UNSUPPORTED;
+  // Fewest CTAs per agent whose share of the window fits; a larger cluster is
+  // preferred when it lets several CTAs share an SM (more warps in flight to
+  // hide the per-iteration barrier).  BI_WINDOW_CS (testing aid) forces a size.
+  int cs_force = 0;
+  if (const char *e = getenv("BI_WINDOW_CS")) cs_force = atoi(e);
+  int best_cs = 0;
+  double best_score = -1.0;
   for (int cs = 1; cs <= 8; cs *= 2) {
+    if (cs_force > 0 && cs != cs_force) continue;
+    const int Tc = (p.T + cs - 1) / cs;
+    if (cs > 1 && Tc * (cs - 1) >= p.T) continue;  // an empty CTA: no gain over the smaller cluster
+    const int warps = (Tc + UPW - 1) / UPW;
+    const int units = warps * UPW;
+    const size_t elems = (size_t)units * TT::P_TILE + 2 * (size_t)(units + 2) * SQ +
+                         (size_t)units * (NB + TT::NCP) + bsz;
+    const size_t b = elems * sizeof(R);
+    if (warps * 32 > 512 || b > (size_t)smem_budget) continue;
+    const int per_sm = (int)std::min<size_t>(8, (size_t)(228 * 1024) / (b + 1024));
+    // useful warps resident per SM, discounted by idle step slots
+    const double score = (double)per_sm * warps * ((double)Tc / units) - 0.01 * cs;
+    if (score > best_score) { best_score = score; best_cs = cs; }
+  }
+  if (best_cs == 0) return BI_ERR_UNSUPPORTED;
+  {
+    const int cs = best_cs;
     const int Tc = (p.T + cs - 1) / cs;
     const int warps = (Tc + UPW - 1) / UPW;
     const int units = warps * UPW;
-    size_t elems = (size_t)units * TT::P_TILE + 2 * (size_t)units * SQ + (size_t)units * (NB + TT::NCP);
-    if (warps * 32 <= 512 && elems * sizeof(R) <= (size_t)smem_budget) {
-      geo.CS = cs; geo.Tc = Tc; geo.units = units;
-      geo.off_q = units * TT::P_TILE;
-      geo.off_se = geo.off_q + 2 * units * SQ;
-      bytes = elems * sizeof(R);
-      threads = warps * 32;
-      found = true;
-      break;
-    }
+    geo.CS = cs; geo.Tc = Tc; geo.units = units;
+    geo.off_q = units * TT::P_TILE;
+    geo.off_se = geo.off_q + 2 * (units + 2) * SQ;
+    geo.off_B = geo.off_se + units * (NB + TT::NCP);
+    bytes = ((size_t)geo.off_B + bsz) * sizeof(R);
+    threads = warps * 32;
+    found = true;
   }
   if (!found) return BI_ERR_UNSUPPORTED;
   const bool stale = sizeof(R) == 8 && p.nmem <= 12;
@@ -285,7 +367,7 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
 
 template <typename R, int ALGO>
 int dispatch_window(const Tile3Params &p, int na, int nb, int nc, int budget, cudaStream_t stream) {
-#define X(A, B, C, S) \
+#define X(A, B, C, S, LS) \
   if (na == A && nb == B && nc == C) return launch_window<R, A, B, C, S, ALGO>(p, budget, stream);
   BI_TILE3_SHAPES(X)
 #undef X
