@@ -305,6 +305,8 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
       lv.last_npad4 = bi_pad4(g.dim[last]) / 4;
       lv.last_qoff = h.offp[g.axis[last]];
       lv.out_npad = bi_pad4(g.dim[last - 1]);
+      lv.last_pv = 4;
+      while (lv.last_pv < lv.last_n) lv.last_pv <<= 1;
       int out_floats = (lv.nrows / g.dim[last - 1]) * lv.out_npad;
       if (l % 2 == 0) V0 = std::max(V0, out_floats); else V1 = std::max(V1, out_floats);
       if (l == 0) rows_max = std::max(rows_max, lv.nrows);
@@ -466,6 +468,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   bi_model *mut = const_cast<bi_model *>(model);
   int rc = bi_launch_tile3(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_warp(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;
 }

@@ -28,6 +28,7 @@ struct BiLevel {
   int32_t last_npad4; // its padded size / 4
   int32_t last_qoff;  // padded belief offset of its factor
   int32_t out_npad;   // padded size of the output tensor's last axis
+  int32_t last_pv;    // last_n rounded up to a power of two, at least 4
 };
 
 // Modalities with the same dependency *set* form one group: their slices add
@@ -50,7 +51,9 @@ struct BiMember {
   int32_t m, modality, P_pad, pad_;
 };
 
-struct BiDev {
+// (16-byte aligned so that its size is a whole number of 16-byte vectors: kernels
+// copy it into shared memory with vector loads)
+struct alignas(16) BiDev {
   int32_t F, M, S, Sp, G, ngroups, nmem, Ltot;
   int32_t n[BI_MAX_F], npad[BI_MAX_F], off[BI_MAX_F], offp[BI_MAX_F], U[BI_MAX_F];
   int32_t m[BI_MAX_M];
@@ -100,6 +103,7 @@ struct BiCall {
 // kernel families; each returns BI_OK, BI_ERR_UNSUPPORTED (not applicable to
 // this model / call: the dispatcher tries the next one) or an error.
 int bi_launch_generic(const BiCall &c, bi_model *mut);
+int bi_launch_warp(const BiCall &c, bi_model *mut);
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
 int bi_launch_tile3_window(const BiCall &c, bi_model *mut);
 // SB of the compiled register-tile shape for packed dims (na, nb, nc), or 0
