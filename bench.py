@@ -73,6 +73,27 @@ def algorithmic_bytes(w, elem_bytes: int) -> float:
     return float(w.N * w.T * slices * elem_bytes + io)
 
 
+def rank_seed(rank: int) -> int:
+    """Seed of the batch a rank draws: agents are independent, so ranks shard by
+    drawing disjoint batches of the same workload (weak scaling)."""
+    return 1000 + HEADLINE + 7919 * rank
+
+
+def max_over_ranks(dist, seconds: float, device) -> float:
+    """Slowest rank's device time (the job finishes when the last rank does)."""
+    if dist is None:
+        return seconds
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(updates_per_rank: int, world: int, seconds: float) -> float:
+    """Whole-job belief updates per second over all ranks."""
+    return updates_per_rank * world / seconds
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while timing runs."""
 
@@ -214,7 +235,7 @@ def main():
 
     # agents are independent: each rank runs its own full-size batch (weak scaling),
     # drawn from its own seed; there is no collective on the data path
-    w = make_config(HEADLINE, seed=1000 + HEADLINE + 7919 * rank)
+    w = make_config(HEADLINE, seed=rank_seed(rank))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
 
     sampler = ClockSampler(local_rank)
@@ -226,11 +247,8 @@ def main():
     torch.cuda.synchronize()
     clocks = sampler.stop()
     sec = head["seconds"]
-    if dist is not None:
-        t = torch.tensor([sec], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        sec = float(t.item())
-    value = w.updates * world / sec
+    sec = max_over_ranks(dist, sec, "cuda")
+    value = aggregate_throughput(w.updates, world, sec)
 
     # ---- end to end: pinned host inputs -> device -> bi_filter -> host beliefs
     md, q = head["model"], head["q"]
@@ -247,11 +265,8 @@ def main():
 
     e2e_times = time_steps(e2e_step, max(3, args.steps // 2), 3, flush, torch)
     e2e_sec = sum(e2e_times) / len(e2e_times)
-    if dist is not None:
-        t = torch.tensor([e2e_sec], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_sec = float(t.item())
-    e2e = {"value": w.updates * world / e2e_sec, "unit": UNIT,
+    e2e_sec = max_over_ranks(dist, e2e_sec, "cuda")
+    e2e = {"value": aggregate_throughput(w.updates, world, e2e_sec), "unit": UNIT,
            "h2d_bytes_per_step": int(w.obs.nbytes + w.act.nbytes), "d2h_bytes_per_step": int(q.numel() * 4)}
 
     flops = algorithmic_flops(w)
