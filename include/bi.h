@@ -159,6 +159,39 @@ int bi_mmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
            const int32_t *act, int32_t iters, float *q_out, float *logq_out,
            int32_t *argmax_out, void *cuda_stream);
 
+/*
+ * Variational filtering without any allocation.  (The paper has no counterpart
+ * to this entry point: it is a deployment convenience of this library.)
+ *
+ * bi_model_create obtains device memory for the packed model, so it cannot be
+ * used by callers that are not allowed to allocate: a control loop on a GPU
+ * whose memory was handed out in full at start-up, a plug-in confined to
+ * another runtime's memory pool, or any path that cannot tolerate the device
+ * synchronisation cudaMalloc and cudaFree imply.  For them this call packs the
+ * model into a fixed scratch array inside the library
+ * (BI_STATIC_SCRATCH_BYTES of device memory per GPU that loads the library,
+ * held until the process exits), runs the general filtering kernel on that
+ * copy in float64 arithmetic and returns; it calls no cudaMalloc, no cudaFree
+ * and no host allocator.
+ *
+ *   desc      as for bi_model_create; only shared models (G == 1)
+ *   others    as for bi_filter
+ * Results are identical to bi_filter on a handle made from the same desc when
+ * that call runs the general kernel.  Returns BI_ERR_UNSUPPORTED if the packed
+ * model (float64 logs of every A_i, transition matrices, priors) needs more
+ * than BI_STATIC_SCRATCH_BYTES or the model is per-agent.
+ * The first call on a device looks up the scratch array's device address; make
+ * that first call outside any stream capture.  All calls share the one array,
+ * which keeps the previous call's contents: every call re-packs the model and
+ * clears its status word, and two calls whose GPU work overlaps (different
+ * streams, different threads) race on it -- serialise them.  Out-of-range
+ * indices are clamped as in bi_filter; no status word is reported.
+ */
+#define BI_STATIC_SCRATCH_BYTES (4u << 20)
+int bi_filter_static(const bi_model_desc *desc, int32_t N, int32_t T, const int32_t *obs,
+                     const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                     int32_t *argmax_out, void *cuda_stream);
+
 /* Synchronises the stream, returns the OR of BI_FLAG_* raised since the last
  * call in *flags (HOST) and clears them. */
 int bi_status(const bi_model_t *model, void *cuda_stream, uint32_t *flags);

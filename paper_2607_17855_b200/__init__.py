@@ -27,7 +27,8 @@ BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
 EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_vmp", "bi_mmp", "bi_status",
-           "bi_last_kernel", "bi_launch_count", "bi_strerror"]
+           "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
+BI_STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class BiError(RuntimeError):
@@ -71,6 +72,10 @@ def lib():
         L.bi_launch_count.argtypes = [ctypes.c_void_p]
         L.bi_strerror.restype = ctypes.c_char_p
         L.bi_strerror.argtypes = [ctypes.c_int]
+        L.bi_filter_static.restype = ctypes.c_int
+        L.bi_filter_static.argtypes = [ctypes.POINTER(_Desc), ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -184,6 +189,39 @@ class Model:
     @property
     def launch_count(self) -> int:
         return int(lib().bi_launch_count(self._h))
+
+
+def bi_filter_static(n, m, dep, U, A, B, D, obs, act, iters, q_out, logq_out=None, argmax_out=None, stream=None):
+    """Filtering for callers that must not allocate (``bi_filter_static``).
+
+    The library packs the shared model ``A``, ``B``, ``D`` (float32 CUDA
+    tensors laid out as for :class:`Model`, ``G == 1``) into its own fixed
+    scratch array on every call instead of using a handle, so no device memory
+    is obtained anywhere on this path; the caller supplies every output
+    tensor.  Calls share that one array: do not let two of them overlap on the
+    GPU.  The model must pack into ``BI_STATIC_SCRATCH_BYTES``.
+    """
+    L = lib()
+    n, m, U = [int(v) for v in n], [int(v) for v in m], [int(v) for v in U]
+    dep = [[int(f) for f in d] for d in dep]
+    d = _Desc()
+    d.F, d.M, d.G = len(n), len(m), 1
+    keep = [_i32(n), _i32(m), _i32([len(x) for x in dep]), _i32([f for x in dep for f in x]), _i32(U)]
+    d.n, d.m, d.dep_len, d.dep, d.U = [ctypes.cast(k, ctypes.c_void_p) for k in keep]
+    pa = (ctypes.c_void_p * max(len(m), 1))(*[a.data_ptr() for a in A])
+    pb = (ctypes.c_void_p * len(n))(*[b.data_ptr() for b in B])
+    pd = (ctypes.c_void_p * len(n))(*[x.data_ptr() for x in D])
+    d.A, d.B, d.D = [ctypes.cast(p, ctypes.c_void_p) for p in (pa, pb, pd)]
+    N, T = int(obs.shape[0]), int(obs.shape[1])
+    rc = L.bi_filter_static(ctypes.byref(d), N, T, ctypes.c_void_p(obs.data_ptr()),
+                            ctypes.c_void_p(act.data_ptr() if act is not None and act.numel() > 0 else None),
+                            int(iters), ctypes.c_void_p(q_out.data_ptr()),
+                            ctypes.c_void_p(logq_out.data_ptr() if logq_out is not None else None),
+                            ctypes.c_void_p(argmax_out.data_ptr() if argmax_out is not None else None),
+                            _stream_ptr(stream))
+    if rc != BI_OK:
+        raise BiError(rc, "bi_filter_static")
+    return q_out
 
 
 def model_from_workload(w, device="cuda", stream=None, arith: str = "f64") -> Model:
