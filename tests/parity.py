@@ -71,6 +71,41 @@ def compare(w, q_gpu, lq_gpu, am_gpu, q_ref, lq_ref, am_ref):
     return res
 
 
+def oracle_self_sensitivity(w, algo, eps=1e-13, seed=0):
+    """Per-agent maximum change of the oracle's own beliefs when its uniform
+    start is perturbed by a relative ``eps``: the conditioning of the K-step
+    Jacobi iteration for that agent.  (On sharp or sparse models the iteration
+    is chaotic: one ulp in the start can flip beliefs.)"""
+    import oracle
+    ref = oracle.run_workload(w, algo)[0]
+    N, T = w.obs.shape[:2]
+    start = np.concatenate([np.full((N, T, int(n)), 1.0 / n) for n in w.n], axis=2)
+    start = start * (1.0 + eps * np.random.default_rng(seed).standard_normal(start.shape))
+    pert = oracle.run_workload(w, algo, q_init=start)[0]
+    return np.abs(pert - ref).reshape(N, -1).max(axis=1)
+
+
+def compare_conditioned(w, algo, q_gpu, lq_gpu, am_gpu, ref):
+    """Parity with the conditioning taken into account.  Agents whose oracle
+    result moves by less than 1e-9 under a 1e-13 perturbation get the full
+    strict comparison (beliefs 1e-5, log-beliefs, argmax).  Every other agent
+    must still be a valid distribution and no further from the oracle than
+    max(1e-5, 10 x the oracle's own movement) (a fully chaotic agent, whose
+    oracle result flips under the probe, is only checked for validity)."""
+    stats = error_stats(w, q_gpu, ref[0])
+    moved = oracle_self_sensitivity(w, algo)
+    err = np.abs(np.asarray(q_gpu, np.float64) - ref[0]).reshape(ref[0].shape[0], -1).max(axis=1)
+    assert (err <= np.maximum(Q_TOL, 10.0 * moved)).all(), (err.max(), moved[err.argmax()])
+    well = np.flatnonzero(moved < 1e-9)
+    if len(well):
+        sub = w.take_agents(well)
+        compare(sub, q_gpu[well], lq_gpu[well] if lq_gpu is not None else None,
+                am_gpu[well] if am_gpu is not None else None, ref[0][well], ref[1][well], ref[2][well])
+    stats["well_conditioned_agents"] = int(len(well))
+    stats["agents"] = int(len(err))
+    return stats
+
+
 def run_gpu(w, algo=None, want_logq=True, want_argmax=True, model=None, arith="f64"):
     """Run the CUDA library on a workload; returns numpy (q, logq, argmax, model)."""
     import torch
@@ -90,7 +125,7 @@ def run_gpu(w, algo=None, want_logq=True, want_argmax=True, model=None, arith="f
             am.cpu().numpy() if am is not None else None, md)
 
 
-def check_workload(w, algo=None, agents=None, arith="f64", strict=True):
+def check_workload(w, algo=None, agents=None, arith="f64", strict=True, conditioned=False):
     """GPU on the whole workload, oracle on ``agents`` (all if None); compares those.
     ``strict=False`` only checks validity and returns the error statistics."""
     import oracle
@@ -102,7 +137,10 @@ def check_workload(w, algo=None, agents=None, arith="f64", strict=True):
         sub = w.take_agents(agents)
         q, lq, am = q[agents], lq[agents], am[agents]
     ref = oracle.run_workload(sub, algo)
-    out = compare(sub, q, lq, am, *ref) if strict else error_stats(sub, q, ref[0])
+    if conditioned:
+        out = compare_conditioned(sub, algo, q, lq, am, ref)
+    else:
+        out = compare(sub, q, lq, am, *ref) if strict else error_stats(sub, q, ref[0])
     out["kernel"] = md.last_kernel
     md.close()
     return out
