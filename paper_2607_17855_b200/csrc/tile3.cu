@@ -16,6 +16,7 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
   __shared__ __align__(16) R sm_e[UPW][NB + NCP];      // gathered e_b, e_c of the current iterate
   __shared__ __align__(16) R sm_q[UPW][NA + NB + NC];  // final beliefs of the previous step
   __shared__ __align__(16) R sm_L[LSMEM ? UPW : 1][LSMEM ? TT::P_TILE : 2];  // large tiles: the step's slice
+  __shared__ __align__(16) R sm_tp[UPW][TT::TP ? TT::TP_UNIT : 2];           // transpose area of the b / c sums
 
   const int lane = threadIdx.x;
   const int unit = lane / LPU;
@@ -26,8 +27,9 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
 
   TT t3;
   t3.init_lane(lane);
+  t3.tp = sm_tp[unit];
   const int a = t3.a, bi = t3.bi, ci = t3.ci;
-  const bool a_ok = t3.a_ok, b_ok = (a >> TT::SHB) < NBL, c_ok = ci < NC;
+  const bool a_ok = t3.a_ok, b_ok = t3.b_ok, c_ok = t3.c_ok;
   const int bsafe = b_ok ? bi : 0, csafe = c_ok ? ci : 0, asafe = a_ok ? a : 0;
   R *se = sm_e[unit], *sq = sm_q[unit];
   for (int i = t3.u; i < NB + NCP; i += LPU) se[i] = (R)0;

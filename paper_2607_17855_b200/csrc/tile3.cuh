@@ -133,10 +133,22 @@ struct Tile3 {
   static_assert(NB % SB == 0, "SB must divide NB");
   static_assert(LPU <= 32 && PB <= NAP && PC <= LPU, "tile does not fit a warp");
 
+  // With one lane per a (SB == 1) the cross-lane sums of the b and c messages
+  // go through a small shared-memory transpose instead of shuffles: lane u
+  // stores its partials as row u, then reads column u.  Fewer instructions
+  // than the butterfly (no selects), and lane u simply owns b = u and c = u.
+  static constexpr bool TP = SB == 1 && NB <= LPU && NC <= LPU;
+  static constexpr int TP_T = NBL + NCP;
+  // row stride: even, = 2 mod 4 elements, so 16-byte row stores of 8 consecutive lanes hit distinct banks
+  static constexpr int TPR = (TP_T % 4 <= 2) ? TP_T - TP_T % 4 + 2 : TP_T + 3;
+  static constexpr int TP_UNIT = LPU * TPR + 8;  // elements per unit (8 extra: units of a half-warp on different banks)
+
   // lane coordinates
   int u, a, bh;       // lane within unit, a index, b half
-  int bi, ci;         // owned b (global index) and c after the reduce-scatters
-  bool a_ok, own_a, own_b, own_c;  // valid a; designated writer of x_a / x_b / x_c
+  int bi, ci;         // owned b (global index) and c
+  bool a_ok, b_ok, c_ok;        // the owned a / b / c index is a real state
+  bool own_a, own_b, own_c;     // designated writer of x_a / x_b / x_c (duplicates exist when SB > 1)
+  R *tp;              // this unit's transpose area (TP only)
 
   R L[NBL][NCP];      // this lane's part of the summed slice
   R ea, eb[NBL], ec[NCP];  // unnormalised beliefs this lane contracts with
@@ -147,12 +159,21 @@ struct Tile3 {
     a = u / SB;
     bh = u % SB;
     a_ok = a < NA;
-    const int ib = a >> SHB;
-    bi = bh * NBL + ib;
-    ci = u >> SHC;
     own_a = a_ok && bh == 0;
-    own_b = ib < NBL && (a & ((1 << SHB) - 1)) == 0;
-    own_c = ci < NC && (u & ((1 << SHC) - 1)) == 0;
+    tp = nullptr;
+    if (TP) {
+      bi = u; ci = u;
+      own_b = b_ok = u < NB;
+      own_c = c_ok = u < NC;
+    } else {
+      const int ib = a >> SHB;
+      bi = bh * NBL + ib;
+      ci = u >> SHC;
+      b_ok = ib < NBL;
+      c_ok = ci < NC;
+      own_b = b_ok && (a & ((1 << SHB) - 1)) == 0;
+      own_c = c_ok && (u & ((1 << SHC) - 1)) == 0;
+    }
   }
 
   // L[b][c] = sum over the group's modalities of their observed slices.  The
@@ -263,13 +284,32 @@ struct Tile3 {
 #pragma unroll
     for (int bl = 0; bl < NBL; ++bl) lav[bl] = V[bl] * eb[bl];
     R la = group_sum<R, SB, 1>(tree_sum<R, NBL>(lav));
-    R pb[PB], pc[PC];
+    R lb, lc;
+    if (TP) {
+      R *row = tp + u * TPR;
 #pragma unroll
-    for (int i = 0; i < PB; ++i) pb[i] = i < NBL ? ea * V[i < NBL ? i : 0] : (R)0;
+      for (int bl = 0; bl < NBL; ++bl) row[bl] = ea * V[bl];
 #pragma unroll
-    for (int c = 0; c < PC; ++c) pc[c] = c < NCP ? ea * W[c < NCP ? c : 0] : (R)0;
-    R lb = reduce_scatter<R, PB, NAP, SB>(pb, a);
-    R lc = reduce_scatter<R, PC, LPU, 1>(pc, u);
+      for (int c = 0; c < NCP; ++c) row[NBL + c] = ea * W[c];
+      __syncwarp();
+      R cb[NAP], cc[NAP];
+#pragma unroll
+      for (int r = 0; r < NAP; ++r) {
+        cb[r] = tp[r * TPR + (b_ok ? u : 0)];
+        cc[r] = tp[r * TPR + NBL + (c_ok ? u : 0)];
+      }
+      lb = tree_sum<R, NAP>(cb);
+      lc = tree_sum<R, NAP>(cc);
+      __syncwarp();
+    } else {
+      R pb[PB], pc[PC];
+#pragma unroll
+      for (int i = 0; i < PB; ++i) pb[i] = i < NBL ? ea * V[i < NBL ? i : 0] : (R)0;
+#pragma unroll
+      for (int c = 0; c < PC; ++c) pc[c] = c < NCP ? ea * W[c < NCP ? c : 0] : (R)0;
+      lb = reduce_scatter<R, PB, NAP, SB>(pb, a);
+      lc = reduce_scatter<R, PC, LPU, 1>(pc, u);
+    }
     xa = la * sa;
     xb = lb * sb;
     xc = lc * sc;

@@ -27,7 +27,7 @@ struct WindowGeom {
   int32_t CS;       // CTAs per cluster (= per agent)
   int32_t Tc;       // time steps per CTA
   int32_t units;    // step slots per CTA (>= Tc; whole warps)
-  int32_t off_q, off_se, off_B;  // element offsets: belief buffers, gather area, transition matrices
+  int32_t off_q, off_se, off_B, off_tp;  // element offsets: belief buffers, gather area, transition matrices, transpose areas
 };
 
 // sum_r M[r][s] q[r] with two interleaved accumulators; M and q in shared memory
@@ -71,8 +71,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
 
   TT t3;
   t3.init_lane(lane);
+  t3.tp = Ls + geo.off_tp + (size_t)tl * TT::TP_UNIT;
   const int a = t3.a, bi = t3.bi, ci = t3.ci;
-  const bool a_ok = t3.a_ok, b_ok = (a >> TT::SHB) < NBL, c_ok = ci < NC;
+  const bool a_ok = t3.a_ok, b_ok = t3.b_ok, c_ok = t3.c_ok;
   const int bsafe = b_ok ? bi : 0, csafe = c_ok ? ci : 0, asafe = a_ok ? a : 0;
   R *se = seb + tl * (NB + NCP);
   R *Lt = Ls + (size_t)tl * PT;
@@ -309,7 +310,7 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
     const int warps = (Tc + UPW - 1) / UPW;
     const int units = warps * UPW;
     const size_t elems = (size_t)units * TT::P_TILE + 2 * (size_t)(units + 2) * SQ +
-                         (size_t)units * (NB + TT::NCP) + bsz;
+                         (size_t)units * (NB + TT::NCP) + bsz + (TT::TP ? (size_t)units * TT::TP_UNIT : 0);
     const size_t b = elems * sizeof(R);
     if (warps * 32 > 512 || b > (size_t)smem_budget) continue;
     const int per_sm = (int)std::min<size_t>(8, (size_t)(228 * 1024) / (b + 1024));
@@ -327,7 +328,8 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
     geo.off_q = units * TT::P_TILE;
     geo.off_se = geo.off_q + 2 * (units + 2) * SQ;
     geo.off_B = geo.off_se + units * (NB + TT::NCP);
-    bytes = ((size_t)geo.off_B + bsz) * sizeof(R);
+    geo.off_tp = geo.off_B + (int)((bsz + 1) & ~(size_t)1);
+    bytes = ((size_t)geo.off_tp + (TT::TP ? (size_t)units * TT::TP_UNIT : 0)) * sizeof(R);
     threads = warps * 32;
     found = true;
   }
