@@ -259,9 +259,13 @@ struct Tile3 {
   // the same with the slice read from shared memory (lane-interleaved layout)
   // instead of registers: for kernels that keep many steps' slices on chip
   __device__ __forceinline__ void messages_smem(const R *__restrict__ Ls, R &xa, R &xb, R &xc) {
-    R V[NBL], W[NCP];
+    // V[b] is accumulated in VE interleaved partial sums: consecutive elements
+    // of a row would otherwise form one chain of dependent multiply-adds
+    R V[NBL], W[NCP], Vp[NBL][VE];
 #pragma unroll
-    for (int bl = 0; bl < NBL; ++bl) V[bl] = (R)0;
+    for (int bl = 0; bl < NBL; ++bl)
+#pragma unroll
+      for (int i = 0; i < VE; ++i) Vp[bl][i] = (R)0;
 #pragma unroll
     for (int c = 0; c < NCP; ++c) W[c] = (R)0;
     const R *p = Ls + u * VE;
@@ -272,10 +276,12 @@ struct Tile3 {
 #pragma unroll
       for (int i = 0; i < VE; ++i) {
         const int bl = (v * VE + i) / NCP, c = (v * VE + i) % NCP;
-        V[bl] = fma(x[i], ec[c], V[bl]);
+        Vp[bl][i] = fma(x[i], ec[c], Vp[bl][i]);
         W[c] = fma(eb[bl], x[i], W[c]);
       }
     }
+#pragma unroll
+    for (int bl = 0; bl < NBL; ++bl) V[bl] = tree_sum<R, VE>(Vp[bl]);
     finish(V, W, xa, xb, xc);
   }
 

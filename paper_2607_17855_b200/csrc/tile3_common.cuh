@@ -6,7 +6,7 @@
 
 // compiled tile shapes: packed dims (a, b, c), the lanes along b, and whether the
 // filtering kernel keeps the step's slice in shared memory (large tiles) or registers
-#define BI_TILE3_SHAPES(X) X(8, 6, 8, 1, false) X(16, 12, 8, 1, true) X(3, 2, 4, 1, false)
+#define BI_TILE3_SHAPES(X) X(8, 6, 8, 1, false) X(16, 12, 8, 2, true) X(3, 2, 4, 1, false) X(10, 6, 8, 1, true)
 
 
 struct Tile3Params {

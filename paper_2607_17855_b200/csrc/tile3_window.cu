@@ -43,8 +43,10 @@ __device__ __forceinline__ R col_dot_smem(const R *col, int stride, const R *q) 
   return s0 + s1;
 }
 
-template <typename R, int NA, int NB, int NC, int SB, int ALGO, bool STALE, bool CLUSTER>
-__global__ void __launch_bounds__(512)
+// LREG: the step's summed slice lives in registers (small tiles); otherwise in
+// shared memory (tiles too large for the register file).
+template <typename R, int NA, int NB, int NC, int SB, bool LREG, int ALGO, bool STALE, bool CLUSTER>
+__global__ void __launch_bounds__(320)
 bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   using TT = Tile3<R, NA, NB, NC, SB>;
   constexpr int LPU = TT::LPU, NBL = TT::NBL, NCP = TT::NCP, NAP = TT::NAP, VE = TT::VE, NV = TT::NV;
@@ -76,11 +78,19 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   const bool a_ok = t3.a_ok, b_ok = t3.b_ok, c_ok = t3.c_ok;
   const int bsafe = b_ok ? bi : 0, csafe = c_ok ? ci : 0, asafe = a_ok ? a : 0;
   R *se = seb + tl * (NB + NCP);
-  R *Lt = Ls + (size_t)tl * PT;
+  R *Lt = Ls + (LREG ? 0 : (size_t)tl * PT);
   for (int i = t3.u; i < NB + NCP; i += LPU) se[i] = (R)0;
 
-  // ---- gather the step's summed slice into shared memory (one HBM read per slice)
-  {
+  // ---- gather the step's summed slice (one HBM read per slice) into registers or shared memory
+  if (LREG) {
+    const size_t ob = ((size_t)agent * T + t) * p.M;
+    const R *slice[BI_MAX_M];
+    for (int mi = 0; mi < p.nmem; ++mi) {
+      int o = clamp_flag(__ldg(p.obs + ob + p.modality[mi]), p.mcount[mi], p.status, BI_FLAG_OBS_RANGE);
+      slice[mi] = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile;
+    }
+    t3.load_slices(slice, p.nmem);
+  } else {
     const size_t ob = ((size_t)agent * T + t) * p.M;
     constexpr int CH = NV % 12 == 0 ? 12 : (NV % 8 == 0 ? 8 : (NV % 6 == 0 ? 6 : NV));  // vectors in flight per pass
     for (int v0 = 0; v0 < NV; v0 += CH) {
@@ -199,7 +209,8 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       }
       ta += va; tb += vb; tc += vc;
     }
-    t3.messages_smem(Lt, xa, xb, xc);
+    if (LREG) t3.messages(xa, xb, xc);
+    else t3.messages_smem(Lt, xa, xb, xc);
     xa = a_ok ? xa + ta : -bi_inf<R>();
     xb = b_ok ? xb + tb : -bi_inf<R>();
     xc = c_ok ? xc + tc : -bi_inf<R>();
@@ -280,7 +291,7 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   }
 }
 
-template <typename R, int NA, int NB, int NC, int SB, int ALGO>
+template <typename R, int NA, int NB, int NC, int SB, bool LREG, int ALGO>
 int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   using TT = Tile3<R, NA, NB, NC, SB>;
   constexpr int SQ = (NA + NB + NC + 1) & ~1;
@@ -309,11 +320,12 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
     if (cs > 1 && Tc * (cs - 1) >= p.T) continue;  // an empty CTA: no gain over the smaller cluster
     const int warps = (Tc + UPW - 1) / UPW;
     const int units = warps * UPW;
-    const size_t elems = (size_t)units * TT::P_TILE + 2 * (size_t)(units + 2) * SQ +
+    const size_t elems = (LREG ? 0 : (size_t)units * TT::P_TILE) + 2 * (size_t)(units + 2) * SQ +
                          (size_t)units * (NB + TT::NCP) + bsz + (TT::TP ? (size_t)units * TT::TP_UNIT : 0);
     const size_t b = elems * sizeof(R);
-    if (warps * 32 > 512 || b > (size_t)smem_budget) continue;
-    const int per_sm = (int)std::min<size_t>(8, (size_t)(228 * 1024) / (b + 1024));
+    if (warps * 32 > (320) || b > (size_t)smem_budget) continue;
+    int per_sm = (int)std::min<size_t>(8, (size_t)(228 * 1024) / (b + 1024));
+    if (LREG) per_sm = std::min(per_sm, std::max(1, 65536 / (warps * 32 * 208)));  // about 200 registers per thread
     // useful warps resident per SM, discounted by idle step slots
     const double score = (double)per_sm * warps * ((double)Tc / units) - 0.01 * cs;
     if (score > best_score) { best_score = score; best_cs = cs; }
@@ -325,7 +337,7 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
     const int warps = (Tc + UPW - 1) / UPW;
     const int units = warps * UPW;
     geo.CS = cs; geo.Tc = Tc; geo.units = units;
-    geo.off_q = units * TT::P_TILE;
+    geo.off_q = LREG ? 0 : units * TT::P_TILE;
     geo.off_se = geo.off_q + 2 * (units + 2) * SQ;
     geo.off_B = geo.off_se + units * (NB + TT::NCP);
     geo.off_tp = geo.off_B + (int)((bsz + 1) & ~(size_t)1);
@@ -350,7 +362,7 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   cudaError_t e;
 #define BI_WIN_LAUNCH(ST, CL)                                                                         \
   do {                                                                                                \
-    auto kern = bi_tile3_window_kernel<R, NA, NB, NC, SB, ALGO, ST, CL>;                             \
+    auto kern = bi_tile3_window_kernel<R, NA, NB, NC, SB, LREG, ALGO, ST, CL>;                             \
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
     if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, kern, p, geo);                                 \
   } while (0)
@@ -370,7 +382,7 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
 template <typename R, int ALGO>
 int dispatch_window(const Tile3Params &p, int na, int nb, int nc, int budget, cudaStream_t stream) {
 #define X(A, B, C, S, LS) \
-  if (na == A && nb == B && nc == C) return launch_window<R, A, B, C, S, ALGO>(p, budget, stream);
+  if (na == A && nb == B && nc == C) return launch_window<R, A, B, C, S, !(LS), ALGO>(p, budget, stream);
   BI_TILE3_SHAPES(X)
 #undef X
   return BI_ERR_UNSUPPORTED;

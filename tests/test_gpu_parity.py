@@ -163,6 +163,10 @@ def test_tile_filter_shapes_and_ragged_batches(arith):
     assert res["kernel"] == f"tile3_filter_{arith}", res
     if not strict:
         assert res["q_max_err"] < 1e-3
+    # a tile kept in shared memory instead of registers (packed dims 10 x 6 x 8)
+    w = _custom(36, [10, 6, 8], [4, 3], [[0, 1, 2], [1, 2, 0]], [2, 1, 3], N=7, T=5, K=6)
+    res = check_workload(w, "filter", arith=arith, strict=strict)
+    assert res["kernel"] == f"tile3_filter_{arith}", res
 
 
 # ---- the register-tile window kernels (VMP / MMP), incl. multi-CTA clusters
@@ -186,6 +190,19 @@ def test_tile_window_kernels(algo):
     w = _custom(33, [4, 3, 2], [3, 5], [[0, 1, 2], [2, 0, 1]], [2, 3, 1], N=7, T=6, K=9, sparsity=0.5)
     res = check_workload(w, algo)
     assert res["kernel"] == f"tile3_{algo}_f64", res
+    # a tile kept in shared memory instead of registers (packed dims 10 x 6 x 8)
+    w = _custom(35, [10, 6, 8], [4, 3], [[0, 1, 2], [1, 2, 0]], [2, 1, 3], N=5, T=9, K=6)
+    res = check_workload(w, algo)
+    assert res["kernel"] == f"tile3_{algo}_f64", res
     # float32 arithmetic: single CTA holds the window
     res = check_workload(make_config(4, N=4, T=20, K=8), algo, arith="f32", strict=False)
     assert res["kernel"] == f"tile3_{algo}_f32", res
+
+
+def test_tile_window_small_tile_across_a_cluster():
+    # 8 lanes per step with the slices in registers: a 40-step window is split
+    # over several CTAs of a cluster (the thread cap of the register variant)
+    res = check_workload(make_config(2, N=5, T=40, K=6), "vmp")
+    assert res["kernel"] == "tile3_vmp_f64", res
+    res = check_workload(make_config(2, N=5, T=64, K=4), "mmp")
+    assert res["kernel"] == "tile3_mmp_f64", res
