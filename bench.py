@@ -34,6 +34,13 @@ FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12   # 37.2
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # 74.4
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the benchmark's
+# workload, from the ncu captures summarised under profiles/ (bytes)
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "tile3_filter_f64": 5.01e6 + 3.6e3,   # profiles/tile3_filter_f64_config2.md
+}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -108,7 +115,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -245,7 +252,6 @@ def main():
     sampler.start()
     head = bench_config(torch, bi, w, "filter", args.arith, args.steps, args.warmup, flush)
     torch.cuda.synchronize()
-    clocks = sampler.stop()
     sec = head["seconds"]
     sec = max_over_ranks(dist, sec, "cuda")
     value = aggregate_throughput(w.updates, world, sec)
@@ -265,6 +271,7 @@ def main():
 
     e2e_times = time_steps(e2e_step, max(3, args.steps // 2), 3, flush, torch)
     e2e_sec = sum(e2e_times) / len(e2e_times)
+    clocks = sampler.stop()  # sampled over both timed regions
     e2e_sec = max_over_ranks(dist, e2e_sec, "cuda")
     e2e = {"value": aggregate_throughput(w.updates, world, e2e_sec), "unit": UNIT,
            "h2d_bytes_per_step": int(w.obs.nbytes + w.act.nbytes), "d2h_bytes_per_step": int(q.numel() * 4)}
@@ -276,10 +283,7 @@ def main():
                 "frac": achieved / peak, "traffic": None,
                 "kernel": head["kernel"],
                 "peak_source": f"derived: 148 SMs x {64 if args.arith == 'f64' else 128} lanes x 2 x 1.965 GHz"}
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(prof):
-        with open(prof) as fh:
-            roofline["traffic"] = json.load(fh).get(head["kernel"])
+    roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(head["kernel"])
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
