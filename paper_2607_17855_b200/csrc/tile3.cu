@@ -70,8 +70,10 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
 
     t3.set_uniform();
     R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
-    float ma = 0.f, mb = 0.f, mc = 0.f;     // softmax shifts in use
-    float pma = 0.f, pmb = 0.f, pmc = 0.f;  // exact maxima of the previous iterate
+    // softmax shifts in use
+    float ma = STALE ? group_max_f<NAP, SB>(a_ok ? (float)lpa : -CUDART_INF_F) : 0.f;
+    float mb = STALE ? group_max_f<LPU, 1>(b_ok ? (float)lpb : -CUDART_INF_F) : 0.f;
+    float mc = STALE ? group_max_f<LPU, 1>(c_ok ? (float)lpc : -CUDART_INF_F) : 0.f;
     for (int k = 0; k < p.K; ++k) {
       if (LSMEM) t3.messages_smem(sm_L[LSMEM ? unit : 0], xa, xb, xc);
       else t3.messages(xa, xb, xc);
@@ -79,18 +81,25 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       xb = b_ok ? xb + lpb : -bi_inf<R>();
       xc = c_ok ? xc + lpc : -bi_inf<R>();
       // Softmax is invariant to the shift; any shift that keeps the exponents
-      // in range is exact.  With STALE the previous iterate's maximum is used
-      // (logits move by less than the range bound between iterates), which
-      // takes the max reduction off the dependency chain.
-      const float cma = group_max_f<NAP, SB>((float)xa);
-      const float cmb = group_max_f<LPU, 1>((float)xb);
-      const float cmc = group_max_f<LPU, 1>((float)xc);
-      if (!STALE || k == 0) { ma = cma; mb = cmb; mc = cmc; }
-      else { ma = pma; mb = pmb; mc = pmc; }
-      pma = cma; pmb = cmb; pmc = cmc;
-      const R ean = a_ok ? bi_exp(xa - (R)ma) : (R)0;
-      const R ebn = b_ok ? bi_exp(xb - (R)mb) : (R)0;
-      const R ecn = c_ok ? bi_exp(xc - (R)mc) : (R)0;
+      // in range is exact.  With STALE the shift is the previous iterate's
+      // maximum (the prior's maximum at the first iterate: the likelihood
+      // message is <= 0 and bounded below by nmem * ln(1e-16)), so the max
+      // reduction sits after the exponentials in program order and its
+      // shuffles no longer delay them (a warp issues in order).
+      if (!STALE) {
+        ma = group_max_f<NAP, SB>((float)xa);
+        mb = group_max_f<LPU, 1>((float)xb);
+        mc = group_max_f<LPU, 1>((float)xc);
+      }
+      const R ean = a_ok ? bi_exp_inline(xa - (R)ma) : (R)0;
+      const R ebn = b_ok ? bi_exp_inline(xb - (R)mb) : (R)0;
+      const R ecn = c_ok ? bi_exp_inline(xc - (R)mc) : (R)0;
+      float nma = ma, nmb = mb, nmc = mc;
+      if (STALE && k + 1 < p.K) {
+        nma = group_max_f<NAP, SB>((float)xa);
+        nmb = group_max_f<LPU, 1>((float)xb);
+        nmc = group_max_f<LPU, 1>((float)xc);
+      }
       if (t3.own_b) se[bi] = ebn;
       if (t3.own_c) se[NB + ci] = ecn;
       za = group_sum<R, NAP, SB>(ean);
@@ -106,6 +115,7 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       t3.sa = rinv * za;
       t3.sb = rinv * zb;
       t3.sc = rinv * zc;
+      if (STALE && k + 1 < p.K) { ma = nma; mb = nmb; mc = nmc; }
       __syncwarp();
     }
 

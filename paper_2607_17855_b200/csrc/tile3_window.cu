@@ -220,9 +220,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     if (!STALE || k == 0) { ma = cma; mb = cmb; mc = cmc; }
     else { ma = pma; mb = pmb; mc = pmc; }
     pma = cma; pmb = cmb; pmc = cmc;
-    const R ean = a_ok ? bi_exp(xa - (R)ma) : (R)0;
-    const R ebn = b_ok ? bi_exp(xb - (R)mb) : (R)0;
-    const R ecn = c_ok ? bi_exp(xc - (R)mc) : (R)0;
+    const R ean = a_ok ? bi_exp_inline(xa - (R)ma) : (R)0;
+    const R ebn = b_ok ? bi_exp_inline(xb - (R)mb) : (R)0;
+    const R ecn = c_ok ? bi_exp_inline(xc - (R)mc) : (R)0;
     __syncwarp();
     if (t3.own_b) se[bi] = ebn;
     if (t3.own_c) se[NB + ci] = ecn;
