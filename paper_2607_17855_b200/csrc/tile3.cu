@@ -62,9 +62,9 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       const R *ta = (const R *)p.BfT[0] + (size_t)g * p.Bstride[0] + (size_t)ua * NA * p.np[0] + asafe;
       const R *tb = (const R *)p.BfT[1] + (size_t)g * p.Bstride[1] + (size_t)ub * NB * p.np[1] + bsafe;
       const R *tc = (const R *)p.BfT[2] + (size_t)g * p.Bstride[2] + (size_t)uc * NC * p.np[2] + csafe;
-      lpa = bi_log(bi_max(col_dot<R, NA>(ta, p.np[0], sq), (R)BI_EPS));
-      lpb = bi_log(bi_max(col_dot<R, NB>(tb, p.np[1], sq + NA), (R)BI_EPS));
-      lpc = bi_log(bi_max(col_dot<R, NC>(tc, p.np[2], sq + NA + NB), (R)BI_EPS));
+      lpa = bi_log_inline(bi_max(col_dot<R, NA>(ta, p.np[0], sq), (R)BI_EPS));
+      lpb = bi_log_inline(bi_max(col_dot<R, NB>(tb, p.np[1], sq + NA), (R)BI_EPS));
+      lpc = bi_log_inline(bi_max(col_dot<R, NC>(tc, p.np[2], sq + NA + NB), (R)BI_EPS));
     }
     __syncwarp();
 

@@ -191,9 +191,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       R vb = col_dot_smem<R, NB>(pa1, p.np[1], qp + NA);
       R vc = col_dot_smem<R, NC>(pa2, p.np[2], qp + NA + NB);
       if (ALGO == BI_ALGO_MMP) {
-        va = (R)0.5 * bi_log(bi_max(va, (R)BI_EPS));
-        vb = (R)0.5 * bi_log(bi_max(vb, (R)BI_EPS));
-        vc = (R)0.5 * bi_log(bi_max(vc, (R)BI_EPS));
+        va = (R)0.5 * bi_log_inline(bi_max(va, (R)BI_EPS));
+        vb = (R)0.5 * bi_log_inline(bi_max(vb, (R)BI_EPS));
+        vc = (R)0.5 * bi_log_inline(bi_max(vc, (R)BI_EPS));
       }
       ta = va; tb = vb; tc = vc;
     }
@@ -203,9 +203,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       R vb = col_dot_smem<R, NB>(fu1, p.np[1], qn + NA);
       R vc = col_dot_smem<R, NC>(fu2, p.np[2], qn + NA + NB);
       if (ALGO == BI_ALGO_MMP) {
-        va = (R)0.5 * bi_log(bi_max(va, (R)BI_EPS));
-        vb = (R)0.5 * bi_log(bi_max(vb, (R)BI_EPS));
-        vc = (R)0.5 * bi_log(bi_max(vc, (R)BI_EPS));
+        va = (R)0.5 * bi_log_inline(bi_max(va, (R)BI_EPS));
+        vb = (R)0.5 * bi_log_inline(bi_max(vb, (R)BI_EPS));
+        vc = (R)0.5 * bi_log_inline(bi_max(vc, (R)BI_EPS));
       }
       ta += va; tb += vb; tc += vc;
     }
