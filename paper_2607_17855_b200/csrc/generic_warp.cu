@@ -173,7 +173,7 @@ __device__ __forceinline__ void softmax_warp(const BiDev &md, const R *ell, R *q
     // the shift only has to be close to the maximum (softmax is shift
     // invariant): a float reduction halves the shuffles of a double one
     R mx = final ? warp_max(x) : (R)warp_max((float)x);
-    R e = lane < n ? bi_exp(x - mx) : (R)0;
+    R e = lane < n ? bi_exp_inline(x - mx) : (R)0;
     R z = warp_sum(e);
     R q = e * bi_rcp(z);
     if (lane < md.npad[f]) qn[op + lane] = lane < n ? q : (R)0;
@@ -249,7 +249,7 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
         } else {
           int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
           const R *col = (const R *)md.BfT[f] + (size_t)g * md.Bstride[f] + (size_t)u * n * md.npad[f] + s;
-          lp = bi_log(bi_max(col_dot_rt<R>(col, md.npad[f], cur + md.offp[f], n), (R)BI_EPS));
+          lp = bi_log_inline(bi_max(col_dot_rt<R>(col, md.npad[f], cur + md.offp[f], n), (R)BI_EPS));
         }
       }
       lpri[idx] = lp;
@@ -325,14 +325,14 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
             const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);  // [previous][next]
             const R *col = M0 + (size_t)g * md.Bstride[f] + (size_t)u * n * np + s;
             R v = col_dot_rt<R>(col, np, cur + (size_t)(t - 1) * Sp + md.offp[f], n);
-            msg = ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log(bi_max(v, (R)BI_EPS));
+            msg = ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
           }
           if (t + 1 < T) {
             int u = clamp_flag(act[((size_t)a * (T - 1) + t) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);  // [next][previous]
             const R *col = M1 + (size_t)g * md.Bstride[f] + (size_t)u * n * np + s;
             R v = col_dot_rt<R>(col, np, cur + (size_t)(t + 1) * Sp + md.offp[f], n);
-            msg += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log(bi_max(v, (R)BI_EPS));
+            msg += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
           }
         }
         ell[idx] = msg;

@@ -36,13 +36,24 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
   __syncwarp();
 
   const size_t out_base = (size_t)agent * p.T;
+  // The index streams are read one step ahead: their DRAM latency then overlaps
+  // the previous step's iterations instead of heading every step's chain.
+  int o_next[BI_MAX_M], u_next[3] = {0, 0, 0};
+  for (int mi = 0; mi < p.nmem; ++mi) o_next[mi] = __ldg(p.obs + out_base * p.M + p.modality[mi]);
   for (int t = 0; t < p.T; ++t) {
     // ---- the step's summed slice: one gather of every modality's observed slice
     const R *slice[BI_MAX_M];
     for (int mi = 0; mi < p.nmem; ++mi) {
-      int o = clamp_flag(__ldg(p.obs + (out_base + t) * p.M + p.modality[mi]), p.mcount[mi], p.status,
-                         BI_FLAG_OBS_RANGE);
+      int o = clamp_flag(o_next[mi], p.mcount[mi], p.status, BI_FLAG_OBS_RANGE);
       slice[mi] = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile;
+    }
+    const int u_cur[3] = {u_next[0], u_next[1], u_next[2]};
+    if (t + 1 < p.T) {
+      for (int mi = 0; mi < p.nmem; ++mi) o_next[mi] = __ldg(p.obs + (out_base + t + 1) * p.M + p.modality[mi]);
+      const int32_t *an = p.act + ((size_t)agent * (p.T - 1) + t) * 3;
+      u_next[0] = __ldg(an + p.fac[0]);
+      u_next[1] = __ldg(an + p.fac[1]);
+      u_next[2] = __ldg(an + p.fac[2]);
     }
     if (LSMEM) t3.load_slices_smem(slice, p.nmem, sm_L[LSMEM ? unit : 0]);
     else t3.load_slices(slice, p.nmem);
@@ -54,10 +65,9 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       lpb = __ldg((const R *)p.logD[1] + (size_t)g * p.Dstride[1] + bsafe);
       lpc = __ldg((const R *)p.logD[2] + (size_t)g * p.Dstride[2] + csafe);
     } else {
-      const int32_t *ac = p.act + ((size_t)agent * (p.T - 1) + (t - 1)) * 3;
-      int ua = clamp_flag(__ldg(ac + p.fac[0]), p.U[0], p.status, BI_FLAG_ACT_RANGE);
-      int ub = clamp_flag(__ldg(ac + p.fac[1]), p.U[1], p.status, BI_FLAG_ACT_RANGE);
-      int uc = clamp_flag(__ldg(ac + p.fac[2]), p.U[2], p.status, BI_FLAG_ACT_RANGE);
+      int ua = clamp_flag(u_cur[0], p.U[0], p.status, BI_FLAG_ACT_RANGE);
+      int ub = clamp_flag(u_cur[1], p.U[1], p.status, BI_FLAG_ACT_RANGE);
+      int uc = clamp_flag(u_cur[2], p.U[2], p.status, BI_FLAG_ACT_RANGE);
       // transposed forward matrices [previous][next]: the lanes of a unit read consecutive next states
       const R *ta = (const R *)p.BfT[0] + (size_t)g * p.Bstride[0] + (size_t)ua * NA * p.np[0] + asafe;
       const R *tb = (const R *)p.BfT[1] + (size_t)g * p.Bstride[1] + (size_t)ub * NB * p.np[1] + bsafe;
