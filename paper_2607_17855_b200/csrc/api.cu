@@ -448,6 +448,7 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
 extern "C" int bi_model_destroy(bi_model_t *model) {
   if (!model) return BI_OK;
   cudaError_t e = cudaDeviceSynchronize();
+  if (model->ws) cudaFree(model->ws);
   free_all(model);
   delete model;
   return e == cudaSuccess ? BI_OK : BI_ERR_CUDA;
@@ -468,6 +469,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   bi_model *mut = const_cast<bi_model *>(model);
   int rc = bi_launch_tile3(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_warp(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;

@@ -89,6 +89,8 @@ struct bi_model {
   int rows_max;     // largest first-level row count over groups
   int64_t launches;
   const char *last_kernel;
+  void *ws;         // workspace of the batched window path (stream-ordered allocation), or NULL
+  size_t ws_bytes;
 };
 
 struct BiCall {
@@ -106,5 +108,6 @@ int bi_launch_generic(const BiCall &c, bi_model *mut);
 int bi_launch_warp(const BiCall &c, bi_model *mut);
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
 int bi_launch_tile3_window(const BiCall &c, bi_model *mut);
+int bi_launch_batch(const BiCall &c, bi_model *mut);
 // SB of the compiled register-tile shape for packed dims (na, nb, nc), or 0
 int bi_tile3_shape(int na, int nb, int nc);

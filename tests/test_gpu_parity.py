@@ -206,3 +206,18 @@ def test_tile_window_small_tile_across_a_cluster():
     assert res["kernel"] == "tile3_vmp_f64", res
     res = check_workload(make_config(2, N=5, T=64, K=4), "mmp")
     assert res["kernel"] == "tile3_mmp_f64", res
+
+
+# ---- batched window kernels (shared model, units bucketed by observed outcome)
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_batched_window_kernels(algo):
+    res = check_workload(make_config(3, N=128, T=16, K=9), algo, agents=range(0, 128, 5))
+    assert res["kernel"] == f"batch_{algo}_f64", res
+    # rank-3 and rank-2 groups, a single-factor modality, an unobserved factor, odd sizes
+    w = _custom(41, [3, 4, 2, 5, 3], [3, 2, 4, 3], [[0, 1, 2], [3, 4], [1], [2, 0, 1]], [2, 1, 3, 2, 2],
+                N=171, T=12, K=7, sparsity=0.5)
+    res = check_workload(w, algo, agents=range(0, 171, 7))
+    assert res["kernel"] == f"batch_{algo}_f64", res
+    res = check_workload(make_config(3, N=160, T=13, K=5), algo, arith="f32", strict=False)
+    assert res["kernel"] == f"batch_{algo}_f32", res
