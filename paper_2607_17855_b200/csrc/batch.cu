@@ -23,7 +23,7 @@
 
 namespace {
 
-constexpr int kTU = 128;   // units per contraction CTA
+constexpr int kTU = 128;   // most units per contraction CTA (the call picks 32, 64 or 128)
 
 // packed dims of the compiled group shapes: rank, then the axis sizes (last axis unpadded)
 #define BI_BATCH_SHAPES(X) \
@@ -44,7 +44,7 @@ struct BatchMember {
 struct BatchParams {
   BatchMember mem[BI_MAX_M];
   int32_t nmem;            // members of rank >= 2
-  int32_t NU, Sp, ntask;
+  int32_t NU, Sp, ntask, tu;   // tu: units per contraction CTA
   const int32_t *perm;     // [nmem][NU] unit ids ordered by observed outcome
   const int4 *task;        // [ntask] (outcome, first position, count, unused)
   void *ellp;              // [nmem][NU][Sp] partial likelihood messages
@@ -185,10 +185,11 @@ bi_batch_bucket_kernel(BatchParams P, const int32_t *__restrict__ obs, int M, ui
   __syncthreads();
   if (threadIdx.x == 0) {
     int pos = 0, slot = mm.task0;
-    const int slot_end = mm.task0 + (NU + kTU - 1) / kTU + m;
+    const int tu = P.tu;
+    const int slot_end = mm.task0 + (NU + tu - 1) / tu + m;
     for (int o = 0; o < m; ++o) {
       cursor[o] = pos;
-      for (int b = 0; b < count[o]; b += kTU) task[slot++] = make_int4(o, pos + b, min(kTU, count[o] - b), 0);
+      for (int b = 0; b < count[o]; b += tu) task[slot++] = make_int4(o, pos + b, min(tu, count[o] - b), 0);
       pos += count[o];
     }
     for (; slot < slot_end; ++slot) task[slot] = make_int4(0, 0, 0, 0);
@@ -215,7 +216,7 @@ bi_batch_contract_kernel(BatchParams P, int cur) {
   if (tk.z == 0) return;
   {  // stage the slice of outcome tk.x
     const R *src = (const R *)mm.logA + (size_t)tk.x * mm.P_pad;
-    for (int i = threadIdx.x * 4; i < mm.P_pad; i += kTU * 4) {
+    for (int i = threadIdx.x * 4; i < mm.P_pad; i += blockDim.x * 4) {
       Vec4<R> v = ldg4(src + i);
       *reinterpret_cast<Vec4<R> *>(L + i) = v;
     }
@@ -241,6 +242,7 @@ struct UpdateArgs {
   int32_t *argmax_out;
   int32_t T, cur, final;
   uint32_t fmask[BI_MAX_F];   // members (rank >= 2) whose group contains factor f
+  uint32_t r1mask[BI_MAX_F];  // descriptor members (modalities) that depend on factor f alone
 };
 
 template <typename R>
@@ -255,74 +257,99 @@ __device__ __forceinline__ R col_dot_g(const R *__restrict__ col, int npad, cons
   return s0 + s1;
 }
 
-template <typename R, int ALGO>
+// LW lanes per unit (the smallest power of two that holds the largest factor),
+// one lane per state: for each factor in turn the lanes gather the partial
+// messages, add the single-factor slices and the two transition messages, and
+// normalise with shuffles inside the lane group.
+struct FactorInfo {
+  int32_t n, np, op, off, U;
+  uint32_t fmask, r1mask;
+  int32_t pad_;
+};
+
+template <int LW, typename R>
+__device__ __forceinline__ R lane_group_sum(R v) {
+#pragma unroll
+  for (int o = LW / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+template <int LW, typename R>
+__device__ __forceinline__ R lane_group_max(R v) {
+#pragma unroll
+  for (int o = LW / 2; o > 0; o >>= 1) v = bi_max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+template <typename R, int ALGO, int LW>
 __global__ void __launch_bounds__(128)
 bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs A) {
-  __shared__ R ell_s[4][BI_MAX_F * BI_MAX_N];
+  __shared__ FactorInfo fi[BI_MAX_F];
   const BiDev &md = *mdp;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int unit = blockIdx.x * 4 + warp;
-  if (unit >= P.NU) return;
-  const int T = A.T, a = unit / T, t = unit - a * T;
-  const int F = md.F, Sp = md.Sp, S = md.S, M = md.M;
-  R *ell = ell_s[warp];
-  const R *qc = (const R *)P.qbuf + (size_t)A.cur * P.NU * Sp;
-  R *qn = (R *)P.qbuf + ((size_t)(A.cur ^ 1) * P.NU + unit) * Sp;
-  for (int idx = lane; idx < Sp; idx += 32) {
-    int f = 0;
-    while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
-    const int s = idx - md.offp[f], n = md.n[f], np = md.npad[f];
-    R x = (R)0;
+  constexpr int UPB = 128 / LW;   // units per CTA
+  const int F = md.F, Sp = md.Sp, S = md.S, M = md.M, T = A.T, NU = P.NU;
+  if ((int)threadIdx.x < F) {
+    const int f = threadIdx.x;
+    FactorInfo x;
+    x.n = md.n[f]; x.np = md.npad[f]; x.op = md.offp[f]; x.off = md.off[f]; x.U = md.U[f];
+    x.fmask = A.fmask[f]; x.r1mask = A.r1mask[f]; x.pad_ = 0;
+    fi[f] = x;
+  }
+  __syncthreads();
+  const int sub = threadIdx.x / LW, s = threadIdx.x % LW;
+  int unit = blockIdx.x * UPB + sub;
+  const bool live = unit < NU;    // dead groups shadow the last unit so that whole warps reach the shuffles
+  if (!live) unit = NU - 1;
+  const int a = unit / T, t = unit - a * T;
+  const R *qc = (const R *)P.qbuf + (size_t)A.cur * NU * Sp;
+  R *qn = (R *)P.qbuf + ((size_t)(A.cur ^ 1) * NU + unit) * Sp;
+  const int32_t *ob = A.obs + (size_t)unit * M;
+  // acp[f]: action into step t (t > 0); acp[F + f]: action out of it (t + 1 < T)
+  const int32_t *acp = A.act + ((ptrdiff_t)a * (T - 1) + (t - 1)) * F;
+  for (int f = 0; f < F; ++f) {
+    const FactorInfo I = fi[f];
+    const int n = I.n, np = I.np, op = I.op;
+    R x = -bi_inf<R>();
     if (s < n) {
-      for (uint32_t mk = A.fmask[f]; mk; mk &= mk - 1) {
+      x = (R)0;
+      for (uint32_t mk = I.fmask; mk; mk &= mk - 1) {
         const int j = __ffs(mk) - 1;
-        x += ((const R *)P.ellp)[((size_t)j * P.NU + unit) * Sp + idx];
+        x += ((const R *)P.ellp)[((size_t)j * NU + unit) * Sp + op + s];
       }
-      for (int gi = 0; gi < md.ngroups; ++gi) {   // single-factor modalities: the slice is the message
-        const BiGroup &gr = md.grp[gi];
-        if (gr.rank != 1 || gr.axis[0] != f) continue;
-        for (int mi = gr.mem_begin; mi < gr.mem_end; ++mi) {
-          const BiMember &mm = md.mem[mi];
-          const int o = clamp_flag(A.obs[(size_t)unit * M + mm.modality], mm.m, md.status, BI_FLAG_OBS_RANGE);
-          x += __ldg((const R *)mm.logA + (size_t)o * mm.P_pad + s);
-        }
+      for (uint32_t mk = I.r1mask; mk; mk &= mk - 1) {   // single-factor modalities: the slice is the message
+        const BiMember &mm = md.mem[__ffs(mk) - 1];
+        const int o = clamp_flag(ob[mm.modality], mm.m, md.status, BI_FLAG_OBS_RANGE);
+        x += __ldg((const R *)mm.logA + (size_t)o * mm.P_pad + s);
       }
       if (t == 0) {
         x += ((const R *)md.logD[f])[s];
       } else {
-        const int u = clamp_flag(A.act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
+        const int u = clamp_flag(acp[f], I.U, md.status, BI_FLAG_ACT_RANGE);
         const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);   // [previous][next]
-        const R v = col_dot_g<R>(M0 + (size_t)u * n * np + s, np, qc + (size_t)(unit - 1) * Sp + md.offp[f], n);
+        const R v = col_dot_g<R>(M0 + (size_t)u * n * np + s, np, qc + (size_t)(unit - 1) * Sp + op, n);
         x += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
       }
       if (t + 1 < T) {
-        const int u = clamp_flag(A.act[((size_t)a * (T - 1) + t) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
+        const int u = clamp_flag(acp[F + f], I.U, md.status, BI_FLAG_ACT_RANGE);
         const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);   // [next][previous]
-        const R v = col_dot_g<R>(M1 + (size_t)u * n * np + s, np, qc + (size_t)(unit + 1) * Sp + md.offp[f], n);
+        const R v = col_dot_g<R>(M1 + (size_t)u * n * np + s, np, qc + (size_t)(unit + 1) * Sp + op, n);
         x += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
       }
     }
-    ell[idx] = x;
-  }
-  __syncwarp();
-  float *qo = A.q_out + (size_t)unit * S;
-  float *lo = A.logq_out ? A.logq_out + (size_t)unit * S : nullptr;
-  for (int f = 0; f < F; ++f) {
-    const int n = md.n[f], op = md.offp[f];
-    const R x = lane < n ? ell[op + lane] : -bi_inf<R>();
-    const R mx = A.final ? warp_max(x) : (R)warp_max((float)x);
-    const R e = lane < n ? bi_exp_inline(x - mx) : (R)0;
-    const R z = warp_sum(e);
+    // any shift near the maximum keeps the exponentials in range; the last iterate takes the exact one
+    const R mx = A.final ? lane_group_max<LW>(x) : (R)lane_group_max<LW>((float)x);
+    const R e = s < n ? bi_exp_inline(x - mx) : (R)0;
+    const R z = lane_group_sum<LW>(e);
     const R q = e * bi_rcp(z);
-    if (lane < md.npad[f]) qn[op + lane] = lane < n ? q : (R)0;
+    if (live && s < np) qn[op + s] = q;
     if (A.final) {
-      if (lane < n) {
-        qo[md.off[f] + lane] = (float)q;
-        if (lo) lo[md.off[f] + lane] = (float)(x - mx - bi_log(z));
+      if (live && s < n) {
+        A.q_out[(size_t)unit * S + I.off + s] = (float)q;
+        if (A.logq_out) A.logq_out[(size_t)unit * S + I.off + s] = (float)(x - mx - bi_log(z));
       }
       if (A.argmax_out) {
-        const unsigned b = __ballot_sync(0xffffffffu, lane < n && x == mx);
-        if (lane == 0) A.argmax_out[(size_t)unit * F + f] = __ffs(b) - 1;
+        unsigned b = __ballot_sync(0xffffffffu, s < n && x == mx);
+        if (LW < 32) b = (b >> ((threadIdx.x & 31) - s)) & ((1u << (LW & 31)) - 1u);
+        if (live && s == 0) A.argmax_out[(size_t)unit * F + f] = __ffs(b) - 1;
       }
     }
   }
@@ -359,6 +386,10 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   const int NU = c.N * c.T;
   BatchParams P;
   memset(&P, 0, sizeof(P));
+  // units per contraction CTA: small enough that the heaviest member alone gives every SM a CTA
+  int tu = kTU;
+  while (tu > 32 && NU / tu < md->sm_count) tu >>= 1;
+  P.tu = tu;
   UpdateArgs A;
   memset(&A, 0, sizeof(A));
   // members of rank >= 2, largest slices first (their tasks are the longest)
@@ -386,7 +417,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
       A.fmask[g.axis[k]] |= 1u << j;
     }
     bm.task0 = ntask;
-    ntask += (NU + kTU - 1) / kTU + mm.m;
+    ntask += (NU + tu - 1) / tu + mm.m;
     max_slice = std::max(max_slice, (size_t)mm.P_pad * sizeof(R));
     max_m = std::max(max_m, mm.m);
   }
@@ -427,14 +458,27 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   if (cudaFuncSetAttribute((const void *)contract, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_slice) !=
       cudaSuccess)
     return BI_ERR_CUDA;
-  const int ugrid = (NU + 3) / 4;
+  for (int gi = 0; gi < h.ngroups; ++gi) {
+    const BiGroup &g = h.grp[gi];
+    if (g.rank != 1) continue;
+    for (int mi = g.mem_begin; mi < g.mem_end; ++mi) A.r1mask[g.axis[0]] |= 1u << mi;
+  }
+  int nmax = 1;
+  for (int f = 0; f < h.F; ++f) nmax = std::max(nmax, (int)h.n[f]);
+  const int lw = nmax <= 8 ? 8 : nmax <= 16 ? 16 : 32, upb = 128 / lw;
+  void (*update)(const BiDev *, BatchParams, UpdateArgs);
+  if (c.algo == BI_ALGO_VMP)
+    update = lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 8>
+                     : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 16> : bi_batch_update_kernel<R, BI_ALGO_VMP, 32>;
+  else
+    update = lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 8>
+                     : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 16> : bi_batch_update_kernel<R, BI_ALGO_MMP, 32>;
   for (int k = 0; k < c.K; ++k) {
     const int cur = k & 1;
-    contract<<<ntask, kTU, max_slice, c.stream>>>(P, cur);
+    contract<<<ntask, tu, max_slice, c.stream>>>(P, cur);
     A.cur = cur;
     A.final = (k == c.K - 1);
-    if (c.algo == BI_ALGO_VMP) bi_batch_update_kernel<R, BI_ALGO_VMP><<<ugrid, 128, 0, c.stream>>>(md->d, P, A);
-    else bi_batch_update_kernel<R, BI_ALGO_MMP><<<ugrid, 128, 0, c.stream>>>(md->d, P, A);
+    update<<<(NU + upb - 1) / upb, 128, 0, c.stream>>>(md->d, P, A);
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += 2 + 2 * c.K;
