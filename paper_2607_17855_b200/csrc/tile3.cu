@@ -13,7 +13,7 @@ template <typename R, int NA, int NB, int NC, int SB, bool LSMEM, bool STALE>
 __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p) {
   using TT = Tile3<R, NA, NB, NC, SB>;
   constexpr int LPU = TT::LPU, UPW = TT::UPW, NBL = TT::NBL, NCP = TT::NCP, NAP = TT::NAP;
-  __shared__ __align__(16) R sm_e[UPW][NB + NCP];      // gathered e_b, e_c of the current iterate
+  __shared__ __align__(16) R sm_e[UPW][NB + NCP + NAP];  // gathered e_b, e_c, e_a of the current iterate
   __shared__ __align__(16) R sm_q[UPW][NA + NB + NC];  // final beliefs of the previous step
   __shared__ __align__(16) R sm_L[LSMEM ? UPW : 1][LSMEM ? TT::P_TILE : 2];  // large tiles: the step's slice
   __shared__ __align__(16) R sm_tp[UPW][TT::TP ? TT::TP_UNIT : 2];           // transpose area of the b / c sums
@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
   const bool a_ok = t3.a_ok, b_ok = t3.b_ok, c_ok = t3.c_ok;
   const int bsafe = b_ok ? bi : 0, csafe = c_ok ? ci : 0, asafe = a_ok ? a : 0;
   R *se = sm_e[unit], *sq = sm_q[unit];
-  for (int i = t3.u; i < NB + NCP; i += LPU) se[i] = (R)0;
+  for (int i = t3.u; i < NB + NCP + NAP; i += LPU) se[i] = (R)0;
   __syncwarp();
 
   const size_t out_base = (size_t)agent * p.T;
@@ -79,14 +79,34 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
     __syncwarp();
 
     t3.set_uniform();
-    R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
+    R xa = 0, xb = 0, xc = 0;
+    // za: sum of the current iterate's e_a over the unit; with the transpose
+    // area in use every lane holds all e_a (read back from shared memory) and
+    // sums them itself, otherwise the lanes sum theirs with shuffles
+    R eav[TT::TP ? NAP : 1];
+#pragma unroll
+    for (int r = 0; r < (TT::TP ? NAP : 1); ++r) eav[r] = r < NA ? (R)1 : (R)0;
+    R za_sh = (R)NA;
     // softmax shifts in use
     float ma = STALE ? group_max_f<NAP, SB>(a_ok ? (float)lpa : -CUDART_INF_F) : 0.f;
     float mb = STALE ? group_max_f<LPU, 1>(b_ok ? (float)lpb : -CUDART_INF_F) : 0.f;
     float mc = STALE ? group_max_f<LPU, 1>(c_ok ? (float)lpc : -CUDART_INF_F) : 0.f;
     for (int k = 0; k < p.K; ++k) {
-      if (LSMEM) t3.messages_smem(sm_L[LSMEM ? unit : 0], xa, xb, xc);
-      else t3.messages(xa, xb, xc);
+      // The normalisers of the current iterate head the loop body, in one
+      // straight-line block with the contraction: their reciprocal is needed
+      // only when the messages are scaled, so its dependency chain runs under
+      // the contraction's multiply-adds instead of ahead of them.
+      {
+        const R za = TT::TP ? tree_sum<R, TT::TP ? NAP : 1>(eav) : za_sh;
+        const R zb = group_sum<R, SB, 1>(tree_sum<R, NBL>(t3.eb));
+        const R zc = tree_sum<R, NCP>(t3.ec);
+        const R rinv = bi_rcp(za * zb * zc);
+        t3.sa = rinv * za;
+        t3.sb = rinv * zb;
+        t3.sc = rinv * zc;
+      }
+      if (LSMEM) t3.messages_smem(sm_L[LSMEM ? unit : 0], xa, xb, xc, TT::TP ? eav : nullptr);
+      else t3.messages(xa, xb, xc, TT::TP ? eav : nullptr);
       xa = a_ok ? xa + lpa : -bi_inf<R>();
       xb = b_ok ? xb + lpb : -bi_inf<R>();
       xc = c_ok ? xc + lpc : -bi_inf<R>();
@@ -104,30 +124,32 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       const R ean = a_ok ? bi_exp_inline(xa - (R)ma) : (R)0;
       const R ebn = b_ok ? bi_exp_inline(xb - (R)mb) : (R)0;
       const R ecn = c_ok ? bi_exp_inline(xc - (R)mc) : (R)0;
-      float nma = ma, nmb = mb, nmc = mc;
-      if (STALE && k + 1 < p.K) {
-        nma = group_max_f<NAP, SB>((float)xa);
-        nmb = group_max_f<LPU, 1>((float)xb);
-        nmc = group_max_f<LPU, 1>((float)xc);
-      }
       if (t3.own_b) se[bi] = ebn;
       if (t3.own_c) se[NB + ci] = ecn;
-      za = group_sum<R, NAP, SB>(ean);
+      if (TT::TP && t3.own_a) se[NB + NCP + a] = ean;
+      if (!TT::TP) za_sh = group_sum<R, NAP, SB>(ean);
       __syncwarp();
       t3.ea = ean;
 #pragma unroll
       for (int bl = 0; bl < NBL; ++bl) t3.eb[bl] = se[t3.bh * NBL + bl];
 #pragma unroll
       for (int c = 0; c < NCP; ++c) t3.ec[c] = se[NB + c];
-      zb = group_sum<R, SB, 1>(tree_sum<R, NBL>(t3.eb));
-      zc = tree_sum<R, NCP>(t3.ec);
-      rinv = bi_rcp(za * zb * zc);
-      t3.sa = rinv * za;
-      t3.sb = rinv * zb;
-      t3.sc = rinv * zc;
-      if (STALE && k + 1 < p.K) { ma = nma; mb = nmb; mc = nmc; }
+      if (TT::TP) {
+#pragma unroll
+        for (int r = 0; r < NAP; ++r) eav[r] = se[NB + NCP + r];
+      }
+      if (STALE && k + 1 < p.K) {
+        ma = group_max_f<NAP, SB>((float)xa);
+        mb = group_max_f<LPU, 1>((float)xb);
+        mc = group_max_f<LPU, 1>((float)xc);
+      }
       __syncwarp();
     }
+    // normalisers of the last iterate
+    const R za = TT::TP ? tree_sum<R, TT::TP ? NAP : 1>(eav) : za_sh;
+    const R zb = group_sum<R, SB, 1>(tree_sum<R, NBL>(t3.eb));
+    const R zc = tree_sum<R, NCP>(t3.ec);
+    const R rinv = bi_rcp(za * zb * zc);
 
     // ---- final beliefs of the step: outputs, and the next step's prior input
     const R qa = t3.ea * (rinv * zb * zc);

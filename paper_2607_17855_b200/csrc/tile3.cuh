@@ -237,7 +237,7 @@ struct Tile3 {
   }
 
   // the three likelihood messages for the logits this lane owns
-  __device__ __forceinline__ void messages(R &xa, R &xb, R &xc) {
+  __device__ __forceinline__ void messages(R &xa, R &xb, R &xc, const R *eav = nullptr) {
     // V[b] = sum_c L[b][c] e_c[c] and W[c] = sum_b e_b[b] L[b][c]: independent
     // accumulators advance together so no multiply-add waits on the previous one
     R V[NBL], W[NCP];
@@ -253,12 +253,12 @@ struct Tile3 {
     for (int bl = 0; bl < NBL; ++bl)
 #pragma unroll
       for (int c = 0; c < NCP; ++c) W[c] = fma(eb[bl], L[bl][c], W[c]);
-    finish(V, W, xa, xb, xc);
+    finish(V, W, xa, xb, xc, eav);
   }
 
   // the same with the slice read from shared memory (lane-interleaved layout)
   // instead of registers: for kernels that keep many steps' slices on chip
-  __device__ __forceinline__ void messages_smem(const R *__restrict__ Ls, R &xa, R &xb, R &xc) {
+  __device__ __forceinline__ void messages_smem(const R *__restrict__ Ls, R &xa, R &xb, R &xc, const R *eav = nullptr) {
     // V[b] is accumulated in VE interleaved partial sums: consecutive elements
     // of a row would otherwise form one chain of dependent multiply-adds
     R V[NBL], W[NCP], Vp[NBL][VE];
@@ -282,30 +282,40 @@ struct Tile3 {
     }
 #pragma unroll
     for (int bl = 0; bl < NBL; ++bl) V[bl] = tree_sum<R, VE>(Vp[bl]);
-    finish(V, W, xa, xb, xc);
+    finish(V, W, xa, xb, xc, eav);
   }
 
-  __device__ __forceinline__ void finish(R (&V)[NBL], R (&W)[NCP], R &xa, R &xb, R &xc) {
-    R lav[NBL];
+  // eav: with the transpose area in use, every lane's copy of all e_a of its
+  // unit (the cross-lane sums are then dot products with it); unused otherwise
+  __device__ __forceinline__ void finish(R (&V)[NBL], R (&W)[NCP], R &xa, R &xb, R &xc, const R *eav = nullptr) {
+    R la0 = (R)0, la1 = (R)0;
 #pragma unroll
-    for (int bl = 0; bl < NBL; ++bl) lav[bl] = V[bl] * eb[bl];
-    R la = group_sum<R, SB, 1>(tree_sum<R, NBL>(lav));
+    for (int bl = 0; bl < NBL; ++bl) {
+      if (bl & 1) la1 = fma(V[bl], eb[bl], la1);
+      else la0 = fma(V[bl], eb[bl], la0);
+    }
+    R la = group_sum<R, SB, 1>(la0 + la1);
     R lb, lc;
     if (TP) {
       R *row = tp + u * TPR;
 #pragma unroll
-      for (int bl = 0; bl < NBL; ++bl) row[bl] = ea * V[bl];
+      const bool dot = eav != nullptr;   // known at compile time once inlined
+      const R wa = dot ? (R)1 : ea;      // without the copies the rows are scaled by this lane's e_a
 #pragma unroll
-      for (int c = 0; c < NCP; ++c) row[NBL + c] = ea * W[c];
+      for (int bl = 0; bl < NBL; ++bl) row[bl] = dot ? V[bl] : wa * V[bl];
+#pragma unroll
+      for (int c = 0; c < NCP; ++c) row[NBL + c] = dot ? W[c] : wa * W[c];
       __syncwarp();
-      R cb[NAP], cc[NAP];
+      R b0 = (R)0, b1 = (R)0, c0 = (R)0, c1 = (R)0;
 #pragma unroll
       for (int r = 0; r < NAP; ++r) {
-        cb[r] = tp[r * TPR + (b_ok ? u : 0)];
-        cc[r] = tp[r * TPR + NBL + (c_ok ? u : 0)];
+        const R vb = tp[r * TPR + (b_ok ? u : 0)], vc = tp[r * TPR + NBL + (c_ok ? u : 0)];
+        const R w = dot ? eav[r] : (R)1;
+        if (r & 1) { b1 = fma(w, vb, b1); c1 = fma(w, vc, c1); }
+        else { b0 = fma(w, vb, b0); c0 = fma(w, vc, c0); }
       }
-      lb = tree_sum<R, NAP>(cb);
-      lc = tree_sum<R, NAP>(cc);
+      lb = b0 + b1;
+      lc = c0 + c1;
       __syncwarp();
     } else {
       R pb[PB], pc[PC];
