@@ -183,31 +183,32 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
   float ma = 0.f, mb = 0.f, mc = 0.f, pma = 0.f, pmb = 0.f, pmc = 0.f;
   for (int k = 0; k < p.K; ++k) {
-    // transition messages from the previous iterate of the neighbouring steps
-    R ta = dprior[0], tb = dprior[1], tc = dprior[2];
-    if (t > 0) {
-      const R *qp = q_cur - SQ;
+    // Transition messages from the previous iterate of the neighbouring steps.
+    // Both edges are evaluated without branches (a window's first and last
+    // step read their halo slot, which always holds valid beliefs, and discard
+    // the result), so this code and the contraction below form one
+    // straight-line block and their dependency chains interleave.
+    R ta, tb, tc;
+    {
+      const R *qp = q_cur - SQ, *qn = q_cur + SQ;
       R va = col_dot_smem<R, NA>(pa0, p.np[0], qp);
       R vb = col_dot_smem<R, NB>(pa1, p.np[1], qp + NA);
       R vc = col_dot_smem<R, NC>(pa2, p.np[2], qp + NA + NB);
+      R wa = col_dot_smem<R, NA>(fu0, p.np[0], qn);
+      R wb = col_dot_smem<R, NB>(fu1, p.np[1], qn + NA);
+      R wc = col_dot_smem<R, NC>(fu2, p.np[2], qn + NA + NB);
       if (ALGO == BI_ALGO_MMP) {
         va = (R)0.5 * bi_log_inline(bi_max(va, (R)BI_EPS));
         vb = (R)0.5 * bi_log_inline(bi_max(vb, (R)BI_EPS));
         vc = (R)0.5 * bi_log_inline(bi_max(vc, (R)BI_EPS));
+        wa = (R)0.5 * bi_log_inline(bi_max(wa, (R)BI_EPS));
+        wb = (R)0.5 * bi_log_inline(bi_max(wb, (R)BI_EPS));
+        wc = (R)0.5 * bi_log_inline(bi_max(wc, (R)BI_EPS));
       }
-      ta = va; tb = vb; tc = vc;
-    }
-    if (t + 1 < T) {
-      const R *qn = q_cur + SQ;
-      R va = col_dot_smem<R, NA>(fu0, p.np[0], qn);
-      R vb = col_dot_smem<R, NB>(fu1, p.np[1], qn + NA);
-      R vc = col_dot_smem<R, NC>(fu2, p.np[2], qn + NA + NB);
-      if (ALGO == BI_ALGO_MMP) {
-        va = (R)0.5 * bi_log_inline(bi_max(va, (R)BI_EPS));
-        vb = (R)0.5 * bi_log_inline(bi_max(vb, (R)BI_EPS));
-        vc = (R)0.5 * bi_log_inline(bi_max(vc, (R)BI_EPS));
-      }
-      ta += va; tb += vb; tc += vc;
+      const bool has_prev = t > 0, has_next = t + 1 < T;
+      ta = (has_prev ? va : dprior[0]) + (has_next ? wa : (R)0);
+      tb = (has_prev ? vb : dprior[1]) + (has_next ? wb : (R)0);
+      tc = (has_prev ? vc : dprior[2]) + (has_next ? wc : (R)0);
     }
     if (LREG) t3.messages(xa, xb, xc);
     else t3.messages_smem(Lt, xa, xb, xc);
