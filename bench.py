@@ -316,6 +316,25 @@ def main():
                                      "frac": gbs / hbm_peak, "peak_source": hbm_src}
             others[f"config{c}_{algo}_{args.arith}"] = entry
             del r
+        # configuration 5: 128 random structures (256 agents, T=10 each), all three algorithms;
+        # aggregate = sum of updates / sum of device time, plus the per-structure spread
+        from biwl import make_sweep_config, SWEEP_SIZE
+        small_flush = torch.empty(0, dtype=torch.uint8, device="cuda")  # working sets here are below L2 anyway
+        sweep = {}
+        members = [make_sweep_config(j) for j in range(SWEEP_SIZE)]
+        for algo in ("filter", "vmp", "mmp"):
+            tot_u, tot_s, rates, kernels = 0, 0.0, [], {}
+            for wj in members:
+                r = bench_config(torch, bi, wj, algo, args.arith, 2, 1, small_flush)
+                tot_u += wj.updates
+                tot_s += r["seconds"]
+                rates.append(wj.updates / r["seconds"])
+                kernels[r["kernel"]] = kernels.get(r["kernel"], 0) + 1
+                del r
+            rates.sort()
+            sweep[algo] = {"value": tot_u / tot_s, "unit": UNIT, "min": rates[0], "median": rates[len(rates) // 2],
+                           "max": rates[-1], "ms_total": tot_s * 1e3, "kernels": kernels}
+        others[f"config5_sweep_{args.arith}"] = sweep
         line["others"] = others
         # ---- the oracle on this machine's host cores, on a bounded sample of the workload
         import oracle

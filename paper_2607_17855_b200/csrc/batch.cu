@@ -13,8 +13,11 @@
 // slice.  A second kernel per iteration adds the transition messages and takes
 // the softmax per unit (Jacobi over steps and factors, Appendix A-2).
 //
-// Compiled for the dependency-group shapes in BI_BATCH_SHAPES; other models use
-// the warp-per-step kernels.
+// The contraction has two forms: fully unrolled code for the dependency-group
+// shapes in BI_BATCH_SHAPES (every accumulator in registers), and a form for any
+// shape of rank 2..5 that is compiled only for the padded size of the last axis
+// (its accumulators in registers, those of the outer axes in per-thread columns
+// of shared memory, the outer loops an odometer shared by the whole CTA).
 #include <algorithm>
 #include <cstring>
 
@@ -37,7 +40,10 @@ constexpr int kTU = 128;   // most units per contraction CTA (the call picks 32,
 struct BatchMember {
   const void *logA;        // packed [m][P_pad]
   int32_t m, P_pad, modality, shape, rank;
-  int32_t offp[4];         // padded belief offsets of the group's axes, packed order
+  int32_t offp[BI_MAX_RANK];   // padded belief offsets of the group's axes, packed order
+  int32_t dim[BI_MAX_RANK];    // axis sizes, packed order (last one unpadded)
+  int32_t ooff[BI_MAX_RANK];   // start of each outer axis in the per-thread shared-memory columns
+  int32_t ncp, rows;       // padded last axis; rows = product of the outer axes
   int32_t task0;           // first task slot of this member
 };
 
@@ -45,6 +51,7 @@ struct BatchParams {
   BatchMember mem[BI_MAX_M];
   int32_t nmem;            // members of rank >= 2
   int32_t NU, Sp, ntask, tu;   // tu: units per contraction CTA
+  int32_t lbuf, so_max;    // any-shape form: elements of the slice staging buffer; most outer states of a member
   const int32_t *perm;     // [nmem][NU] unit ids ordered by observed outcome
   const int4 *task;        // [ntask] (outcome, first position, count, unused)
   void *ellp;              // [nmem][NU][Sp] partial likelihood messages
@@ -235,6 +242,163 @@ bi_batch_contract_kernel(BatchParams P, int cur) {
   }
 }
 
+// ---- contraction for any shape: compiled for the padded last axis only ----
+// Same arithmetic as the unrolled forms.  For a row of the slice (all outer
+// indices fixed) v = sum_c L[row][c] q_c[c] and acc_c[c] += W L[row][c], with W
+// the product of the outer beliefs.  v then climbs the outer axes from the
+// innermost: at axis j the message accumulator of index s_j receives
+// (product of the beliefs of axes before j) * v, the running sum p_{j-1}
+// receives q_j[s_j] * v, and when s_j was the axis' last index that sum becomes
+// the value handed to axis j - 1.  The indices are an odometer that is the same
+// for every thread of a warp, so its branches are uniform and a slice row is a
+// broadcast load.  qs / as: per-thread columns (state-major, thread-minor: no
+// bank conflicts) holding the outer axes' beliefs and message accumulators.
+//
+// Small batches do not have enough units to fill the machine with one thread
+// per unit, so a CTA is tu units x rs row splits: split r contracts the rows of
+// a contiguous range of the first axis' indices for the same tu units, and the
+// partial messages of the splits are added through shared memory at the end
+// (fixed order: deterministic).
+template <typename R, int NCP>
+__device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__restrict__ slice, R *Lbuf, int lbuf,
+                                            R *qs, R *as, int *unit_s, const BatchParams &P, int cur, int4 tk,
+                                            int mi) {
+  const int tid = threadIdx.x, nt = blockDim.x, tu = P.tu, rs = nt / tu;
+  const int u = tid % tu, r = tid / tu;
+  const bool has_unit = u < tk.z;
+  const int unit = has_unit ? P.perm[(size_t)mi * P.NU + tk.y + u] : 0;
+  if (r == 0) unit_s[u] = unit;
+  const R *q = (const R *)P.qbuf + ((size_t)cur * P.NU + unit) * P.Sp;
+  const int K1 = mm.rank - 1, NC = mm.dim[K1];
+  R qc[NCP], accc[NCP];
+#pragma unroll
+  for (int c = 0; c < NCP; ++c) {
+    qc[c] = (has_unit && c < NC) ? q[mm.offp[K1] + c] : (R)0;
+    accc[c] = (R)0;
+  }
+  for (int j = 0; j < K1; ++j)
+    for (int sj = 0; sj < mm.dim[j]; ++sj) {
+      qs[(mm.ooff[j] + sj) * nt + tid] = has_unit ? q[mm.offp[j] + sj] : (R)0;
+      as[(mm.ooff[j] + sj) * nt + tid] = (R)0;
+    }
+  // this split's range of the first axis, and of rows
+  const int d0 = mm.dim[0], rps = mm.rows / d0;
+  const int s0a = (int)((long long)r * d0 / rs), s0b = (int)((long long)(r + 1) * d0 / rs);
+  const int row_a = s0a * rps, row_b = s0b * rps;
+  const int most = ((d0 + rs - 1) / rs) * rps;   // rows of the largest split: the common trip count
+  int dig[4] = {s0a < d0 ? s0a : 0, 0, 0, 0};
+  R p[4] = {(R)0, (R)0, (R)0, (R)0}, Wp[4] = {(R)1, (R)1, (R)1, (R)1};
+#pragma unroll
+  for (int lv = 0; lv < 4; ++lv)
+    if (lv < K1) Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * nt + tid];
+  const int lrows = lbuf / rs / NCP;   // rows of one split's staging area
+  R *Lr = Lbuf + (size_t)r * lrows * NCP;
+  for (int c0 = 0; c0 < most; c0 += lrows) {
+    const int ra = row_a + c0;
+    const int nr = max(0, min(lrows, row_b - ra));
+    __syncthreads();   // the previous rows are consumed
+    {
+      const R *src = slice + (size_t)ra * NCP;
+      for (int i = u * 4; i < nr * NCP; i += tu * 4) *reinterpret_cast<Vec4<R> *>(Lr + i) = ldg4(src + i);
+    }
+    __syncthreads();
+    if (!has_unit) continue;
+    for (int rr = 0; rr < nr; ++rr) {
+      constexpr int VE = 16 / (int)sizeof(R);
+      const R *row = Lr + rr * NCP;
+      const R wf = K1 == 1 ? Wp[0] : K1 == 2 ? Wp[1] : K1 == 3 ? Wp[2] : Wp[3];
+      R v0 = (R)0, v1 = (R)0;
+#pragma unroll
+      for (int cc = 0; cc < NCP; cc += VE) {
+        R x[VE];
+        lds_vec(row + cc, x);
+#pragma unroll
+        for (int i = 0; i < VE; ++i) {
+          if (i & 1) v1 = fma(x[i], qc[cc + i], v1);
+          else v0 = fma(x[i], qc[cc + i], v0);
+          accc[cc + i] = fma(wf, x[i], accc[cc + i]);
+        }
+      }
+      R val = v0 + v1;
+      bool act = true;
+      int top = K1;
+#pragma unroll
+      for (int lv = 3; lv >= 0; --lv) {
+        if (lv < K1 && act) {
+          const int sj = dig[lv];
+          const int idx = (mm.ooff[lv] + sj) * nt + tid;
+          const R wprev = lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1;
+          as[idx] = fma(wprev, val, as[idx]);
+          if (lv > 0) p[lv > 0 ? lv - 1 : 0] = fma(qs[idx], val, p[lv > 0 ? lv - 1 : 0]);
+          if (sj + 1 == mm.dim[lv]) {
+            dig[lv] = 0;
+            if (lv > 0) {
+              val = p[lv > 0 ? lv - 1 : 0];
+              p[lv > 0 ? lv - 1 : 0] = (R)0;
+            }
+          } else {
+            dig[lv] = sj + 1;
+            act = false;
+          }
+          top = lv;
+        }
+      }
+      // prefix products of the outer beliefs, from the first axis whose index changed
+#pragma unroll
+      for (int lv = 0; lv < 4; ++lv)
+        if (lv < K1 && lv >= top)
+          Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * nt + tid];
+    }
+  }
+  // ---- add the splits' partial messages and write them out
+  __syncthreads();
+#pragma unroll
+  for (int c = 0; c < NCP; ++c) qs[c * nt + tid] = accc[c];   // the belief columns are no longer needed
+  __syncthreads();
+  const int so = mm.ooff[K1];   // outer states of this member
+  for (int i = tid; i < (so + NC) * tu; i += nt) {
+    const int uu = i % tu, st = i / tu;
+    if (uu >= tk.z) continue;
+    const R *col = st < so ? as + (size_t)st * nt + uu : qs + (size_t)(st - so) * nt + uu;
+    R sum = col[0];
+    for (int k = 1; k < rs; ++k) sum += col[k * tu];
+    int j = K1, base = so;   // st >= so: the last axis
+    if (st < so) {
+      j = 0;
+      while (j + 1 < K1 && st >= mm.ooff[j + 1]) ++j;
+      base = mm.ooff[j];
+    }
+    ((R *)P.ellp)[((size_t)mi * P.NU + unit_s[uu]) * P.Sp + mm.offp[j] + (st - base)] = sum;
+  }
+}
+
+template <typename R>
+__global__ void __launch_bounds__(256)
+bi_batch_contract_rt_kernel(BatchParams P, int cur) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  R *Lbuf = reinterpret_cast<R *>(smem_raw);
+  R *qs = Lbuf + P.lbuf;
+  R *as = qs + (size_t)P.so_max * blockDim.x;
+  int *unit_s = reinterpret_cast<int *>(as + (size_t)P.so_max * blockDim.x);
+  int mi = 0;
+  while (mi + 1 < P.nmem && (int)blockIdx.x >= P.mem[mi + 1].task0) ++mi;
+  const BatchMember &mm = P.mem[mi];
+  const int4 tk = P.task[blockIdx.x];
+  if (tk.z == 0) return;
+  const R *slice = (const R *)mm.logA + (size_t)tk.x * mm.P_pad;
+  switch (mm.ncp) {
+    case 4: contract_rt<R, 4>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 8: contract_rt<R, 8>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 12: contract_rt<R, 12>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 16: contract_rt<R, 16>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 20: contract_rt<R, 20>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 24: contract_rt<R, 24>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 28: contract_rt<R, 28>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 32: contract_rt<R, 32>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    default: break;
+  }
+}
+
 // ---- per unit: sum the partial messages, add rank-1 slices and transition messages, softmax ----
 struct UpdateArgs {
   const int32_t *obs, *act;
@@ -394,16 +558,18 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   memset(&A, 0, sizeof(A));
   // members of rank >= 2, largest slices first (their tasks are the longest)
   int order[BI_MAX_M], cnt = 0;
+  bool any_shape = false;   // some group has no unrolled form: every member takes the any-shape form
   for (int gi = 0; gi < h.ngroups; ++gi) {
     const BiGroup &g = h.grp[gi];
     if (g.rank < 2) continue;
-    if (g.rank > 4 || shape_of(g) < 0) return BI_ERR_UNSUPPORTED;
+    if (g.rank > BI_MAX_RANK) return BI_ERR_UNSUPPORTED;
+    if (shape_of(g) < 0) any_shape = true;
     for (int mi = g.mem_begin; mi < g.mem_end; ++mi) order[cnt++] = mi;
   }
   if (cnt == 0) return BI_ERR_UNSUPPORTED;
   std::sort(order, order + cnt, [&](int x, int y) { return h.mem[x].P_pad > h.mem[y].P_pad; });
   size_t max_slice = 0;
-  int max_m = 1, ntask = 0;
+  int max_m = 1, so_max = 1;
   for (int j = 0; j < cnt; ++j) {
     const BiMember &mm = h.mem[order[j]];
     int gi = 0;
@@ -412,16 +578,50 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     BatchMember &bm = P.mem[j];
     bm.logA = mm.logA; bm.m = mm.m; bm.P_pad = mm.P_pad; bm.modality = mm.modality;
     bm.shape = shape_of(g); bm.rank = g.rank;
+    int so = 0, rows = 1;
     for (int k = 0; k < g.rank; ++k) {
       bm.offp[k] = h.offp[g.axis[k]];
+      bm.dim[k] = g.dim[k];
+      bm.ooff[k] = so;
+      if (k + 1 < g.rank) { so += g.dim[k]; rows *= g.dim[k]; }
       A.fmask[g.axis[k]] |= 1u << j;
     }
-    bm.task0 = ntask;
-    ntask += (NU + tu - 1) / tu + mm.m;
+    bm.ncp = bi_pad4(g.dim[g.rank - 1]);
+    bm.rows = rows;
+    if ((long long)rows * bm.ncp != mm.P_pad || bm.ncp > 32) return BI_ERR_UNSUPPORTED;
+    so_max = std::max(so_max, so);
     max_slice = std::max(max_slice, (size_t)mm.P_pad * sizeof(R));
     max_m = std::max(max_m, mm.m);
   }
-  if (max_slice > (size_t)md->max_smem_optin - 1024 || max_m > 4096) return BI_ERR_UNSUPPORTED;
+  if (max_m > 4096) return BI_ERR_UNSUPPORTED;
+  // shared memory and shape of a contraction CTA
+  size_t csmem = max_slice;
+  int rs = 1;
+  if (any_shape) {
+    // row splits: enough warps for about two per scheduler when the batch is small
+    if (tu == 32) rs = NU <= 32 * 4 * md->sm_count ? 8 : 4;
+    else if (tu == 64) rs = 2;
+    // two columns per thread and outer state (at least 32 rows: the columns also carry the last
+    // axis' partial messages to the final sum), and a staging area of whole rows per split
+    // (48 KB in all at most); fewer splits, then fewer units, when that does not fit
+    P.so_max = std::max(so_max, 32);
+    for (;;) {
+      P.lbuf = (int)std::min<size_t>(max_slice / sizeof(R), 48 * 1024 / sizeof(R));
+      P.lbuf = (std::max(P.lbuf, 32 * rs) + 32 * rs - 1) / (32 * rs) * (32 * rs);
+      csmem = ((size_t)P.lbuf + 2 * (size_t)P.so_max * tu * rs) * sizeof(R) + (size_t)tu * sizeof(int);
+      if (csmem <= (size_t)md->max_smem_optin - 1024) break;
+      if (rs > 1) rs >>= 1;
+      else if (tu > 32) tu >>= 1;
+      else break;
+    }
+    P.tu = tu;
+  }
+  if (csmem > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
+  int ntask = 0;
+  for (int j = 0; j < cnt; ++j) {
+    P.mem[j].task0 = ntask;
+    ntask += (NU + tu - 1) / tu + P.mem[j].m;
+  }
   P.nmem = cnt; P.NU = NU; P.Sp = h.Sp; P.ntask = ntask;
 
   // ---- workspace (stream-ordered; kept in the handle and grown on demand)
@@ -454,8 +654,8 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
 
   bi_batch_init_kernel<R><<<256, 256, 0, c.stream>>>(md->d, (R *)P.qbuf, NU);
   bi_batch_bucket_kernel<<<cnt, 1024, 2 * max_m * sizeof(int32_t), c.stream>>>(P, c.obs, h.M, h.status, perm, task);
-  auto contract = bi_batch_contract_kernel<R>;
-  if (cudaFuncSetAttribute((const void *)contract, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_slice) !=
+  void (*contract)(BatchParams, int) = any_shape ? bi_batch_contract_rt_kernel<R> : bi_batch_contract_kernel<R>;
+  if (cudaFuncSetAttribute((const void *)contract, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csmem) !=
       cudaSuccess)
     return BI_ERR_CUDA;
   for (int gi = 0; gi < h.ngroups; ++gi) {
@@ -475,7 +675,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
                      : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 16> : bi_batch_update_kernel<R, BI_ALGO_MMP, 32>;
   for (int k = 0; k < c.K; ++k) {
     const int cur = k & 1;
-    contract<<<ntask, tu, max_slice, c.stream>>>(P, cur);
+    contract<<<ntask, tu * rs, csmem, c.stream>>>(P, cur);
     A.cur = cur;
     A.final = (k == c.K - 1);
     update<<<(NU + upb - 1) / upb, 128, 0, c.stream>>>(md->d, P, A);

@@ -298,7 +298,6 @@ struct Tile3 {
     R lb, lc;
     if (TP) {
       R *row = tp + u * TPR;
-#pragma unroll
       const bool dot = eav != nullptr;   // known at compile time once inlined
       const R wa = dot ? (R)1 : ea;      // without the copies the rows are scaled by this lane's e_a
 #pragma unroll

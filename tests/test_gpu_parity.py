@@ -221,3 +221,22 @@ def test_batched_window_kernels(algo):
     assert res["kernel"] == f"batch_{algo}_f64", res
     res = check_workload(make_config(3, N=160, T=13, K=5), algo, arith="f32", strict=False)
     assert res["kernel"] == f"batch_{algo}_f32", res
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_batched_any_shape(algo):
+    # rank 5 with a two-state last axis (padded to 4); last axes of 7, 13 and 32 states; a slice of
+    # 20 x 20 x 20 that is staged in several pieces; a single-factor modality
+    w = _custom(43, [3, 4, 5, 3, 2], [3, 4, 2], [[0, 1, 2, 3, 4], [1, 2], [3]], [2, 1, 2, 3, 1],
+                N=150, T=14, K=6, sparsity=0.5)
+    res = check_workload(w, algo, agents=range(0, 150, 6))
+    assert res["kernel"] == f"batch_{algo}_f64", res
+    w = _custom(44, [7, 13, 32, 9], [5, 3, 2, 6], [[0, 1], [1, 2], [0, 3, 2], [3, 0]], [2, 2, 1, 3],
+                N=128, T=16, K=5)
+    res = check_workload(w, algo, agents=range(0, 128, 5))
+    assert res["kernel"] == f"batch_{algo}_f64", res
+    w = _custom(45, [20, 20, 20], [3, 2], [[0, 1, 2], [2, 0]], [1, 2, 2], N=129, T=16, K=4, sparsity=0.9)
+    res = check_workload(w, algo, agents=range(0, 129, 8), conditioned=True)
+    assert res["kernel"] == f"batch_{algo}_f64", res
+    res = check_workload(w, algo, arith="f32", strict=False)
+    assert res["kernel"] == f"batch_{algo}_f32", res
