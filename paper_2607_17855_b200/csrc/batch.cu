@@ -566,7 +566,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     if (shape_of(g) < 0) any_shape = true;
     for (int mi = g.mem_begin; mi < g.mem_end; ++mi) order[cnt++] = mi;
   }
-  if (cnt == 0) return BI_ERR_UNSUPPORTED;
+  // (cnt == 0: every modality depends on a single factor; the update kernel alone does the work)
   std::sort(order, order + cnt, [&](int x, int y) { return h.mem[x].P_pad > h.mem[y].P_pad; });
   size_t max_slice = 0;
   int max_m = 1, so_max = 1;
@@ -653,7 +653,8 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   A.T = c.T;
 
   bi_batch_init_kernel<R><<<256, 256, 0, c.stream>>>(md->d, (R *)P.qbuf, NU);
-  bi_batch_bucket_kernel<<<cnt, 1024, 2 * max_m * sizeof(int32_t), c.stream>>>(P, c.obs, h.M, h.status, perm, task);
+  if (cnt > 0)
+    bi_batch_bucket_kernel<<<cnt, 1024, 2 * max_m * sizeof(int32_t), c.stream>>>(P, c.obs, h.M, h.status, perm, task);
   void (*contract)(BatchParams, int) = any_shape ? bi_batch_contract_rt_kernel<R> : bi_batch_contract_kernel<R>;
   if (cudaFuncSetAttribute((const void *)contract, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csmem) !=
       cudaSuccess)
@@ -675,13 +676,13 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
                      : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 16> : bi_batch_update_kernel<R, BI_ALGO_MMP, 32>;
   for (int k = 0; k < c.K; ++k) {
     const int cur = k & 1;
-    contract<<<ntask, tu * rs, csmem, c.stream>>>(P, cur);
+    if (cnt > 0) contract<<<ntask, tu * rs, csmem, c.stream>>>(P, cur);
     A.cur = cur;
     A.final = (k == c.K - 1);
     update<<<(NU + upb - 1) / upb, 128, 0, c.stream>>>(md->d, P, A);
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
-  mut->launches += 2 + 2 * c.K;
+  mut->launches += cnt > 0 ? 2 + 2 * c.K : 1 + c.K;
   const bool f64 = sizeof(R) == 8;
   mut->last_kernel = c.algo == BI_ALGO_VMP ? (f64 ? "batch_vmp_f64" : "batch_vmp_f32")
                                            : (f64 ? "batch_mmp_f64" : "batch_mmp_f32");

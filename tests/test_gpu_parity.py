@@ -240,3 +240,11 @@ def test_batched_any_shape(algo):
     assert res["kernel"] == f"batch_{algo}_f64", res
     res = check_workload(w, algo, arith="f32", strict=False)
     assert res["kernel"] == f"batch_{algo}_f32", res
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_batched_single_factor_modalities_only(algo):
+    # no contraction at all: the observed slices are the messages
+    w = _custom(46, [5, 9], [4, 3, 6], [[0], [1], [0]], [2, 3], N=150, T=14, K=5)
+    res = check_workload(w, algo, agents=range(0, 150, 4))
+    assert res["kernel"] == f"batch_{algo}_f64", res
