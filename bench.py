@@ -37,7 +37,7 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # 74.4
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the benchmark's
 # workload, from the ncu captures summarised under profiles/ (bytes)
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "tile3_filter_f64": 5.01e6 + 3.6e3,   # profiles/tile3_filter_f64_config2.md
+    "tile3_filter_f64": 5.01e6 + 4.1e3,   # profiles/tile3_filter_f64_config2.md
 }
 
 
@@ -316,10 +316,20 @@ def main():
                                      "frac": gbs / hbm_peak, "peak_source": hbm_src}
             others[f"config{c}_{algo}_{args.arith}"] = entry
             del r
+        # configuration 1 (8 agents, 0.5 KB working set): latency per call, beside a one-element fill
+        # kernel timed the same way (what a launch alone costs here)
+        w1 = make_config(1)
+        small_flush = torch.empty(0, dtype=torch.uint8, device="cuda")  # nothing to flush: below L2 anyway
+        r = bench_config(torch, bi, w1, "filter", args.arith, 20, 3, small_flush)
+        one = torch.empty(1, device="cuda")
+        null_times = time_steps(lambda: one.zero_(), 20, 3, small_flush, torch)
+        others[f"config1_filter_{args.arith}"] = {"us_per_call": r["seconds"] * 1e6, "kernel": r["kernel"],
+                                                  "one_element_fill_us": sum(null_times) / len(null_times) * 1e6,
+                                                  "value": w1.updates / r["seconds"], "unit": UNIT}
+        del r
         # configuration 5: 128 random structures (256 agents, T=10 each), all three algorithms;
         # aggregate = sum of updates / sum of device time, plus the per-structure spread
         from biwl import make_sweep_config, SWEEP_SIZE
-        small_flush = torch.empty(0, dtype=torch.uint8, device="cuda")  # working sets here are below L2 anyway
         sweep = {}
         members = [make_sweep_config(j) for j in range(SWEEP_SIZE)]
         for algo in ("filter", "vmp", "mmp"):

@@ -70,6 +70,8 @@ enum {
 /* bits of the device status word read by bi_status */
 #define BI_FLAG_OBS_RANGE 1u /* an observation index was outside [0, m_i): clamped */
 #define BI_FLAG_ACT_RANGE 2u /* an action index was outside [0, U_f): clamped      */
+#define BI_FLAG_COPY_TIMEOUT 4u /* an asynchronous copy inside a kernel did not complete within its
+                                   probe limit: the CTA left early and the call's outputs are invalid */
 
 typedef struct bi_model bi_model_t; /* opaque; owns the packed device copies */
 

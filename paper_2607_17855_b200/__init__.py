@@ -21,6 +21,7 @@ ERRORS = {0: "BI_OK", -1: "BI_ERR_INVALID_ARG", -2: "BI_ERR_SHAPE", -3: "BI_ERR_
           -4: "BI_ERR_ALLOC", -5: "BI_ERR_CUDA"}
 BI_FLAG_OBS_RANGE = 1
 BI_FLAG_ACT_RANGE = 2
+BI_FLAG_COPY_TIMEOUT = 4
 
 BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1

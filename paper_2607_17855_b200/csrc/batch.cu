@@ -56,6 +56,7 @@ struct BatchParams {
   const int4 *task;        // [ntask] (outcome, first position, count, unused)
   void *ellp;              // [nmem][NU][Sp] partial likelihood messages
   void *qbuf;              // [2][NU][Sp] beliefs
+  uint32_t *status;        // the handle's status word
 };
 
 // ---- one unit against one slice: every message of the group in one pass ----
@@ -221,18 +222,22 @@ bi_batch_contract_kernel(BatchParams P, int cur) {
   const BatchMember &mm = P.mem[mi];
   const int4 tk = P.task[blockIdx.x];
   if (tk.z == 0) return;
-  {  // stage the slice of outcome tk.x
-    const R *src = (const R *)mm.logA + (size_t)tk.x * mm.P_pad;
-    for (int i = threadIdx.x * 4; i < mm.P_pad; i += blockDim.x * 4) {
-      Vec4<R> v = ldg4(src + i);
-      *reinterpret_cast<Vec4<R> *>(L + i) = v;
-    }
-  }
+  // stage the slice of outcome tk.x: one bulk asynchronous copy, global -> shared, issued by one
+  // thread; the others meanwhile look up their unit
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x == 0) bi_mbar_init(&bar, 1);
   __syncthreads();
-  if ((int)threadIdx.x >= tk.z) return;
-  const int unit = P.perm[(size_t)mi * P.NU + tk.y + threadIdx.x];
+  if (threadIdx.x == 0)
+    bi_bulk_load(L, (const R *)mm.logA + (size_t)tk.x * mm.P_pad, (uint32_t)(mm.P_pad * sizeof(R)), &bar);
+  const bool has_unit = (int)threadIdx.x < tk.z;
+  const int unit = has_unit ? P.perm[(size_t)mi * P.NU + tk.y + threadIdx.x] : 0;
   const R *q = (const R *)P.qbuf + ((size_t)cur * P.NU + unit) * P.Sp;
   R *out = (R *)P.ellp + ((size_t)mi * P.NU + unit) * P.Sp;
+  if (!bi_mbar_wait(&bar, 0)) {
+    if (threadIdx.x == 0) atomicOr(P.status, BI_FLAG_COPY_TIMEOUT);
+    return;
+  }
+  if (!has_unit) return;
   switch (mm.shape) {
 #define X(ID, RANK, D0, D1, D2, D3) \
   case ID: contract_shape<R, RANK, D0, D1, D2, D3>(L, q, out, mm.offp); break;
@@ -293,16 +298,24 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
     if (lv < K1) Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * nt + tid];
   const int lrows = lbuf / rs / NCP;   // rows of one split's staging area
   R *Lr = Lbuf + (size_t)r * lrows * NCP;
+  __shared__ __align__(8) unsigned long long bar[8];   // one per split
+  if (tid < rs) bi_mbar_init(&bar[tid], 1);
+  uint32_t phase = 0;
+  bool failed = false;
   for (int c0 = 0; c0 < most; c0 += lrows) {
     const int ra = row_a + c0;
     const int nr = max(0, min(lrows, row_b - ra));
     __syncthreads();   // the previous rows are consumed
-    {
-      const R *src = slice + (size_t)ra * NCP;
-      for (int i = u * 4; i < nr * NCP; i += tu * 4) *reinterpret_cast<Vec4<R> *>(Lr + i) = ldg4(src + i);
+    if (nr > 0) {
+      // this split's rows: one bulk asynchronous copy issued by the split's first thread
+      if (u == 0) bi_bulk_load(Lr, slice + (size_t)ra * NCP, (uint32_t)(nr * NCP * sizeof(R)), &bar[r]);
+      if (!bi_mbar_wait(&bar[r], phase)) {
+        if (u == 0) atomicOr(P.status, BI_FLAG_COPY_TIMEOUT);
+        failed = true;
+      }
+      phase ^= 1u;
     }
-    __syncthreads();
-    if (!has_unit) continue;
+    if (!has_unit || failed) continue;
     for (int rr = 0; rr < nr; ++rr) {
       constexpr int VE = 16 / (int)sizeof(R);
       const R *row = Lr + rr * NCP;
@@ -649,6 +662,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   P.task = task;
   P.ellp = w + b_perm + b_task;
   P.qbuf = w + b_perm + b_task + b_ellp;
+  P.status = h.status;
   A.obs = c.obs; A.act = c.act; A.q_out = c.q_out; A.logq_out = c.logq_out; A.argmax_out = c.argmax_out;
   A.T = c.T;
 

@@ -126,3 +126,42 @@ __device__ __forceinline__ int clamp_flag(int v, int hi, uint32_t *status, uint3
   }
   return v;
 }
+
+// ---- bulk asynchronous copy, global -> shared, completed on an mbarrier ----
+// (the copy engine's untiled form: cp.async.bulk; both addresses 16-byte
+// aligned, the size a multiple of 16 bytes, no multicast)
+__device__ __forceinline__ uint32_t bi_smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void bi_mbar_init(unsigned long long *bar, int arrivals) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bi_smem_addr(bar)), "r"(arrivals) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// one thread: announce `bytes` on the barrier (its one arrival) and start the copy
+__device__ __forceinline__ void bi_bulk_load(void *dst_smem, const void *src_global, uint32_t bytes,
+                                             unsigned long long *bar) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bi_smem_addr(bar)), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   bi_smem_addr(dst_smem)),
+               "l"(src_global), "r"(bytes), "r"(bi_smem_addr(bar))
+               : "memory");
+}
+
+// Waits for the barrier's phase of the given parity with a bounded number of
+// probes; false when the limit ran out (the caller raises a status flag and
+// leaves: nothing here spins without an end).
+__device__ __forceinline__ bool bi_mbar_wait(unsigned long long *bar, uint32_t parity, int limit = 1 << 18) {
+  for (int i = 0; i < limit; ++i) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bi_smem_addr(bar)), "r"(parity)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
