@@ -57,12 +57,15 @@ def _ptr_array(arrs):
 
 def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G: int,
         A, B, D, obs: np.ndarray, act: Optional[np.ndarray], K: int, *,
-        q_init: Optional[np.ndarray] = None, threads: int = 0, round32: bool = False):
+        q_init: Optional[np.ndarray] = None, threads: int = 0, round32: bool = False,
+        q_prev: Optional[np.ndarray] = None, act_prev: Optional[np.ndarray] = None):
     """Run ``algo`` ('filter' | 'vmp' | 'mmp') and return ``(q, logq, argmax)``.
 
     ``obs`` is ``[N, T, M]`` int32, ``act`` ``[N, T-1, F]`` int32 (ignored when
     T == 1); ``q`` and ``logq`` come back as float64 ``[N, T, S]``, ``argmax`` as
-    int32 ``[N, T, F]``.
+    int32 ``[N, T, F]``.  ``q_prev`` ``[N, S]`` with ``act_prev`` ``[N, F]``
+    (filtering only) continue a stream: the first step's prior is
+    ``B_u q_prev`` instead of ``D``.
     """
     lib = _load()
     n = np.ascontiguousarray(n, dtype=np.int32)
@@ -96,6 +99,24 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
         q_init = np.ascontiguousarray(q_init, dtype=np.float64)
         assert q_init.shape == (N, T, S)
     Ap, Bp, Dp = _ptr_array(A), _ptr_array(B), _ptr_array(D)
+    if q_prev is not None or act_prev is not None:
+        assert algo == "filter" and q_init is None and not round32
+        q_prev = np.ascontiguousarray(q_prev, dtype=np.float64)
+        act_prev = np.ascontiguousarray(act_prev, dtype=np.int32)
+        assert q_prev.shape == (N, S) and act_prev.shape == (N, F)
+        rc = lib.bi_ref_filter_from(
+            ctypes.c_int(F), ctypes.c_int(M),
+            ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),
+            ctypes.c_void_p(dep_len.ctypes.data), ctypes.c_void_p(dep_flat.ctypes.data),
+            ctypes.c_void_p(U.ctypes.data), ctypes.c_int(G), Ap, Bp, Dp,
+            ctypes.c_int(N), ctypes.c_int(T), ctypes.c_void_p(obs.ctypes.data),
+            ctypes.c_void_p(act_p), ctypes.c_int(K),
+            ctypes.c_void_p(q_prev.ctypes.data), ctypes.c_void_p(act_prev.ctypes.data),
+            ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(lq.ctypes.data),
+            ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads))
+        if rc != 0:
+            raise ValueError(f"bi_ref_filter_from rejected its arguments (code {rc})")
+        return q, lq, am
     rc = lib.bi_ref_run(
         ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),
         ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),

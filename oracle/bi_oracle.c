@@ -151,8 +151,12 @@ static void set_initial(const model_t *md, const double *q_init, double *q)
 }
 
 /* ---- variational filtering (FPI) for one agent ------------------------- */
+/* q_prev / act_prev (both NULL, or both given): the belief of the step before the
+ * window, [S], and the action taken at that step, [F]; the first step's prior is
+ * then B_u q_prev, the same recursion as every later step, instead of D. */
 static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *obs,
-                         const int32_t *act, const double *q_init, double *q_out,
+                         const int32_t *act, const double *q_init, const double *q_prev,
+                         const int32_t *act_prev, double *q_out,
                          double *lq_out, int32_t *am_out)
 {
     int S = md->S, F = md->F;
@@ -166,11 +170,11 @@ static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *
             int nf = md->n[f], o = md->off[f];
             for (int s = 0; s < nf; ++s) {
                 double p;
-                if (t == 0) {
+                if (t == 0 && !q_prev) {
                     p = (double)md->D[f][(size_t)g * nf + s];
                 } else {
-                    int u = act[(size_t)(t - 1) * F + f];
-                    const double *qp = q_out + (size_t)(t - 1) * S + o;
+                    int u = t == 0 ? act_prev[f] : act[(size_t)(t - 1) * F + f];
+                    const double *qp = t == 0 ? q_prev + o : q_out + (size_t)(t - 1) * S + o;
                     p = 0.0;
                     for (int r = 0; r < nf; ++r) p += B_at(md, g, f, u, s, r) * qp[r];
                 }
@@ -267,14 +271,16 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
  * OpenMP default; agents are independent, so threading is over agents only.
  * Returns 0, or a negative value for an invalid argument.
  */
-int bi_ref_run(int algo, int F, int M, const int32_t *n, const int32_t *m,
-               const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
-               const float *const *A, const float *const *B, const float *const *D,
-               int N, int T, const int32_t *obs, const int32_t *act, int K,
-               const double *q_init, double *q_out, double *logq_out,
-               int32_t *argmax_out, int threads, int round32)
+static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
+                    const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+                    const float *const *A, const float *const *B, const float *const *D,
+                    int N, int T, const int32_t *obs, const int32_t *act, int K,
+                    const double *q_init, const double *q_prev, const int32_t *act_prev,
+                    double *q_out, double *logq_out,
+                    int32_t *argmax_out, int threads, int round32)
 {
     if (algo < 0 || algo > 2 || F < 1 || M < 0 || N < 0 || T < 1 || K < 1) return -1;
+    if ((q_prev != NULL) != (act_prev != NULL) || (q_prev && algo != ALGO_FILTER)) return -1;
     if (!(G == 1 || G == N)) return -1;
     model_t md;
     md.F = F; md.M = M; md.G = G; md.n = n; md.m = m; md.dep_len = dep_len; md.dep = dep;
@@ -312,11 +318,43 @@ int bi_ref_run(int algo, int F, int M, const int32_t *n, const int32_t *m,
         double *qo = q_out + (size_t)a * T * S;
         double *lo = logq_out ? logq_out + (size_t)a * T * S : NULL;
         int32_t *ao = argmax_out ? argmax_out + (size_t)a * T * F : NULL;
-        if (algo == ALGO_FILTER) filter_agent(&md, g, T, K, ob, ac, qi, qo, lo, ao);
+        if (algo == ALGO_FILTER)
+            filter_agent(&md, g, T, K, ob, ac, qi, q_prev ? q_prev + (size_t)a * S : NULL,
+                         act_prev ? act_prev + (size_t)a * F : NULL, qo, lo, ao);
         else window_agent(&md, algo, g, T, K, ob, ac, qi, qo, lo, ao);
     }
     free(md.off); free(md.dep_off); free(md.P);
     return 0;
+}
+
+int bi_ref_run(int algo, int F, int M, const int32_t *n, const int32_t *m,
+               const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+               const float *const *A, const float *const *B, const float *const *D,
+               int N, int T, const int32_t *obs, const int32_t *act, int K,
+               const double *q_init, double *q_out, double *logq_out,
+               int32_t *argmax_out, int threads, int round32)
+{
+    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, act, K, q_init, NULL, NULL,
+                    q_out, logq_out, argmax_out, threads, round32);
+}
+
+/*
+ * Filtering continued from a known belief: q_prev [N][S] is every agent's belief
+ * at the step before the window and act_prev [N][F] the action taken there, so
+ * the first step's prior is B_u q_prev (the recursion of Section III-B entered
+ * mid-stream) instead of D.  Everything else as bi_ref_run with the filtering
+ * algorithm.
+ */
+int bi_ref_filter_from(int F, int M, const int32_t *n, const int32_t *m,
+                       const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+                       const float *const *A, const float *const *B, const float *const *D,
+                       int N, int T, const int32_t *obs, const int32_t *act, int K,
+                       const double *q_prev, const int32_t *act_prev,
+                       double *q_out, double *logq_out, int32_t *argmax_out, int threads)
+{
+    if (!q_prev || !act_prev) return -1;
+    return run_impl(ALGO_FILTER, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, act, K, NULL, q_prev,
+                    act_prev, q_out, logq_out, argmax_out, threads, 0);
 }
 
 int bi_ref_max_threads(void)

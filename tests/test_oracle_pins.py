@@ -313,3 +313,40 @@ def test_zero_probabilities_use_the_clamped_log():
     want = np.array([1e-16, 0.5]) / (1e-16 + 0.5)
     np.testing.assert_allclose(q[0, 0], want, rtol=1e-12)
     assert np.isfinite(lq).all()
+
+
+# ---- filtering continued from a known belief (the recursion entered mid-stream) ----
+
+def test_filter_continuation_equals_the_uninterrupted_run():
+    w = tiny(61, [4, 3, 2], [3, 4], [[0, 1], [1, 2, 0]], [2, 3, 1], T=9, N=3, sparsity=0.5)
+    q, lq, am = run("filter", w, 5)
+    for cut in (1, 4, 8):
+        head = dict(w, obs=w["obs"][:, :cut], act=w["act"][:, :cut - 1])
+        tail = dict(w, obs=w["obs"][:, cut:], act=w["act"][:, cut:])
+        qh, _, _ = run("filter", head, 5)
+        np.testing.assert_array_equal(qh, q[:, :cut])
+        qt, lqt, amt = run("filter", tail, 5, q_prev=qh[:, -1], act_prev=w["act"][:, cut - 1])
+        np.testing.assert_array_equal(qt, q[:, cut:])
+        np.testing.assert_array_equal(lqt, lq[:, cut:])
+        np.testing.assert_array_equal(amt, am[:, cut:])
+
+
+def test_single_factor_continuation_is_one_bayes_step():
+    # softmax(ln A[o] + ln(B_u q_prev)), written out directly
+    w = tiny(62, [5], [4], [[0]], [3], T=1, N=4)
+    rng = np.random.default_rng(7)
+    q_prev = rng.dirichlet(np.ones(5), size=4)
+    act_prev = rng.integers(0, 3, size=(4, 1)).astype(np.int32)
+    q, lq, _ = run("filter", w, 3, q_prev=q_prev, act_prev=act_prev)
+    A, B = w["A"][0][0].astype(np.float64), w["B"][0][0].astype(np.float64)
+    for a in range(4):
+        post = A[w["obs"][a, 0, 0]] * (B[:, :, act_prev[a, 0]] @ q_prev[a])
+        post /= post.sum()
+        np.testing.assert_allclose(q[a, 0], post, atol=1e-14)
+        np.testing.assert_allclose(lq[a, 0], np.log(post), atol=1e-12)
+
+
+def test_continuation_arguments_are_checked():
+    w = tiny(63, [3], [2], [[0]], [2], T=2)
+    with pytest.raises((ValueError, AssertionError)):
+        run("vmp", w, 2, q_prev=np.full((1, 3), 1 / 3), act_prev=np.zeros((1, 1), np.int32))
