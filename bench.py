@@ -28,6 +28,7 @@ sys.path.insert(0, ROOT)
 METRIC = "belief_updates_per_sec"
 UNIT = "updates/s"
 HEADLINE = 2  # configuration the metric is quoted on
+E2E_CHUNKS = 5  # the end-to-end run filters the trajectory in this many consecutive blocks of steps
 
 # Nominal ALU peaks derived from the unit counts: 148 SMs x lanes x 2 flops x 1.965 GHz.
 FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12   # 37.2
@@ -256,25 +257,73 @@ def main():
     sec = max_over_ranks(dist, sec, "cuda")
     value = aggregate_throughput(w.updates, world, sec)
 
-    # ---- end to end: pinned host inputs -> device -> bi_filter -> host beliefs
+    # ---- end to end: pinned host inputs -> device -> filtering -> host beliefs.  The trajectory is
+    # run as E2E_CHUNKS consecutive blocks of steps (bi_filter, then bi_filter_from continuing from the
+    # previous block's last belief), so a block's beliefs travel to the host while the next block runs.
     md, q = head["model"], head["q"]
-    h_obs = torch.from_numpy(w.obs).pin_memory()
-    h_act = torch.from_numpy(w.act).pin_memory()
-    h_q = torch.empty(q.shape, dtype=torch.float32).pin_memory()
-    d_obs, d_act = head["obs"], head["act"]
+    nchunk = E2E_CHUNKS if w.T % E2E_CHUNKS == 0 else 1
+    tc = w.T // nchunk
+    copy_out, copy_in = torch.cuda.Stream(), torch.cuda.Stream()
+    # host inputs block by block, packed into two pinned buffers (the first block; the rest) so that each
+    # reaches the device in one copy: the second one while the first block is being filtered
+    parts = []
+    for i in range(nchunk):
+        t0 = i * tc
+        parts.append([np.ascontiguousarray(w.obs[:, t0:t0 + tc]), np.ascontiguousarray(w.act[:, t0:t0 + tc - 1]),
+                      np.ascontiguousarray(w.act[:, t0 - 1]) if i else np.empty((w.N, 0), np.int32)])
+    def pack(blocks):
+        flat = np.concatenate([x.reshape(-1) for blk in blocks for x in blk]) if blocks else np.empty(0, np.int32)
+        return torch.from_numpy(flat.astype(np.int32)).pin_memory()
+    h_first, h_rest = pack(parts[:1]), pack(parts[1:])
+    d_first = torch.empty(h_first.shape, dtype=torch.int32, device="cuda")
+    d_rest = torch.empty(h_rest.shape, dtype=torch.int32, device="cuda")
+    d_in = []
+    for i, blk in enumerate(parts):
+        buf, pos, views = (d_first, 0, []) if i == 0 else (d_rest, d_in[-1][3] if i > 1 else 0, [])
+        for x in blk:
+            views.append(buf[pos:pos + x.size].view(x.shape))
+            pos += x.size
+        d_in.append((views[0], views[1], views[2], pos))
+    d_q = [torch.empty((w.N, tc, w.S), dtype=torch.float32, device="cuda") for _ in range(nchunk)]
+    h_q = [torch.empty((w.N, tc, w.S), dtype=torch.float32).pin_memory() for _ in range(nchunk)]
+    done = [torch.cuda.Event() for _ in range(nchunk)]
+    arrived = torch.cuda.Event()
+    q_prev = torch.empty((w.N, w.S), dtype=torch.float32, device="cuda")
 
     def e2e_step():
-        d_obs.copy_(h_obs, non_blocking=True)
-        d_act.copy_(h_act, non_blocking=True)
-        md.bi_filter(d_obs, d_act, w.K, q_out=q)
-        h_q.copy_(q, non_blocking=True)
+        cur = torch.cuda.current_stream()
+        copy_in.wait_stream(cur)
+        d_first.copy_(h_first, non_blocking=True)
+        with torch.cuda.stream(copy_in):
+            d_rest.copy_(h_rest, non_blocking=True)
+            arrived.record(copy_in)
+        for i in range(nchunk):
+            obs_i, act_i, actp_i, _ = d_in[i]
+            if i == 0:
+                md.bi_filter(obs_i, act_i, w.K, q_out=d_q[0])
+            else:
+                if i == 1:
+                    cur.wait_event(arrived)
+                q_prev.copy_(d_q[i - 1][:, -1])
+                md.bi_filter_from(obs_i, act_i, q_prev, actp_i, w.K, q_out=d_q[i])
+            done[i].record(cur)
+            copy_out.wait_event(done[i])
+            with torch.cuda.stream(copy_out):
+                h_q[i].copy_(d_q[i], non_blocking=True)
+        cur.wait_stream(copy_out)   # the step ends when the last block has reached the host
 
     e2e_times = time_steps(e2e_step, max(3, args.steps // 2), 3, flush, torch)
     e2e_sec = sum(e2e_times) / len(e2e_times)
     clocks = sampler.stop()  # sampled over both timed regions
     e2e_sec = max_over_ranks(dist, e2e_sec, "cuda")
+    # the blockwise result against the single call's (continuing from float32 beliefs re-rounds the
+    # carried state once per block; the iteration amplifies that on ill-conditioned agents)
+    torch.cuda.synchronize()
+    diff = (torch.cat(h_q, dim=1) - q.cpu()).abs().reshape(w.N, -1).max(dim=1).values
+    blocks_agree = float((diff <= 1e-5).float().mean())
     e2e = {"value": aggregate_throughput(w.updates, world, e2e_sec), "unit": UNIT,
-           "h2d_bytes_per_step": int(w.obs.nbytes + w.act.nbytes), "d2h_bytes_per_step": int(q.numel() * 4)}
+           "h2d_bytes_per_step": int(w.obs.nbytes + w.act.nbytes), "d2h_bytes_per_step": int(q.numel() * 4),
+           "blocks_of_steps": nchunk, "agents_within_1e-5_of_single_call": blocks_agree}
 
     flops = algorithmic_flops(w)
     peak = FP64_PEAK_TFLOPS if args.arith == "f64" else FP32_PEAK_TFLOPS

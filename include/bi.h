@@ -162,6 +162,29 @@ int bi_mmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
            int32_t *argmax_out, void *cuda_stream);
 
 /*
+ * Variational filtering continued from a known belief: the recursion of
+ * bi_filter (Section III-B: prior of a step = B_u applied to the previous
+ * step's belief) entered mid-stream.  For an agent that receives its
+ * observations over time -- one call per tick, or per block of ticks -- and
+ * for splitting a long trajectory into pieces whose results can be copied out
+ * while the next piece runs.
+ *   q_prev    DEVICE [N][S] float32: each agent's belief at the step before this
+ *             window (normally the last step of the previous call's q_out)
+ *   act_prev  DEVICE [N][F] int32: the action taken at that step, u in [0, U_f)
+ *   others    as for bi_filter (act is [N][T-1][F]; may be NULL when T == 1)
+ * The first step's prior is B_{act_prev} q_prev instead of D; everything else is
+ * bi_filter.  Because q_prev carries float32 rounding, a split run equals the
+ * uninterrupted one only up to that rounding (and to what the iteration makes of
+ * it).  Each agent's q_prev row is read before that agent's outputs are written,
+ * so with T == 1 q_prev and q_out may be the same buffer (an in-place tick).
+ * Returns BI_ERR_INVALID_ARG when q_prev or act_prev is NULL.
+ */
+int bi_filter_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                   const int32_t *act, const float *q_prev, const int32_t *act_prev,
+                   int32_t iters, float *q_out, float *logq_out, int32_t *argmax_out,
+                   void *cuda_stream);
+
+/*
  * Variational filtering without any allocation.  (The paper has no counterpart
  * to this entry point: it is a deployment convenience of this library.)
  *

@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_vmp", "bi_mmp", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -65,6 +65,10 @@ def lib():
             fn.restype = ctypes.c_int
             fn.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                            ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.bi_filter_from.restype = ctypes.c_int
+        L.bi_filter_from.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.bi_status.restype = ctypes.c_int
         L.bi_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
         L.bi_last_kernel.restype = ctypes.c_char_p
@@ -164,6 +168,25 @@ class Model:
     def bi_filter(self, obs, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
         """Variational filtering; ``obs`` int32 ``[N,T,M]``, ``act`` int32 ``[N,T-1,F]`` (CUDA)."""
         return self._run("bi_filter", obs, act, iters, q_out, logq_out, argmax_out, stream)
+
+    def bi_filter_from(self, obs, act, q_prev, act_prev, iters, q_out=None, logq_out=None, argmax_out=None,
+                       stream=None):
+        """Filtering continued from ``q_prev`` float32 ``[N,S]`` (the belief of the step before
+        this window) and ``act_prev`` int32 ``[N,F]`` (the action taken there)."""
+        import torch
+        N, T = int(obs.shape[0]), int(obs.shape[1])
+        if q_out is None:
+            q_out = torch.empty((N, T, self.S), dtype=torch.float32, device=obs.device)
+        rc = lib().bi_filter_from(self._h, N, T, ctypes.c_void_p(obs.data_ptr()),
+                                  ctypes.c_void_p(act.data_ptr() if act is not None and act.numel() > 0 else None),
+                                  ctypes.c_void_p(q_prev.data_ptr()), ctypes.c_void_p(act_prev.data_ptr()),
+                                  int(iters), ctypes.c_void_p(q_out.data_ptr()),
+                                  ctypes.c_void_p(logq_out.data_ptr() if logq_out is not None else None),
+                                  ctypes.c_void_p(argmax_out.data_ptr() if argmax_out is not None else None),
+                                  _stream_ptr(stream))
+        if rc != BI_OK:
+            raise BiError(rc, "bi_filter_from")
+        return q_out
 
     def bi_vmp(self, obs, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
         """Variational message passing over one window."""

@@ -456,7 +456,8 @@ extern "C" int bi_model_destroy(bi_model_t *model) {
 
 static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, const int32_t *obs,
                     const int32_t *act, int32_t iters, float *q_out, float *logq_out,
-                    int32_t *argmax_out, void *cuda_stream) {
+                    int32_t *argmax_out, void *cuda_stream, const float *q_prev = nullptr,
+                    const int32_t *act_prev = nullptr) {
   if (!model || N < 0 || T < 1 || iters < 1) return BI_ERR_INVALID_ARG;
   if (N == 0) return BI_OK;
   if (!q_out || (model->h.M > 0 && !obs) || (T > 1 && !act)) return BI_ERR_INVALID_ARG;
@@ -465,6 +466,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   BiCall c;
   c.model = model; c.algo = algo; c.N = N; c.T = T; c.K = iters;
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
+  c.q_prev = q_prev; c.act_prev = act_prev;
   c.stream = (cudaStream_t)cuda_stream;
   bi_model *mut = const_cast<bi_model *>(model);
   int rc = bi_launch_tile3(c, mut);
@@ -479,6 +481,15 @@ extern "C" int bi_filter(const bi_model_t *model, int32_t N, int32_t T, const in
                          const int32_t *act, int32_t iters, float *q_out, float *logq_out,
                          int32_t *argmax_out, void *cuda_stream) {
   return run_call(model, BI_ALGO_FILTER, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream);
+}
+
+extern "C" int bi_filter_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                              const int32_t *act, const float *q_prev, const int32_t *act_prev,
+                              int32_t iters, float *q_out, float *logq_out, int32_t *argmax_out,
+                              void *cuda_stream) {
+  if (!q_prev || !act_prev) return BI_ERR_INVALID_ARG;
+  return run_call(model, BI_ALGO_FILTER, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, q_prev,
+                  act_prev);
 }
 
 extern "C" int bi_vmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,

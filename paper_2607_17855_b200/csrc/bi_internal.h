@@ -97,6 +97,8 @@ struct BiCall {
   const bi_model *model;
   int algo, N, T, K;
   const int32_t *obs, *act;
+  const float *q_prev;       // filtering continued from a belief [N][S], or NULL
+  const int32_t *act_prev;   // [N][F], with q_prev
   float *q_out, *logq_out;
   int32_t *argmax_out;
   cudaStream_t stream;

@@ -216,8 +216,9 @@ __device__ __forceinline__ void all_groups(const BiDev &md, int g, const int32_t
 template <typename R, int ALGO, bool STAGED>
 __global__ void __launch_bounds__(256)
 bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
-                  const int32_t *__restrict__ act, int K, float *__restrict__ q_out,
-                  float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, GenSmem sm) {
+                  const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
+                  int K, float *q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out,
+                  GenSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *smem = reinterpret_cast<R *>(smem_raw);
   const BiDev &md = *mdp;
@@ -242,6 +243,15 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
 
   if (ALGO == BI_ALGO_FILTER) {
     R *cur = q0, *nxt = q1;
+    if (q_prev) {  // continued filtering: the belief of the step before the window
+      for (int idx = tid; idx < Sp; idx += NT) {
+        int f = 0;
+        while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+        const int s = idx - md.offp[f];
+        cur[idx] = s < md.n[f] ? (R)q_prev[(size_t)a * S + md.off[f] + s] : (R)0;
+      }
+      __syncthreads();
+    }
     for (int t = 0; t < T; ++t) {
       // ln prior: D at the first step, else B_u q_{t-1} (cur still holds step t-1)
       for (int idx = tid; idx < Sp; idx += NT) {
@@ -250,10 +260,11 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
         const int s = idx - md.offp[f], n = md.n[f];
         R lp = (R)0;
         if (s < n) {
-          if (t == 0) {
+          if (t == 0 && !q_prev) {
             lp = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
           } else {
-            int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
+            const int ur = t == 0 ? act_prev[(size_t)a * F + f] : act[((size_t)a * (T - 1) + (t - 1)) * F + f];
+            int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *row = (const R *)md.Bf[f] + (size_t)g * md.Bstride[f] + ((size_t)u * n + s) * md.npad[f];
             R p = (R)0;
             for (int r = 0; r < n; ++r) p = fma(row[r], cur[md.offp[f] + r], p);
@@ -355,8 +366,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   sm.total_bytes = (int)(o * sizeof(R));
   if ((size_t)sm.total_bytes > budget) return BI_ERR_UNSUPPORTED;
 
-  using KernelT = void (*)(const BiDev *, int, int, const int32_t *, const int32_t *, int, float *,
-                           float *, int32_t *, GenSmem);
+  using KernelT = void (*)(const BiDev *, int, int, const int32_t *, const int32_t *, const float *,
+                           const int32_t *, int, float *, float *, int32_t *, GenSmem);
   KernelT kern = nullptr;
   const char *name = "";
   const bool f64 = sizeof(R) == 8;
@@ -376,8 +387,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes) !=
       cudaSuccess)
     return BI_ERR_CUDA;
-  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.K, c.q_out, c.logq_out,
-                                               c.argmax_out, sm);
+  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.K, c.q_out,
+                                               c.logq_out, c.argmax_out, sm);
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += 1;
   mut->last_kernel = name;

@@ -215,8 +215,9 @@ __device__ __forceinline__ void copy_descriptor(const BiDev *src, void *dst) {
 template <typename R>
 __global__ void __launch_bounds__(512)
 bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
-                      const int32_t *__restrict__ act, int K, float *__restrict__ q_out,
-                      float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, WarpSmem sm) {
+                      const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
+                      int K, float *q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out,
+                      WarpSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   copy_descriptor(mdp, smem_raw);
   const BiDev &md = *reinterpret_cast<const BiDev *>(smem_raw);
@@ -232,6 +233,15 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
   const R **sl = reinterpret_cast<const R **>(wb + sm.o_sl);
   for (int i = lane; i < sm.o_sl - sm.o_q0; i += 32) cur[i] = (R)0;  // q0, q1, V0, V1 are adjacent
   __syncwarp();
+  if (q_prev) {  // continued filtering: the belief of the step before the window
+    for (int idx = lane; idx < Sp; idx += 32) {
+      int f = 0;
+      while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+      const int s = idx - md.offp[f];
+      if (s < md.n[f]) cur[idx] = (R)q_prev[(size_t)a * S + md.off[f] + s];
+    }
+    __syncwarp();
+  }
 
   float *q_a = q_out + (size_t)a * T * S;
   float *lq_a = logq_out ? logq_out + (size_t)a * T * S : nullptr;
@@ -244,10 +254,11 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
       const int s = idx - md.offp[f], n = md.n[f];
       R lp = (R)0;
       if (s < n) {
-        if (t == 0) {
+        if (t == 0 && !q_prev) {
           lp = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
         } else {
-          int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
+          const int ur = t == 0 ? act_prev[(size_t)a * F + f] : act[((size_t)a * (T - 1) + (t - 1)) * F + f];
+          int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
           const R *col = (const R *)md.BfT[f] + (size_t)g * md.Bstride[f] + (size_t)u * n * md.npad[f] + s;
           lp = bi_log_inline(bi_max(col_dot_rt<R>(col, md.npad[f], cur + md.offp[f], n), (R)BI_EPS));
         }
@@ -404,8 +415,9 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
     auto kern = bi_warp_filter_kernel<R>;
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
-    kern<<<(c.N + W - 1) / W, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.K, c.q_out,
-                                                                   c.logq_out, c.argmax_out, sm);
+    kern<<<(c.N + W - 1) / W, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev,
+                                                                   c.act_prev, c.K, c.q_out, c.logq_out,
+                                                                   c.argmax_out, sm);
     name = f64 ? "warp_filter_f64" : "warp_filter_f32";
   } else if (c.algo == BI_ALGO_VMP) {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_VMP>;

@@ -40,6 +40,20 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
   // the previous step's iterations instead of heading every step's chain.
   int o_next[BI_MAX_M], u_next[3] = {0, 0, 0};
   for (int mi = 0; mi < p.nmem; ++mi) o_next[mi] = __ldg(p.obs + out_base * p.M + p.modality[mi]);
+  // Continued filtering: the belief of the step before the window takes the
+  // place of "the previous step's final belief", and its action that of u_{t-1}.
+  const bool from_prev = p.q_prev != nullptr;
+  if (from_prev) {
+    const float *qp = p.q_prev + (size_t)agent * p.S;
+    if (t3.own_a) sq[a] = (R)__ldg(qp + p.off[0] + a);
+    if (t3.own_b) sq[NA + bi] = (R)__ldg(qp + p.off[1] + bi);
+    if (t3.own_c) sq[NA + NB + ci] = (R)__ldg(qp + p.off[2] + ci);
+    const int32_t *ap = p.act_prev + (size_t)agent * p.F;
+    u_next[0] = __ldg(ap + p.fac[0]);
+    u_next[1] = __ldg(ap + p.fac[1]);
+    u_next[2] = __ldg(ap + p.fac[2]);
+    __syncwarp();
+  }
   for (int t = 0; t < p.T; ++t) {
     // ---- the step's summed slice: one gather of every modality's observed slice
     const R *slice[BI_MAX_M];
@@ -60,7 +74,7 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
 
     // ---- ln prior of the logits this lane owns: D, or B_u times the previous step's belief
     R lpa, lpb, lpc;
-    if (t == 0) {
+    if (t == 0 && !from_prev) {
       lpa = __ldg((const R *)p.logD[0] + (size_t)g * p.Dstride[0] + asafe);
       lpb = __ldg((const R *)p.logD[1] + (size_t)g * p.Dstride[1] + bsafe);
       lpc = __ldg((const R *)p.logD[2] + (size_t)g * p.Dstride[2] + csafe);

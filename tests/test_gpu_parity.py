@@ -248,3 +248,60 @@ def test_batched_single_factor_modalities_only(algo):
     w = _custom(46, [5, 9], [4, 3, 6], [[0], [1], [0]], [2, 3], N=150, T=14, K=5)
     res = check_workload(w, algo, agents=range(0, 150, 4))
     assert res["kernel"] == f"batch_{algo}_f64", res
+
+
+# ---- filtering continued from a known belief (bi_filter_from)
+
+def _continued(w, cut, arith="f64"):
+    """Run the first `cut` steps with bi_filter, the rest with bi_filter_from; returns the joined
+    beliefs, the oracle's result for the same two calls, and the kernels used."""
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    md = bi.model_from_workload(w, arith=arith)
+    obs = torch.from_numpy(w.obs).cuda()
+    act = torch.from_numpy(w.act).cuda()
+    q_head = md.bi_filter(obs[:, :cut].contiguous(), act[:, :cut - 1].contiguous(), w.K)
+    q_prev = q_head[:, -1].contiguous()
+    act_prev = act[:, cut - 1].contiguous()
+    q_tail = md.bi_filter_from(obs[:, cut:].contiguous(), act[:, cut:].contiguous(), q_prev, act_prev, w.K)
+    kernel = md.last_kernel
+    assert md.status() == 0
+    # the oracle continues from the very same float32 belief
+    ref_tail = oracle.run("filter", w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, w.obs[:, cut:], w.act[:, cut:], w.K,
+                          q_prev=q_prev.cpu().numpy().astype(np.float64), act_prev=w.act[:, cut - 1])[0]
+    md.close()
+    return q_tail.cpu().numpy(), ref_tail, kernel
+
+
+@pytest.mark.parametrize("case", ["tile", "warp", "per_agent"])
+def test_filter_continuation(case):
+    if case == "tile":
+        w, kern = make_config(2, N=37, T=9, K=8), "tile3_filter_f64"
+    elif case == "warp":
+        w, kern = make_config(3, N=21, T=7, K=6), "warp_filter_f64"
+    else:
+        w, kern = _custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=5, G=5), None
+    for cut in (1, 4):
+        q, ref, kernel = _continued(w, cut)
+        if kern:
+            assert kernel == kern, kernel
+        assert np.abs(q - ref).max() <= 1e-5, (case, cut, np.abs(q - ref).max())
+    # a single tick in place: q_prev and q_out are the same buffer
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    md = bi.model_from_workload(w)
+    obs = torch.from_numpy(w.obs).cuda()
+    act = torch.from_numpy(w.act).cuda()
+    buf = md.bi_filter(obs[:, :1].contiguous(), None, w.K)          # [N, 1, S]
+    start = buf[:, 0].cpu().numpy().astype(np.float64)
+    md.bi_filter_from(obs[:, 1:2].contiguous(), None, buf.view(w.N, -1), act[:, 0].contiguous(), w.K, q_out=buf)
+    ref = oracle.run("filter", w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, w.obs[:, 1:2], w.act[:, :0], w.K,
+                     q_prev=start, act_prev=w.act[:, 0])[0]
+    assert np.abs(buf.cpu().numpy() - ref).max() <= 1e-5
+    null = torch.empty(0, dtype=torch.int32, device="cuda")      # data_ptr() == 0
+    with pytest.raises(bi.BiError) as e:
+        md.bi_filter_from(obs[:, 1:2].contiguous(), None, buf.view(w.N, -1), null, w.K)
+    assert e.value.code == -1
+    md.close()
