@@ -185,6 +185,24 @@ int bi_filter_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t 
                    void *cuda_stream);
 
 /*
+ * bi_vmp / bi_mmp started from given beliefs instead of the uniform ones: the
+ * warm start of a sliding inference window (Section III-A: inference over a
+ * horizon that advances with t), where the previous window's result, shifted by
+ * one step, is the natural starting point.
+ *   q_init    DEVICE [N][T][S] float32: the starting belief of every step, laid out
+ *             like q_out; each factor's block is used as given (not renormalised).
+ *             Must not overlap q_out.
+ *   others    as for bi_vmp / bi_mmp
+ * The iterates are the same Jacobi sweeps; only iterate 0 differs.
+ */
+int bi_vmp_warm(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                const int32_t *act, const float *q_init, int32_t iters, float *q_out,
+                float *logq_out, int32_t *argmax_out, void *cuda_stream);
+int bi_mmp_warm(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                const int32_t *act, const float *q_init, int32_t iters, float *q_out,
+                float *logq_out, int32_t *argmax_out, void *cuda_stream);
+
+/*
  * Variational filtering without any allocation.  (The paper has no counterpart
  * to this entry point: it is a deployment convenience of this library.)
  *

@@ -457,7 +457,7 @@ extern "C" int bi_model_destroy(bi_model_t *model) {
 static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, const int32_t *obs,
                     const int32_t *act, int32_t iters, float *q_out, float *logq_out,
                     int32_t *argmax_out, void *cuda_stream, const float *q_prev = nullptr,
-                    const int32_t *act_prev = nullptr) {
+                    const int32_t *act_prev = nullptr, const float *q_init = nullptr) {
   if (!model || N < 0 || T < 1 || iters < 1) return BI_ERR_INVALID_ARG;
   if (N == 0) return BI_OK;
   if (!q_out || (model->h.M > 0 && !obs) || (T > 1 && !act)) return BI_ERR_INVALID_ARG;
@@ -466,7 +466,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   BiCall c;
   c.model = model; c.algo = algo; c.N = N; c.T = T; c.K = iters;
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
-  c.q_prev = q_prev; c.act_prev = act_prev;
+  c.q_prev = q_prev; c.act_prev = act_prev; c.q_init = q_init;
   c.stream = (cudaStream_t)cuda_stream;
   bi_model *mut = const_cast<bi_model *>(model);
   int rc = bi_launch_tile3(c, mut);
@@ -502,6 +502,22 @@ extern "C" int bi_mmp(const bi_model_t *model, int32_t N, int32_t T, const int32
                       const int32_t *act, int32_t iters, float *q_out, float *logq_out,
                       int32_t *argmax_out, void *cuda_stream) {
   return run_call(model, BI_ALGO_MMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream);
+}
+
+extern "C" int bi_vmp_warm(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                           const int32_t *act, const float *q_init, int32_t iters, float *q_out,
+                           float *logq_out, int32_t *argmax_out, void *cuda_stream) {
+  if (!q_init) return BI_ERR_INVALID_ARG;
+  return run_call(model, BI_ALGO_VMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, nullptr,
+                  nullptr, q_init);
+}
+
+extern "C" int bi_mmp_warm(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                           const int32_t *act, const float *q_init, int32_t iters, float *q_out,
+                           float *logq_out, int32_t *argmax_out, void *cuda_stream) {
+  if (!q_init) return BI_ERR_INVALID_ARG;
+  return run_call(model, BI_ALGO_MMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, nullptr,
+                  nullptr, q_init);
 }
 
 extern "C" int bi_status(const bi_model_t *model, void *cuda_stream, uint32_t *flags) {

@@ -533,14 +533,17 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
 }
 
 template <typename R>
-__global__ void bi_batch_init_kernel(const BiDev *__restrict__ mdp, R *q, int NU) {
+__global__ void bi_batch_init_kernel(const BiDev *__restrict__ mdp, R *q, int NU, const float *__restrict__ q_init) {
   const BiDev &md = *mdp;
   const size_t total = (size_t)NU * md.Sp;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int p = (int)(i % md.Sp);
     int f = 0;
     while (f + 1 < md.F && p >= md.offp[f + 1]) ++f;
-    q[i] = (p - md.offp[f]) < md.n[f] ? (R)1 / (R)md.n[f] : (R)0;
+    const int s = p - md.offp[f];
+    R v = (R)0;
+    if (s < md.n[f]) v = q_init ? (R)q_init[(i / md.Sp) * md.S + md.off[f] + s] : (R)1 / (R)md.n[f];
+    q[i] = v;
   }
 }
 
@@ -666,7 +669,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   A.obs = c.obs; A.act = c.act; A.q_out = c.q_out; A.logq_out = c.logq_out; A.argmax_out = c.argmax_out;
   A.T = c.T;
 
-  bi_batch_init_kernel<R><<<256, 256, 0, c.stream>>>(md->d, (R *)P.qbuf, NU);
+  bi_batch_init_kernel<R><<<256, 256, 0, c.stream>>>(md->d, (R *)P.qbuf, NU, c.q_init);
   if (cnt > 0)
     bi_batch_bucket_kernel<<<cnt, 1024, 2 * max_m * sizeof(int32_t), c.stream>>>(P, c.obs, h.M, h.status, perm, task);
   void (*contract)(BatchParams, int) = any_shape ? bi_batch_contract_rt_kernel<R> : bi_batch_contract_kernel<R>;

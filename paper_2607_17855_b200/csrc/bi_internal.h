@@ -99,6 +99,7 @@ struct BiCall {
   const int32_t *obs, *act;
   const float *q_prev;       // filtering continued from a belief [N][S], or NULL
   const int32_t *act_prev;   // [N][F], with q_prev
+  const float *q_init;       // window algorithms: starting beliefs [N][T][S], or NULL (uniform)
   float *q_out, *logq_out;
   int32_t *argmax_out;
   cudaStream_t stream;

@@ -217,8 +217,8 @@ template <typename R, int ALGO, bool STAGED>
 __global__ void __launch_bounds__(256)
 bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
                   const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
-                  int K, float *q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out,
-                  GenSmem sm) {
+                  const float *__restrict__ q_init, int K, float *q_out, float *__restrict__ logq_out,
+                  int32_t *__restrict__ argmax_out, GenSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *smem = reinterpret_cast<R *>(smem_raw);
   const BiDev &md = *mdp;
@@ -291,6 +291,14 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
     // ---- window algorithms: beliefs of all T steps, Jacobi over (t, f)
     R *cur = q0, *nxt = q1;
     set_uniform<R>(md, cur, T);
+    if (q_init) {  // warm start: the given beliefs replace the uniform ones (pad entries stay zero)
+      for (int idx = tid; idx < T * Sp; idx += NT) {
+        int p = idx % Sp, f = 0;
+        while (f + 1 < F && p >= md.offp[f + 1]) ++f;
+        const int s = p - md.offp[f];
+        if (s < md.n[f]) cur[idx] = (R)q_init[((size_t)a * T + idx / Sp) * S + md.off[f] + s];
+      }
+    }
     if (STAGED)
       for (int t = 0; t < T; ++t) stage_step<R>(md, g, obs_s + t * M, Lst + (size_t)t * md.Ltot);
     __syncthreads();
@@ -367,7 +375,7 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if ((size_t)sm.total_bytes > budget) return BI_ERR_UNSUPPORTED;
 
   using KernelT = void (*)(const BiDev *, int, int, const int32_t *, const int32_t *, const float *,
-                           const int32_t *, int, float *, float *, int32_t *, GenSmem);
+                           const int32_t *, const float *, int, float *, float *, int32_t *, GenSmem);
   KernelT kern = nullptr;
   const char *name = "";
   const bool f64 = sizeof(R) == 8;
@@ -387,8 +395,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes) !=
       cudaSuccess)
     return BI_ERR_CUDA;
-  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.K, c.q_out,
-                                               c.logq_out, c.argmax_out, sm);
+  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.q_init, c.K,
+                                               c.q_out, c.logq_out, c.argmax_out, sm);
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += 1;
   mut->last_kernel = name;

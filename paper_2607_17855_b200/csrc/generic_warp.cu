@@ -286,8 +286,9 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
 template <typename R, int ALGO>
 __global__ void __launch_bounds__(512)
 bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
-                      const int32_t *__restrict__ act, int K, float *__restrict__ q_out,
-                      float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, WarpSmem sm) {
+                      const int32_t *__restrict__ act, const float *__restrict__ q_init, int K,
+                      float *__restrict__ q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out,
+                      WarpSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   copy_descriptor(mdp, smem_raw);
   const BiDev &md = *reinterpret_cast<const BiDev *>(smem_raw);
@@ -308,7 +309,11 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
     const int pidx = i % Sp;
     int f = 0;
     while (f + 1 < F && pidx >= md.offp[f + 1]) ++f;
-    qb[i] = (pidx - md.offp[f]) < md.n[f] ? (R)1 / (R)md.n[f] : (R)0;
+    const int s = pidx - md.offp[f];
+    R v = (R)0;
+    if (s < md.n[f])
+      v = (q_init && i < T * Sp) ? (R)q_init[((size_t)a * T + i / Sp) * S + md.off[f] + s] : (R)1 / (R)md.n[f];
+    qb[i] = v;
   }
   __syncthreads();
 
@@ -423,15 +428,15 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_VMP>;
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
-    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.K, c.q_out, c.logq_out,
-                                                    c.argmax_out, sm);
+    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.K, c.q_out,
+                                                    c.logq_out, c.argmax_out, sm);
     name = f64 ? "warp_vmp_f64" : "warp_vmp_f32";
   } else {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_MMP>;
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
-    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.K, c.q_out, c.logq_out,
-                                                    c.argmax_out, sm);
+    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.K, c.q_out,
+                                                    c.logq_out, c.argmax_out, sm);
     name = f64 ? "warp_mmp_f64" : "warp_mmp_f32";
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;

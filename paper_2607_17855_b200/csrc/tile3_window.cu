@@ -178,6 +178,26 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     qb[i] = s < NA ? (R)1 / (R)NA : s < NA + NB ? (R)1 / (R)NB : s < NA + NB + NC ? (R)1 / (R)NC : (R)0;
   }
   t3.set_uniform();
+  if (p.q_init) {
+    // Warm start: every slot that stands for a real step (halos included) takes that step's
+    // given beliefs; this lane group then holds them as e with normalisers of 1.
+    __syncthreads();
+    for (int i = threadIdx.x; i < (geo.units + 2) * SQ; i += blockDim.x) {
+      const int slot = i / SQ, s = i % SQ, ts = rank * geo.Tc + slot - 1;
+      if (ts < 0 || ts >= T || s >= NA + NB + NC) continue;
+      const int j = s < NA ? 0 : s < NA + NB ? 1 : 2;
+      const int sj = s - (j == 0 ? 0 : j == 1 ? NA : NA + NB);
+      qb[i] = (R)__ldg(p.q_init + ((size_t)agent * T + ts) * p.S + p.off[j] + sj);
+    }
+    __syncthreads();
+    const R *qs = qb + (size_t)(tl + 1) * SQ;   // this group's own step (idle groups shadow a valid slot's layout)
+    t3.ea = a_ok ? qs[asafe] : (R)0;
+#pragma unroll
+    for (int bl = 0; bl < TT::NBL; ++bl) t3.eb[bl] = qs[NA + t3.bh * TT::NBL + bl];
+#pragma unroll
+    for (int c = 0; c < TT::NCP; ++c) t3.ec[c] = c < NC ? qs[NA + NB + c] : (R)0;
+    t3.sa = t3.sb = t3.sc = (R)1;
+  }
   if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
 
   R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;

@@ -305,3 +305,45 @@ def test_filter_continuation(case):
         md.bi_filter_from(obs[:, 1:2].contiguous(), None, buf.view(w.N, -1), null, w.K)
     assert e.value.code == -1
     md.close()
+
+
+# ---- warm-started window algorithms (bi_vmp_warm / bi_mmp_warm)
+
+def _random_beliefs(w, seed):
+    rng = np.random.default_rng(seed)
+    blocks = [rng.dirichlet(np.full(int(nf), 2.0), size=(w.N, w.T)) for nf in w.n]
+    return np.concatenate(blocks, axis=2).astype(np.float32)
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "per_agent"])
+def test_warm_started_windows(case, algo):
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w, kern = {
+        "tile": (make_config(2, N=9, T=11, K=3), f"tile3_{algo}_f64"),
+        "tile_cluster": (make_config(4, N=4, T=20, K=3), f"tile3_{algo}_f64"),
+        "batch": (make_config(3, N=128, T=16, K=3), f"batch_{algo}_f64"),
+        "warp": (make_config(3, N=10, T=7, K=3), f"warp_{algo}_f64"),
+        "per_agent": (_custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=3, G=5), None),
+    }[case]
+    q_init = _random_beliefs(w, 77)
+    md = bi.model_from_workload(w)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    fn = md.bi_vmp_warm if algo == "vmp" else md.bi_mmp_warm
+    lq = torch.empty((w.N, w.T, w.S), dtype=torch.float32, device="cuda")
+    q = fn(obs, act, torch.from_numpy(q_init).cuda(), w.K, logq_out=lq).cpu().numpy()
+    if kern:
+        assert md.last_kernel == kern, md.last_kernel
+    assert md.status() == 0
+    sel = list(range(0, w.N, max(1, w.N // 16)))
+    sub = w.take_agents(sel)
+    ref, lref, _ = oracle.run_workload(sub, algo, q_init=q_init[sel].astype(np.float64))
+    assert np.abs(q[sel] - ref).max() <= 1e-5, np.abs(q[sel] - ref).max()
+    big = lref > -30
+    assert np.abs(lq.cpu().numpy()[sel][big] - lref[big]).max() <= 1e-4
+    # and the start matters: the uniform-start call gives something else after so few sweeps
+    q_cold = md.run(algo, obs, act, w.K).cpu().numpy()
+    assert np.abs(q_cold - q).max() > 1e-4
+    md.close()
