@@ -58,14 +58,17 @@ def _ptr_array(arrs):
 def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G: int,
         A, B, D, obs: np.ndarray, act: Optional[np.ndarray], K: int, *,
         q_init: Optional[np.ndarray] = None, threads: int = 0, round32: bool = False,
-        q_prev: Optional[np.ndarray] = None, act_prev: Optional[np.ndarray] = None):
+        q_prev: Optional[np.ndarray] = None, act_prev: Optional[np.ndarray] = None,
+        obs_soft: Optional[np.ndarray] = None):
     """Run ``algo`` ('filter' | 'vmp' | 'mmp') and return ``(q, logq, argmax)``.
 
     ``obs`` is ``[N, T, M]`` int32, ``act`` ``[N, T-1, F]`` int32 (ignored when
     T == 1); ``q`` and ``logq`` come back as float64 ``[N, T, S]``, ``argmax`` as
     int32 ``[N, T, F]``.  ``q_prev`` ``[N, S]`` with ``act_prev`` ``[N, F]``
     (filtering only) continue a stream: the first step's prior is
-    ``B_u q_prev`` instead of ``D``.
+    ``B_u q_prev`` instead of ``D``.  ``obs_soft`` float32 ``[N, T, sum(m)]``
+    replaces ``obs`` (pass ``obs=None``): every observation is a categorical
+    vector per modality and the log-likelihood is ``log(A_i) . o^i``.
     """
     lib = _load()
     n = np.ascontiguousarray(n, dtype=np.int32)
@@ -77,9 +80,15 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
     A = [np.ascontiguousarray(a, dtype=np.float32) for a in A]
     B = [np.ascontiguousarray(b, dtype=np.float32) for b in B]
     D = [np.ascontiguousarray(d, dtype=np.float32) for d in D]
-    obs = np.ascontiguousarray(obs, dtype=np.int32)
-    N, T = int(obs.shape[0]), int(obs.shape[1])
-    assert obs.shape == (N, T, M)
+    if obs_soft is not None:
+        assert obs is None and q_init is None and q_prev is None and not round32
+        obs_soft = np.ascontiguousarray(obs_soft, dtype=np.float32)
+        N, T = int(obs_soft.shape[0]), int(obs_soft.shape[1])
+        assert obs_soft.shape == (N, T, int(m.sum()))
+    else:
+        obs = np.ascontiguousarray(obs, dtype=np.int32)
+        N, T = int(obs.shape[0]), int(obs.shape[1])
+        assert obs.shape == (N, T, M)
     if T > 1:
         act = np.ascontiguousarray(act, dtype=np.int32)
         assert act.shape == (N, T - 1, F)
@@ -99,6 +108,19 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
         q_init = np.ascontiguousarray(q_init, dtype=np.float64)
         assert q_init.shape == (N, T, S)
     Ap, Bp, Dp = _ptr_array(A), _ptr_array(B), _ptr_array(D)
+    if obs_soft is not None:
+        rc = lib.bi_ref_run_soft(
+            ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),
+            ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),
+            ctypes.c_void_p(dep_len.ctypes.data), ctypes.c_void_p(dep_flat.ctypes.data),
+            ctypes.c_void_p(U.ctypes.data), ctypes.c_int(G), Ap, Bp, Dp,
+            ctypes.c_int(N), ctypes.c_int(T), ctypes.c_void_p(obs_soft.ctypes.data),
+            ctypes.c_void_p(act_p), ctypes.c_int(K),
+            ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(lq.ctypes.data),
+            ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads))
+        if rc != 0:
+            raise ValueError(f"bi_ref_run_soft rejected its arguments (code {rc})")
+        return q, lq, am
     if q_prev is not None or act_prev is not None:
         assert algo == "filter" and q_init is None and not round32
         q_prev = np.ascontiguousarray(q_prev, dtype=np.float64)

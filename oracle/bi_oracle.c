@@ -71,6 +71,8 @@ typedef struct {
     int *off;      /* [F] offset of factor f in a belief vector */
     int *dep_off;  /* [M] offset of modality i's list in dep     */
     int64_t *P;    /* [M] product of the sizes of the factors in dep(i) */
+    int *moff;     /* [M] offset of modality i's block in a soft observation vector */
+    int Mtot;      /* sum of m_i */
     int round32;   /* conditioning probe: round logs and beliefs to float32 */
 } model_t;
 
@@ -93,8 +95,12 @@ static double B_at(const model_t *md, int g, int f, int u, int s_next, int s_pre
  * Section IV):
  *   ell_f[s] = sum_{i: f in dep(i)} sum_{s_dep(i) \ f}
  *              ln A_i[o_i, s_dep(i) with s_f = s] * prod_{g in dep(i), g != f} q_g[s_g].
+ * With soft_t (the step's observation given as one categorical vector per
+ * modality, Section III-B; [Mtot] floats, modality blocks in order) the term
+ * ln A_i[o_i, .] is the contraction over the observation axis of Section
+ * III-C, log(A_i) . o^i = sum_o o^i[o] ln A_i[o, .]; obs_t is then unused.
  */
-static void likelihood_messages(const model_t *md, int g, const int32_t *obs_t,
+static void likelihood_messages(const model_t *md, int g, const int32_t *obs_t, const float *soft_t,
                                 const double *q, double *ell)
 {
     for (int s = 0; s < md->S; ++s) ell[s] = 0.0;
@@ -102,11 +108,18 @@ static void likelihood_messages(const model_t *md, int g, const int32_t *obs_t,
         int k = md->dep_len[i];
         const int32_t *d = md->dep + md->dep_off[i];
         int64_t P = md->P[i];
-        const float *slice = md->A[i] + ((size_t)g * md->m[i] + (size_t)obs_t[i]) * (size_t)P;
+        const float *slice = md->A[i] + ((size_t)g * md->m[i] + (size_t)(soft_t ? 0 : obs_t[i])) * (size_t)P;
         int idx[BI_REF_MAXK];
         for (int j = 0; j < k; ++j) idx[j] = 0;
         for (int64_t e = 0; e < P; ++e) {
-            double la = log_eps((double)slice[e], md->round32);
+            double la;
+            if (soft_t) {
+                la = 0.0;
+                for (int o = 0; o < md->m[i]; ++o)
+                    la += (double)soft_t[md->moff[i] + o] * log_eps((double)slice[(size_t)o * (size_t)P + e], md->round32);
+            } else {
+                la = log_eps((double)slice[e], md->round32);
+            }
             for (int j = 0; j < k; ++j) {
                 double w = 1.0;
                 for (int jj = 0; jj < k; ++jj)
@@ -154,7 +167,7 @@ static void set_initial(const model_t *md, const double *q_init, double *q)
 /* q_prev / act_prev (both NULL, or both given): the belief of the step before the
  * window, [S], and the action taken at that step, [F]; the first step's prior is
  * then B_u q_prev, the same recursion as every later step, instead of D. */
-static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *obs,
+static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *obs, const float *soft,
                          const int32_t *act, const double *q_init, const double *q_prev,
                          const int32_t *act_prev, double *q_out,
                          double *lq_out, int32_t *am_out)
@@ -183,7 +196,8 @@ static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *
         }
         set_initial(md, q_init ? q_init + (size_t)t * S : NULL, cur);
         for (int k = 0; k < K; ++k) {
-            likelihood_messages(md, g, obs + (size_t)t * md->M, cur, ell);
+            likelihood_messages(md, g, obs ? obs + (size_t)t * md->M : NULL,
+                                soft ? soft + (size_t)t * md->Mtot : NULL, cur, ell);
             for (int f = 0; f < F; ++f) {
                 int nf = md->n[f], o = md->off[f];
                 for (int s = 0; s < nf; ++s) x[o + s] = ell[o + s] + lprior[o + s];
@@ -200,7 +214,7 @@ static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *
 
 /* ---- VMP / MMP over one window for one agent --------------------------- */
 static void window_agent(const model_t *md, int algo, int g, int T, int K,
-                         const int32_t *obs, const int32_t *act, const double *q_init,
+                         const int32_t *obs, const float *soft, const int32_t *act, const double *q_init,
                          double *q_out, double *lq_out, int32_t *am_out)
 {
     int S = md->S, F = md->F;
@@ -213,7 +227,8 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
     for (int k = 0; k < K; ++k) {
         for (int t = 0; t < T; ++t) {
             const double *qt = cur + (size_t)t * S;
-            likelihood_messages(md, g, obs + (size_t)t * md->M, qt, ell);
+            likelihood_messages(md, g, obs ? obs + (size_t)t * md->M : NULL,
+                                soft ? soft + (size_t)t * md->Mtot : NULL, qt, ell);
             for (int f = 0; f < F; ++f) {
                 int nf = md->n[f], o = md->off[f];
                 for (int s = 0; s < nf; ++s) {
@@ -274,7 +289,7 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
 static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
                     const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
                     const float *const *A, const float *const *B, const float *const *D,
-                    int N, int T, const int32_t *obs, const int32_t *act, int K,
+                    int N, int T, const int32_t *obs, const float *obs_soft, const int32_t *act, int K,
                     const double *q_init, const double *q_prev, const int32_t *act_prev,
                     double *q_out, double *logq_out,
                     int32_t *argmax_out, int threads, int round32)
@@ -288,6 +303,9 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
     md.off = malloc(sizeof(int) * F);
     md.dep_off = malloc(sizeof(int) * (M > 0 ? M : 1));
     md.P = malloc(sizeof(int64_t) * (M > 0 ? M : 1));
+    md.moff = malloc(sizeof(int) * (M > 0 ? M : 1));
+    md.Mtot = 0;
+    for (int i = 0; i < M; ++i) { md.moff[i] = md.Mtot; md.Mtot += m[i]; }
     int S = 0;
     for (int f = 0; f < F; ++f) { md.off[f] = S; S += n[f]; }
     md.S = S;
@@ -303,7 +321,7 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
         md.P[i] = P;
         o += dep_len[i];
     }
-    if (bad) { free(md.off); free(md.dep_off); free(md.P); return -1; }
+    if (bad) { free(md.off); free(md.dep_off); free(md.P); free(md.moff); return -1; }
 #ifdef _OPENMP
     if (threads > 0) omp_set_num_threads(threads);
 #else
@@ -312,18 +330,19 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
 #pragma omp parallel for schedule(dynamic, 1)
     for (int a = 0; a < N; ++a) {
         int g = (G == 1) ? 0 : a;
-        const int32_t *ob = obs + (size_t)a * T * M;
+        const int32_t *ob = obs ? obs + (size_t)a * T * M : NULL;
+        const float *so = obs_soft ? obs_soft + (size_t)a * T * md.Mtot : NULL;
         const int32_t *ac = act ? act + (size_t)a * (T - 1) * F : NULL;
         const double *qi = q_init ? q_init + (size_t)a * T * S : NULL;
         double *qo = q_out + (size_t)a * T * S;
         double *lo = logq_out ? logq_out + (size_t)a * T * S : NULL;
         int32_t *ao = argmax_out ? argmax_out + (size_t)a * T * F : NULL;
         if (algo == ALGO_FILTER)
-            filter_agent(&md, g, T, K, ob, ac, qi, q_prev ? q_prev + (size_t)a * S : NULL,
+            filter_agent(&md, g, T, K, ob, so, ac, qi, q_prev ? q_prev + (size_t)a * S : NULL,
                          act_prev ? act_prev + (size_t)a * F : NULL, qo, lo, ao);
-        else window_agent(&md, algo, g, T, K, ob, ac, qi, qo, lo, ao);
+        else window_agent(&md, algo, g, T, K, ob, so, ac, qi, qo, lo, ao);
     }
-    free(md.off); free(md.dep_off); free(md.P);
+    free(md.off); free(md.dep_off); free(md.P); free(md.moff);
     return 0;
 }
 
@@ -334,8 +353,26 @@ int bi_ref_run(int algo, int F, int M, const int32_t *n, const int32_t *m,
                const double *q_init, double *q_out, double *logq_out,
                int32_t *argmax_out, int threads, int round32)
 {
-    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, act, K, q_init, NULL, NULL,
+    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, NULL, NULL,
                     q_out, logq_out, argmax_out, threads, round32);
+}
+
+/*
+ * bi_ref_run with every observation given as categorical vectors instead of
+ * indices: obs_soft is [N][T][sum_i m_i] float32, the modalities' blocks in
+ * order (Section III-B: an observation modality is represented as a categorical
+ * probability vector; Section III-C: the log-likelihood is log(A_i) . o^i).
+ * A one-hot vector reproduces the index form.
+ */
+int bi_ref_run_soft(int algo, int F, int M, const int32_t *n, const int32_t *m,
+                    const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+                    const float *const *A, const float *const *B, const float *const *D,
+                    int N, int T, const float *obs_soft, const int32_t *act, int K,
+                    double *q_out, double *logq_out, int32_t *argmax_out, int threads)
+{
+    if (!obs_soft && M > 0) return -1;
+    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, NULL, obs_soft, act, K, NULL, NULL, NULL,
+                    q_out, logq_out, argmax_out, threads, 0);
 }
 
 /*
@@ -353,7 +390,7 @@ int bi_ref_filter_from(int F, int M, const int32_t *n, const int32_t *m,
                        double *q_out, double *logq_out, int32_t *argmax_out, int threads)
 {
     if (!q_prev || !act_prev) return -1;
-    return run_impl(ALGO_FILTER, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, act, K, NULL, q_prev,
+    return run_impl(ALGO_FILTER, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, NULL, q_prev,
                     act_prev, q_out, logq_out, argmax_out, threads, 0);
 }
 

@@ -350,3 +350,76 @@ def test_continuation_arguments_are_checked():
     w = tiny(63, [3], [2], [[0]], [2], T=2)
     with pytest.raises((ValueError, AssertionError)):
         run("vmp", w, 2, q_prev=np.full((1, 3), 1 / 3), act_prev=np.zeros((1, 1), np.int32))
+
+
+# ---- observations as categorical vectors: log-likelihood = log(A_i) . o^i (Section III-C) ----
+
+def one_hot(w):
+    N, T, M = w["obs"].shape
+    out = np.zeros((N, T, int(np.sum(w["m"]))), np.float32)
+    off = np.concatenate([[0], np.cumsum(w["m"])]).astype(int)
+    for i in range(M):
+        np.put_along_axis(out[:, :, off[i]:off[i + 1]], w["obs"][:, :, i:i + 1], 1.0, axis=2)
+    return out
+
+
+def run_soft(algo, w, K, soft):
+    return oracle.run(algo, w["n"], w["m"], w["dep"], w["U"], w["G"], w["A"], w["B"], w["D"], None, w["act"], K,
+                      obs_soft=soft)
+
+
+@pytest.mark.parametrize("algo", ["filter", "vmp", "mmp"])
+def test_one_hot_vectors_reproduce_index_observations(algo):
+    w = tiny(71, [4, 3, 2], [3, 4, 2], [[0, 1], [1, 2, 0], [2]], [2, 3, 1], T=5, N=3, sparsity=0.5)
+    q, lq, am = run(algo, w, 4)
+    qs, lqs, ams = run_soft(algo, w, 4, one_hot(w))
+    np.testing.assert_array_equal(qs, q)
+    np.testing.assert_array_equal(lqs, lq)
+    np.testing.assert_array_equal(ams, am)
+
+
+def test_single_factor_soft_observation_is_a_geometric_mixture():
+    # q proportional to D * prod_o A[o, :]^{w[o]}, written out directly
+    w = tiny(72, [5], [4], [[0]], [2], T=1, N=3)
+    rng = np.random.default_rng(3)
+    soft = rng.dirichlet(np.ones(4), size=(3, 1)).astype(np.float32)
+    q, lq, _ = run_soft("filter", w, 2, soft)
+    A, D = w["A"][0][0].astype(np.float64), w["D"][0][0].astype(np.float64)
+    for a in range(3):
+        post = D * np.prod(A ** soft[a, 0].astype(np.float64)[:, None], axis=0)
+        post /= post.sum()
+        np.testing.assert_allclose(q[a, 0], post, rtol=1e-12)
+
+
+def test_soft_log_likelihood_is_linear_in_the_observation_vector():
+    # one sweep from the uniform start: the logits are prior + likelihood message, and the message is
+    # linear in every modality's vector, so log-beliefs of a mixture are the mixture of log-beliefs up to
+    # one constant per factor
+    w = tiny(73, [3, 4], [3, 2], [[0, 1], [1]], [2, 2], T=1, N=1)
+    o1 = one_hot(w)
+    w2 = dict(w, obs=(w["obs"] + 1) % np.asarray(w["m"], np.int32))
+    o2 = one_hot(w2)
+    alpha = 0.3
+    mix = (alpha * o1 + (1 - alpha) * o2).astype(np.float32)
+    _, l1, _ = run_soft("filter", w, 1, o1)
+    _, l2, _ = run_soft("filter", w, 1, o2)
+    _, lm, _ = run_soft("filter", w, 1, mix)
+    # float32 weights: use the values the oracle actually saw
+    a32 = float(mix[0, 0, w["obs"][0, 0, 0]])
+    for lo, hi in ((0, 3), (3, 7)):
+        d = lm[0, 0, lo:hi] - (a32 * l1[0, 0, lo:hi] + (1 - a32) * l2[0, 0, lo:hi])
+        np.testing.assert_allclose(d, d[0], atol=1e-6)
+
+
+def test_soft_observations_weight_each_modality_separately():
+    # a uniform vector on one modality carries no information about a factor only that modality sees ...
+    w = tiny(74, [3, 2], [4, 3], [[0], [1]], [1, 1], T=1)
+    soft = one_hot(w)
+    soft[0, 0, :4] = 0.25
+    q, _, _ = run_soft("filter", w, 3, soft)
+    A0, D0 = w["A"][0][0].astype(np.float64), w["D"][0][0].astype(np.float64)
+    post = D0 * np.exp(0.25 * np.log(np.maximum(A0, 1e-16)).sum(axis=0))
+    np.testing.assert_allclose(q[0, 0, :3], post / post.sum(), rtol=1e-10)
+    # ... and leaves the other factor's exact posterior untouched
+    qh, _, _ = run("filter", w, 3)
+    np.testing.assert_allclose(q[0, 0, 3:], qh[0, 0, 3:], rtol=1e-12)
