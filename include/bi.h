@@ -203,6 +203,33 @@ int bi_mmp_warm(const bi_model_t *model, int32_t N, int32_t T, const int32_t *ob
                 float *logq_out, int32_t *argmax_out, void *cuda_stream);
 
 /*
+ * The three algorithms with every observation given as categorical vectors
+ * (Section III-B: an observation modality is represented as a categorical
+ * probability vector of length m_i) instead of an index.  The log-likelihood
+ * term of modality i at a step is then log(A_i) . o^i = sum_o o^i[o] ln A_i[o, .]
+ * (Section III-C); a one-hot vector reproduces the index form.
+ *   obs_soft  DEVICE [N][T][sum_i m_i] float32: per step the modalities' vectors one
+ *             after the other, in modality order; used as weights as given (not
+ *             checked or renormalised)
+ *   others    as for bi_filter / bi_vmp / bi_mmp
+ * The call first forms the weighted slices of every (agent, step) in a workspace
+ * of N * T * (sum over dependency groups of the padded slice size) elements of
+ * the handle's arithmetic type (twice that for register-tile models), obtained
+ * from the stream-ordered allocator on first use and kept in the handle, then
+ * runs the same inference kernels on them.  BI_ERR_ALLOC if the workspace cannot
+ * be obtained; BI_ERR_UNSUPPORTED if sum_i m_i exceeds 768 (1536 in float32 arithmetic).
+ */
+int bi_filter_soft(const bi_model_t *model, int32_t N, int32_t T, const float *obs_soft,
+                   const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                   int32_t *argmax_out, void *cuda_stream);
+int bi_vmp_soft(const bi_model_t *model, int32_t N, int32_t T, const float *obs_soft,
+                const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                int32_t *argmax_out, void *cuda_stream);
+int bi_mmp_soft(const bi_model_t *model, int32_t N, int32_t T, const float *obs_soft,
+                const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                int32_t *argmax_out, void *cuda_stream);
+
+/*
  * Variational filtering without any allocation.  (The paper has no counterpart
  * to this entry point: it is a deployment convenience of this library.)
  *

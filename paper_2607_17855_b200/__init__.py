@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -60,7 +60,7 @@ def lib():
         L.bi_model_arith.argtypes = [ctypes.c_void_p]
         L.bi_model_destroy.restype = ctypes.c_int
         L.bi_model_destroy.argtypes = [ctypes.c_void_p]
-        for name in ("bi_filter", "bi_vmp", "bi_mmp"):
+        for name in ("bi_filter", "bi_vmp", "bi_mmp", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft"):
             fn = getattr(L, name)
             fn.restype = ctypes.c_int
             fn.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
@@ -224,6 +224,12 @@ class Model:
     def bi_mmp_warm(self, obs, act, q_init, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
         """``bi_mmp`` started from ``q_init`` float32 ``[N,T,S]`` instead of uniform beliefs."""
         return self._run_warm("bi_mmp_warm", obs, act, q_init, iters, q_out, logq_out, argmax_out, stream)
+
+    def run_soft(self, algo, obs_soft, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
+        """``bi_filter_soft`` / ``bi_vmp_soft`` / ``bi_mmp_soft``: observations as categorical vectors,
+        ``obs_soft`` float32 ``[N,T,sum(m)]`` (CUDA)."""
+        return self._run({"filter": "bi_filter_soft", "vmp": "bi_vmp_soft", "mmp": "bi_mmp_soft"}[algo], obs_soft,
+                         act, iters, q_out, logq_out, argmax_out, stream)
 
     def run(self, algo, *a, **k):
         return {"filter": self.bi_filter, "vmp": self.bi_vmp, "mmp": self.bi_mmp}[algo](*a, **k)

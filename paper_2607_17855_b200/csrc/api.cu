@@ -449,9 +449,19 @@ extern "C" int bi_model_destroy(bi_model_t *model) {
   if (!model) return BI_OK;
   cudaError_t e = cudaDeviceSynchronize();
   if (model->ws) cudaFree(model->ws);
+  if (model->ws_soft) cudaFree(model->ws_soft);
   free_all(model);
   delete model;
   return e == cudaSuccess ? BI_OK : BI_ERR_CUDA;
+}
+
+int bi_dispatch(const BiCall &c, bi_model *mut) {
+  int rc = bi_launch_tile3(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_warp(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
+  return rc;
 }
 
 static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, const int32_t *obs,
@@ -468,13 +478,37 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
   c.q_prev = q_prev; c.act_prev = act_prev; c.q_init = q_init;
   c.stream = (cudaStream_t)cuda_stream;
-  bi_model *mut = const_cast<bi_model *>(model);
-  int rc = bi_launch_tile3(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_warp(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
-  return rc;
+  return bi_dispatch(c, const_cast<bi_model *>(model));
+}
+
+static int run_soft(const bi_model_t *model, int algo, int32_t N, int32_t T, const float *obs_soft,
+                    const int32_t *act, int32_t iters, float *q_out, float *logq_out, int32_t *argmax_out,
+                    void *cuda_stream) {
+  if (!model || N < 0 || T < 1 || iters < 1) return BI_ERR_INVALID_ARG;
+  if (N == 0) return BI_OK;
+  if (!q_out || (model->h.M > 0 && !obs_soft) || (T > 1 && !act)) return BI_ERR_INVALID_ARG;
+  if (model->h.G != 1 && model->h.G != N) return BI_ERR_SHAPE;
+  if (algo != BI_ALGO_FILTER && T > BI_MAX_T) return BI_ERR_UNSUPPORTED;
+  return bi_run_soft(model, algo, N, T, obs_soft, act, iters, q_out, logq_out, argmax_out,
+                     (cudaStream_t)cuda_stream);
+}
+
+extern "C" int bi_filter_soft(const bi_model_t *model, int32_t N, int32_t T, const float *obs_soft,
+                              const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                              int32_t *argmax_out, void *cuda_stream) {
+  return run_soft(model, BI_ALGO_FILTER, N, T, obs_soft, act, iters, q_out, logq_out, argmax_out, cuda_stream);
+}
+
+extern "C" int bi_vmp_soft(const bi_model_t *model, int32_t N, int32_t T, const float *obs_soft,
+                           const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                           int32_t *argmax_out, void *cuda_stream) {
+  return run_soft(model, BI_ALGO_VMP, N, T, obs_soft, act, iters, q_out, logq_out, argmax_out, cuda_stream);
+}
+
+extern "C" int bi_mmp_soft(const bi_model_t *model, int32_t N, int32_t T, const float *obs_soft,
+                           const int32_t *act, int32_t iters, float *q_out, float *logq_out,
+                           int32_t *argmax_out, void *cuda_stream) {
+  return run_soft(model, BI_ALGO_MMP, N, T, obs_soft, act, iters, q_out, logq_out, argmax_out, cuda_stream);
 }
 
 extern "C" int bi_filter(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,

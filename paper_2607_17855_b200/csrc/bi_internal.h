@@ -91,6 +91,8 @@ struct bi_model {
   const char *last_kernel;
   void *ws;         // workspace of the batched window path (stream-ordered allocation), or NULL
   size_t ws_bytes;
+  void *ws_soft;    // workspace of the calls that take observation vectors, or NULL
+  size_t ws_soft_bytes;
 };
 
 struct BiCall {
@@ -112,5 +114,10 @@ int bi_launch_warp(const BiCall &c, bi_model *mut);
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
 int bi_launch_tile3_window(const BiCall &c, bi_model *mut);
 int bi_launch_batch(const BiCall &c, bi_model *mut);
+// tries the kernel families in order (the dispatcher behind every inference call)
+int bi_dispatch(const BiCall &c, bi_model *mut);
+// inference with observations given as categorical vectors [N][T][sum m_i]
+int bi_run_soft(const bi_model *model, int algo, int N, int T, const float *obs_soft, const int32_t *act, int iters,
+                float *q_out, float *logq_out, int32_t *argmax_out, cudaStream_t stream);
 // SB of the compiled register-tile shape for packed dims (na, nb, nc), or 0
 int bi_tile3_shape(int na, int nb, int nc);

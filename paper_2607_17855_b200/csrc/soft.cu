@@ -1,0 +1,223 @@
+// Observations given as categorical vectors (Section III-B) instead of indices.
+//
+// The log-likelihood term of a modality is then the contraction over its
+// observation axis, log(A_i) . o^i (Section III-C), and everything after it is
+// unchanged.  So the call first forms, for every (agent, step) and dependency
+// group, the group's slice  sum_{i in group} sum_o o^i[o] ln A_i[o, .]  in the
+// layouts the inference kernels read, and then runs those kernels on a shadow
+// model in which every group has one modality with T "outcomes" per agent: the
+// slices just formed, selected by the step index.
+#include <algorithm>
+#include <cstring>
+
+#include "bi_device.cuh"
+#include "bi_internal.h"
+
+namespace {
+
+constexpr int kTT = 16;   // steps accumulated per pass over a modality's outcomes
+
+struct SoftMember {
+  const void *src;     // ln A of one modality in the layout being produced: [G][m][P]
+  int64_t gstride;     // elements per model (0 when the model is shared)
+  int32_t m, moff;     // outcomes; offset of the modality's block in an observation vector
+};
+
+struct SoftJob {
+  SoftMember mem[BI_MAX_M];
+  int32_t nmem, P, T, Mtot;
+  const float *soft;   // [N][T][Mtot]
+  void *dst;           // [N][T][P]
+};
+
+// kEPT slice elements of one agent per thread; a modality's outcomes are read
+// once per block of kTT steps and weighted into kTT accumulators per element
+// (a step's weight is one broadcast shared-memory load for kEPT multiply-adds).
+// The vectors are converted to the arithmetic type once, when they are staged.
+template <typename R, int kEPT>
+__global__ void __launch_bounds__(128) bi_soft_slices_kernel(const SoftJob J) {
+  extern __shared__ __align__(16) unsigned char w_raw[];
+  R *w_s = reinterpret_cast<R *>(w_raw);   // [kTT][Mtot] this agent's vectors for the current steps
+  const int a = blockIdx.y;
+  const int e0 = blockIdx.x * (kEPT * 128) + threadIdx.x;   // elements e0 + j * 128
+  R *dst = (R *)J.dst + (size_t)a * J.T * J.P;
+  for (int t0 = 0; t0 < J.T; t0 += kTT) {
+    const int nt = min(kTT, J.T - t0);
+    __syncthreads();
+    for (int i = threadIdx.x; i < nt * J.Mtot; i += blockDim.x)
+      w_s[i] = (R)J.soft[((size_t)a * J.T + t0) * J.Mtot + i];
+    for (int i = nt * J.Mtot + threadIdx.x; i < kTT * J.Mtot; i += blockDim.x) w_s[i] = (R)0;
+    __syncthreads();
+    R acc[kEPT][kTT];
+#pragma unroll
+    for (int j = 0; j < kEPT; ++j)
+#pragma unroll
+      for (int tt = 0; tt < kTT; ++tt) acc[j][tt] = (R)0;
+    for (int mi = 0; mi < J.nmem; ++mi) {
+      const SoftMember &mm = J.mem[mi];
+      const R *src = (const R *)mm.src + (size_t)a * mm.gstride;
+      for (int o = 0; o < mm.m; ++o) {
+        R la[kEPT];
+#pragma unroll
+        for (int j = 0; j < kEPT; ++j) {
+          const int e = e0 + j * 128;
+          la[j] = e < J.P ? __ldg(src + (size_t)o * J.P + e) : (R)0;
+        }
+        const R *wo = w_s + mm.moff + o;
+#pragma unroll
+        for (int tt = 0; tt < kTT; ++tt) {
+          const R wv = wo[tt * J.Mtot];
+#pragma unroll
+          for (int j = 0; j < kEPT; ++j) acc[j][tt] = fma(wv, la[j], acc[j][tt]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kEPT; ++j) {
+      const int e = e0 + j * 128;
+      if (e < J.P) {
+#pragma unroll
+        for (int tt = 0; tt < kTT; ++tt)
+          if (tt < nt) dst[(size_t)(t0 + tt) * J.P + e] = acc[j][tt];
+      }
+    }
+  }
+}
+
+__global__ void bi_soft_step_index_kernel(int32_t *obs, int N, int T, int M) {
+  const size_t total = (size_t)N * T * M;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+    obs[i] = (int32_t)((i / M) % T);
+}
+
+size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+template <typename R>
+int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_soft, const int32_t *act, int iters,
+               float *q_out, float *logq_out, int32_t *argmax_out, cudaStream_t stream) {
+  bi_model *mut = const_cast<bi_model *>(model);
+  const BiDev &h = model->h;
+  int moff[BI_MAX_M], Mtot = 0;
+  for (int i = 0; i < h.M; ++i) { moff[i] = Mtot; Mtot += h.m[i]; }
+  if ((size_t)kTT * Mtot * sizeof(R) > 96 * 1024) return BI_ERR_UNSUPPORTED;
+  const bool tile = model->tile_sb > 0;
+  const size_t NT = (size_t)N * T;
+
+  // ---- workspace: per group the packed slices (and the lane-interleaved ones of a tile model),
+  // the step-index "observations", the shadow descriptor
+  size_t off_pack[BI_MAX_GROUPS], off_tile = 0, need = 0;
+  for (int k = 0; k < h.ngroups; ++k) {
+    off_pack[k] = need;
+    need += up256(NT * h.grp[k].P_pad * sizeof(R));
+  }
+  if (tile) { off_tile = need; need += up256(NT * model->tile_P * sizeof(R)); }
+  const size_t off_obs = need;
+  need += up256(NT * h.ngroups * sizeof(int32_t));
+  const size_t off_desc = need;
+  need += up256(sizeof(BiDev));
+  if (mut->ws_soft_bytes < need) {
+    if (mut->ws_soft && cudaFreeAsync(mut->ws_soft, stream) != cudaSuccess) return BI_ERR_CUDA;
+    mut->ws_soft = nullptr;
+    mut->ws_soft_bytes = 0;
+    void *pnew = nullptr;
+    if (cudaMallocAsync(&pnew, need, stream) != cudaSuccess) {
+      cudaGetLastError();
+      return BI_ERR_ALLOC;
+    }
+    mut->ws_soft = pnew;
+    mut->ws_soft_bytes = need;
+  }
+  unsigned char *w = static_cast<unsigned char *>(mut->ws_soft);
+
+  // ---- the slices.  A register-tile model's kernels read only the lane-interleaved layout, so
+  // that one is formed first; the packed layout follows only if those kernels decline the call.
+  const size_t wsmem = (size_t)kTT * Mtot * sizeof(R);
+  void (*kerns[4])(const SoftJob) = {bi_soft_slices_kernel<R, 1>, bi_soft_slices_kernel<R, 2>,
+                                     bi_soft_slices_kernel<R, 3>, bi_soft_slices_kernel<R, 4>};
+  for (auto kf : kerns)
+    if (cudaFuncSetAttribute((const void *)kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem) != cudaSuccess)
+      return BI_ERR_CUDA;
+  int launches = 0;
+  auto form = [&](int layout) {
+    for (int k = 0; k < (layout ? 1 : h.ngroups); ++k) {
+      const BiGroup &g = h.grp[k];
+      SoftJob J;
+      memset(&J, 0, sizeof(J));
+      J.nmem = g.mem_end - g.mem_begin;
+      J.P = layout ? model->tile_P : g.P_pad;
+      J.T = T; J.Mtot = Mtot; J.soft = obs_soft;
+      J.dst = w + (layout ? off_tile : off_pack[k]);
+      for (int i = 0; i < J.nmem; ++i) {
+        const BiMember &mm = h.mem[g.mem_begin + i];
+        J.mem[i].src = layout ? mm.logA_tile : mm.logA;
+        J.mem[i].gstride = h.G == 1 ? 0 : (int64_t)mm.m * J.P;
+        J.mem[i].m = mm.m;
+        J.mem[i].moff = moff[mm.modality];
+      }
+      // elements per thread: 4 for large slices, else just enough to cover the slice with one CTA
+      const int ept = J.P >= 512 ? 4 : (J.P + 127) / 128;
+      kerns[ept - 1]<<<dim3((J.P + ept * 128 - 1) / (ept * 128), N), 128, wsmem, stream>>>(J);
+      ++launches;
+    }
+  };
+  form(tile ? 1 : 0);
+  int32_t *obs_idx = reinterpret_cast<int32_t *>(w + off_obs);
+  bi_soft_step_index_kernel<<<256, 256, 0, stream>>>(obs_idx, N, T, h.ngroups);
+  ++launches;
+  if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
+
+  // ---- the shadow model: one modality per group, T outcomes per agent, selected by the step index
+  bi_model sh = *model;
+  sh.h.G = N;
+  sh.h.M = h.ngroups;
+  sh.h.nmem = h.ngroups;
+  for (int k = 0; k < h.ngroups; ++k) {
+    BiGroup &g = sh.h.grp[k];
+    g.mem_begin = k;
+    g.mem_end = k + 1;
+    BiMember &mm = sh.h.mem[k];
+    mm.logA = w + off_pack[k];
+    mm.logA_tile = tile && k == 0 ? w + off_tile : nullptr;
+    mm.gstride = (int64_t)T * g.P_pad;
+    mm.m = T;
+    mm.modality = k;
+    mm.P_pad = g.P_pad;
+    sh.h.m[k] = T;
+  }
+  sh.d = reinterpret_cast<BiDev *>(w + off_desc);
+  sh.ws = nullptr;
+  sh.ws_bytes = 0;
+  if (cudaMemcpyAsync(sh.d, &sh.h, sizeof(BiDev), cudaMemcpyHostToDevice, stream) != cudaSuccess) return BI_ERR_CUDA;
+
+  BiCall c;
+  c.model = &sh; c.algo = algo; c.N = N; c.T = T; c.K = iters;
+  c.obs = obs_idx; c.act = act; c.q_prev = nullptr; c.act_prev = nullptr; c.q_init = nullptr;
+  c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
+  c.stream = stream;
+  const int64_t before = sh.launches;
+  int rc;
+  if (tile) {
+    rc = bi_launch_tile3(c, &sh);
+    if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, &sh);
+    if (rc == BI_ERR_UNSUPPORTED) {
+      form(0);
+      if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
+      rc = bi_launch_warp(c, &sh);
+      if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, &sh);
+    }
+  } else {
+    rc = bi_dispatch(c, &sh);
+  }
+  mut->launches += launches + (sh.launches - before);
+  mut->last_kernel = sh.last_kernel;
+  return rc;
+}
+
+}  // namespace
+
+int bi_run_soft(const bi_model *model, int algo, int N, int T, const float *obs_soft, const int32_t *act, int iters,
+                float *q_out, float *logq_out, int32_t *argmax_out, cudaStream_t stream) {
+  return model->arith == BI_ARITH_F64
+             ? run_soft_t<double>(model, algo, N, T, obs_soft, act, iters, q_out, logq_out, argmax_out, stream)
+             : run_soft_t<float>(model, algo, N, T, obs_soft, act, iters, q_out, logq_out, argmax_out, stream);
+}

@@ -25,6 +25,7 @@ def main():
     ap.add_argument("--iters", type=int, default=None, help="iterations K")
     ap.add_argument("--arith", default="f64", choices=["f64", "f32"])
     ap.add_argument("--reps", type=int, default=3, help="warm-up calls before the timed one")
+    ap.add_argument("--soft", action="store_true", help="give the observations as (one-hot) categorical vectors")
     args = ap.parse_args()
 
     import torch
@@ -40,17 +41,27 @@ def main():
     obs = torch.from_numpy(w.obs).cuda()
     act = torch.from_numpy(w.act).cuda() if w.act.size else None
     q = torch.empty((w.N, w.T, w.S), device="cuda")
+    if args.soft:
+        import numpy as np
+        off = np.concatenate([[0], np.cumsum(w.m)]).astype(int)
+        soft = np.zeros((w.N, w.T, int(off[-1])), np.float32)
+        for i in range(w.M):
+            np.put_along_axis(soft[:, :, off[i]:off[i + 1]], w.obs[:, :, i:i + 1], 1.0, axis=2)
+        soft = torch.from_numpy(soft).cuda()
+        call = lambda: md.run_soft(algo, soft, act, w.K, q_out=q)  # noqa: E731
+    else:
+        call = lambda: md.run(algo, obs, act, w.K, q_out=q)  # noqa: E731
     for _ in range(args.reps):
-        md.run(algo, obs, act, w.K, q_out=q)
+        call()
     torch.cuda.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
-    md.run(algo, obs, act, w.K, q_out=q)
+    call()
     b.record()
     b.synchronize()
     ms = a.elapsed_time(b)
     print(json.dumps({"workload": w.name, "algo": algo, "agents": w.N, "T": w.T, "K": w.K, "arith": args.arith,
-                      "kernel": md.last_kernel, "ms": ms, "updates_per_s": w.updates / (ms * 1e-3)}))
+                      "soft": bool(args.soft), "kernel": md.last_kernel, "ms": ms, "updates_per_s": w.updates / (ms * 1e-3)}))
 
 
 if __name__ == "__main__":

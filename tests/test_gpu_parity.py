@@ -347,3 +347,57 @@ def test_warm_started_windows(case, algo):
     q_cold = md.run(algo, obs, act, w.K).cpu().numpy()
     assert np.abs(q_cold - q).max() > 1e-4
     md.close()
+
+
+# ---- observations as categorical vectors (bi_filter_soft / bi_vmp_soft / bi_mmp_soft)
+
+def _soft_vectors(w, seed, sharp=False):
+    """Random categorical vectors per modality; `sharp` gives one-hot vectors of w.obs."""
+    off = np.concatenate([[0], np.cumsum(w.m)]).astype(int)
+    out = np.zeros((w.N, w.T, int(off[-1])), np.float32)
+    rng = np.random.default_rng(seed)
+    for i, mi in enumerate(w.m):
+        if sharp:
+            np.put_along_axis(out[:, :, off[i]:off[i + 1]], w.obs[:, :, i:i + 1], 1.0, axis=2)
+        else:
+            out[:, :, off[i]:off[i + 1]] = rng.dirichlet(np.full(int(mi), 0.7), size=(w.N, w.T))
+    return out
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("case", ["tile_shared", "tile_per_agent", "groups", "mixed_ranks"])
+def test_soft_observations(case, algo):
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = {
+        "tile_shared": make_config(2, N=21, T=9, K=4),
+        "tile_per_agent": make_config(4, N=5, T=6, K=4),
+        "groups": make_config(3, N=12, T=7, K=4),
+        "mixed_ranks": _custom(51, [3, 4, 2, 5, 3], [3, 2, 4, 3], [[0, 1, 2], [3, 4], [1], [2, 0, 1]], [2, 1, 3, 2, 2],
+                               N=9, T=8, K=4, sparsity=0.5),
+    }[case]
+    md = bi.model_from_workload(w)
+    act = torch.from_numpy(w.act).cuda()
+    # one-hot vectors reproduce the index form
+    hard = md.run(algo, torch.from_numpy(w.obs).cuda(), act, w.K).cpu().numpy()
+    sharp = md.run_soft(algo, torch.from_numpy(_soft_vectors(w, 0, sharp=True)).cuda(), act, w.K).cpu().numpy()
+    assert np.abs(sharp - hard).max() <= 2e-6, np.abs(sharp - hard).max()
+    # random vectors against the oracle
+    soft = _soft_vectors(w, 5)
+    lq = torch.empty((w.N, w.T, w.S), dtype=torch.float32, device="cuda")
+    am = torch.empty((w.N, w.T, w.F), dtype=torch.int32, device="cuda")
+    q = md.run_soft(algo, torch.from_numpy(soft).cuda(), act, w.K, logq_out=lq, argmax_out=am).cpu().numpy()
+    assert md.status() == 0
+    ref, lref, amref = oracle.run(algo, w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, None, w.act, w.K, obs_soft=soft)
+    print(case, algo, md.last_kernel, np.abs(q - ref).max())
+    assert np.abs(q - ref).max() <= 1e-5
+    big = lref > -30
+    assert np.abs(lq.cpu().numpy()[big] - lref[big]).max() <= 1e-4
+    # argmax wherever the oracle's top two are further apart than the tolerance
+    off = np.concatenate([[0], np.cumsum(w.n)]).astype(int)
+    for f in range(w.F):
+        blk = np.sort(ref[:, :, off[f]:off[f + 1]], axis=2)
+        clear = (blk[:, :, -1] - blk[:, :, -2] > 2e-5) if blk.shape[2] > 1 else np.ones(blk.shape[:2], bool)
+        assert (am.cpu().numpy()[:, :, f][clear] == amref[:, :, f][clear]).all()
+    md.close()
