@@ -114,8 +114,19 @@ int bi_model_create_arith(const bi_model_desc *desc, int arith, void *cuda_strea
 /* BI_ARITH_* of a handle, or BI_ERR_INVALID_ARG for NULL. */
 int bi_model_arith(const bi_model_t *model);
 
-/* Synchronises the device, frees the packed copies.  NULL is accepted. */
+/* Synchronises the device, frees the packed copies and the handle's workspaces.  NULL is accepted. */
 int bi_model_destroy(bi_model_t *model);
+
+/*
+ * Threads and streams.  A handle may be used from any thread, but its inference
+ * calls must not overlap on the GPU: the status word, the launch bookkeeping and
+ * two workspaces (of the batched window path for shared models and of the calls
+ * that take observation vectors; both obtained from the stream-ordered allocator
+ * on first need, grown on demand and kept until bi_model_destroy) belong to the
+ * handle.  Issue a handle's calls on one stream, or order the streams with
+ * events; for concurrent inference on one model create one handle per stream.
+ * All other calls allocate nothing.
+ */
 
 /*
  * Variational filtering by fixed-point iteration ("FPI", Sections I and IV).
