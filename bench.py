@@ -166,7 +166,11 @@ def time_steps(fn, steps, warmup, flush, torch):
 
 
 def bench_config(torch, bi, w, algo, arith, steps, warmup, flush):
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
     md = bi.model_from_workload(w, arith=arith)
+    torch.cuda.synchronize()
+    pack_ms = (time.perf_counter() - t0) * 1e3   # host arrays -> device, packing kernels, handle
     obs = torch.from_numpy(w.obs).cuda()
     act = torch.from_numpy(w.act).cuda() if w.act.size else None
     q = torch.empty((w.N, w.T, w.S), dtype=torch.float32, device="cuda")
@@ -174,7 +178,8 @@ def bench_config(torch, bi, w, algo, arith, steps, warmup, flush):
     times = time_steps(lambda: md.run(algo, obs, act, w.K, q_out=q), steps, warmup, flush, torch)
     launches = (md.launch_count - l0) // (steps + warmup)
     assert md.status() == 0
-    res = {"seconds": sum(times) / len(times), "best": min(times), "kernel": md.last_kernel,
+    res = {"seconds": sum(times) / len(times), "best": min(times), "median": sorted(times)[len(times) // 2],
+           "pack_ms": pack_ms, "kernel": md.last_kernel,
            "launches_per_step": launches, "model": md, "obs": obs, "act": act, "q": q}
     return res
 
@@ -341,7 +346,8 @@ def main():
         "config": {"workload": "config 2: variational filtering, 4096 agents sharing one model, "
                                "n=[8,8,6], m=[16,8,8], T=50, K=16",
                    "updates_per_step": w.updates, "l2": "flushed with a 256 MiB write before every timed step",
-                   "agents_per_gpu": w.N},
+                   "agents_per_gpu": w.N, "ms_median": head["median"] * 1e3, "ms_best": head["best"] * 1e3,
+                   "agent_steps_per_s": w.N * w.T * world / sec, "model_pack_ms": head["pack_ms"]},
         "e2e": e2e, "gpu_launches": head["launches_per_step"] * args.steps, "clocks": clocks,
         "roofline": roofline,
     }
@@ -414,6 +420,7 @@ def main():
             rates.sort()
             sweep[algo] = {"value": tot_u / tot_s, "unit": UNIT, "min": rates[0], "median": rates[len(rates) // 2],
                            "max": rates[-1], "ms_total": tot_s * 1e3, "kernels": kernels}
+        sweep["cap_entries_per_modality"] = 2 ** 18
         others[f"config5_sweep_{args.arith}"] = sweep
         line["others"] = others
         # ---- the oracle on this machine's host cores, on a bounded sample of the workload
@@ -423,9 +430,16 @@ def main():
         t0 = time.perf_counter()
         oracle.run_workload(sub)
         dt = time.perf_counter() - t0
-        line["cpu_baseline"] = {"value": sub.updates / dt, "unit": UNIT, "cores": oracle.max_threads(),
+        cores = oracle.max_threads()
+        one = w.take_agents(range(64))
+        t0 = time.perf_counter()
+        oracle.run_workload(one, threads=1)
+        dt1 = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": sub.updates / dt, "unit": UNIT, "cores": cores,
                                 "kind": "oracle", "sample": f"first {sample} of 4096 agents, all 50 steps, "
-                                                            f"16 iterations ({dt:.1f} s wall)"}
+                                                            f"16 iterations ({dt:.1f} s wall)",
+                                "single_thread_value": one.updates / dt1,
+                                "single_thread_sample": f"first 64 agents ({dt1:.1f} s)"}
     elif rank == 0:
         line["cpu_baseline"] = None
 
