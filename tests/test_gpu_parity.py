@@ -401,3 +401,26 @@ def test_soft_observations(case, algo):
         clear = (blk[:, :, -1] - blk[:, :, -2] > 2e-5) if blk.shape[2] > 1 else np.ones(blk.shape[:2], bool)
         assert (am.cpu().numpy()[:, :, f][clear] == amref[:, :, f][clear]).all()
     md.close()
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_batched_window_of_a_single_step(algo):
+    # T = 1: no actions at all, every unit is both the first and the last step of its window
+    w = _custom(47, [4, 6, 3], [3, 5], [[0, 1, 2], [1, 2]], [2, 2, 1], N=2100, T=1, K=5)
+    res = check_workload(w, algo, agents=range(0, 2100, 50))
+    assert res["kernel"] == f"batch_{algo}_f64", res
+
+
+def test_soft_observations_single_step_and_empty_batch():
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = _custom(48, [4, 3], [3, 2], [[0, 1], [1]], [2, 2], N=6, T=1, K=3)
+    md = bi.model_from_workload(w)
+    soft = _soft_vectors(w, 9)
+    q = md.run_soft("filter", torch.from_numpy(soft).cuda(), None, w.K).cpu().numpy()
+    ref = oracle.run("filter", w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, None, w.act, w.K, obs_soft=soft)[0]
+    assert np.abs(q - ref).max() <= 1e-5
+    empty = torch.empty((0, 3, 5), dtype=torch.float32, device="cuda")
+    assert md.run_soft("vmp", empty, torch.empty((0, 2, 2), dtype=torch.int32, device="cuda"), 2).shape == (0, 3, w.S)
+    md.close()
