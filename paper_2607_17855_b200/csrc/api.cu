@@ -459,6 +459,16 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
   int rc = bi_launch_tile3(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER && c.N <= 2 * mut->sm_count) {
+    // Filtering exposes one unit per agent.  With about as few agents as SMs, a CTA per agent keeps
+    // more of the machine busy than a warp per agent once the slices are large (measured on the 128
+    // random structures: faster from about 2000 slice elements per step at 64 and 256 agents, slower
+    // at 1024 agents whatever the size).
+    long long elems = 0;
+    for (int gi = 0; gi < mut->h.ngroups; ++gi)
+      if (mut->h.grp[gi].rank >= 2) elems += mut->h.grp[gi].P_pad;
+    if (elems >= 2000) rc = bi_launch_generic(c, mut);
+  }
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_warp(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;

@@ -274,12 +274,14 @@ def _continued(w, cut, arith="f64"):
     return q_tail.cpu().numpy(), ref_tail, kernel
 
 
-@pytest.mark.parametrize("case", ["tile", "warp", "per_agent"])
+@pytest.mark.parametrize("case", ["tile", "warp", "cta", "per_agent"])
 def test_filter_continuation(case):
     if case == "tile":
         w, kern = make_config(2, N=37, T=9, K=8), "tile3_filter_f64"
     elif case == "warp":
-        w, kern = make_config(3, N=21, T=7, K=6), "warp_filter_f64"
+        w, kern = _custom(49, [5, 4, 3, 2], [3, 4], [[0, 1], [1, 2, 3]], [2, 2, 1, 2], N=21, T=7, K=6), "warp_filter_f64"
+    elif case == "cta":   # few agents and large slices: a CTA per agent
+        w, kern = make_config(3, N=21, T=7, K=6), "generic_filter_staged_f64"
     else:
         w, kern = _custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=5, G=5), None
     for cut in (1, 4):
