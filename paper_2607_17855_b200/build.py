@@ -36,17 +36,30 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".tmp{os.getpid()}"
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
-    cmd = [nvcc] + flags + ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()
+    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math") and f != "-shared"]
+    common = [nvcc] + flags + ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-        raise RuntimeError("nvcc failed building libbi.so")
+        common += ["-Xptxas", "-v"]
+    # one object per source, compiled side by side, then one link
+    import tempfile
+    from concurrent.futures import ThreadPoolExecutor
+    with tempfile.TemporaryDirectory(prefix="bi_build_") as objdir:
+        def compile_one(src):
+            obj = os.path.join(objdir, os.path.basename(src) + ".o")
+            return src, obj, subprocess.run(common + ["-c", src, "-o", obj], capture_output=True, text=True)
+        with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+            results = list(pool.map(compile_one, sources()))
+        log = "".join(r.stdout + r.stderr for _, _, r in results)
+        if any(r.returncode != 0 for _, _, r in results):
+            sys.stderr.write(log)
+            raise RuntimeError("nvcc failed building libbi.so")
+        res = subprocess.run([nvcc, "-shared", "-Xcompiler", "-fPIC", "-gencode", "arch=compute_100a,code=sm_100a",
+                              "-o", tmp] + [obj for _, obj, _ in results], capture_output=True, text=True)
+        if res.returncode != 0:
+            sys.stderr.write(log + res.stdout + res.stderr)
+            raise RuntimeError("nvcc failed linking libbi.so")
     if verbose:
-        sys.stderr.write(res.stderr)
+        sys.stderr.write(log)
     os.replace(tmp, LIB)
     return LIB
 
