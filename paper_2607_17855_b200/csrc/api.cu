@@ -274,6 +274,33 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
       long vb = (long)bi_pad4(nb) * nj, vj = (long)bi_pad4(nj) * nb;  // compare pad(nb)/nb vs pad(nj)/nj
       if (vj < vb || (vj == vb && nj < nb)) best = j;
     }
+    // Orders with unrolled kernels (the register tiles, the batched shapes) are kept as they are.
+    // For every other group of rank 3 or more the largest of the remaining axes goes first: the
+    // batched contraction splits a small batch's work along the first axis.
+    {
+      std::vector<int> trial(axes);
+      int lf = trial[best];
+      trial.erase(trial.begin() + best);
+      trial.push_back(lf);
+      int d[BI_MAX_RANK] = {0, 0, 0, 0, 0};
+      for (int j = 0; j < k && j < BI_MAX_RANK; ++j) d[j] = h.n[trial[j]];
+      const bool unrolled = (k == 3 && bi_tile3_shape(d[0], d[1], d[2]) > 0) || bi_batch_shape(k, d) >= 0;
+      if (!unrolled && k >= 3) {
+        // largest outer axis first (stable otherwise)
+        int first = -1;
+        for (int j = 0; j < k; ++j)
+          if (j != best && (first < 0 || h.n[axes[j]] > h.n[axes[first]])) first = j;
+        const int ff = axes[first], lf2 = axes[best];
+        std::vector<int> rest;
+        for (int j = 0; j < k; ++j)
+          if (j != first && j != best) rest.push_back(axes[j]);
+        axes.clear();
+        axes.push_back(ff);
+        for (int f2 : rest) axes.push_back(f2);
+        axes.push_back(lf2);
+        best = k - 1;
+      }
+    }
     int lastf = axes[best];
     axes.erase(axes.begin() + best);
     axes.push_back(lastf);

@@ -708,6 +708,14 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
 
 }  // namespace
 
+int bi_batch_shape(int rank, const int *dim) {
+  BiGroup g;
+  memset(&g, 0, sizeof(g));
+  g.rank = rank;
+  for (int k = 0; k < rank && k < BI_MAX_RANK; ++k) g.dim[k] = dim[k];
+  return rank >= 2 && rank <= 4 ? shape_of(g) : -1;
+}
+
 // Applies to window calls on a shared model with enough (agent, step) units to
 // fill the machine and whose dependency groups all have a compiled shape.
 int bi_launch_batch(const BiCall &c, bi_model *mut) {

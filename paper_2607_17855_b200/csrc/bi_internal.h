@@ -119,5 +119,7 @@ int bi_dispatch(const BiCall &c, bi_model *mut);
 // inference with observations given as categorical vectors [N][T][sum m_i]
 int bi_run_soft(const bi_model *model, int algo, int N, int T, const float *obs_soft, const int32_t *act, int iters,
                 float *q_out, float *logq_out, int32_t *argmax_out, cudaStream_t stream);
+// id of the batched path's unrolled shape for packed dims (rank, then the axis sizes), or -1
+int bi_batch_shape(int rank, const int *dim);
 // SB of the compiled register-tile shape for packed dims (na, nb, nc), or 0
 int bi_tile3_shape(int na, int nb, int nc);

@@ -173,6 +173,25 @@ extern "C" int bi_filter_static(const bi_model_desc *desc, int32_t N, int32_t T,
       long vb = (long)bi_pad4(nb) * nj, vj = (long)bi_pad4(nj) * nb;
       if (vj < vb || (vj == vb && nj < nb)) best = j;
     }
+    {  // same rule as bi_model_create: orders with unrolled kernels stay, otherwise the largest outer axis goes first
+      int d[BI_MAX_RANK] = {0, 0, 0, 0, 0}, p = 0;
+      for (int j = 0; j < k; ++j)
+        if (j != best && p < BI_MAX_RANK) d[p++] = h.n[axes[j]];
+      if (p < BI_MAX_RANK) d[p] = h.n[axes[best]];
+      const bool unrolled = (k == 3 && bi_tile3_shape(d[0], d[1], d[2]) > 0) || bi_batch_shape(k, d) >= 0;
+      if (!unrolled && k >= 3) {
+        int first = -1;
+        for (int j = 0; j < k; ++j)
+          if (j != best && (first < 0 || h.n[axes[j]] > h.n[axes[first]])) first = j;
+        int tmp[BI_MAX_F], q = 0;
+        tmp[q++] = axes[first];
+        for (int j = 0; j < k; ++j)
+          if (j != first && j != best) tmp[q++] = axes[j];
+        tmp[q++] = axes[best];
+        for (int j = 0; j < k; ++j) axes[j] = tmp[j];
+        best = k - 1;
+      }
+    }
     const int lastf = axes[best];
     for (int j = best; j + 1 < k; ++j) axes[j] = axes[j + 1];
     axes[k - 1] = lastf;
