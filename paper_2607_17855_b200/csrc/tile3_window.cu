@@ -208,27 +208,43 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     // step read their halo slot, which always holds valid beliefs, and discard
     // the result), so this code and the contraction below form one
     // straight-line block and their dependency chains interleave.
+    // Where a state is owned by two or more lanes of the group (more lanes than
+    // states), one of them evaluates the past edge and its neighbour the future
+    // edge at the same time, and a shuffle adds the two: half the dot products
+    // and half the logarithms per lane.
     R ta, tb, tc;
     {
       const R *qp = q_cur - SQ, *qn = q_cur + SQ;
-      R va = col_dot_smem<R, NA>(pa0, p.np[0], qp);
-      R vb = col_dot_smem<R, NB>(pa1, p.np[1], qp + NA);
-      R vc = col_dot_smem<R, NC>(pa2, p.np[2], qp + NA + NB);
-      R wa = col_dot_smem<R, NA>(fu0, p.np[0], qn);
-      R wb = col_dot_smem<R, NB>(fu1, p.np[1], qn + NA);
-      R wc = col_dot_smem<R, NC>(fu2, p.np[2], qn + NA + NB);
-      if (ALGO == BI_ALGO_MMP) {
-        va = (R)0.5 * bi_log_inline(bi_max(va, (R)BI_EPS));
-        vb = (R)0.5 * bi_log_inline(bi_max(vb, (R)BI_EPS));
-        vc = (R)0.5 * bi_log_inline(bi_max(vc, (R)BI_EPS));
-        wa = (R)0.5 * bi_log_inline(bi_max(wa, (R)BI_EPS));
-        wb = (R)0.5 * bi_log_inline(bi_max(wb, (R)BI_EPS));
-        wc = (R)0.5 * bi_log_inline(bi_max(wc, (R)BI_EPS));
-      }
       const bool has_prev = t > 0, has_next = t + 1 < T;
-      ta = (has_prev ? va : dprior[0]) + (has_next ? wa : (R)0);
-      tb = (has_prev ? vb : dprior[1]) + (has_next ? wb : (R)0);
-      tc = (has_prev ? vc : dprior[2]) + (has_next ? wc : (R)0);
+      auto edge = [&](R dot, bool future, R prior) -> R {
+        const R v = ALGO == BI_ALGO_MMP ? (R)0.5 * bi_log_inline(bi_max(dot, (R)BI_EPS)) : dot;
+        return future ? (has_next ? v : (R)0) : (has_prev ? v : prior);
+      };
+      constexpr bool DUPA = SB >= 2, DUPB = !TT::TP && TT::SHB >= 1, DUPC = !TT::TP && TT::SHC >= 1;
+      if (DUPA) {
+        const bool fut = (t3.u & 1) != 0;   // u = a * SB + bh: the lowest bit tells the two apart
+        const R v = edge(col_dot_smem<R, NA>(fut ? fu0 : pa0, p.np[0], fut ? qn : qp), fut, dprior[0]);
+        ta = v + __shfl_xor_sync(0xffffffffu, v, 1);
+      } else {
+        ta = edge(col_dot_smem<R, NA>(pa0, p.np[0], qp), false, dprior[0]) +
+             edge(col_dot_smem<R, NA>(fu0, p.np[0], qn), true, (R)0);
+      }
+      if (DUPB) {
+        const bool fut = (a & 1) != 0;      // duplicates of a b owner differ in the low bits of a
+        const R v = edge(col_dot_smem<R, NB>(fut ? fu1 : pa1, p.np[1], (fut ? qn : qp) + NA), fut, dprior[1]);
+        tb = v + __shfl_xor_sync(0xffffffffu, v, SB);
+      } else {
+        tb = edge(col_dot_smem<R, NB>(pa1, p.np[1], qp + NA), false, dprior[1]) +
+             edge(col_dot_smem<R, NB>(fu1, p.np[1], qn + NA), true, (R)0);
+      }
+      if (DUPC) {
+        const bool fut = (t3.u & 1) != 0;   // duplicates of a c owner differ in the low bits of u
+        const R v = edge(col_dot_smem<R, NC>(fut ? fu2 : pa2, p.np[2], (fut ? qn : qp) + NA + NB), fut, dprior[2]);
+        tc = v + __shfl_xor_sync(0xffffffffu, v, 1);
+      } else {
+        tc = edge(col_dot_smem<R, NC>(pa2, p.np[2], qp + NA + NB), false, dprior[2]) +
+             edge(col_dot_smem<R, NC>(fu2, p.np[2], qn + NA + NB), true, (R)0);
+      }
     }
     if (LREG) t3.messages(xa, xb, xc);
     else t3.messages_smem(Lt, xa, xb, xc);
