@@ -65,11 +65,13 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
     ``obs`` is ``[N, T, M]`` int32, ``act`` ``[N, T-1, F]`` int32 (ignored when
     T == 1); ``q`` and ``logq`` come back as float64 ``[N, T, S]``, ``argmax`` as
     int32 ``[N, T, F]``.  ``q_prev`` ``[N, S]`` with ``act_prev`` ``[N, F]``
-    (filtering only) continue a stream: the first step's prior is
-    ``B_u q_prev`` instead of ``D``.  ``obs_soft`` float32 ``[N, T, sum(m)]``
+    continue a stream: the first step's prior is ``B_u q_prev`` instead of
+    ``D`` (for the window algorithms at full weight, like ``D``).  ``obs_soft`` float32 ``[N, T, sum(m)]``
     replaces ``obs`` (pass ``obs=None``): every observation is a categorical
     vector per modality and the log-likelihood is ``log(A_i) . o^i``.
     """
+    if (q_prev is None) != (act_prev is None):
+        raise ValueError("q_prev and act_prev go together")
     lib = _load()
     n = np.ascontiguousarray(n, dtype=np.int32)
     m = np.ascontiguousarray(m, dtype=np.int32)
@@ -120,6 +122,25 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
             ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads))
         if rc != 0:
             raise ValueError(f"bi_ref_run_soft rejected its arguments (code {rc})")
+        return q, lq, am
+    if (q_prev is not None or act_prev is not None) and algo != "filter":
+        assert not round32
+        q_prev = np.ascontiguousarray(q_prev, dtype=np.float64)
+        act_prev = np.ascontiguousarray(act_prev, dtype=np.int32)
+        assert q_prev.shape == (N, S) and act_prev.shape == (N, F)
+        rc = lib.bi_ref_window_from(
+            ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),
+            ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),
+            ctypes.c_void_p(dep_len.ctypes.data), ctypes.c_void_p(dep_flat.ctypes.data),
+            ctypes.c_void_p(U.ctypes.data), ctypes.c_int(G), Ap, Bp, Dp,
+            ctypes.c_int(N), ctypes.c_int(T), ctypes.c_void_p(obs.ctypes.data),
+            ctypes.c_void_p(act_p), ctypes.c_int(K),
+            ctypes.c_void_p(q_init.ctypes.data if q_init is not None else None),
+            ctypes.c_void_p(q_prev.ctypes.data), ctypes.c_void_p(act_prev.ctypes.data),
+            ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(lq.ctypes.data),
+            ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads))
+        if rc != 0:
+            raise ValueError(f"bi_ref_window_from rejected its arguments (code {rc})")
         return q, lq, am
     if q_prev is not None or act_prev is not None:
         assert algo == "filter" and q_init is None and not round32

@@ -213,8 +213,13 @@ static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *
 }
 
 /* ---- VMP / MMP over one window for one agent --------------------------- */
+/* q_prev / act_prev (both NULL, or both given): as for filter_agent, the belief of
+ * the step before the window and the action taken there; the first step's past
+ * message is then ln(B_u q_prev) at full weight, i.e. the window's prior D is
+ * replaced by the predictive prior the filtering recursion would use. */
 static void window_agent(const model_t *md, int algo, int g, int T, int K,
                          const int32_t *obs, const float *soft, const int32_t *act, const double *q_init,
+                         const double *q_prev, const int32_t *act_prev,
                          double *q_out, double *lq_out, int32_t *am_out)
 {
     int S = md->S, F = md->F;
@@ -233,7 +238,11 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
                 int nf = md->n[f], o = md->off[f];
                 for (int s = 0; s < nf; ++s) {
                     double past, future = 0.0;
-                    if (t == 0) {
+                    if (t == 0 && q_prev) {
+                        double p = 0.0;
+                        for (int r = 0; r < nf; ++r) p += B_at(md, g, f, act_prev[f], s, r) * q_prev[o + r];
+                        past = log_eps(p, md->round32);
+                    } else if (t == 0) {
                         past = log_eps((double)md->D[f][(size_t)g * nf + s], md->round32);
                     } else {
                         int u = act[(size_t)(t - 1) * F + f];
@@ -295,7 +304,7 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
                     int32_t *argmax_out, int threads, int round32)
 {
     if (algo < 0 || algo > 2 || F < 1 || M < 0 || N < 0 || T < 1 || K < 1) return -1;
-    if ((q_prev != NULL) != (act_prev != NULL) || (q_prev && algo != ALGO_FILTER)) return -1;
+    if ((q_prev != NULL) != (act_prev != NULL)) return -1;
     if (!(G == 1 || G == N)) return -1;
     model_t md;
     md.F = F; md.M = M; md.G = G; md.n = n; md.m = m; md.dep_len = dep_len; md.dep = dep;
@@ -340,7 +349,8 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
         if (algo == ALGO_FILTER)
             filter_agent(&md, g, T, K, ob, so, ac, qi, q_prev ? q_prev + (size_t)a * S : NULL,
                          act_prev ? act_prev + (size_t)a * F : NULL, qo, lo, ao);
-        else window_agent(&md, algo, g, T, K, ob, so, ac, qi, qo, lo, ao);
+        else window_agent(&md, algo, g, T, K, ob, so, ac, qi, q_prev ? q_prev + (size_t)a * S : NULL,
+                          act_prev ? act_prev + (size_t)a * F : NULL, qo, lo, ao);
     }
     free(md.off); free(md.dep_off); free(md.P); free(md.moff);
     return 0;
@@ -391,6 +401,23 @@ int bi_ref_filter_from(int F, int M, const int32_t *n, const int32_t *m,
 {
     if (!q_prev || !act_prev) return -1;
     return run_impl(ALGO_FILTER, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, NULL, q_prev,
+                    act_prev, q_out, logq_out, argmax_out, threads, 0);
+}
+
+/*
+ * VMP / MMP over a window that continues a stream: as bi_ref_filter_from, the
+ * first step's prior is B_u q_prev (at full weight, in the place of D); q_init
+ * may be NULL (uniform start).
+ */
+int bi_ref_window_from(int algo, int F, int M, const int32_t *n, const int32_t *m,
+                       const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+                       const float *const *A, const float *const *B, const float *const *D,
+                       int N, int T, const int32_t *obs, const int32_t *act, int K,
+                       const double *q_init, const double *q_prev, const int32_t *act_prev,
+                       double *q_out, double *logq_out, int32_t *argmax_out, int threads)
+{
+    if (!q_prev || !act_prev || (algo != ALGO_VMP && algo != ALGO_MMP)) return -1;
+    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, q_prev,
                     act_prev, q_out, logq_out, argmax_out, threads, 0);
 }
 

@@ -349,7 +349,35 @@ def test_single_factor_continuation_is_one_bayes_step():
 def test_continuation_arguments_are_checked():
     w = tiny(63, [3], [2], [[0]], [2], T=2)
     with pytest.raises((ValueError, AssertionError)):
-        run("vmp", w, 2, q_prev=np.full((1, 3), 1 / 3), act_prev=np.zeros((1, 1), np.int32))
+        run("vmp", w, 2, q_prev=np.full((1, 3), 1 / 3))          # act_prev missing
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_window_continuation_replaces_the_prior_by_the_predictive_one(algo):
+    # a window continued from q_prev equals the same window on a model whose D is B_u q_prev
+    w = tiny(64, [4, 3], [3, 4], [[0, 1], [1]], [2, 3], T=4, sparsity=0.5)
+    rng = np.random.default_rng(11)
+    q_prev = np.concatenate([rng.dirichlet(np.ones(4)), rng.dirichlet(np.ones(3))])[None]
+    act_prev = np.array([[1, 2]], np.int32)
+    q, lq, am = run(algo, w, 5, q_prev=q_prev, act_prev=act_prev)
+    D2 = []
+    for f, (lo, hi) in enumerate([(0, 4), (4, 7)]):
+        Bu = w["B"][f][0][:, :, act_prev[0, f]].astype(np.float64)
+        D2.append((Bu @ q_prev[0, lo:hi]).astype(np.float32)[None])
+    q2, _, _ = run(algo, dict(w, D=D2), 5)
+    np.testing.assert_allclose(q, q2, atol=2e-6)      # D2 was rounded to float32
+
+
+def test_single_step_windows_continue_like_the_filter():
+    # T = 1: VMP = MMP = one filtering step, also when the step continues a stream
+    w = tiny(65, [3, 4], [3, 2], [[0, 1], [1]], [2, 2], T=1, N=2)
+    rng = np.random.default_rng(12)
+    q_prev = np.concatenate([rng.dirichlet(np.ones(3), size=2), rng.dirichlet(np.ones(4), size=2)], axis=1)
+    act_prev = rng.integers(0, 2, size=(2, 2)).astype(np.int32)
+    qf, _, _ = run("filter", w, 4, q_prev=q_prev, act_prev=act_prev)
+    for algo in ("vmp", "mmp"):
+        qw, _, _ = run(algo, w, 4, q_prev=q_prev, act_prev=act_prev)
+        np.testing.assert_allclose(qw, qf, atol=1e-12)
 
 
 # ---- observations as categorical vectors: log-likelihood = log(A_i) . o^i (Section III-C) ----
