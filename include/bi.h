@@ -120,8 +120,8 @@ int bi_model_destroy(bi_model_t *model);
 /*
  * Threads and streams.  A handle may be used from any thread, but its inference
  * calls must not overlap on the GPU: the status word, the launch bookkeeping and
- * two workspaces (of the batched window path for shared models and of the calls
- * that take observation vectors; both obtained from the stream-ordered allocator
+ * its workspaces (of the batched window path for shared models, of the calls that
+ * take observation vectors and of the continued window calls; all obtained from the stream-ordered allocator
  * on first need, grown on demand and kept until bi_model_destroy) belong to the
  * handle.  Issue a handle's calls on one stream, or order the streams with
  * events; for concurrent inference on one model create one handle per stream.
@@ -212,6 +212,25 @@ int bi_vmp_warm(const bi_model_t *model, int32_t N, int32_t T, const int32_t *ob
 int bi_mmp_warm(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
                 const int32_t *act, const float *q_init, int32_t iters, float *q_out,
                 float *logq_out, int32_t *argmax_out, void *cuda_stream);
+
+/*
+ * bi_vmp / bi_mmp over a window that continues a stream (the sliding inference
+ * window of Section III-B: the current step together with the preceding h
+ * steps).  As in bi_filter_from, q_prev [N][S] is each agent's belief at the
+ * step before the window and act_prev [N][F] the action taken there; the first
+ * step's past message is then ln(B_{act_prev} q_prev) at full weight, i.e. the
+ * model's prior D is replaced, per agent, by the predictive prior.  q_init may
+ * be NULL (uniform start) or DEVICE [N][T][S] as in bi_vmp_warm.  A small
+ * [N][S] workspace is obtained from the stream-ordered allocator on first use.
+ */
+int bi_vmp_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                const int32_t *act, const float *q_prev, const int32_t *act_prev,
+                const float *q_init, int32_t iters, float *q_out, float *logq_out,
+                int32_t *argmax_out, void *cuda_stream);
+int bi_mmp_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                const int32_t *act, const float *q_prev, const int32_t *act_prev,
+                const float *q_init, int32_t iters, float *q_out, float *logq_out,
+                int32_t *argmax_out, void *cuda_stream);
 
 /*
  * The three algorithms with every observation given as categorical vectors

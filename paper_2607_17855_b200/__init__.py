@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -75,6 +75,12 @@ def lib():
             fn.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                            ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                            ctypes.c_void_p]
+        for name in ("bi_vmp_from", "bi_mmp_from"):
+            fn = getattr(L, name)
+            fn.restype = ctypes.c_int
+            fn.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
+                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.bi_status.restype = ctypes.c_int
         L.bi_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
         L.bi_last_kernel.restype = ctypes.c_char_p
@@ -224,6 +230,29 @@ class Model:
     def bi_mmp_warm(self, obs, act, q_init, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
         """``bi_mmp`` started from ``q_init`` float32 ``[N,T,S]`` instead of uniform beliefs."""
         return self._run_warm("bi_mmp_warm", obs, act, q_init, iters, q_out, logq_out, argmax_out, stream)
+
+    def run_from(self, algo, obs, act, q_prev, act_prev, iters, q_init=None, q_out=None, logq_out=None,
+                 argmax_out=None, stream=None):
+        """``bi_filter_from`` / ``bi_vmp_from`` / ``bi_mmp_from``: the call continues a stream from
+        ``q_prev`` float32 ``[N,S]`` and ``act_prev`` int32 ``[N,F]``."""
+        if algo == "filter":
+            return self.bi_filter_from(obs, act, q_prev, act_prev, iters, q_out, logq_out, argmax_out, stream)
+        import torch
+        N, T = int(obs.shape[0]), int(obs.shape[1])
+        if q_out is None:
+            q_out = torch.empty((N, T, self.S), dtype=torch.float32, device=obs.device)
+        name = "bi_vmp_from" if algo == "vmp" else "bi_mmp_from"
+        rc = getattr(lib(), name)(self._h, N, T, ctypes.c_void_p(obs.data_ptr()),
+                                  ctypes.c_void_p(act.data_ptr() if act is not None and act.numel() > 0 else None),
+                                  ctypes.c_void_p(q_prev.data_ptr()), ctypes.c_void_p(act_prev.data_ptr()),
+                                  ctypes.c_void_p(q_init.data_ptr() if q_init is not None else None), int(iters),
+                                  ctypes.c_void_p(q_out.data_ptr()),
+                                  ctypes.c_void_p(logq_out.data_ptr() if logq_out is not None else None),
+                                  ctypes.c_void_p(argmax_out.data_ptr() if argmax_out is not None else None),
+                                  _stream_ptr(stream))
+        if rc != BI_OK:
+            raise BiError(rc, name)
+        return q_out
 
     def run_soft(self, algo, obs_soft, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
         """``bi_filter_soft`` / ``bi_vmp_soft`` / ``bi_mmp_soft``: observations as categorical vectors,

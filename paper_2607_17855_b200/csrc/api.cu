@@ -6,6 +6,7 @@
 #include <new>
 #include <vector>
 
+#include "bi_device.cuh"
 #include "bi_internal.h"
 
 namespace {
@@ -477,9 +478,29 @@ extern "C" int bi_model_destroy(bi_model_t *model) {
   cudaError_t e = cudaDeviceSynchronize();
   if (model->ws) cudaFree(model->ws);
   if (model->ws_soft) cudaFree(model->ws_soft);
+  if (model->ws_prior) cudaFree(model->ws_prior);
   free_all(model);
   delete model;
   return e == cudaSuccess ? BI_OK : BI_ERR_CUDA;
+}
+
+// ln max(B_u q_prev, eps) for every agent and state: the prior a continued window starts from
+template <typename R>
+__global__ void bi_predictive_prior_kernel(const BiDev *__restrict__ mdp, int N, const float *__restrict__ q_prev,
+                                           const int32_t *__restrict__ act_prev, R *__restrict__ out) {
+  const BiDev &md = *mdp;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N * md.S) return;
+  const int a = i / md.S, p = i - a * md.S;
+  int f = 0;
+  while (f + 1 < md.F && p >= md.off[f + 1]) ++f;
+  const int s = p - md.off[f], n = md.n[f], np = md.npad[f];
+  const int g = md.G == 1 ? 0 : a;
+  const int u = clamp_flag(act_prev[(size_t)a * md.F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
+  const R *row = (const R *)md.Bf[f] + (size_t)g * md.Bstride[f] + ((size_t)u * n + s) * np;   // [next][previous]
+  R acc = (R)0;
+  for (int r = 0; r < n; ++r) acc = fma(row[r], (R)q_prev[(size_t)a * md.S + md.off[f] + r], acc);
+  out[i] = bi_log(bi_max(acc, (R)BI_EPS));
 }
 
 int bi_dispatch(const BiCall &c, bi_model *mut) {
@@ -513,7 +534,37 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   BiCall c;
   c.model = model; c.algo = algo; c.N = N; c.T = T; c.K = iters;
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
-  c.q_prev = q_prev; c.act_prev = act_prev; c.q_init = q_init;
+  c.q_prev = q_prev; c.act_prev = act_prev; c.q_init = q_init; c.lnprior = nullptr;
+  c.stream = (cudaStream_t)cuda_stream;
+  if (algo != BI_ALGO_FILTER && q_prev) {
+    // window continued from a belief: ln(B_u q_prev) per agent, once, in the place of ln D
+    bi_model *mh = const_cast<bi_model *>(model);
+    const size_t need = (size_t)N * model->h.S * (model->arith == BI_ARITH_F64 ? 8 : 4);
+    if (mh->ws_prior_bytes < need) {
+      if (mh->ws_prior && cudaFreeAsync(mh->ws_prior, c.stream) != cudaSuccess) return BI_ERR_CUDA;
+      mh->ws_prior = nullptr;
+      mh->ws_prior_bytes = 0;
+      void *pnew = nullptr;
+      if (cudaMallocAsync(&pnew, need, c.stream) != cudaSuccess) {
+        cudaGetLastError();
+        return BI_ERR_ALLOC;
+      }
+      mh->ws_prior = pnew;
+      mh->ws_prior_bytes = need;
+    }
+    const int total = N * model->h.S;
+    if (model->arith == BI_ARITH_F64)
+      bi_predictive_prior_kernel<double><<<(total + 255) / 256, 256, 0, c.stream>>>(model->d, N, q_prev, act_prev,
+                                                                                   (double *)mh->ws_prior);
+    else
+      bi_predictive_prior_kernel<float><<<(total + 255) / 256, 256, 0, c.stream>>>(model->d, N, q_prev, act_prev,
+                                                                                  (float *)mh->ws_prior);
+    if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
+    mh->launches += 1;
+    c.lnprior = mh->ws_prior;
+    c.q_prev = nullptr;
+    c.act_prev = nullptr;
+  }
   c.stream = (cudaStream_t)cuda_stream;
   return bi_dispatch(c, const_cast<bi_model *>(model));
 }
@@ -589,6 +640,24 @@ extern "C" int bi_mmp_warm(const bi_model_t *model, int32_t N, int32_t T, const 
   if (!q_init) return BI_ERR_INVALID_ARG;
   return run_call(model, BI_ALGO_MMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, nullptr,
                   nullptr, q_init);
+}
+
+extern "C" int bi_vmp_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                           const int32_t *act, const float *q_prev, const int32_t *act_prev,
+                           const float *q_init, int32_t iters, float *q_out, float *logq_out,
+                           int32_t *argmax_out, void *cuda_stream) {
+  if (!q_prev || !act_prev) return BI_ERR_INVALID_ARG;
+  return run_call(model, BI_ALGO_VMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, q_prev,
+                  act_prev, q_init);
+}
+
+extern "C" int bi_mmp_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                           const int32_t *act, const float *q_prev, const int32_t *act_prev,
+                           const float *q_init, int32_t iters, float *q_out, float *logq_out,
+                           int32_t *argmax_out, void *cuda_stream) {
+  if (!q_prev || !act_prev) return BI_ERR_INVALID_ARG;
+  return run_call(model, BI_ALGO_MMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, q_prev,
+                  act_prev, q_init);
 }
 
 extern "C" int bi_status(const bi_model_t *model, void *cuda_stream, uint32_t *flags) {

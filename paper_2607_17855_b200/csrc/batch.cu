@@ -418,6 +418,7 @@ struct UpdateArgs {
   float *q_out, *logq_out;
   int32_t *argmax_out;
   int32_t T, cur, final;
+  const void *lnprior;        // [N][S] log-priors used in the place of ln D at a window's first step, or NULL
   uint32_t fmask[BI_MAX_F];   // members (rank >= 2) whose group contains factor f
   uint32_t r1mask[BI_MAX_F];  // descriptor members (modalities) that depend on factor f alone
 };
@@ -498,7 +499,7 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
         x += __ldg((const R *)mm.logA + (size_t)o * mm.P_pad + s);
       }
       if (t == 0) {
-        x += ((const R *)md.logD[f])[s];
+        x += A.lnprior ? ((const R *)A.lnprior)[(size_t)a * S + I.off + s] : ((const R *)md.logD[f])[s];
       } else {
         const int u = clamp_flag(acp[f], I.U, md.status, BI_FLAG_ACT_RANGE);
         const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);   // [previous][next]
@@ -668,6 +669,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   P.status = h.status;
   A.obs = c.obs; A.act = c.act; A.q_out = c.q_out; A.logq_out = c.logq_out; A.argmax_out = c.argmax_out;
   A.T = c.T;
+  A.lnprior = c.lnprior;
 
   bi_batch_init_kernel<R><<<256, 256, 0, c.stream>>>(md->d, (R *)P.qbuf, NU, c.q_init);
   if (cnt > 0)

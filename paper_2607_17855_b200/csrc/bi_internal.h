@@ -93,6 +93,8 @@ struct bi_model {
   size_t ws_bytes;
   void *ws_soft;    // workspace of the calls that take observation vectors, or NULL
   size_t ws_soft_bytes;
+  void *ws_prior;   // predictive log-priors of continued window calls, or NULL
+  size_t ws_prior_bytes;
 };
 
 struct BiCall {
@@ -102,6 +104,8 @@ struct BiCall {
   const float *q_prev;       // filtering continued from a belief [N][S], or NULL
   const int32_t *act_prev;   // [N][F], with q_prev
   const float *q_init;       // window algorithms: starting beliefs [N][T][S], or NULL (uniform)
+  const void *lnprior;       // window algorithms continued from a belief: ln(B_u q_prev) per agent,
+                             // [N][S] in the handle's arithmetic type, used in the place of ln D; or NULL
   float *q_out, *logq_out;
   int32_t *argmax_out;
   cudaStream_t stream;

@@ -217,8 +217,8 @@ template <typename R, int ALGO, bool STAGED>
 __global__ void __launch_bounds__(256)
 bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
                   const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
-                  const float *__restrict__ q_init, int K, float *q_out, float *__restrict__ logq_out,
-                  int32_t *__restrict__ argmax_out, GenSmem sm) {
+                  const float *__restrict__ q_init, const void *__restrict__ lnprior, int K, float *q_out,
+                  float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, GenSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *smem = reinterpret_cast<R *>(smem_raw);
   const BiDev &md = *mdp;
@@ -314,7 +314,8 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
           R msg = (R)0;
           if (s < n) {
             if (t == 0) {
-              msg = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
+              msg = lnprior ? ((const R *)lnprior)[(size_t)a * S + md.off[f] + s]
+                            : ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
             } else {
               int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
               const R *qp = cur + (t - 1) * Sp + md.offp[f];
@@ -375,7 +376,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if ((size_t)sm.total_bytes > budget) return BI_ERR_UNSUPPORTED;
 
   using KernelT = void (*)(const BiDev *, int, int, const int32_t *, const int32_t *, const float *,
-                           const int32_t *, const float *, int, float *, float *, int32_t *, GenSmem);
+                           const int32_t *, const float *, const void *, int, float *, float *, int32_t *,
+                           GenSmem);
   KernelT kern = nullptr;
   const char *name = "";
   const bool f64 = sizeof(R) == 8;
@@ -395,8 +397,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes) !=
       cudaSuccess)
     return BI_ERR_CUDA;
-  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.q_init, c.K,
-                                               c.q_out, c.logq_out, c.argmax_out, sm);
+  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.q_init,
+                                               c.lnprior, c.K, c.q_out, c.logq_out, c.argmax_out, sm);
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += 1;
   mut->last_kernel = name;

@@ -286,9 +286,9 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
 template <typename R, int ALGO>
 __global__ void __launch_bounds__(512)
 bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
-                      const int32_t *__restrict__ act, const float *__restrict__ q_init, int K,
-                      float *__restrict__ q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out,
-                      WarpSmem sm) {
+                      const int32_t *__restrict__ act, const float *__restrict__ q_init,
+                      const void *__restrict__ lnprior, int K, float *__restrict__ q_out,
+                      float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, WarpSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   copy_descriptor(mdp, smem_raw);
   const BiDev &md = *reinterpret_cast<const BiDev *>(smem_raw);
@@ -335,7 +335,8 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
         R msg = (R)0;
         if (s < n) {
           if (t == 0) {
-            msg = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
+            msg = lnprior ? ((const R *)lnprior)[(size_t)a * S + md.off[f] + s]
+                          : ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
           } else {
             int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);  // [previous][next]
@@ -428,14 +429,14 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_VMP>;
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
-    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.K, c.q_out,
+    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.lnprior, c.K, c.q_out,
                                                     c.logq_out, c.argmax_out, sm);
     name = f64 ? "warp_vmp_f64" : "warp_vmp_f32";
   } else {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_MMP>;
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
-    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.K, c.q_out,
+    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.lnprior, c.K, c.q_out,
                                                     c.logq_out, c.argmax_out, sm);
     name = f64 ? "warp_mmp_f64" : "warp_mmp_f32";
   }

@@ -139,7 +139,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
         Bs[boff + msz + i] = __ldg(Mf + i);
       }
       int up = 0, uf = 0;
-      if (t == 0) dprior[j] = __ldg((const R *)p.logD[j] + (size_t)g * p.Dstride[j] + own[j]);
+      if (t == 0)
+        dprior[j] = p.lnprior ? __ldg((const R *)p.lnprior + (size_t)agent * p.S + p.off[j] + own[j])
+                              : __ldg((const R *)p.logD[j] + (size_t)g * p.Dstride[j] + own[j]);
       else up = clamp_flag(__ldg(p.act + ((size_t)agent * (T - 1) + (t - 1)) * 3 + p.fac[j]), p.U[j], p.status,
                            BI_FLAG_ACT_RANGE);
       if (t + 1 < T)

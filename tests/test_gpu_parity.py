@@ -426,3 +426,44 @@ def test_soft_observations_single_step_and_empty_batch():
     empty = torch.empty((0, 3, 5), dtype=torch.float32, device="cuda")
     assert md.run_soft("vmp", empty, torch.empty((0, 2, 2), dtype=torch.int32, device="cuda"), 2).shape == (0, 3, w.S)
     md.close()
+
+
+# ---- window algorithms continued from a belief (bi_vmp_from / bi_mmp_from)
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "per_agent"])
+def test_continued_windows(case, algo):
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w, kern = {
+        "tile": (make_config(2, N=9, T=11, K=4), f"tile3_{algo}_f64"),
+        "tile_cluster": (make_config(4, N=4, T=20, K=4), f"tile3_{algo}_f64"),
+        "batch": (make_config(3, N=128, T=16, K=4), f"batch_{algo}_f64"),
+        "warp": (make_config(3, N=10, T=7, K=4), f"warp_{algo}_f64"),
+        "per_agent": (_custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=4, G=5), None),
+    }[case]
+    rng = np.random.default_rng(91)
+    q_prev = np.concatenate([rng.dirichlet(np.full(int(nf), 1.5), size=w.N) for nf in w.n], axis=1).astype(np.float32)
+    act_prev = np.stack([rng.integers(0, int(u), size=w.N) for u in w.U], axis=1).astype(np.int32)
+    md = bi.model_from_workload(w)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    q = md.run_from(algo, obs, act, torch.from_numpy(q_prev).cuda(), torch.from_numpy(act_prev).cuda(), w.K)
+    q = q.cpu().numpy()
+    if kern:
+        assert md.last_kernel == kern, md.last_kernel
+    assert md.status() == 0
+    sel = list(range(0, w.N, max(1, w.N // 16)))
+    sub = w.take_agents(sel)
+    ref = oracle.run_workload(sub, algo, q_prev=q_prev[sel].astype(np.float64), act_prev=act_prev[sel])[0]
+    assert np.abs(q[sel] - ref).max() <= 1e-5, np.abs(q[sel] - ref).max()
+    # the prior matters: the plain call (prior D) differs
+    assert np.abs(md.run(algo, obs, act, w.K).cpu().numpy() - q).max() > 1e-4
+    # ... and both a continued prior and a warm start at once
+    q_init = _random_beliefs(w, 78)
+    q2 = md.run_from(algo, obs, act, torch.from_numpy(q_prev).cuda(), torch.from_numpy(act_prev).cuda(), w.K,
+                     q_init=torch.from_numpy(q_init).cuda()).cpu().numpy()
+    ref2 = oracle.run_workload(sub, algo, q_init=q_init[sel].astype(np.float64), q_prev=q_prev[sel].astype(np.float64),
+                               act_prev=act_prev[sel])[0]
+    assert np.abs(q2[sel] - ref2).max() <= 1e-5
+    md.close()
