@@ -59,7 +59,7 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
         A, B, D, obs: np.ndarray, act: Optional[np.ndarray], K: int, *,
         q_init: Optional[np.ndarray] = None, threads: int = 0, round32: bool = False,
         q_prev: Optional[np.ndarray] = None, act_prev: Optional[np.ndarray] = None,
-        obs_soft: Optional[np.ndarray] = None):
+        obs_soft: Optional[np.ndarray] = None, damping: float = 1.0):
     """Run ``algo`` ('filter' | 'vmp' | 'mmp') and return ``(q, logq, argmax)``.
 
     ``obs`` is ``[N, T, M]`` int32, ``act`` ``[N, T-1, F]`` int32 (ignored when
@@ -69,6 +69,7 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
     ``D`` (for the window algorithms at full weight, like ``D``).  ``obs_soft`` float32 ``[N, T, sum(m)]``
     replaces ``obs`` (pass ``obs=None``): every observation is a categorical
     vector per modality and the log-likelihood is ``log(A_i) . o^i``.
+    ``damping`` in (0, 1]: step size of the update on log-beliefs (1 = plain).
     """
     if (q_prev is None) != (act_prev is None):
         raise ValueError("q_prev and act_prev go together")
@@ -110,6 +111,29 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
         q_init = np.ascontiguousarray(q_init, dtype=np.float64)
         assert q_init.shape == (N, T, S)
     Ap, Bp, Dp = _ptr_array(A), _ptr_array(B), _ptr_array(D)
+    if damping != 1.0:
+        if q_prev is not None:
+            q_prev = np.ascontiguousarray(q_prev, dtype=np.float64)
+            act_prev = np.ascontiguousarray(act_prev, dtype=np.int32)
+            assert q_prev.shape == (N, S) and act_prev.shape == (N, F)
+        rc = lib.bi_ref_run_opts(
+            ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),
+            ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),
+            ctypes.c_void_p(dep_len.ctypes.data), ctypes.c_void_p(dep_flat.ctypes.data),
+            ctypes.c_void_p(U.ctypes.data), ctypes.c_int(G), Ap, Bp, Dp,
+            ctypes.c_int(N), ctypes.c_int(T),
+            ctypes.c_void_p(obs.ctypes.data if obs is not None else None),
+            ctypes.c_void_p(obs_soft.ctypes.data if obs_soft is not None else None),
+            ctypes.c_void_p(act_p), ctypes.c_int(K),
+            ctypes.c_void_p(q_init.ctypes.data if q_init is not None else None),
+            ctypes.c_void_p(q_prev.ctypes.data if q_prev is not None else None),
+            ctypes.c_void_p(act_prev.ctypes.data if act_prev is not None else None),
+            ctypes.c_double(float(damping)),
+            ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(lq.ctypes.data),
+            ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads), ctypes.c_int(int(round32)))
+        if rc != 0:
+            raise ValueError(f"bi_ref_run_opts rejected its arguments (code {rc})")
+        return q, lq, am
     if obs_soft is not None:
         rc = lib.bi_ref_run_soft(
             ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),

@@ -74,6 +74,7 @@ typedef struct {
     int *moff;     /* [M] offset of modality i's block in a soft observation vector */
     int Mtot;      /* sum of m_i */
     int round32;   /* conditioning probe: round logs and beliefs to float32 */
+    double lambda; /* damping of the log-belief update: 1 = the plain fixed-point map */
 } model_t;
 
 static double log_eps(double x, int round32)
@@ -195,12 +196,15 @@ static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *
             }
         }
         set_initial(md, q_init ? q_init + (size_t)t * S : NULL, cur);
+        for (int s = 0; s < S; ++s) lq[s] = log_eps(cur[s], 0);
         for (int k = 0; k < K; ++k) {
             likelihood_messages(md, g, obs ? obs + (size_t)t * md->M : NULL,
                                 soft ? soft + (size_t)t * md->Mtot : NULL, cur, ell);
             for (int f = 0; f < F; ++f) {
                 int nf = md->n[f], o = md->off[f];
-                for (int s = 0; s < nf; ++s) x[o + s] = ell[o + s] + lprior[o + s];
+                /* damped update on log-beliefs: ln q' = (1 - lambda) ln q + lambda (message + ln prior) + const */
+                for (int s = 0; s < nf; ++s)
+                    x[o + s] = (1.0 - md->lambda) * lq[o + s] + md->lambda * (ell[o + s] + lprior[o + s]);
                 am[f] = softmax_vec(x + o, nf, nxt + o, lq + o, md->round32);
             }
             double *tmp = cur; cur = nxt; nxt = tmp;
@@ -229,6 +233,7 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
     double *x = malloc(sizeof(double) * S);
     int32_t *am = malloc(sizeof(int32_t) * (size_t)T * F);
     for (int t = 0; t < T; ++t) set_initial(md, q_init ? q_init + (size_t)t * S : NULL, cur + (size_t)t * S);
+    for (size_t i = 0; i < TS; ++i) lq[i] = log_eps(cur[i], 0);
     for (int k = 0; k < K; ++k) {
         for (int t = 0; t < T; ++t) {
             const double *qt = cur + (size_t)t * S;
@@ -275,7 +280,7 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
                             future = 0.5 * log_eps(p, md->round32);
                         }
                     }
-                    x[o + s] = ell[o + s] + past + future;
+                    x[o + s] = (1.0 - md->lambda) * lq[(size_t)t * S + o + s] + md->lambda * (ell[o + s] + past + future);
                 }
                 am[(size_t)t * F + f] = softmax_vec(x + o, nf, nxt + (size_t)t * S + o,
                                                     lq + (size_t)t * S + o, md->round32);
@@ -301,14 +306,15 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
                     int N, int T, const int32_t *obs, const float *obs_soft, const int32_t *act, int K,
                     const double *q_init, const double *q_prev, const int32_t *act_prev,
                     double *q_out, double *logq_out,
-                    int32_t *argmax_out, int threads, int round32)
+                    int32_t *argmax_out, int threads, int round32, double lambda)
 {
     if (algo < 0 || algo > 2 || F < 1 || M < 0 || N < 0 || T < 1 || K < 1) return -1;
+    if (!(lambda > 0.0 && lambda <= 1.0)) return -1;
     if ((q_prev != NULL) != (act_prev != NULL)) return -1;
     if (!(G == 1 || G == N)) return -1;
     model_t md;
     md.F = F; md.M = M; md.G = G; md.n = n; md.m = m; md.dep_len = dep_len; md.dep = dep;
-    md.U = U; md.A = A; md.B = B; md.D = D; md.round32 = round32;
+    md.U = U; md.A = A; md.B = B; md.D = D; md.round32 = round32; md.lambda = lambda;
     md.off = malloc(sizeof(int) * F);
     md.dep_off = malloc(sizeof(int) * (M > 0 ? M : 1));
     md.P = malloc(sizeof(int64_t) * (M > 0 ? M : 1));
@@ -364,7 +370,7 @@ int bi_ref_run(int algo, int F, int M, const int32_t *n, const int32_t *m,
                int32_t *argmax_out, int threads, int round32)
 {
     return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, NULL, NULL,
-                    q_out, logq_out, argmax_out, threads, round32);
+                    q_out, logq_out, argmax_out, threads, round32, 1.0);
 }
 
 /*
@@ -382,7 +388,7 @@ int bi_ref_run_soft(int algo, int F, int M, const int32_t *n, const int32_t *m,
 {
     if (!obs_soft && M > 0) return -1;
     return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, NULL, obs_soft, act, K, NULL, NULL, NULL,
-                    q_out, logq_out, argmax_out, threads, 0);
+                    q_out, logq_out, argmax_out, threads, 0, 1.0);
 }
 
 /*
@@ -401,7 +407,7 @@ int bi_ref_filter_from(int F, int M, const int32_t *n, const int32_t *m,
 {
     if (!q_prev || !act_prev) return -1;
     return run_impl(ALGO_FILTER, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, NULL, q_prev,
-                    act_prev, q_out, logq_out, argmax_out, threads, 0);
+                    act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0);
 }
 
 /*
@@ -418,7 +424,24 @@ int bi_ref_window_from(int algo, int F, int M, const int32_t *n, const int32_t *
 {
     if (!q_prev || !act_prev || (algo != ALGO_VMP && algo != ALGO_MMP)) return -1;
     return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, q_prev,
-                    act_prev, q_out, logq_out, argmax_out, threads, 0);
+                    act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0);
+}
+
+/*
+ * Every option at once, plus damping: the update becomes
+ *   ln q' = (1 - lambda) ln q + lambda (likelihood message + transition messages) + const,
+ * a step of size lambda on the log-beliefs towards the plain update (lambda = 1).
+ * Unused options are NULL; obs_soft replaces obs when given.
+ */
+int bi_ref_run_opts(int algo, int F, int M, const int32_t *n, const int32_t *m,
+                    const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+                    const float *const *A, const float *const *B, const float *const *D,
+                    int N, int T, const int32_t *obs, const float *obs_soft, const int32_t *act, int K,
+                    const double *q_init, const double *q_prev, const int32_t *act_prev, double lambda,
+                    double *q_out, double *logq_out, int32_t *argmax_out, int threads, int round32)
+{
+    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, obs_soft, act, K, q_init, q_prev,
+                    act_prev, q_out, logq_out, argmax_out, threads, round32, lambda);
 }
 
 int bi_ref_max_threads(void)

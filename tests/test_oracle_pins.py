@@ -451,3 +451,52 @@ def test_soft_observations_weight_each_modality_separately():
     # ... and leaves the other factor's exact posterior untouched
     qh, _, _ = run("filter", w, 3)
     np.testing.assert_allclose(q[0, 0, 3:], qh[0, 0, 3:], rtol=1e-12)
+
+
+# ---- damped update on log-beliefs ----
+
+def test_damping_one_is_the_plain_update_and_small_steps_interpolate():
+    w = tiny(81, [3, 4], [3, 2], [[0, 1], [1]], [2, 2], T=3)
+    for algo in ("filter", "vmp", "mmp"):
+        q, lq, _ = run(algo, w, 4)
+        q1, lq1, _ = run(algo, w, 4, damping=1.0 - 1e-12)
+        np.testing.assert_allclose(q1, q, atol=1e-9)
+
+
+def test_single_factor_damped_filter_has_a_closed_form():
+    # one factor: the plain update is the exact posterior p* whatever q is, so after k damped steps from
+    # the uniform start  ln q_k = (1 - (1 - lambda)^k) ln p* + const
+    w = tiny(82, [5], [4], [[0]], [2], T=1, N=2)
+    lam = 0.35
+    p_star, _, _ = run("filter", w, 1)
+    for K in (1, 2, 5):
+        q, _, _ = run("filter", w, K, damping=lam)
+        for a in range(2):
+            want = p_star[a, 0] ** (1.0 - (1.0 - lam) ** K)
+            np.testing.assert_allclose(q[a, 0], want / want.sum(), rtol=1e-12)
+
+
+def test_damping_keeps_the_fixed_points():
+    # a fixed point of the plain map is a fixed point of the damped one: start both at a converged
+    # belief (a decoupled model converges in one sweep) and nothing moves
+    w = tiny(83, [3, 2], [3, 2, 2], [[0], [1], [0]], [2, 1], T=1)
+    q, _, _ = run("filter", w, 3)
+    q_init = q.copy()
+    qd, _, _ = run("filter", w, 4, q_init=q_init, damping=0.4)
+    np.testing.assert_allclose(qd, q, atol=1e-12)
+
+
+def test_damped_windows_start_from_log_q_init():
+    # the first damped step mixes the plain update with ln q_init
+    w = tiny(84, [3, 4], [3, 2], [[0, 1], [1]], [2, 2], T=2)
+    rng = np.random.default_rng(5)
+    q_init = np.concatenate([rng.dirichlet(np.ones(3), size=(1, 2)), rng.dirichlet(np.ones(4), size=(1, 2))], axis=2)
+    lam = 0.6
+    for algo in ("vmp", "mmp"):
+        _, lplain, _ = run(algo, w, 1, q_init=q_init)            # log of the plain update from q_init
+        qd, _, _ = run(algo, w, 1, q_init=q_init, damping=lam)
+        for lo, hi in ((0, 3), (3, 7)):
+            mix = (1 - lam) * np.log(q_init[0, :, lo:hi]) + lam * lplain[0, :, lo:hi]
+            want = np.exp(mix - mix.max(axis=1, keepdims=True))
+            want /= want.sum(axis=1, keepdims=True)
+            np.testing.assert_allclose(qd[0, :, lo:hi], want, rtol=1e-11)
