@@ -118,6 +118,17 @@ int bi_model_arith(const bi_model_t *model);
 int bi_model_destroy(bi_model_t *model);
 
 /*
+ * Damped updates (optional; the paper's iteration is the plain one, lambda = 1).
+ * Every later inference call on the handle replaces the update of a factor by
+ *   ln q' = (1 - lambda) ln q + lambda (likelihood message + transition messages) + const,
+ * a step of size lambda on the log-beliefs towards the plain update; ln q of a
+ * starting belief is ln max(q, 1e-16).  The plain Jacobi map oscillates on many
+ * models (see BI_ARITH_*); a step below 1 damps that and, with it, the
+ * amplification of rounding errors.  0 < lambda <= 1, else BI_ERR_INVALID_ARG.
+ */
+int bi_model_set_damping(bi_model_t *model, double lambda);
+
+/*
  * Threads and streams.  A handle may be used from any thread, but its inference
  * calls must not overlap on the GPU: the status word, the launch bookkeeping and
  * its workspaces (of the batched window path for shared models, of the calls that

@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -81,6 +81,8 @@ def lib():
             fn.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.bi_model_set_damping.restype = ctypes.c_int
+        L.bi_model_set_damping.argtypes = [ctypes.c_void_p, ctypes.c_double]
         L.bi_status.restype = ctypes.c_int
         L.bi_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
         L.bi_last_kernel.restype = ctypes.c_char_p
@@ -262,6 +264,12 @@ class Model:
 
     def run(self, algo, *a, **k):
         return {"filter": self.bi_filter, "vmp": self.bi_vmp, "mmp": self.bi_mmp}[algo](*a, **k)
+
+    def set_damping(self, lam: float):
+        """Step size of the update on log-beliefs for every later call (1 = the plain update)."""
+        rc = lib().bi_model_set_damping(self._h, float(lam))
+        if rc != BI_OK:
+            raise BiError(rc, "bi_model_set_damping")
 
     def status(self, stream=None) -> int:
         v = ctypes.c_uint32(0)

@@ -208,6 +208,7 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
   bi_model *md = new (std::nothrow) bi_model();
   if (!md) return BI_ERR_ALLOC;
   memset(md, 0, sizeof(*md));
+  md->damping = 1.0;
   md->last_kernel = "";
   md->arith = arith;
   if (cudaGetDevice(&md->device) != cudaSuccess) {
@@ -535,6 +536,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   c.model = model; c.algo = algo; c.N = N; c.T = T; c.K = iters;
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
   c.q_prev = q_prev; c.act_prev = act_prev; c.q_init = q_init; c.lnprior = nullptr;
+  c.lambda = model->damping;
   c.stream = (cudaStream_t)cuda_stream;
   if (algo != BI_ALGO_FILTER && q_prev) {
     // window continued from a belief: ln(B_u q_prev) per agent, once, in the place of ln D
@@ -658,6 +660,12 @@ extern "C" int bi_mmp_from(const bi_model_t *model, int32_t N, int32_t T, const 
   if (!q_prev || !act_prev) return BI_ERR_INVALID_ARG;
   return run_call(model, BI_ALGO_MMP, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, q_prev,
                   act_prev, q_init);
+}
+
+extern "C" int bi_model_set_damping(bi_model_t *model, double lambda) {
+  if (!model || !(lambda > 0.0 && lambda <= 1.0)) return BI_ERR_INVALID_ARG;
+  model->damping = lambda;
+  return BI_OK;
 }
 
 extern "C" int bi_status(const bi_model_t *model, void *cuda_stream, uint32_t *flags) {

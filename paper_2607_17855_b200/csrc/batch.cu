@@ -419,6 +419,10 @@ struct UpdateArgs {
   int32_t *argmax_out;
   int32_t T, cur, final;
   const void *lnprior;        // [N][S] log-priors used in the place of ln D at a window's first step, or NULL
+  double lambda;              // damping step; 1 = plain update
+  void *xprev;                // [NU][Sp] previous iterate's logits (damped calls only), or NULL
+  int32_t first;              // first iteration of the call
+  const float *q_init;        // warm start (for the first damped step's ln q), or NULL
   uint32_t fmask[BI_MAX_F];   // members (rank >= 2) whose group contains factor f
   uint32_t r1mask[BI_MAX_F];  // descriptor members (modalities) that depend on factor f alone
 };
@@ -511,6 +515,18 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
         const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);   // [next][previous]
         const R v = col_dot_g<R>(M1 + (size_t)u * n * np + s, np, qc + (size_t)(unit + 1) * Sp + op, n);
         x += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
+      }
+    }
+    if (A.xprev) {
+      // damped step on the logits; the first one starts from ln q of the starting belief (uniform: a
+      // constant, taken as 0)
+      R *xp = (R *)A.xprev + (size_t)unit * Sp + op;
+      if (s < n) {
+        R prev = (R)0;
+        if (!A.first) prev = xp[s];
+        else if (A.q_init) prev = bi_log(bi_max((R)A.q_init[(size_t)unit * S + I.off + s], (R)BI_EPS));
+        x = fma((R)A.lambda, x, ((R)1 - (R)A.lambda) * prev);
+        if (live) xp[s] = x;
       }
     }
     // any shift near the maximum keeps the exponentials in range; the last iterate takes the exact one
@@ -646,7 +662,8 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   const size_t b_task = up256((size_t)ntask * sizeof(int4));
   const size_t b_ellp = up256((size_t)cnt * NU * h.Sp * sizeof(R));
   const size_t b_q = up256(2 * (size_t)NU * h.Sp * sizeof(R));
-  const size_t need = b_perm + b_task + b_ellp + b_q;
+  const size_t b_x = c.lambda != 1.0 ? up256((size_t)NU * h.Sp * sizeof(R)) : 0;
+  const size_t need = b_perm + b_task + b_ellp + b_q + b_x;
   if (mut->ws_bytes < need) {
     if (mut->ws && cudaFreeAsync(mut->ws, c.stream) != cudaSuccess) return BI_ERR_CUDA;
     mut->ws = nullptr;
@@ -670,6 +687,9 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   A.obs = c.obs; A.act = c.act; A.q_out = c.q_out; A.logq_out = c.logq_out; A.argmax_out = c.argmax_out;
   A.T = c.T;
   A.lnprior = c.lnprior;
+  A.lambda = c.lambda;
+  A.xprev = b_x ? w + b_perm + b_task + b_ellp + b_q : nullptr;
+  A.q_init = c.q_init;
 
   bi_batch_init_kernel<R><<<256, 256, 0, c.stream>>>(md->d, (R *)P.qbuf, NU, c.q_init);
   if (cnt > 0)
@@ -698,6 +718,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     if (cnt > 0) contract<<<ntask, tu * rs, csmem, c.stream>>>(P, cur);
     A.cur = cur;
     A.final = (k == c.K - 1);
+    A.first = (k == 0);
     update<<<(NU + upb - 1) / upb, 128, 0, c.stream>>>(md->d, P, A);
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;

@@ -95,6 +95,7 @@ struct bi_model {
   size_t ws_soft_bytes;
   void *ws_prior;   // predictive log-priors of continued window calls, or NULL
   size_t ws_prior_bytes;
+  double damping;   // step of the update on log-beliefs, (0, 1]; 1 = the plain fixed-point map
 };
 
 struct BiCall {
@@ -104,6 +105,7 @@ struct BiCall {
   const float *q_prev;       // filtering continued from a belief [N][S], or NULL
   const int32_t *act_prev;   // [N][F], with q_prev
   const float *q_init;       // window algorithms: starting beliefs [N][T][S], or NULL (uniform)
+  double lambda;             // damping: ln q' = (1 - lambda) ln q + lambda (messages) + const; 1 = plain
   const void *lnprior;       // window algorithms continued from a belief: ln(B_u q_prev) per agent,
                              // [N][S] in the handle's arithmetic type, used in the place of ln D; or NULL
   float *q_out, *logq_out;

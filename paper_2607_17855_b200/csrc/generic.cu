@@ -17,6 +17,7 @@ namespace {
 
 struct GenSmem {  // element offsets (units of R) into dynamic shared memory
   int q0, q1, lpri, ell, Lst, V0, V1, red, obs, total_bytes;
+  int xp;      // damped calls: previous logits, Tq steps; -1 otherwise
   int Tq;      // belief steps kept (1 for filtering, T for windows)
   int staged;  // summed slices staged in shared memory
 };
@@ -143,11 +144,16 @@ __device__ __forceinline__ void contract_group(const BiGroup &g, const LD &first
 // writes the next beliefs (padded layout) and, if final, the outputs.
 template <typename R>
 __device__ __forceinline__ void softmax_step(const BiDev &md, const R *ell, R *qn, bool final,
-                                             float *q_out, float *logq_out, int32_t *argmax_out) {
+                                             float *q_out, float *logq_out, int32_t *argmax_out,
+                                             R *xp = nullptr, R lam = (R)1) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
   for (int f = warp; f < md.F; f += nw) {
     const int n = md.n[f], op = md.offp[f];
     R x = lane < n ? ell[op + lane] : -bi_inf<R>();
+    if (xp && lane < n) {   // damped step on the logits; xp: the previous iterate's
+      x = fma(lam, x, ((R)1 - lam) * xp[op + lane]);
+      xp[op + lane] = x;
+    }
     R mx = warp_max(x);
     R e = lane < n ? bi_exp(x - mx) : (R)0;
     R z = warp_sum(e);
@@ -217,8 +223,8 @@ template <typename R, int ALGO, bool STAGED>
 __global__ void __launch_bounds__(256)
 bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
                   const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
-                  const float *__restrict__ q_init, const void *__restrict__ lnprior, int K, float *q_out,
-                  float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, GenSmem sm) {
+                  const float *__restrict__ q_init, const void *__restrict__ lnprior, double lambda, int K,
+                  float *q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, GenSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *smem = reinterpret_cast<R *>(smem_raw);
   const BiDev &md = *mdp;
@@ -227,6 +233,7 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
   const int tid = threadIdx.x, NT = blockDim.x;
   const int S = md.S, Sp = md.Sp, F = md.F, M = md.M;
   R *q0 = smem + sm.q0, *q1 = smem + sm.q1, *lpri = smem + sm.lpri, *ell = smem + sm.ell;
+  R *xpb = sm.xp >= 0 ? smem + sm.xp : nullptr;   // previous logits (damped calls)
   R *Lst = smem + sm.Lst, *V0 = smem + sm.V0, *V1 = smem + sm.V1, *red = smem + sm.red;
   int32_t *obs_s = reinterpret_cast<int32_t *>(smem + sm.obs);
 
@@ -276,13 +283,15 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
       if (STAGED) stage_step<R>(md, g, obs_s + t * M, Lst);
       __syncthreads();
       set_uniform<R>(md, cur, 1);
+      if (xpb)
+        for (int idx = tid; idx < Sp; idx += NT) xpb[idx] = (R)0;   // logits of the uniform start: a constant
       __syncthreads();
       for (int k = 0; k < K; ++k) {
         for (int idx = tid; idx < Sp; idx += NT) ell[idx] = lpri[idx];
         __syncthreads();
         all_groups<R, STAGED>(md, g, obs_s + t * M, Lst, cur, ell, V0, V1, red);
         softmax_step<R>(md, ell, nxt, k == K - 1, q_a + (size_t)t * S, lq_a ? lq_a + (size_t)t * S : nullptr,
-                        am_a ? am_a + (size_t)t * F : nullptr);
+                        am_a ? am_a + (size_t)t * F : nullptr, xpb, (R)lambda);
         __syncthreads();
         R *tmp = cur; cur = nxt; nxt = tmp;
       }
@@ -297,6 +306,14 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
         while (f + 1 < F && p >= md.offp[f + 1]) ++f;
         const int s = p - md.offp[f];
         if (s < md.n[f]) cur[idx] = (R)q_init[((size_t)a * T + idx / Sp) * S + md.off[f] + s];
+      }
+    }
+    if (xpb) {   // damped calls start from the logarithms of the starting beliefs (uniform: a constant)
+      __syncthreads();
+      for (int idx = tid; idx < T * Sp; idx += NT) {
+        int p = idx % Sp, f = 0;
+        while (f + 1 < F && p >= md.offp[f + 1]) ++f;
+        xpb[idx] = (q_init && p - md.offp[f] < md.n[f]) ? bi_log(bi_max(cur[idx], (R)BI_EPS)) : (R)0;
       }
     }
     if (STAGED)
@@ -340,7 +357,8 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
         __syncthreads();
         all_groups<R, STAGED>(md, g, obs_s + t * M, Lst + (size_t)t * md.Ltot, qt, ell, V0, V1, red);
         softmax_step<R>(md, ell, nxt + t * Sp, k == K - 1, q_a + (size_t)t * S,
-                        lq_a ? lq_a + (size_t)t * S : nullptr, am_a ? am_a + (size_t)t * F : nullptr);
+                        lq_a ? lq_a + (size_t)t * S : nullptr, am_a ? am_a + (size_t)t * F : nullptr,
+                        xpb ? xpb + t * Sp : nullptr, (R)lambda);
         __syncthreads();
       }
       R *tmp = cur; cur = nxt; nxt = tmp;
@@ -367,6 +385,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   sm.V1 = o; o += bi_pad4(md->V1max);
   sm.red = o; o += nwarps * 32;
   sm.obs = o; o += bi_pad4(c.T * h.M + 1);
+  sm.xp = c.lambda != 1.0 ? o : -1;
+  if (c.lambda != 1.0) o += sm.Tq * h.Sp;
   const size_t budget = (size_t)md->max_smem_optin - 1024;
   const size_t stage = (size_t)(window ? c.T : 1) * h.Ltot;
   sm.staged = stage > 0 && ((size_t)o + stage) * sizeof(R) <= budget;
@@ -376,7 +396,7 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if ((size_t)sm.total_bytes > budget) return BI_ERR_UNSUPPORTED;
 
   using KernelT = void (*)(const BiDev *, int, int, const int32_t *, const int32_t *, const float *,
-                           const int32_t *, const float *, const void *, int, float *, float *, int32_t *,
+                           const int32_t *, const float *, const void *, double, int, float *, float *, int32_t *,
                            GenSmem);
   KernelT kern = nullptr;
   const char *name = "";
@@ -398,7 +418,7 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
       cudaSuccess)
     return BI_ERR_CUDA;
   kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.q_init,
-                                               c.lnprior, c.K, c.q_out, c.logq_out, c.argmax_out, sm);
+                                               c.lnprior, c.lambda, c.K, c.q_out, c.logq_out, c.argmax_out, sm);
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += 1;
   mut->last_kernel = name;

@@ -31,6 +31,8 @@ struct WarpSmem {       // element offsets (units of R) into dynamic shared memo
   int md_bytes;         // bytes reserved for the model descriptor copy
   int total_bytes;
   int W;                // warps per CTA
+  int o_xp;             // filtering, damped calls: per-warp previous logits [Sp]; -1 otherwise
+  int xp;               // window, damped calls: [T][Sp] previous logits shared by the CTA; -1 otherwise
 };
 
 template <typename R>
@@ -166,10 +168,15 @@ __device__ __forceinline__ void slice_table(const BiDev &md, int g, const int32_
 // softmax of every factor of one step from the logits in ell
 template <typename R>
 __device__ __forceinline__ void softmax_warp(const BiDev &md, const R *ell, R *qn, bool final, float *q_out,
-                                             float *logq_out, int32_t *argmax_out, int lane) {
+                                             float *logq_out, int32_t *argmax_out, int lane, R *xp = nullptr,
+                                             R lam = (R)1) {
   for (int f = 0; f < md.F; ++f) {
     const int n = md.n[f], op = md.offp[f];
     R x = lane < n ? ell[op + lane] : -bi_inf<R>();
+    if (xp && lane < n) {   // damped step on the logits; xp: the previous iterate's
+      x = fma(lam, x, ((R)1 - lam) * xp[op + lane]);
+      xp[op + lane] = x;
+    }
     // the shift only has to be close to the maximum (softmax is shift
     // invariant): a float reduction halves the shuffles of a double one
     R mx = final ? warp_max(x) : (R)warp_max((float)x);
@@ -216,8 +223,8 @@ template <typename R>
 __global__ void __launch_bounds__(512)
 bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
                       const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
-                      int K, float *q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out,
-                      WarpSmem sm) {
+                      double lambda, int K, float *q_out, float *__restrict__ logq_out,
+                      int32_t *__restrict__ argmax_out, WarpSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   copy_descriptor(mdp, smem_raw);
   const BiDev &md = *reinterpret_cast<const BiDev *>(smem_raw);
@@ -231,6 +238,7 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
   R *ell = wb + sm.o_ell, *lpri = wb + sm.o_lpri, *cur = wb + sm.o_q0, *nxt = wb + sm.o_q1;
   R *V0 = wb + sm.o_V0, *V1 = wb + sm.o_V1;
   const R **sl = reinterpret_cast<const R **>(wb + sm.o_sl);
+  R *xpw = sm.o_xp >= 0 ? wb + sm.o_xp : nullptr;
   for (int i = lane; i < sm.o_sl - sm.o_q0; i += 32) cur[i] = (R)0;  // q0, q1, V0, V1 are adjacent
   __syncwarp();
   if (q_prev) {  // continued filtering: the belief of the step before the window
@@ -270,6 +278,7 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
       int f = 0;
       while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
       cur[idx] = (idx - md.offp[f]) < md.n[f] ? (R)1 / (R)md.n[f] : (R)0;
+      if (xpw) xpw[idx] = (R)0;   // logits of the uniform start: a constant
     }
     __syncwarp();
     for (int k = 0; k < K; ++k) {
@@ -277,7 +286,7 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
       __syncwarp();
       likelihood_warp<R>(md, sl, cur, ell, V0, V1, lane);
       softmax_warp<R>(md, ell, nxt, k == K - 1, q_a + (size_t)t * S, lq_a ? lq_a + (size_t)t * S : nullptr,
-                      am_a ? am_a + (size_t)t * F : nullptr, lane);
+                      am_a ? am_a + (size_t)t * F : nullptr, lane, xpw, (R)lambda);
       R *tmp = cur; cur = nxt; nxt = tmp;
     }
   }
@@ -287,7 +296,7 @@ template <typename R, int ALGO>
 __global__ void __launch_bounds__(512)
 bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
                       const int32_t *__restrict__ act, const float *__restrict__ q_init,
-                      const void *__restrict__ lnprior, int K, float *__restrict__ q_out,
+                      const void *__restrict__ lnprior, double lambda, int K, float *__restrict__ q_out,
                       float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, WarpSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   copy_descriptor(mdp, smem_raw);
@@ -314,6 +323,8 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
     if (s < md.n[f])
       v = (q_init && i < T * Sp) ? (R)q_init[((size_t)a * T + i / Sp) * S + md.off[f] + s] : (R)1 / (R)md.n[f];
     qb[i] = v;
+    if (sm.xp >= 0 && i < T * Sp)   // damped calls: logits of the start (uniform: a constant)
+      (base + sm.xp)[i] = (q_init && s < md.n[f]) ? bi_log(bi_max(v, (R)BI_EPS)) : (R)0;
   }
   __syncthreads();
 
@@ -357,7 +368,8 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
       __syncwarp();
       likelihood_warp<R>(md, sl, qt, ell, V0, V1, lane);
       softmax_warp<R>(md, ell, nxt + (size_t)t * Sp, k == K - 1, q_a + (size_t)t * S,
-                      lq_a ? lq_a + (size_t)t * S : nullptr, am_a ? am_a + (size_t)t * F : nullptr, lane);
+                      lq_a ? lq_a + (size_t)t * S : nullptr, am_a ? am_a + (size_t)t * F : nullptr, lane,
+                      sm.xp >= 0 ? base + sm.xp + (size_t)t * Sp : nullptr, (R)lambda);
     }
     __syncthreads();
     R *tmp = cur; cur = nxt; nxt = tmp;
@@ -379,6 +391,9 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
   sm.o_V0 = o; o += bi_pad4(md->V0max);
   sm.o_V1 = o; o += bi_pad4(md->V1max);
   sm.o_sl = o; o += (int)(BI_MAX_M * sizeof(void *) / sizeof(R));
+  const bool damped = c.lambda != 1.0;
+  sm.o_xp = (!window && damped) ? o : -1;
+  if (!window && damped) o += h.Sp;
   sm.per_warp = o;
   const size_t budget = 100 * 1024;  // at least two CTAs per SM
   size_t shared_elems = 0;
@@ -387,7 +402,10 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
     shared_elems = 2 * (size_t)c.T * h.Sp;
     sm.obs = (int)shared_elems;
     shared_elems += (size_t)bi_pad4((int)(((size_t)c.T * h.M * sizeof(int32_t) + sizeof(R) - 1) / sizeof(R)) + 1);
+    sm.xp = damped ? (int)shared_elems : -1;
+    if (damped) shared_elems += (size_t)c.T * h.Sp;
   } else {
+    sm.xp = -1;
     sm.q = 0;
     sm.obs = 0;
   }
@@ -422,22 +440,22 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
     kern<<<(c.N + W - 1) / W, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev,
-                                                                   c.act_prev, c.K, c.q_out, c.logq_out,
+                                                                   c.act_prev, c.lambda, c.K, c.q_out, c.logq_out,
                                                                    c.argmax_out, sm);
     name = f64 ? "warp_filter_f64" : "warp_filter_f32";
   } else if (c.algo == BI_ALGO_VMP) {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_VMP>;
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
-    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.lnprior, c.K, c.q_out,
-                                                    c.logq_out, c.argmax_out, sm);
+    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.lnprior, c.lambda, c.K,
+                                                    c.q_out, c.logq_out, c.argmax_out, sm);
     name = f64 ? "warp_vmp_f64" : "warp_vmp_f32";
   } else {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_MMP>;
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
-    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.lnprior, c.K, c.q_out,
-                                                    c.logq_out, c.argmax_out, sm);
+    kern<<<c.N, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_init, c.lnprior, c.lambda, c.K,
+                                                    c.q_out, c.logq_out, c.argmax_out, sm);
     name = f64 ? "warp_mmp_f64" : "warp_mmp_f32";
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;

@@ -191,7 +191,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
 
   BiCall c;
   c.model = &sh; c.algo = algo; c.N = N; c.T = T; c.K = iters;
-  c.obs = obs_idx; c.act = act; c.q_prev = nullptr; c.act_prev = nullptr; c.q_init = nullptr; c.lnprior = nullptr;
+  c.obs = obs_idx; c.act = act; c.q_prev = nullptr; c.act_prev = nullptr; c.q_init = nullptr; c.lnprior = nullptr; c.lambda = model->damping;
   c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
   c.stream = stream;
   const int64_t before = sh.launches;

@@ -30,6 +30,7 @@ struct Tile3Params {
   float *q_out, *logq_out;
   int32_t *argmax_out;
   uint32_t *status;
+  double lambda;             // damping step (1 = plain update)
 };
 
 // sum_r M[r][s] q[r] for this lane's s: col points at M[0][s], rows are `stride` apart
@@ -78,6 +79,6 @@ static inline void bi_tile3_fill_params(const BiCall &c, Tile3Params &p) {
   }
   p.N = c.N; p.T = c.T; p.K = c.K; p.M = h.M; p.S = h.S; p.G = h.G;
   p.obs = c.obs; p.act = c.act; p.q_out = c.q_out; p.logq_out = c.logq_out;
-  p.q_prev = c.q_prev; p.act_prev = c.act_prev; p.q_init = c.q_init; p.lnprior = c.lnprior; p.F = c.model->h.F;
+  p.q_prev = c.q_prev; p.act_prev = c.act_prev; p.q_init = c.q_init; p.lnprior = c.lnprior; p.lambda = c.lambda; p.F = c.model->h.F;
   p.argmax_out = c.argmax_out; p.status = h.status;
 }

@@ -45,7 +45,7 @@ __device__ __forceinline__ R col_dot_smem(const R *col, int stride, const R *q) 
 
 // LREG: the step's summed slice lives in registers (small tiles); otherwise in
 // shared memory (tiles too large for the register file).
-template <typename R, int NA, int NB, int NC, int SB, bool LREG, int ALGO, bool STALE, bool CLUSTER>
+template <typename R, int NA, int NB, int NC, int SB, bool LREG, int ALGO, bool STALE, bool CLUSTER, bool DAMPED>
 __global__ void __launch_bounds__(320)
 bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   using TT = Tile3<R, NA, NB, NC, SB>;
@@ -180,6 +180,8 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     qb[i] = s < NA ? (R)1 / (R)NA : s < NA + NB ? (R)1 / (R)NB : s < NA + NB + NC ? (R)1 / (R)NC : (R)0;
   }
   t3.set_uniform();
+  R pxa = 0, pxb = 0, pxc = 0;   // previous iterate's logits (uniform start: a constant, taken as 0)
+  const R lam = (R)p.lambda, oml = (R)1 - lam;
   if (p.q_init) {
     // Warm start: every slot that stands for a real step (halos included) takes that step's
     // given beliefs; this lane group then holds them as e with normalisers of 1.
@@ -199,6 +201,10 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
 #pragma unroll
     for (int c = 0; c < TT::NCP; ++c) t3.ec[c] = c < NC ? qs[NA + NB + c] : (R)0;
     t3.sa = t3.sb = t3.sc = (R)1;
+    // the damped update starts from the logarithms of the given beliefs
+    if (DAMPED) pxa = a_ok ? bi_log(bi_max(qs[asafe], (R)BI_EPS)) : (R)0;
+    if (DAMPED) pxb = b_ok ? bi_log(bi_max(qs[NA + bsafe], (R)BI_EPS)) : (R)0;
+    if (DAMPED) pxc = c_ok ? bi_log(bi_max(qs[NA + NB + csafe], (R)BI_EPS)) : (R)0;
   }
   if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
 
@@ -253,6 +259,12 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     xa = a_ok ? xa + ta : -bi_inf<R>();
     xb = b_ok ? xb + tb : -bi_inf<R>();
     xc = c_ok ? xc + tc : -bi_inf<R>();
+    if (DAMPED) {   // damped step on the logits (a shift per factor does not matter)
+      xa = a_ok ? fma(lam, xa, oml * pxa) : xa;
+      xb = b_ok ? fma(lam, xb, oml * pxb) : xb;
+      xc = c_ok ? fma(lam, xc, oml * pxc) : xc;
+      pxa = a_ok ? xa : (R)0; pxb = b_ok ? xb : (R)0; pxc = c_ok ? xc : (R)0;
+    }
     const float cma = group_max_f<NAP, SB>((float)xa);
     const float cmb = group_max_f<LPU, 1>((float)xb);
     const float cmc = group_max_f<LPU, 1>((float)xc);
@@ -399,16 +411,21 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   cfg.attrs = attr;
   cfg.numAttrs = geo.CS > 1 ? 1 : 0;
   cudaError_t e;
-#define BI_WIN_LAUNCH(ST, CL)                                                                         \
+#define BI_WIN_LAUNCH(ST, CL, DA)                                                                     \
   do {                                                                                                \
-    auto kern = bi_tile3_window_kernel<R, NA, NB, NC, SB, LREG, ALGO, ST, CL>;                             \
+    auto kern = bi_tile3_window_kernel<R, NA, NB, NC, SB, LREG, ALGO, ST, CL, DA>;                         \
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
     if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, kern, p, geo);                                 \
   } while (0)
+  // (a damped call is a separate instantiation, so that the plain update carries none of it)
   if (geo.CS > 1) {
-    if (stale) BI_WIN_LAUNCH(true, true); else BI_WIN_LAUNCH(false, true);
+    if (p.lambda != 1.0) BI_WIN_LAUNCH(false, true, true);
+    else if (stale) BI_WIN_LAUNCH(true, true, false);
+    else BI_WIN_LAUNCH(false, true, false);
   } else {
-    if (stale) BI_WIN_LAUNCH(true, false); else BI_WIN_LAUNCH(false, false);
+    if (p.lambda != 1.0) BI_WIN_LAUNCH(false, false, true);
+    else if (stale) BI_WIN_LAUNCH(true, false, false);
+    else BI_WIN_LAUNCH(false, false, false);
   }
 #undef BI_WIN_LAUNCH
   if (e != cudaSuccess) {

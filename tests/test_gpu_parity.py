@@ -467,3 +467,50 @@ def test_continued_windows(case, algo):
                                act_prev=act_prev[sel])[0]
     assert np.abs(q2[sel] - ref2).max() <= 1e-5
     md.close()
+
+
+# ---- damped updates (bi_model_set_damping)
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "cta", "per_agent"])
+def test_damped_updates(case, algo):
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = {
+        "tile": make_config(2, N=9, T=11, K=6),
+        "tile_cluster": make_config(4, N=4, T=20, K=6),
+        "batch": make_config(3, N=128, T=16, K=6),
+        "warp": _custom(49, [5, 4, 3, 2], [3, 4], [[0, 1], [1, 2, 3]], [2, 2, 1, 2], N=10, T=7, K=6),
+        "cta": make_config(3, N=10, T=7, K=6),
+        "per_agent": _custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=6, G=5),
+    }[case]
+    lam = 0.45
+    md = bi.model_from_workload(w)
+    md.set_damping(lam)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    lq = torch.empty((w.N, w.T, w.S), dtype=torch.float32, device="cuda")
+    q = md.run(algo, obs, act, w.K, logq_out=lq).cpu().numpy()
+    kernel = md.last_kernel
+    assert md.status() == 0
+    sel = list(range(0, w.N, max(1, w.N // 12)))
+    sub = w.take_agents(sel)
+    ref, lref, _ = oracle.run_workload(sub, algo, damping=lam)
+    print(case, algo, kernel, np.abs(q[sel] - ref).max())
+    assert np.abs(q[sel] - ref).max() <= 1e-5
+    big = lref > -30
+    assert np.abs(lq.cpu().numpy()[sel][big] - lref[big]).max() <= 1e-4
+    if algo != "filter":   # damped and warm-started: the first step mixes with ln q_init
+        q_init = _random_beliefs(w, 79)
+        fn = md.bi_vmp_warm if algo == "vmp" else md.bi_mmp_warm
+        q2 = fn(obs, act, torch.from_numpy(q_init).cuda(), w.K).cpu().numpy()
+        ref2 = oracle.run_workload(sub, algo, q_init=q_init[sel].astype(np.float64), damping=lam)[0]
+        assert np.abs(q2[sel] - ref2).max() <= 1e-5
+    # back to the plain update
+    md.set_damping(1.0)
+    q1 = md.run(algo, obs, act, w.K).cpu().numpy()
+    ref1 = oracle.run_workload(sub, algo)[0]
+    assert np.abs(q1[sel] - ref1).max() <= 1e-5
+    with pytest.raises(bi.BiError):
+        md.set_damping(0.0)
+    md.close()
