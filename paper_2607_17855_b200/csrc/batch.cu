@@ -44,6 +44,7 @@ struct BatchMember {
   int32_t dim[BI_MAX_RANK];    // axis sizes, packed order (last one unpadded)
   int32_t ooff[BI_MAX_RANK];   // start of each outer axis in the per-thread shared-memory columns
   int32_t ncp, rows;       // padded last axis; rows = product of the outer axes
+  int64_t gstride;         // elements per agent's model (per-agent models), 0 when shared
   int32_t task0;           // first task slot of this member
 };
 
@@ -57,6 +58,8 @@ struct BatchParams {
   void *ellp;              // [nmem][NU][Sp] partial likelihood messages
   void *qbuf;              // [2][NU][Sp] beliefs
   uint32_t *status;        // the handle's status word
+  const int32_t *obs;      // [NU][M] (per-agent models: every unit reads its own slice)
+  int32_t M, T;
 };
 
 // ---- one unit against one slice: every message of the group in one pass ----
@@ -211,6 +214,16 @@ bi_batch_bucket_kernel(BatchParams P, const int32_t *__restrict__ obs, int M, ui
   }
 }
 
+// Per-agent models: no two units share a slice, so the "buckets" are just runs of consecutive units.
+__global__ void bi_batch_identity_tasks_kernel(BatchParams P, int32_t *perm, int4 *task) {
+  const int mi = blockIdx.y, NU = P.NU, tu = P.tu;
+  const int nchunk = (NU + tu - 1) / tu;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < NU; i += gridDim.x * blockDim.x)
+    perm[(size_t)mi * NU + i] = i;
+  for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < nchunk + P.mem[mi].m; k += gridDim.x * blockDim.x)
+    task[P.mem[mi].task0 + k] = k < nchunk ? make_int4(0, k * tu, min(tu, NU - k * tu), 0) : make_int4(0, 0, 0, 0);
+}
+
 // ---- contraction: one task = one slice, up to kTU units, one thread per unit ----
 template <typename R>
 __global__ void __launch_bounds__(kTU)
@@ -264,7 +277,10 @@ bi_batch_contract_kernel(BatchParams P, int cur) {
 // a contiguous range of the first axis' indices for the same tu units, and the
 // partial messages of the splits are added through shared memory at the end
 // (fixed order: deterministic).
-template <typename R, int NCP>
+// PERUNIT (per-agent models): nothing is shared between units, so nothing is staged; every thread
+// reads the rows of its own unit's slice straight from global memory (consecutive rows of one
+// thread share cache lines, so L1 serves most of the loads).
+template <typename R, int NCP, bool PERUNIT>
 __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__restrict__ slice, R *Lbuf, int lbuf,
                                             R *qs, R *as, int *unit_s, const BatchParams &P, int cur, int4 tk,
                                             int mi) {
@@ -296,17 +312,22 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
 #pragma unroll
   for (int lv = 0; lv < 4; ++lv)
     if (lv < K1) Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * nt + tid];
-  const int lrows = lbuf / rs / NCP;   // rows of one split's staging area
-  R *Lr = Lbuf + (size_t)r * lrows * NCP;
+  const int lrows = PERUNIT ? most : lbuf / rs / NCP;   // rows of one split's staging area (PERUNIT: all at once)
+  R *Lr = Lbuf + (size_t)r * (PERUNIT ? 0 : lrows) * NCP;
   __shared__ __align__(8) unsigned long long bar[8];   // one per split
-  if (tid < rs) bi_mbar_init(&bar[tid], 1);
+  if (!PERUNIT && tid < rs) bi_mbar_init(&bar[tid], 1);
   uint32_t phase = 0;
   bool failed = false;
+  const R *mine = nullptr;   // PERUNIT: this unit's slice
+  if (PERUNIT && has_unit) {
+    const int o = clamp_flag(P.obs[(size_t)unit * P.M + mm.modality], mm.m, P.status, BI_FLAG_OBS_RANGE);
+    mine = (const R *)mm.logA + (size_t)(unit / P.T) * mm.gstride + (size_t)o * mm.P_pad;
+  }
   for (int c0 = 0; c0 < most; c0 += lrows) {
     const int ra = row_a + c0;
     const int nr = max(0, min(lrows, row_b - ra));
-    __syncthreads();   // the previous rows are consumed
-    if (nr > 0) {
+    if (!PERUNIT) __syncthreads();   // the previous rows are consumed
+    if (!PERUNIT && nr > 0) {
       // this split's rows: one bulk asynchronous copy issued by the split's first thread
       if (u == 0) bi_bulk_load(Lr, slice + (size_t)ra * NCP, (uint32_t)(nr * NCP * sizeof(R)), &bar[r]);
       if (!bi_mbar_wait(&bar[r], phase)) {
@@ -318,13 +339,14 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
     if (!has_unit || failed) continue;
     for (int rr = 0; rr < nr; ++rr) {
       constexpr int VE = 16 / (int)sizeof(R);
-      const R *row = Lr + rr * NCP;
+      const R *row = PERUNIT ? mine + (size_t)(ra + rr) * NCP : Lr + rr * NCP;
       const R wf = K1 == 1 ? Wp[0] : K1 == 2 ? Wp[1] : K1 == 3 ? Wp[2] : Wp[3];
       R v0 = (R)0, v1 = (R)0;
 #pragma unroll
       for (int cc = 0; cc < NCP; cc += VE) {
         R x[VE];
-        lds_vec(row + cc, x);
+        if (PERUNIT) ldg_vec(row + cc, x);
+        else lds_vec(row + cc, x);
 #pragma unroll
         for (int i = 0; i < VE; ++i) {
           if (i & 1) v1 = fma(x[i], qc[cc + i], v1);
@@ -385,7 +407,7 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
   }
 }
 
-template <typename R>
+template <typename R, bool PERUNIT>
 __global__ void __launch_bounds__(256)
 bi_batch_contract_rt_kernel(BatchParams P, int cur) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -400,14 +422,14 @@ bi_batch_contract_rt_kernel(BatchParams P, int cur) {
   if (tk.z == 0) return;
   const R *slice = (const R *)mm.logA + (size_t)tk.x * mm.P_pad;
   switch (mm.ncp) {
-    case 4: contract_rt<R, 4>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 8: contract_rt<R, 8>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 12: contract_rt<R, 12>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 16: contract_rt<R, 16>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 20: contract_rt<R, 20>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 24: contract_rt<R, 24>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 28: contract_rt<R, 28>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 32: contract_rt<R, 32>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 4: contract_rt<R, 4, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 8: contract_rt<R, 8, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 12: contract_rt<R, 12, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 16: contract_rt<R, 16, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 20: contract_rt<R, 20, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 24: contract_rt<R, 24, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 28: contract_rt<R, 28, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 32: contract_rt<R, 32, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
     default: break;
   }
 }
@@ -482,6 +504,7 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
   const bool live = unit < NU;    // dead groups shadow the last unit so that whole warps reach the shuffles
   if (!live) unit = NU - 1;
   const int a = unit / T, t = unit - a * T;
+  const int g = md.G == 1 ? 0 : a;   // per-agent models: this agent's matrices and slices
   const R *qc = (const R *)P.qbuf + (size_t)A.cur * NU * Sp;
   R *qn = (R *)P.qbuf + ((size_t)(A.cur ^ 1) * NU + unit) * Sp;
   const int32_t *ob = A.obs + (size_t)unit * M;
@@ -500,20 +523,22 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
       for (uint32_t mk = I.r1mask; mk; mk &= mk - 1) {   // single-factor modalities: the slice is the message
         const BiMember &mm = md.mem[__ffs(mk) - 1];
         const int o = clamp_flag(ob[mm.modality], mm.m, md.status, BI_FLAG_OBS_RANGE);
-        x += __ldg((const R *)mm.logA + (size_t)o * mm.P_pad + s);
+        x += __ldg((const R *)mm.logA + (size_t)g * mm.gstride + (size_t)o * mm.P_pad + s);
       }
       if (t == 0) {
-        x += A.lnprior ? ((const R *)A.lnprior)[(size_t)a * S + I.off + s] : ((const R *)md.logD[f])[s];
+        x += A.lnprior ? ((const R *)A.lnprior)[(size_t)a * S + I.off + s] : ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
       } else {
         const int u = clamp_flag(acp[f], I.U, md.status, BI_FLAG_ACT_RANGE);
         const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);   // [previous][next]
-        const R v = col_dot_g<R>(M0 + (size_t)u * n * np + s, np, qc + (size_t)(unit - 1) * Sp + op, n);
+        const R v = col_dot_g<R>(M0 + (size_t)g * md.Bstride[f] + (size_t)u * n * np + s, np,
+                                 qc + (size_t)(unit - 1) * Sp + op, n);
         x += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
       }
       if (t + 1 < T) {
         const int u = clamp_flag(acp[F + f], I.U, md.status, BI_FLAG_ACT_RANGE);
         const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);   // [next][previous]
-        const R v = col_dot_g<R>(M1 + (size_t)u * n * np + s, np, qc + (size_t)(unit + 1) * Sp + op, n);
+        const R v = col_dot_g<R>(M1 + (size_t)g * md.Bstride[f] + (size_t)u * n * np + s, np,
+                                 qc + (size_t)(unit + 1) * Sp + op, n);
         x += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
       }
     }
@@ -591,7 +616,8 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   memset(&A, 0, sizeof(A));
   // members of rank >= 2, largest slices first (their tasks are the longest)
   int order[BI_MAX_M], cnt = 0;
-  bool any_shape = false;   // some group has no unrolled form: every member takes the any-shape form
+  const bool per_unit = h.G != 1;   // per-agent models: every unit contracts its own slice
+  bool any_shape = per_unit;        // (also set when some group has no unrolled form)
   for (int gi = 0; gi < h.ngroups; ++gi) {
     const BiGroup &g = h.grp[gi];
     if (g.rank < 2) continue;
@@ -610,6 +636,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     const BiGroup &g = h.grp[gi];
     BatchMember &bm = P.mem[j];
     bm.logA = mm.logA; bm.m = mm.m; bm.P_pad = mm.P_pad; bm.modality = mm.modality;
+    bm.gstride = mm.gstride;
     bm.shape = shape_of(g); bm.rank = g.rank;
     int so = 0, rows = 1;
     for (int k = 0; k < g.rank; ++k) {
@@ -684,6 +711,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   P.ellp = w + b_perm + b_task;
   P.qbuf = w + b_perm + b_task + b_ellp;
   P.status = h.status;
+  P.obs = c.obs; P.M = h.M; P.T = c.T;
   A.obs = c.obs; A.act = c.act; A.q_out = c.q_out; A.logq_out = c.logq_out; A.argmax_out = c.argmax_out;
   A.T = c.T;
   A.lnprior = c.lnprior;
@@ -692,9 +720,13 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   A.q_init = c.q_init;
 
   bi_batch_init_kernel<R><<<256, 256, 0, c.stream>>>(md->d, (R *)P.qbuf, NU, c.q_init);
-  if (cnt > 0)
+  if (cnt > 0 && per_unit)
+    bi_batch_identity_tasks_kernel<<<dim3(64, cnt), 256, 0, c.stream>>>(P, perm, task);
+  else if (cnt > 0)
     bi_batch_bucket_kernel<<<cnt, 1024, 2 * max_m * sizeof(int32_t), c.stream>>>(P, c.obs, h.M, h.status, perm, task);
-  void (*contract)(BatchParams, int) = any_shape ? bi_batch_contract_rt_kernel<R> : bi_batch_contract_kernel<R>;
+  void (*contract)(BatchParams, int) = per_unit    ? bi_batch_contract_rt_kernel<R, true>
+                                       : any_shape ? bi_batch_contract_rt_kernel<R, false>
+                                                   : bi_batch_contract_kernel<R>;
   if (cudaFuncSetAttribute((const void *)contract, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csmem) !=
       cudaSuccess)
     return BI_ERR_CUDA;
@@ -739,11 +771,22 @@ int bi_batch_shape(int rank, const int *dim) {
   return rank >= 2 && rank <= 4 ? shape_of(g) : -1;
 }
 
-// Applies to window calls on a shared model with enough (agent, step) units to
-// fill the machine and whose dependency groups all have a compiled shape.
+// Applies to window calls with enough (agent, step) units to fill the machine.  Shared models
+// bucket the units by observed outcome and share a staged slice; per-agent models run the
+// any-shape contraction with every unit reading its own slice.
 int bi_launch_batch(const BiCall &c, bi_model *mut) {
   const bi_model *md = c.model;
-  if (c.algo == BI_ALGO_FILTER || md->h.G != 1) return BI_ERR_UNSUPPORTED;
+  if (c.algo == BI_ALGO_FILTER) return BI_ERR_UNSUPPORTED;
+  if (md->h.G != 1) {
+    // per-agent models: the slices are re-read every iteration, which pays only while they stay in L2
+    // (measured on config 3's model with per-step slices: faster than the warp-per-step kernels at
+    // 112 MB of slices, slower at 224 MB)
+    double bytes = 0;
+    for (int gi = 0; gi < md->h.ngroups; ++gi)
+      if (md->h.grp[gi].rank >= 2) bytes += (double)md->h.grp[gi].P_pad * (md->h.grp[gi].mem_end - md->h.grp[gi].mem_begin);
+    bytes *= (double)c.N * c.T * (md->arith == BI_ARITH_F64 ? 8 : 4);
+    if (bytes > 120e6) return BI_ERR_UNSUPPORTED;
+  }
   if ((long long)c.N * c.T < 2048) return BI_ERR_UNSUPPORTED;
   return md->arith == BI_ARITH_F64 ? launch_batch_t<double>(c, mut) : launch_batch_t<float>(c, mut);
 }

@@ -185,8 +185,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     sh.h.m[k] = T;
   }
   sh.d = reinterpret_cast<BiDev *>(w + off_desc);
-  sh.ws = nullptr;
-  sh.ws_bytes = 0;
+  // (the shadow borrows the handle's batched-path workspace and hands it back below)
   if (cudaMemcpyAsync(sh.d, &sh.h, sizeof(BiDev), cudaMemcpyHostToDevice, stream) != cudaSuccess) return BI_ERR_CUDA;
 
   BiCall c;
@@ -208,6 +207,8 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
   } else {
     rc = bi_dispatch(c, &sh);
   }
+  mut->ws = sh.ws;
+  mut->ws_bytes = sh.ws_bytes;
   mut->launches += launches + (sh.launches - before);
   mut->last_kernel = sh.last_kernel;
   return rc;

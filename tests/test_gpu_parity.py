@@ -514,3 +514,27 @@ def test_damped_updates(case, algo):
     with pytest.raises(bi.BiError):
         md.set_damping(0.0)
     md.close()
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_batched_window_with_per_agent_models(algo):
+    # per-agent models without a register tile: every unit contracts its own slice
+    w = _custom(52, [5, 7, 3, 4], [4, 3, 5], [[0, 1, 3], [1, 2], [2]], [2, 1, 3, 2], N=140, T=16, K=5, G=140,
+                sparsity=0.5)
+    res = check_workload(w, algo, agents=range(0, 140, 7))
+    assert res["kernel"] == f"batch_{algo}_f64", res
+    # the same through observation vectors on a shared model (slices become per agent and step)
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = make_config(3, N=130, T=16, K=4)            # 130 x 16 x 5460 x 8 B = 91 MB of slices: L2-resident
+    md = bi.model_from_workload(w)
+    soft = _soft_vectors(w, 6)
+    q = md.run_soft(algo, torch.from_numpy(soft).cuda(), torch.from_numpy(w.act).cuda(), w.K).cpu().numpy()
+    assert md.last_kernel == f"batch_{algo}_f64", md.last_kernel
+    sel = list(range(0, 130, 13))
+    sub = w.take_agents(sel)
+    ref = oracle.run(algo, sub.n, sub.m, sub.dep, sub.U, sub.G, sub.A, sub.B, sub.D, None, sub.act, sub.K,
+                     obs_soft=soft[sel])[0]
+    assert np.abs(q[sel] - ref).max() <= 1e-5
+    md.close()
