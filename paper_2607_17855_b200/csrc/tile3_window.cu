@@ -222,6 +222,8 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     // and half the logarithms per lane.
     R ta, tb, tc;
     {
+      // row strides of the staged matrices: each factor's padded state count, known at compile time
+      constexpr int NPA = (NA + 3) & ~3, NPB = (NB + 3) & ~3, NPC = (NC + 3) & ~3;
       const R *qp = q_cur - SQ, *qn = q_cur + SQ;
       const bool has_prev = t > 0, has_next = t + 1 < T;
       auto edge = [&](R dot, bool future, R prior) -> R {
@@ -231,27 +233,27 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       constexpr bool DUPA = SB >= 2, DUPB = !TT::TP && TT::SHB >= 1, DUPC = !TT::TP && TT::SHC >= 1;
       if (DUPA) {
         const bool fut = (t3.u & 1) != 0;   // u = a * SB + bh: the lowest bit tells the two apart
-        const R v = edge(col_dot_smem<R, NA>(fut ? fu0 : pa0, p.np[0], fut ? qn : qp), fut, dprior[0]);
+        const R v = edge(col_dot_smem<R, NA>(fut ? fu0 : pa0, NPA, fut ? qn : qp), fut, dprior[0]);
         ta = v + __shfl_xor_sync(0xffffffffu, v, 1);
       } else {
-        ta = edge(col_dot_smem<R, NA>(pa0, p.np[0], qp), false, dprior[0]) +
-             edge(col_dot_smem<R, NA>(fu0, p.np[0], qn), true, (R)0);
+        ta = edge(col_dot_smem<R, NA>(pa0, NPA, qp), false, dprior[0]) +
+             edge(col_dot_smem<R, NA>(fu0, NPA, qn), true, (R)0);
       }
       if (DUPB) {
         const bool fut = (a & 1) != 0;      // duplicates of a b owner differ in the low bits of a
-        const R v = edge(col_dot_smem<R, NB>(fut ? fu1 : pa1, p.np[1], (fut ? qn : qp) + NA), fut, dprior[1]);
+        const R v = edge(col_dot_smem<R, NB>(fut ? fu1 : pa1, NPB, (fut ? qn : qp) + NA), fut, dprior[1]);
         tb = v + __shfl_xor_sync(0xffffffffu, v, SB);
       } else {
-        tb = edge(col_dot_smem<R, NB>(pa1, p.np[1], qp + NA), false, dprior[1]) +
-             edge(col_dot_smem<R, NB>(fu1, p.np[1], qn + NA), true, (R)0);
+        tb = edge(col_dot_smem<R, NB>(pa1, NPB, qp + NA), false, dprior[1]) +
+             edge(col_dot_smem<R, NB>(fu1, NPB, qn + NA), true, (R)0);
       }
       if (DUPC) {
         const bool fut = (t3.u & 1) != 0;   // duplicates of a c owner differ in the low bits of u
-        const R v = edge(col_dot_smem<R, NC>(fut ? fu2 : pa2, p.np[2], (fut ? qn : qp) + NA + NB), fut, dprior[2]);
+        const R v = edge(col_dot_smem<R, NC>(fut ? fu2 : pa2, NPC, (fut ? qn : qp) + NA + NB), fut, dprior[2]);
         tc = v + __shfl_xor_sync(0xffffffffu, v, 1);
       } else {
-        tc = edge(col_dot_smem<R, NC>(pa2, p.np[2], qp + NA + NB), false, dprior[2]) +
-             edge(col_dot_smem<R, NC>(fu2, p.np[2], qn + NA + NB), true, (R)0);
+        tc = edge(col_dot_smem<R, NC>(pa2, NPC, qp + NA + NB), false, dprior[2]) +
+             edge(col_dot_smem<R, NC>(fu2, NPC, qn + NA + NB), true, (R)0);
       }
     }
     if (LREG) t3.messages(xa, xb, xc);
