@@ -206,16 +206,22 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     if (DAMPED) pxb = b_ok ? bi_log(bi_max(qs[NA + bsafe], (R)BI_EPS)) : (R)0;
     if (DAMPED) pxc = c_ok ? bi_log(bi_max(qs[NA + NB + csafe], (R)BI_EPS)) : (R)0;
   }
-  if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
+  // The barrier between iterations is split: a CTA arrives as soon as its beliefs are published and
+  // waits only when it needs its neighbours', with the contraction (own data only) in between.
+  // (A launch without a cluster attribute is a cluster of one CTA, so the same barrier serves both.)
+  cg::this_cluster().barrier_arrive();
 
   R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
   float ma = 0.f, mb = 0.f, mc = 0.f, pma = 0.f, pmb = 0.f, pmc = 0.f;
   for (int k = 0; k < p.K; ++k) {
+    // likelihood messages from this step's own beliefs, while the other CTAs finish publishing theirs
+    if (LREG) t3.messages(xa, xb, xc);
+    else t3.messages_smem(Lt, xa, xb, xc);
+    cg::this_cluster().barrier_wait();
     // Transition messages from the previous iterate of the neighbouring steps.
     // Both edges are evaluated without branches (a window's first and last
     // step read their halo slot, which always holds valid beliefs, and discard
-    // the result), so this code and the contraction below form one
-    // straight-line block and their dependency chains interleave.
+    // the result).
     // Where a state is owned by two or more lanes of the group (more lanes than
     // states), one of them evaluates the past edge and its neighbour the future
     // edge at the same time, and a shuffle adds the two: half the dot products
@@ -256,8 +262,6 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
              edge(col_dot_smem<R, NC>(fu2, NPC, qn + NA + NB), true, (R)0);
       }
     }
-    if (LREG) t3.messages(xa, xb, xc);
-    else t3.messages_smem(Lt, xa, xb, xc);
     xa = a_ok ? xa + ta : -bi_inf<R>();
     xb = b_ok ? xb + tb : -bi_inf<R>();
     xc = c_ok ? xc + tc : -bi_inf<R>();
@@ -340,8 +344,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     { R *tmp = q_cur; q_cur = q_nxt; q_nxt = tmp; }
     { R *tmp = r_prev_cur; r_prev_cur = r_prev_nxt; r_prev_nxt = tmp; }
     { R *tmp = r_next_cur; r_next_cur = r_next_nxt; r_next_nxt = tmp; }
-    if (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
+    cg::this_cluster().barrier_arrive();
   }
+  cg::this_cluster().barrier_wait();   // nobody leaves while a neighbour may still write into its halo
 }
 
 template <typename R, int NA, int NB, int NC, int SB, bool LREG, int ALGO>
