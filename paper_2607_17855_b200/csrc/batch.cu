@@ -26,6 +26,14 @@
 
 namespace {
 
+// Programmatic dependent launch: the iteration loop queues its kernels so that the next one may be
+// scheduled while the previous one drains.  A kernel first does what needs none of its
+// predecessor's results (its task, the slice copy, index loads), then waits for the predecessor to
+// complete (bi_grid_wait; a no-op when launched without the attribute) and only then lets its own
+// successor be scheduled: when a kernel starts, everything before its predecessor is complete.
+__device__ __forceinline__ void bi_grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void bi_grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 constexpr int kTU = 128;   // most units per contraction CTA (the call picks 32, 64 or 128)
 
 // packed dims of the compiled group shapes: rank, then the axis sizes (last axis unpadded)
@@ -227,14 +235,20 @@ __global__ void bi_batch_identity_tasks_kernel(BatchParams P, int32_t *perm, int
 // ---- contraction: one task = one slice, up to kTU units, one thread per unit ----
 template <typename R>
 __global__ void __launch_bounds__(kTU)
-bi_batch_contract_kernel(BatchParams P, int cur) {
+bi_batch_contract_kernel(BatchParams P, int cur, int first) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *L = reinterpret_cast<R *>(smem_raw);
+  if (first) {   // the tasks were written by the kernel just before this one
+    bi_grid_wait();
+    bi_grid_launch_dependents();
+  }
   int mi = 0;
   while (mi + 1 < P.nmem && (int)blockIdx.x >= P.mem[mi + 1].task0) ++mi;
   const BatchMember &mm = P.mem[mi];
   const int4 tk = P.task[blockIdx.x];
-  if (tk.z == 0) return;
+  if (tk.z == 0) {   // an unused task slot (an exiting CTA counts as having released its dependents)
+    return;
+  }
   // stage the slice of outcome tk.x: one bulk asynchronous copy, global -> shared, issued by one
   // thread; the others meanwhile look up their unit
   __shared__ __align__(8) unsigned long long bar;
@@ -246,6 +260,10 @@ bi_batch_contract_kernel(BatchParams P, int cur) {
   const int unit = has_unit ? P.perm[(size_t)mi * P.NU + tk.y + threadIdx.x] : 0;
   const R *q = (const R *)P.qbuf + ((size_t)cur * P.NU + unit) * P.Sp;
   R *out = (R *)P.ellp + ((size_t)mi * P.NU + unit) * P.Sp;
+  if (!first) {   // beliefs of the previous update, and the right to overwrite the messages it read
+    bi_grid_wait();
+    bi_grid_launch_dependents();
+  }
   if (!bi_mbar_wait(&bar, 0)) {
     if (threadIdx.x == 0) atomicOr(P.status, BI_FLAG_COPY_TIMEOUT);
     return;
@@ -409,7 +427,11 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
 
 template <typename R, bool PERUNIT>
 __global__ void __launch_bounds__(256)
-bi_batch_contract_rt_kernel(BatchParams P, int cur) {
+bi_batch_contract_rt_kernel(BatchParams P, int cur, int first) {
+  // (this form reads beliefs from its first instruction on, so it waits at once)
+  bi_grid_wait();
+  bi_grid_launch_dependents();
+  (void)first;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *Lbuf = reinterpret_cast<R *>(smem_raw);
   R *qs = Lbuf + P.lbuf;
@@ -499,6 +521,8 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
     fi[f] = x;
   }
   __syncthreads();
+  bi_grid_wait();   // the contraction's messages (and, for the beliefs, everything before it)
+  bi_grid_launch_dependents();
   const int sub = threadIdx.x / LW, s = threadIdx.x % LW;
   int unit = blockIdx.x * UPB + sub;
   const bool live = unit < NU;    // dead groups shadow the last unit so that whole warps reach the shuffles
@@ -724,7 +748,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     bi_batch_identity_tasks_kernel<<<dim3(64, cnt), 256, 0, c.stream>>>(P, perm, task);
   else if (cnt > 0)
     bi_batch_bucket_kernel<<<cnt, 1024, 2 * max_m * sizeof(int32_t), c.stream>>>(P, c.obs, h.M, h.status, perm, task);
-  void (*contract)(BatchParams, int) = per_unit    ? bi_batch_contract_rt_kernel<R, true>
+  void (*contract)(BatchParams, int, int) = per_unit    ? bi_batch_contract_rt_kernel<R, true>
                                        : any_shape ? bi_batch_contract_rt_kernel<R, false>
                                                    : bi_batch_contract_kernel<R>;
   if (cudaFuncSetAttribute((const void *)contract, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csmem) !=
@@ -745,13 +769,29 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   else
     update = lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 8>
                      : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 16> : bi_batch_update_kernel<R, BI_ALGO_MMP, 32>;
+  // every launch of the loop may be scheduled while its predecessor drains (see bi_grid_wait)
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
   for (int k = 0; k < c.K; ++k) {
     const int cur = k & 1;
-    if (cnt > 0) contract<<<ntask, tu * rs, csmem, c.stream>>>(P, cur);
     A.cur = cur;
     A.final = (k == c.K - 1);
     A.first = (k == 0);
-    update<<<(NU + upb - 1) / upb, 128, 0, c.stream>>>(md->d, P, A);
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = c.stream;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    if (cnt > 0) {
+      cfg.gridDim = dim3((unsigned)ntask);
+      cfg.blockDim = dim3((unsigned)(tu * rs));
+      cfg.dynamicSmemBytes = csmem;
+      if (cudaLaunchKernelEx(&cfg, contract, P, cur, (int)(k == 0)) != cudaSuccess) return BI_ERR_CUDA;
+    }
+    cfg.gridDim = dim3((unsigned)((NU + upb - 1) / upb));
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0;
+    if (cudaLaunchKernelEx(&cfg, update, (const BiDev *)md->d, P, A) != cudaSuccess) return BI_ERR_CUDA;
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += cnt > 0 ? 2 + 2 * c.K : 1 + c.K;
