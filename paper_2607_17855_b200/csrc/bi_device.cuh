@@ -78,6 +78,36 @@ __device__ __forceinline__ double bi_exp_inline(double x) {
 }
 __device__ __forceinline__ float bi_exp_inline(float x) { return expf(x); }
 
+// The same with a 32-entry table of 2^(j/32) (in shared memory: tab): the reduced
+// argument is then below ln2/64 and a degree-6 polynomial suffices, 13 FP64
+// operations instead of 19.  exp(x) = 2^(k>>5) * tab[k&31] * exp(r),
+// k = round(x * 32/ln2), r = x - k ln2/32.  Same range and accuracy.
+__device__ __forceinline__ double bi_exp_tab(double x, const double *tab) {
+  const double K32 = 46.166241308446828384, LH = 6.93147180369123816490e-01 / 32.0, LL = 1.90821492927058770002e-10 / 32.0;
+  const double MAGIC = 6755399441055744.0;
+  double t = fma(x, K32, MAGIC);
+  const int k = __double2loint(t);
+  const double kd = t - MAGIC;
+  double r = fma(kd, -LH, x);
+  r = fma(kd, -LL, r);
+  const double T = tab[k & 31];
+  const double r2 = r * r;
+  const double a = fma(r, 1.0 / 6.0, 0.5);
+  double b = fma(r, 1.0 / 120.0, 1.0 / 24.0);
+  b = fma(r2, 1.0 / 720.0, b);
+  const double c = fma(r2, b, a);
+  const double p = fma(r2, c, r);
+  const double res = fma(T, p, T);
+  const double out = __hiloint2double(__double2hiint(res) + ((k >> 5) << 20), __double2loint(res));
+  return x < -700.0 ? 0.0 : out;
+}
+__device__ __forceinline__ float bi_exp_tab(float x, const float *) { return expf(x); }
+// fills tab[0..32) with 2^(j/32); call with at least 32 threads, then synchronise them
+__device__ __forceinline__ void bi_exp_tab_init(double *tab, int lane) {
+  if (lane < 32) tab[lane] = exp2((double)lane / 32.0);
+}
+__device__ __forceinline__ void bi_exp_tab_init(float *, int) {}
+
 // Branch-free natural log of a positive normal double (the messages take logs
 // of probabilities clamped at 1e-16 and of sums of exponentials: never zero,
 // subnormal, infinite or NaN).  Same motive as bi_exp_inline: the six logs of
@@ -115,6 +145,7 @@ __device__ __forceinline__ double bi_log_inline(double x) {
   return dk * ln2_hi - ((hfsq - (s * (hfsq + (t2 + t1)) + dk * ln2_lo)) - f);
 }
 __device__ __forceinline__ float bi_log_inline(float x) { return logf(x); }
+
 __device__ __forceinline__ float bi_log(float x) { return logf(x); }
 __device__ __forceinline__ double bi_log(double x) { return log(x); }
 

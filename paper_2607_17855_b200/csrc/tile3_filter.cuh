@@ -20,6 +20,8 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
   __shared__ __align__(16) R sm_L[LSMEM ? UPW : 1][LSMEM ? TT::P_TILE : 2];  // large tiles: the step's slice
   __shared__ __align__(16) R sm_tp[UPW][TT::TP ? TT::TP_UNIT : 2];           // transpose area of the b / c sums
 
+  __shared__ R exp_tab[32];   // 2^(j/32) for the table-driven exponential
+  bi_exp_tab_init(exp_tab, (int)threadIdx.x);
   const int lane = threadIdx.x;
   const int unit = lane / LPU;
   int agent = blockIdx.x * UPW + unit;
@@ -145,9 +147,9 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
         mb = group_max_f<LPU, 1>((float)xb);
         mc = group_max_f<LPU, 1>((float)xc);
       }
-      const R ean = a_ok ? bi_exp_inline(xa - (R)ma) : (R)0;
-      const R ebn = b_ok ? bi_exp_inline(xb - (R)mb) : (R)0;
-      const R ecn = c_ok ? bi_exp_inline(xc - (R)mc) : (R)0;
+      const R ean = a_ok ? bi_exp_tab(xa - (R)ma, exp_tab) : (R)0;
+      const R ebn = b_ok ? bi_exp_tab(xb - (R)mb, exp_tab) : (R)0;
+      const R ecn = c_ok ? bi_exp_tab(xc - (R)mc, exp_tab) : (R)0;
       if (t3.own_b) se[bi] = ebn;
       if (t3.own_c) se[NB + ci] = ecn;
       if (TT::TP && t3.own_a) se[NB + NCP + a] = ean;

@@ -60,6 +60,8 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   R *seb = Ls + geo.off_se;                  // [units][NB + NCP] gathered e_b, e_c
   R *Bs = Ls + geo.off_B;                    // this agent's transition matrices, every action
 
+  __shared__ R exp_tab[32];   // 2^(j/32) for the table-driven exponential (synchronised with the staging below)
+  bi_exp_tab_init(exp_tab, (int)threadIdx.x);
   int rank = 0;
   if (CLUSTER) rank = (int)cg::this_cluster().block_rank();
   const int agent = blockIdx.x / geo.CS;
@@ -277,9 +279,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     if (!STALE || k == 0) { ma = cma; mb = cmb; mc = cmc; }
     else { ma = pma; mb = pmb; mc = pmc; }
     pma = cma; pmb = cmb; pmc = cmc;
-    const R ean = a_ok ? bi_exp_inline(xa - (R)ma) : (R)0;
-    const R ebn = b_ok ? bi_exp_inline(xb - (R)mb) : (R)0;
-    const R ecn = c_ok ? bi_exp_inline(xc - (R)mc) : (R)0;
+    const R ean = a_ok ? bi_exp_tab(xa - (R)ma, exp_tab) : (R)0;
+    const R ebn = b_ok ? bi_exp_tab(xb - (R)mb, exp_tab) : (R)0;
+    const R ecn = c_ok ? bi_exp_tab(xc - (R)mc, exp_tab) : (R)0;
     __syncwarp();
     if (t3.own_b) se[bi] = ebn;
     if (t3.own_c) se[NB + ci] = ecn;
