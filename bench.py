@@ -338,6 +338,26 @@ def main():
                 "kernel": head["kernel"],
                 "peak_source": f"derived: 148 SMs x {64 if args.arith == 'f64' else 128} lanes x 2 x 1.965 GHz"}
     roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(head["kernel"])
+    # the same run's own measurements beside the derived peak: the rate of independent multiply-add
+    # chains in this arithmetic, and a large device-to-device copy
+    try:
+        fma_peak = bi.bi_probe_fma(args.arith)
+        src = torch.empty(1 << 28, dtype=torch.float32, device="cuda")   # 1 GiB
+        dst = torch.empty_like(src)
+        for _ in range(2):
+            dst.copy_(src)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(5):
+            dst.copy_(src)
+        ev1.record()
+        ev1.synchronize()
+        copy_gbs = 5 * 2 * src.numel() * 4 / (ev0.elapsed_time(ev1) * 1e-3) / 1e9
+        del src, dst
+        roofline["measured_in_this_run"] = {"fma_tflops": fma_peak, "frac_of_fma": achieved / fma_peak,
+                                            "copy_gbs": copy_gbs}
+    except Exception as exc:  # noqa: BLE001  (a measurement aid must not fail the benchmark)
+        roofline["measured_in_this_run"] = {"error": str(exc)}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -303,6 +303,15 @@ int bi_filter_static(const bi_model_desc *desc, int32_t N, int32_t T, const int3
                      const int32_t *act, int32_t iters, float *q_out, float *logq_out,
                      int32_t *argmax_out, void *cuda_stream);
 
+/*
+ * Measurement aid (no part of the method): times a kernel of independent
+ * multiply-add chains in the given arithmetic (BI_ARITH_*) on the current device
+ * and returns the rate in TFLOP/s in *tflops (HOST), so that a benchmark can set
+ * its achieved arithmetic against a peak measured in the same run.  Allocates one
+ * word of device memory for the duration of the call and synchronises the stream.
+ */
+int bi_probe_fma(int arith, double *tflops, void *cuda_stream);
+
 /* Synchronises the stream, returns the OR of BI_FLAG_* raised since the last
  * call in *flags (HOST) and clears them. */
 int bi_status(const bi_model_t *model, void *cuda_stream, uint32_t *flags);

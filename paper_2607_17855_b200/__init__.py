@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_probe_fma", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -83,6 +83,8 @@ def lib():
                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.bi_model_set_damping.restype = ctypes.c_int
         L.bi_model_set_damping.argtypes = [ctypes.c_void_p, ctypes.c_double]
+        L.bi_probe_fma.restype = ctypes.c_int
+        L.bi_probe_fma.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
         L.bi_status.restype = ctypes.c_int
         L.bi_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
         L.bi_last_kernel.restype = ctypes.c_char_p
@@ -285,6 +287,15 @@ class Model:
     @property
     def launch_count(self) -> int:
         return int(lib().bi_launch_count(self._h))
+
+
+def bi_probe_fma(arith: str = "f64", stream=None) -> float:
+    """Measured multiply-add rate of this GPU in TFLOP/s (``bi_probe_fma``; a measurement aid)."""
+    v = ctypes.c_double(0.0)
+    rc = lib().bi_probe_fma(ARITH[arith], ctypes.byref(v), _stream_ptr(stream))
+    if rc != BI_OK:
+        raise BiError(rc, "bi_probe_fma")
+    return float(v.value)
 
 
 def bi_filter_static(n, m, dep, U, A, B, D, obs, act, iters, q_out, logq_out=None, argmax_out=None, stream=None):

@@ -538,3 +538,9 @@ def test_batched_window_with_per_agent_models(algo):
                      obs_soft=soft[sel])[0]
     assert np.abs(q[sel] - ref).max() <= 1e-5
     md.close()
+
+
+def test_fma_probe_reports_a_plausible_rate():
+    import paper_2607_17855_b200 as bi
+    f64, f32 = bi.bi_probe_fma("f64"), bi.bi_probe_fma("f32")
+    assert 1.0 < f64 < 200.0 and f64 < f32 < 400.0, (f64, f32)
