@@ -165,35 +165,60 @@ __device__ __forceinline__ void slice_table(const BiDev &md, int g, const int32_
   __syncwarp();
 }
 
+// reductions over the NW lanes that hold a factor's states (NW: the power of two at or above n, at
+// least 4): a small factor needs two or three shuffle steps, not five
+template <int NW, typename T>
+__device__ __forceinline__ T group_sum_w(T v) {
+#pragma unroll
+  for (int o = NW / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+template <int NW, typename T>
+__device__ __forceinline__ T group_max_w(T v) {
+#pragma unroll
+  for (int o = NW / 2; o > 0; o >>= 1) v = bi_max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+template <typename R, int NW>
+__device__ __forceinline__ void softmax_factor(const BiDev &md, int f, const R *ell, R *qn, bool final, float *q_out,
+                                               float *logq_out, int32_t *argmax_out, int lane, R *xp, R lam) {
+  const int n = md.n[f], op = md.offp[f];
+  R x = lane < n ? ell[op + lane] : -bi_inf<R>();
+  if (xp && lane < n) {   // damped step on the logits; xp: the previous iterate's
+    x = fma(lam, x, ((R)1 - lam) * xp[op + lane]);
+    xp[op + lane] = x;
+  }
+  // the shift only has to be close to the maximum (softmax is shift
+  // invariant): a float reduction halves the shuffles of a double one
+  R mx = final ? group_max_w<NW>(x) : (R)group_max_w<NW>((float)x);
+  R e = lane < n ? bi_exp_inline(x - mx) : (R)0;
+  R z = group_sum_w<NW>(e);
+  R q = e * bi_rcp(z);
+  if (lane < md.npad[f]) qn[op + lane] = lane < n ? q : (R)0;
+  if (final) {
+    if (lane < n) {
+      q_out[md.off[f] + lane] = (float)q;
+      if (logq_out) logq_out[md.off[f] + lane] = (float)(x - mx - bi_log(z));
+    }
+    if (argmax_out) {
+      unsigned b = __ballot_sync(0xffffffffu, lane < n && x == mx);
+      if (lane == 0) argmax_out[f] = __ffs(b) - 1;
+    }
+  }
+}
+
 // softmax of every factor of one step from the logits in ell
 template <typename R>
 __device__ __forceinline__ void softmax_warp(const BiDev &md, const R *ell, R *qn, bool final, float *q_out,
                                              float *logq_out, int32_t *argmax_out, int lane, R *xp = nullptr,
                                              R lam = (R)1) {
   for (int f = 0; f < md.F; ++f) {
-    const int n = md.n[f], op = md.offp[f];
-    R x = lane < n ? ell[op + lane] : -bi_inf<R>();
-    if (xp && lane < n) {   // damped step on the logits; xp: the previous iterate's
-      x = fma(lam, x, ((R)1 - lam) * xp[op + lane]);
-      xp[op + lane] = x;
-    }
-    // the shift only has to be close to the maximum (softmax is shift
-    // invariant): a float reduction halves the shuffles of a double one
-    R mx = final ? warp_max(x) : (R)warp_max((float)x);
-    R e = lane < n ? bi_exp_inline(x - mx) : (R)0;
-    R z = warp_sum(e);
-    R q = e * bi_rcp(z);
-    if (lane < md.npad[f]) qn[op + lane] = lane < n ? q : (R)0;
-    if (final) {
-      if (lane < n) {
-        q_out[md.off[f] + lane] = (float)q;
-        if (logq_out) logq_out[md.off[f] + lane] = (float)(x - mx - bi_log(z));
-      }
-      if (argmax_out) {
-        unsigned b = __ballot_sync(0xffffffffu, lane < n && x == mx);
-        if (lane == 0) argmax_out[f] = __ffs(b) - 1;
-      }
-    }
+    const int n = md.n[f];
+    if (n <= 4) softmax_factor<R, 4>(md, f, ell, qn, final, q_out, logq_out, argmax_out, lane, xp, lam);
+    else if (n <= 8) softmax_factor<R, 8>(md, f, ell, qn, final, q_out, logq_out, argmax_out, lane, xp, lam);
+    else if (n <= 16) softmax_factor<R, 16>(md, f, ell, qn, final, q_out, logq_out, argmax_out, lane, xp, lam);
+    else softmax_factor<R, 32>(md, f, ell, qn, final, q_out, logq_out, argmax_out, lane, xp, lam);
   }
   __syncwarp();
 }
