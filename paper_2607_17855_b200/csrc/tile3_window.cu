@@ -43,6 +43,29 @@ __device__ __forceinline__ R col_dot_smem(const R *col, int stride, const R *q) 
   return s0 + s1;
 }
 
+// the same with the column held in registers; the beliefs are read two at a time where their
+// offset allows (broadcast loads: half the shared-memory wavefronts)
+template <typename R, int N, bool PAIRS>
+__device__ __forceinline__ R reg_dot_smem(const R (&col)[N], const R *q) {
+  R s0 = (R)0, s1 = (R)0;
+  if constexpr (PAIRS && sizeof(R) == 8) {
+#pragma unroll
+    for (int r = 0; r + 1 < N; r += 2) {
+      const double2 x = *reinterpret_cast<const double2 *>(q + r);
+      s0 = fma(col[r], x.x, s0);
+      s1 = fma(col[r + 1], x.y, s1);
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r + 1 < N; r += 2) {
+      s0 = fma(col[r], q[r], s0);
+      s1 = fma(col[r + 1], q[r + 1], s1);
+    }
+  }
+  if (N & 1) s0 = fma(col[N - 1], q[N - 1], s0);
+  return s0 + s1;
+}
+
 // LREG: the step's summed slice lives in registers (small tiles); otherwise in
 // shared memory (tiles too large for the register file).
 template <typename R, int NA, int NB, int NC, int SB, bool LREG, int ALGO, bool STALE, bool CLUSTER, bool DAMPED>
@@ -208,6 +231,34 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     if (DAMPED) pxb = b_ok ? bi_log(bi_max(qs[NA + bsafe], (R)BI_EPS)) : (R)0;
     if (DAMPED) pxc = c_ok ? bi_log(bi_max(qs[NA + NB + csafe], (R)BI_EPS)) : (R)0;
   }
+  // With the slices in shared memory the register file has room for the transition-matrix column
+  // of each owned state (for the one edge this lane evaluates): they do not change between
+  // iterations, and reading them from shared memory again every time was a third of the
+  // kernel's shared-memory traffic.
+  constexpr int NPA_ = (NA + 3) & ~3, NPB_ = (NB + 3) & ~3, NPC_ = (NC + 3) & ~3;
+  constexpr bool DUPA_ = SB >= 2, DUPB_ = !TT::TP && TT::SHB >= 1, DUPC_ = !TT::TP && TT::SHC >= 1;
+  // (the a and b columns: with the c column as well the kernel spills at the 168 registers a
+  // ten-warp CTA may use, and measured slower)
+  constexpr bool BRA = !LREG && DUPA_, BRB = !LREG && DUPB_, BRC = false;
+  R bca[BRA ? NA : 1], bcb[BRB ? NB : 1], bcc[BRC ? NC : 1];
+  if (BRA || BRB || BRC) {
+    __syncthreads();
+    if (BRA) {
+      const R *col = (t3.u & 1) ? fu0 : pa0;
+#pragma unroll
+      for (int r = 0; r < (BRA ? NA : 1); ++r) bca[r] = col[r * NPA_];
+    }
+    if (BRB) {
+      const R *col = (a & 1) ? fu1 : pa1;
+#pragma unroll
+      for (int r = 0; r < (BRB ? NB : 1); ++r) bcb[r] = col[r * NPB_];
+    }
+    if (BRC) {
+      const R *col = (t3.u & 1) ? fu2 : pa2;
+#pragma unroll
+      for (int r = 0; r < (BRC ? NC : 1); ++r) bcc[r] = col[r * NPC_];
+    }
+  }
   // The barrier between iterations is split: a CTA arrives as soon as its beliefs are published and
   // waits only when it needs its neighbours', with the contraction (own data only) in between.
   // (A launch without a cluster attribute is a cluster of one CTA, so the same barrier serves both.)
@@ -241,7 +292,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       constexpr bool DUPA = SB >= 2, DUPB = !TT::TP && TT::SHB >= 1, DUPC = !TT::TP && TT::SHC >= 1;
       if (DUPA) {
         const bool fut = (t3.u & 1) != 0;   // u = a * SB + bh: the lowest bit tells the two apart
-        const R v = edge(col_dot_smem<R, NA>(fut ? fu0 : pa0, NPA, fut ? qn : qp), fut, dprior[0]);
+        const R dot = BRA ? reg_dot_smem<R, BRA ? NA : 1, true>(bca, fut ? qn : qp)
+                          : col_dot_smem<R, NA>(fut ? fu0 : pa0, NPA, fut ? qn : qp);
+        const R v = edge(dot, fut, dprior[0]);
         ta = v + __shfl_xor_sync(0xffffffffu, v, 1);
       } else {
         ta = edge(col_dot_smem<R, NA>(pa0, NPA, qp), false, dprior[0]) +
@@ -249,7 +302,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       }
       if (DUPB) {
         const bool fut = (a & 1) != 0;      // duplicates of a b owner differ in the low bits of a
-        const R v = edge(col_dot_smem<R, NB>(fut ? fu1 : pa1, NPB, (fut ? qn : qp) + NA), fut, dprior[1]);
+        const R dot = BRB ? reg_dot_smem<R, BRB ? NB : 1, NA % 2 == 0>(bcb, (fut ? qn : qp) + NA)
+                          : col_dot_smem<R, NB>(fut ? fu1 : pa1, NPB, (fut ? qn : qp) + NA);
+        const R v = edge(dot, fut, dprior[1]);
         tb = v + __shfl_xor_sync(0xffffffffu, v, SB);
       } else {
         tb = edge(col_dot_smem<R, NB>(pa1, NPB, qp + NA), false, dprior[1]) +
@@ -257,7 +312,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       }
       if (DUPC) {
         const bool fut = (t3.u & 1) != 0;   // duplicates of a c owner differ in the low bits of u
-        const R v = edge(col_dot_smem<R, NC>(fut ? fu2 : pa2, NPC, (fut ? qn : qp) + NA + NB), fut, dprior[2]);
+        const R dot = BRC ? reg_dot_smem<R, BRC ? NC : 1, (NA + NB) % 2 == 0>(bcc, (fut ? qn : qp) + NA + NB)
+                          : col_dot_smem<R, NC>(fut ? fu2 : pa2, NPC, (fut ? qn : qp) + NA + NB);
+        const R v = edge(dot, fut, dprior[2]);
         tc = v + __shfl_xor_sync(0xffffffffu, v, 1);
       } else {
         tc = edge(col_dot_smem<R, NC>(pa2, NPC, qp + NA + NB), false, dprior[2]) +
@@ -288,10 +345,23 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     za = group_sum<R, NAP, SB>(ean);
     __syncwarp();
     t3.ea = ean;
+    if constexpr (sizeof(R) == 8 && NBL % 2 == 0 && NB % 2 == 0) {   // 16-byte broadcast loads
 #pragma unroll
-    for (int bl = 0; bl < NBL; ++bl) t3.eb[bl] = se[t3.bh * NBL + bl];
+      for (int bl = 0; bl < NBL; bl += 2) {
+        const double2 x = *reinterpret_cast<const double2 *>(se + t3.bh * NBL + bl);
+        t3.eb[bl] = x.x; t3.eb[bl + 1] = x.y;
+      }
 #pragma unroll
-    for (int c = 0; c < NCP; ++c) t3.ec[c] = se[NB + c];
+      for (int c = 0; c < NCP; c += 2) {
+        const double2 x = *reinterpret_cast<const double2 *>(se + NB + c);
+        t3.ec[c] = x.x; t3.ec[c + 1] = x.y;
+      }
+    } else {
+#pragma unroll
+      for (int bl = 0; bl < NBL; ++bl) t3.eb[bl] = se[t3.bh * NBL + bl];
+#pragma unroll
+      for (int c = 0; c < NCP; ++c) t3.ec[c] = se[NB + c];
+    }
     zb = group_sum<R, SB, 1>(tree_sum<R, NBL>(t3.eb));
     zc = tree_sum<R, NCP>(t3.ec);
     rinv = bi_rcp(za * zb * zc);
@@ -372,6 +442,15 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   // hide the per-iteration barrier).  BI_WINDOW_CS (testing aid) forces a size.
   int cs_force = 0;
   if (const char *e = getenv("BI_WINDOW_CS")) cs_force = atoi(e);
+  const bool stale = sizeof(R) == 8 && p.nmem <= 12;
+  // (a damped call is a separate instantiation, so that the plain update carries none of it)
+  auto pick = [&](bool cl) -> const void * {
+#define BI_WIN_KERN(ST, CL, DA) ((const void *)bi_tile3_window_kernel<R, NA, NB, NC, SB, LREG, ALGO, ST, CL, DA>)
+    if (p.lambda != 1.0) return cl ? BI_WIN_KERN(false, true, true) : BI_WIN_KERN(false, false, true);
+    if (stale) return cl ? BI_WIN_KERN(true, true, false) : BI_WIN_KERN(true, false, false);
+    return cl ? BI_WIN_KERN(false, true, false) : BI_WIN_KERN(false, false, false);
+#undef BI_WIN_KERN
+  };
   int best_cs = 0;
   double best_score = -1.0;
   for (int cs = 1; cs <= 8; cs *= 2) {
@@ -384,8 +463,16 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
                          (size_t)units * (NB + TT::NCP) + bsz + (TT::TP ? (size_t)units * TT::TP_UNIT : 0);
     const size_t b = elems * sizeof(R);
     if (warps * 32 > (320) || b > (size_t)smem_budget) continue;
-    int per_sm = (int)std::min<size_t>(8, (size_t)(228 * 1024) / (b + 1024));
-    if (LREG) per_sm = std::min(per_sm, std::max(1, 65536 / (warps * 32 * 208)));  // about 200 registers per thread
+    // CTAs that fit an SM together (shared memory and registers), as the runtime counts them
+    const void *kf = pick(cs > 1);
+    int per_sm = 0;
+    if (cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)b) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kf, warps * 32, b) != cudaSuccess) {
+      cudaGetLastError();
+      continue;
+    }
+    per_sm = std::min(per_sm, 8);
+    if (per_sm < 1) continue;
     // useful warps resident per SM, discounted by idle step slots
     const double score = (double)per_sm * warps * ((double)Tc / units) - 0.01 * cs;
     if (score > best_score) { best_score = score; best_cs = cs; }
@@ -406,7 +493,6 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
     found = true;
   }
   if (!found) return BI_ERR_UNSUPPORTED;
-  const bool stale = sizeof(R) == 8 && p.nmem <= 12;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(p.N * geo.CS));
   cfg.blockDim = dim3((unsigned)threads);
@@ -419,24 +505,10 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = geo.CS > 1 ? 1 : 0;
-  cudaError_t e;
-#define BI_WIN_LAUNCH(ST, CL, DA)                                                                     \
-  do {                                                                                                \
-    auto kern = bi_tile3_window_kernel<R, NA, NB, NC, SB, LREG, ALGO, ST, CL, DA>;                         \
-    e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, kern, p, geo);                                 \
-  } while (0)
-  // (a damped call is a separate instantiation, so that the plain update carries none of it)
-  if (geo.CS > 1) {
-    if (p.lambda != 1.0) BI_WIN_LAUNCH(false, true, true);
-    else if (stale) BI_WIN_LAUNCH(true, true, false);
-    else BI_WIN_LAUNCH(false, true, false);
-  } else {
-    if (p.lambda != 1.0) BI_WIN_LAUNCH(false, false, true);
-    else if (stale) BI_WIN_LAUNCH(true, false, false);
-    else BI_WIN_LAUNCH(false, false, false);
-  }
-#undef BI_WIN_LAUNCH
+  const void *kern = pick(geo.CS > 1);
+  void *args[2] = {(void *)&p, (void *)&geo};
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) e = cudaLaunchKernelExC(&cfg, kern, args);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return BI_ERR_CUDA;
