@@ -262,7 +262,18 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   // The barrier between iterations is split: a CTA arrives as soon as its beliefs are published and
   // waits only when it needs its neighbours', with the contraction (own data only) in between.
   // (A launch without a cluster attribute is a cluster of one CTA, so the same barrier serves both.)
-  cg::this_cluster().barrier_arrive();
+  // Only the warps that store into a neighbouring CTA's halo need the arrival to release at cluster
+  // scope; for the others every store before it is to this CTA's own shared memory, so a fence at
+  // CTA scope and a relaxed arrival give the same ordering without the wider fence's latency.
+  // (The wait keeps its acquire: it orders the halo reads after the neighbours' stores.)
+  const bool remote_writer =
+      CLUSTER && __any_sync(0xffffffffu, r_prev_cur != nullptr || r_next_cur != nullptr) != 0;
+  auto arrive = [&]() {
+    if (remote_writer) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    else asm volatile("fence.acq_rel.cta;\n\tbarrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  };
+  auto wait = [&]() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); };
+  arrive();
 
   R xa = 0, xb = 0, xc = 0, za = 1, zb = 1, zc = 1, rinv = 1;
   float ma = 0.f, mb = 0.f, mc = 0.f, pma = 0.f, pmb = 0.f, pmc = 0.f;
@@ -270,7 +281,7 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     // likelihood messages from this step's own beliefs, while the other CTAs finish publishing theirs
     if (LREG) t3.messages(xa, xb, xc);
     else t3.messages_smem(Lt, xa, xb, xc);
-    cg::this_cluster().barrier_wait();
+    wait();
     // Transition messages from the previous iterate of the neighbouring steps.
     // Both edges are evaluated without branches (a window's first and last
     // step read their halo slot, which always holds valid beliefs, and discard
@@ -416,9 +427,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     { R *tmp = q_cur; q_cur = q_nxt; q_nxt = tmp; }
     { R *tmp = r_prev_cur; r_prev_cur = r_prev_nxt; r_prev_nxt = tmp; }
     { R *tmp = r_next_cur; r_next_cur = r_next_nxt; r_next_nxt = tmp; }
-    cg::this_cluster().barrier_arrive();
+    arrive();
   }
-  cg::this_cluster().barrier_wait();   // nobody leaves while a neighbour may still write into its halo
+  wait();   // nobody leaves while a neighbour may still write into its halo
 }
 
 template <typename R, int NA, int NB, int NC, int SB, bool LREG, int ALGO>
