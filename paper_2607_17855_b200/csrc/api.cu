@@ -508,15 +508,17 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
   int rc = bi_launch_tile3(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER && c.N <= 2 * mut->sm_count) {
-    // Filtering exposes one unit per agent.  With about as few agents as SMs, a CTA per agent keeps
-    // more of the machine busy than a warp per agent once the slices are large (measured on the 128
-    // random structures: faster from about 2000 slice elements per step at 64 and 256 agents, slower
-    // at 1024 agents whatever the size).
+  if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) {
+    // Filtering exposes one unit per agent.  With few agents per SM a CTA per agent keeps more of
+    // the machine busy than a warp per agent.  Measured on the 128 random structures: the CTA
+    // kernel is faster for every structure at 256 and 512 agents (sum of times 95 against 145 ms,
+    // 139 against 186 ms), for all but the largest slices at 1024 agents, and slower for most at
+    // 2048.  BI_CTA_MAXN (testing aid) sets the batch up to which it is used whatever the size.
     long long elems = 0;
-    for (int gi = 0; gi < mut->h.ngroups; ++gi)
-      if (mut->h.grp[gi].rank >= 2) elems += mut->h.grp[gi].P_pad;
-    if (elems >= 2000) rc = bi_launch_generic(c, mut);
+    for (int gi = 0; gi < mut->h.ngroups; ++gi) elems += mut->h.grp[gi].P_pad;
+    bool cta = c.N <= 4 * mut->sm_count || (c.N <= 8 * mut->sm_count && elems < 3000);
+    if (const char *e = getenv("BI_CTA_MAXN")) cta = c.N <= atoll(e);
+    if (cta) rc = bi_launch_cta_filter(c, mut);
   }
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_warp(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);

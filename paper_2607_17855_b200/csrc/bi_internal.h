@@ -117,6 +117,7 @@ struct BiCall {
 // this model / call: the dispatcher tries the next one) or an error.
 int bi_launch_generic(const BiCall &c, bi_model *mut);
 int bi_launch_warp(const BiCall &c, bi_model *mut);
+int bi_launch_cta_filter(const BiCall &c, bi_model *mut);   // filtering only; slices staged per step
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
 int bi_launch_tile3_window(const BiCall &c, bi_model *mut);
 int bi_launch_batch(const BiCall &c, bi_model *mut);

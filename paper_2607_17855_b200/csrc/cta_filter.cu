@@ -1,0 +1,413 @@
+// Variational filtering with one CTA per agent, for batches too small to fill
+// the machine with one warp per agent and models whose groups do not fit a
+// compiled tile.
+//
+// The time recursion and the iteration loop run inside one launch (Section
+// III-C names the launch overhead of looping small contractions as a cost).
+// Per step the summed slices of every dependency group are staged in shared
+// memory once.  One Jacobi iteration (Section IV, marginalisation) is three
+// phases with one CTA barrier after each:
+//
+//   A  every group's first contraction level, its rows strided over all the
+//      CTA's threads: V[r] = sum_c L[r,c] q_last[c] for the next level, and the
+//      per-warp partial sums of (prod_j q_j[r_j]) L[r,c] for the message to the
+//      last axis;
+//   B  one warp per group finishes that group alone (its deeper levels are
+//      small): partial sums added in a fixed order, remaining levels, the fully
+//      contracted vector, all written to the group's own message row;
+//   C  one warp per factor: log-prior plus the groups' messages in a fixed
+//      order, softmax, next beliefs (and the outputs after the last iteration).
+//
+// Sums are taken in a fixed order: results do not depend on scheduling.
+#include <algorithm>
+
+#include "bi_internal.h"
+#include "tile3.cuh"
+
+namespace {
+
+struct CtaGeom {   // element offsets (units of R) into dynamic shared memory
+  int desc, q0, q1, lpri, xp, ellg, part, obs;
+  int Lst[BI_MAX_GROUPS];    // per group: its staged slice, rows `lstride` apart
+  int lstride[BI_MAX_GROUPS];
+  int V[BI_MAX_GROUPS][2];   // per group: the two buffers its levels alternate between
+  int vtot_begin, vtot_end;  // the range holding every V buffer (zeroed once: pad columns stay zero)
+  // Groups of rank >= 2 whose last axis is the same factor form a class: a thread adds their
+  // column sums in registers and the warp reduces once per class.  order[] lists those groups
+  // class by class; class c is order[cls_begin[c] .. cls_begin[c + 1]).
+  int ncls, order[BI_MAX_GROUPS], cls_begin[BI_MAX_GROUPS + 1], cls_pv[BI_MAX_GROUPS];
+  int row_start[BI_MAX_GROUPS];   // thread that takes the group's row 0 (rows go round the CTA's threads)
+  int cls_wmask[BI_MAX_GROUPS];   // warps that hold rows of the class
+  int total_bytes;
+};
+
+// Row stride in shared memory for rows of npad elements (npad a multiple of 4) read by one thread
+// per row with 16-byte loads: the stride in 16-byte units must be odd, or the lanes of a quarter
+// warp fall on the same banks.
+template <typename R>
+__host__ __device__ inline int row_stride(int npad) {
+  const int per16 = 16 / (int)sizeof(R);
+  return ((npad / per16) % 2 == 1) ? npad : npad + per16;
+}
+
+template <typename R>
+__device__ __forceinline__ Vec4<R> lds4(const R *p) {
+  return *reinterpret_cast<const Vec4<R> *>(p);
+}
+
+// Rows r0, r0 + step, ... of one level: writes V, accumulates the column sums in acc.
+template <typename R, int PV>
+__device__ __forceinline__ void peel_rows(const BiLevel &lv, const R *L, int lstride, const R *qt, R *Vout,
+                                          int ostride, int r0, int step, R (&acc)[PV]) {
+  const int npad4 = lv.last_npad4, ndig = lv.ndig, nrows = lv.nrows;
+  uint32_t magic[4], dim[4];
+  const R *qd[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    magic[i] = i < ndig ? lv.magic[i] : 0u;
+    dim[i] = i < ndig ? (uint32_t)lv.dim[i] : 1u;
+    qd[i] = qt + (i < ndig ? lv.qoff[i] : 0);
+  }
+  const R *q4 = qt + lv.last_qoff;
+  for (int r = r0; r < nrows; r += step) {
+    uint32_t rem = (uint32_t)r;
+    R w = (R)1;
+    int lastdig = 0, hi = 0;
+#pragma unroll
+    for (int i = 3; i >= 0; --i) {
+      if (i < ndig) {
+        const uint32_t qq = __umulhi(rem, magic[i]);
+        const int dg = (int)(rem - qq * dim[i]);
+        rem = qq;
+        w *= qd[i][dg];
+        if (i == ndig - 1) { lastdig = dg; hi = (int)qq; }
+      }
+    }
+    R v0 = (R)0, v1 = (R)0;
+#pragma unroll
+    for (int c4 = 0; c4 < PV / 4; ++c4) {
+      if (c4 < npad4) {
+        const Vec4<R> x = lds4(L + r * lstride + 4 * c4);
+        const Vec4<R> qq = lds4(q4 + 4 * c4);
+        v0 = fma(x.x, qq.x, v0); v1 = fma(x.y, qq.y, v1);
+        v0 = fma(x.z, qq.z, v0); v1 = fma(x.w, qq.w, v1);
+        acc[4 * c4 + 0] = fma(w, x.x, acc[4 * c4 + 0]);
+        acc[4 * c4 + 1] = fma(w, x.y, acc[4 * c4 + 1]);
+        acc[4 * c4 + 2] = fma(w, x.z, acc[4 * c4 + 2]);
+        acc[4 * c4 + 3] = fma(w, x.w, acc[4 * c4 + 3]);
+      }
+    }
+    Vout[hi * ostride + lastdig] = v0 + v1;
+  }
+}
+
+// phase A for one class of groups: this thread's rows of their first levels; the warp's column sums go to part_w[c]
+template <typename R, int PV>
+__device__ __forceinline__ void first_levels(const BiDev &md, const CtaGeom &sm, int cls, R *smem, const R *qt,
+                                             R *part_w, int lane) {
+  R acc[PV];
+#pragma unroll
+  for (int c = 0; c < PV; ++c) acc[c] = (R)0;
+  const int NT = blockDim.x;
+  for (int i = sm.cls_begin[cls]; i < sm.cls_begin[cls + 1]; ++i) {
+    const int gi = sm.order[i];
+    const BiLevel &lv = md.grp[gi].lev[0];
+    int r0 = (int)threadIdx.x - sm.row_start[gi];
+    if (r0 < 0) r0 += NT;
+    peel_rows<R, PV>(lv, smem + sm.Lst[gi], sm.lstride[gi], qt, smem + sm.V[gi][0], row_stride<R>(lv.out_npad), r0, NT,
+                     acc);
+  }
+  const R tot = reduce_scatter<R, PV, 32, 1>(acc, lane);
+  constexpr int SH = 5 - Log2<PV>::v;
+  if ((lane & ((1 << SH) - 1)) == 0) part_w[lane >> SH] = tot;
+}
+
+// phase B for one deeper level, by one warp: message entries are written (each level feeds another factor)
+template <typename R, int PV>
+__device__ __forceinline__ void deeper_level(const BiLevel &lv, const R *L, const R *qt, R *Vout, R *ell_g, int lane) {
+  R acc[PV];
+#pragma unroll
+  for (int c = 0; c < PV; ++c) acc[c] = (R)0;
+  peel_rows<R, PV>(lv, L, row_stride<R>(lv.last_npad4 * 4), qt, Vout, row_stride<R>(lv.out_npad), lane, 32, acc);
+  const R tot = reduce_scatter<R, PV, 32, 1>(acc, lane);
+  constexpr int SH = 5 - Log2<PV>::v;
+  const int idx = lane >> SH;
+  if ((lane & ((1 << SH) - 1)) == 0 && idx < lv.last_n) ell_g[lv.last_qoff + idx] = tot;
+  __syncwarp();
+}
+
+template <typename R>
+__global__ void __launch_bounds__(256, 2)
+bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__restrict__ obs,
+                     const int32_t *__restrict__ act, const float *q_prev,
+                     const int32_t *__restrict__ act_prev, double lambda, int K, float *q_out,
+                     float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, const CtaGeom sm) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  R *smem = reinterpret_cast<R *>(smem_raw);
+  {  // the model's description, read from shared memory from here on
+    const int4 *s = reinterpret_cast<const int4 *>(mdp);
+    int4 *d = reinterpret_cast<int4 *>(smem + sm.desc);
+    for (int i = threadIdx.x; i < (int)(sizeof(BiDev) / sizeof(int4)); i += blockDim.x) d[i] = __ldg(s + i);
+    __syncthreads();
+  }
+  const BiDev &md = *reinterpret_cast<const BiDev *>(smem + sm.desc);
+  const int a = blockIdx.x, g = md.G == 1 ? 0 : a;
+  const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5, NW = NT >> 5;
+  const int S = md.S, Sp = md.Sp, F = md.F, M = md.M, NG = md.ngroups;
+  R *cur = smem + sm.q0, *nxt = smem + sm.q1, *lpri = smem + sm.lpri;
+  R *xp = sm.xp >= 0 ? smem + sm.xp : nullptr;   // previous logits (damped calls)
+  R *ellg = smem + sm.ellg;                      // [NG][Sp] the groups' messages
+  R *part = smem + sm.part;                      // [classes][NW][32] per-warp column sums of the first levels
+  int32_t *obs_s = reinterpret_cast<int32_t *>(smem + sm.obs);
+  const R lam = (R)lambda;
+
+  for (int i = tid; i < T * M; i += NT)
+    obs_s[i] = clamp_flag(__ldg(obs + (size_t)a * T * M + i), md.m[i % M], md.status, BI_FLAG_OBS_RANGE);
+  for (int i = tid; i < 2 * Sp; i += NT) cur[i] = (R)0;   // q0 and q1 are adjacent
+  for (int i = tid; i < NG * Sp; i += NT) ellg[i] = (R)0;  // entries of factors outside a group stay zero
+  for (int i = sm.vtot_begin + tid; i < sm.vtot_end; i += NT) smem[i] = (R)0;
+  __syncthreads();
+  if (q_prev) {  // continued filtering: the belief of the step before the first
+    for (int idx = tid; idx < Sp; idx += NT) {
+      int f = 0;
+      while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+      const int s = idx - md.offp[f];
+      cur[idx] = s < md.n[f] ? (R)q_prev[(size_t)a * S + md.off[f] + s] : (R)0;   // (may alias q_out: plain load)
+    }
+    __syncthreads();
+  }
+
+  for (int t = 0; t < T; ++t) {
+    // ln prior: D at the first step, else B_u q_{t-1} (cur still holds step t-1)
+    for (int idx = tid; idx < Sp; idx += NT) {
+      int f = 0;
+      while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+      const int s = idx - md.offp[f], n = md.n[f];
+      R lp = (R)0;
+      if (s < n) {
+        if (t == 0 && !q_prev) {
+          lp = __ldg((const R *)md.logD[f] + (size_t)g * md.Dstride[f] + s);
+        } else {
+          const int ur = t == 0 ? __ldg(act_prev + (size_t)a * F + f)
+                                : __ldg(act + ((size_t)a * (T - 1) + (t - 1)) * F + f);
+          const int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
+          const R *row = (const R *)md.Bf[f] + (size_t)g * md.Bstride[f] + ((size_t)u * n + s) * md.npad[f];
+          const R *qf = cur + md.offp[f];
+          R p0 = (R)0, p1 = (R)0;
+          int r = 0;
+          for (; r + 1 < n; r += 2) {
+            p0 = fma(__ldg(row + r), qf[r], p0);
+            p1 = fma(__ldg(row + r + 1), qf[r + 1], p1);
+          }
+          if (r < n) p0 = fma(__ldg(row + r), qf[r], p0);
+          lp = bi_log(bi_max(p0 + p1, (R)BI_EPS));
+        }
+      }
+      lpri[idx] = lp;
+    }
+    // the step's summed slices, rows at their padded stride
+    for (int gi = 0; gi < NG; ++gi) {
+      const BiGroup &gr = md.grp[gi];
+      const int nm = gr.mem_end - gr.mem_begin;
+      const R *src[BI_MAX_M];
+      for (int mi = 0; mi < nm; ++mi) {
+        const BiMember &mm = md.mem[gr.mem_begin + mi];
+        src[mi] = (const R *)mm.logA + (size_t)g * mm.gstride + (size_t)obs_s[t * M + mm.modality] * mm.P_pad;
+      }
+      const int npad4 = gr.rank > 1 ? gr.lev[0].last_npad4 : bi_pad4(gr.first_n) / 4;
+      R *dst = smem + sm.Lst[gi];
+      const int ls = sm.lstride[gi];
+      for (int e4 = tid; e4 < gr.P_pad / 4; e4 += NT) {
+        Vec4<R> v = ldg4(src[0] + 4 * e4);
+        for (int mi = 1; mi < nm; ++mi) {
+          const Vec4<R> x = ldg4(src[mi] + 4 * e4);
+          v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
+        }
+        const int row = e4 / npad4, c4 = e4 - row * npad4;
+        *reinterpret_cast<Vec4<R> *>(dst + row * ls + 4 * c4) = v;
+      }
+    }
+    __syncthreads();
+    // uniform start
+    for (int idx = tid; idx < Sp; idx += NT) {
+      int f = 0;
+      while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+      cur[idx] = (idx - md.offp[f]) < md.n[f] ? (R)1 / (R)md.n[f] : (R)0;
+      if (xp) xp[idx] = (R)0;   // logits of the uniform start: a constant
+    }
+    __syncthreads();
+
+    for (int k = 0; k < K; ++k) {
+      // ---- A: first levels, all threads
+      for (int cls = 0; cls < sm.ncls; ++cls) {
+        if (!((sm.cls_wmask[cls] >> warp) & 1)) continue;   // none of the class' rows fall to this warp
+        R *pw = part + ((size_t)cls * NW + warp) * 32;
+        switch (sm.cls_pv[cls]) {
+          case 4: first_levels<R, 4>(md, sm, cls, smem, cur, pw, lane); break;
+          case 8: first_levels<R, 8>(md, sm, cls, smem, cur, pw, lane); break;
+          case 16: first_levels<R, 16>(md, sm, cls, smem, cur, pw, lane); break;
+          default: first_levels<R, 32>(md, sm, cls, smem, cur, pw, lane); break;
+        }
+      }
+      __syncthreads();
+      // ---- B: one warp per group
+      for (int gi = warp; gi < NG; gi += NW) {
+        const BiGroup &gr = md.grp[gi];
+        R *eg = ellg + (size_t)gi * Sp;
+        if (gr.rank < 2) {   // rank-1 slice: it is the message itself
+          if (lane < gr.first_n) eg[gr.first_qoff + lane] = smem[sm.Lst[gi] + lane];
+          continue;
+        }
+        for (int cls = 0; cls < sm.ncls; ++cls) {   // the head of a class adds up the class' partial sums
+          if (sm.order[sm.cls_begin[cls]] != gi) continue;
+          const BiLevel &lv = gr.lev[0];
+          if (lane < lv.last_n) {
+            R s = (R)0;
+            for (int w = 0; w < NW; ++w)
+              if ((sm.cls_wmask[cls] >> w) & 1) s += part[((size_t)cls * NW + w) * 32 + lane];
+            eg[lv.last_qoff + lane] = s;
+          }
+        }
+        int bin = 0;
+        for (int l = 1; l + 1 < gr.rank; ++l) {
+          const BiLevel &lv = gr.lev[l];
+          const R *L = smem + sm.V[gi][bin];
+          R *Vout = smem + sm.V[gi][bin ^ 1];
+          switch (lv.last_pv) {
+            case 4: deeper_level<R, 4>(lv, L, cur, Vout, eg, lane); break;
+            case 8: deeper_level<R, 8>(lv, L, cur, Vout, eg, lane); break;
+            case 16: deeper_level<R, 16>(lv, L, cur, Vout, eg, lane); break;
+            default: deeper_level<R, 32>(lv, L, cur, Vout, eg, lane); break;
+          }
+          bin ^= 1;
+        }
+        if (lane < gr.first_n) eg[gr.first_qoff + lane] = smem[sm.V[gi][bin] + lane];
+      }
+      __syncthreads();
+      // ---- C: one warp per factor
+      const bool final = k == K - 1;
+      for (int f = warp; f < F; f += NW) {
+        const int n = md.n[f], op = md.offp[f];
+        R x = -bi_inf<R>();
+        if (lane < n) {
+          x = lpri[op + lane];
+          for (int gi = 0; gi < NG; ++gi) x += ellg[(size_t)gi * Sp + op + lane];
+          if (xp) {   // damped step on the logits; xp: the previous iterate's
+            x = fma(lam, x, ((R)1 - lam) * xp[op + lane]);
+            xp[op + lane] = x;
+          }
+        }
+        const R mx = final ? warp_max(x) : (R)warp_max((float)x);
+        const R e = lane < n ? bi_exp_inline(x - mx) : (R)0;
+        const R z = warp_sum(e);
+        const R q = e * bi_rcp(z);
+        if (lane < md.npad[f]) nxt[op + lane] = lane < n ? q : (R)0;
+        if (final) {
+          const size_t ob = (size_t)a * T + t;
+          if (lane < n) {
+            q_out[ob * S + md.off[f] + lane] = (float)q;
+            if (logq_out) logq_out[ob * S + md.off[f] + lane] = (float)(x - mx - bi_log(z));
+          }
+          if (argmax_out) {
+            const unsigned b = __ballot_sync(0xffffffffu, lane < n && x == mx);
+            if (lane == 0) argmax_out[ob * F + f] = __ffs(b) - 1;
+          }
+        }
+      }
+      __syncthreads();
+      R *tmp = cur; cur = nxt; nxt = tmp;
+    }
+  }
+}
+
+template <typename R>
+int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
+  const bi_model *md = c.model;
+  const BiDev &h = md->h;
+  int NT = 64;
+  while (NT < md->rows_max && NT < 256) NT <<= 1;
+  const int NW = NT / 32;
+  CtaGeom sm;
+  int o = 0;
+  sm.desc = o; o += (int)((sizeof(BiDev) + sizeof(R) - 1) / sizeof(R));
+  o = (o + 3) & ~3;
+  sm.q0 = o; o += h.Sp;
+  sm.q1 = o; o += h.Sp;
+  sm.lpri = o; o += h.Sp;
+  sm.xp = c.lambda != 1.0 ? o : -1;
+  if (c.lambda != 1.0) o += h.Sp;
+  sm.ellg = o; o += h.ngroups * h.Sp;
+  // classes of rank >= 2 groups by the factor of their last axis
+  sm.ncls = 0;
+  {
+    bool taken[BI_MAX_GROUPS] = {};
+    int pos = 0, start = 0;
+    for (int gi = 0; gi < h.ngroups; ++gi) {
+      if (taken[gi] || h.grp[gi].rank < 2) continue;
+      sm.cls_begin[sm.ncls] = pos;
+      sm.cls_pv[sm.ncls] = h.grp[gi].lev[0].last_pv;
+      sm.cls_wmask[sm.ncls] = 0;
+      for (int gj = gi; gj < h.ngroups; ++gj) {
+        if (taken[gj] || h.grp[gj].rank < 2 || h.grp[gj].lev[0].last_qoff != h.grp[gi].lev[0].last_qoff) continue;
+        taken[gj] = true;
+        sm.order[pos++] = gj;
+        // rows go round the CTA's threads from where the previous group's ended (a whole warp on)
+        sm.row_start[gj] = start % NT;
+        const int nr = h.grp[gj].lev[0].nrows;
+        for (int w = 0; w < NW; ++w) {
+          int first = w * 32 - sm.row_start[gj];   // the row of this warp's first thread
+          if (first < 0) first += NT;
+          if (nr >= NT || first < nr || first + 31 >= NT) sm.cls_wmask[sm.ncls] |= 1 << w;
+        }
+        start = (start + nr + 31) & ~31;
+      }
+      ++sm.ncls;
+    }
+    sm.cls_begin[sm.ncls] = pos;
+  }
+  sm.part = o; o += std::max(1, sm.ncls) * NW * 32;
+  sm.vtot_begin = o;
+  for (int gi = 0; gi < BI_MAX_GROUPS; ++gi) sm.V[gi][0] = sm.V[gi][1] = o;
+  for (int gi = 0; gi < h.ngroups; ++gi) {
+    const BiGroup &g = h.grp[gi];
+    int need[2] = {4, 4};
+    for (int l = 0; l + 1 < g.rank; ++l) {
+      const BiLevel &lv = g.lev[l];
+      const int out = (lv.nrows / lv.dim[lv.ndig - 1]) * row_stride<R>(lv.out_npad);
+      need[l & 1] = std::max(need[l & 1], out);
+    }
+    sm.V[gi][0] = o; o += bi_pad4(need[0]);
+    sm.V[gi][1] = o; o += bi_pad4(need[1]);
+  }
+  sm.vtot_end = o;
+  sm.obs = o; o += bi_pad4(c.T * h.M + 1);
+  for (int gi = 0; gi < BI_MAX_GROUPS; ++gi) { sm.Lst[gi] = o; sm.lstride[gi] = 4; }
+  for (int gi = 0; gi < h.ngroups; ++gi) {
+    const BiGroup &g = h.grp[gi];
+    const int npad = g.rank > 1 ? g.lev[0].last_npad4 * 4 : bi_pad4(g.first_n);
+    const int rows = g.P_pad / npad;
+    sm.lstride[gi] = row_stride<R>(npad);
+    sm.Lst[gi] = o;
+    o += bi_pad4(rows * sm.lstride[gi]);
+  }
+  sm.total_bytes = (int)((size_t)o * sizeof(R));
+  if ((size_t)o * sizeof(R) > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
+
+  auto kern = bi_cta_filter_kernel<R>;
+  if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes) !=
+      cudaSuccess)
+    return BI_ERR_CUDA;
+  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.lambda, c.K, c.q_out,
+                                               c.logq_out, c.argmax_out, sm);
+  if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
+  mut->launches += 1;
+  mut->last_kernel = sizeof(R) == 8 ? "cta_filter_f64" : "cta_filter_f32";
+  return BI_OK;
+}
+
+}  // namespace
+
+int bi_launch_cta_filter(const BiCall &c, bi_model *mut) {
+  if (c.algo != BI_ALGO_FILTER) return BI_ERR_UNSUPPORTED;
+  return c.model->arith == BI_ARITH_F64 ? launch_cta_filter_t<double>(c, mut) : launch_cta_filter_t<float>(c, mut);
+}

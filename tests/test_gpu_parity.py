@@ -1,5 +1,8 @@
 """GPU parity: the CUDA library (through its C ABI) against the CPU oracle,
 element by element on the same seeded inputs."""
+import contextlib
+import os
+
 import numpy as np
 import pytest
 
@@ -9,6 +12,21 @@ from biwl import make_config, make_model, make_sweep_config, sample_streams, Wor
 from parity import check_workload, compare, run_gpu  # noqa: E402
 
 ALGOS = ["filter", "vmp", "mmp"]
+
+
+@contextlib.contextmanager
+def warp_filter_forced():
+    """Small filtering batches go to the CTA-per-agent kernel; the library's testing aid BI_CTA_MAXN=0
+    sends them to the warp-per-agent kernel instead, so that it can be checked on oracle-sized inputs."""
+    old = os.environ.get("BI_CTA_MAXN")
+    os.environ["BI_CTA_MAXN"] = "0"
+    try:
+        yield
+    finally:
+        if old is None:
+            del os.environ["BI_CTA_MAXN"]
+        else:
+            os.environ["BI_CTA_MAXN"] = old
 
 
 def _custom(seed, n, m, dep, U, N, T, K, G=1, sparsity=0.0):
@@ -281,11 +299,12 @@ def test_filter_continuation(case):
     elif case == "warp":
         w, kern = _custom(49, [5, 4, 3, 2], [3, 4], [[0, 1], [1, 2, 3]], [2, 2, 1, 2], N=21, T=7, K=6), "warp_filter_f64"
     elif case == "cta":   # few agents and large slices: a CTA per agent
-        w, kern = make_config(3, N=21, T=7, K=6), "generic_filter_staged_f64"
+        w, kern = make_config(3, N=21, T=7, K=6), "cta_filter_f64"
     else:
         w, kern = _custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=5, G=5), None
     for cut in (1, 4):
-        q, ref, kernel = _continued(w, cut)
+        with (warp_filter_forced() if case == "warp" else contextlib.nullcontext()):
+            q, ref, kernel = _continued(w, cut)
         if kern:
             assert kernel == kern, kernel
         assert np.abs(q - ref).max() <= 1e-5, (case, cut, np.abs(q - ref).max())
@@ -490,8 +509,11 @@ def test_damped_updates(case, algo):
     md.set_damping(lam)
     obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
     lq = torch.empty((w.N, w.T, w.S), dtype=torch.float32, device="cuda")
-    q = md.run(algo, obs, act, w.K, logq_out=lq).cpu().numpy()
+    with (warp_filter_forced() if case == "warp" else contextlib.nullcontext()):
+        q = md.run(algo, obs, act, w.K, logq_out=lq).cpu().numpy()
     kernel = md.last_kernel
+    if algo == "filter" and case in ("warp", "cta"):
+        assert kernel == f"{case}_filter_f64", kernel
     assert md.status() == 0
     sel = list(range(0, w.N, max(1, w.N // 12)))
     sub = w.take_agents(sel)
@@ -538,6 +560,51 @@ def test_batched_window_with_per_agent_models(algo):
                      obs_soft=soft[sel])[0]
     assert np.abs(q[sel] - ref).max() <= 1e-5
     md.close()
+
+
+@pytest.mark.parametrize("j", [0, 3, 7, 19, 42, 68, 77, 101, 127])
+def test_warp_filter_kernel_on_small_batches(j):
+    """The warp-per-agent filtering kernel serves large batches; here it is forced onto oracle-sized ones."""
+    w = make_sweep_config(j, N=12)
+    with warp_filter_forced():
+        res = check_workload(w, "filter")
+    assert res["kernel"] == "warp_filter_f64", res
+
+
+@pytest.mark.parametrize("arith", ["f64", "f32"])
+def test_filter_kernel_choice_by_batch_size(arith):
+    """Few agents: a CTA per agent.  Many agents: a warp per agent.  Both against the oracle on sampled agents."""
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = _custom(53, [5, 4, 3, 6], [3, 4, 5], [[0, 1], [1, 2, 3], [3]], [2, 2, 1, 3], N=1400, T=5, K=6)
+    md = bi.model_from_workload(w, arith=arith)
+    sel = list(range(0, w.N, 100))
+    ref = oracle.run_workload(w.take_agents(sel), "filter")[0]
+    for n, kern in ((40, "cta_filter"), (600, "cta_filter"), (1400, "warp_filter")):
+        sub = w.take_agents(list(range(n)))
+        q, _, _, _ = run_gpu(sub, "filter", model=md, arith=arith)
+        assert md.last_kernel == f"{kern}_{arith}", (n, md.last_kernel)
+        pick = [i for i in sel if i < n]
+        err = np.abs(q[pick] - ref[:len(pick)]).max()
+        assert err <= (1e-5 if arith == "f64" else 5e-3), (n, err)
+    md.close()
+
+
+@pytest.mark.parametrize("case", ["rank1_only", "rank5", "per_agent", "many_groups", "wide_last_axis"])
+def test_cta_filter_kernel_shapes(case):
+    """Shapes that stress the CTA-per-agent kernel's phases: no contraction at all, four levels, per-agent slices,
+    several groups sharing a last axis (one merged reduction) next to groups that do not, a 32-state last axis."""
+    w = {
+        "rank1_only": _custom(61, [7, 3], [4, 5, 2], [[0], [1], [0]], [2, 1], N=6, T=5, K=5),
+        "rank5": _custom(62, [3, 4, 2, 5, 3], [4, 3], [[0, 1, 2, 3, 4], [2, 4]], [2, 1, 2, 1, 3], N=5, T=4, K=5),
+        "per_agent": _custom(63, [6, 5, 7, 2], [4, 3, 2], [[2, 0, 1], [1, 2], [3]], [2, 2, 2, 1], N=7, T=5, K=5, G=7,
+                             sparsity=0.5),
+        "many_groups": _custom(64, [9, 4, 6, 5], [3, 4, 2, 5, 3, 2], [[0, 1], [2, 0], [3, 0], [1, 2], [0, 1, 2, 3], [3]],
+                               [2, 1, 3, 2], N=9, T=5, K=6),
+        "wide_last_axis": _custom(65, [32, 31, 2], [3, 4], [[0, 1], [1, 2, 0]], [2, 2, 1], N=4, T=4, K=5),
+    }[case]
+    res = check_workload(w, "filter")
+    assert res["kernel"] == "cta_filter_f64", res
 
 
 def test_fma_probe_reports_a_plausible_rate():
