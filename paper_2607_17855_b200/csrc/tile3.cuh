@@ -22,6 +22,10 @@ template <> struct Pow2Ceil<1> { static constexpr int v = 1; };
 template <int X> struct Log2 { static constexpr int v = 1 + Log2<X / 2>::v; };
 template <> struct Log2<1> { static constexpr int v = 0; };
 
+// an empty statement the optimiser cannot see through: x stays a value in a register
+__device__ __forceinline__ void bi_opaque(float &x) { asm("" : "+f"(x)); }
+__device__ __forceinline__ void bi_opaque(double &x) { asm("" : "+d"(x)); }
+
 // Sum v[i] over the NL lanes {lane ^ (k * STR)}; afterwards v[0] holds the
 // total of element (sub >> (log2 NL - log2 PV)), where sub is the lane's index
 // within the NL lanes.  PV and NL are powers of two, PV <= NL.
@@ -36,8 +40,13 @@ __device__ __forceinline__ R reduce_scatter(R (&v)[PV], int sub) {
       const int half = cur / 2;
 #pragma unroll
       for (int i = 0; i < half; ++i) {
-        R send = up ? v[i] : v[i + half];
-        R keep = up ? v[i + half] : v[i];
+        // (both values are read first and made opaque: a conditional between two array elements can
+        // compile to a load through a selected address, which puts the whole array in local memory)
+        R lo = v[i], hi = v[i + half];
+        bi_opaque(lo);
+        bi_opaque(hi);
+        const R send = up ? lo : hi;
+        const R keep = up ? hi : lo;
         v[i] = keep + __shfl_xor_sync(0xffffffffu, send, d * STR);
       }
       cur = half;
