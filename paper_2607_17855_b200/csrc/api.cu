@@ -510,13 +510,11 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
   if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) {
     // Filtering exposes one unit per agent.  With few agents per SM a CTA per agent keeps more of
-    // the machine busy than a warp per agent.  Measured on the 128 random structures: the CTA
-    // kernel is faster for every structure at 256 and 512 agents (sum of times 95 against 145 ms,
-    // 139 against 186 ms), for all but the largest slices at 1024 agents, and slower for most at
-    // 2048.  BI_CTA_MAXN (testing aid) sets the batch up to which it is used whatever the size.
-    long long elems = 0;
-    for (int gi = 0; gi < mut->h.ngroups; ++gi) elems += mut->h.grp[gi].P_pad;
-    bool cta = c.N <= 4 * mut->sm_count || (c.N <= 8 * mut->sm_count && elems < 3000);
+    // the machine busy than a warp per agent.  Measured on the 128 random structures (sum of their
+    // times, CTA against warp kernel): 66 against 99 ms at 256 agents, 91 against 118 ms at 512,
+    // 139 against 160 ms at 1024 (faster for all but six structures), 261 against 227 ms at 2048
+    // (slower for three quarters of them).  BI_CTA_MAXN (testing aid) moves the boundary.
+    bool cta = c.N <= 8 * mut->sm_count;
     if (const char *e = getenv("BI_CTA_MAXN")) cta = c.N <= atoll(e);
     if (cta) rc = bi_launch_cta_filter(c, mut);
   }
