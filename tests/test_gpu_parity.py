@@ -590,7 +590,7 @@ def test_filter_kernel_choice_by_batch_size(arith):
     md.close()
 
 
-@pytest.mark.parametrize("case", ["rank1_only", "rank5", "per_agent", "many_groups", "wide_last_axis"])
+@pytest.mark.parametrize("case", ["rank1_only", "rank5", "per_agent", "many_groups", "wide_last_axis", "max_counts"])
 def test_cta_filter_kernel_shapes(case):
     """Shapes that stress the CTA-per-agent kernel's phases: no contraction at all, four levels, per-agent slices,
     several groups sharing a last axis (one merged reduction) next to groups that do not, a 32-state last axis."""
@@ -602,6 +602,10 @@ def test_cta_filter_kernel_shapes(case):
         "many_groups": _custom(64, [9, 4, 6, 5], [3, 4, 2, 5, 3, 2], [[0, 1], [2, 0], [3, 0], [1, 2], [0, 1, 2, 3], [3]],
                                [2, 1, 3, 2], N=9, T=5, K=6),
         "wide_last_axis": _custom(65, [32, 31, 2], [3, 4], [[0, 1], [1, 2, 0]], [2, 2, 1], N=4, T=4, K=5),
+        # the most factors and modalities a model may have, sixteen distinct dependency sets
+        "max_counts": _custom(66, [3, 2, 4, 3, 2, 5, 2, 3], [2, 3, 2, 4, 3, 2, 3, 2, 4, 2, 3, 2, 3, 2, 2, 3],
+                              [[0], [1, 2], [2, 3, 4], [5], [6, 7], [0, 1, 2, 3, 4], [7, 0], [3, 5], [4], [1, 6], [2, 7, 5],
+                               [0, 3], [6], [5, 1], [4, 7], [2, 0, 6]], [2, 1, 2, 1, 3, 1, 2, 2], N=5, T=4, K=5),
     }[case]
     res = check_workload(w, "filter")
     assert res["kernel"] == "cta_filter_f64", res
