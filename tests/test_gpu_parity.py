@@ -611,6 +611,19 @@ def test_cta_filter_kernel_shapes(case):
     assert res["kernel"] == "cta_filter_f64", res
 
 
+@pytest.mark.parametrize("j", list(range(2, 128, 5)))
+def test_filter_kernels_on_random_structures_with_ragged_sizes(j):
+    """Every fifth structure of the sweep with ragged agent, step and iteration counts, through both general
+    filtering kernels (the CTA-per-agent one by dispatch, the warp-per-agent one forced)."""
+    rng = np.random.default_rng(1000 + j)
+    w = make_sweep_config(j, N=int(rng.integers(1, 14)), T=int(rng.integers(1, 9)), K=int(rng.integers(1, 7)))
+    res = check_workload(w, "filter", conditioned=True)
+    assert res["kernel"] == "cta_filter_f64", res
+    with warp_filter_forced():
+        res = check_workload(w, "filter", conditioned=True)
+    assert res["kernel"] == "warp_filter_f64", res
+
+
 def test_fma_probe_reports_a_plausible_rate():
     import paper_2607_17855_b200 as bi
     f64, f32 = bi.bi_probe_fma("f64"), bi.bi_probe_fma("f32")
