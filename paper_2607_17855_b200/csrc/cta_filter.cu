@@ -12,11 +12,14 @@
 //      CTA's threads: V[r] = sum_c L[r,c] q_last[c] for the next level, and the
 //      per-warp partial sums of (prod_j q_j[r_j]) L[r,c] for the message to the
 //      last axis;
-//   B  one warp per group finishes that group alone (its deeper levels are
-//      small): partial sums added in a fixed order, remaining levels, the fully
-//      contracted vector, all written to the group's own message row;
-//   C  one warp per factor: log-prior plus the groups' messages in a fixed
-//      order, softmax, next beliefs (and the outputs after the last iteration).
+//   B  one warp per group of rank 3 or more finishes that group alone (its
+//      deeper levels are small): remaining levels and the fully contracted
+//      vector, written to the group's own message row (models without such a
+//      group skip this phase and its barrier);
+//   C  one warp per factor: log-prior, the per-warp partial sums of the classes
+//      that end in this factor, the vectors of rank-2 groups, rank-1 slices and
+//      phase B's rows, all in a fixed order; softmax, next beliefs (and the
+//      outputs after the last iteration).
 //
 // Sums are taken in a fixed order: results do not depend on scheduling.
 #include <algorithm>
@@ -38,6 +41,11 @@ struct CtaGeom {   // element offsets (units of R) into dynamic shared memory
   int ncls, order[BI_MAX_GROUPS], cls_begin[BI_MAX_GROUPS + 1], cls_pv[BI_MAX_GROUPS];
   int row_start[BI_MAX_GROUPS];   // thread that takes the group's row 0 (rows go round the CTA's threads)
   int cls_wmask[BI_MAX_GROUPS];   // warps that hold rows of the class
+  // what phase C adds up for factor f, as bit masks: classes whose last axis is f, rank-2 groups whose
+  // first axis is f (their first level leaves the fully contracted vector), rank-1 groups on f (the
+  // slice is the message), groups of rank >= 3 that contain f (finished by phase B)
+  unsigned f_cls[BI_MAX_F], f_vec[BI_MAX_F], f_r1[BI_MAX_F], f_deep[BI_MAX_F];
+  int deep;                       // any group of rank >= 3: phase B and its barrier are needed
   int total_bytes;
 };
 
@@ -250,48 +258,45 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
         }
       }
       __syncthreads();
-      // ---- B: one warp per group
-      for (int gi = warp; gi < NG; gi += NW) {
-        const BiGroup &gr = md.grp[gi];
-        R *eg = ellg + (size_t)gi * Sp;
-        if (gr.rank < 2) {   // rank-1 slice: it is the message itself
-          if (lane < gr.first_n) eg[gr.first_qoff + lane] = smem[sm.Lst[gi] + lane];
-          continue;
-        }
-        for (int cls = 0; cls < sm.ncls; ++cls) {   // the head of a class adds up the class' partial sums
-          if (sm.order[sm.cls_begin[cls]] != gi) continue;
-          const BiLevel &lv = gr.lev[0];
-          if (lane < lv.last_n) {
-            R s = (R)0;
-            for (int w = 0; w < NW; ++w)
-              if ((sm.cls_wmask[cls] >> w) & 1) s += part[((size_t)cls * NW + w) * 32 + lane];
-            eg[lv.last_qoff + lane] = s;
+      // ---- B: one warp per group of rank >= 3
+      if (sm.deep) {
+        for (int gi = warp; gi < NG; gi += NW) {
+          const BiGroup &gr = md.grp[gi];
+          if (gr.rank < 3) continue;
+          R *eg = ellg + (size_t)gi * Sp;
+          int bin = 0;
+          for (int l = 1; l + 1 < gr.rank; ++l) {
+            const BiLevel &lv = gr.lev[l];
+            const R *L = smem + sm.V[gi][bin];
+            R *Vout = smem + sm.V[gi][bin ^ 1];
+            switch (lv.last_pv) {
+              case 4: deeper_level<R, 4>(lv, L, cur, Vout, eg, lane); break;
+              case 8: deeper_level<R, 8>(lv, L, cur, Vout, eg, lane); break;
+              case 16: deeper_level<R, 16>(lv, L, cur, Vout, eg, lane); break;
+              default: deeper_level<R, 32>(lv, L, cur, Vout, eg, lane); break;
+            }
+            bin ^= 1;
           }
+          if (lane < gr.first_n) eg[gr.first_qoff + lane] = smem[sm.V[gi][bin] + lane];
         }
-        int bin = 0;
-        for (int l = 1; l + 1 < gr.rank; ++l) {
-          const BiLevel &lv = gr.lev[l];
-          const R *L = smem + sm.V[gi][bin];
-          R *Vout = smem + sm.V[gi][bin ^ 1];
-          switch (lv.last_pv) {
-            case 4: deeper_level<R, 4>(lv, L, cur, Vout, eg, lane); break;
-            case 8: deeper_level<R, 8>(lv, L, cur, Vout, eg, lane); break;
-            case 16: deeper_level<R, 16>(lv, L, cur, Vout, eg, lane); break;
-            default: deeper_level<R, 32>(lv, L, cur, Vout, eg, lane); break;
-          }
-          bin ^= 1;
-        }
-        if (lane < gr.first_n) eg[gr.first_qoff + lane] = smem[sm.V[gi][bin] + lane];
+        __syncthreads();
       }
-      __syncthreads();
       // ---- C: one warp per factor
       const bool final = k == K - 1;
       for (int f = warp; f < F; f += NW) {
         const int n = md.n[f], op = md.offp[f];
         R x = -bi_inf<R>();
         if (lane < n) {
-          x = lpri[op + lane];
-          for (int gi = 0; gi < NG; ++gi) x += ellg[(size_t)gi * Sp + op + lane];
+          R x0 = lpri[op + lane], x1 = (R)0;
+          for (unsigned mk = sm.f_cls[f]; mk; mk &= mk - 1) {
+            const int cls = __ffs(mk) - 1;
+            const R *pc = part + (size_t)cls * NW * 32 + lane;
+            for (unsigned wm = (unsigned)sm.cls_wmask[cls]; wm; wm &= wm - 1) x1 += pc[(__ffs(wm) - 1) * 32];
+          }
+          for (unsigned mk = sm.f_vec[f]; mk; mk &= mk - 1) x0 += smem[sm.V[__ffs(mk) - 1][0] + lane];
+          for (unsigned mk = sm.f_r1[f]; mk; mk &= mk - 1) x0 += smem[sm.Lst[__ffs(mk) - 1] + lane];
+          for (unsigned mk = sm.f_deep[f]; mk; mk &= mk - 1) x1 += ellg[(size_t)(__ffs(mk) - 1) * Sp + op + lane];
+          x = x0 + x1;
           if (xp) {   // damped step on the logits; xp: the previous iterate's
             x = fma(lam, x, ((R)1 - lam) * xp[op + lane]);
             xp[op + lane] = x;
@@ -364,6 +369,23 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
       ++sm.ncls;
     }
     sm.cls_begin[sm.ncls] = pos;
+  }
+  sm.deep = 0;
+  for (int f = 0; f < BI_MAX_F; ++f) sm.f_cls[f] = sm.f_vec[f] = sm.f_r1[f] = sm.f_deep[f] = 0;
+  for (int f = 0; f < h.F; ++f) {
+    for (int cls = 0; cls < sm.ncls; ++cls)
+      if (h.grp[sm.order[sm.cls_begin[cls]]].lev[0].last_qoff == h.offp[f]) sm.f_cls[f] |= 1u << cls;
+    for (int gi = 0; gi < h.ngroups; ++gi) {
+      const BiGroup &g = h.grp[gi];
+      if (g.rank <= 2) {
+        if (g.first_qoff == h.offp[f]) (g.rank == 2 ? sm.f_vec[f] : sm.f_r1[f]) |= 1u << gi;
+      } else {
+        sm.deep = 1;
+        // every axis but the last is finished by phase B (the last axis' message comes from the class)
+        for (int j = 0; j + 1 < g.rank; ++j)
+          if (g.axis[j] == f) sm.f_deep[f] |= 1u << gi;
+      }
+    }
   }
   sm.part = o; o += std::max(1, sm.ncls) * NW * 32;
   sm.vtot_begin = o;
