@@ -580,7 +580,7 @@ def test_filter_kernel_choice_by_batch_size(arith):
     md = bi.model_from_workload(w, arith=arith)
     sel = list(range(0, w.N, 100))
     ref = oracle.run_workload(w.take_agents(sel), "filter")[0]
-    for n, kern in ((40, "cta_filter"), (600, "cta_filter"), (1400, "warp_filter")):
+    for n, kern in ((40, "cta_filter"), (400, "cta_filter"), (600, "cta_filter"), (1400, "warp_filter")):   # (the CTA kernel with 8, 4 and 2 warps)
         sub = w.take_agents(list(range(n)))
         q, _, _, _ = run_gpu(sub, "filter", model=md, arith=arith)
         assert md.last_kernel == f"{kern}_{arith}", (n, md.last_kernel)
