@@ -511,9 +511,9 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
   if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) {
     // Filtering exposes one unit per agent.  With few agents per SM a CTA per agent keeps more of
     // the machine busy than a warp per agent.  Measured on the 128 random structures (sum of their
-    // times, CTA against warp kernel): 66 against 99 ms at 256 agents, 91 against 118 ms at 512,
-    // 139 against 160 ms at 1024 (faster for all but six structures), 261 against 227 ms at 2048
-    // (slower for three quarters of them).  BI_CTA_MAXN (testing aid) moves the boundary.
+    // times, CTA against warp kernel): 54 against 99 ms at 256 agents, 78 against 118 ms at 512,
+    // 133 against 160 ms at 1024, 213 against 196 ms at 1536, 249 against 227 ms at 2048.
+    // BI_CTA_MAXN (testing aid) moves the boundary.
     bool cta = c.N <= 8 * mut->sm_count;
     if (const char *e = getenv("BI_CTA_MAXN")) cta = c.N <= atoll(e);
     if (cta) rc = bi_launch_cta_filter(c, mut);
