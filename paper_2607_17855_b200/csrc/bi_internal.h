@@ -12,6 +12,13 @@
 enum { BI_ALGO_FILTER = 0, BI_ALGO_VMP = 1, BI_ALGO_MMP = 2 };
 
 static __host__ __device__ inline int bi_pad4(int x) { return (x + 3) & ~3; }
+// Row stride in shared memory for rows of npad elements (npad a multiple of 4, elements of esize
+// bytes) read by one thread per row with 16-byte loads: an odd number of 16-byte units, or the lanes
+// of a quarter warp fall on the same banks.
+static __host__ __device__ inline int bi_row_stride(int npad, int esize) {
+  const int per16 = 16 / esize;
+  return ((npad / per16) % 2 == 1) ? npad : npad + per16;
+}
 
 // One contraction level of a dependency group.  The group's summed slice is a
 // tensor with `ndig` leading axes and one last axis; the level contracts the

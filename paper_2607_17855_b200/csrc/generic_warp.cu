@@ -65,7 +65,8 @@ __device__ __forceinline__ void peel_level_warp(const BiLevel &lv, const LD &ld,
   for (int c = 0; c < PV; ++c) acc[c] = (R)0;
   // the level's description is read into registers once: it lives in shared
   // memory, and the stores below would otherwise force a reload per row
-  const int npad4 = lv.last_npad4, ndig = lv.ndig, nrows = lv.nrows, onp = lv.out_npad;
+  const int npad4 = lv.last_npad4, ndig = lv.ndig, nrows = lv.nrows;
+  const int onp = bi_row_stride(lv.out_npad, (int)sizeof(R));   // rows of the partial tensor at a conflict-free stride
   uint32_t magic[4], dim[4];
   const R *qd_base[4];
 #pragma unroll
@@ -143,7 +144,7 @@ __device__ __forceinline__ void likelihood_warp(const BiDev &md, const R *const 
     peel_dispatch<R>(gr.lev[0], first, qt, V0, ell, lane);
     R *vin = V0, *vout = V1;
     for (int l = 1; l + 1 < gr.rank; ++l) {
-      SmemRows<R> rows{vin, gr.lev[l].last_npad4 * 4};
+      SmemRows<R> rows{vin, bi_row_stride(gr.lev[l].last_npad4 * 4, (int)sizeof(R))};
       peel_dispatch<R>(gr.lev[l], rows, qt, vout, ell, lane);
       R *t = vin; vin = vout; vout = t;
     }
@@ -413,8 +414,16 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
   sm.o_lpri = o; o += window ? 0 : h.Sp;
   sm.o_q0 = o; o += window ? 0 : h.Sp;
   sm.o_q1 = o; o += window ? 0 : h.Sp;
-  sm.o_V0 = o; o += bi_pad4(md->V0max);
-  sm.o_V1 = o; o += bi_pad4(md->V1max);
+  // the two buffers the levels' partial tensors alternate between, rows at their padded strides
+  int v0 = 4, v1 = 4;
+  for (int gi = 0; gi < h.ngroups; ++gi)
+    for (int l = 0; l + 1 < h.grp[gi].rank; ++l) {
+      const BiLevel &lv = h.grp[gi].lev[l];
+      const int out = (lv.nrows / lv.dim[lv.ndig - 1]) * bi_row_stride(lv.out_npad, (int)sizeof(R));
+      (l % 2 == 0 ? v0 : v1) = std::max(l % 2 == 0 ? v0 : v1, out);
+    }
+  sm.o_V0 = o; o += bi_pad4(v0);
+  sm.o_V1 = o; o += bi_pad4(v1);
   sm.o_sl = o; o += (int)(BI_MAX_M * sizeof(void *) / sizeof(R));
   const bool damped = c.lambda != 1.0;
   sm.o_xp = (!window && damped) ? o : -1;
