@@ -50,15 +50,6 @@ struct CtaGeom {   // element offsets (units of R) into dynamic shared memory
   int total_bytes;
 };
 
-// Row stride in shared memory for rows of npad elements (npad a multiple of 4) read by one thread
-// per row with 16-byte loads: the stride in 16-byte units must be odd, or the lanes of a quarter
-// warp fall on the same banks.
-template <typename R>
-__host__ __device__ inline int row_stride(int npad) {
-  const int per16 = 16 / (int)sizeof(R);
-  return ((npad / per16) % 2 == 1) ? npad : npad + per16;
-}
-
 template <typename R>
 __device__ __forceinline__ Vec4<R> lds4(const R *p) {
   return *reinterpret_cast<const Vec4<R> *>(p);
@@ -123,7 +114,7 @@ __device__ __forceinline__ void first_levels(const BiDev &md, const CtaGeom &sm,
     const BiLevel &lv = md.grp[gi].lev[0];
     int r0 = (int)threadIdx.x - sm.row_start[gi];
     if (r0 < 0) r0 += NT;
-    peel_rows<R, PV>(lv, smem + sm.Lst[gi], sm.lstride[gi], qt, smem + sm.V[gi][0], row_stride<R>(lv.out_npad), r0, NT,
+    peel_rows<R, PV>(lv, smem + sm.Lst[gi], sm.lstride[gi], qt, smem + sm.V[gi][0], bi_row_stride(lv.out_npad, (int)sizeof(R)), r0, NT,
                      acc);
   }
   const R tot = reduce_scatter<R, PV, 32, 1>(acc, lane);
@@ -137,7 +128,7 @@ __device__ __forceinline__ void deeper_level(const BiLevel &lv, const R *L, cons
   R acc[PV];
 #pragma unroll
   for (int c = 0; c < PV; ++c) acc[c] = (R)0;
-  peel_rows<R, PV>(lv, L, row_stride<R>(lv.last_npad4 * 4), qt, Vout, row_stride<R>(lv.out_npad), lane, 32, acc);
+  peel_rows<R, PV>(lv, L, bi_row_stride(lv.last_npad4 * 4, (int)sizeof(R)), qt, Vout, bi_row_stride(lv.out_npad, (int)sizeof(R)), lane, 32, acc);
   const R tot = reduce_scatter<R, PV, 32, 1>(acc, lane);
   constexpr int SH = 5 - Log2<PV>::v;
   const int idx = lane >> SH;
@@ -402,7 +393,7 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
     int need[2] = {4, 4};
     for (int l = 0; l + 1 < g.rank; ++l) {
       const BiLevel &lv = g.lev[l];
-      const int out = (lv.nrows / lv.dim[lv.ndig - 1]) * row_stride<R>(lv.out_npad);
+      const int out = (lv.nrows / lv.dim[lv.ndig - 1]) * bi_row_stride(lv.out_npad, (int)sizeof(R));
       need[l & 1] = std::max(need[l & 1], out);
     }
     sm.V[gi][0] = o; o += bi_pad4(need[0]);
@@ -415,7 +406,7 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
     const BiGroup &g = h.grp[gi];
     const int npad = g.rank > 1 ? g.lev[0].last_npad4 * 4 : bi_pad4(g.first_n);
     const int rows = g.P_pad / npad;
-    sm.lstride[gi] = row_stride<R>(npad);
+    sm.lstride[gi] = bi_row_stride(npad, (int)sizeof(R));
     sm.Lst[gi] = o;
     o += bi_pad4(rows * sm.lstride[gi]);
   }
