@@ -136,6 +136,39 @@ __device__ __forceinline__ void deeper_level(const BiLevel &lv, const R *L, cons
   __syncwarp();
 }
 
+// The last level of a group, by one warp: a matrix L[r][c] over the group's first two axes (at most
+// 32 x 32).  Both of its results are plain loops, one lane per row and one lane per column, with no
+// cross-lane sums: vec[r] = sum_c L[r][c] q1[c] (the message to the first axis) and
+// msg[c] = sum_r q0[r] L[r][c] (the message to the second).
+template <typename R>
+__device__ __forceinline__ void last_level(const BiLevel &lv, const R *L, const R *qt, R *ell_g, int first_qoff,
+                                           int lane) {
+  const int lstride = bi_row_stride(lv.last_npad4 * 4, (int)sizeof(R));
+  const int nrows = lv.nrows, npad4 = lv.last_npad4, n1 = lv.last_n;
+  const R *q0 = qt + lv.qoff[0], *q1 = qt + lv.last_qoff;
+  if (lane < nrows) {
+    R v0 = (R)0, v1 = (R)0;
+    for (int c4 = 0; c4 < npad4; ++c4) {
+      const Vec4<R> x = lds4(L + lane * lstride + 4 * c4);
+      const Vec4<R> qq = lds4(q1 + 4 * c4);
+      v0 = fma(x.x, qq.x, v0); v1 = fma(x.y, qq.y, v1);
+      v0 = fma(x.z, qq.z, v0); v1 = fma(x.w, qq.w, v1);
+    }
+    ell_g[first_qoff + lane] = v0 + v1;
+  }
+  if (lane < n1) {
+    R m0 = (R)0, m1 = (R)0;
+    int r = 0;
+    for (; r + 1 < nrows; r += 2) {
+      m0 = fma(q0[r], L[r * lstride + lane], m0);
+      m1 = fma(q0[r + 1], L[(r + 1) * lstride + lane], m1);
+    }
+    if (r < nrows) m0 = fma(q0[r], L[r * lstride + lane], m0);
+    ell_g[lv.last_qoff + lane] = m0 + m1;
+  }
+  __syncwarp();
+}
+
 template <typename R>
 __global__ void __launch_bounds__(256, 2)
 bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__restrict__ obs,
@@ -257,7 +290,7 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
           if (gr.rank < 3) continue;
           R *eg = ellg + (size_t)gi * Sp;
           int bin = 0;
-          for (int l = 1; l + 1 < gr.rank; ++l) {
+          for (int l = 1; l + 2 < gr.rank; ++l) {
             const BiLevel &lv = gr.lev[l];
             const R *L = smem + sm.V[gi][bin];
             R *Vout = smem + sm.V[gi][bin ^ 1];
@@ -269,7 +302,7 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
             }
             bin ^= 1;
           }
-          if (lane < gr.first_n) eg[gr.first_qoff + lane] = smem[sm.V[gi][bin] + lane];
+          last_level<R>(gr.lev[gr.rank - 2], smem + sm.V[gi][bin], cur, eg, gr.first_qoff, lane);
         }
         __syncthreads();
       }
