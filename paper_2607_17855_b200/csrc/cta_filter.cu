@@ -8,8 +8,8 @@
 // memory once.  One Jacobi iteration (Section IV, marginalisation) is three
 // phases with one CTA barrier after each:
 //
-//   A  every group's first contraction level, its rows strided over all the
-//      CTA's threads: V[r] = sum_c L[r,c] q_last[c] for the next level, and the
+//   A  the first contraction level of every group of rank 3 or more, its rows
+//      dealt round all the CTA's threads: V[r] = sum_c L[r,c] q_last[c] for the next level, and the
 //      per-warp partial sums of (prod_j q_j[r_j]) L[r,c] for the message to the
 //      last axis;
 //   B  one warp per group of rank 3 or more finishes that group alone (its
@@ -17,9 +17,11 @@
 //      vector, written to the group's own message row (models without such a
 //      group skip this phase and its barrier);
 //   C  one warp per factor: log-prior, the per-warp partial sums of the classes
-//      that end in this factor, the vectors of rank-2 groups, rank-1 slices and
-//      phase B's rows, all in a fixed order; softmax, next beliefs (and the
-//      outputs after the last iteration).
+//      that end in this factor, the rank-2 groups' messages (a matrix of at most
+//      32 x 32: the factor's warp sums its rows or columns itself), rank-1
+//      slices and phase B's rows, all in a fixed order; softmax, next beliefs
+//      (and the outputs after the last iteration).
+// Phases A and B and their barriers are skipped by models without such groups.
 //
 // Sums are taken in a fixed order: results do not depend on scheduling.
 #include <algorithm>
@@ -36,16 +38,16 @@ struct CtaGeom {   // element offsets (units of R) into dynamic shared memory
   int lstride[BI_MAX_GROUPS];
   int V[BI_MAX_GROUPS][2];   // per group: the two buffers its levels alternate between
   int vtot_begin, vtot_end;  // the range holding every V buffer (zeroed once: pad columns stay zero)
-  // Groups of rank >= 2 whose last axis is the same factor form a class: a thread adds their
+  // Groups of rank >= 3 whose last axis is the same factor form a class: a thread adds their
   // column sums in registers and the warp reduces once per class.  order[] lists those groups
   // class by class; class c is order[cls_begin[c] .. cls_begin[c + 1]).
   int ncls, order[BI_MAX_GROUPS], cls_begin[BI_MAX_GROUPS + 1], cls_pv[BI_MAX_GROUPS];
   int row_start[BI_MAX_GROUPS];   // thread that takes the group's row 0 (rows go round the CTA's threads)
   int cls_wmask[BI_MAX_GROUPS];   // warps that hold rows of the class
-  // what phase C adds up for factor f, as bit masks: classes whose last axis is f, rank-2 groups whose
-  // first axis is f (their first level leaves the fully contracted vector), rank-1 groups on f (the
+  // what phase C adds up for factor f, as bit masks: classes whose last axis is f, rank-2 groups
+  // whose first / second axis is f (contracted by the factor's own warp), rank-1 groups on f (the
   // slice is the message), groups of rank >= 3 that contain f (finished by phase B)
-  unsigned f_cls[BI_MAX_F], f_vec[BI_MAX_F], f_r1[BI_MAX_F], f_deep[BI_MAX_F];
+  unsigned f_cls[BI_MAX_F], f_m0[BI_MAX_F], f_m1[BI_MAX_F], f_r1[BI_MAX_F], f_deep[BI_MAX_F];
   int deep;                       // any group of rank >= 3: phase B and its barrier are needed
   int total_bytes;
 };
@@ -169,6 +171,31 @@ __device__ __forceinline__ void last_level(const BiLevel &lv, const R *L, const 
   __syncwarp();
 }
 
+// rank-2 group, matrix L[r][c] at row stride ls: the messages to its first axis (this lane's row) and
+// to its second axis (this lane's column)
+template <typename R>
+__device__ __forceinline__ R matrix_row_dot(const R *L, int ls, int row, const R *q1, int npad4) {
+  R v0 = (R)0, v1 = (R)0;
+  for (int c4 = 0; c4 < npad4; ++c4) {
+    const Vec4<R> x = lds4(L + row * ls + 4 * c4);
+    const Vec4<R> qq = lds4(q1 + 4 * c4);
+    v0 = fma(x.x, qq.x, v0); v1 = fma(x.y, qq.y, v1);
+    v0 = fma(x.z, qq.z, v0); v1 = fma(x.w, qq.w, v1);
+  }
+  return v0 + v1;
+}
+template <typename R>
+__device__ __forceinline__ R matrix_col_dot(const R *L, int ls, int col, const R *q0, int nrows) {
+  R m0 = (R)0, m1 = (R)0;
+  int r = 0;
+  for (; r + 1 < nrows; r += 2) {
+    m0 = fma(q0[r], L[r * ls + col], m0);
+    m1 = fma(q0[r + 1], L[(r + 1) * ls + col], m1);
+  }
+  if (r < nrows) m0 = fma(q0[r], L[r * ls + col], m0);
+  return m0 + m1;
+}
+
 template <typename R>
 __global__ void __launch_bounds__(256, 2)
 bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__restrict__ obs,
@@ -271,7 +298,7 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
     __syncthreads();
 
     for (int k = 0; k < K; ++k) {
-      // ---- A: first levels, all threads
+      // ---- A: first levels of the groups of rank >= 3, all threads
       for (int cls = 0; cls < sm.ncls; ++cls) {
         if (!((sm.cls_wmask[cls] >> warp) & 1)) continue;   // none of the class' rows fall to this warp
         R *pw = part + ((size_t)cls * NW + warp) * 32;
@@ -282,9 +309,9 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
           default: first_levels<R, 32>(md, sm, cls, smem, cur, pw, lane); break;
         }
       }
-      __syncthreads();
       // ---- B: one warp per group of rank >= 3
       if (sm.deep) {
+        __syncthreads();
         for (int gi = warp; gi < NG; gi += NW) {
           const BiGroup &gr = md.grp[gi];
           if (gr.rank < 3) continue;
@@ -318,7 +345,16 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
             const R *pc = part + (size_t)cls * NW * 32 + lane;
             for (unsigned wm = (unsigned)sm.cls_wmask[cls]; wm; wm &= wm - 1) x1 += pc[(__ffs(wm) - 1) * 32];
           }
-          for (unsigned mk = sm.f_vec[f]; mk; mk &= mk - 1) x0 += smem[sm.V[__ffs(mk) - 1][0] + lane];
+          for (unsigned mk = sm.f_m0[f]; mk; mk &= mk - 1) {   // rank-2 groups with f as first axis
+            const int gi = __ffs(mk) - 1;
+            const BiLevel &lv = md.grp[gi].lev[0];
+            x0 += matrix_row_dot<R>(smem + sm.Lst[gi], sm.lstride[gi], lane, cur + lv.last_qoff, lv.last_npad4);
+          }
+          for (unsigned mk = sm.f_m1[f]; mk; mk &= mk - 1) {   // ... and as second axis
+            const int gi = __ffs(mk) - 1;
+            const BiLevel &lv = md.grp[gi].lev[0];
+            x1 += matrix_col_dot<R>(smem + sm.Lst[gi], sm.lstride[gi], lane, cur + lv.qoff[0], lv.nrows);
+          }
           for (unsigned mk = sm.f_r1[f]; mk; mk &= mk - 1) x0 += smem[sm.Lst[__ffs(mk) - 1] + lane];
           for (unsigned mk = sm.f_deep[f]; mk; mk &= mk - 1) x1 += ellg[(size_t)(__ffs(mk) - 1) * Sp + op + lane];
           x = x0 + x1;
@@ -373,18 +409,18 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
   sm.xp = c.lambda != 1.0 ? o : -1;
   if (c.lambda != 1.0) o += h.Sp;
   sm.ellg = o; o += h.ngroups * h.Sp;
-  // classes of rank >= 2 groups by the factor of their last axis
+  // classes of rank >= 3 groups by the factor of their last axis
   sm.ncls = 0;
   {
     bool taken[BI_MAX_GROUPS] = {};
     int pos = 0, start = 0;
     for (int gi = 0; gi < h.ngroups; ++gi) {
-      if (taken[gi] || h.grp[gi].rank < 2) continue;
+      if (taken[gi] || h.grp[gi].rank < 3) continue;
       sm.cls_begin[sm.ncls] = pos;
       sm.cls_pv[sm.ncls] = h.grp[gi].lev[0].last_pv;
       sm.cls_wmask[sm.ncls] = 0;
       for (int gj = gi; gj < h.ngroups; ++gj) {
-        if (taken[gj] || h.grp[gj].rank < 2 || h.grp[gj].lev[0].last_qoff != h.grp[gi].lev[0].last_qoff) continue;
+        if (taken[gj] || h.grp[gj].rank < 3 || h.grp[gj].lev[0].last_qoff != h.grp[gi].lev[0].last_qoff) continue;
         taken[gj] = true;
         sm.order[pos++] = gj;
         // rows go round the CTA's threads from where the previous group's ended (a whole warp on)
@@ -402,14 +438,17 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
     sm.cls_begin[sm.ncls] = pos;
   }
   sm.deep = 0;
-  for (int f = 0; f < BI_MAX_F; ++f) sm.f_cls[f] = sm.f_vec[f] = sm.f_r1[f] = sm.f_deep[f] = 0;
+  for (int f = 0; f < BI_MAX_F; ++f) sm.f_cls[f] = sm.f_m0[f] = sm.f_m1[f] = sm.f_r1[f] = sm.f_deep[f] = 0;
   for (int f = 0; f < h.F; ++f) {
     for (int cls = 0; cls < sm.ncls; ++cls)
       if (h.grp[sm.order[sm.cls_begin[cls]]].lev[0].last_qoff == h.offp[f]) sm.f_cls[f] |= 1u << cls;
     for (int gi = 0; gi < h.ngroups; ++gi) {
       const BiGroup &g = h.grp[gi];
-      if (g.rank <= 2) {
-        if (g.first_qoff == h.offp[f]) (g.rank == 2 ? sm.f_vec[f] : sm.f_r1[f]) |= 1u << gi;
+      if (g.rank == 1) {
+        if (g.first_qoff == h.offp[f]) sm.f_r1[f] |= 1u << gi;
+      } else if (g.rank == 2) {
+        if (g.axis[0] == f) sm.f_m0[f] |= 1u << gi;
+        if (g.axis[1] == f) sm.f_m1[f] |= 1u << gi;
       } else {
         sm.deep = 1;
         // every axis but the last is finished by phase B (the last axis' message comes from the class)
