@@ -12,16 +12,17 @@
 //      dealt round all the CTA's threads: V[r] = sum_c L[r,c] q_last[c] for the next level, and the
 //      per-warp partial sums of (prod_j q_j[r_j]) L[r,c] for the message to the
 //      last axis;
-//   B  one warp per group of rank 3 or more finishes that group alone (its
-//      deeper levels are small): remaining levels and the fully contracted
-//      vector, written to the group's own message row (models without such a
-//      group skip this phase and its barrier);
+//   B  one warp per group of rank 4 or more takes that group down to its last
+//      two axes (these levels are small) and writes their messages to the
+//      group's own message row;
 //   C  one warp per factor: log-prior, the per-warp partial sums of the classes
-//      that end in this factor, the rank-2 groups' messages (a matrix of at most
-//      32 x 32: the factor's warp sums its rows or columns itself), rank-1
-//      slices and phase B's rows, all in a fixed order; softmax, next beliefs
-//      (and the outputs after the last iteration).
-// Phases A and B and their barriers are skipped by models without such groups.
+//      that end in this factor, the messages from groups of rank 2 and 3 (what
+//      is left of them is a matrix of at most 32 x 32 over their first two
+//      axes: the factor's warp sums its rows or columns itself), rank-1 slices
+//      and phase B's rows, all in a fixed order; softmax, next beliefs (and the
+//      outputs after the last iteration).
+// Models without a group of rank 3 or more skip phase A, models without one of rank 4 or
+// more phase B, each with its barrier.
 //
 // Sums are taken in a fixed order: results do not depend on scheduling.
 #include <algorithm>
@@ -44,11 +45,14 @@ struct CtaGeom {   // element offsets (units of R) into dynamic shared memory
   int ncls, order[BI_MAX_GROUPS], cls_begin[BI_MAX_GROUPS + 1], cls_pv[BI_MAX_GROUPS];
   int row_start[BI_MAX_GROUPS];   // thread that takes the group's row 0 (rows go round the CTA's threads)
   int cls_wmask[BI_MAX_GROUPS];   // warps that hold rows of the class
-  // what phase C adds up for factor f, as bit masks: classes whose last axis is f, rank-2 groups
-  // whose first / second axis is f (contracted by the factor's own warp), rank-1 groups on f (the
-  // slice is the message), groups of rank >= 3 that contain f (finished by phase B)
+  // what phase C adds up for factor f, as bit masks: classes whose last axis is f, groups of rank 2
+  // or 3 whose first / second axis is f (a matrix contracted by the factor's own warp), rank-1
+  // groups on f (the slice is the message), groups of rank >= 4 that contain f (finished by phase B)
   unsigned f_cls[BI_MAX_F], f_m0[BI_MAX_F], f_m1[BI_MAX_F], f_r1[BI_MAX_F], f_deep[BI_MAX_F];
-  int deep;                       // any group of rank >= 3: phase B and its barrier are needed
+  // the matrix over a group's first two axes that phase C contracts: a rank-2 group's staged slice, a
+  // rank-3 group's first partial tensor; its offset, row stride and the level that describes it
+  int mat_off[BI_MAX_GROUPS], mat_ls[BI_MAX_GROUPS], mat_lev[BI_MAX_GROUPS];
+  int deep;                       // any group of rank >= 4: phase B and its barrier are needed
   int total_bytes;
 };
 
@@ -309,12 +313,12 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
           default: first_levels<R, 32>(md, sm, cls, smem, cur, pw, lane); break;
         }
       }
-      // ---- B: one warp per group of rank >= 3
+      if (sm.ncls) __syncthreads();
+      // ---- B: one warp per group of rank >= 4
       if (sm.deep) {
-        __syncthreads();
         for (int gi = warp; gi < NG; gi += NW) {
           const BiGroup &gr = md.grp[gi];
-          if (gr.rank < 3) continue;
+          if (gr.rank < 4) continue;
           R *eg = ellg + (size_t)gi * Sp;
           int bin = 0;
           for (int l = 1; l + 2 < gr.rank; ++l) {
@@ -345,15 +349,15 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
             const R *pc = part + (size_t)cls * NW * 32 + lane;
             for (unsigned wm = (unsigned)sm.cls_wmask[cls]; wm; wm &= wm - 1) x1 += pc[(__ffs(wm) - 1) * 32];
           }
-          for (unsigned mk = sm.f_m0[f]; mk; mk &= mk - 1) {   // rank-2 groups with f as first axis
+          for (unsigned mk = sm.f_m0[f]; mk; mk &= mk - 1) {   // groups of rank 2 or 3 with f as first axis
             const int gi = __ffs(mk) - 1;
-            const BiLevel &lv = md.grp[gi].lev[0];
-            x0 += matrix_row_dot<R>(smem + sm.Lst[gi], sm.lstride[gi], lane, cur + lv.last_qoff, lv.last_npad4);
+            const BiLevel &lv = md.grp[gi].lev[sm.mat_lev[gi]];
+            x0 += matrix_row_dot<R>(smem + sm.mat_off[gi], sm.mat_ls[gi], lane, cur + lv.last_qoff, lv.last_npad4);
           }
           for (unsigned mk = sm.f_m1[f]; mk; mk &= mk - 1) {   // ... and as second axis
             const int gi = __ffs(mk) - 1;
-            const BiLevel &lv = md.grp[gi].lev[0];
-            x1 += matrix_col_dot<R>(smem + sm.Lst[gi], sm.lstride[gi], lane, cur + lv.qoff[0], lv.nrows);
+            const BiLevel &lv = md.grp[gi].lev[sm.mat_lev[gi]];
+            x1 += matrix_col_dot<R>(smem + sm.mat_off[gi], sm.mat_ls[gi], lane, cur + lv.qoff[0], lv.nrows);
           }
           for (unsigned mk = sm.f_r1[f]; mk; mk &= mk - 1) x0 += smem[sm.Lst[__ffs(mk) - 1] + lane];
           for (unsigned mk = sm.f_deep[f]; mk; mk &= mk - 1) x1 += ellg[(size_t)(__ffs(mk) - 1) * Sp + op + lane];
@@ -446,7 +450,7 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
       const BiGroup &g = h.grp[gi];
       if (g.rank == 1) {
         if (g.first_qoff == h.offp[f]) sm.f_r1[f] |= 1u << gi;
-      } else if (g.rank == 2) {
+      } else if (g.rank <= 3) {
         if (g.axis[0] == f) sm.f_m0[f] |= 1u << gi;
         if (g.axis[1] == f) sm.f_m1[f] |= 1u << gi;
       } else {
@@ -481,6 +485,17 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
     sm.lstride[gi] = bi_row_stride(npad, (int)sizeof(R));
     sm.Lst[gi] = o;
     o += bi_pad4(rows * sm.lstride[gi]);
+  }
+  for (int gi = 0; gi < BI_MAX_GROUPS; ++gi) sm.mat_off[gi] = sm.mat_ls[gi] = sm.mat_lev[gi] = 0;
+  for (int gi = 0; gi < h.ngroups; ++gi) {
+    const BiGroup &g = h.grp[gi];
+    if (g.rank == 2) {
+      sm.mat_off[gi] = sm.Lst[gi]; sm.mat_ls[gi] = sm.lstride[gi]; sm.mat_lev[gi] = 0;
+    } else if (g.rank == 3) {   // the first level's output: rows at the padded stride of its last axis
+      sm.mat_off[gi] = sm.V[gi][0];
+      sm.mat_ls[gi] = bi_row_stride(g.lev[0].out_npad, (int)sizeof(R));
+      sm.mat_lev[gi] = 1;
+    }
   }
   sm.total_bytes = (int)((size_t)o * sizeof(R));
   if ((size_t)o * sizeof(R) > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
