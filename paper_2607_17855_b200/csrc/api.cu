@@ -509,12 +509,13 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
   if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) {
-    // Filtering exposes one unit per agent.  With few agents per SM a CTA per agent keeps more of
-    // the machine busy than a warp per agent.  Measured on the 128 random structures (sum of their
-    // times, CTA against warp kernel): 54 against 99 ms at 256 agents, 78 against 118 ms at 512,
-    // 133 against 160 ms at 1024, 213 against 196 ms at 1536, 249 against 227 ms at 2048.
-    // BI_CTA_MAXN (testing aid) moves the boundary.
-    bool cta = c.N <= 8 * mut->sm_count;
+    // Filtering exposes one unit per agent, so a CTA per agent keeps more of the machine busy than
+    // a warp per agent, and its staged slices and per-factor warps pay at every batch size measured
+    // on the 128 random structures (sum of times, CTA against warp kernel): 44 against 99 ms at 256
+    // agents, 109 against 160 ms at 1024, 207 against 224 ms at 2048, 406 against 434 ms at 4096,
+    // 784 against 846 ms at 8192.  The warp kernel serves the models whose slices do not fit in
+    // shared memory.  BI_CTA_MAXN (testing aid) caps the batch that goes to the CTA kernel.
+    bool cta = true;
     if (const char *e = getenv("BI_CTA_MAXN")) cta = c.N <= atoll(e);
     if (cta) rc = bi_launch_cta_filter(c, mut);
   }

@@ -572,17 +572,19 @@ def test_warp_filter_kernel_on_small_batches(j):
 
 
 @pytest.mark.parametrize("arith", ["f64", "f32"])
-def test_filter_kernel_choice_by_batch_size(arith):
-    """Few agents: a CTA per agent.  Many agents: a warp per agent.  Both against the oracle on sampled agents."""
+def test_filter_kernels_across_batch_sizes(arith):
+    """The CTA-per-agent kernel at the batch sizes that select its 8-, 4- and 2-warp CTAs, and the
+    warp-per-agent kernel on the largest batch, all against the oracle on sampled agents."""
     import oracle
     import paper_2607_17855_b200 as bi
     w = _custom(53, [5, 4, 3, 6], [3, 4, 5], [[0, 1], [1, 2, 3], [3]], [2, 2, 1, 3], N=1400, T=5, K=6)
     md = bi.model_from_workload(w, arith=arith)
     sel = list(range(0, w.N, 100))
     ref = oracle.run_workload(w.take_agents(sel), "filter")[0]
-    for n, kern in ((40, "cta_filter"), (400, "cta_filter"), (600, "cta_filter"), (1400, "warp_filter")):   # (the CTA kernel with 8, 4 and 2 warps)
+    for n, kern in ((40, "cta_filter"), (400, "cta_filter"), (1400, "cta_filter"), (1400, "warp_filter")):
         sub = w.take_agents(list(range(n)))
-        q, _, _, _ = run_gpu(sub, "filter", model=md, arith=arith)
+        with (warp_filter_forced() if kern == "warp_filter" else contextlib.nullcontext()):
+            q, _, _, _ = run_gpu(sub, "filter", model=md, arith=arith)
         assert md.last_kernel == f"{kern}_{arith}", (n, md.last_kernel)
         pick = [i for i in sel if i < n]
         err = np.abs(q[pick] - ref[:len(pick)]).max()
