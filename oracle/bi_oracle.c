@@ -36,10 +36,14 @@
  *     q_{t+1}) (0 at the last step), Bdag = transpose of B_u with every column
  *     renormalised (a zero sum gives a uniform column).
  * Pins: filtering, VMP and the free-energy property are pinned by closed forms
- * and brute-force enumeration in the CPU tests.  The MMP reading itself (the
- * 1/2 weights and Bdag) has no statement in the paper to check against:
- * PARITY UNPINNED for that reading; the tests pin only that the code
- * implements it (closed-form special cases).
+ * and brute-force enumeration in the CPU tests.  MMP is pinned by a hand-worked
+ * two-step window whose backward message varies over states, by a permutation
+ * transition, by an unreachable-state case, and by a restatement of the update
+ * from the model's definition (likelihood by enumeration, Bayes reversal of the
+ * transition by conditioning an enumerated joint table).  What no test can
+ * settle is whether this reading of "MMP" (1/2 weights, reversed transition
+ * under a uniform prior, D at full weight) is the one the paper's authors ran:
+ * Section IV names the algorithm and prints no equation.
  *
  * Layouts (row-major):
  *   A[i]: [G][m_i][n_{dep(i)[0]}]...[n_{dep(i)[k-1]}]   float32

@@ -129,3 +129,67 @@ def hmm_forward(A, B, D, obs, act):
         alpha /= alpha.sum()
         out.append(alpha)
     return np.stack(out)
+
+
+def reversed_transition(Bu):
+    """P(s_t = s | s_{t+1} = r) for a single factor whose s_t has a uniform
+    prior, by enumerating the joint table of the pair (s_t, s_{t+1}) and
+    conditioning on the second coordinate -- Bayes' rule on the definition
+    p(s_{t+1} | s_t) = Bu[s_{t+1}, s_t] (Section III-B), no closed formula.
+    Returns R[s, r].  A next state r that no s_t can reach has no posterior;
+    there the marginal-message reading takes the prior itself (uniform)."""
+    Bu = np.asarray(Bu, np.float64)
+    n = Bu.shape[0]
+    joint = np.zeros((n, n))            # joint[s, r] = p(s_t = s) p(s_{t+1} = r | s_t = s)
+    for s in range(n):
+        for r in range(n):
+            joint[s, r] = (1.0 / n) * Bu[r, s]
+    R = np.zeros((n, n))
+    for r in range(n):
+        evidence = sum(joint[s, r] for s in range(n))
+        for s in range(n):
+            R[s, r] = joint[s, r] / evidence if evidence > 0.0 else 1.0 / n
+    return R
+
+
+def mmp_update_by_definition(model, q):
+    """One Jacobi marginal-message-passing update of every (t, f) of a TinyModel
+    from the beliefs q [T, S], written from the reading's own words rather
+    than from message formulas: the new belief is proportional to
+        exp(E_{q_t \\ f}[ln p(o_t | s_t)])                       (likelihood, by enumeration)
+      * p(s_1)                      at t = 1, else sqrt of the one-step prediction of s_t from q_{t-1}
+      * sqrt of the one-step retrodiction of s_t from q_{t+1}     (none at the last step),
+    the retrodiction being sum_r P(s_t | s_{t+1} = r) q_{t+1}[r] with the
+    reversed kernel of reversed_transition.  Probabilities enter through the
+    same floor 1e-16 as everywhere."""
+    out = np.zeros_like(q)
+    for t in range(model.T):
+        for f in range(model.F):
+            lo, hi = model.off[f], model.off[f + 1]
+            x = np.zeros(model.n[f])
+            for s in model.states:          # E over the other factors of ln p(o_t | s_t)
+                w = 1.0
+                for ff in range(model.F):
+                    if ff != f:
+                        w *= q[t, model.off[ff] + s[ff]]
+                x[s[f]] += w * model.ln_emit(t, s)
+            if t == 0:
+                x += _ln(model.D[f])
+            else:
+                pred = np.zeros(model.n[f])
+                Bu = model.B[f][:, :, model.act[t - 1, f]]
+                for s_next in range(model.n[f]):
+                    for s_prev in range(model.n[f]):
+                        pred[s_next] += Bu[s_next, s_prev] * q[t - 1, lo + s_prev]
+                x += 0.5 * _ln(pred)
+            if t + 1 < model.T:
+                R = reversed_transition(model.B[f][:, :, model.act[t, f]])
+                retro = np.zeros(model.n[f])
+                for s in range(model.n[f]):
+                    for r in range(model.n[f]):
+                        retro[s] += R[s, r] * q[t + 1, lo + r]
+                x += 0.5 * _ln(retro)
+            x -= x.max()
+            e = np.exp(x)
+            out[t, lo:hi] = e / e.sum()
+    return out

@@ -15,7 +15,7 @@ import pytest
 
 import oracle
 from biwl import make_config, make_model, sample_streams
-from bruteforce import TinyModel, hmm_forward
+from bruteforce import TinyModel, hmm_forward, mmp_update_by_definition, reversed_transition
 from conftest import read_golden
 
 
@@ -173,6 +173,115 @@ def test_jacobi_schedule_composes():
         for _ in range(3):
             q, _, _ = run(algo, w, 1, q_init=q)
         np.testing.assert_allclose(q, q3, atol=1e-14)
+
+
+# ---- the marginal-message-passing reading: half weights and the reversed transition ----
+
+def test_golden_mmp_future_message(golden_dir):
+    # a transition matrix with unequal row sums and a mixed belief at the later step: the backward
+    # message varies over states, so the reversed matrix's normalisation axis and the 1/2 weight show
+    g = read_golden(os.path.join(golden_dir, "mmp_future_message.txt"))
+    A = [g["A"].reshape(1, 2, 2).astype(np.float32)]
+    B = [g["B"].reshape(1, 2, 2, 1).astype(np.float32)]
+    D = [g["D"].reshape(1, 2).astype(np.float32)]
+    obs = g["obs"].astype(np.int32).reshape(1, 2, 1)
+    act = np.zeros((1, 1, 1), np.int32)
+    start = np.stack([g["q1_start"], g["q2_start"]])[None]
+    for algo in ("mmp", "vmp"):
+        q, lq, _ = oracle.run(algo, [2], [2], [[0]], [1], 1, A, B, D, obs, act, 1, q_init=start)
+        np.testing.assert_allclose(q[0, 0], g["q1_" + algo], atol=2e-7)     # inputs are float32
+        np.testing.assert_allclose(q[0, 1], g["q2_" + algo], atol=2e-7)
+        np.testing.assert_allclose(np.exp(lq), q, atol=1e-14)
+
+
+def test_reversed_transition_of_a_permutation_is_its_transpose():
+    # a deterministic, invertible transition: knowing s_{t+1} fixes s_t, so the backward message is
+    # the later belief carried back through the permutation, whatever the prior on s_t
+    perm = [2, 0, 3, 1]                      # s_{t+1} = perm[s_t]
+    Bu = np.zeros((4, 4))
+    for s, r in enumerate(perm):
+        Bu[r, s] = 1.0
+    np.testing.assert_array_equal(reversed_transition(Bu), Bu.T)
+    A = [np.full((1, 2, 4), 0.5, np.float32)]
+    B = [Bu.reshape(1, 4, 4, 1).astype(np.float32)]
+    D = [np.full((1, 4), 0.25, np.float32)]
+    q2 = np.array([0.1, 0.2, 0.3, 0.4])
+    start = np.stack([np.full(4, 0.25), q2])[None]
+    q, _, _ = oracle.run("mmp", [4], [2], [[0]], [1], 1, A, B, D, np.zeros((1, 2, 1), np.int32),
+                         np.zeros((1, 1, 1), np.int32), 1, q_init=start)
+    want = np.sqrt(q2[perm])                 # q_1[s] ∝ sqrt(q_2[perm[s]])
+    np.testing.assert_allclose(q[0, 0], want / want.sum(), atol=1e-14)
+
+
+@pytest.mark.parametrize("seed,n,m,dep,U,sparsity", [
+    (91, [3], [3], [[0]], [2], 0.0),
+    (92, [2, 3], [2, 3], [[0, 1], [1]], [2, 1], 0.0),
+    (93, [3, 2], [3, 2], [[1, 0], [0]], [1, 3], 0.5),
+])
+def test_mmp_update_matches_the_reading_written_from_the_definition(seed, n, m, dep, U, sparsity):
+    w = tiny(seed, n, m, dep, U, T=3, sparsity=sparsity)
+    model = tm(w)
+    rng = np.random.default_rng(seed)
+    q0 = np.concatenate([rng.dirichlet(np.ones(k), size=3) for k in n], axis=1)
+    q1, _, _ = run("mmp", w, 1, q_init=q0[None])
+    np.testing.assert_allclose(q1[0], mmp_update_by_definition(model, q0), atol=1e-12)
+    # and the iteration is that update composed with itself
+    q2, _, _ = run("mmp", w, 2, q_init=q0[None])
+    np.testing.assert_allclose(q2[0], mmp_update_by_definition(model, mmp_update_by_definition(model, q0)),
+                               atol=1e-12)
+
+
+def test_mmp_unreachable_next_state_gives_a_uniform_backward_column():
+    # state 2 can never be entered (its row of B is zero): conditioning on s_{t+1} = 2 is undefined and
+    # the reading takes the uniform prior there; a later belief with mass on state 2 exercises it
+    Bu = np.array([[0.6, 0.2, 1.0], [0.4, 0.8, 0.0], [0.0, 0.0, 0.0]])
+    R = reversed_transition(Bu)
+    np.testing.assert_allclose(R[:, 2], 1.0 / 3.0)
+    A = [np.array([[[0.5, 0.3, 0.2], [0.5, 0.7, 0.8]]], np.float32)]
+    B = [Bu.reshape(1, 3, 3, 1).astype(np.float32)]
+    D = [np.array([[0.2, 0.3, 0.5]], np.float32)]
+    obs = np.array([[[1], [0]]], np.int32)
+    q2 = np.array([0.25, 0.15, 0.6])
+    start = np.stack([np.full(3, 1.0 / 3.0), q2])[None]
+    q, _, _ = oracle.run("mmp", [3], [2], [[0]], [1], 1, A, B, D, obs, np.zeros((1, 1, 1), np.int32), 1,
+                         q_init=start)
+    Bf = B[0][0, :, :, 0].astype(np.float64)
+    retro = np.array([0.25 * Bf[0, s] / Bf[0].sum() + 0.15 * Bf[1, s] / Bf[1].sum() + 0.6 / 3.0 for s in range(3)])
+    want = D[0][0].astype(np.float64) * A[0][0, 1].astype(np.float64) * np.sqrt(retro)
+    np.testing.assert_allclose(q[0, 0], want / want.sum(), atol=1e-14)
+
+
+# ---- P6: Gauss-Seidel sweeps reach a fixed point, free energy never rising ---------
+
+def test_gauss_seidel_sweeps_reach_a_fixed_point():
+    w = tiny(32, [2, 3], [2, 3], [[0, 1], [1]], [2, 2], T=2)
+    model = tm(w)
+    rng = np.random.default_rng(1)
+    q = np.concatenate([rng.dirichlet(np.ones(2), size=2), rng.dirichlet(np.ones(3), size=2)], axis=1)
+    coords = list(itertools.product(range(2), range(2)))
+
+    def sweep(q):
+        for t, f in coords:           # one coordinate at a time: the Jacobi result, one block taken
+            upd, _, _ = run("vmp", w, 1, q_init=q[None])
+            q = q.copy()
+            q[t, model.off[f]:model.off[f + 1]] = upd[0, t, model.off[f]:model.off[f + 1]]
+        return q
+
+    f_prev = model.free_energy(q)
+    for i in range(500):
+        q = sweep(q)
+        if i < 40 or i % 20 == 0:     # the enumeration is the slow part; checked densely early on
+            f_new = model.free_energy(q)
+            assert f_new <= f_prev + 1e-12
+            f_prev = f_new
+    q_next = sweep(q)
+    assert np.abs(q_next - q).max() < 1e-12
+    assert model.free_energy(q_next) <= f_prev + 1e-12
+    assert f_prev >= -model.ln_evidence() - 1e-12
+    # at the fixed point every coordinate is its own enumerated optimum
+    for t, f in coords:
+        np.testing.assert_allclose(q[t, model.off[f]:model.off[f + 1]], model.coordinate_optimum(q, t, f),
+                                   atol=1e-10)
 
 
 # ---- P4: window edge conventions ------------------------------------------------
