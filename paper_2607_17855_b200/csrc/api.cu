@@ -127,6 +127,32 @@ __global__ void bi_pack_tile_kernel(PackTile p) {
   ((R *)p.dst)[e] = out;
 }
 
+// Pre-summed slices of a register-tile group: out[g][combo][e] = sum over the group's members, in
+// member order (the order the kernels add them in), of that member's slice for its outcome in combo.
+struct PackComb {
+  const void *src[4];
+  int32_t m[4], mul[4];
+  int32_t nmem, ncomb, P_tile;
+  int64_t total;   // G * ncomb * P_tile
+  void *dst;
+};
+template <typename R>
+__global__ void bi_pack_comb_kernel(PackComb p) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= p.total) return;
+  const int e = (int)(i % p.P_tile);
+  const int64_t gc = i / p.P_tile;
+  int combo = (int)(gc % p.ncomb);
+  const int64_t g = gc / p.ncomb;
+  R acc = (R)0;
+  for (int mi = 0; mi < p.nmem; ++mi) {
+    const int o = combo / p.mul[mi];
+    combo -= o * p.mul[mi];
+    acc += ((const R *)p.src[mi])[((size_t)g * p.m[mi] + o) * p.P_tile + e];
+  }
+  ((R *)p.dst)[i] = acc;
+}
+
 template <typename R>
 __global__ void bi_pack_D_kernel(const float *__restrict__ D, int G, int n, int npad, R *logD) {
   int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -424,6 +450,50 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
         if (arith == BI_ARITH_F64) bi_pack_tile_kernel<double><<<(unsigned)tb, threads, 0, stream>>>(q);
         else bi_pack_tile_kernel<float><<<(unsigned)tb, threads, 0, stream>>>(q);
         if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+      }
+    }
+  }
+  // register-tile models: the pre-summed table over every outcome combination, while it stays small
+  // enough to live in L2 beside everything else (at most 4 modalities, at most 8 MiB)
+  md->tile_comb = nullptr;
+  md->tile_ncomb = 0;
+  if (rc == BI_OK && md->tile_sb == 1 && arith == BI_ARITH_F64) {   // (read by the float64 filtering kernel only)
+    const BiGroup &g0 = h.grp[0];
+    const int nm = g0.mem_end - g0.mem_begin;
+    double ncomb = 1.0;
+    for (int mi = g0.mem_begin; mi < g0.mem_end; ++mi) ncomb *= h.mem[mi].m;
+    const double bytes = ncomb * (double)G * md->tile_P * (double)esz;
+    if (nm == 1) {
+      md->tile_comb = const_cast<void *>(h.mem[g0.mem_begin].logA_tile);
+      md->tile_ncomb = h.mem[g0.mem_begin].m;
+      md->tile_comb_mul[0] = 1;
+    } else if (nm <= 4 && bytes <= 8.0 * 1024 * 1024) {
+      PackComb q;
+      memset(&q, 0, sizeof(q));
+      q.nmem = nm;
+      q.ncomb = (int)ncomb;
+      q.P_tile = md->tile_P;
+      int mul = 1;
+      for (int j = nm - 1; j >= 0; --j) {
+        const BiMember &mm = h.mem[g0.mem_begin + j];
+        q.src[j] = mm.logA_tile;
+        q.m[j] = mm.m;
+        q.mul[j] = mul;
+        md->tile_comb_mul[j] = mul;
+        mul *= mm.m;
+      }
+      q.total = (int64_t)G * q.ncomb * q.P_tile;
+      void *td = nullptr;
+      rc = dev_alloc(md, &td, (size_t)q.total * esz);
+      if (rc == BI_OK) {
+        q.dst = td;
+        const int threads = 256;
+        const int64_t tb = (q.total + threads - 1) / threads;
+        if (arith == BI_ARITH_F64) bi_pack_comb_kernel<double><<<(unsigned)tb, threads, 0, stream>>>(q);
+        else bi_pack_comb_kernel<float><<<(unsigned)tb, threads, 0, stream>>>(q);
+        if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+        md->tile_comb = td;
+        md->tile_ncomb = q.ncomb;
       }
     }
   }

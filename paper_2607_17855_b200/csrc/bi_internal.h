@@ -84,7 +84,7 @@ struct alignas(16) BiDev {
 struct bi_model {
   BiDev h;          // host copy (device pointers inside)
   BiDev *d;         // device copy
-  void *allocs[8 + 2 * BI_MAX_M + 8 * BI_MAX_F];  // status, descriptor, 2 per modality, 7 per factor
+  void *allocs[10 + 2 * BI_MAX_M + 8 * BI_MAX_F];  // status, descriptor, pre-summed table, 2 per modality, 7 per factor
   int nalloc;
   int arith;        // BI_ARITH_F64 or BI_ARITH_F32
   int device;
@@ -92,6 +92,13 @@ struct bi_model {
   int max_smem_optin;
   int tile_sb;      // > 0: a register-tile shape matches; lanes along b per (agent, step)
   int tile_P;       // elements per lane-interleaved slice
+  // Register-tile models with few outcome combinations: the group's slices pre-summed for every
+  // combination, [G][tile_ncomb][tile_P] in the lane-interleaved layout (one gather per step instead of
+  // one per modality and no additions); combination index = sum_i outcome_i * tile_comb_mul[i] over the
+  // group's members.  NULL when the table would be too large.
+  void *tile_comb;
+  int tile_ncomb;
+  int tile_comb_mul[BI_MAX_M];
   int V0max, V1max; // floats needed by the generic kernel's two intermediate buffers
   int rows_max;     // largest first-level row count over groups
   int64_t launches;

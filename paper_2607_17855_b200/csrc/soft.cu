@@ -184,6 +184,10 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     mm.P_pad = g.P_pad;
     sh.h.m[k] = T;
   }
+  // (a group of one modality is its own pre-summed table: the shadow's T per-agent slices)
+  sh.tile_comb = tile ? w + off_tile : nullptr;
+  sh.tile_ncomb = T;
+  sh.tile_comb_mul[0] = 1;
   sh.d = reinterpret_cast<BiDev *>(w + off_desc);
   // (the shadow borrows the handle's batched-path workspace and hands it back below)
   if (cudaMemcpyAsync(sh.d, &sh.h, sizeof(BiDev), cudaMemcpyHostToDevice, stream) != cudaSuccess) return BI_ERR_CUDA;

@@ -10,6 +10,8 @@
 
 // (the damped update's instantiations live in tile3_damped.cu)
 int bi_tile3_filter_damped(const Tile3Params &p, int arith, int na, int nb, int nc, cudaStream_t stream);
+// (the float64 kernel of the plain update, for the tile shapes it covers, in tile3_filter_f64.cu)
+int bi_tile3_filter_f64(const Tile3Params &p, int na, int nb, int nc, cudaStream_t stream);
 
 
 int bi_tile3_shape(int na, int nb, int nc) {
@@ -33,10 +35,11 @@ int bi_launch_tile3(const BiCall &c, bi_model *mut) {
   int rc;
   if (p.lambda != 1.0)
     rc = bi_tile3_filter_damped(p, md->arith, g.dim[0], g.dim[1], g.dim[2], c.stream);
-  else
-    rc = md->arith == BI_ARITH_F64
-             ? tile3_filter::dispatch_filter<double, false>(p, g.dim[0], g.dim[1], g.dim[2], c.stream)
-             : tile3_filter::dispatch_filter<float, false>(p, g.dim[0], g.dim[1], g.dim[2], c.stream);
+  else if (md->arith == BI_ARITH_F64) {
+    rc = bi_tile3_filter_f64(p, g.dim[0], g.dim[1], g.dim[2], c.stream);
+    if (rc == BI_ERR_UNSUPPORTED) rc = tile3_filter::dispatch_filter<double, false>(p, g.dim[0], g.dim[1], g.dim[2], c.stream);
+  } else
+    rc = tile3_filter::dispatch_filter<float, false>(p, g.dim[0], g.dim[1], g.dim[2], c.stream);
   if (rc == BI_OK) {
     mut->launches += 1;
     mut->last_kernel = md->arith == BI_ARITH_F64 ? "tile3_filter_f64" : "tile3_filter_f32";

@@ -14,6 +14,8 @@ struct Tile3Params {
   int64_t gstride[BI_MAX_M];
   int32_t modality[BI_MAX_M], mcount[BI_MAX_M];
   int32_t nmem, P_tile;
+  const void *Lcomb;        // the group's slices pre-summed for every outcome combination [G][ncomb][P_tile], or NULL
+  int32_t ncomb, comb_mul[BI_MAX_M];   // combination index = sum_i outcome_i * comb_mul[i]
   int32_t fac[3];   // factor ids of the axes a, b, c
   int32_t off[3];   // offsets of those factors in an output belief vector
   int32_t np[3];    // padded row length of their transition matrices
@@ -57,6 +59,9 @@ static inline void bi_tile3_fill_params(const BiCall &c, Tile3Params &p) {
   const BiDev &h = md->h;
   const BiGroup &g = h.grp[0];
   p.nmem = g.mem_end - g.mem_begin;
+  p.Lcomb = md->tile_comb;
+  p.ncomb = md->tile_ncomb;
+  for (int i = 0; i < p.nmem; ++i) p.comb_mul[i] = md->tile_comb_mul[i];
   p.P_tile = md->tile_P;
   for (int i = 0; i < p.nmem; ++i) {
     const BiMember &mm = h.mem[g.mem_begin + i];
