@@ -630,3 +630,37 @@ def test_fma_probe_reports_a_plausible_rate():
     import paper_2607_17855_b200 as bi
     f64, f32 = bi.bi_probe_fma("f64"), bi.bi_probe_fma("f32")
     assert 1.0 < f64 < 200.0 and f64 < f32 < 400.0, (f64, f32)
+
+
+def test_golden_mmp_backward_message_on_the_gpu(golden_dir):
+    """The hand-worked two-step window whose backward message varies over states (unequal row sums of
+    the transition matrix), one iteration from the fixture's start, through bi_mmp_warm / bi_vmp_warm."""
+    import torch
+    import paper_2607_17855_b200 as bi
+    from conftest import read_golden
+    g = read_golden(os.path.join(golden_dir, "mmp_future_message.txt"))
+    A = [torch.tensor(g["A"].reshape(1, 2, 2), dtype=torch.float32, device="cuda")]
+    B = [torch.tensor(g["B"].reshape(1, 2, 2, 1), dtype=torch.float32, device="cuda")]
+    D = [torch.tensor(g["D"].reshape(1, 2), dtype=torch.float32, device="cuda")]
+    md = bi.Model([2], [2], [[0]], [1], 1, A, B, D)
+    obs = torch.tensor(g["obs"].reshape(1, 2, 1), dtype=torch.int32, device="cuda")
+    act = torch.zeros((1, 1, 1), dtype=torch.int32, device="cuda")
+    start = torch.tensor(np.stack([g["q1_start"], g["q2_start"]])[None], dtype=torch.float32, device="cuda")
+    for algo, fn in (("mmp", md.bi_mmp_warm), ("vmp", md.bi_vmp_warm)):
+        q = fn(obs, act, start, 1).cpu().numpy()
+        np.testing.assert_allclose(q[0, 0], g["q1_" + algo], atol=3e-7)
+        np.testing.assert_allclose(q[0, 1], g["q2_" + algo], atol=3e-7)
+    # a permutation transition: the backward message carries the later belief back through it
+    perm = [2, 0, 3, 1]
+    Bu = np.zeros((4, 4), np.float32)
+    for s_, r_ in enumerate(perm):
+        Bu[r_, s_] = 1.0
+    md2 = bi.Model([4], [2], [[0]], [1], 1, [torch.full((1, 2, 4), 0.5, device="cuda")],
+                   [torch.tensor(Bu.reshape(1, 4, 4, 1), device="cuda")], [torch.full((1, 4), 0.25, device="cuda")])
+    q2 = np.array([0.1, 0.2, 0.3, 0.4])
+    start = torch.tensor(np.stack([np.full(4, 0.25), q2])[None], dtype=torch.float32, device="cuda")
+    q = md2.bi_mmp_warm(torch.zeros((1, 2, 1), dtype=torch.int32, device="cuda"), act, start, 1).cpu().numpy()
+    want = np.sqrt(q2[perm])
+    np.testing.assert_allclose(q[0, 0], want / want.sum(), atol=3e-7)
+    md.close()
+    md2.close()
