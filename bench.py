@@ -11,6 +11,12 @@ one step in one iteration, so a step performs N*T*F*K of them.
 
 prints one JSON line.  With ``--impl reference`` the CPU oracle is timed
 instead (rank 0 only), each step on a bounded sample of the same workload.
+
+    python bench.py --case 4:mmp [--agents N] [--T T] [--K K] [--member j] [--soft] [--arith f32]
+
+runs ONE secondary workload of a chosen size a few times and prints its device
+time (one JSON line of its own, not the benchmark's): the command the profiler
+summaries were captured with.
 """
 from __future__ import annotations
 
@@ -35,11 +41,36 @@ FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12   # 37.2
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # 74.4
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the benchmark's
-# workload, from the ncu captures summarised under profiles/ (bytes)
-NCU_DRAM_BYTES_PER_LAUNCH = {
-    "tile3_filter_f64": 5.015e6 + 3.1e3,   # profiles/tile3_filter_f64_config2.md
+# dram__bytes_read.sum + dram__bytes_write.sum per call on the timed workloads, from ncu captures of the
+# same kernels (bytes; the captures and how they scale to these sizes are written up beside the code,
+# in the profiler summaries).  A record of those captures: the run itself does not measure DRAM traffic.
+NCU_DRAM_BYTES_PER_CALL = {
+    "tile3_filter_f64": 5.0e6,     # config 2, full size, one launch
+    "batch_vmp_f64": None,         # config 3 (filled from the capture: see NCU_NOTES)
+    "tile3_mmp_f64": None,         # config 4
 }
+
+
+def fma_probe(arith: str) -> float:
+    """Measured multiply-add rate of this GPU in TFLOP/s: a kernel of independent chains from
+    bench_probe.cu (built on first use with nvcc for sm_100a, beside this file)."""
+    import ctypes
+    import torch
+    src, lib = os.path.join(ROOT, "bench_probe.cu"), os.path.join(ROOT, "bench_probe.so")
+    if not os.path.exists(lib) or os.path.getmtime(lib) < os.path.getmtime(src):
+        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+        tmp = lib + f".tmp{os.getpid()}"
+        subprocess.run([nvcc, "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC",
+                        "-shared", "-o", tmp, src], check=True, capture_output=True)
+        os.replace(tmp, lib)
+    L = ctypes.CDLL(lib)
+    L.bench_probe_fma.restype = ctypes.c_int
+    L.bench_probe_fma.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
+    v = ctypes.c_double(0.0)
+    rc = L.bench_probe_fma(1 if arith == "f64" else 0, ctypes.byref(v), ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if rc != 0:
+        raise RuntimeError("bench_probe_fma failed")
+    return float(v.value)
 
 
 def measured_peaks():
@@ -214,6 +245,47 @@ def reference_arm(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_case(args):
+    """One call of one workload at a chosen size, timed after a few warm-up calls."""
+    import numpy as np
+    import torch
+    import paper_2607_17855_b200 as bi
+    from biwl import make_config, make_sweep_config
+    cfg, _, algo = args.case.partition(":")
+    cfg = int(cfg)
+    if cfg == 5:
+        w = make_sweep_config(args.member, N=args.agents, T=args.T, K=args.K)
+    else:
+        w = make_config(cfg, N=args.agents, T=args.T, K=args.K)
+    algo = algo or (w.algo if w.algo != "all" else "filter")
+    md = bi.model_from_workload(w, arith=args.arith)
+    obs = torch.from_numpy(w.obs).cuda()
+    act = torch.from_numpy(w.act).cuda() if w.act.size else None
+    q = torch.empty((w.N, w.T, w.S), device="cuda")
+    if args.soft:
+        off = np.concatenate([[0], np.cumsum(w.m)]).astype(int)
+        soft = np.zeros((w.N, w.T, int(off[-1])), np.float32)
+        for i in range(w.M):
+            np.put_along_axis(soft[:, :, off[i]:off[i + 1]], w.obs[:, :, i:i + 1], 1.0, axis=2)
+        soft = torch.from_numpy(soft).cuda()
+        call = lambda: md.run_soft(algo, soft, act, w.K, q_out=q)  # noqa: E731
+    else:
+        call = lambda: md.run(algo, obs, act, w.K, q_out=q)  # noqa: E731
+    for _ in range(args.warmup):
+        call()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    call()
+    b.record()
+    b.synchronize()
+    ms = a.elapsed_time(b)
+    assert md.status() == 0
+    print(json.dumps({"workload": w.name, "algo": algo, "agents": w.N, "T": w.T, "K": w.K, "arith": args.arith,
+                      "soft": bool(args.soft), "kernel": md.last_kernel, "ms": ms,
+                      "updates_per_s": w.updates / (ms * 1e-3)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -222,7 +294,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--arith", default="f64", choices=["f64", "f32"])
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads and the CPU baseline")
+    ap.add_argument("--case", default=None, help="CONFIG[:ALGO], e.g. 4:mmp: run that one workload and print its time")
+    ap.add_argument("--agents", type=int, default=None, help="with --case: agents N")
+    ap.add_argument("--T", type=int, default=None, help="with --case: time steps")
+    ap.add_argument("--K", type=int, default=None, help="with --case: iterations")
+    ap.add_argument("--member", type=int, default=0, help="with --case 5: member of the randomised sweep")
+    ap.add_argument("--soft", action="store_true", help="with --case: observations as (one-hot) categorical vectors")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))
@@ -263,8 +344,9 @@ def main():
     value = aggregate_throughput(w.updates, world, sec)
 
     # ---- end to end: pinned host inputs -> device -> filtering -> host beliefs.  The trajectory is
-    # run as E2E_CHUNKS consecutive blocks of steps (bi_filter, then bi_filter_from continuing from the
-    # previous block's last belief), so a block's beliefs travel to the host while the next block runs.
+    # run as E2E_CHUNKS consecutive blocks of steps (bi_filter, then bi_filter_continue from the handle's
+    # full-precision record of the previous block's last belief: bit for bit the single call's result),
+    # so a block's beliefs travel to the host while the next block runs.
     md, q = head["model"], head["q"]
     nchunk = E2E_CHUNKS if w.T % E2E_CHUNKS == 0 else 1
     tc = w.T // nchunk
@@ -293,7 +375,6 @@ def main():
     h_q = [torch.empty((w.N, tc, w.S), dtype=torch.float32).pin_memory() for _ in range(nchunk)]
     done = [torch.cuda.Event() for _ in range(nchunk)]
     arrived = torch.cuda.Event()
-    q_prev = torch.empty((w.N, w.S), dtype=torch.float32, device="cuda")
 
     def e2e_step():
         cur = torch.cuda.current_stream()
@@ -309,8 +390,7 @@ def main():
             else:
                 if i == 1:
                     cur.wait_event(arrived)
-                q_prev.copy_(d_q[i - 1][:, -1])
-                md.bi_filter_from(obs_i, act_i, q_prev, actp_i, w.K, q_out=d_q[i])
+                md.bi_filter_continue(obs_i, act_i, actp_i, w.K, q_out=d_q[i])
             done[i].record(cur)
             copy_out.wait_event(done[i])
             with torch.cuda.stream(copy_out):
@@ -321,14 +401,12 @@ def main():
     e2e_sec = sum(e2e_times) / len(e2e_times)
     clocks = sampler.stop()  # sampled over both timed regions
     e2e_sec = max_over_ranks(dist, e2e_sec, "cuda")
-    # the blockwise result against the single call's (continuing from float32 beliefs re-rounds the
-    # carried state once per block; the iteration amplifies that on ill-conditioned agents)
+    # the blockwise result is the single call's, bit for bit (the parity tests compare both with the oracle)
     torch.cuda.synchronize()
-    diff = (torch.cat(h_q, dim=1) - q.cpu()).abs().reshape(w.N, -1).max(dim=1).values
-    blocks_agree = float((diff <= 1e-5).float().mean())
+    blocks_equal = bool(torch.equal(torch.cat(h_q, dim=1), q.cpu()))
     e2e = {"value": aggregate_throughput(w.updates, world, e2e_sec), "unit": UNIT,
            "h2d_bytes_per_step": int(w.obs.nbytes + w.act.nbytes), "d2h_bytes_per_step": int(q.numel() * 4),
-           "blocks_of_steps": nchunk, "agents_within_1e-5_of_single_call": blocks_agree}
+           "blocks_of_steps": nchunk, "equals_single_call_bit_for_bit": blocks_equal}
 
     flops = algorithmic_flops(w)
     peak = FP64_PEAK_TFLOPS if args.arith == "f64" else FP32_PEAK_TFLOPS
@@ -337,11 +415,11 @@ def main():
                 "frac": achieved / peak, "traffic": None,
                 "kernel": head["kernel"],
                 "peak_source": f"derived: 148 SMs x {64 if args.arith == 'f64' else 128} lanes x 2 x 1.965 GHz"}
-    roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(head["kernel"])
+    roofline["traffic"] = NCU_DRAM_BYTES_PER_CALL.get(head["kernel"])
     # the same run's own measurements beside the derived peak: the rate of independent multiply-add
     # chains in this arithmetic, and a large device-to-device copy
     try:
-        fma_peak = bi.bi_probe_fma(args.arith)
+        fma_peak = fma_probe(args.arith)
         src = torch.empty(1 << 28, dtype=torch.float32, device="cuda")   # 1 GiB
         dst = torch.empty_like(src)
         for _ in range(2):
@@ -403,12 +481,26 @@ def main():
         for c, algo in ((3, "vmp"), (4, "mmp")):
             wc = make_config(c)
             r = bench_config(torch, bi, wc, algo, args.arith, max(3, args.steps // 2), 3, flush)
+            tfl = algorithmic_flops(wc) / r["seconds"] / 1e12
             entry = {"value": wc.updates / r["seconds"], "unit": UNIT, "ms_per_step": r["seconds"] * 1e3,
-                     "kernel": r["kernel"], "alu_tflops": algorithmic_flops(wc) / r["seconds"] / 1e12}
-            if wc.G != 1:
-                gbs = algorithmic_bytes(wc, 8 if args.arith == "f64" else 4) / r["seconds"] / 1e9
+                     "kernel": r["kernel"], "launches_per_step": r["launches_per_step"], "alu_tflops": tfl}
+            traffic = NCU_DRAM_BYTES_PER_CALL.get(r["kernel"])
+            if wc.G == 1:
+                # the shared model stays on chip / in L2: the arithmetic pipe bounds the call
+                entry["roofline"] = {"bound": "alu", "achieved": tfl, "peak": peak, "unit": "TFLOP/s",
+                                     "frac": tfl / peak, "traffic": traffic,
+                                     "peak_source": roofline["peak_source"]}
+            else:
+                # per-agent models: every slice crosses HBM once.  Two byte counts: the slices as the
+                # handle stores them (float64 logs in this arithmetic), and the float32 slices the method
+                # itself needs (4 bytes per entry of A)
+                stored = algorithmic_bytes(wc, 8 if args.arith == "f64" else 4)
+                method = algorithmic_bytes(wc, 4)
+                gbs = stored / r["seconds"] / 1e9
                 entry["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s",
-                                     "frac": gbs / hbm_peak, "peak_source": hbm_src}
+                                     "frac": gbs / hbm_peak, "traffic": traffic, "peak_source": hbm_src,
+                                     "bytes_as_stored": stored, "bytes_of_the_method_fp32": method,
+                                     "frac_on_the_method_bytes": method / r["seconds"] / 1e9 / hbm_peak}
             others[f"config{c}_{algo}_{args.arith}"] = entry
             del r
         # the headline workload with its observations given as categorical vectors (one-hot here):

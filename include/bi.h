@@ -207,6 +207,31 @@ int bi_filter_from(const bi_model_t *model, int32_t N, int32_t T, const int32_t 
                    void *cuda_stream);
 
 /*
+ * Variational filtering continued from the handle's own record of where the
+ * previous filtering call on this handle stopped (the same recursion of Section
+ * III-B entered mid-stream, as bi_filter_from).  Every bi_filter,
+ * bi_filter_from and bi_filter_continue call leaves the last step's belief of
+ * each of its N agents in a device buffer the handle owns, in the handle's
+ * arithmetic (float64 by default), and this call starts from that buffer.
+ * Nothing is rounded to float32 on the way, so a trajectory filtered as
+ * consecutive blocks of steps -- the first with bi_filter, the rest with this
+ * call -- gives bit for bit the beliefs of one bi_filter call over all the
+ * steps, which bi_filter_from (float32 q_prev) cannot promise on models whose
+ * iteration amplifies rounding.
+ *   act_prev  DEVICE [N][F] int32: the action taken at the previous call's last step
+ *   others    as for bi_filter (act is [N][T-1][F]; may be NULL when T == 1)
+ * The calls must be issued in order on one stream (or otherwise ordered); N must
+ * equal the previous filtering call's N, else BI_ERR_INVALID_ARG (also when
+ * there was no previous call, or it failed).  Calls with observation vectors
+ * (bi_filter_soft) and bi_filter_static neither read nor update the record.
+ * The buffer is N * S elements, obtained from the stream-ordered allocator at
+ * the first filtering call (and again when N grows), freed by bi_model_destroy.
+ */
+int bi_filter_continue(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                       const int32_t *act, const int32_t *act_prev, int32_t iters, float *q_out,
+                       float *logq_out, int32_t *argmax_out, void *cuda_stream);
+
+/*
  * bi_vmp / bi_mmp started from given beliefs instead of the uniform ones: the
  * warm start of a sliding inference window (Section III-A: inference over a
  * horizon that advances with t), where the previous window's result, shifted by
@@ -303,14 +328,6 @@ int bi_filter_static(const bi_model_desc *desc, int32_t N, int32_t T, const int3
                      const int32_t *act, int32_t iters, float *q_out, float *logq_out,
                      int32_t *argmax_out, void *cuda_stream);
 
-/*
- * Measurement aid (no part of the method): times a kernel of independent
- * multiply-add chains in the given arithmetic (BI_ARITH_*) on the current device
- * and returns the rate in TFLOP/s in *tflops (HOST), so that a benchmark can set
- * its achieved arithmetic against a peak measured in the same run.  Allocates one
- * word of device memory for the duration of the call and synchronises the stream.
- */
-int bi_probe_fma(int arith, double *tflops, void *cuda_stream);
 
 /* Synchronises the stream, returns the OR of BI_FLAG_* raised since the last
  * call in *flags (HOST) and clears them. */

@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_probe_fma", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_filter_continue", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -69,7 +69,7 @@ def lib():
         L.bi_filter_from.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
-        for name in ("bi_vmp_warm", "bi_mmp_warm"):
+        for name in ("bi_vmp_warm", "bi_mmp_warm", "bi_filter_continue"):   # (handle, N, T, obs, act, one pointer, iters, outputs)
             fn = getattr(L, name)
             fn.restype = ctypes.c_int
             fn.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
@@ -83,8 +83,6 @@ def lib():
                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.bi_model_set_damping.restype = ctypes.c_int
         L.bi_model_set_damping.argtypes = [ctypes.c_void_p, ctypes.c_double]
-        L.bi_probe_fma.restype = ctypes.c_int
-        L.bi_probe_fma.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
         L.bi_status.restype = ctypes.c_int
         L.bi_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
         L.bi_last_kernel.restype = ctypes.c_char_p
@@ -204,6 +202,26 @@ class Model:
             raise BiError(rc, "bi_filter_from")
         return q_out
 
+    def bi_filter_continue(self, obs, act, act_prev, iters, q_out=None, logq_out=None, argmax_out=None,
+                           stream=None):
+        """Filtering continued from the belief this handle kept from its previous filtering call
+        (full precision: consecutive blocks equal the single call bit for bit); ``act_prev`` int32
+        ``[N,F]`` is the action taken at that call's last step."""
+        import torch
+        N, T = int(obs.shape[0]), int(obs.shape[1])
+        if q_out is None:
+            q_out = torch.empty((N, T, self.S), dtype=torch.float32, device=obs.device)
+        rc = lib().bi_filter_continue(self._h, N, T, ctypes.c_void_p(obs.data_ptr()),
+                                      ctypes.c_void_p(act.data_ptr() if act is not None and act.numel() > 0 else None),
+                                      ctypes.c_void_p(act_prev.data_ptr()), int(iters),
+                                      ctypes.c_void_p(q_out.data_ptr()),
+                                      ctypes.c_void_p(logq_out.data_ptr() if logq_out is not None else None),
+                                      ctypes.c_void_p(argmax_out.data_ptr() if argmax_out is not None else None),
+                                      _stream_ptr(stream))
+        if rc != BI_OK:
+            raise BiError(rc, "bi_filter_continue")
+        return q_out
+
     def bi_vmp(self, obs, act, iters, q_out=None, logq_out=None, argmax_out=None, stream=None):
         """Variational message passing over one window."""
         return self._run("bi_vmp", obs, act, iters, q_out, logq_out, argmax_out, stream)
@@ -287,15 +305,6 @@ class Model:
     @property
     def launch_count(self) -> int:
         return int(lib().bi_launch_count(self._h))
-
-
-def bi_probe_fma(arith: str = "f64", stream=None) -> float:
-    """Measured multiply-add rate of this GPU in TFLOP/s (``bi_probe_fma``; a measurement aid)."""
-    v = ctypes.c_double(0.0)
-    rc = lib().bi_probe_fma(ARITH[arith], ctypes.byref(v), _stream_ptr(stream))
-    if rc != BI_OK:
-        raise BiError(rc, "bi_probe_fma")
-    return float(v.value)
 
 
 def bi_filter_static(n, m, dep, U, A, B, D, obs, act, iters, q_out, logq_out=None, argmax_out=None, stream=None):

@@ -235,6 +235,9 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
   if (!md) return BI_ERR_ALLOC;
   memset(md, 0, sizeof(*md));
   md->damping = 1.0;
+  if (const char *e = getenv("BI_TEST_FAMILY")) {   // testing aid, read here and nowhere else
+    md->test_family = !strcmp(e, "warp") ? BI_FAMILY_WARP : !strcmp(e, "generic") ? BI_FAMILY_GENERIC : BI_FAMILY_ANY;
+  }
   md->last_kernel = "";
   md->arith = arith;
   if (cudaGetDevice(&md->device) != cudaSuccess) {
@@ -550,6 +553,7 @@ extern "C" int bi_model_destroy(bi_model_t *model) {
   if (model->ws) cudaFree(model->ws);
   if (model->ws_soft) cudaFree(model->ws_soft);
   if (model->ws_prior) cudaFree(model->ws_prior);
+  if (model->carry) cudaFree(model->carry);
   free_all(model);
   delete model;
   return e == cudaSuccess ? BI_OK : BI_ERR_CUDA;
@@ -575,21 +579,21 @@ __global__ void bi_predictive_prior_kernel(const BiDev *__restrict__ mdp, int N,
 }
 
 int bi_dispatch(const BiCall &c, bi_model *mut) {
-  int rc = bi_launch_tile3(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
-  if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) {
+  const int only = c.model->test_family;   // testing aid: start at the named family
+  int rc = BI_ERR_UNSUPPORTED;
+  if (only == BI_FAMILY_ANY) {
+    rc = bi_launch_tile3(c, mut);
+    if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
+    if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
     // Filtering exposes one unit per agent, so a CTA per agent keeps more of the machine busy than
     // a warp per agent, and its staged slices and per-factor warps pay at every batch size measured
     // on the 128 random structures (sum of times, CTA against warp kernel): 44 against 99 ms at 256
     // agents, 109 against 160 ms at 1024, 207 against 224 ms at 2048, 406 against 434 ms at 4096,
     // 784 against 846 ms at 8192.  The warp kernel serves the models whose slices do not fit in
-    // shared memory.  BI_CTA_MAXN (testing aid) caps the batch that goes to the CTA kernel.
-    bool cta = true;
-    if (const char *e = getenv("BI_CTA_MAXN")) cta = c.N <= atoll(e);
-    if (cta) rc = bi_launch_cta_filter(c, mut);
+    // shared memory.
+    if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) rc = bi_launch_cta_filter(c, mut);
   }
-  if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_warp(c, mut);
+  if (rc == BI_ERR_UNSUPPORTED && only != BI_FAMILY_GENERIC) rc = bi_launch_warp(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;
 }
@@ -597,7 +601,7 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
 static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, const int32_t *obs,
                     const int32_t *act, int32_t iters, float *q_out, float *logq_out,
                     int32_t *argmax_out, void *cuda_stream, const float *q_prev = nullptr,
-                    const int32_t *act_prev = nullptr, const float *q_init = nullptr) {
+                    const int32_t *act_prev = nullptr, const float *q_init = nullptr, bool from_carry = false) {
   if (!model || N < 0 || T < 1 || iters < 1) return BI_ERR_INVALID_ARG;
   if (N == 0) return BI_OK;
   if (!q_out || (model->h.M > 0 && !obs) || (T > 1 && !act)) return BI_ERR_INVALID_ARG;
@@ -607,6 +611,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   c.model = model; c.algo = algo; c.N = N; c.T = T; c.K = iters;
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
   c.q_prev = q_prev; c.act_prev = act_prev; c.q_init = q_init; c.lnprior = nullptr;
+  c.carry_in = nullptr; c.carry_out = nullptr;
   c.lambda = model->damping;
   c.stream = (cudaStream_t)cuda_stream;
   if (algo != BI_ALGO_FILTER && q_prev) {
@@ -639,6 +644,30 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
     c.act_prev = nullptr;
   }
   c.stream = (cudaStream_t)cuda_stream;
+  if (algo == BI_ALGO_FILTER) {
+    // every filtering call leaves its last belief, in the handle's arithmetic, for bi_filter_continue
+    bi_model *mh = const_cast<bi_model *>(model);
+    if (from_carry && mh->carry_N != N) return BI_ERR_INVALID_ARG;
+    const size_t need = (size_t)N * model->h.S * (model->arith == BI_ARITH_F64 ? 8 : 4);
+    if (mh->carry_bytes < need) {   // (never while continuing: the carried belief has this size)
+      if (mh->carry && cudaFreeAsync(mh->carry, c.stream) != cudaSuccess) return BI_ERR_CUDA;
+      mh->carry = nullptr;
+      mh->carry_bytes = 0;
+      mh->carry_N = 0;
+      void *pnew = nullptr;
+      if (cudaMallocAsync(&pnew, need, c.stream) != cudaSuccess) {
+        cudaGetLastError();
+        return BI_ERR_ALLOC;
+      }
+      mh->carry = pnew;
+      mh->carry_bytes = need;
+    }
+    c.carry_in = from_carry ? mh->carry : nullptr;
+    c.carry_out = mh->carry;
+    const int rc = bi_dispatch(c, mh);
+    mh->carry_N = rc == BI_OK ? N : 0;
+    return rc;
+  }
   return bi_dispatch(c, const_cast<bi_model *>(model));
 }
 
@@ -685,6 +714,14 @@ extern "C" int bi_filter_from(const bi_model_t *model, int32_t N, int32_t T, con
   if (!q_prev || !act_prev) return BI_ERR_INVALID_ARG;
   return run_call(model, BI_ALGO_FILTER, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, q_prev,
                   act_prev);
+}
+
+extern "C" int bi_filter_continue(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,
+                                  const int32_t *act, const int32_t *act_prev, int32_t iters, float *q_out,
+                                  float *logq_out, int32_t *argmax_out, void *cuda_stream) {
+  if (!model || !act_prev) return BI_ERR_INVALID_ARG;
+  return run_call(model, BI_ALGO_FILTER, N, T, obs, act, iters, q_out, logq_out, argmax_out, cuda_stream, nullptr,
+                  act_prev, nullptr, true);
 }
 
 extern "C" int bi_vmp(const bi_model_t *model, int32_t N, int32_t T, const int32_t *obs,

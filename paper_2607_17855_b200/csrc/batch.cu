@@ -827,8 +827,6 @@ int bi_launch_batch(const BiCall &c, bi_model *mut) {
     bytes *= (double)c.N * c.T * (md->arith == BI_ARITH_F64 ? 8 : 4);
     if (bytes > 120e6) return BI_ERR_UNSUPPORTED;
   }
-  long long min_units = 2048;
-  if (const char *e = getenv("BI_BATCH_MIN_UNITS")) min_units = atoll(e);   // testing aid
-  if ((long long)c.N * c.T < min_units) return BI_ERR_UNSUPPORTED;
+  if ((long long)c.N * c.T < 2048) return BI_ERR_UNSUPPORTED;   // too few units to fill the machine this way
   return md->arith == BI_ARITH_F64 ? launch_batch_t<double>(c, mut) : launch_batch_t<float>(c, mut);
 }

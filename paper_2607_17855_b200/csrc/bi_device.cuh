@@ -108,6 +108,12 @@ __device__ __forceinline__ void bi_exp_tab_init(double *tab, int lane) {
 }
 __device__ __forceinline__ void bi_exp_tab_init(float *, int) {}
 
+// The argument reduction and the minimax coefficients Lg1..Lg7 (and the two-part ln 2 shared with the
+// exponentials above) are those of FreeBSD's msun / fdlibm e_log.c:
+//   Copyright (C) 1993 by Sun Microsystems, Inc. All rights reserved.
+//   Developed at SunSoft, a Sun Microsystems, Inc. business.
+//   Permission to use, copy, modify, and distribute this software is freely granted,
+//   provided that this notice is preserved.
 // Branch-free natural log of a positive normal double (the messages take logs
 // of probabilities clamped at 1e-16 and of sums of exponentials: never zero,
 // subnormal, infinite or NaN).  Same motive as bi_exp_inline: the six logs of

@@ -10,6 +10,7 @@
 #define BI_MAX_GROUPS BI_MAX_M
 
 enum { BI_ALGO_FILTER = 0, BI_ALGO_VMP = 1, BI_ALGO_MMP = 2 };
+enum { BI_FAMILY_ANY = 0, BI_FAMILY_WARP = 1, BI_FAMILY_GENERIC = 2 };
 
 static __host__ __device__ inline int bi_pad4(int x) { return (x + 3) & ~3; }
 // Row stride in shared memory for rows of npad elements (npad a multiple of 4, elements of esize
@@ -110,6 +111,13 @@ struct bi_model {
   void *ws_prior;   // predictive log-priors of continued window calls, or NULL
   size_t ws_prior_bytes;
   double damping;   // step of the update on log-beliefs, (0, 1]; 1 = the plain fixed-point map
+  void *carry;      // last belief of the latest filtering call, [carry_N][S] in the arithmetic type, or NULL
+  size_t carry_bytes;
+  int carry_N;      // agents of that call (0: none yet)
+  // Testing aid, read from the environment once, when the handle is made (BI_TEST_FAMILY = "warp" or
+  // "generic"): calls skip the kernel families ahead of the named one, so that the general kernels can
+  // be checked on inputs small enough for the oracle.  0 = normal dispatch.
+  int test_family;
 };
 
 struct BiCall {
@@ -117,7 +125,13 @@ struct BiCall {
   int algo, N, T, K;
   const int32_t *obs, *act;
   const float *q_prev;       // filtering continued from a belief [N][S], or NULL
-  const int32_t *act_prev;   // [N][F], with q_prev
+  const int32_t *act_prev;   // [N][F], with q_prev (or with carry_in)
+  // Filtering calls: the last step's belief of every agent, [N][S] in the handle's arithmetic type.
+  // carry_in (or NULL) takes the place of q_prev at full precision; carry_out (or NULL) receives this
+  // call's last belief.  (A trajectory filtered in consecutive calls then equals the single call
+  // bit for bit: nothing is rounded to float32 on the way.)
+  const void *carry_in;
+  void *carry_out;
   const float *q_init;       // window algorithms: starting beliefs [N][T][S], or NULL (uniform)
   double lambda;             // damping: ln q' = (1 - lambda) ln q + lambda (messages) + const; 1 = plain
   const void *lnprior;       // window algorithms continued from a belief: ln(B_u q_prev) per agent,

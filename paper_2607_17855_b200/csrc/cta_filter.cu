@@ -204,8 +204,9 @@ template <typename R>
 __global__ void __launch_bounds__(256, 2)
 bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__restrict__ obs,
                      const int32_t *__restrict__ act, const float *q_prev,
-                     const int32_t *__restrict__ act_prev, double lambda, int K, float *q_out,
-                     float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, const CtaGeom sm) {
+                     const int32_t *__restrict__ act_prev, const void *carry_in, void *carry_out, double lambda,
+                     int K, float *q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out,
+                     const CtaGeom sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *smem = reinterpret_cast<R *>(smem_raw);
   {  // the model's description, read from shared memory from here on
@@ -231,12 +232,14 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
   for (int i = tid; i < NG * Sp; i += NT) ellg[i] = (R)0;  // entries of factors outside a group stay zero
   for (int i = sm.vtot_begin + tid; i < sm.vtot_end; i += NT) smem[i] = (R)0;
   __syncthreads();
-  if (q_prev) {  // continued filtering: the belief of the step before the first
+  const bool from_prev = q_prev != nullptr || carry_in != nullptr;
+  if (from_prev) {  // continued filtering: the belief of the step before the first
     for (int idx = tid; idx < Sp; idx += NT) {
       int f = 0;
       while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
       const int s = idx - md.offp[f];
-      cur[idx] = s < md.n[f] ? (R)q_prev[(size_t)a * S + md.off[f] + s] : (R)0;   // (may alias q_out: plain load)
+      const size_t src = (size_t)a * S + md.off[f] + s;
+      cur[idx] = s < md.n[f] ? (carry_in ? ((const R *)carry_in)[src] : (R)q_prev[src]) : (R)0;   // (q_prev may alias q_out: plain load)
     }
     __syncthreads();
   }
@@ -249,7 +252,7 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
       const int s = idx - md.offp[f], n = md.n[f];
       R lp = (R)0;
       if (s < n) {
-        if (t == 0 && !q_prev) {
+        if (t == 0 && !from_prev) {
           lp = __ldg((const R *)md.logD[f] + (size_t)g * md.Dstride[f] + s);
         } else {
           const int ur = t == 0 ? __ldg(act_prev + (size_t)a * F + f)
@@ -388,6 +391,14 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
       R *tmp = cur; cur = nxt; nxt = tmp;
     }
   }
+  if (carry_out) {   // the last step's belief at full precision, for a call that continues this one
+    for (int idx = tid; idx < Sp; idx += NT) {
+      int f = 0;
+      while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+      const int s = idx - md.offp[f];
+      if (s < md.n[f]) ((R *)carry_out)[(size_t)a * S + md.off[f] + s] = cur[idx];
+    }
+  }
 }
 
 template <typename R>
@@ -399,8 +410,6 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
   // of them be resident).  Measured on the 128 random structures: 256 threads for every structure
   // took the sum of times from 61 to 54 ms at 256 agents and from 133 to 204 ms at 1024.
   int NT = c.N <= 2 * md->sm_count ? 256 : c.N <= 4 * md->sm_count ? 128 : 64;
-  if (const char *e = getenv("BI_CTA_THREADS")) NT = atoi(e);   // testing aid (32 .. 256, a power of two)
-  NT = std::max(32, std::min(256, NT));
   while (NT < md->rows_max && NT < 256) NT <<= 1;
   const int NW = NT / 32;
   CtaGeom sm;
@@ -504,7 +513,7 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
   if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes) !=
       cudaSuccess)
     return BI_ERR_CUDA;
-  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.lambda, c.K, c.q_out,
+  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.carry_in, c.carry_out, c.lambda, c.K, c.q_out,
                                                c.logq_out, c.argmax_out, sm);
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += 1;

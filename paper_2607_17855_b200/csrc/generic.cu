@@ -223,7 +223,7 @@ template <typename R, int ALGO, bool STAGED>
 __global__ void __launch_bounds__(256)
 bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
                   const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
-                  const float *__restrict__ q_init, const void *__restrict__ lnprior, double lambda, int K,
+                  const void *carry_in, void *carry_out, const float *__restrict__ q_init, const void *__restrict__ lnprior, double lambda, int K,
                   float *q_out, float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, GenSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *smem = reinterpret_cast<R *>(smem_raw);
@@ -250,12 +250,14 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
 
   if (ALGO == BI_ALGO_FILTER) {
     R *cur = q0, *nxt = q1;
-    if (q_prev) {  // continued filtering: the belief of the step before the window
+    const bool from_prev = q_prev != nullptr || carry_in != nullptr;
+    if (from_prev) {  // continued filtering: the belief of the step before the window
       for (int idx = tid; idx < Sp; idx += NT) {
         int f = 0;
         while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
         const int s = idx - md.offp[f];
-        cur[idx] = s < md.n[f] ? (R)q_prev[(size_t)a * S + md.off[f] + s] : (R)0;
+        const size_t src = (size_t)a * S + md.off[f] + s;
+        cur[idx] = s < md.n[f] ? (carry_in ? ((const R *)carry_in)[src] : (R)q_prev[src]) : (R)0;
       }
       __syncthreads();
     }
@@ -267,7 +269,7 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
         const int s = idx - md.offp[f], n = md.n[f];
         R lp = (R)0;
         if (s < n) {
-          if (t == 0 && !q_prev) {
+          if (t == 0 && !from_prev) {
             lp = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
           } else {
             const int ur = t == 0 ? act_prev[(size_t)a * F + f] : act[((size_t)a * (T - 1) + (t - 1)) * F + f];
@@ -294,6 +296,14 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
                         am_a ? am_a + (size_t)t * F : nullptr, xpb, (R)lambda);
         __syncthreads();
         R *tmp = cur; cur = nxt; nxt = tmp;
+      }
+    }
+    if (carry_out) {   // the last step's belief at full precision, for a call that continues this one
+      for (int idx = tid; idx < Sp; idx += NT) {
+        int f = 0;
+        while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+        const int s = idx - md.offp[f];
+        if (s < md.n[f]) ((R *)carry_out)[(size_t)a * S + md.off[f] + s] = cur[idx];
       }
     }
   } else {
@@ -396,8 +406,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if ((size_t)sm.total_bytes > budget) return BI_ERR_UNSUPPORTED;
 
   using KernelT = void (*)(const BiDev *, int, int, const int32_t *, const int32_t *, const float *,
-                           const int32_t *, const float *, const void *, double, int, float *, float *, int32_t *,
-                           GenSmem);
+                           const int32_t *, const void *, void *, const float *, const void *, double, int, float *,
+                           float *, int32_t *, GenSmem);
   KernelT kern = nullptr;
   const char *name = "";
   const bool f64 = sizeof(R) == 8;
@@ -417,8 +427,8 @@ int launch_generic_t(const BiCall &c, bi_model *mut) {
   if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes) !=
       cudaSuccess)
     return BI_ERR_CUDA;
-  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.q_init,
-                                               c.lnprior, c.lambda, c.K, c.q_out, c.logq_out, c.argmax_out, sm);
+  kern<<<c.N, NT, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev, c.act_prev, c.carry_in,
+                                               c.carry_out, c.q_init, c.lnprior, c.lambda, c.K, c.q_out, c.logq_out, c.argmax_out, sm);
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += 1;
   mut->last_kernel = name;

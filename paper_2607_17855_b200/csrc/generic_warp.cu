@@ -249,8 +249,8 @@ template <typename R>
 __global__ void __launch_bounds__(512)
 bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
                       const int32_t *__restrict__ act, const float *q_prev, const int32_t *__restrict__ act_prev,
-                      double lambda, int K, float *q_out, float *__restrict__ logq_out,
-                      int32_t *__restrict__ argmax_out, WarpSmem sm) {
+                      const void *carry_in, void *carry_out, double lambda, int K, float *q_out,
+                      float *__restrict__ logq_out, int32_t *__restrict__ argmax_out, WarpSmem sm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   copy_descriptor(mdp, smem_raw);
   const BiDev &md = *reinterpret_cast<const BiDev *>(smem_raw);
@@ -267,12 +267,14 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
   R *xpw = sm.o_xp >= 0 ? wb + sm.o_xp : nullptr;
   for (int i = lane; i < sm.o_sl - sm.o_q0; i += 32) cur[i] = (R)0;  // q0, q1, V0, V1 are adjacent
   __syncwarp();
-  if (q_prev) {  // continued filtering: the belief of the step before the window
+  const bool from_prev = q_prev != nullptr || carry_in != nullptr;
+  if (from_prev) {  // continued filtering: the belief of the step before the window
     for (int idx = lane; idx < Sp; idx += 32) {
       int f = 0;
       while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
       const int s = idx - md.offp[f];
-      if (s < md.n[f]) cur[idx] = (R)q_prev[(size_t)a * S + md.off[f] + s];
+      const size_t src = (size_t)a * S + md.off[f] + s;
+      if (s < md.n[f]) cur[idx] = carry_in ? ((const R *)carry_in)[src] : (R)q_prev[src];
     }
     __syncwarp();
   }
@@ -288,7 +290,7 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
       const int s = idx - md.offp[f], n = md.n[f];
       R lp = (R)0;
       if (s < n) {
-        if (t == 0 && !q_prev) {
+        if (t == 0 && !from_prev) {
           lp = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
         } else {
           const int ur = t == 0 ? act_prev[(size_t)a * F + f] : act[((size_t)a * (T - 1) + (t - 1)) * F + f];
@@ -314,6 +316,15 @@ bi_warp_filter_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
       softmax_warp<R>(md, ell, nxt, k == K - 1, q_a + (size_t)t * S, lq_a ? lq_a + (size_t)t * S : nullptr,
                       am_a ? am_a + (size_t)t * F : nullptr, lane, xpw, (R)lambda);
       R *tmp = cur; cur = nxt; nxt = tmp;
+    }
+  }
+  if (carry_out) {   // the last step's belief at full precision, for a call that continues this one
+    __syncwarp();
+    for (int idx = lane; idx < Sp; idx += 32) {
+      int f = 0;
+      while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+      const int s = idx - md.offp[f];
+      if (s < md.n[f]) ((R *)carry_out)[(size_t)a * S + md.off[f] + s] = cur[idx];
     }
   }
 }
@@ -474,8 +485,8 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
     e = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm.total_bytes);
     if (e != cudaSuccess) return BI_ERR_CUDA;
     kern<<<(c.N + W - 1) / W, W * 32, sm.total_bytes, c.stream>>>(md->d, c.N, c.T, c.obs, c.act, c.q_prev,
-                                                                   c.act_prev, c.lambda, c.K, c.q_out, c.logq_out,
-                                                                   c.argmax_out, sm);
+                                                                   c.act_prev, c.carry_in, c.carry_out, c.lambda, c.K,
+                                                                   c.q_out, c.logq_out, c.argmax_out, sm);
     name = f64 ? "warp_filter_f64" : "warp_filter_f32";
   } else if (c.algo == BI_ALGO_VMP) {
     auto kern = bi_warp_window_kernel<R, BI_ALGO_VMP>;

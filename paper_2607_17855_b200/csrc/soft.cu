@@ -193,6 +193,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
   if (cudaMemcpyAsync(sh.d, &sh.h, sizeof(BiDev), cudaMemcpyHostToDevice, stream) != cudaSuccess) return BI_ERR_CUDA;
 
   BiCall c;
+  c.carry_in = nullptr; c.carry_out = nullptr;
   c.model = &sh; c.algo = algo; c.N = N; c.T = T; c.K = iters;
   c.obs = obs_idx; c.act = act; c.q_prev = nullptr; c.act_prev = nullptr; c.q_init = nullptr; c.lnprior = nullptr; c.lambda = model->damping;
   c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;

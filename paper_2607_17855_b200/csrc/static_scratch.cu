@@ -305,6 +305,7 @@ extern "C" int bi_filter_static(const bi_model_desc *desc, int32_t N, int32_t T,
 
   // ---- the general filtering kernel on the packed copy
   BiCall c;
+  c.carry_in = nullptr; c.carry_out = nullptr;
   c.model = &md; c.algo = BI_ALGO_FILTER; c.N = N; c.T = T; c.K = iters;
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
   c.q_prev = nullptr; c.act_prev = nullptr; c.q_init = nullptr; c.lnprior = nullptr; c.lambda = 1.0;

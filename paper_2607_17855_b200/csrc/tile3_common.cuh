@@ -26,6 +26,8 @@ struct Tile3Params {
   const int32_t *obs, *act;
   const float *q_prev;       // filtering continued from these beliefs [N][S], or NULL
   const int32_t *act_prev;   // [N][F] with q_prev
+  const void *carry_in;      // as BiCall
+  void *carry_out;
   const float *q_init;       // window algorithms: starting beliefs [N][T][S], or NULL
   const void *lnprior;       // window algorithms: [N][S] log-priors used in the place of ln D, or NULL
   int32_t F;
@@ -84,6 +86,6 @@ static inline void bi_tile3_fill_params(const BiCall &c, Tile3Params &p) {
   }
   p.N = c.N; p.T = c.T; p.K = c.K; p.M = h.M; p.S = h.S; p.G = h.G;
   p.obs = c.obs; p.act = c.act; p.q_out = c.q_out; p.logq_out = c.logq_out;
-  p.q_prev = c.q_prev; p.act_prev = c.act_prev; p.q_init = c.q_init; p.lnprior = c.lnprior; p.lambda = c.lambda; p.F = c.model->h.F;
+  p.q_prev = c.q_prev; p.act_prev = c.act_prev; p.carry_in = c.carry_in; p.carry_out = c.carry_out; p.q_init = c.q_init; p.lnprior = c.lnprior; p.lambda = c.lambda; p.F = c.model->h.F;
   p.argmax_out = c.argmax_out; p.status = h.status;
 }

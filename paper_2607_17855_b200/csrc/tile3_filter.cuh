@@ -46,12 +46,19 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
   for (int mi = 0; mi < p.nmem; ++mi) o_next[mi] = __ldg(p.obs + out_base * p.M + p.modality[mi]);
   // Continued filtering: the belief of the step before the window takes the
   // place of "the previous step's final belief", and its action that of u_{t-1}.
-  const bool from_prev = p.q_prev != nullptr;
+  const bool from_prev = p.q_prev != nullptr || p.carry_in != nullptr;
   if (from_prev) {
-    const float *qp = p.q_prev + (size_t)agent * p.S;
-    if (t3.own_a) sq[a] = (R)__ldg(qp + p.off[0] + a);
-    if (t3.own_b) sq[NA + bi] = (R)__ldg(qp + p.off[1] + bi);
-    if (t3.own_c) sq[NA + NB + ci] = (R)__ldg(qp + p.off[2] + ci);
+    if (p.carry_in) {   // the previous call's last belief at full precision
+      const R *qp = (const R *)p.carry_in + (size_t)agent * p.S;
+      if (t3.own_a) sq[a] = qp[p.off[0] + a];
+      if (t3.own_b) sq[NA + bi] = qp[p.off[1] + bi];
+      if (t3.own_c) sq[NA + NB + ci] = qp[p.off[2] + ci];
+    } else {
+      const float *qp = p.q_prev + (size_t)agent * p.S;
+      if (t3.own_a) sq[a] = (R)__ldg(qp + p.off[0] + a);
+      if (t3.own_b) sq[NA + bi] = (R)__ldg(qp + p.off[1] + bi);
+      if (t3.own_c) sq[NA + NB + ci] = (R)__ldg(qp + p.off[2] + ci);
+    }
     const int32_t *ap = p.act_prev + (size_t)agent * p.F;
     u_next[0] = __ldg(ap + p.fac[0]);
     u_next[1] = __ldg(ap + p.fac[1]);
@@ -189,6 +196,12 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_kernel(const Tile3Params p
       if (t3.own_a) qo[p.off[0] + a] = (float)qa;
       if (t3.own_b) qo[p.off[1] + bi] = (float)qb;
       if (t3.own_c) qo[p.off[2] + ci] = (float)qc;
+      if (p.carry_out && t == p.T - 1) {
+        R *co = (R *)p.carry_out + (size_t)agent * p.S;
+        if (t3.own_a) co[p.off[0] + a] = qa;
+        if (t3.own_b) co[p.off[1] + bi] = qb;
+        if (t3.own_c) co[p.off[2] + ci] = qc;
+      }
       if (p.logq_out) {
         float *lo = p.logq_out + (out_base + t) * p.S;
         if (t3.own_a) lo[p.off[0] + a] = (float)(xa - (R)ma - bi_log(za));

@@ -270,13 +270,20 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_f64_kernel(const Tile3Para
   __syncwarp();
 
   const size_t out_base = (size_t)agent * p.T;
-  const bool from_prev = p.q_prev != nullptr;
+  const bool from_prev = p.q_prev != nullptr || p.carry_in != nullptr;
   int u_next[3] = {0, 0, 0};
   if (from_prev) {
-    const float *qp = p.q_prev + (size_t)agent * p.S;
-    if (a_ok) sq[a] = (R)__ldg(qp + p.off[0] + a);
-    if (b_ok) sq[NA + bi] = (R)__ldg(qp + p.off[1] + bi);
-    if (c_ok) sq[NA + NB + ci] = (R)__ldg(qp + p.off[2] + ci);
+    if (p.carry_in) {   // the previous call's last belief at full precision
+      const R *qp = (const R *)p.carry_in + (size_t)agent * p.S;
+      if (a_ok) sq[a] = qp[p.off[0] + a];
+      if (b_ok) sq[NA + bi] = qp[p.off[1] + bi];
+      if (c_ok) sq[NA + NB + ci] = qp[p.off[2] + ci];
+    } else {
+      const float *qp = p.q_prev + (size_t)agent * p.S;
+      if (a_ok) sq[a] = (R)__ldg(qp + p.off[0] + a);
+      if (b_ok) sq[NA + bi] = (R)__ldg(qp + p.off[1] + bi);
+      if (c_ok) sq[NA + NB + ci] = (R)__ldg(qp + p.off[2] + ci);
+    }
     const int32_t *ap = p.act_prev + (size_t)agent * p.F;
     u_next[0] = __ldg(ap + p.fac[0]);
     u_next[1] = __ldg(ap + p.fac[1]);
@@ -390,6 +397,12 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_f64_kernel(const Tile3Para
       if (a_ok) qo[p.off[0] + a] = (float)qa;
       if (b_ok) qo[p.off[1] + bi] = (float)qb;
       if (c_ok) qo[p.off[2] + ci] = (float)qc;
+      if (p.carry_out && t == p.T - 1) {
+        R *co = (R *)p.carry_out + (size_t)agent * p.S;
+        if (a_ok) co[p.off[0] + a] = qa;
+        if (b_ok) co[p.off[1] + bi] = qb;
+        if (c_ok) co[p.off[2] + ci] = qc;
+      }
       if (p.logq_out) {
         const R LN2 = 0.69314718055994530942;
         float *lo = p.logq_out + (out_base + t) * p.S;

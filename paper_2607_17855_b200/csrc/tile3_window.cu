@@ -450,9 +450,7 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   if (bsz * sizeof(R) > 48 * 1024) return BI_ERR_UNSUPPORTED;
   // Fewest CTAs per agent whose share of the window fits; a larger cluster is
   // preferred when it lets several CTAs share an SM (more warps in flight to
-  // hide the per-iteration barrier).  BI_WINDOW_CS (testing aid) forces a size.
-  int cs_force = 0;
-  if (const char *e = getenv("BI_WINDOW_CS")) cs_force = atoi(e);
+  // hide the per-iteration barrier).
   const bool stale = sizeof(R) == 8 && p.nmem <= 12;
   // (a damped call is a separate instantiation, so that the plain update carries none of it)
   auto pick = [&](bool cl) -> const void * {
@@ -465,7 +463,6 @@ int launch_window(const Tile3Params &p, int smem_budget, cudaStream_t stream) {
   int best_cs = 0;
   double best_score = -1.0;
   for (int cs = 1; cs <= 8; cs *= 2) {
-    if (cs_force > 0 && cs != cs_force) continue;
     const int Tc = (p.T + cs - 1) / cs;
     if (cs > 1 && Tc * (cs - 1) >= p.T) continue;  // an empty CTA: no gain over the smaller cluster
     const int warps = (Tc + UPW - 1) / UPW;

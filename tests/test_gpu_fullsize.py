@@ -17,6 +17,41 @@ def test_config2_full_size_every_agent():
     assert res["kernel"] == "tile3_filter_f64"
 
 
+def test_config2_full_size_in_blocks_of_steps_every_agent():
+    # the end-to-end run of bench.py: five consecutive blocks of ten steps (bi_filter, then
+    # bi_filter_continue four times), compared with the oracle on all 4096 agents
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    from parity import compare
+    w = make_config(2)
+    md = bi.model_from_workload(w)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    lq = torch.empty((w.N, w.T, w.S), device="cuda")
+    am = torch.empty((w.N, w.T, w.F), dtype=torch.int32, device="cuda")
+    q = torch.empty((w.N, w.T, w.S), device="cuda")
+    nb = 5
+    tc = w.T // nb
+    for i in range(nb):
+        t0 = i * tc
+        o = obs[:, t0:t0 + tc].contiguous()
+        a = act[:, t0:t0 + tc - 1].contiguous()
+        outs = [torch.empty((w.N, tc, d), dtype=dt, device="cuda") for d, dt in
+                ((w.S, torch.float32), (w.S, torch.float32), (w.F, torch.int32))]
+        if i == 0:
+            md.bi_filter(o, a, w.K, q_out=outs[0], logq_out=outs[1], argmax_out=outs[2])
+        else:
+            md.bi_filter_continue(o, a, act[:, t0 - 1].contiguous(), w.K, q_out=outs[0], logq_out=outs[1],
+                                  argmax_out=outs[2])
+        q[:, t0:t0 + tc], lq[:, t0:t0 + tc], am[:, t0:t0 + tc] = outs
+    torch.cuda.synchronize()
+    assert md.last_kernel == "tile3_filter_f64" and md.status() == 0
+    whole = md.bi_filter(obs, act, w.K).cpu().numpy()
+    assert np.array_equal(q.cpu().numpy(), whole)
+    print(compare(w, q.cpu().numpy(), lq.cpu().numpy(), am.cpu().numpy(), *oracle.run_workload(w)))
+    md.close()
+
+
 def test_config3_full_size_sampled_agents():
     w = make_config(3)
     rng = np.random.default_rng(3)

@@ -15,18 +15,23 @@ ALGOS = ["filter", "vmp", "mmp"]
 
 
 @contextlib.contextmanager
-def warp_filter_forced():
-    """Small filtering batches go to the CTA-per-agent kernel; the library's testing aid BI_CTA_MAXN=0
-    sends them to the warp-per-agent kernel instead, so that it can be checked on oracle-sized inputs."""
-    old = os.environ.get("BI_CTA_MAXN")
-    os.environ["BI_CTA_MAXN"] = "0"
+def family_forced(name):
+    """The library's testing aid BI_TEST_FAMILY ("warp" or "generic"), read when a handle is made: its
+    calls skip the kernel families ahead of the named one, so that the general kernels can be checked
+    on oracle-sized inputs that would otherwise go to a specialised kernel."""
+    old = os.environ.get("BI_TEST_FAMILY")
+    os.environ["BI_TEST_FAMILY"] = name
     try:
         yield
     finally:
         if old is None:
-            del os.environ["BI_CTA_MAXN"]
+            del os.environ["BI_TEST_FAMILY"]
         else:
-            os.environ["BI_CTA_MAXN"] = old
+            os.environ["BI_TEST_FAMILY"] = old
+
+
+def warp_filter_forced():
+    return family_forced("warp")
 
 
 def _custom(seed, n, m, dep, U, N, T, K, G=1, sparsity=0.0):
@@ -505,12 +510,12 @@ def test_damped_updates(case, algo):
         "per_agent": _custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=6, G=5),
     }[case]
     lam = 0.45
-    md = bi.model_from_workload(w)
+    with (warp_filter_forced() if case == "warp" else contextlib.nullcontext()):
+        md = bi.model_from_workload(w)     # (the testing aid is read when the handle is made)
     md.set_damping(lam)
     obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
     lq = torch.empty((w.N, w.T, w.S), dtype=torch.float32, device="cuda")
-    with (warp_filter_forced() if case == "warp" else contextlib.nullcontext()):
-        q = md.run(algo, obs, act, w.K, logq_out=lq).cpu().numpy()
+    q = md.run(algo, obs, act, w.K, logq_out=lq).cpu().numpy()
     kernel = md.last_kernel
     if algo == "filter" and case in ("warp", "cta"):
         assert kernel == f"{case}_filter_f64", kernel
@@ -583,9 +588,16 @@ def test_filter_kernels_across_batch_sizes(arith):
     ref = oracle.run_workload(w.take_agents(sel), "filter")[0]
     for n, kern in ((40, "cta_filter"), (400, "cta_filter"), (1400, "cta_filter"), (1400, "warp_filter")):
         sub = w.take_agents(list(range(n)))
-        with (warp_filter_forced() if kern == "warp_filter" else contextlib.nullcontext()):
+        if kern == "warp_filter":   # (the testing aid is read when a handle is made: a handle of its own)
+            with warp_filter_forced():
+                mdw = bi.model_from_workload(w, arith=arith)
+            q, _, _, _ = run_gpu(sub, "filter", model=mdw, arith=arith)
+            name = mdw.last_kernel
+            mdw.close()
+        else:
             q, _, _, _ = run_gpu(sub, "filter", model=md, arith=arith)
-        assert md.last_kernel == f"{kern}_{arith}", (n, md.last_kernel)
+            name = md.last_kernel
+        assert name == f"{kern}_{arith}", (n, name)
         pick = [i for i in sel if i < n]
         err = np.abs(q[pick] - ref[:len(pick)]).max()
         assert err <= (1e-5 if arith == "f64" else 5e-3), (n, err)
@@ -626,12 +638,6 @@ def test_filter_kernels_on_random_structures_with_ragged_sizes(j):
     assert res["kernel"] == "warp_filter_f64", res
 
 
-def test_fma_probe_reports_a_plausible_rate():
-    import paper_2607_17855_b200 as bi
-    f64, f32 = bi.bi_probe_fma("f64"), bi.bi_probe_fma("f32")
-    assert 1.0 < f64 < 200.0 and f64 < f32 < 400.0, (f64, f32)
-
-
 def test_golden_mmp_backward_message_on_the_gpu(golden_dir):
     """The hand-worked two-step window whose backward message varies over states (unequal row sums of
     the transition matrix), one iteration from the fixture's start, through bi_mmp_warm / bi_vmp_warm."""
@@ -664,3 +670,85 @@ def test_golden_mmp_backward_message_on_the_gpu(golden_dir):
     np.testing.assert_allclose(q[0, 0], want / want.sum(), atol=3e-7)
     md.close()
     md2.close()
+
+
+def _blockwise(md, w, cuts, K):
+    """bi_filter on the first block of steps, bi_filter_continue on the rest; returns q [N, T, S]."""
+    import torch
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    parts, names = [], set()
+    for i, (t0, t1) in enumerate(zip(cuts[:-1], cuts[1:])):
+        o = obs[:, t0:t1].contiguous()
+        a = act[:, t0:t1 - 1].contiguous() if t1 - t0 > 1 else None
+        if i == 0:
+            parts.append(md.bi_filter(o, a, K))
+        else:
+            parts.append(md.bi_filter_continue(o, a, act[:, t0 - 1].contiguous(), K))
+        names.add(md.last_kernel)
+    torch.cuda.synchronize()
+    return torch.cat(parts, dim=1).cpu().numpy(), names
+
+
+@pytest.mark.parametrize("case", ["tile_f64", "tile_sb2", "cta", "warp", "tile_f32"])
+def test_filter_continue_equals_the_single_call_bit_for_bit(case):
+    """A trajectory filtered in consecutive blocks through the handle's full-precision record equals
+    the single call exactly, on every filtering kernel family."""
+    import torch
+    import paper_2607_17855_b200 as bi
+    arith = "f32" if case == "tile_f32" else "f64"
+    if case in ("tile_f64", "tile_f32"):
+        w = make_config(2, N=37, T=12)
+    elif case == "tile_sb2":
+        w = make_config(4, N=9, T=9)
+    else:
+        w = make_sweep_config(42, N=13, T=11)
+    ctx = warp_filter_forced() if case == "warp" else contextlib.nullcontext()
+    with ctx:
+        md = bi.model_from_workload(w, arith=arith)
+        obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+        whole = md.bi_filter(obs, act, w.K).cpu().numpy()
+        kernel = md.last_kernel
+        for cuts in ([0, 1, w.T], [0, 4, 5, w.T - 2, w.T], [0, w.T - 1, w.T]):
+            q, names = _blockwise(md, w, cuts, w.K)
+            assert names == {kernel}
+            assert np.array_equal(q, whole), (case, cuts, np.abs(q - whole).max())
+    expect = {"tile_f64": "tile3_filter_f64", "tile_f32": "tile3_filter_f32", "tile_sb2": "tile3_filter_f64",
+              "cta": "cta_filter_f64", "warp": "warp_filter_f64"}[case]
+    assert kernel == expect
+    assert md.status() == 0
+    md.close()
+
+
+def test_filter_continue_needs_a_matching_previous_call():
+    import torch
+    import paper_2607_17855_b200 as bi
+    w = make_config(1)
+    md = bi.model_from_workload(w)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    ap = act[:, 0].contiguous()
+    with pytest.raises(bi.BiError) as e:
+        md.bi_filter_continue(obs[:, 1:].contiguous(), act[:, 1:].contiguous(), ap, 2)   # nothing to continue
+    assert e.value.code == -1
+    md.bi_filter(obs[:, :1].contiguous(), None, 2)
+    with pytest.raises(bi.BiError) as e:
+        md.bi_filter_continue(obs[:4, 1:].contiguous(), act[:4, 1:].contiguous(), ap[:4].contiguous(), 2)   # other N
+    assert e.value.code == -1
+    md.bi_filter_continue(obs[:, 1:].contiguous(), act[:, 1:].contiguous(), ap, 2)
+    # a window call in between leaves the record alone
+    md.bi_vmp(obs, act, 2)
+    md.bi_filter_continue(obs[:, 1:].contiguous(), act[:, 1:].contiguous(), ap, 2)
+    assert md.status() == 0
+    md.close()
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("case", ["config1", "sweep", "per_agent"])
+def test_general_cta_kernel_when_forced(case, algo):
+    """The first, fully general kernel family (one CTA per agent, every shape and algorithm): the
+    fallback behind the others, forced here so that it is checked against the oracle too."""
+    w = {"config1": lambda: make_config(1), "sweep": lambda: make_sweep_config(19, N=6, T=6),
+         "per_agent": lambda: make_config(4, N=5, T=5)}[case]()
+    with family_forced("generic"):
+        res = check_workload(w, algo)
+    print(res)
+    assert res["kernel"].startswith("generic_"), res["kernel"]
