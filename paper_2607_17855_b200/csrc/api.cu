@@ -235,7 +235,8 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
   if (!md) return BI_ERR_ALLOC;
   memset(md, 0, sizeof(*md));
   md->damping = 1.0;
-  if (const char *e = getenv("BI_TEST_FAMILY")) {   // testing aid, read here and nowhere else
+  if (const char *e = getenv("BI_TEST_DROP_COPY")) md->test_drop_copy = atoi(e) > 0 ? atoi(e) : 0;   // testing aids,
+  if (const char *e = getenv("BI_TEST_FAMILY")) {                                                  // read here only
     md->test_family = !strcmp(e, "warp") ? BI_FAMILY_WARP : !strcmp(e, "generic") ? BI_FAMILY_GENERIC : BI_FAMILY_ANY;
   }
   md->last_kernel = "";

@@ -68,6 +68,7 @@ struct BatchParams {
   uint32_t *status;        // the handle's status word
   const int32_t *obs;      // [NU][M] (per-agent models: every unit reads its own slice)
   int32_t M, T;
+  int32_t drop_copy;       // testing aid: the contraction announces its slice copy and does not issue it
 };
 
 // ---- one unit against one slice: every message of the group in one pass ----
@@ -254,8 +255,10 @@ bi_batch_contract_kernel(BatchParams P, int cur, int first) {
   __shared__ __align__(8) unsigned long long bar;
   if (threadIdx.x == 0) bi_mbar_init(&bar, 1);
   __syncthreads();
-  if (threadIdx.x == 0)
-    bi_bulk_load(L, (const R *)mm.logA + (size_t)tk.x * mm.P_pad, (uint32_t)(mm.P_pad * sizeof(R)), &bar);
+  if (threadIdx.x == 0) {
+    if (P.drop_copy) bi_mbar_expect(&bar, (uint32_t)(mm.P_pad * sizeof(R)));   // (testing aid: the copy never comes)
+    else bi_bulk_load(L, (const R *)mm.logA + (size_t)tk.x * mm.P_pad, (uint32_t)(mm.P_pad * sizeof(R)), &bar);
+  }
   const bool has_unit = (int)threadIdx.x < tk.z;
   const int unit = has_unit ? P.perm[(size_t)mi * P.NU + tk.y + threadIdx.x] : 0;
   const R *q = (const R *)P.qbuf + ((size_t)cur * P.NU + unit) * P.Sp;
@@ -264,7 +267,9 @@ bi_batch_contract_kernel(BatchParams P, int cur, int first) {
     bi_grid_wait();
     bi_grid_launch_dependents();
   }
-  if (!bi_mbar_wait(&bar, 0)) {
+  // a copy that does not arrive within the probe limit: the block reports it and leaves (nothing of
+  // its own is in flight then; the call's outputs are invalid)
+  if (!bi_mbar_wait(&bar, 0, P.drop_copy ? 256 : 1 << 18)) {
     if (threadIdx.x == 0) atomicOr(P.status, BI_FLAG_COPY_TIMEOUT);
     return;
   }
@@ -735,6 +740,11 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   P.ellp = w + b_perm + b_task;
   P.qbuf = w + b_perm + b_task + b_ellp;
   P.status = h.status;
+  P.drop_copy = 0;
+  if (mut->test_drop_copy > 0) {   // testing aid: this many calls lose their copies
+    P.drop_copy = 1;
+    mut->test_drop_copy -= 1;
+  }
   P.obs = c.obs; P.M = h.M; P.T = c.T;
   A.obs = c.obs; A.act = c.act; A.q_out = c.q_out; A.logq_out = c.logq_out; A.argmax_out = c.argmax_out;
   A.T = c.T;

@@ -185,6 +185,13 @@ __device__ __forceinline__ void bi_bulk_load(void *dst_smem, const void *src_glo
                : "memory");
 }
 
+// the announcement alone: `bytes` expected on the barrier, and this thread's arrival (a testing aid uses
+// it without the copy, to make the bounded wait below run out)
+__device__ __forceinline__ void bi_mbar_expect(unsigned long long *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bi_smem_addr(bar)), "r"(bytes)
+               : "memory");
+}
+
 // Waits for the barrier's phase of the given parity with a bounded number of
 // probes; false when the limit ran out (the caller raises a status flag and
 // leaves: nothing here spins without an end).

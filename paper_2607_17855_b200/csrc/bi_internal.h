@@ -118,6 +118,10 @@ struct bi_model {
   // "generic"): calls skip the kernel families ahead of the named one, so that the general kernels can
   // be checked on inputs small enough for the oracle.  0 = normal dispatch.
   int test_family;
+  // Testing aid (BI_TEST_DROP_COPY = n, read when the handle is made): the next n batched window calls
+  // announce their slice copies without issuing them, so that the bounded wait on the copy runs out and
+  // the status flag BI_FLAG_COPY_TIMEOUT is raised; nothing faults, nothing is left in flight.
+  int test_drop_copy;
 };
 
 struct BiCall {

@@ -752,3 +752,35 @@ def test_general_cta_kernel_when_forced(case, algo):
         res = check_workload(w, algo)
     print(res)
     assert res["kernel"].startswith("generic_"), res["kernel"]
+
+
+def test_a_copy_that_never_arrives_is_reported_not_waited_for():
+    """The bounded wait on a block's own bulk copy.  The testing aid BI_TEST_DROP_COPY=1 (read when the
+    handle is made) makes the next batched window call announce its slice copies on their barriers
+    without issuing them; every contraction block must give up after its probe limit, raise
+    BI_FLAG_COPY_TIMEOUT and leave -- nothing is in flight, nothing faults, the context stays usable --
+    and the next call on the same handle is an ordinary, correct one."""
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = make_config(3, N=128, T=16, K=4)
+    old = os.environ.get("BI_TEST_DROP_COPY")
+    os.environ["BI_TEST_DROP_COPY"] = "1"
+    try:
+        md = bi.model_from_workload(w)
+    finally:
+        if old is None:
+            del os.environ["BI_TEST_DROP_COPY"]
+        else:
+            os.environ["BI_TEST_DROP_COPY"] = old
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    md.bi_vmp(obs, act, w.K)
+    assert md.last_kernel == "batch_vmp_f64"
+    flags = md.status()                 # synchronises; returns and clears the flags
+    assert flags & 4, flags             # BI_FLAG_COPY_TIMEOUT
+    q = md.bi_vmp(obs, act, w.K).cpu().numpy()
+    assert md.status() == 0
+    sel = list(range(0, w.N, 16))
+    ref = oracle.run_workload(w.take_agents(sel), "vmp")[0]
+    assert np.abs(q[sel] - ref).max() <= 1e-5
+    md.close()
