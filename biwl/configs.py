@@ -50,6 +50,7 @@ class Workload:
     obs: np.ndarray
     act: np.ndarray
     meta: dict = field(default_factory=dict)
+    bdep: Optional[List[List[int]]] = None  # B-dependencies (None: every factor depends on itself only)
 
     @property
     def F(self) -> int:
@@ -85,7 +86,7 @@ class Workload:
             name=self.name, algo=self.algo, n=self.n, m=self.m, dep=self.dep,
             U=self.U, G=G, A=A, B=B, D=D, N=len(idx), T=self.T, K=self.K,
             obs=np.ascontiguousarray(self.obs[idx]),
-            act=np.ascontiguousarray(self.act[idx]), meta=dict(self.meta))
+            act=np.ascontiguousarray(self.act[idx]), meta=dict(self.meta), bdep=self.bdep)
 
 
 # --------------------------------------------------------------------------
@@ -120,8 +121,10 @@ def _sparsify(rng: np.random.Generator, a: np.ndarray, frac: float, axis: int) -
 def make_model(rng: np.random.Generator, n, m, dep, U, G: int, *,
                a_alpha: float = 1.0, sparsity: float = 0.0,
                b_alpha: float = 1.0, b_diag: float = 0.0,
-               d_alpha: Optional[float] = None, chunk: int = 128):
-    """Draw A, B, D for the given structure.  ``d_alpha=None`` gives uniform D."""
+               d_alpha: Optional[float] = None, chunk: int = 128, bdep=None, b_sparsity: float = 0.0):
+    """Draw A, B, D for the given structure.  ``d_alpha=None`` gives uniform D.
+    ``bdep`` (per factor, the factors its transition depends on; None = its own previous state)
+    gives ``B[f]`` of shape ``[G, n_f, n_bdep..., U_f]``."""
     n = np.asarray(n, dtype=np.int32)
     m = np.asarray(m, dtype=np.int32)
     U = np.asarray(U, dtype=np.int32)
@@ -138,6 +141,12 @@ def make_model(rng: np.random.Generator, n, m, dep, U, G: int, *,
     B = []
     for f in range(len(n)):
         nf, uf = int(n[f]), int(U[f])
+        if bdep is not None:
+            par = tuple(int(n[g]) for g in bdep[f])
+            b = _dirichlet_axis(rng, (G, nf) + par + (uf,), b_alpha, axis=1)
+            b = _sparsify(rng, b, b_sparsity, axis=1)
+            B.append(b.astype(np.float32))
+            continue
         b = _dirichlet_axis(rng, (G, nf, nf, uf), b_alpha, axis=1)
         if b_diag > 0.0:
             b = b + b_diag * np.eye(nf)[None, :, :, None]
@@ -166,7 +175,7 @@ def _categorical(rng: np.random.Generator, p: np.ndarray) -> np.ndarray:
     return np.minimum(idx, p.shape[1] - 1).astype(np.int32)
 
 
-def sample_streams(rng: np.random.Generator, n, m, dep, U, G, A, B, D, N: int, T: int):
+def sample_streams(rng: np.random.Generator, n, m, dep, U, G, A, B, D, N: int, T: int, bdep=None):
     """Sample per-agent observation and action index streams from the model."""
     F, M = len(n), len(m)
     gi = np.zeros(N, dtype=np.int64) if G == 1 else np.arange(N, dtype=np.int64)
@@ -183,10 +192,14 @@ def sample_streams(rng: np.random.Generator, n, m, dep, U, G, A, B, D, N: int, T
             # advanced indices separated by a slice put the broadcast axis first
             obs[:, t, i] = _categorical(rng, p)
         if t + 1 < T:
+            s_prev = s.copy()   # every factor's transition reads the states of step t
             for f in range(F):
                 u = rng.integers(0, int(U[f]), size=N).astype(np.int32)
                 act[:, t, f] = u
-                p = B[f][gi, :, s[:, f], u]
+                if bdep is None:
+                    p = B[f][gi, :, s_prev[:, f], u]
+                else:
+                    p = B[f][(gi, slice(None)) + tuple(s_prev[:, g] for g in bdep[f]) + (u,)]
                 s[:, f] = _categorical(rng, p)
     return obs, act
 

@@ -59,7 +59,7 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
         A, B, D, obs: np.ndarray, act: Optional[np.ndarray], K: int, *,
         q_init: Optional[np.ndarray] = None, threads: int = 0, round32: bool = False,
         q_prev: Optional[np.ndarray] = None, act_prev: Optional[np.ndarray] = None,
-        obs_soft: Optional[np.ndarray] = None, damping: float = 1.0):
+        obs_soft: Optional[np.ndarray] = None, damping: float = 1.0, bdep=None):
     """Run ``algo`` ('filter' | 'vmp' | 'mmp') and return ``(q, logq, argmax)``.
 
     ``obs`` is ``[N, T, M]`` int32, ``act`` ``[N, T-1, F]`` int32 (ignored when
@@ -70,6 +70,8 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
     replaces ``obs`` (pass ``obs=None``): every observation is a categorical
     vector per modality and the log-likelihood is ``log(A_i) . o^i``.
     ``damping`` in (0, 1]: step size of the update on log-beliefs (1 = plain).
+    ``bdep`` (a list of factor lists, or None): B-dependencies -- factor f's transition depends on the
+    previous states of ``bdep[f]`` and ``B[f]`` is ``[G, n_f, n_bdep..., U_f]``; filtering and VMP only.
     """
     if (q_prev is None) != (act_prev is None):
         raise ValueError("q_prev and act_prev go together")
@@ -102,7 +104,8 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
     for i, a in enumerate(A):
         assert a.shape == (G, int(m[i])) + tuple(int(n[f]) for f in dep[i]), (i, a.shape)
     for f in range(F):
-        assert B[f].shape == (G, int(n[f]), int(n[f]), int(U[f])), (f, B[f].shape)
+        par = tuple(int(n[g]) for g in bdep[f]) if bdep is not None else (int(n[f]),)
+        assert B[f].shape == (G, int(n[f])) + par + (int(U[f]),), (f, B[f].shape)
         assert D[f].shape == (G, int(n[f]))
     q = np.empty((N, T, S), dtype=np.float64)
     lq = np.empty((N, T, S), dtype=np.float64)
@@ -111,6 +114,29 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
         q_init = np.ascontiguousarray(q_init, dtype=np.float64)
         assert q_init.shape == (N, T, S)
     Ap, Bp, Dp = _ptr_array(A), _ptr_array(B), _ptr_array(D)
+    if bdep is not None:
+        assert obs_soft is None and damping == 1.0 and not round32
+        bl = np.ascontiguousarray([len(d) for d in bdep], dtype=np.int32)
+        bf = np.ascontiguousarray([g for d in bdep for g in d], dtype=np.int32)
+        if q_prev is not None:
+            q_prev = np.ascontiguousarray(q_prev, dtype=np.float64)
+            act_prev = np.ascontiguousarray(act_prev, dtype=np.int32)
+            assert q_prev.shape == (N, S) and act_prev.shape == (N, F)
+        rc = lib.bi_ref_run_bdep(
+            ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),
+            ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),
+            ctypes.c_void_p(dep_len.ctypes.data), ctypes.c_void_p(dep_flat.ctypes.data),
+            ctypes.c_void_p(U.ctypes.data), ctypes.c_int(G), Ap, Bp, Dp,
+            ctypes.c_void_p(bl.ctypes.data), ctypes.c_void_p(bf.ctypes.data),
+            ctypes.c_int(N), ctypes.c_int(T), ctypes.c_void_p(obs.ctypes.data), ctypes.c_void_p(act_p),
+            ctypes.c_int(K), ctypes.c_void_p(q_init.ctypes.data if q_init is not None else None),
+            ctypes.c_void_p(q_prev.ctypes.data if q_prev is not None else None),
+            ctypes.c_void_p(act_prev.ctypes.data if act_prev is not None else None),
+            ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(lq.ctypes.data),
+            ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads))
+        if rc != 0:
+            raise ValueError(f"bi_ref_run_bdep rejected its arguments (code {rc})")
+        return q, lq, am
     if damping != 1.0:
         if q_prev is not None:
             q_prev = np.ascontiguousarray(q_prev, dtype=np.float64)
@@ -201,4 +227,6 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
 
 def run_workload(w, algo: Optional[str] = None, **kw):
     """Convenience: run on an object with the workload generator's field names."""
+    if getattr(w, "bdep", None) is not None:
+        kw.setdefault("bdep", w.bdep)
     return run(algo or w.algo, w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, w.obs, w.act, w.K, **kw)

@@ -45,9 +45,21 @@
  * under a uniform prior, D at full weight) is the one the paper's authors ran:
  * Section IV names the algorithm and prints no equation.
  *
+ * Non-trivial B-dependencies (the extension Section VI leaves as future work; Section III-B restricts
+ * itself to the trivial case): factor f's transition may depend on the previous states of a list
+ * bdep(f) of factors, p(s^f_{t+1} | s^{bdep(f)}_t, u^f_t) = B_f[s', s_bdep..., u].  The same mean-field
+ * update (Section III-A) then gives
+ *   - filtering: prior_t,f[s'] = sum_{s_par} B_f[s', s_par, u] prod_{g in bdep(f)} q_{t-1,g}[s_g];
+ *   - VMP past message to (t, f): sum_{s_par} ln B_f[s', s_par, u_{t-1}] prod_g q_{t-1,g}[s_g];
+ *     future message to (t, g): sum over the factors h with g in bdep(h) of
+ *       sum_{s'} q_{t+1,h}[s'] sum_{s_par \ g} ln B_h[s', s_par, u_t] prod_{j in bdep(h), j != g} q_{t,j}[s_j];
+ *   - MMP is not defined for them here (its reversed transition has no counterpart with several
+ *     parents): such a call is rejected.
+ *
  * Layouts (row-major):
  *   A[i]: [G][m_i][n_{dep(i)[0]}]...[n_{dep(i)[k-1]}]   float32
  *   B[f]: [G][n_f next][n_f prev][U_f]                   float32
+ *         (with B-dependencies: [G][n_f next][n_{bdep(f)[0]}]...[n_{bdep(f)[k-1]}][U_f])
  *   D[f]: [G][n_f]                                       float32
  *   obs:  [N][T][M] int32     act: [N][T-1][F] int32
  *   q, logq: [N][T][S] float64 (factor f at offset sum_{g<f} n_g)
@@ -79,6 +91,10 @@ typedef struct {
     int Mtot;      /* sum of m_i */
     int round32;   /* conditioning probe: round logs and beliefs to float32 */
     double lambda; /* damping of the log-belief update: 1 = the plain fixed-point map */
+    /* B-dependencies: NULL = trivial (every factor depends on its own previous state) */
+    const int32_t *bdep_len, *bdep;
+    int *bdep_off;  /* [F] offset of factor f's list in bdep */
+    int64_t *PB;    /* [F] product of the sizes of the factors in bdep(f) */
 } model_t;
 
 static double log_eps(double x, int round32)
@@ -92,6 +108,66 @@ static double B_at(const model_t *md, int g, int f, int u, int s_next, int s_pre
 {
     int nf = md->n[f], Uf = md->U[f];
     return (double)md->B[f][(((size_t)g * nf + s_next) * nf + s_prev) * Uf + u];
+}
+
+/* B_f[s_next, parents, u] of model g with B-dependencies; par is the row-major index of the parents'
+ * states in bdep(f) order */
+static double B_par(const model_t *md, int g, int f, int u, int s_next, int64_t par)
+{
+    int nf = md->n[f], Uf = md->U[f];
+    return (double)md->B[f][((((size_t)g * nf + s_next) * (size_t)md->PB[f]) + (size_t)par) * Uf + u];
+}
+
+/* sum_{parents} X(B_f[s_next, parents, u]) prod_{g in bdep(f)} q_g[s_g], X = identity or the clamped log;
+ * q is one step's belief vector [S] */
+static double transition_expectation(const model_t *md, int g, int f, int u, int s_next, const double *q, int take_log)
+{
+    int k = md->bdep_len[f];
+    const int32_t *d = md->bdep + md->bdep_off[f];
+    int idx[BI_REF_MAXK];
+    for (int j = 0; j < k; ++j) idx[j] = 0;
+    double total = 0.0;
+    for (int64_t e = 0; e < md->PB[f]; ++e) {
+        double w = 1.0;
+        for (int j = 0; j < k; ++j) w *= q[md->off[d[j]] + idx[j]];
+        double b = B_par(md, g, f, u, s_next, e);
+        total += (take_log ? log_eps(b, md->round32) : b) * w;
+        for (int j = k - 1; j >= 0; --j) {
+            if (++idx[j] < md->n[d[j]]) break;
+            idx[j] = 0;
+        }
+    }
+    return total;
+}
+
+/* VMP future message to factor f0 at a step, state s: over every factor h whose transition depends on f0,
+ * sum_{s'} qn_h[s'] sum_{parents with s_f0 = s} ln B_h[s', parents, u_h] prod_{other parents} q_j[s_j];
+ * q: this step's beliefs, qn: the next step's, act_t: the actions taken at this step [F] */
+static double future_message_bdep(const model_t *md, int g, int f0, int s, const double *q, const double *qn,
+                                  const int32_t *act_t)
+{
+    double total = 0.0;
+    for (int h = 0; h < md->F; ++h) {
+        int k = md->bdep_len[h], pos = -1;
+        const int32_t *d = md->bdep + md->bdep_off[h];
+        for (int j = 0; j < k; ++j) if (d[j] == f0) pos = j;
+        if (pos < 0) continue;
+        int idx[BI_REF_MAXK];
+        for (int j = 0; j < k; ++j) idx[j] = 0;
+        for (int64_t e = 0; e < md->PB[h]; ++e) {
+            if (idx[pos] == s) {
+                double w = 1.0;
+                for (int j = 0; j < k; ++j) if (j != pos) w *= q[md->off[d[j]] + idx[j]];
+                for (int sn = 0; sn < md->n[h]; ++sn)
+                    total += qn[md->off[h] + sn] * log_eps(B_par(md, g, h, act_t[h], sn, e), md->round32) * w;
+            }
+            for (int j = k - 1; j >= 0; --j) {
+                if (++idx[j] < md->n[d[j]]) break;
+                idx[j] = 0;
+            }
+        }
+    }
+    return total;
 }
 
 /*
@@ -194,7 +270,8 @@ static void filter_agent(const model_t *md, int g, int T, int K, const int32_t *
                     int u = t == 0 ? act_prev[f] : act[(size_t)(t - 1) * F + f];
                     const double *qp = t == 0 ? q_prev + o : q_out + (size_t)(t - 1) * S + o;
                     p = 0.0;
-                    for (int r = 0; r < nf; ++r) p += B_at(md, g, f, u, s, r) * qp[r];
+                    if (md->bdep_len) p = transition_expectation(md, g, f, u, s, qp - o, 0);
+                    else for (int r = 0; r < nf; ++r) p += B_at(md, g, f, u, s, r) * qp[r];
                 }
                 lprior[o + s] = log_eps(p, md->round32);
             }
@@ -249,14 +326,17 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
                     double past, future = 0.0;
                     if (t == 0 && q_prev) {
                         double p = 0.0;
-                        for (int r = 0; r < nf; ++r) p += B_at(md, g, f, act_prev[f], s, r) * q_prev[o + r];
+                        if (md->bdep_len) p = transition_expectation(md, g, f, act_prev[f], s, q_prev, 0);
+                        else for (int r = 0; r < nf; ++r) p += B_at(md, g, f, act_prev[f], s, r) * q_prev[o + r];
                         past = log_eps(p, md->round32);
                     } else if (t == 0) {
                         past = log_eps((double)md->D[f][(size_t)g * nf + s], md->round32);
                     } else {
                         int u = act[(size_t)(t - 1) * F + f];
                         const double *qp = cur + (size_t)(t - 1) * S + o;
-                        if (algo == ALGO_VMP) {
+                        if (algo == ALGO_VMP && md->bdep_len) {
+                            past = transition_expectation(md, g, f, u, s, qp - o, 1);
+                        } else if (algo == ALGO_VMP) {
                             past = 0.0;
                             for (int r = 0; r < nf; ++r)
                                 past += log_eps(B_at(md, g, f, u, s, r), md->round32) * qp[r];
@@ -269,7 +349,9 @@ static void window_agent(const model_t *md, int algo, int g, int T, int K,
                     if (t + 1 < T) {
                         int u = act[(size_t)t * F + f];
                         const double *qn = cur + (size_t)(t + 1) * S + o;
-                        if (algo == ALGO_VMP) {
+                        if (algo == ALGO_VMP && md->bdep_len) {
+                            future = future_message_bdep(md, g, f, s, qt, qn - o, act + (size_t)t * F);
+                        } else if (algo == ALGO_VMP) {
                             for (int r = 0; r < nf; ++r)
                                 future += log_eps(B_at(md, g, f, u, r, s), md->round32) * qn[r];
                         } else {
@@ -310,15 +392,21 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
                     int N, int T, const int32_t *obs, const float *obs_soft, const int32_t *act, int K,
                     const double *q_init, const double *q_prev, const int32_t *act_prev,
                     double *q_out, double *logq_out,
-                    int32_t *argmax_out, int threads, int round32, double lambda)
+                    int32_t *argmax_out, int threads, int round32, double lambda,
+                    const int32_t *bdep_len, const int32_t *bdep)
 {
     if (algo < 0 || algo > 2 || F < 1 || M < 0 || N < 0 || T < 1 || K < 1) return -1;
+    if ((bdep_len != NULL) != (bdep != NULL)) return -1;
+    if (bdep_len && algo == ALGO_MMP) return -1;   /* not defined for several parents */
     if (!(lambda > 0.0 && lambda <= 1.0)) return -1;
     if ((q_prev != NULL) != (act_prev != NULL)) return -1;
     if (!(G == 1 || G == N)) return -1;
     model_t md;
     md.F = F; md.M = M; md.G = G; md.n = n; md.m = m; md.dep_len = dep_len; md.dep = dep;
     md.U = U; md.A = A; md.B = B; md.D = D; md.round32 = round32; md.lambda = lambda;
+    md.bdep_len = bdep_len; md.bdep = bdep;
+    md.bdep_off = malloc(sizeof(int) * F);
+    md.PB = malloc(sizeof(int64_t) * F);
     md.off = malloc(sizeof(int) * F);
     md.dep_off = malloc(sizeof(int) * (M > 0 ? M : 1));
     md.P = malloc(sizeof(int64_t) * (M > 0 ? M : 1));
@@ -340,7 +428,21 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
         md.P[i] = P;
         o += dep_len[i];
     }
-    if (bad) { free(md.off); free(md.dep_off); free(md.P); free(md.moff); return -1; }
+    if (bdep_len) {
+        int bo = 0;
+        for (int f = 0; f < F && !bad; ++f) {
+            md.bdep_off[f] = bo;
+            if (bdep_len[f] < 1 || bdep_len[f] > BI_REF_MAXK) { bad = 1; break; }
+            int64_t P = 1;
+            for (int j = 0; j < bdep_len[f]; ++j) {
+                if (bdep[bo + j] < 0 || bdep[bo + j] >= F) { bad = 1; break; }
+                P *= n[bdep[bo + j]];
+            }
+            md.PB[f] = P;
+            bo += bdep_len[f];
+        }
+    }
+    if (bad) { free(md.off); free(md.dep_off); free(md.P); free(md.moff); free(md.bdep_off); free(md.PB); return -1; }
 #ifdef _OPENMP
     if (threads > 0) omp_set_num_threads(threads);
 #else
@@ -362,7 +464,7 @@ static int run_impl(int algo, int F, int M, const int32_t *n, const int32_t *m,
         else window_agent(&md, algo, g, T, K, ob, so, ac, qi, q_prev ? q_prev + (size_t)a * S : NULL,
                           act_prev ? act_prev + (size_t)a * F : NULL, qo, lo, ao);
     }
-    free(md.off); free(md.dep_off); free(md.P); free(md.moff);
+    free(md.off); free(md.dep_off); free(md.P); free(md.moff); free(md.bdep_off); free(md.PB);
     return 0;
 }
 
@@ -374,7 +476,7 @@ int bi_ref_run(int algo, int F, int M, const int32_t *n, const int32_t *m,
                int32_t *argmax_out, int threads, int round32)
 {
     return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, NULL, NULL,
-                    q_out, logq_out, argmax_out, threads, round32, 1.0);
+                    q_out, logq_out, argmax_out, threads, round32, 1.0, NULL, NULL);
 }
 
 /*
@@ -392,7 +494,7 @@ int bi_ref_run_soft(int algo, int F, int M, const int32_t *n, const int32_t *m,
 {
     if (!obs_soft && M > 0) return -1;
     return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, NULL, obs_soft, act, K, NULL, NULL, NULL,
-                    q_out, logq_out, argmax_out, threads, 0, 1.0);
+                    q_out, logq_out, argmax_out, threads, 0, 1.0, NULL, NULL);
 }
 
 /*
@@ -411,7 +513,7 @@ int bi_ref_filter_from(int F, int M, const int32_t *n, const int32_t *m,
 {
     if (!q_prev || !act_prev) return -1;
     return run_impl(ALGO_FILTER, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, NULL, q_prev,
-                    act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0);
+                    act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0, NULL, NULL);
 }
 
 /*
@@ -428,7 +530,7 @@ int bi_ref_window_from(int algo, int F, int M, const int32_t *n, const int32_t *
 {
     if (!q_prev || !act_prev || (algo != ALGO_VMP && algo != ALGO_MMP)) return -1;
     return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, q_prev,
-                    act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0);
+                    act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0, NULL, NULL);
 }
 
 /*
@@ -445,7 +547,25 @@ int bi_ref_run_opts(int algo, int F, int M, const int32_t *n, const int32_t *m,
                     double *q_out, double *logq_out, int32_t *argmax_out, int threads, int round32)
 {
     return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, obs_soft, act, K, q_init, q_prev,
-                    act_prev, q_out, logq_out, argmax_out, threads, round32, lambda);
+                    act_prev, q_out, logq_out, argmax_out, threads, round32, lambda, NULL, NULL);
+}
+
+/*
+ * Filtering or VMP on a model with B-dependencies: bdep_len [F] and bdep [sum] list, per factor, the
+ * factors whose previous states its transition depends on (B[f] laid out [G][n_f][parents...][U_f]).
+ * Other options as bi_ref_run_opts (no observation vectors, no damping).
+ */
+int bi_ref_run_bdep(int algo, int F, int M, const int32_t *n, const int32_t *m,
+                    const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+                    const float *const *A, const float *const *B, const float *const *D,
+                    const int32_t *bdep_len, const int32_t *bdep,
+                    int N, int T, const int32_t *obs, const int32_t *act, int K,
+                    const double *q_init, const double *q_prev, const int32_t *act_prev,
+                    double *q_out, double *logq_out, int32_t *argmax_out, int threads)
+{
+    if (!bdep_len || !bdep) return -1;
+    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, q_prev,
+                    act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0, bdep_len, bdep);
 }
 
 int bi_ref_max_threads(void)

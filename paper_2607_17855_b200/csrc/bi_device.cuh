@@ -114,6 +114,56 @@ __device__ __forceinline__ void bi_exp_tab_init(float *, int) {}
 //   Developed at SunSoft, a Sun Microsystems, Inc. business.
 //   Permission to use, copy, modify, and distribute this software is freely granted,
 //   provided that this notice is preserved.
+// ---- table-driven exp and log in float64, for kernels whose pace is set by FP64 instructions ----
+// Tables in shared memory, filled by the block (bi_fast_tabs_init, then a block-wide barrier).
+//   exp: x = k ln2/512 + r with k = round(x 512/ln 2), |r| <= ln2/1024; exp(x) = 2^(k >> 9) *
+//        2^((k & 511)/512) * (1 + r + r^2/2 + r^3/6): 7 operations, within 1e-14 relative.  k ln2/512 is
+//        exact inside the fused multiply-add, so one constant serves the reduction (error |x| 1.1e-16).
+//   log: x = 2^k m, m in [1, 2); c_j = 1 + (j + 1/2)/128 for the j-th of 128 mantissa intervals;
+//        ln x = k ln 2 + ln c_j + log1p(r), r = m / c_j - 1, |r| <= 1/256, log1p to the fifth power:
+//        9 operations (25 for the table-free form below), absolute error below 1e-15 for the
+//        probabilities and normalisers it is used on (|k| <= 54).
+constexpr int BI_EXP_TAB = 512, BI_EXP_BITS = 9, BI_LOG_TAB = 128;
+__device__ __forceinline__ void bi_fast_tabs_init(double *exp_tab, double2 *log_tab, int tid, int nthreads) {
+  for (int j = tid; j < BI_EXP_TAB; j += nthreads) exp_tab[j] = exp2((double)j * (1.0 / BI_EXP_TAB));
+  for (int j = tid; j < BI_LOG_TAB; j += nthreads) {
+    const double c = 1.0 + ((double)j + 0.5) * (1.0 / BI_LOG_TAB);
+    log_tab[j] = make_double2(1.0 / c, log(c));
+  }
+}
+__device__ __forceinline__ void bi_fast_tabs_init(float *, float2 *, int, int) {}
+// exact zero below -700 (the true value is below 1e-304)
+__device__ __forceinline__ double bi_exp_fast(double x, const double *__restrict__ tab) {
+  const double KL = 738.6598609351493, LK = 0.0013538030870311431, MAGIC = 6755399441055744.0;
+  const double t = fma(x, KL, MAGIC);
+  const int k = __double2loint(t);
+  const double kd = t - MAGIC;
+  const double r = fma(kd, -LK, x);
+  const double T = tab[k & (BI_EXP_TAB - 1)];
+  const double a = fma(r, 1.0 / 6.0, 0.5);
+  const double r2 = r * r;
+  const double p = fma(r2, a, r);
+  const double res = fma(T, p, T);
+  const double out = __hiloint2double(__double2hiint(res) + ((k >> BI_EXP_BITS) << 20), __double2loint(res));
+  return x < -700.0 ? 0.0 : out;
+}
+__device__ __forceinline__ float bi_exp_fast(float x, const float *) { return expf(x); }
+// x a positive normal double
+__device__ __forceinline__ double bi_log_fast(double x, const double2 *__restrict__ tab) {
+  const int hx = __double2hiint(x);
+  const int k = (hx >> 20) - 1023;
+  const double2 cj = tab[(hx >> 13) & (BI_LOG_TAB - 1)];
+  const double m = __hiloint2double((hx & 0x000fffff) | 0x3ff00000, __double2loint(x));
+  const double r = fma(m, cj.x, -1.0);
+  const double r2 = r * r;
+  const double a = fma(r, 1.0 / 3.0, -0.5);
+  const double b = fma(r, 0.2, -0.25);
+  const double c = fma(r2, b, a);
+  const double p = fma(r2, c, r);
+  return fma((double)k, 0.69314718055994530942, cj.y) + p;
+}
+__device__ __forceinline__ float bi_log_fast(float x, const float2 *) { return logf(x); }
+
 // Branch-free natural log of a positive normal double (the messages take logs
 // of probabilities clamped at 1e-16 and of sums of exponentials: never zero,
 // subnormal, infinite or NaN).  Same motive as bi_exp_inline: the six logs of

@@ -13,6 +13,7 @@
 #include <cooperative_groups.h>
 
 #include <algorithm>
+#include <type_traits>
 #include <cstdlib>
 
 #include "bi_internal.h"
@@ -83,8 +84,11 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   R *seb = Ls + geo.off_se;                  // [units][NB + NCP] gathered e_b, e_c
   R *Bs = Ls + geo.off_B;                    // this agent's transition matrices, every action
 
-  __shared__ R exp_tab[32];   // 2^(j/32) for the table-driven exponential (synchronised with the staging below)
-  bi_exp_tab_init(exp_tab, (int)threadIdx.x);
+  // tables of the fast exponential and logarithm (float64; synchronised with the staging below)
+  using R2 = typename std::conditional<sizeof(R) == 8, double2, float2>::type;
+  __shared__ __align__(16) R exp_tab[sizeof(R) == 8 ? BI_EXP_TAB : 2];
+  __shared__ __align__(16) R2 log_tab[sizeof(R) == 8 ? BI_LOG_TAB : 1];
+  bi_fast_tabs_init(exp_tab, log_tab, (int)threadIdx.x, (int)blockDim.x);
   int rank = 0;
   if (CLUSTER) rank = (int)cg::this_cluster().block_rank();
   const int agent = blockIdx.x / geo.CS;
@@ -297,7 +301,7 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       const R *qp = q_cur - SQ, *qn = q_cur + SQ;
       const bool has_prev = t > 0, has_next = t + 1 < T;
       auto edge = [&](R dot, bool future, R prior) -> R {
-        const R v = ALGO == BI_ALGO_MMP ? (R)0.5 * bi_log_inline(bi_max(dot, (R)BI_EPS)) : dot;
+        const R v = ALGO == BI_ALGO_MMP ? (R)0.5 * bi_log_fast(bi_max(dot, (R)BI_EPS), log_tab) : dot;
         return future ? (has_next ? v : (R)0) : (has_prev ? v : prior);
       };
       constexpr bool DUPA = SB >= 2, DUPB = !TT::TP && TT::SHB >= 1, DUPC = !TT::TP && TT::SHC >= 1;
@@ -347,9 +351,9 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
     if (!STALE || k == 0) { ma = cma; mb = cmb; mc = cmc; }
     else { ma = pma; mb = pmb; mc = pmc; }
     pma = cma; pmb = cmb; pmc = cmc;
-    const R ean = a_ok ? bi_exp_tab(xa - (R)ma, exp_tab) : (R)0;
-    const R ebn = b_ok ? bi_exp_tab(xb - (R)mb, exp_tab) : (R)0;
-    const R ecn = c_ok ? bi_exp_tab(xc - (R)mc, exp_tab) : (R)0;
+    const R ean = a_ok ? bi_exp_fast(xa - (R)ma, exp_tab) : (R)0;
+    const R ebn = b_ok ? bi_exp_fast(xb - (R)mb, exp_tab) : (R)0;
+    const R ecn = c_ok ? bi_exp_fast(xc - (R)mc, exp_tab) : (R)0;
     __syncwarp();
     if (t3.own_b) se[bi] = ebn;
     if (t3.own_c) se[NB + ci] = ecn;
@@ -541,7 +545,7 @@ int bi_launch_tile3_window(const BiCall &c, bi_model *mut) {
   const BiGroup &g = md->h.grp[0];
   Tile3Params p;
   bi_tile3_fill_params(c, p);
-  const int budget = md->max_smem_optin - 1024;
+  const int budget = md->max_smem_optin - 1024 - 6400;   // (the kernel's static tables)
   int rc;
   const bool f64 = md->arith == BI_ARITH_F64;
   if (c.algo == BI_ALGO_VMP)

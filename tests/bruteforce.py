@@ -21,7 +21,7 @@ def _ln(x):
 class TinyModel:
     """One agent, shared model (G = 1 arrays indexed at g = 0)."""
 
-    def __init__(self, n, m, dep, U, A, B, D, obs, act):
+    def __init__(self, n, m, dep, U, A, B, D, obs, act, bdep=None):
         self.n = [int(v) for v in n]
         self.m = [int(v) for v in m]
         self.dep = [list(d) for d in dep]
@@ -35,6 +35,8 @@ class TinyModel:
         self.F = len(self.n)
         self.off = np.concatenate([[0], np.cumsum(self.n)]).astype(int)
         self.states = list(itertools.product(*[range(k) for k in self.n]))
+        # B-dependencies: factor f's transition reads the previous states of bdep[f] (default: its own)
+        self.bdep = [list(d) for d in bdep] if bdep is not None else [[f] for f in range(self.F)]
 
     # log p(o_t | s_t) for a joint state tuple
     def ln_emit(self, t, s):
@@ -48,7 +50,7 @@ class TinyModel:
 
     def ln_trans(self, t, s_next, s_prev):
         """ln p(s_t = s_next | s_{t-1} = s_prev, u_{t-1}); t >= 1."""
-        return float(sum(_ln(self.B[f][s_next[f], s_prev[f], self.act[t - 1, f]])
+        return float(sum(_ln(self.B[f][(s_next[f],) + tuple(s_prev[g] for g in self.bdep[f]) + (self.act[t - 1, f],)])
                          for f in range(self.F)))
 
     def trajectories(self):

@@ -284,6 +284,111 @@ def test_gauss_seidel_sweeps_reach_a_fixed_point():
                                    atol=1e-10)
 
 
+# ---- non-trivial B-dependencies (transitions that read other factors' previous states) ----
+
+def tiny_bdep(seed, n, m, dep, U, bdep, T, *, N=1, sparsity=0.0, b_sparsity=0.0):
+    rng = np.random.default_rng(seed)
+    A, B, D = make_model(rng, n, m, dep, U, 1, sparsity=sparsity, d_alpha=1.0, bdep=bdep, b_sparsity=b_sparsity)
+    obs, act = sample_streams(rng, n, m, dep, U, 1, A, B, D, N, T, bdep=bdep)
+    return dict(n=n, m=m, dep=dep, U=U, G=1, A=A, B=B, D=D, obs=obs, act=act, bdep=bdep)
+
+
+def run_b(algo, w, K, **kw):
+    return oracle.run(algo, w["n"], w["m"], w["dep"], w["U"], w["G"], w["A"], w["B"], w["D"], w["obs"], w["act"], K,
+                      bdep=w["bdep"], **kw)
+
+
+@pytest.mark.parametrize("seed,bdep,b_sparsity", [(101, [[0, 1], [1]], 0.0), (102, [[1], [0, 1]], 0.0),
+                                                  (103, [[1, 0], [0]], 0.4)])
+def test_vmp_with_b_dependencies_is_the_enumerated_coordinate_optimum(seed, bdep, b_sparsity):
+    # the generic update of Section III-A on a model whose transitions read other factors' states:
+    # every (t, f) block of one Jacobi iteration equals the optimum found by enumerating trajectories
+    w = tiny_bdep(seed, [2, 3], [2, 3], [[0, 1], [1]], [2, 2], bdep, T=3, b_sparsity=b_sparsity)
+    model = TinyModel(w["n"], w["m"], w["dep"], w["U"], w["A"], w["B"], w["D"], w["obs"][0], w["act"][0], bdep=bdep)
+    rng = np.random.default_rng(seed)
+    q0 = np.concatenate([rng.dirichlet(np.ones(2), size=3), rng.dirichlet(np.ones(3), size=3)], axis=1)
+    q1, lq1, _ = run_b("vmp", w, 1, q_init=q0[None])
+    for t in range(3):
+        for f in range(2):
+            np.testing.assert_allclose(q1[0, t, model.off[f]:model.off[f + 1]], model.coordinate_optimum(q0, t, f),
+                                       atol=1e-12)
+    np.testing.assert_allclose(np.exp(lq1), q1, atol=1e-12)
+
+
+def test_filter_prior_with_b_dependencies_is_the_product_of_marginals_prediction():
+    # step 2 of the filter equals a fresh one-step problem whose D is sum_parents B prod q_1, taken with
+    # plain loops over the joint parent states
+    bdep = [[0, 1], [1, 0]]
+    w = tiny_bdep(111, [3, 2], [3, 2], [[0, 1], [1]], [2, 2], bdep, T=2)
+    q, _, _ = run_b("filter", w, 5)
+    D2 = []
+    for f, (lo, hi) in enumerate([(0, 3), (3, 5)]):
+        u = int(w["act"][0, 0, f])
+        pred = np.zeros(hi - lo)
+        for sn in range(hi - lo):
+            for par in itertools.product(*[range(w["n"][g]) for g in bdep[f]]):
+                wgt = 1.0
+                for g, sg in zip(bdep[f], par):
+                    wgt *= q[0, 0, [0, 3][g] + sg]
+                pred[sn] += float(w["B"][f][(0, sn) + par + (u,)]) * wgt
+        D2.append(pred.astype(np.float32)[None])
+    w2 = dict(w, D=D2, obs=w["obs"][:, 1:], act=w["act"][:, :0])
+    q2, _, _ = run_b("filter", w2, 5)
+    np.testing.assert_allclose(q2[0, 0], q[0, 1], atol=5e-7)   # D2 was rounded to float32
+
+
+def test_b_dependencies_on_the_factor_itself_are_the_plain_model():
+    w = tiny(112, [3, 4, 2], [3, 2], [[0, 1], [1, 2]], [2, 3, 1], T=4, N=2, sparsity=0.5)
+    for algo in ("filter", "vmp"):
+        a = run(algo, w, 4)
+        b = oracle.run(algo, w["n"], w["m"], w["dep"], w["U"], 1, w["A"], w["B"], w["D"], w["obs"], w["act"], 4,
+                       bdep=[[0], [1], [2]])
+        for x, y in zip(a, b):
+            np.testing.assert_allclose(y, x, atol=1e-13)
+    # a transition declared on a superset of its true parents (B replicated along the new axis): same beliefs
+    B = list(w["B"])
+    B[1] = np.ascontiguousarray(np.repeat(w["B"][1][:, :, :, None, :], 2, axis=3))   # [1, 4, 4, n_2 = 2, 3]
+    for algo in ("filter", "vmp"):
+        a = run(algo, w, 4)[0]
+        b = oracle.run(algo, w["n"], w["m"], w["dep"], w["U"], 1, w["A"], B, w["D"], w["obs"], w["act"], 4,
+                       bdep=[[0], [1, 2], [2]])[0]
+        np.testing.assert_allclose(b, a, atol=1e-12)
+
+
+def test_deterministic_parents_give_the_exact_transition_column():
+    # when the previous beliefs are point masses the prior is the transition's own column, whatever the
+    # number of parents; and MMP is refused on such models
+    bdep = [[0, 1], [1]]
+    w = tiny_bdep(113, [3, 2], [3, 2], [[0], [1]], [2, 1], bdep, T=1, N=1)
+    q_prev = np.array([[0.0, 1.0, 0.0, 1.0, 0.0]])
+    act_prev = np.array([[1, 0]], np.int32)
+    q, _, _ = run_b("filter", w, 1, q_prev=q_prev, act_prev=act_prev)
+    A0 = w["A"][0][0].astype(np.float64)
+    col = w["B"][0][0, :, 1, 0, 1].astype(np.float64)          # parents (s_0, s_1) = (1, 0), action 1
+    want = A0[w["obs"][0, 0, 0]] * col
+    np.testing.assert_allclose(q[0, 0, :3], want / want.sum(), atol=1e-12)
+    with pytest.raises(ValueError):
+        run_b("mmp", dict(w, obs=np.repeat(w["obs"], 2, axis=1), act=np.zeros((1, 1, 2), np.int32)), 2)
+
+
+def test_free_energy_with_b_dependencies_never_increases():
+    bdep = [[0, 1], [0]]
+    w = tiny_bdep(114, [2, 2], [2, 2], [[0, 1], [0]], [2, 1], bdep, T=3)
+    model = TinyModel(w["n"], w["m"], w["dep"], w["U"], w["A"], w["B"], w["D"], w["obs"][0], w["act"][0], bdep=bdep)
+    rng = np.random.default_rng(0)
+    q = np.concatenate([rng.dirichlet(np.ones(2), size=3), rng.dirichlet(np.ones(2), size=3)], axis=1)
+    f_prev = model.free_energy(q)
+    for sweep in range(2):
+        for t, f in itertools.product(range(3), range(2)):
+            upd, _, _ = run_b("vmp", w, 1, q_init=q[None])
+            q = q.copy()
+            q[t, model.off[f]:model.off[f + 1]] = upd[0, t, model.off[f]:model.off[f + 1]]
+            f_new = model.free_energy(q)
+            assert f_new <= f_prev + 1e-12
+            f_prev = f_new
+    assert f_prev >= -model.ln_evidence() - 1e-12
+
+
 # ---- P4: window edge conventions ------------------------------------------------
 
 def test_single_step_window_equals_filter_step():
