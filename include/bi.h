@@ -115,6 +115,27 @@ int bi_model_create_arith(const bi_model_desc *desc, int arith, void *cuda_strea
 int bi_model_arith(const bi_model_t *model);
 
 /* Synchronises the device, frees the packed copies and the handle's workspaces.  NULL is accepted. */
+/*
+ * A model whose transitions have non-trivial B-dependencies: factor f's next state depends on the
+ * previous states of a list of factors, p(s^f_{t+1} | s^{bdep(f)}_t, u^f_t) (Section III-B restricts
+ * itself to the trivial case bdep(f) = {f}; Section VI names the general case as the next step).
+ *   bdep_len  HOST [F]: k_f >= 1, at most BI_MAX_RANK
+ *   bdep      HOST [sum k_f]: 0-based factor ids, no repeats within a list (f itself need not be in it)
+ *   desc->B[f] DEVICE [G][n_f next][n_{bdep(f)[0]}]...[n_{bdep(f)[k-1]}][U_f] row-major, at most 2^20
+ *             entries per model; everything else of desc as for bi_model_create
+ * The mean-field update of Section III-A then gives: filtering, prior of a step = the transition
+ * tensor contracted with the previous step's beliefs of all its parents; VMP, past message = the
+ * tensor of logarithms contracted likewise, future message to a factor = the sum, over the factors
+ * whose transitions read it, of the log-tensor contracted with the next step's belief of that factor
+ * and this step's beliefs of the other parents.  Such handles serve bi_filter, bi_filter_from,
+ * bi_filter_continue, bi_vmp and bi_vmp_warm (one general kernel family; damping applies).  Marginal
+ * message passing has no reversed transition for several parents: bi_mmp and its variants, the calls
+ * with observation vectors and bi_vmp_from return BI_ERR_UNSUPPORTED on such a handle.
+ * Errors as bi_model_create; BI_ERR_INVALID_ARG for a malformed list, BI_ERR_UNSUPPORTED beyond the limits.
+ */
+int bi_model_create_bdep(const bi_model_desc *desc, const int32_t *bdep_len, const int32_t *bdep, int arith,
+                         void *cuda_stream, bi_model_t **out);
+
 int bi_model_destroy(bi_model_t *model);
 
 /*

@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_filter_continue", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_create_bdep", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_filter_continue", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -56,6 +56,9 @@ def lib():
         L.bi_model_create_arith.restype = ctypes.c_int
         L.bi_model_create_arith.argtypes = [ctypes.POINTER(_Desc), ctypes.c_int, ctypes.c_void_p,
                                             ctypes.POINTER(ctypes.c_void_p)]
+        L.bi_model_create_bdep.restype = ctypes.c_int
+        L.bi_model_create_bdep.argtypes = [ctypes.POINTER(_Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                           ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)]
         L.bi_model_arith.restype = ctypes.c_int
         L.bi_model_arith.argtypes = [ctypes.c_void_p]
         L.bi_model_destroy.restype = ctypes.c_int
@@ -117,10 +120,13 @@ class Model:
     header documents: ``A[i]: [G, m_i, n_dep...]``, ``B[f]: [G, n, n, U]``,
     ``D[f]: [G, n]``.  ``arith`` selects the kernels' arithmetic: ``"f64"``
     (default; reproduces a float64 evaluation to 1e-5) or ``"f32"`` (fast).
+    ``bdep`` (per factor, the factors its transition depends on) makes a model
+    with non-trivial B-dependencies (``bi_model_create_bdep``): ``B[f]`` is then
+    ``[G, n_f, n_bdep..., U_f]``.
     """
 
     def __init__(self, n: Sequence[int], m: Sequence[int], dep: Sequence[Sequence[int]], U: Sequence[int],
-                 G: int, A: List, B: List, D: List, stream=None, arith: str = "f64"):
+                 G: int, A: List, B: List, D: List, stream=None, arith: str = "f64", bdep=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("bi needs a CUDA device: there is no CPU path")
@@ -141,7 +147,12 @@ class Model:
         pd = (ctypes.c_void_p * self.F)(*[x.data_ptr() for x in D])
         d.A, d.B, d.D = [ctypes.cast(p, ctypes.c_void_p) for p in (pa, pb, pd)]
         h = ctypes.c_void_p()
-        if arith == "f64":
+        self.bdep = [[int(g) for g in x] for x in bdep] if bdep is not None else None
+        if self.bdep is not None:
+            bl, bf = _i32([len(x) for x in self.bdep]), _i32([g for x in self.bdep for g in x])
+            rc = L.bi_model_create_bdep(ctypes.byref(d), ctypes.cast(bl, ctypes.c_void_p), ctypes.cast(bf, ctypes.c_void_p),
+                                        ARITH[arith], _stream_ptr(stream), ctypes.byref(h))
+        elif arith == "f64":
             rc = L.bi_model_create(ctypes.byref(d), _stream_ptr(stream), ctypes.byref(h))
         else:
             rc = L.bi_model_create_arith(ctypes.byref(d), ARITH[arith], _stream_ptr(stream), ctypes.byref(h))
@@ -346,6 +357,6 @@ def model_from_workload(w, device="cuda", stream=None, arith: str = "f64") -> Mo
     A = [torch.from_numpy(a).to(device) for a in w.A]
     B = [torch.from_numpy(b).to(device) for b in w.B]
     D = [torch.from_numpy(d).to(device) for d in w.D]
-    md = Model(w.n, w.m, w.dep, w.U, w.G, A, B, D, stream=stream, arith=arith)
+    md = Model(w.n, w.m, w.dep, w.U, w.G, A, B, D, stream=stream, arith=arith, bdep=getattr(w, "bdep", None))
     torch.cuda.synchronize()
     return md

@@ -153,6 +153,23 @@ __global__ void bi_pack_comb_kernel(PackComb p) {
   ((R *)p.dst)[i] = acc;
 }
 
+// transition tensors with B-dependencies: source [G][n][PB][U] -> [G][U][n][PB], plain and clamped log
+template <typename R>
+__global__ void bi_pack_Bfull_kernel(const float *__restrict__ B, int64_t total, int n, int64_t PB, int U, R *Bfull,
+                                     R *logBfull) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int64_t par = e % PB;
+  int64_t r = e / PB;
+  const int sn = (int)(r % n);
+  r /= n;
+  const int u = (int)(r % U);
+  const int64_t g = r / U;
+  const float v = B[((g * n + sn) * PB + par) * U + u];
+  Bfull[e] = (R)v;
+  logBfull[e] = (R)log(fmax((double)v, 1e-16));
+}
+
 template <typename R>
 __global__ void bi_pack_D_kernel(const float *__restrict__ D, int G, int n, int npad, R *logD) {
   int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -222,13 +239,45 @@ extern "C" int bi_model_create(const bi_model_desc *desc, void *cuda_stream, bi_
 
 extern "C" int bi_model_arith(const bi_model_t *model) { return model ? model->arith : BI_ERR_INVALID_ARG; }
 
+static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep_len, const int32_t *bdep,
+                       void *cuda_stream, bi_model_t **out);
+
 extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void *cuda_stream, bi_model_t **out) {
+  return create_impl(desc, arith, nullptr, nullptr, cuda_stream, out);
+}
+
+extern "C" int bi_model_create_bdep(const bi_model_desc *desc, const int32_t *bdep_len, const int32_t *bdep, int arith,
+                                    void *cuda_stream, bi_model_t **out) {
+  if (!bdep_len || !bdep) return BI_ERR_INVALID_ARG;
+  return create_impl(desc, arith, bdep_len, bdep, cuda_stream, out);
+}
+
+static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep_len, const int32_t *bdep,
+                       void *cuda_stream, bi_model_t **out) {
   if (!out) return BI_ERR_INVALID_ARG;
   *out = nullptr;
   if (arith != BI_ARITH_F64 && arith != BI_ARITH_F32) return BI_ERR_INVALID_ARG;
   const size_t esz = arith == BI_ARITH_F64 ? 8 : 4;
   int rc = validate_desc(desc);
   if (rc != BI_OK) return rc;
+  if (bdep_len) {   // B-dependency lists: in range, no repeats, tensors of bounded size
+    int o = 0;
+    for (int f = 0; f < desc->F; ++f) {
+      if (bdep_len[f] < 1) return BI_ERR_INVALID_ARG;
+      if (bdep_len[f] > BI_MAX_RANK) return BI_ERR_UNSUPPORTED;
+      uint32_t seen = 0;
+      double entries = (double)desc->n[f] * desc->U[f];
+      for (int j = 0; j < bdep_len[f]; ++j) {
+        const int gq = bdep[o + j];
+        if (gq < 0 || gq >= desc->F) return BI_ERR_INVALID_ARG;
+        if (seen & (1u << gq)) return BI_ERR_SHAPE;
+        seen |= 1u << gq;
+        entries *= desc->n[gq];
+      }
+      if (entries > (double)(1 << 20)) return BI_ERR_UNSUPPORTED;
+      o += bdep_len[f];
+    }
+  }
   cudaStream_t stream = (cudaStream_t)cuda_stream;
 
   bi_model *md = new (std::nothrow) bi_model();
@@ -386,7 +435,7 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
 
   // a register-tile shape applies when the model is one rank-3 group over exactly its factors
   md->tile_sb = 0;
-  if (h.ngroups == 1 && F == 3 && h.grp[0].rank == 3)
+  if (!bdep_len && h.ngroups == 1 && F == 3 && h.grp[0].rank == 3)
     md->tile_sb = bi_tile3_shape(h.grp[0].dim[0], h.grp[0].dim[1], h.grp[0].dim[2]);
 
   // ---- allocate and pack
@@ -501,7 +550,39 @@ extern "C" int bi_model_create_arith(const bi_model_desc *desc, int arith, void 
       }
     }
   }
-  for (int f = 0; f < F && rc == BI_OK; ++f) {
+  h.has_bdep = bdep_len ? 1 : 0;
+  for (int f = 0, bo = 0; f < F && rc == BI_OK && bdep_len; ++f) {
+    // transition tensors of a model with B-dependencies (and ln D; the per-factor matrix forms are not made)
+    h.bdep_len[f] = bdep_len[f];
+    int64_t PB = 1;
+    for (int j = 0; j < bdep_len[f]; ++j) {
+      h.bdep[f][j] = bdep[bo + j];
+      PB *= h.n[bdep[bo + j]];
+    }
+    bo += bdep_len[f];
+    h.PB[f] = (int32_t)PB;
+    const int n = h.n[f], npad = h.npad[f], U = h.U[f];
+    const int64_t total = (int64_t)G * U * n * PB;
+    void *bfull, *lbfull, *ld;
+    if ((rc = dev_alloc(md, &bfull, (size_t)total * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &lbfull, (size_t)total * esz)) != BI_OK) break;
+    if ((rc = dev_alloc(md, &ld, (size_t)G * npad * esz)) != BI_OK) break;
+    h.Bfull[f] = bfull; h.logBfull[f] = lbfull; h.logD[f] = ld;
+    h.Bfull_stride[f] = (G == 1) ? 0 : (int64_t)U * n * PB;
+    h.Dstride[f] = (G == 1) ? 0 : npad;
+    const int threads = 256;
+    const unsigned gb = (unsigned)((total + threads - 1) / threads);
+    const unsigned gd = (unsigned)(((size_t)G * npad + threads - 1) / threads);
+    if (arith == BI_ARITH_F64) {
+      bi_pack_Bfull_kernel<double><<<gb, threads, 0, stream>>>(desc->B[f], total, n, PB, U, (double *)bfull, (double *)lbfull);
+      bi_pack_D_kernel<double><<<gd, threads, 0, stream>>>(desc->D[f], G, n, npad, (double *)ld);
+    } else {
+      bi_pack_Bfull_kernel<float><<<gb, threads, 0, stream>>>(desc->B[f], total, n, PB, U, (float *)bfull, (float *)lbfull);
+      bi_pack_D_kernel<float><<<gd, threads, 0, stream>>>(desc->D[f], G, n, npad, (float *)ld);
+    }
+    if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+  }
+  for (int f = 0; f < F && rc == BI_OK && !bdep_len; ++f) {
     int n = h.n[f], npad = h.npad[f], U = h.U[f];
     size_t count = (size_t)G * U * n * npad;
     void *bf, *lb, *lt, *bd, *ld, *bft, *bdt;
@@ -580,6 +661,7 @@ __global__ void bi_predictive_prior_kernel(const BiDev *__restrict__ mdp, int N,
 }
 
 int bi_dispatch(const BiCall &c, bi_model *mut) {
+  if (c.model->h.has_bdep) return bi_launch_generic(c, mut);   // the one family that contracts transition tensors
   const int only = c.model->test_family;   // testing aid: start at the named family
   int rc = BI_ERR_UNSUPPORTED;
   if (only == BI_FAMILY_ANY) {
@@ -608,6 +690,7 @@ static int run_call(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   if (!q_out || (model->h.M > 0 && !obs) || (T > 1 && !act)) return BI_ERR_INVALID_ARG;
   if (model->h.G != 1 && model->h.G != N) return BI_ERR_SHAPE;
   if (algo != BI_ALGO_FILTER && T > BI_MAX_T) return BI_ERR_UNSUPPORTED;
+  if (model->h.has_bdep && (algo == BI_ALGO_MMP || (algo != BI_ALGO_FILTER && q_prev))) return BI_ERR_UNSUPPORTED;
   BiCall c;
   c.model = model; c.algo = algo; c.N = N; c.T = T; c.K = iters;
   c.obs = obs; c.act = act; c.q_out = q_out; c.logq_out = logq_out; c.argmax_out = argmax_out;
@@ -680,6 +763,7 @@ static int run_soft(const bi_model_t *model, int algo, int32_t N, int32_t T, con
   if (!q_out || (model->h.M > 0 && !obs_soft) || (T > 1 && !act)) return BI_ERR_INVALID_ARG;
   if (model->h.G != 1 && model->h.G != N) return BI_ERR_SHAPE;
   if (algo != BI_ALGO_FILTER && T > BI_MAX_T) return BI_ERR_UNSUPPORTED;
+  if (model->h.has_bdep) return BI_ERR_UNSUPPORTED;
   return bi_run_soft(model, algo, N, T, obs_soft, act, iters, q_out, logq_out, argmax_out,
                      (cudaStream_t)cuda_stream);
 }

@@ -77,6 +77,14 @@ struct alignas(16) BiDev {
   const void *BdagT[BI_MAX_F]; // [s_next][s_prev]      = B[s_next, s_prev, u] / sum_r B[s_next, r, u]
   const void *logD[BI_MAX_F];  // [G][npad]
   int64_t Bstride[BI_MAX_F];    // floats per model in each B array (0 when shared)
+  // Non-trivial B-dependencies (has_bdep != 0): factor f's transition reads the previous states of the
+  // factors bdep[f][0..bdep_len[f]); PB[f] = product of their state counts.  The transition tensors,
+  // per model g and action u: [n_f (next)][PB[f]] with the parents in list order, last fastest; the six
+  // per-factor matrix forms above are not made for such a model.
+  int32_t has_bdep, bdep_len[BI_MAX_F], bdep[BI_MAX_F][BI_MAX_RANK], PB[BI_MAX_F];
+  const void *Bfull[BI_MAX_F];     // B[s_next, parents, u]
+  const void *logBfull[BI_MAX_F];  // ln max(., 1e-16) of the same
+  int64_t Bfull_stride[BI_MAX_F];  // elements per model (0 when shared)
   int64_t Dstride[BI_MAX_F];
   uint32_t *status;
 };
@@ -85,7 +93,7 @@ struct alignas(16) BiDev {
 struct bi_model {
   BiDev h;          // host copy (device pointers inside)
   BiDev *d;         // device copy
-  void *allocs[10 + 2 * BI_MAX_M + 8 * BI_MAX_F];  // status, descriptor, pre-summed table, 2 per modality, 7 per factor
+  void *allocs[10 + 2 * BI_MAX_M + 10 * BI_MAX_F];  // status, descriptor, pre-summed table, 2 per modality, 7 per factor
   int nalloc;
   int arith;        // BI_ARITH_F64 or BI_ARITH_F32
   int device;

@@ -219,6 +219,68 @@ __device__ __forceinline__ void all_groups(const BiDev &md, int g, const int32_t
   }
 }
 
+// ---- transition tensors with several parents (non-trivial B-dependencies) ----
+// One warp per output value, lanes over the joint states of the parents; sums in a fixed order.
+// X: the tensor's rows for one model and action, [n_f][PB]; q: one step's beliefs (padded layout).
+
+// sum_{parents} X[s_next][parents] prod_j q_{parent_j}[s_j]
+template <typename R>
+__device__ R bdep_expect(const BiDev &md, int f, const R *__restrict__ Xrow, const R *q, int lane) {
+  const int k = md.bdep_len[f], PB = md.PB[f];
+  R acc = (R)0;
+  for (int e = lane; e < PB; e += 32) {
+    int rem = e;
+    R w = (R)1;
+    for (int j = k - 1; j >= 0; --j) {
+      const int gq = md.bdep[f][j], nj = md.n[gq];
+      const int d = rem % nj;
+      rem /= nj;
+      w *= q[md.offp[gq] + d];
+    }
+    acc = fma(Xrow[e], w, acc);
+  }
+  return warp_sum(acc);
+}
+
+// VMP future message to state s of factor f0 at a step: over every factor h whose transition reads f0,
+// sum_{s'} qn_h[s'] sum_{parents with s_f0 = s} ln B_h[s'][parents] prod_{other parents} q[...];
+// act_t: the actions taken at this step
+template <typename R>
+__device__ R bdep_future(const BiDev &md, int g, int f0, int s, const R *q, const R *qn,
+                         const int32_t *__restrict__ act_t, int lane) {
+  R acc = (R)0;
+  for (int h = 0; h < md.F; ++h) {
+    const int k = md.bdep_len[h];
+    int pos = -1;
+    for (int j = 0; j < k; ++j)
+      if (md.bdep[h][j] == f0) pos = j;
+    if (pos < 0) continue;
+    const int nh = md.n[h], PB = md.PB[h];
+    const int u = clamp_flag(act_t[h], md.U[h], md.status, BI_FLAG_ACT_RANGE);
+    const R *X = (const R *)md.logBfull[h] + (size_t)g * md.Bfull_stride[h] + (size_t)u * nh * PB;
+    const int others = PB / md.n[f0];
+    for (int i = lane; i < nh * others; i += 32) {
+      const int sn = i / others;
+      int rem = i - sn * others, e = 0, stride = 1;
+      R w = (R)1;
+      for (int j = k - 1; j >= 0; --j) {
+        const int gq = md.bdep[h][j], nj = md.n[gq];
+        int d;
+        if (j == pos) d = s;
+        else {
+          d = rem % nj;
+          rem /= nj;
+          w *= q[md.offp[gq] + d];
+        }
+        e += d * stride;
+        stride *= nj;
+      }
+      acc = fma(qn[md.offp[h] + sn] * w, X[(size_t)sn * PB + e], acc);
+    }
+  }
+  return warp_sum(acc);
+}
+
 template <typename R, int ALGO, bool STAGED>
 __global__ void __launch_bounds__(256)
 bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__restrict__ obs,
@@ -263,6 +325,25 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
     }
     for (int t = 0; t < T; ++t) {
       // ln prior: D at the first step, else B_u q_{t-1} (cur still holds step t-1)
+      if (md.has_bdep) {   // transition tensors with several parents: a warp per state
+        for (int idx = tid >> 5; idx < Sp; idx += NT >> 5) {
+          int f = 0;
+          while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+          const int s = idx - md.offp[f], n = md.n[f];
+          R lp = (R)0;
+          if (s < n) {
+            if (t == 0 && !from_prev) {
+              lp = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
+            } else {
+              const int ur = t == 0 ? act_prev[(size_t)a * F + f] : act[((size_t)a * (T - 1) + (t - 1)) * F + f];
+              const int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
+              const R *row = (const R *)md.Bfull[f] + (size_t)g * md.Bfull_stride[f] + ((size_t)u * n + s) * md.PB[f];
+              lp = bi_log(bi_max(bdep_expect<R>(md, f, row, cur, tid & 31), (R)BI_EPS));
+            }
+          }
+          if ((tid & 31) == 0) lpri[idx] = lp;
+        }
+      } else
       for (int idx = tid; idx < Sp; idx += NT) {
         int f = 0;
         while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
@@ -334,6 +415,26 @@ bi_generic_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t *__
         const R *qt = cur + t * Sp;
         // transition messages (Section IV: low-rank contractions of B with the
         // neighbouring steps' beliefs)
+        if (md.has_bdep) {   // transition tensors with several parents (VMP only): a warp per state
+          for (int idx = tid >> 5; idx < Sp; idx += NT >> 5) {
+            int f = 0;
+            while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+            const int s = idx - md.offp[f], n = md.n[f];
+            R msg = (R)0;
+            if (s < n) {
+              if (t == 0) {
+                msg = ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
+              } else {
+                const int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
+                const R *row = (const R *)md.logBfull[f] + (size_t)g * md.Bfull_stride[f] + ((size_t)u * n + s) * md.PB[f];
+                msg = bdep_expect<R>(md, f, row, cur + (t - 1) * Sp, tid & 31);
+              }
+              if (t + 1 < T)
+                msg += bdep_future<R>(md, g, f, s, qt, cur + (t + 1) * Sp, act + ((size_t)a * (T - 1) + t) * F, tid & 31);
+            }
+            if ((tid & 31) == 0) ell[idx] = msg;
+          }
+        } else
         for (int idx = tid; idx < Sp; idx += NT) {
           int f = 0;
           while (f + 1 < F && idx >= md.offp[f + 1]) ++f;

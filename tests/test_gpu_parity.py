@@ -784,3 +784,77 @@ def test_a_copy_that_never_arrives_is_reported_not_waited_for():
     ref = oracle.run_workload(w.take_agents(sel), "vmp")[0]
     assert np.abs(q[sel] - ref).max() <= 1e-5
     md.close()
+
+
+# ---- non-trivial B-dependencies (bi_model_create_bdep) ----
+
+def _bdep_workload(seed, n, m, dep, U, bdep, N, T, K, G=1, sparsity=0.0, b_sparsity=0.0):
+    rng = np.random.default_rng(seed)
+    A, B, D = make_model(rng, n, m, dep, U, G, sparsity=sparsity, d_alpha=1.0, bdep=bdep, b_sparsity=b_sparsity)
+    obs, act = sample_streams(rng, n, m, dep, U, G, A, B, D, N, T, bdep=bdep)
+    return Workload(name="bdep", algo="filter", n=np.asarray(n, np.int32), m=np.asarray(m, np.int32), dep=dep,
+                    U=np.asarray(U, np.int32), G=G, A=A, B=B, D=D, N=N, T=T, K=K, obs=obs, act=act, bdep=bdep)
+
+
+BDEP_CASES = {
+    "two_parents": dict(n=[4, 3], m=[5, 4], dep=[[0, 1], [1]], U=[2, 2], bdep=[[0, 1], [1]], N=9, T=6, K=6),
+    "cross": dict(n=[3, 5, 2], m=[4, 3], dep=[[0, 1], [2, 1]], U=[2, 1, 3], bdep=[[1], [0, 2], [2, 1, 0]], N=7, T=5, K=5,
+                  sparsity=0.5, b_sparsity=0.5),
+    "wide": dict(n=[6, 5, 4, 3], m=[3, 4, 2], dep=[[0, 1, 2], [3], [1, 3]], U=[1, 2, 2, 1],
+                 bdep=[[0, 1, 2, 3], [1], [3, 2], [0, 3]], N=5, T=4, K=4),
+    "per_agent": dict(n=[3, 4], m=[3, 2], dep=[[0, 1], [1]], U=[2, 2], bdep=[[1, 0], [0]], N=4, T=5, K=4, G=4, sparsity=0.6),
+    "ragged_edge": dict(n=[32, 2], m=[2], dep=[[0]], U=[1, 1], bdep=[[0, 1], [1, 0]], N=1, T=1, K=1),
+}
+
+
+@pytest.mark.parametrize("algo", ["filter", "vmp"])
+@pytest.mark.parametrize("case", sorted(BDEP_CASES))
+def test_b_dependencies(case, algo):
+    """Transitions that read other factors' previous states, against the oracle's enumerated reading."""
+    w = _bdep_workload(1200 + sorted(BDEP_CASES).index(case), **BDEP_CASES[case])
+    res = check_workload(w, algo)
+    print(case, algo, res)
+    assert res["kernel"].startswith("generic_")
+
+
+def test_b_dependencies_call_forms_and_refusals():
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = _bdep_workload(1300, [4, 3], [5, 4], [[0, 1], [1]], [2, 2], [[0, 1], [1, 0]], N=6, T=6, K=5)
+    md = bi.model_from_workload(w)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    # blocks of steps through the handle's record equal the single call; a float32 q_prev is within tolerance
+    whole = md.bi_filter(obs, act, w.K).cpu().numpy()
+    head = md.bi_filter(obs[:, :2].contiguous(), act[:, :1].contiguous(), w.K)
+    tail = md.bi_filter_continue(obs[:, 2:].contiguous(), act[:, 2:].contiguous(), act[:, 1].contiguous(), w.K)
+    assert np.array_equal(torch.cat([head, tail], dim=1).cpu().numpy(), whole)
+    tail32 = md.bi_filter_from(obs[:, 2:].contiguous(), act[:, 2:].contiguous(), head[:, -1].contiguous(),
+                               act[:, 1].contiguous(), w.K).cpu().numpy()
+    ref = oracle.run_workload(w, "filter")[0]
+    assert np.abs(whole - ref).max() <= 1e-5 and np.abs(tail32 - ref[:, 2:]).max() <= 1e-5
+    # a warm start
+    rng = np.random.default_rng(5)
+    q_init = np.concatenate([rng.dirichlet(np.full(int(k), 2.0), size=(w.N, w.T)) for k in w.n], axis=2).astype(np.float32)
+    q = md.bi_vmp_warm(obs, act, torch.from_numpy(q_init).cuda(), 3).cpu().numpy()
+    ref = oracle.run("vmp", w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, w.obs, w.act, 3,
+                     q_init=q_init.astype(np.float64), bdep=w.bdep)[0]
+    assert np.abs(q - ref).max() <= 1e-5
+    # what has no counterpart with several parents is refused
+    for call in (lambda: md.bi_mmp(obs, act, 2),
+                 lambda: md.bi_mmp_warm(obs, act, torch.from_numpy(q_init).cuda(), 2),
+                 lambda: md.run_from("vmp", obs, act, head[:, -1].contiguous(), act[:, 1].contiguous(), 2),
+                 lambda: md.run_soft("filter", torch.zeros((w.N, w.T, int(w.m.sum())), device="cuda"), act, 2)):
+        with pytest.raises(bi.BiError) as e:
+            call()
+        assert e.value.code == -3
+    assert md.status() == 0
+    md.close()
+    # malformed lists
+    A = [torch.from_numpy(a).cuda() for a in w.A]
+    B = [torch.from_numpy(b).cuda() for b in w.B]
+    D = [torch.from_numpy(d).cuda() for d in w.D]
+    for bad, code in (([[0, 0], [1]], -2), ([[0, 2], [1]], -1), ([[], [1]], -1)):
+        with pytest.raises(bi.BiError) as e:
+            bi.Model(w.n, w.m, w.dep, w.U, 1, A, B, D, bdep=bad)
+        assert e.value.code == code, (bad, e.value.code)
