@@ -111,6 +111,29 @@ int bi_model_create(const bi_model_desc *desc, void *cuda_stream, bi_model_t **o
 /* As bi_model_create (which uses BI_ARITH_F64) with the arithmetic chosen. */
 int bi_model_create_arith(const bi_model_desc *desc, int arith, void *cuda_stream, bi_model_t **out);
 
+/*
+ * Storage of a per-agent model's observation slices in the layout the window kernels gather from
+ * (HOST outputs, bytes): *dense as full slices, *compressed as the handle keeps them when most of A is
+ * zero -- the paper's motive for sparse storage, Section III-D: its BCOO variants cut parameter counts
+ * 14-fold without a speed-up, Section V-B.  Here a slice becomes one 64-bit mask per lane (which of the
+ * lane's elements are not the floor ln 1e-16) plus those values; bi_vmp / bi_mmp read that form, so the
+ * gather's HBM traffic shrinks with the share of zeros; the result is bit for bit that of the dense
+ * form.  Made automatically by bi_model_create for per-agent register-tile models (G > 1, up to four
+ * modalities) when it is under 60 % of the dense size; sizing it needs the non-zero counts on the
+ * host, so creating such a handle synchronises the stream.  Both are 0 when the handle has no
+ * compressed form.
+ */
+int bi_model_slice_bytes(const bi_model_t *model, int64_t *dense, int64_t *compressed);
+
+/*
+ * Chooses the form later bi_vmp / bi_mmp calls on this handle gather from: on != 0 the compressed
+ * one (BI_ERR_UNSUPPORTED when the handle has none), 0 the dense one (the default).  Measured on a
+ * B200 with 70 % zeros: a third of the bytes from HBM, but the calls are not bound by that gather,
+ * and decoding costs about 5 % more time; the switch is for deployments where HBM traffic or
+ * capacity is the scarcer resource.
+ */
+int bi_model_set_compressed(bi_model_t *model, int on);
+
 /* BI_ARITH_* of a handle, or BI_ERR_INVALID_ARG for NULL. */
 int bi_model_arith(const bi_model_t *model);
 

@@ -27,7 +27,7 @@ BI_ARITH_F64 = 0
 BI_ARITH_F32 = 1
 ARITH = {"f64": BI_ARITH_F64, "f32": BI_ARITH_F32}
 
-EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_create_bdep", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_filter_continue", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_status",
+EXPORTS = ["bi_model_create", "bi_model_create_arith", "bi_model_create_bdep", "bi_model_slice_bytes", "bi_model_set_compressed", "bi_model_arith", "bi_model_destroy", "bi_filter", "bi_filter_from", "bi_filter_continue", "bi_vmp", "bi_mmp", "bi_vmp_warm", "bi_mmp_warm", "bi_vmp_from", "bi_mmp_from", "bi_filter_soft", "bi_vmp_soft", "bi_mmp_soft", "bi_model_set_damping", "bi_status",
            "bi_last_kernel", "bi_launch_count", "bi_strerror", "bi_filter_static"]
 BI_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -59,6 +59,10 @@ def lib():
         L.bi_model_create_bdep.restype = ctypes.c_int
         L.bi_model_create_bdep.argtypes = [ctypes.POINTER(_Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
                                            ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)]
+        L.bi_model_set_compressed.restype = ctypes.c_int
+        L.bi_model_set_compressed.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        L.bi_model_slice_bytes.restype = ctypes.c_int
+        L.bi_model_slice_bytes.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]
         L.bi_model_arith.restype = ctypes.c_int
         L.bi_model_arith.argtypes = [ctypes.c_void_p]
         L.bi_model_destroy.restype = ctypes.c_int
@@ -308,6 +312,21 @@ class Model:
         if rc != BI_OK:
             raise BiError(rc, "bi_status")
         return int(v.value)
+
+    def set_compressed(self, on: bool):
+        """Window calls gather from the compressed slices (``bi_model_set_compressed``)."""
+        rc = lib().bi_model_set_compressed(self._h, int(bool(on)))
+        if rc != BI_OK:
+            raise BiError(rc, "bi_model_set_compressed")
+
+    def slice_bytes(self):
+        """(dense, compressed) bytes of a per-agent model's slices as the window kernels gather them
+        (``bi_model_slice_bytes``); (0, 0) when the handle keeps no compressed form."""
+        a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+        rc = lib().bi_model_slice_bytes(self._h, ctypes.byref(a), ctypes.byref(b))
+        if rc != BI_OK:
+            raise BiError(rc, "bi_model_slice_bytes")
+        return int(a.value), int(b.value)
 
     @property
     def last_kernel(self) -> str:

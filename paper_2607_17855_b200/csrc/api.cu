@@ -127,6 +127,48 @@ __global__ void bi_pack_tile_kernel(PackTile p) {
   ((R *)p.dst)[e] = out;
 }
 
+// ---- compressed lane-interleaved slices (sparse per-agent models) ----
+// A slice in the lane-interleaved layout: 16-byte vector v of lane u at (v * LPU + u) * VE, so lane u's
+// local element i = v * VE + w sits at ((i / VE) * LPU + u) * VE + i % VE.
+template <typename R>
+__global__ void bi_floor_log_kernel(R *out) { out[0] = (R)log(fmax(0.0, 1e-16)); }
+
+// masks[slice][u]: bit i set when lane u's i-th element differs from the floor; counts[slice]: set bits
+template <typename R>
+__global__ void bi_compress_count_kernel(const R *__restrict__ tile, int64_t nslices, int P_tile, int LPU, int VE,
+                                         const R *__restrict__ flr, unsigned long long *masks, int32_t *counts) {
+  const int64_t sl = (int64_t)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+  const int lane = threadIdx.x & 31;
+  if (sl >= nslices) return;
+  const R f = flr[0];
+  const int nloc = P_tile / LPU;
+  int total = 0;
+  for (int u = lane; u < LPU; u += 32) {
+    unsigned long long m = 0ull;
+    for (int i = 0; i < nloc; ++i)
+      if (tile[sl * P_tile + ((size_t)(i / VE) * LPU + u) * VE + i % VE] != f) m |= 1ull << i;
+    masks[sl * LPU + u] = m;
+    total += __popcll(m);
+  }
+  for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+  if (lane == 0) counts[sl] = total;
+}
+// the values that are not the floor, lane after lane, at the slice's offset
+template <typename R>
+__global__ void bi_compress_fill_kernel(const R *__restrict__ tile, int64_t nslices, int P_tile, int LPU, int VE,
+                                        const unsigned long long *__restrict__ masks,
+                                        const long long *__restrict__ off, R *vals) {
+  const int64_t sl = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (sl >= nslices) return;
+  long long o = off[sl];
+  const int nloc = P_tile / LPU;
+  for (int u = 0; u < LPU; ++u) {
+    unsigned long long m = masks[sl * LPU + u];
+    for (int i = 0; i < nloc; ++i, m >>= 1)
+      if (m & 1ull) vals[o++] = tile[sl * P_tile + ((size_t)(i / VE) * LPU + u) * VE + i % VE];
+  }
+}
+
 // Pre-summed slices of a register-tile group: out[g][combo][e] = sum over the group's members, in
 // member order (the order the kernels add them in), of that member's slice for its outcome in combo.
 struct PackComb {
@@ -239,6 +281,20 @@ extern "C" int bi_model_create(const bi_model_desc *desc, void *cuda_stream, bi_
 
 extern "C" int bi_model_arith(const bi_model_t *model) { return model ? model->arith : BI_ERR_INVALID_ARG; }
 
+extern "C" int bi_model_set_compressed(bi_model_t *model, int on) {
+  if (!model) return BI_ERR_INVALID_ARG;
+  if (on && model->slice_bytes_compressed == 0) return BI_ERR_UNSUPPORTED;
+  model->use_compressed = on ? 1 : 0;
+  return BI_OK;
+}
+
+extern "C" int bi_model_slice_bytes(const bi_model_t *model, int64_t *dense, int64_t *compressed) {
+  if (!model || !dense || !compressed) return BI_ERR_INVALID_ARG;
+  *dense = model->slice_bytes_dense;
+  *compressed = model->slice_bytes_compressed;
+  return BI_OK;
+}
+
 static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep_len, const int32_t *bdep,
                        void *cuda_stream, bi_model_t **out);
 
@@ -284,6 +340,7 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
   if (!md) return BI_ERR_ALLOC;
   memset(md, 0, sizeof(*md));
   md->damping = 1.0;
+  if (const char *e = getenv("BI_TEST_NO_COMPRESS")) md->test_no_compress = atoi(e) != 0;
   if (const char *e = getenv("BI_TEST_DROP_COPY")) md->test_drop_copy = atoi(e) > 0 ? atoi(e) : 0;   // testing aids,
   if (const char *e = getenv("BI_TEST_FAMILY")) {                                                  // read here only
     md->test_family = !strcmp(e, "warp") ? BI_FAMILY_WARP : !strcmp(e, "generic") ? BI_FAMILY_GENERIC : BI_FAMILY_ANY;
@@ -548,6 +605,96 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
         md->tile_comb = td;
         md->tile_ncomb = q.ncomb;
       }
+    }
+  }
+  // Per-agent register-tile models whose slices are mostly the floor ln 1e-16 (sparse A): a compressed
+  // copy of the lane-interleaved slices for the window kernels' gather (a mask per lane and the other
+  // values).  Sizing it needs the counts on the host, so making such a handle synchronises the stream.
+  md->slice_bytes_dense = md->slice_bytes_compressed = 0;
+  if (rc == BI_OK && md->tile_sb > 0) {
+    void *fl = nullptr;
+    rc = dev_alloc(md, &fl, 16);
+    if (rc == BI_OK) {
+      md->tile_floor = fl;
+      if (arith == BI_ARITH_F64) bi_floor_log_kernel<double><<<1, 1, 0, stream>>>((double *)fl);
+      else bi_floor_log_kernel<float><<<1, 1, 0, stream>>>((float *)fl);
+      if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+    }
+  }
+  if (rc == BI_OK && md->tile_sb > 0 && G > 1 && !md->test_no_compress) {
+    const BiGroup &g0 = h.grp[0];
+    const int nm = g0.mem_end - g0.mem_begin;
+    int NAP = 1;
+    while (NAP < g0.dim[0]) NAP <<= 1;
+    const int LPU = NAP * md->tile_sb, VE = (int)(16 / esz), P_tile = md->tile_P;
+    if (nm <= 4 && P_tile / LPU <= 64) {
+      std::vector<unsigned long long *> masks(nm, nullptr);
+      std::vector<std::vector<long long>> offs(nm);
+      long long dense = 0, comp = 0;
+      // pass 1: masks and counts of every member; offsets on the host
+      for (int j = 0; j < nm && rc == BI_OK; ++j) {
+        const BiMember &mm = h.mem[g0.mem_begin + j];
+        const int64_t ns = (int64_t)G * mm.m;
+        int32_t *cnt = nullptr;
+        if (cudaMalloc(&masks[j], (size_t)ns * LPU * 8) != cudaSuccess || cudaMalloc(&cnt, (size_t)ns * 4) != cudaSuccess) {
+          cudaGetLastError();
+          if (cnt) cudaFree(cnt);
+          rc = BI_ERR_ALLOC;
+          break;
+        }
+        const unsigned blocks = (unsigned)((ns + 7) / 8);
+        if (arith == BI_ARITH_F64)
+          bi_compress_count_kernel<double><<<blocks, 256, 0, stream>>>((const double *)mm.logA_tile, ns, P_tile, LPU, VE,
+                                                                       (const double *)md->tile_floor, masks[j], cnt);
+        else
+          bi_compress_count_kernel<float><<<blocks, 256, 0, stream>>>((const float *)mm.logA_tile, ns, P_tile, LPU, VE,
+                                                                      (const float *)md->tile_floor, masks[j], cnt);
+        std::vector<int32_t> hc((size_t)ns);
+        if (cudaMemcpyAsync(hc.data(), cnt, (size_t)ns * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess)
+          rc = BI_ERR_CUDA;
+        cudaFree(cnt);
+        offs[j].assign((size_t)ns + 1, 0);
+        for (int64_t i = 0; i < ns; ++i) offs[j][(size_t)i + 1] = offs[j][(size_t)i] + hc[(size_t)i];
+        dense += ns * (long long)P_tile * (long long)esz;
+        comp += offs[j][(size_t)ns] * (long long)esz + ns * (long long)LPU * 8 + (ns + 1) * 8;
+      }
+      // worth it when the compressed form is under 60 % of the dense one
+      if (rc == BI_OK && comp * 10 < dense * 6) {
+        for (int j = 0; j < nm && rc == BI_OK; ++j) {
+          BiMember &mm = h.mem[g0.mem_begin + j];
+          const int64_t ns = (int64_t)G * mm.m;
+          void *dv = nullptr, *doff = nullptr, *dm = nullptr;
+          if ((rc = dev_alloc(md, &dv, (size_t)offs[j][(size_t)ns] * esz)) != BI_OK) break;
+          if ((rc = dev_alloc(md, &doff, (size_t)(ns + 1) * 8)) != BI_OK) break;
+          if ((rc = dev_alloc(md, &dm, (size_t)ns * LPU * 8)) != BI_OK) break;
+          if (cudaMemcpyAsync(doff, offs[j].data(), (size_t)(ns + 1) * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+              cudaMemcpyAsync(dm, masks[j], (size_t)ns * LPU * 8, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+            rc = BI_ERR_CUDA;
+            break;
+          }
+          const unsigned blocks = (unsigned)((ns + 127) / 128);
+          if (arith == BI_ARITH_F64)
+            bi_compress_fill_kernel<double><<<blocks, 128, 0, stream>>>((const double *)mm.logA_tile, ns, P_tile, LPU, VE,
+                                                                        (const unsigned long long *)dm,
+                                                                        (const long long *)doff, (double *)dv);
+          else
+            bi_compress_fill_kernel<float><<<blocks, 128, 0, stream>>>((const float *)mm.logA_tile, ns, P_tile, LPU, VE,
+                                                                       (const unsigned long long *)dm,
+                                                                       (const long long *)doff, (float *)dv);
+          if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+          // (the host offsets must outlive their asynchronous copy)
+          if (rc == BI_OK && cudaStreamSynchronize(stream) != cudaSuccess) rc = BI_ERR_CUDA;
+          mm.cmask = (const unsigned long long *)dm;
+          mm.cvals = dv;
+          mm.coff = (const long long *)doff;
+        }
+        md->slice_bytes_dense = dense;
+        md->slice_bytes_compressed = comp;
+      }
+      cudaStreamSynchronize(stream);
+      for (int j = 0; j < nm; ++j)
+        if (masks[j]) cudaFree(masks[j]);
     }
   }
   h.has_bdep = bdep_len ? 1 : 0;

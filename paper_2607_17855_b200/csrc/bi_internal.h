@@ -55,6 +55,13 @@ struct BiGroup {
 struct BiMember {
   const void *logA;   // packed [G][m][P_pad], float or double (the handle's arithmetic)
   const void *logA_tile;  // lane-interleaved copy [G][m][P_tile] for the register-tile kernels, or NULL
+  // Compressed form of the lane-interleaved copy for sparse per-agent models (or NULL): most entries
+  // of such a slice are the floor ln 1e-16 (a zero of A), so a slice is stored as one 64-bit mask per
+  // lane of a unit (bit i set: the lane's i-th element is not the floor) plus the other values, packed
+  // lane after lane.  cmask: [G * m][LPU]; coff: [G * m + 1] element offsets into cvals.
+  const unsigned long long *cmask;
+  const void *cvals;
+  const long long *coff;
   int64_t gstride;    // floats per model (0 when the model is shared)
   int32_t m, modality, P_pad, pad_;
 };
@@ -93,7 +100,7 @@ struct alignas(16) BiDev {
 struct bi_model {
   BiDev h;          // host copy (device pointers inside)
   BiDev *d;         // device copy
-  void *allocs[10 + 2 * BI_MAX_M + 10 * BI_MAX_F];  // status, descriptor, pre-summed table, 2 per modality, 7 per factor
+  void *allocs[24 + 2 * BI_MAX_M + 10 * BI_MAX_F];  // status, descriptor, pre-summed table, 2 per modality, 7 per factor
   int nalloc;
   int arith;        // BI_ARITH_F64 or BI_ARITH_F32
   int device;
@@ -101,6 +108,10 @@ struct bi_model {
   int max_smem_optin;
   int tile_sb;      // > 0: a register-tile shape matches; lanes along b per (agent, step)
   int tile_P;       // elements per lane-interleaved slice
+  const void *tile_floor;   // device scalar: ln 1e-16 in the arithmetic type, as the pack kernels compute it
+  long long slice_bytes_dense, slice_bytes_compressed;   // per-agent tile models: bytes of the two forms (0: none)
+  int test_no_compress;     // testing aid (BI_TEST_NO_COMPRESS, read when the handle is made)
+  int use_compressed;       // window calls gather from the compressed form (bi_model_set_compressed)
   // Register-tile models with few outcome combinations: the group's slices pre-summed for every
   // combination, [G][tile_ncomb][tile_P] in the lane-interleaved layout (one gather per step instead of
   // one per modality and no additions); combination index = sum_i outcome_i * tile_comb_mul[i] over the

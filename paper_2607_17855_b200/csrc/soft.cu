@@ -178,6 +178,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     BiMember &mm = sh.h.mem[k];
     mm.logA = w + off_pack[k];
     mm.logA_tile = tile && k == 0 ? w + off_tile : nullptr;
+    mm.cmask = nullptr; mm.cvals = nullptr; mm.coff = nullptr;   // (the slices formed above are dense)
     mm.gstride = (int64_t)T * g.P_pad;
     mm.m = T;
     mm.modality = k;

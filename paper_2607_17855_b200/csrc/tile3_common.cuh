@@ -14,6 +14,10 @@ struct Tile3Params {
   int64_t gstride[BI_MAX_M];
   int32_t modality[BI_MAX_M], mcount[BI_MAX_M];
   int32_t nmem, P_tile;
+  const unsigned long long *cmask[BI_MAX_M];   // compressed slices (BiMember), all NULL when the model has none
+  const void *cvals[BI_MAX_M];
+  const long long *coff[BI_MAX_M];
+  const void *floor_log;     // device scalar ln 1e-16
   const void *Lcomb;        // the group's slices pre-summed for every outcome combination [G][ncomb][P_tile], or NULL
   int32_t ncomb, comb_mul[BI_MAX_M];   // combination index = sum_i outcome_i * comb_mul[i]
   int32_t fac[3];   // factor ids of the axes a, b, c
@@ -61,6 +65,7 @@ static inline void bi_tile3_fill_params(const BiCall &c, Tile3Params &p) {
   const BiDev &h = md->h;
   const BiGroup &g = h.grp[0];
   p.nmem = g.mem_end - g.mem_begin;
+  p.floor_log = md->tile_floor;
   p.Lcomb = md->tile_comb;
   p.ncomb = md->tile_ncomb;
   for (int i = 0; i < p.nmem; ++i) p.comb_mul[i] = md->tile_comb_mul[i];
@@ -71,6 +76,8 @@ static inline void bi_tile3_fill_params(const BiCall &c, Tile3Params &p) {
     p.gstride[i] = mm.gstride;
     p.modality[i] = mm.modality;
     p.mcount[i] = mm.m;
+    const bool comp = md->use_compressed != 0;
+    p.cmask[i] = comp ? mm.cmask : nullptr; p.cvals[i] = comp ? mm.cvals : nullptr; p.coff[i] = comp ? mm.coff : nullptr;
   }
   for (int j = 0; j < 3; ++j) {
     const int f = g.axis[j];

@@ -119,6 +119,61 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
       slice[mi] = (const R *)p.logA[mi] + ((size_t)g * p.mcount[mi] + (size_t)o) * p.P_tile;
     }
     t3.load_slices(slice, p.nmem);
+  } else if (p.cmask[0] != nullptr) {
+    // Compressed slices (sparse per-agent models): per lane one 64-bit mask of the elements that are
+    // not the floor ln 1e-16, and those values packed lane after lane; the HBM traffic of the gather
+    // shrinks with the share of zeros in A.  This lane's values start at the slice's offset plus the
+    // other lanes' counts before it (a scan over the unit's lanes).
+    static_assert(NV * VE <= 64, "a lane's part of a slice must fit one mask");
+    constexpr int MAXC = 4;   // the packing layer compresses groups of up to four modalities
+    const size_t ob = ((size_t)agent * T + t) * p.M;
+    const R flr = __ldg((const R *)p.floor_log);
+    unsigned long long mk[MAXC];
+    const R *vp[MAXC];
+#pragma unroll
+    for (int mi = 0; mi < MAXC; ++mi) {
+      mk[mi] = 0ull;
+      vp[mi] = nullptr;
+      if (mi < p.nmem) {
+        const int o = clamp_flag(__ldg(p.obs + ob + p.modality[mi]), p.mcount[mi], p.status, BI_FLAG_OBS_RANGE);
+        const size_t sl = (size_t)g * p.mcount[mi] + (size_t)o;
+        mk[mi] = __ldg(p.cmask[mi] + sl * LPU + t3.u);
+        const int cnt = __popcll(mk[mi]);
+        int incl = cnt;
+#pragma unroll
+        for (int d = 1; d < LPU; d <<= 1) {
+          const int up = __shfl_up_sync(0xffffffffu, incl, d, LPU);
+          if (t3.u >= d) incl += up;
+        }
+        vp[mi] = (const R *)p.cvals[mi] + __ldg(p.coff[mi] + sl) + (incl - cnt);
+      }
+    }
+    constexpr int CH = NV % 12 == 0 ? 12 : (NV % 8 == 0 ? 8 : (NV % 6 == 0 ? 6 : NV));
+    for (int v0 = 0; v0 < NV; v0 += CH) {
+      R acc[CH][VE];
+#pragma unroll
+      for (int v = 0; v < CH; ++v)
+#pragma unroll
+        for (int i = 0; i < VE; ++i) acc[v][i] = (R)0;
+#pragma unroll
+      for (int mi = 0; mi < MAXC; ++mi) {
+        if (mi < p.nmem) {
+#pragma unroll
+          for (int v = 0; v < CH; ++v)
+#pragma unroll
+            for (int i = 0; i < VE; ++i) {
+              const bool bit = (mk[mi] & 1ull) != 0ull;
+              mk[mi] >>= 1;
+              acc[v][i] += bit ? __ldg(vp[mi]) : flr;
+              vp[mi] += bit ? 1 : 0;
+            }
+        }
+      }
+#pragma unroll
+      for (int v = 0; v < CH; ++v)
+#pragma unroll
+        for (int i = 0; i < VE; ++i) Lt[((v0 + v) * LPU + t3.u) * VE + i] = acc[v][i];
+    }
   } else {
     const size_t ob = ((size_t)agent * T + t) * p.M;
     constexpr int CH = NV % 12 == 0 ? 12 : (NV % 8 == 0 ? 8 : (NV % 6 == 0 ? 6 : NV));  // vectors in flight per pass

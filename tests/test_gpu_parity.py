@@ -858,3 +858,58 @@ def test_b_dependencies_call_forms_and_refusals():
         with pytest.raises(bi.BiError) as e:
             bi.Model(w.n, w.m, w.dep, w.U, 1, A, B, D, bdep=bad)
         assert e.value.code == code, (bad, e.value.code)
+
+
+# ---- compressed slices for sparse per-agent models ----
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+def test_compressed_slices_give_the_dense_result_bit_for_bit(algo):
+    """Per-agent models with 70 % zeros keep their slices as a mask per lane plus the non-floor values;
+    the window kernels gather from that form.  Same values, same order of additions: the beliefs equal
+    those of a handle made without compression (testing aid BI_TEST_NO_COMPRESS) exactly, and the oracle's
+    within tolerance.  A dense per-agent model is left uncompressed."""
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = make_config(4, N=24, T=7)
+    md = bi.model_from_workload(w)
+    dense_b, comp_b = md.slice_bytes()
+    assert 0 < comp_b < 0.6 * dense_b, (dense_b, comp_b)
+    md.set_compressed(True)
+    old = os.environ.get("BI_TEST_NO_COMPRESS")
+    os.environ["BI_TEST_NO_COMPRESS"] = "1"
+    try:
+        md_dense = bi.model_from_workload(w)
+    finally:
+        if old is None:
+            del os.environ["BI_TEST_NO_COMPRESS"]
+        else:
+            os.environ["BI_TEST_NO_COMPRESS"] = old
+    assert md_dense.slice_bytes() == (0, 0)
+    with pytest.raises(bi.BiError) as e:
+        md_dense.set_compressed(True)
+    assert e.value.code == -3
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    outs = []
+    for m_ in (md, md_dense):
+        lq = torch.empty((w.N, w.T, w.S), device="cuda")
+        am = torch.empty((w.N, w.T, w.F), dtype=torch.int32, device="cuda")
+        q = m_.run(algo, obs, act, w.K, logq_out=lq, argmax_out=am)
+        assert m_.last_kernel == f"tile3_{algo}_f64" and m_.status() == 0
+        outs.append((q.cpu().numpy(), lq.cpu().numpy(), am.cpu().numpy()))
+    for x, y in zip(*outs):
+        assert np.array_equal(x, y)
+    from parity import compare_conditioned
+    print(compare_conditioned(w, algo, *outs[0], oracle.run_workload(w, algo)))
+    # filtering on the same handle reads the dense form
+    qf = md.bi_filter(obs, act, w.K).cpu().numpy()
+    assert np.array_equal(qf, md_dense.bi_filter(obs, act, w.K).cpu().numpy())
+    md.close()
+    md_dense.close()
+    # a dense per-agent model of the same shape: nothing to gain, nothing made
+    rng = np.random.default_rng(9)
+    A, B, D = make_model(rng, w.n, w.m, w.dep, w.U, 6, sparsity=0.0, d_alpha=1.0)
+    md2 = bi.Model(w.n, w.m, w.dep, w.U, 6, [torch.from_numpy(a).cuda() for a in A],
+                   [torch.from_numpy(b).cuda() for b in B], [torch.from_numpy(d).cuda() for d in D])
+    assert md2.slice_bytes() == (0, 0)
+    md2.close()
