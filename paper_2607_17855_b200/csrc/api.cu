@@ -343,7 +343,8 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
   if (const char *e = getenv("BI_TEST_NO_COMPRESS")) md->test_no_compress = atoi(e) != 0;
   if (const char *e = getenv("BI_TEST_DROP_COPY")) md->test_drop_copy = atoi(e) > 0 ? atoi(e) : 0;   // testing aids,
   if (const char *e = getenv("BI_TEST_FAMILY")) {                                                  // read here only
-    md->test_family = !strcmp(e, "warp") ? BI_FAMILY_WARP : !strcmp(e, "generic") ? BI_FAMILY_GENERIC : BI_FAMILY_ANY;
+    md->test_family = !strcmp(e, "warp") ? BI_FAMILY_WARP : !strcmp(e, "generic") ? BI_FAMILY_GENERIC
+                      : !strcmp(e, "cta") ? BI_FAMILY_CTA : BI_FAMILY_ANY;
   }
   md->last_kernel = "";
   md->arith = arith;
@@ -495,6 +496,16 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
   if (!bdep_len && h.ngroups == 1 && F == 3 && h.grp[0].rank == 3)
     md->tile_sb = bi_tile3_shape(h.grp[0].dim[0], h.grp[0].dim[1], h.grp[0].dim[2]);
 
+  // at most one group over two factors, none over more: the pair filtering kernel's models
+  {
+    int r2 = 0, deep = 0;
+    for (int gi = 0; gi < h.ngroups; ++gi) {
+      if (h.grp[gi].rank == 2) ++r2;
+      if (h.grp[gi].rank > 2) ++deep;
+    }
+    md->pair_ok = !bdep_len && deep == 0 && r2 <= 1;
+  }
+
   // ---- allocate and pack
   rc = dev_alloc(md, (void **)&h.status, sizeof(uint32_t));
   if (rc == BI_OK && cudaMemsetAsync(h.status, 0, sizeof(uint32_t), stream) != cudaSuccess) rc = BI_ERR_CUDA;
@@ -535,6 +546,23 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
       if (arith == BI_ARITH_F64) bi_pack_A_kernel<double><<<(unsigned)blocks, threads, 0, stream>>>(p);
       else bi_pack_A_kernel<float><<<(unsigned)blocks, threads, 0, stream>>>(p);
       if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+      if (rc == BI_OK && md->pair_ok && g.rank == 2 && arith == BI_ARITH_F64) {
+        // the same slices with the two axes exchanged, for the pair filtering kernel's column copy
+        PackA t = p;
+        const size_t tcount = (size_t)G * mm.m * g.dim[1] * bi_pad4(g.dim[0]);
+        void *tdst = nullptr;
+        rc = dev_alloc(md, &tdst, tcount * esz);
+        if (rc != BI_OK) break;
+        t.dst = tdst;
+        t.total = (int64_t)tcount;
+        t.P_pad = g.dim[1] * bi_pad4(g.dim[0]);
+        t.dim[0] = g.dim[1]; t.dim[1] = g.dim[0];
+        t.sstride[0] = p.sstride[1]; t.sstride[1] = p.sstride[0];
+        t.npad = bi_pad4(g.dim[0]);
+        bi_pack_A_kernel<double><<<(unsigned)((t.total + threads - 1) / threads), threads, 0, stream>>>(t);
+        if (cudaGetLastError() != cudaSuccess) rc = BI_ERR_CUDA;
+        mm.logA_T = tdst;
+      }
       if (rc == BI_OK && md->tile_sb > 0) {
         PackTile q;
         memset(&q, 0, sizeof(q));
@@ -814,6 +842,7 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
   if (only == BI_FAMILY_ANY) {
     rc = bi_launch_tile3(c, mut);
     if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
+    if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_pair_filter(c, mut);
     if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
     // Filtering exposes one unit per agent, so a CTA per agent keeps more of the machine busy than
     // a warp per agent, and its staged slices and per-factor warps pay at every batch size measured
@@ -823,6 +852,7 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
     // shared memory.
     if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) rc = bi_launch_cta_filter(c, mut);
   }
+  if (only == BI_FAMILY_CTA && c.algo == BI_ALGO_FILTER) rc = bi_launch_cta_filter(c, mut);
   if (rc == BI_ERR_UNSUPPORTED && only != BI_FAMILY_GENERIC) rc = bi_launch_warp(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;

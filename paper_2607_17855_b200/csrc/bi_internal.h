@@ -10,7 +10,7 @@
 #define BI_MAX_GROUPS BI_MAX_M
 
 enum { BI_ALGO_FILTER = 0, BI_ALGO_VMP = 1, BI_ALGO_MMP = 2 };
-enum { BI_FAMILY_ANY = 0, BI_FAMILY_WARP = 1, BI_FAMILY_GENERIC = 2 };
+enum { BI_FAMILY_ANY = 0, BI_FAMILY_WARP = 1, BI_FAMILY_GENERIC = 2, BI_FAMILY_CTA = 3 };
 
 static __host__ __device__ inline int bi_pad4(int x) { return (x + 3) & ~3; }
 // Row stride in shared memory for rows of npad elements (npad a multiple of 4, elements of esize
@@ -59,6 +59,7 @@ struct BiMember {
   // of such a slice are the floor ln 1e-16 (a zero of A), so a slice is stored as one 64-bit mask per
   // lane of a unit (bit i set: the lane's i-th element is not the floor) plus the other values, packed
   // lane after lane.  cmask: [G * m][LPU]; coff: [G * m + 1] element offsets into cvals.
+  const void *logA_T;     // groups over two factors of pair models: the slices transposed, [G][m][dim1][pad4(dim0)], or NULL
   const unsigned long long *cmask;
   const void *cvals;
   const long long *coff;
@@ -100,7 +101,7 @@ struct alignas(16) BiDev {
 struct bi_model {
   BiDev h;          // host copy (device pointers inside)
   BiDev *d;         // device copy
-  void *allocs[24 + 2 * BI_MAX_M + 10 * BI_MAX_F];  // status, descriptor, pre-summed table, 2 per modality, 7 per factor
+  void *allocs[24 + 3 * BI_MAX_M + 10 * BI_MAX_F];  // status, descriptor, pre-summed table, 2 per modality, 7 per factor
   int nalloc;
   int arith;        // BI_ARITH_F64 or BI_ARITH_F32
   int device;
@@ -108,6 +109,7 @@ struct bi_model {
   int max_smem_optin;
   int tile_sb;      // > 0: a register-tile shape matches; lanes along b per (agent, step)
   int tile_P;       // elements per lane-interleaved slice
+  int pair_ok;      // at most one group over two factors and none over more: the pair filtering kernel applies
   const void *tile_floor;   // device scalar: ln 1e-16 in the arithmetic type, as the pack kernels compute it
   long long slice_bytes_dense, slice_bytes_compressed;   // per-agent tile models: bytes of the two forms (0: none)
   int test_no_compress;     // testing aid (BI_TEST_NO_COMPRESS, read when the handle is made)
@@ -133,7 +135,7 @@ struct bi_model {
   void *carry;      // last belief of the latest filtering call, [carry_N][S] in the arithmetic type, or NULL
   size_t carry_bytes;
   int carry_N;      // agents of that call (0: none yet)
-  // Testing aid, read from the environment once, when the handle is made (BI_TEST_FAMILY = "warp" or
+  // Testing aid, read from the environment once, when the handle is made (BI_TEST_FAMILY = "cta", "warp" or
   // "generic"): calls skip the kernel families ahead of the named one, so that the general kernels can
   // be checked on inputs small enough for the oracle.  0 = normal dispatch.
   int test_family;
@@ -169,6 +171,7 @@ struct BiCall {
 int bi_launch_generic(const BiCall &c, bi_model *mut);
 int bi_launch_warp(const BiCall &c, bi_model *mut);
 int bi_launch_cta_filter(const BiCall &c, bi_model *mut);   // filtering only; slices staged per step
+int bi_launch_pair_filter(const BiCall &c, bi_model *mut);  // filtering only; models coupled in at most one pair of factors
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
 int bi_launch_tile3_window(const BiCall &c, bi_model *mut);
 int bi_launch_batch(const BiCall &c, bi_model *mut);

@@ -16,7 +16,7 @@ ALGOS = ["filter", "vmp", "mmp"]
 
 @contextlib.contextmanager
 def family_forced(name):
-    """The library's testing aid BI_TEST_FAMILY ("warp" or "generic"), read when a handle is made: its
+    """The library's testing aid BI_TEST_FAMILY ("cta", "warp" or "generic"), read when a handle is made: its
     calls skip the kernel families ahead of the named one, so that the general kernels can be checked
     on oracle-sized inputs that would otherwise go to a specialised kernel."""
     old = os.environ.get("BI_TEST_FAMILY")
@@ -622,6 +622,9 @@ def test_cta_filter_kernel_shapes(case):
                                [0, 3], [6], [5, 1], [4, 7], [2, 0, 6]], [2, 1, 2, 1, 3, 1, 2, 2], N=5, T=4, K=5),
     }[case]
     res = check_workload(w, "filter")
+    assert res["kernel"] == ("pair_filter_f64" if case == "rank1_only" else "cta_filter_f64"), res
+    with family_forced("cta"):
+        res = check_workload(w, "filter")
     assert res["kernel"] == "cta_filter_f64", res
 
 
@@ -632,6 +635,9 @@ def test_filter_kernels_on_random_structures_with_ragged_sizes(j):
     rng = np.random.default_rng(1000 + j)
     w = make_sweep_config(j, N=int(rng.integers(1, 14)), T=int(rng.integers(1, 9)), K=int(rng.integers(1, 7)))
     res = check_workload(w, "filter", conditioned=True)
+    assert res["kernel"] in ("cta_filter_f64", "pair_filter_f64"), res
+    with family_forced("cta"):
+        res = check_workload(w, "filter", conditioned=True)
     assert res["kernel"] == "cta_filter_f64", res
     with warp_filter_forced():
         res = check_workload(w, "filter", conditioned=True)
@@ -913,3 +919,55 @@ def test_compressed_slices_give_the_dense_result_bit_for_bit(algo):
                    [torch.from_numpy(b).cuda() for b in B], [torch.from_numpy(d).cuda() for d in D])
     assert md2.slice_bytes() == (0, 0)
     md2.close()
+
+
+# ---- the pair filtering kernel (models coupled in at most one pair of factors) ----
+
+PAIR_CASES = {
+    "config1": lambda: make_config(1),
+    "lanes4_many_agents": lambda: _custom(91, [4, 3], [5, 4, 3], [[0, 1], [1, 0], [1]], [2, 2], N=37, T=6, K=7),
+    "lanes8_extra_factors": lambda: _custom(92, [6, 8, 3, 1], [4, 3, 2, 5], [[1, 0], [2], [0], [3]], [2, 1, 3, 1], N=11, T=5, K=6),
+    "lanes16_sparse": lambda: _custom(93, [9, 13], [6, 3], [[0, 1], [0, 1]], [3, 2], N=5, T=7, K=8, sparsity=0.7),
+    "lanes32": lambda: _custom(94, [32, 31], [3, 4, 2], [[1, 0], [0], [1]], [2, 2], N=3, T=4, K=5),
+    "no_pair": lambda: _custom(95, [7, 5, 12], [4, 3, 5, 2], [[0], [2], [2], [0]], [2, 3, 1], N=9, T=6, K=4),
+    "per_agent": lambda: _custom(96, [5, 7], [4, 3], [[0, 1], [1]], [2, 2], N=6, T=5, K=6, G=6, sparsity=0.5),
+    "one_agent_one_step": lambda: _custom(97, [5, 3], [4], [[0, 1]], [1, 1], N=1, T=1, K=1),
+}
+
+
+@pytest.mark.parametrize("case", sorted(PAIR_CASES))
+def test_pair_filter_kernel(case):
+    w = PAIR_CASES[case]()
+    res = check_workload(w, "filter", conditioned=True)
+    print(case, res)
+    assert res["kernel"] == "pair_filter_f64", res
+
+
+@pytest.mark.parametrize("j", [8, 15, 19, 0, 13, 90, 127])
+def test_pair_filter_kernel_on_sweep_structures(j):
+    w = make_sweep_config(j, N=21, T=7)
+    res = check_workload(w, "filter", conditioned=True)
+    assert res["kernel"] == "pair_filter_f64", res
+
+
+def test_pair_filter_continued_calls():
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = _custom(98, [6, 8, 3], [4, 3, 2], [[1, 0], [2], [0]], [2, 1, 3], N=11, T=9, K=6)
+    md = bi.model_from_workload(w)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    whole = md.bi_filter(obs, act, w.K).cpu().numpy()
+    assert md.last_kernel == "pair_filter_f64"
+    q, names = _blockwise(md, w, [0, 2, 3, 7, w.T], w.K)
+    assert names == {"pair_filter_f64"} and np.array_equal(q, whole)
+    head = md.bi_filter(obs[:, :4].contiguous(), act[:, :3].contiguous(), w.K)
+    tail = md.bi_filter_from(obs[:, 4:].contiguous(), act[:, 4:].contiguous(), head[:, -1].contiguous(),
+                             act[:, 3].contiguous(), w.K).cpu().numpy()
+    ref = oracle.run_workload(w, "filter")[0]
+    assert np.abs(whole - ref).max() <= 1e-5 and np.abs(tail - ref[:, 4:]).max() <= 1e-5
+    # a damped call is not this kernel's
+    md.set_damping(0.5)
+    md.bi_filter(obs, act, w.K)
+    assert md.last_kernel == "cta_filter_f64" and md.status() == 0
+    md.close()

