@@ -45,9 +45,11 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # 74.4
 # same kernels (bytes; the captures and how they scale to these sizes are written up beside the code,
 # in the profiler summaries).  A record of those captures: the run itself does not measure DRAM traffic.
 NCU_DRAM_BYTES_PER_CALL = {
-    "tile3_filter_f64": 5.0e6,     # config 2, full size, one launch
-    "batch_vmp_f64": None,         # config 3 (filled from the capture: see NCU_NOTES)
-    "tile3_mmp_f64": None,         # config 4
+    "tile3_filter_f64": 8.05e6,    # config 2, full size, one launch (read 8.05 MB, written 3.3 KB: outputs stay in L2)
+    "batch_vmp_f64": 6.8e8,        # config 3: 16 x (9.6 + 2.3 MB contraction, 30.5 MB update), each launch with the
+                                   # cold L2 the profiler gives it; back to back the partial messages stay in L2
+    "tile3_mmp_f64": 7.3e8,        # config 4: (101.8 + 3.4) MB captured on 296 agents x 2048 / 296 (per-agent models:
+                                   # traffic grows in proportion to the agents)
 }
 
 
