@@ -295,6 +295,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--arith", default="f64", choices=["f64", "f32"])
+    ap.add_argument("--e2e-blocks", type=int, default=E2E_CHUNKS,
+                    help="the end-to-end run filters the trajectory in this many consecutive blocks of steps")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads and the CPU baseline")
     ap.add_argument("--case", default=None, help="CONFIG[:ALGO], e.g. 4:mmp: run that one workload and print its time")
     ap.add_argument("--agents", type=int, default=None, help="with --case: agents N")
@@ -350,7 +352,7 @@ def main():
     # full-precision record of the previous block's last belief: bit for bit the single call's result),
     # so a block's beliefs travel to the host while the next block runs.
     md, q = head["model"], head["q"]
-    nchunk = E2E_CHUNKS if w.T % E2E_CHUNKS == 0 else 1
+    nchunk = args.e2e_blocks if args.e2e_blocks >= 1 and w.T % args.e2e_blocks == 0 else 1
     tc = w.T // nchunk
     copy_out, copy_in = torch.cuda.Stream(), torch.cuda.Stream()
     # host inputs block by block, packed into two pinned buffers (the first block; the rest) so that each

@@ -344,7 +344,7 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
   if (const char *e = getenv("BI_TEST_DROP_COPY")) md->test_drop_copy = atoi(e) > 0 ? atoi(e) : 0;   // testing aids,
   if (const char *e = getenv("BI_TEST_FAMILY")) {                                                  // read here only
     md->test_family = !strcmp(e, "warp") ? BI_FAMILY_WARP : !strcmp(e, "generic") ? BI_FAMILY_GENERIC
-                      : !strcmp(e, "cta") ? BI_FAMILY_CTA : BI_FAMILY_ANY;
+                      : !strcmp(e, "cta") ? BI_FAMILY_CTA : !strcmp(e, "batch") ? BI_FAMILY_BATCH : BI_FAMILY_ANY;
   }
   md->last_kernel = "";
   md->arith = arith;
@@ -843,6 +843,7 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
     rc = bi_launch_tile3(c, mut);
     if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_tile3_window(c, mut);
     if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_pair_filter(c, mut);
+    if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_pair_window(c, mut);
     if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_batch(c, mut);
     // Filtering exposes one unit per agent, so a CTA per agent keeps more of the machine busy than
     // a warp per agent, and its staged slices and per-factor warps pay at every batch size measured
@@ -853,6 +854,10 @@ int bi_dispatch(const BiCall &c, bi_model *mut) {
     if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) rc = bi_launch_cta_filter(c, mut);
   }
   if (only == BI_FAMILY_CTA && c.algo == BI_ALGO_FILTER) rc = bi_launch_cta_filter(c, mut);
+  if (only == BI_FAMILY_BATCH) {   // the batched window kernels and what follows them
+    rc = bi_launch_batch(c, mut);
+    if (rc == BI_ERR_UNSUPPORTED && c.algo == BI_ALGO_FILTER) rc = bi_launch_cta_filter(c, mut);
+  }
   if (rc == BI_ERR_UNSUPPORTED && only != BI_FAMILY_GENERIC) rc = bi_launch_warp(c, mut);
   if (rc == BI_ERR_UNSUPPORTED) rc = bi_launch_generic(c, mut);
   return rc;

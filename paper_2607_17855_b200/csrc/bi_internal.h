@@ -10,7 +10,7 @@
 #define BI_MAX_GROUPS BI_MAX_M
 
 enum { BI_ALGO_FILTER = 0, BI_ALGO_VMP = 1, BI_ALGO_MMP = 2 };
-enum { BI_FAMILY_ANY = 0, BI_FAMILY_WARP = 1, BI_FAMILY_GENERIC = 2, BI_FAMILY_CTA = 3 };
+enum { BI_FAMILY_ANY = 0, BI_FAMILY_WARP = 1, BI_FAMILY_GENERIC = 2, BI_FAMILY_CTA = 3, BI_FAMILY_BATCH = 4 };
 
 static __host__ __device__ inline int bi_pad4(int x) { return (x + 3) & ~3; }
 // Row stride in shared memory for rows of npad elements (npad a multiple of 4, elements of esize
@@ -135,8 +135,8 @@ struct bi_model {
   void *carry;      // last belief of the latest filtering call, [carry_N][S] in the arithmetic type, or NULL
   size_t carry_bytes;
   int carry_N;      // agents of that call (0: none yet)
-  // Testing aid, read from the environment once, when the handle is made (BI_TEST_FAMILY = "cta", "warp" or
-  // "generic"): calls skip the kernel families ahead of the named one, so that the general kernels can
+  // Testing aid, read from the environment once, when the handle is made (BI_TEST_FAMILY = "batch", "cta", "warp"
+  // or "generic"): calls skip the kernel families ahead of the named one, so that the general kernels can
   // be checked on inputs small enough for the oracle.  0 = normal dispatch.
   int test_family;
   // Testing aid (BI_TEST_DROP_COPY = n, read when the handle is made): the next n batched window calls
@@ -172,6 +172,7 @@ int bi_launch_generic(const BiCall &c, bi_model *mut);
 int bi_launch_warp(const BiCall &c, bi_model *mut);
 int bi_launch_cta_filter(const BiCall &c, bi_model *mut);   // filtering only; slices staged per step
 int bi_launch_pair_filter(const BiCall &c, bi_model *mut);  // filtering only; models coupled in at most one pair of factors
+int bi_launch_pair_window(const BiCall &c, bi_model *mut);  // window calls on the same models; a CTA per agent
 int bi_launch_tile3(const BiCall &c, bi_model *mut);
 int bi_launch_tile3_window(const BiCall &c, bi_model *mut);
 int bi_launch_batch(const BiCall &c, bi_model *mut);

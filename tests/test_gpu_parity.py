@@ -16,7 +16,7 @@ ALGOS = ["filter", "vmp", "mmp"]
 
 @contextlib.contextmanager
 def family_forced(name):
-    """The library's testing aid BI_TEST_FAMILY ("cta", "warp" or "generic"), read when a handle is made: its
+    """The library's testing aid BI_TEST_FAMILY ("batch", "cta", "warp" or "generic"), read when a handle is made: its
     calls skip the kernel families ahead of the named one, so that the general kernels can be checked
     on oracle-sized inputs that would otherwise go to a specialised kernel."""
     old = os.environ.get("BI_TEST_FAMILY")
@@ -269,8 +269,11 @@ def test_batched_any_shape(algo):
 def test_batched_single_factor_modalities_only(algo):
     # no contraction at all: the observed slices are the messages
     w = _custom(46, [5, 9], [4, 3, 6], [[0], [1], [0]], [2, 3], N=150, T=14, K=5)
-    res = check_workload(w, algo, agents=range(0, 150, 4))
+    with family_forced("batch"):   # (by itself the dispatcher gives such a model to the pair window kernel)
+        res = check_workload(w, algo, agents=range(0, 150, 4))
     assert res["kernel"] == f"batch_{algo}_f64", res
+    res = check_workload(w, algo, agents=range(0, 150, 4))
+    assert res["kernel"] == f"pair_{algo}_f64", res
 
 
 # ---- filtering continued from a known belief (bi_filter_from)
@@ -342,7 +345,7 @@ def _random_beliefs(w, seed):
 
 
 @pytest.mark.parametrize("algo", ["vmp", "mmp"])
-@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "per_agent"])
+@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "per_agent", "pair"])
 def test_warm_started_windows(case, algo):
     import torch
     import oracle
@@ -353,6 +356,8 @@ def test_warm_started_windows(case, algo):
         "batch": (make_config(3, N=128, T=16, K=3), f"batch_{algo}_f64"),
         "warp": (make_config(3, N=10, T=7, K=3), f"warp_{algo}_f64"),
         "per_agent": (_custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=3, G=5), None),
+        "pair": (_custom(92, [6, 8, 3, 1], [4, 3, 2, 5], [[1, 0], [2], [0], [3]], [2, 1, 3, 1], N=11, T=5, K=3),
+                 f"pair_{algo}_f64"),
     }[case]
     q_init = _random_beliefs(w, 77)
     md = bi.model_from_workload(w)
@@ -455,7 +460,7 @@ def test_soft_observations_single_step_and_empty_batch():
 # ---- window algorithms continued from a belief (bi_vmp_from / bi_mmp_from)
 
 @pytest.mark.parametrize("algo", ["vmp", "mmp"])
-@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "per_agent"])
+@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "per_agent", "pair"])
 def test_continued_windows(case, algo):
     import torch
     import oracle
@@ -466,6 +471,8 @@ def test_continued_windows(case, algo):
         "batch": (make_config(3, N=128, T=16, K=4), f"batch_{algo}_f64"),
         "warp": (make_config(3, N=10, T=7, K=4), f"warp_{algo}_f64"),
         "per_agent": (_custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=4, G=5), None),
+        "pair": (_custom(92, [6, 8, 3, 1], [4, 3, 2, 5], [[1, 0], [2], [0], [3]], [2, 1, 3, 1], N=11, T=5, K=4),
+                 f"pair_{algo}_f64"),
     }[case]
     rng = np.random.default_rng(91)
     q_prev = np.concatenate([rng.dirichlet(np.full(int(nf), 1.5), size=w.N) for nf in w.n], axis=1).astype(np.float32)
@@ -948,6 +955,41 @@ def test_pair_filter_kernel_on_sweep_structures(j):
     w = make_sweep_config(j, N=21, T=7)
     res = check_workload(w, "filter", conditioned=True)
     assert res["kernel"] == "pair_filter_f64", res
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+@pytest.mark.parametrize("case", sorted(PAIR_CASES))
+def test_pair_window_kernel(case, algo):
+    w = PAIR_CASES[case]()
+    res = check_workload(w, algo, conditioned=True)
+    print(case, algo, res)
+    assert res["kernel"] == f"pair_{algo}_f64", res
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+@pytest.mark.parametrize("j", [8, 15, 19, 0, 13, 90, 127])
+def test_pair_window_kernel_on_sweep_structures(j, algo):
+    w = make_sweep_config(j, N=21, T=7)
+    res = check_workload(w, algo, conditioned=True)
+    assert res["kernel"] == f"pair_{algo}_f64", res
+
+
+def test_pair_window_kernel_limits():
+    """A window whose steps do not fit one CTA goes to another kernel family; so does a damped call."""
+    import torch
+    import paper_2607_17855_b200 as bi
+    w = _custom(99, [32, 31], [3, 4], [[1, 0], [0]], [2, 2], N=40, T=20, K=3)   # 20 steps x 32 lanes > 512 threads
+    res = check_workload(w, "vmp", agents=range(0, 40, 5))
+    assert not res["kernel"].startswith("pair_"), res
+    w = _custom(98, [6, 8, 3], [4, 3, 2], [[1, 0], [2], [0]], [2, 1, 3], N=11, T=9, K=6)
+    md = bi.model_from_workload(w)
+    obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
+    md.bi_vmp(obs, act, w.K)
+    assert md.last_kernel == "pair_vmp_f64"
+    md.set_damping(0.5)
+    md.bi_vmp(obs, act, w.K)
+    assert not md.last_kernel.startswith("pair_") and md.status() == 0
+    md.close()
 
 
 def test_pair_filter_continued_calls():
