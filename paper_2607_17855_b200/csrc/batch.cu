@@ -21,6 +21,8 @@
 #include <algorithm>
 #include <cstring>
 
+#include <type_traits>
+
 #include "bi_internal.h"
 #include "tile3.cuh"
 
@@ -476,16 +478,30 @@ struct UpdateArgs {
   uint32_t r1mask[BI_MAX_F];  // descriptor members (modalities) that depend on factor f alone
 };
 
+// Both transition messages' dot products at once: dp = sum_r Mp[r][s] qp[r] and df = sum_r Mf[r][s] qf[r],
+// r < n, the matrices read [summation index][own state] from global memory (L1), the beliefs as pairs
+// from shared memory (their padding entries are zero); pointers advance by additions only.
 template <typename R>
-__device__ __forceinline__ R col_dot_g(const R *__restrict__ col, int npad, const R *__restrict__ q, int n) {
-  R s0 = (R)0, s1 = (R)0;
+__device__ __forceinline__ void edge_dots_g(const R *__restrict__ mp, const R *__restrict__ mf, int npad,
+                                            const R *qp, const R *qf, int n, R &dp, R &df) {
+  using V2 = typename std::conditional<sizeof(R) == 8, double2, float2>::type;
+  R p0 = (R)0, p1 = (R)0, f0 = (R)0, f1 = (R)0;
+  const int st2 = 2 * npad;
   int r = 0;
+#pragma unroll 2
   for (; r + 1 < n; r += 2) {
-    s0 = fma(__ldg(col + (size_t)r * npad), q[r], s0);
-    s1 = fma(__ldg(col + (size_t)(r + 1) * npad), q[r + 1], s1);
+    const V2 x = *reinterpret_cast<const V2 *>(qp + r), y = *reinterpret_cast<const V2 *>(qf + r);
+    p0 = fma(__ldg(mp), x.x, p0); p1 = fma(__ldg(mp + npad), x.y, p1);
+    f0 = fma(__ldg(mf), y.x, f0); f1 = fma(__ldg(mf + npad), y.y, f1);
+    mp += st2;
+    mf += st2;
   }
-  if (r < n) s0 = fma(__ldg(col + (size_t)r * npad), q[r], s0);
-  return s0 + s1;
+  if (r < n) {
+    p0 = fma(__ldg(mp), qp[r], p0);
+    f0 = fma(__ldg(mf), qf[r], f0);
+  }
+  dp = p0 + p1;
+  df = f0 + f1;
 }
 
 // LW lanes per unit (the smallest power of two that holds the largest factor),
@@ -511,10 +527,18 @@ __device__ __forceinline__ R lane_group_max(R v) {
   return v;
 }
 
+// A first pass gathers, with loads that do not depend on one another (one position of the unit's
+// state vector per lane and trip), everything that comes from L2: the sum of the partial messages,
+// the single-factor slices, the first step's log-prior, and the two neighbouring steps' beliefs, into
+// the unit's part of shared memory.  The per-factor pass then reads shared memory and the transition
+// matrices (L1) only.  (With the L2 reads inside the per-factor loop every factor paid several
+// dependent round trips: 35 us per launch on 20 480 units, `long_scoreboard` 8.9 stall cycles per issue.)
 template <typename R, int ALGO, int LW>
 __global__ void __launch_bounds__(128)
 bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs A) {
   __shared__ FactorInfo fi[BI_MAX_F];
+  __shared__ unsigned char pfac[BI_MAX_F * 32];   // factor of each padded state position
+  extern __shared__ __align__(16) unsigned char upd_smem[];
   const BiDev &md = *mdp;
   constexpr int UPB = 128 / LW;   // units per CTA
   const int F = md.F, Sp = md.Sp, S = md.S, M = md.M, T = A.T, NU = P.NU;
@@ -524,6 +548,11 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
     x.n = md.n[f]; x.np = md.npad[f]; x.op = md.offp[f]; x.off = md.off[f]; x.U = md.U[f];
     x.fmask = A.fmask[f]; x.r1mask = A.r1mask[f]; x.pad_ = 0;
     fi[f] = x;
+  }
+  for (int p = threadIdx.x; p < Sp; p += blockDim.x) {
+    int f = 0;
+    while (f + 1 < F && p >= md.offp[f + 1]) ++f;
+    pfac[p] = (unsigned char)f;
   }
   __syncthreads();
   bi_grid_wait();   // the contraction's messages (and, for the beliefs, everything before it)
@@ -539,37 +568,50 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
   const int32_t *ob = A.obs + (size_t)unit * M;
   // acp[f]: action into step t (t > 0); acp[F + f]: action out of it (t + 1 < T)
   const int32_t *acp = A.act + ((ptrdiff_t)a * (T - 1) + (t - 1)) * F;
+  R *base = reinterpret_cast<R *>(upd_smem) + (size_t)sub * 3 * Sp;   // [Sp] logit constants, [Sp] q(t-1), [Sp] q(t+1)
+  R *qprev = base + Sp, *qnext = base + 2 * Sp;
+  for (int p = s; p < Sp; p += LW) {
+    const int f = pfac[p];
+    const FactorInfo I = fi[f];
+    const int sl = p - I.op;
+    R x = (R)0;
+    if (sl < I.n) {
+      const R *ep = (const R *)P.ellp + (size_t)unit * Sp + p;   // member j's entry: NU * Sp elements further per j
+      const size_t mstride = (size_t)NU * Sp;
+      for (uint32_t mk = I.fmask; mk; mk &= mk - 1) x += ep[(__ffs(mk) - 1) * mstride];
+      for (uint32_t mk = I.r1mask; mk; mk &= mk - 1) {   // single-factor modalities: the slice is the message
+        const BiMember &mm = md.mem[__ffs(mk) - 1];
+        const int o = clamp_flag(ob[mm.modality], mm.m, md.status, BI_FLAG_OBS_RANGE);
+        x += __ldg((const R *)mm.logA + (size_t)g * mm.gstride + (size_t)o * mm.P_pad + sl);
+      }
+      if (t == 0)
+        x += A.lnprior ? ((const R *)A.lnprior)[(size_t)a * S + I.off + sl]
+                       : ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + sl];
+    }
+    base[p] = x;
+    qprev[p] = t > 0 ? qc[(size_t)(unit - 1) * Sp + p] : (R)0;
+    qnext[p] = t + 1 < T ? qc[(size_t)(unit + 1) * Sp + p] : (R)0;
+  }
+  __syncwarp();
   for (int f = 0; f < F; ++f) {
     const FactorInfo I = fi[f];
     const int n = I.n, np = I.np, op = I.op;
     R x = -bi_inf<R>();
     if (s < n) {
-      x = (R)0;
-      for (uint32_t mk = I.fmask; mk; mk &= mk - 1) {
-        const int j = __ffs(mk) - 1;
-        x += ((const R *)P.ellp)[((size_t)j * NU + unit) * Sp + op + s];
+      x = base[op + s];
+      // both edges are evaluated (a window's end reads zeros and discards the result)
+      const int up = t > 0 ? clamp_flag(acp[f], I.U, md.status, BI_FLAG_ACT_RANGE) : 0;
+      const int uf = t + 1 < T ? clamp_flag(acp[F + f], I.U, md.status, BI_FLAG_ACT_RANGE) : 0;
+      const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);   // [previous][next]
+      const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);   // [next][previous]
+      const size_t mo = (size_t)g * md.Bstride[f] + s;
+      R dp, df;
+      edge_dots_g<R>(M0 + mo + up * n * np, M1 + mo + uf * n * np, np, qprev + op, qnext + op, n, dp, df);
+      if (ALGO == BI_ALGO_MMP) {
+        dp = (R)0.5 * bi_log_inline(bi_max(dp, (R)BI_EPS));
+        df = (R)0.5 * bi_log_inline(bi_max(df, (R)BI_EPS));
       }
-      for (uint32_t mk = I.r1mask; mk; mk &= mk - 1) {   // single-factor modalities: the slice is the message
-        const BiMember &mm = md.mem[__ffs(mk) - 1];
-        const int o = clamp_flag(ob[mm.modality], mm.m, md.status, BI_FLAG_OBS_RANGE);
-        x += __ldg((const R *)mm.logA + (size_t)g * mm.gstride + (size_t)o * mm.P_pad + s);
-      }
-      if (t == 0) {
-        x += A.lnprior ? ((const R *)A.lnprior)[(size_t)a * S + I.off + s] : ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
-      } else {
-        const int u = clamp_flag(acp[f], I.U, md.status, BI_FLAG_ACT_RANGE);
-        const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);   // [previous][next]
-        const R v = col_dot_g<R>(M0 + (size_t)g * md.Bstride[f] + (size_t)u * n * np + s, np,
-                                 qc + (size_t)(unit - 1) * Sp + op, n);
-        x += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
-      }
-      if (t + 1 < T) {
-        const int u = clamp_flag(acp[F + f], I.U, md.status, BI_FLAG_ACT_RANGE);
-        const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);   // [next][previous]
-        const R v = col_dot_g<R>(M1 + (size_t)g * md.Bstride[f] + (size_t)u * n * np + s, np,
-                                 qc + (size_t)(unit + 1) * Sp + op, n);
-        x += ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
-      }
+      x += (t > 0 ? dp : (R)0) + (t + 1 < T ? df : (R)0);
     }
     if (A.xprev) {
       // damped step on the logits; the first one starts from ln q of the starting belief (uniform: a
@@ -800,7 +842,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     }
     cfg.gridDim = dim3((unsigned)((NU + upb - 1) / upb));
     cfg.blockDim = dim3(128);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = (size_t)upb * 3 * h.Sp * sizeof(R);
     if (cudaLaunchKernelEx(&cfg, update, (const BiDev *)md->d, P, A) != cudaSuccess) return BI_ERR_CUDA;
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
