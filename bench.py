@@ -34,7 +34,9 @@ sys.path.insert(0, ROOT)
 METRIC = "belief_updates_per_sec"
 UNIT = "updates/s"
 HEADLINE = 2  # configuration the metric is quoted on
-E2E_CHUNKS = 5  # the end-to-end run filters the trajectory in this many consecutive blocks of steps
+# the end-to-end run filters the trajectory in consecutive blocks of steps of these lengths (short last
+# blocks: the last block's beliefs are the only ones whose way to the host nothing overlaps)
+E2E_BLOCKS = "8,14,14,9,5"
 
 # Nominal ALU peaks derived from the unit counts: 148 SMs x lanes x 2 flops x 1.965 GHz.
 FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12   # 37.2
@@ -295,8 +297,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--arith", default="f64", choices=["f64", "f32"])
-    ap.add_argument("--e2e-blocks", type=int, default=E2E_CHUNKS,
-                    help="the end-to-end run filters the trajectory in this many consecutive blocks of steps")
+    ap.add_argument("--e2e-blocks", default=E2E_BLOCKS,
+                    help="the end-to-end run filters the trajectory in consecutive blocks of steps: their number, "
+                         "or their lengths as a comma-separated list")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads and the CPU baseline")
     ap.add_argument("--case", default=None, help="CONFIG[:ALGO], e.g. 4:mmp: run that one workload and print its time")
     ap.add_argument("--agents", type=int, default=None, help="with --case: agents N")
@@ -348,52 +351,57 @@ def main():
     value = aggregate_throughput(w.updates, world, sec)
 
     # ---- end to end: pinned host inputs -> device -> filtering -> host beliefs.  The trajectory is
-    # run as E2E_CHUNKS consecutive blocks of steps (bi_filter, then bi_filter_continue from the handle's
+    # run as consecutive blocks of steps (bi_filter, then bi_filter_continue from the handle's
     # full-precision record of the previous block's last belief: bit for bit the single call's result),
     # so a block's beliefs travel to the host while the next block runs.
     md, q = head["model"], head["q"]
-    nchunk = args.e2e_blocks if args.e2e_blocks >= 1 and w.T % args.e2e_blocks == 0 else 1
-    tc = w.T // nchunk
+    spec = str(args.e2e_blocks)
+    if "," in spec:
+        lens = [int(x) for x in spec.split(",")]
+    else:
+        nb = max(1, int(spec))
+        lens = [w.T // nb] * nb if w.T % nb == 0 else [w.T]
+    if sum(lens) != w.T or min(lens) < 1:
+        lens = [w.T]
+    nchunk = len(lens)
+    starts = [sum(lens[:i]) for i in range(nchunk)]
     copy_out, copy_in = torch.cuda.Stream(), torch.cuda.Stream()
-    # host inputs block by block, packed into two pinned buffers (the first block; the rest) so that each
-    # reaches the device in one copy: the second one while the first block is being filtered
+    # host inputs block by block, each block packed into one pinned buffer so that it reaches the device
+    # in one copy; the copies are issued in order on one stream (side by side they would share the link and
+    # the first block would wait for all of them) and a block's call waits for its own copy only
     parts = []
     for i in range(nchunk):
-        t0 = i * tc
+        t0, tc = starts[i], lens[i]
         parts.append([np.ascontiguousarray(w.obs[:, t0:t0 + tc]), np.ascontiguousarray(w.act[:, t0:t0 + tc - 1]),
                       np.ascontiguousarray(w.act[:, t0 - 1]) if i else np.empty((w.N, 0), np.int32)])
-    def pack(blocks):
-        flat = np.concatenate([x.reshape(-1) for blk in blocks for x in blk]) if blocks else np.empty(0, np.int32)
-        return torch.from_numpy(flat.astype(np.int32)).pin_memory()
-    h_first, h_rest = pack(parts[:1]), pack(parts[1:])
-    d_first = torch.empty(h_first.shape, dtype=torch.int32, device="cuda")
-    d_rest = torch.empty(h_rest.shape, dtype=torch.int32, device="cuda")
+    h_in = [torch.from_numpy(np.concatenate([x.reshape(-1) for x in blk]).astype(np.int32)).pin_memory()
+            for blk in parts]
+    d_buf = [torch.empty(h.shape, dtype=torch.int32, device="cuda") for h in h_in]
     d_in = []
-    for i, blk in enumerate(parts):
-        buf, pos, views = (d_first, 0, []) if i == 0 else (d_rest, d_in[-1][3] if i > 1 else 0, [])
+    for buf, blk in zip(d_buf, parts):
+        pos, views = 0, []
         for x in blk:
             views.append(buf[pos:pos + x.size].view(x.shape))
             pos += x.size
-        d_in.append((views[0], views[1], views[2], pos))
-    d_q = [torch.empty((w.N, tc, w.S), dtype=torch.float32, device="cuda") for _ in range(nchunk)]
-    h_q = [torch.empty((w.N, tc, w.S), dtype=torch.float32).pin_memory() for _ in range(nchunk)]
+        d_in.append(views)
+    d_q = [torch.empty((w.N, tc, w.S), dtype=torch.float32, device="cuda") for tc in lens]
+    h_q = [torch.empty((w.N, tc, w.S), dtype=torch.float32).pin_memory() for tc in lens]
     done = [torch.cuda.Event() for _ in range(nchunk)]
-    arrived = torch.cuda.Event()
+    arrived = [torch.cuda.Event() for _ in range(nchunk)]
 
     def e2e_step():
         cur = torch.cuda.current_stream()
         copy_in.wait_stream(cur)
-        d_first.copy_(h_first, non_blocking=True)
         with torch.cuda.stream(copy_in):
-            d_rest.copy_(h_rest, non_blocking=True)
-            arrived.record(copy_in)
+            for i in range(nchunk):
+                d_buf[i].copy_(h_in[i], non_blocking=True)
+                arrived[i].record(copy_in)
         for i in range(nchunk):
-            obs_i, act_i, actp_i, _ = d_in[i]
+            obs_i, act_i, actp_i = d_in[i]
+            cur.wait_event(arrived[i])
             if i == 0:
                 md.bi_filter(obs_i, act_i, w.K, q_out=d_q[0])
             else:
-                if i == 1:
-                    cur.wait_event(arrived)
                 md.bi_filter_continue(obs_i, act_i, actp_i, w.K, q_out=d_q[i])
             done[i].record(cur)
             copy_out.wait_event(done[i])
@@ -410,7 +418,7 @@ def main():
     blocks_equal = bool(torch.equal(torch.cat(h_q, dim=1), q.cpu()))
     e2e = {"value": aggregate_throughput(w.updates, world, e2e_sec), "unit": UNIT,
            "h2d_bytes_per_step": int(w.obs.nbytes + w.act.nbytes), "d2h_bytes_per_step": int(q.numel() * 4),
-           "blocks_of_steps": nchunk, "equals_single_call_bit_for_bit": blocks_equal}
+           "blocks_of_steps": lens, "equals_single_call_bit_for_bit": blocks_equal}
 
     flops = algorithmic_flops(w)
     peak = FP64_PEAK_TFLOPS if args.arith == "f64" else FP32_PEAK_TFLOPS
