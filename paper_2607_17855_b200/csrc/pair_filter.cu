@@ -73,8 +73,15 @@ __device__ __forceinline__ int unit_argmax(R x, int idx) {
 
 constexpr int WARPS = 4;
 
-template <int LPU>
+// WARPMAX: the pair's softmax shifts by the largest binary exponent of the whole warp (one reduction
+// instruction) instead of the unit's (a shuffle per halving of the unit): every unit of the warp is then
+// scaled by the same power of two, which is exact, and safe while a logit cannot differ from another
+// agent's by more than the exponent range, which the caller checks from the number of modalities.
+template <int LPU, bool WARPMAX>
 __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairParams p) {
+  // small units take the normalisers from the exchanged copies every lane reads anyway (a few additions
+  // in the shadow of the products) instead of a shuffle sum at the end of the sweep's dependency chain
+  constexpr bool ZLOCAL = LPU <= 8;
   constexpr int UPW = 32 / LPU;
   constexpr int QS = BI_MAX_F * LPU;                  // previous beliefs of one unit: [factor][state]
   __shared__ __align__(16) R exp_tab[EXP_TAB];
@@ -185,7 +192,7 @@ __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairPa
     se[LPU + u] = eb;
     __syncwarp();
     for (int k = 0; k < p.K; ++k) {
-      R v0 = 0.0, v1 = 0.0, w0 = 0.0, w1 = 0.0;
+      R v0 = 0.0, v1 = 0.0, w0 = 0.0, w1 = 0.0, sa0 = 0.0, sa1 = 0.0, sb0 = 0.0, sb1 = 0.0;
 #pragma unroll
       for (int i = 0; i < LPU; i += 2) {
         R b0, b1, a0, a1;
@@ -193,25 +200,37 @@ __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairPa
         lds2(se + i, a0, a1);
         v0 = fma(L[i], b0, v0); v1 = fma(L[i + 1], b1, v1);
         w0 = fma(LT[i], a0, w0); w1 = fma(LT[i + 1], a1, w1);
+        if (ZLOCAL) { sa0 += a0; sa1 += a1; sb0 += b0; sb1 += b1; }
+      }
+      if (ZLOCAL) {   // (one Newton step: 1e-13 relative on a message's scale; the final beliefs take two)
+        za = sa0 + sa1; zb = sb0 + sb1;
+        rza = rcp_fast(za); rzb = rcp_fast(zb);
       }
       xa = fma(v0 + v1, rzb, ca);
       xb = fma(w0 + w1, rza, cb);
       int ka, kb;
       const R ma = exp_mant(xa, exp_tab, ka);
       const R mb = exp_mant(xb, exp_tab, kb);
-      Ma = max_k<LPU, true>(a_ok ? ka : INT_MIN) >> EXP_BITS;
-      Mb = max_k<LPU, true>(b_ok ? kb : INT_MIN) >> EXP_BITS;
+      Ma = max_k<LPU, !WARPMAX>(a_ok ? ka : INT_MIN) >> EXP_BITS;
+      Mb = max_k<LPU, !WARPMAX>(b_ok ? kb : INT_MIN) >> EXP_BITS;
       ea = a_ok ? exp_scale(ma, (ka >> EXP_BITS) - Ma) : 0.0;
       eb = b_ok ? exp_scale(mb, (kb >> EXP_BITS) - Mb) : 0.0;
       __syncwarp();          // every lane has read the previous iterate
       se[u] = ea;
       se[LPU + u] = eb;
+      if (!ZLOCAL) {
+        za = unit_sum<LPU>(ea);
+        zb = unit_sum<LPU>(eb);
+        rza = rcp_fast(za); rzb = rcp_fast(zb);
+      }
+      __syncwarp();
+    }
+    {   // the last iterate's normalisers, to full precision: they scale the step's beliefs
       za = unit_sum<LPU>(ea);
       zb = unit_sum<LPU>(eb);
       const R ra = rcp_fast(za), rb = rcp_fast(zb);
-      rza = ra * (2.0 - za * ra);   // (a second Newton step: these scale the messages and the final beliefs)
+      rza = ra * (2.0 - za * ra);
       rzb = rb * (2.0 - zb * rb);
-      __syncwarp();
     }
     const R qa = ea * rza, qb = eb * rzb;
     sq[p.fa * LPU + u] = qa;
@@ -245,7 +264,11 @@ __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairPa
 template <int LPU>
 int launch(const PairParams &p, cudaStream_t stream) {
   constexpr int per_cta = WARPS * (32 / LPU);
-  bi_pair_filter_kernel<LPU><<<(p.N + per_cta - 1) / per_cta, WARPS * 32, 0, stream>>>(p);
+  const int grid = (p.N + per_cta - 1) / per_cta;
+  // (logits are sums of at most M + 1 terms of magnitude below 37: with few modalities two agents'
+  // logits are within a few hundred binary exponents of each other)
+  if (p.M <= 5) bi_pair_filter_kernel<LPU, true><<<grid, WARPS * 32, 0, stream>>>(p);
+  else bi_pair_filter_kernel<LPU, false><<<grid, WARPS * 32, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? BI_OK : BI_ERR_CUDA;
 }
 
