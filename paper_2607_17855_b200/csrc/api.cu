@@ -27,6 +27,7 @@ struct PackA {
   int32_t dim[BI_MAX_RANK];      // packed axis sizes
   int64_t sstride[BI_MAX_RANK];  // source stride of each packed axis
   int32_t npad;                  // padded size of the last packed axis (rank > 0)
+  uint32_t *wide;                // set to 1 when an entry exceeds 1 (see BiDev::status)
 };
 
 // ln(max(A, eps)) in float64, rounded once; outcome slices contiguous, axes in
@@ -40,7 +41,11 @@ __global__ void bi_pack_A_kernel(PackA p) {
   R out = (R)0;
   if (p.rank == 0) {
     // every axis has a single state: the slice is one number (padded to 4)
-    if (idx == 0) out = (R)log(fmax((double)p.src[go * p.P], 1e-16));
+    if (idx == 0) {
+      const float v = p.src[go * p.P];
+      if (v > 1.0f) atomicOr(p.wide, 1u);
+      out = (R)log(fmax((double)v, 1e-16));
+    }
   } else {
     int32_t last = idx % p.npad, rest = idx / p.npad;
     if (last < p.dim[p.rank - 1]) {
@@ -50,7 +55,9 @@ __global__ void bi_pack_A_kernel(PackA p) {
         rest /= p.dim[j];
         s += (int64_t)dg * p.sstride[j];
       }
-      out = (R)log(fmax((double)p.src[s], 1e-16));
+      const float v = p.src[s];
+      if (v > 1.0f) atomicOr(p.wide, 1u);
+      out = (R)log(fmax((double)v, 1e-16));
     }
   }
   ((R *)p.dst)[e] = out;
@@ -507,8 +514,8 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
   }
 
   // ---- allocate and pack
-  rc = dev_alloc(md, (void **)&h.status, sizeof(uint32_t));
-  if (rc == BI_OK && cudaMemsetAsync(h.status, 0, sizeof(uint32_t), stream) != cudaSuccess) rc = BI_ERR_CUDA;
+  rc = dev_alloc(md, (void **)&h.status, 2 * sizeof(uint32_t));   // the flags, and the wide-range mark
+  if (rc == BI_OK && cudaMemsetAsync(h.status, 0, 2 * sizeof(uint32_t), stream) != cudaSuccess) rc = BI_ERR_CUDA;
   for (int gi = 0; gi < h.ngroups && rc == BI_OK; ++gi) {
     BiGroup &g = h.grp[gi];
     for (int mi = g.mem_begin; mi < g.mem_end && rc == BI_OK; ++mi) {
@@ -523,6 +530,7 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
       memset(&p, 0, sizeof(p));
       p.src = desc->A[i];
       p.dst = dst;
+      p.wide = h.status + 1;
       p.total = (int64_t)count;
       p.P_pad = g.P_pad;
       p.rank = g.rank;

@@ -94,6 +94,9 @@ struct alignas(16) BiDev {
   const void *logBfull[BI_MAX_F];  // ln max(., 1e-16) of the same
   int64_t Bfull_stride[BI_MAX_F];  // elements per model (0 when shared)
   int64_t Dstride[BI_MAX_F];
+  // status[0]: the BI_FLAG_* bits bi_status reports and clears.  status[1]: set when the model was packed
+  // if an entry of A exceeds 1 (not a probability): kernels that shift several agents' softmaxes by one
+  // common power of two then shift per agent, because such logits can lie too far apart for one shift.
   uint32_t *status;
 };
 
@@ -109,6 +112,7 @@ struct bi_model {
   int max_smem_optin;
   int tile_sb;      // > 0: a register-tile shape matches; lanes along b per (agent, step)
   int tile_P;       // elements per lane-interleaved slice
+  int soft_shadow;  // this is the shadow model of a call with observation vectors (weights chosen by the caller)
   int pair_ok;      // at most one group over two factors and none over more: the pair filtering kernel applies
   const void *tile_floor;   // device scalar: ln 1e-16 in the arithmetic type, as the pack kernels compute it
   long long slice_bytes_dense, slice_bytes_compressed;   // per-agent tile models: bytes of the two forms (0: none)

@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairPa
   // small units take the normalisers from the exchanged copies every lane reads anyway (a few additions
   // in the shadow of the products) instead of a shuffle sum at the end of the sweep's dependency chain
   constexpr bool ZLOCAL = LPU <= 8;
+  const bool unit_shift = __ldg(p.status + 1) != 0;   // entries of A above 1: no common shift (BiDev::status)
   constexpr int UPW = 32 / LPU;
   constexpr int QS = BI_MAX_F * LPU;                  // previous beliefs of one unit: [factor][state]
   __shared__ __align__(16) R exp_tab[EXP_TAB];
@@ -211,8 +212,13 @@ __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairPa
       int ka, kb;
       const R ma = exp_mant(xa, exp_tab, ka);
       const R mb = exp_mant(xb, exp_tab, kb);
-      Ma = max_k<LPU, !WARPMAX>(a_ok ? ka : INT_MIN) >> EXP_BITS;
-      Mb = max_k<LPU, !WARPMAX>(b_ok ? kb : INT_MIN) >> EXP_BITS;
+      if (WARPMAX && !unit_shift) {
+        Ma = max_k<LPU, false>(a_ok ? ka : INT_MIN) >> EXP_BITS;
+        Mb = max_k<LPU, false>(b_ok ? kb : INT_MIN) >> EXP_BITS;
+      } else {
+        Ma = max_k<LPU, true>(a_ok ? ka : INT_MIN) >> EXP_BITS;
+        Mb = max_k<LPU, true>(b_ok ? kb : INT_MIN) >> EXP_BITS;
+      }
       ea = a_ok ? exp_scale(ma, (ka >> EXP_BITS) - Ma) : 0.0;
       eb = b_ok ? exp_scale(mb, (kb >> EXP_BITS) - Mb) : 0.0;
       __syncwarp();          // every lane has read the previous iterate

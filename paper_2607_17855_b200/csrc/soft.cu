@@ -186,6 +186,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     sh.h.m[k] = T;
   }
   // (a group of one modality is its own pre-summed table: the shadow's T per-agent slices)
+  sh.soft_shadow = 1;
   sh.pair_ok = 0;   // (no transposed copy of the slices formed above: the pair kernel does not apply)
   sh.tile_comb = tile ? w + off_tile : nullptr;
   sh.tile_ncomb = T;

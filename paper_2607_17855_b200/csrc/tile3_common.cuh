@@ -39,6 +39,7 @@ struct Tile3Params {
   int32_t *argmax_out;
   uint32_t *status;
   double lambda;             // damping step (1 = plain update)
+  int32_t unit_shift;        // softmax shifts per agent even where a warp-wide one would do (see BiDev::status)
 };
 
 // sum_r M[r][s] q[r] for this lane's s: col points at M[0][s], rows are `stride` apart
@@ -66,6 +67,7 @@ static inline void bi_tile3_fill_params(const BiCall &c, Tile3Params &p) {
   const BiGroup &g = h.grp[0];
   p.nmem = g.mem_end - g.mem_begin;
   p.floor_log = md->tile_floor;
+  p.unit_shift = md->soft_shadow;
   p.Lcomb = md->tile_comb;
   p.ncomb = md->tile_ncomb;
   for (int i = 0; i < p.nmem; ++i) p.comb_mul[i] = md->tile_comb_mul[i];

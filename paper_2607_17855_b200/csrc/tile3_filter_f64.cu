@@ -8,14 +8,11 @@ template <int NA, int NB, int NC>
 int launch(const Tile3Params &p, cudaStream_t stream) {
   using G = tile3_f64::Geo<NA, NB, NC>;
   const int grid = (p.N + G::UPW - 1) / G::UPW;
-  // One warp-wide reduction finds the softmax shift of all the warp's agents at once; an agent whose
-  // logits lie far below another's then carries small numerators, and the product of its three
-  // normalisers must stay a normal number: a logit is at least (modalities + 1) ln 1e-16, i.e.
-  // 53.2 (modalities + 1) binary orders below zero, three times that must stay under 1022.
-  if (p.nmem <= 5)
-    tile3_f64::bi_tile3_filter_f64_kernel<NA, NB, NC, false><<<grid, 32, 0, stream>>>(p);
-  else
-    tile3_f64::bi_tile3_filter_f64_kernel<NA, NB, NC, true><<<grid, 32, 0, stream>>>(p);
+  // (an agent whose logits lie far below another's of the same warp carries small numerators under a
+  // common shift, and the product of its three normalisers must stay a normal number: with probabilities
+  // in A a logit is at least (modalities + 1) ln 1e-16, i.e. 53.2 (modalities + 1) binary orders below
+  // zero, and three times that must stay under 1022: the kernel shifts per agent beyond five modalities)
+  tile3_f64::bi_tile3_filter_f64_kernel<NA, NB, NC><<<grid, 32, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? BI_OK : BI_ERR_CUDA;
 }
 

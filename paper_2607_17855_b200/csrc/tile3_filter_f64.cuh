@@ -137,7 +137,7 @@ struct Geo {
 
 // Per-step state of one lane and the sweep.  Everything is indexed with compile-time constants once
 // inlined, so the members live in registers.
-template <class G, bool UNITMAX>
+template <class G>
 struct Sweep {
   using R = double;
   static constexpr int NA = G::NA, NB = G::NB, NC = G::NC, LPU = G::LPU, NBP = G::NBP, NCP = G::NCP;
@@ -172,6 +172,7 @@ struct Sweep {
     Ma = Mb = Mc = 0;
   }
 
+  template <bool UNITMAX>
   __device__ __forceinline__ void sweep() {
     R V[G::NP], W[G::NP];
 #pragma unroll
@@ -238,11 +239,11 @@ struct Sweep {
   }
 };
 
-template <int NA, int NB, int NC, bool UNITMAX>
+template <int NA, int NB, int NC>
 __global__ void __launch_bounds__(32) bi_tile3_filter_f64_kernel(const Tile3Params p) {
   using R = double;
   using G = Geo<NA, NB, NC>;
-  using SW = Sweep<G, UNITMAX>;
+  using SW = Sweep<G>;
   constexpr int LPU = G::LPU, UPW = G::UPW, NCP = G::NCP, NV = G::NV;
   __shared__ __align__(16) R exp_tab[EXP_TAB];
   __shared__ __align__(16) R sm_q[UPW][(NA + NB + NC + 1) & ~1];   // final beliefs of the previous step
@@ -250,6 +251,10 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_f64_kernel(const Tile3Para
   __shared__ __align__(16) R sm_se[UPW][G::SE];
   const int lane = threadIdx.x;
   for (int j = lane; j < EXP_TAB; j += 32) exp_tab[j] = exp2((double)j * (1.0 / EXP_TAB));
+  // One warp-wide reduction finds the softmax shift of all the warp's agents at once, unless the model's
+  // logits can lie too far apart for a common shift (many modalities, entries of A above 1, observation
+  // vectors with the caller's weights): then every agent takes its own.
+  const bool unit_shift = p.unit_shift != 0 || p.nmem > 5 || __ldg(p.status + 1) != 0;
   const int unit = lane / LPU, u = lane % LPU;
   int agent = blockIdx.x * UPW + unit;
   const bool live = agent < p.N;
@@ -382,7 +387,8 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_f64_kernel(const Tile3Para
     sw.lpc = c_ok ? lpc : 0.0;
 
     sw.start();
-    for (int k = 0; k < p.K; ++k) sw.sweep();
+    if (unit_shift) for (int k = 0; k < p.K; ++k) sw.template sweep<true>();
+    else for (int k = 0; k < p.K; ++k) sw.template sweep<false>();
 
     // ---- final beliefs of the step: outputs, and the next step's prior input
     // (1/za = sc zb, 1/zb = sc za, 1/zc = sa zb)

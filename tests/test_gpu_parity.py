@@ -47,6 +47,26 @@ def test_config1(algo):
     print(check_workload(make_config(1), algo))
 
 
+@pytest.mark.parametrize("case", ["tile", "pair"])
+def test_unnormalised_likelihoods_far_above_one(case):
+    """The inputs are used as given.  With entries of A far above 1 for some outcomes and far below for
+    others, agents of one warp see logits hundreds of binary orders apart: the kernels that share one
+    softmax shift among a warp's agents must then shift per agent."""
+    import dataclasses
+    w = make_config(2, N=41, T=6, K=6) if case == "tile" else make_config(1)
+    scale = [10.0 ** e for e in (30, -8, 12, 0, -20, 25, 3, -3)]
+    A = []
+    for a in w.A:
+        a = a.astype(np.float64)
+        for o in range(a.shape[1]):
+            a[:, o] *= scale[o % len(scale)]
+        A.append(a.astype(np.float32))
+    w = dataclasses.replace(w, A=A)
+    res = check_workload(w, "filter", conditioned=True)
+    print(case, res)
+    assert res["kernel"] == ("tile3_filter_f64" if case == "tile" else "pair_filter_f64"), res
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_config2_small(algo):
     print(check_workload(make_config(2, N=96, T=12), algo))
