@@ -536,6 +536,42 @@ def main():
             "slice_forming_gflop": slice_flops / 1e9}
         md_s.close()
         del d_soft, q_s
+        # configuration 4 again with the handle's compressed slices switched on (sparse per-agent models:
+        # a mask per lane and the values above the floor; bit for bit the dense result), with both sizes
+        w4 = make_config(4)
+        md4 = bi.model_from_workload(w4, arith=args.arith)
+        d_obs4, d_act4 = torch.from_numpy(w4.obs).cuda(), torch.from_numpy(w4.act).cuda()
+        q4 = torch.empty((w4.N, w4.T, w4.S), dtype=torch.float32, device="cuda")
+        dense_b, comp_b = md4.slice_bytes()
+        if comp_b:
+            md4.set_compressed(True)
+            ts = time_steps(lambda: md4.bi_mmp(d_obs4, d_act4, w4.K, q_out=q4), max(3, args.steps // 4), 3, flush, torch)
+            sec4 = sum(ts) / len(ts)
+            others[f"config4_mmp_compressed_{args.arith}"] = {
+                "value": w4.updates / sec4, "unit": UNIT, "ms_per_step": sec4 * 1e3, "kernel": md4.last_kernel,
+                "slice_bytes_dense": int(dense_b), "slice_bytes_compressed": int(comp_b)}
+        md4.close()
+        del d_obs4, d_act4, q4, w4
+        # a model with non-trivial B-dependencies (transitions that read other factors' previous states):
+        # config 3's factors and modalities, every factor's transition depending on itself and its
+        # neighbour; filtering and VMP on the general kernel that contracts transition tensors
+        from biwl import make_model, sample_streams, Workload
+        rngb = np.random.default_rng(4242)
+        nb_, mb_, depb, Ub = [10, 10, 8, 6], [12, 10, 8, 6], [[0, 1], [1, 2], [0, 2, 3], [0, 1, 2, 3]], [3, 3, 3, 3]
+        bdep = [[0, 1], [1, 2], [2, 3], [3, 0]]
+        Ab, Bb, Db = make_model(rngb, nb_, mb_, depb, Ub, 1, bdep=bdep)
+        Nb, Tb = 1024, 20
+        ob_, ab_ = sample_streams(rngb, nb_, mb_, depb, Ub, 1, Ab, Bb, Db, Nb, Tb, bdep=bdep)
+        wb = Workload(name="bdep", algo="filter", n=np.asarray(nb_, np.int32), m=np.asarray(mb_, np.int32), dep=depb,
+                      U=np.asarray(Ub, np.int32), G=1, A=Ab, B=Bb, D=Db, N=Nb, T=Tb, K=16, obs=ob_, act=ab_, bdep=bdep)
+        entry = {}
+        for algo in ("filter", "vmp"):
+            r = bench_config(torch, bi, wb, algo, args.arith, 3, 3, flush)
+            entry[algo] = {"value": wb.updates / r["seconds"], "unit": UNIT, "ms_per_step": r["seconds"] * 1e3,
+                           "kernel": r["kernel"]}
+            del r
+        entry["workload"] = "1024 agents, n=[10,10,8,6], T=20, K=16, two parents per transition"
+        others[f"bdep_{args.arith}"] = entry
         # configuration 1 (8 agents, 0.5 KB working set): latency per call, beside a one-element fill
         # kernel timed the same way (what a launch alone costs here)
         w1 = make_config(1)

@@ -151,7 +151,7 @@ int bi_model_arith(const bi_model_t *model);
  * tensor of logarithms contracted likewise, future message to a factor = the sum, over the factors
  * whose transitions read it, of the log-tensor contracted with the next step's belief of that factor
  * and this step's beliefs of the other parents.  Such handles serve bi_filter, bi_filter_from,
- * bi_filter_continue, bi_vmp and bi_vmp_warm (one general kernel family; damping applies).  Marginal
+ * bi_filter_continue, bi_vmp and bi_vmp_warm (the general kernel families; damping applies).  Marginal
  * message passing has no reversed transition for several parents: bi_mmp and its variants, the calls
  * with observation vectors and bi_vmp_from return BI_ERR_UNSUPPORTED on such a handle.
  * Errors as bi_model_create; BI_ERR_INVALID_ARG for a malformed list, BI_ERR_UNSUPPORTED beyond the limits.

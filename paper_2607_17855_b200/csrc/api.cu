@@ -844,7 +844,15 @@ __global__ void bi_predictive_prior_kernel(const BiDev *__restrict__ mdp, int N,
 }
 
 int bi_dispatch(const BiCall &c, bi_model *mut) {
-  if (c.model->h.has_bdep) return bi_launch_generic(c, mut);   // the one family that contracts transition tensors
+  if (c.model->h.has_bdep) {
+    // Transition tensors with several parents.  In filtering they enter only the prior, formed once per
+    // step, which the CTA-per-agent filtering kernel computes; window calls (VMP) need them in every
+    // message: the warp-per-step kernel's lanes sum them, the general kernel where that one does not fit.
+    int rc = BI_ERR_UNSUPPORTED;
+    if (c.model->test_family == BI_FAMILY_ANY)
+      rc = c.algo == BI_ALGO_FILTER ? bi_launch_cta_filter(c, mut) : bi_launch_warp(c, mut);
+    return rc == BI_ERR_UNSUPPORTED ? bi_launch_generic(c, mut) : rc;
+  }
   const int only = c.model->test_family;   // testing aid: start at the named family
   int rc = BI_ERR_UNSUPPORTED;
   if (only == BI_FAMILY_ANY) {

@@ -200,6 +200,28 @@ __device__ __forceinline__ R matrix_col_dot(const R *L, int ls, int col, const R
   return m0 + m1;
 }
 
+// Non-trivial B-dependencies (a transition that reads several factors' previous states): the prior of
+// state s_next is sum_{parents} X[s_next][parents] prod_j q_{parent_j}[s_j], summed by a warp in a fixed
+// order.  It is the only place where such a model differs from a plain one in filtering: the prior is
+// formed once per step, outside the iteration.
+template <typename R>
+__device__ R cta_bdep_expect(const BiDev &md, int f, const R *__restrict__ Xrow, const R *q, int lane) {
+  const int k = md.bdep_len[f], PB = md.PB[f];
+  R acc = (R)0;
+  for (int e = lane; e < PB; e += 32) {
+    int rem = e;
+    R w = (R)1;
+    for (int j = k - 1; j >= 0; --j) {
+      const int gq = md.bdep[f][j], nj = md.n[gq];
+      const int d = rem % nj;
+      rem /= nj;
+      w *= q[md.offp[gq] + d];
+    }
+    acc = fma(__ldg(Xrow + e), w, acc);
+  }
+  return warp_sum(acc);
+}
+
 template <typename R>
 __global__ void __launch_bounds__(256, 2)
 bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__restrict__ obs,
@@ -246,6 +268,22 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
 
   for (int t = 0; t < T; ++t) {
     // ln prior: D at the first step, else B_u q_{t-1} (cur still holds step t-1)
+    if (md.has_bdep && (t > 0 || from_prev)) {   // a warp per state: the expectation of the transition tensor
+      for (int idx = warp; idx < Sp; idx += NW) {
+        int f = 0;
+        while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+        const int s = idx - md.offp[f], n = md.n[f];
+        R lp = (R)0;
+        if (s < n) {
+          const int ur = t == 0 ? __ldg(act_prev + (size_t)a * F + f)
+                                : __ldg(act + ((size_t)a * (T - 1) + (t - 1)) * F + f);
+          const int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
+          const R *row = (const R *)md.Bfull[f] + (size_t)g * md.Bfull_stride[f] + ((size_t)u * n + s) * md.PB[f];
+          lp = bi_log(bi_max(cta_bdep_expect<R>(md, f, row, cur, lane), (R)BI_EPS));
+        }
+        if (lane == 0) lpri[idx] = lp;
+      }
+    } else
     for (int idx = tid; idx < Sp; idx += NT) {
       int f = 0;
       while (f + 1 < F && idx >= md.offp[f + 1]) ++f;

@@ -237,6 +237,65 @@ __device__ __forceinline__ R col_dot_rt(const R *__restrict__ col, int npad, con
   return s0 + s1;
 }
 
+// Non-trivial B-dependencies (VMP only): the two transition messages of one state, summed by its lane.
+// Past: sum_{parents} ln B_f[s][parents] prod_j q_{t-1, parent_j}[s_j].
+template <typename R>
+__device__ R bdep_past_lane(const BiDev &md, int f, const R *__restrict__ Xrow, const R *qprev) {
+  const int k = md.bdep_len[f], PB = md.PB[f];
+  R acc = (R)0;
+  for (int e = 0; e < PB; ++e) {
+    int rem = e;
+    R w = (R)1;
+    for (int j = k - 1; j >= 0; --j) {
+      const int gq = md.bdep[f][j], nj = md.n[gq];
+      const int d = rem % nj;
+      rem /= nj;
+      w *= qprev[md.offp[gq] + d];
+    }
+    acc = fma(__ldg(Xrow + e), w, acc);
+  }
+  return acc;
+}
+// Future, to state s of factor f0: over every factor h whose transition reads f0,
+// sum_{s'} q_{t+1,h}[s'] sum_{parents with s_f0 = s} ln B_h[s'][parents] prod_{other parents} q_t[...];
+// act_t: the actions taken at this step.
+template <typename R>
+__device__ R bdep_future_lane(const BiDev &md, int g, int f0, int s, const R *q, const R *qn,
+                              const int32_t *__restrict__ act_t) {
+  R acc = (R)0;
+  for (int h = 0; h < md.F; ++h) {
+    const int k = md.bdep_len[h];
+    int pos = -1;
+    for (int j = 0; j < k; ++j)
+      if (md.bdep[h][j] == f0) pos = j;
+    if (pos < 0) continue;
+    const int nh = md.n[h], PB = md.PB[h];
+    const int u = clamp_flag(act_t[h], md.U[h], md.status, BI_FLAG_ACT_RANGE);
+    const R *X = (const R *)md.logBfull[h] + (size_t)g * md.Bfull_stride[h] + (size_t)u * nh * PB;
+    const int others = PB / md.n[f0];
+    for (int i = 0; i < others; ++i) {
+      int rem = i, e = 0, stride = 1;
+      R w = (R)1;
+      for (int j = k - 1; j >= 0; --j) {
+        const int gq = md.bdep[h][j], nj = md.n[gq];
+        int d;
+        if (j == pos) d = s;
+        else {
+          d = rem % nj;
+          rem /= nj;
+          w *= q[md.offp[gq] + d];
+        }
+        e += d * stride;
+        stride *= nj;
+      }
+      R inner = (R)0;
+      for (int sn = 0; sn < nh; ++sn) inner = fma(qn[md.offp[h] + sn], __ldg(X + (size_t)sn * PB + e), inner);
+      acc = fma(w, inner, acc);
+    }
+  }
+  return acc;
+}
+
 static_assert(sizeof(BiDev) % sizeof(int4) == 0, "descriptor is copied as 16-byte vectors");
 __device__ __forceinline__ void copy_descriptor(const BiDev *src, void *dst) {
   const int4 *s = reinterpret_cast<const int4 *>(src);
@@ -385,6 +444,10 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
           if (t == 0) {
             msg = lnprior ? ((const R *)lnprior)[(size_t)a * S + md.off[f] + s]
                           : ((const R *)md.logD[f])[(size_t)g * md.Dstride[f] + s];
+          } else if (md.has_bdep) {
+            const int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
+            const R *row = (const R *)md.logBfull[f] + (size_t)g * md.Bfull_stride[f] + ((size_t)u * n + s) * md.PB[f];
+            msg = bdep_past_lane<R>(md, f, row, cur + (size_t)(t - 1) * Sp);
           } else {
             int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);  // [previous][next]
@@ -392,7 +455,9 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
             R v = col_dot_rt<R>(col, np, cur + (size_t)(t - 1) * Sp + md.offp[f], n);
             msg = ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
           }
-          if (t + 1 < T) {
+          if (t + 1 < T && md.has_bdep) {
+            msg += bdep_future_lane<R>(md, g, f, s, qt, cur + (size_t)(t + 1) * Sp, act + ((size_t)a * (T - 1) + t) * F);
+          } else if (t + 1 < T) {
             int u = clamp_flag(act[((size_t)a * (T - 1) + t) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);  // [next][previous]
             const R *col = M1 + (size_t)g * md.Bstride[f] + (size_t)u * n * np + s;

@@ -847,7 +847,17 @@ def test_b_dependencies(case, algo):
     w = _bdep_workload(1200 + sorted(BDEP_CASES).index(case), **BDEP_CASES[case])
     res = check_workload(w, algo)
     print(case, algo, res)
-    assert res["kernel"].startswith("generic_")
+    # (in filtering the transition tensors enter only the prior: the CTA-per-agent filtering kernel forms it)
+    if algo == "vmp":   # the warp-per-step kernel's lanes sum the transition tensors' messages
+        assert res["kernel"] == "warp_vmp_f64", res
+        with family_forced("generic"):
+            res = check_workload(w, algo)
+        assert res["kernel"].startswith("generic_"), res
+    else:
+        assert res["kernel"] == "cta_filter_f64", res
+        with family_forced("generic"):
+            res = check_workload(w, algo)
+        assert res["kernel"].startswith("generic_"), res
 
 
 def test_b_dependencies_call_forms_and_refusals():
