@@ -115,14 +115,14 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
         assert q_init.shape == (N, T, S)
     Ap, Bp, Dp = _ptr_array(A), _ptr_array(B), _ptr_array(D)
     if bdep is not None:
-        assert obs_soft is None and damping == 1.0 and not round32
+        assert obs_soft is None and not round32
         bl = np.ascontiguousarray([len(d) for d in bdep], dtype=np.int32)
         bf = np.ascontiguousarray([g for d in bdep for g in d], dtype=np.int32)
         if q_prev is not None:
             q_prev = np.ascontiguousarray(q_prev, dtype=np.float64)
             act_prev = np.ascontiguousarray(act_prev, dtype=np.int32)
             assert q_prev.shape == (N, S) and act_prev.shape == (N, F)
-        rc = lib.bi_ref_run_bdep(
+        rc = lib.bi_ref_run_bdep_damped(
             ctypes.c_int(ALGOS[algo]), ctypes.c_int(F), ctypes.c_int(M),
             ctypes.c_void_p(n.ctypes.data), ctypes.c_void_p(m.ctypes.data),
             ctypes.c_void_p(dep_len.ctypes.data), ctypes.c_void_p(dep_flat.ctypes.data),
@@ -132,6 +132,7 @@ def run(algo: str, n: Sequence[int], m: Sequence[int], dep, U: Sequence[int], G:
             ctypes.c_int(K), ctypes.c_void_p(q_init.ctypes.data if q_init is not None else None),
             ctypes.c_void_p(q_prev.ctypes.data if q_prev is not None else None),
             ctypes.c_void_p(act_prev.ctypes.data if act_prev is not None else None),
+            ctypes.c_double(float(damping)),
             ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(lq.ctypes.data),
             ctypes.c_void_p(am.ctypes.data), ctypes.c_int(threads))
         if rc != 0:

@@ -568,6 +568,24 @@ int bi_ref_run_bdep(int algo, int F, int M, const int32_t *n, const int32_t *m,
                     act_prev, q_out, logq_out, argmax_out, threads, 0, 1.0, bdep_len, bdep);
 }
 
+/*
+ * The same with the damped update of bi_ref_run_opts (lambda in (0, 1]; 1 = plain): the step on the
+ * log-beliefs is taken after the messages are formed, in the code the plain model runs, so nothing
+ * about it depends on how many parents a transition has.
+ */
+int bi_ref_run_bdep_damped(int algo, int F, int M, const int32_t *n, const int32_t *m,
+                           const int32_t *dep_len, const int32_t *dep, const int32_t *U, int G,
+                           const float *const *A, const float *const *B, const float *const *D,
+                           const int32_t *bdep_len, const int32_t *bdep,
+                           int N, int T, const int32_t *obs, const int32_t *act, int K,
+                           const double *q_init, const double *q_prev, const int32_t *act_prev, double lambda,
+                           double *q_out, double *logq_out, int32_t *argmax_out, int threads)
+{
+    if (!bdep_len || !bdep) return -1;
+    return run_impl(algo, F, M, n, m, dep_len, dep, U, G, A, B, D, N, T, obs, NULL, act, K, q_init, q_prev,
+                    act_prev, q_out, logq_out, argmax_out, threads, 0, lambda, bdep_len, bdep);
+}
+
 int bi_ref_max_threads(void)
 {
 #ifdef _OPENMP

@@ -860,6 +860,29 @@ def test_b_dependencies(case, algo):
         assert res["kernel"].startswith("generic_"), res
 
 
+@pytest.mark.parametrize("algo", ["filter", "vmp"])
+def test_b_dependencies_damped(algo):
+    """The damped update on a model with several parents per transition, on the kernels the dispatcher
+    picks and on the general kernel."""
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = _bdep_workload(1400, [4, 3, 5], [5, 4], [[0, 1], [1, 2]], [2, 2, 1], [[0, 1], [1, 2], [2, 0]], N=8, T=6, K=7)
+    ref = oracle.run_workload(w, algo, damping=0.6)[0]
+    for forced in (None, "generic"):
+        with (family_forced(forced) if forced else contextlib.nullcontext()):
+            md = bi.model_from_workload(w)
+        md.set_damping(0.6)
+        q = md.run(algo, torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda(), w.K).cpu().numpy()
+        assert md.status() == 0
+        if forced:
+            assert md.last_kernel.startswith("generic_"), md.last_kernel
+        else:
+            assert md.last_kernel == ("cta_filter_f64" if algo == "filter" else "warp_vmp_f64"), md.last_kernel
+        assert np.abs(q - ref).max() <= 1e-5, (forced, md.last_kernel, np.abs(q - ref).max())
+        md.close()
+
+
 def test_b_dependencies_call_forms_and_refusals():
     import torch
     import oracle

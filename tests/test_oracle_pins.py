@@ -345,6 +345,16 @@ def test_b_dependencies_on_the_factor_itself_are_the_plain_model():
                        bdep=[[0], [1], [2]])
         for x, y in zip(a, b):
             np.testing.assert_allclose(y, x, atol=1e-13)
+    # ... and so does the damped update (the step on the log-beliefs does not see the parents)
+    for algo in ("filter", "vmp"):
+        a = oracle.run(algo, w["n"], w["m"], w["dep"], w["U"], 1, w["A"], w["B"], w["D"], w["obs"], w["act"], 5,
+                       damping=0.6)
+        b = oracle.run(algo, w["n"], w["m"], w["dep"], w["U"], 1, w["A"], w["B"], w["D"], w["obs"], w["act"], 5,
+                       damping=0.6, bdep=[[0], [1], [2]])
+        plain = run(algo, w, 5)
+        assert np.abs(a[0] - plain[0]).max() > 1e-4          # the damping does something here
+        for x, y in zip(a, b):
+            np.testing.assert_allclose(y, x, atol=1e-13)
     # a transition declared on a superset of its true parents (B replicated along the new axis): same beliefs
     B = list(w["B"])
     B[1] = np.ascontiguousarray(np.repeat(w["B"][1][:, :, :, None, :], 2, axis=3))   # [1, 4, 4, n_2 = 2, 3]
