@@ -1,6 +1,6 @@
 // Filtering kernel for models whose factors are coupled at most in one pair: every modality depends
 // on a single factor, except for the modalities of at most one dependency group over two factors
-// (a, b).  (Of the 128 random structures of the randomised benchmark sweep, 86 are of this kind, and
+// (a, b).  (Of the 128 random structures of the randomised benchmark sweep, 77 are of this kind, and
 // so is the smallest benchmark configuration.)  For such a model
 //   * a factor outside the pair receives no message that depends on another factor's belief: its
 //     logits are prior + its modalities' slices, the same in every iteration, so its belief is one
