@@ -511,6 +511,7 @@ static int create_impl(const bi_model_desc *desc, int arith, const int32_t *bdep
       if (h.grp[gi].rank > 2) ++deep;
     }
     md->pair_ok = !bdep_len && deep == 0 && r2 <= 1;
+    md->rank2_ok = !bdep_len && deep == 0;   // any number of groups over two factors: the pair window kernel's models
   }
 
   // ---- allocate and pack

@@ -113,6 +113,7 @@ struct bi_model {
   int tile_sb;      // > 0: a register-tile shape matches; lanes along b per (agent, step)
   int tile_P;       // elements per lane-interleaved slice
   int soft_shadow;  // this is the shadow model of a call with observation vectors (weights chosen by the caller)
+  int rank2_ok;     // no group over more than two factors: the pair window kernel applies
   int pair_ok;      // at most one group over two factors and none over more: the pair filtering kernel applies
   const void *tile_floor;   // device scalar: ln 1e-16 in the arithmetic type, as the pack kernels compute it
   long long slice_bytes_dense, slice_bytes_compressed;   // per-agent tile models: bytes of the two forms (0: none)

@@ -1,6 +1,6 @@
-// Window kernel (VMP and MMP) for models whose factors are coupled at most in one pair: every
-// modality depends on a single factor, except for the modalities of at most one dependency group
-// over two factors (the models pair_filter.cu serves for filtering).
+// Window kernel (VMP and MMP) for models whose dependency groups span at most two factors: every
+// modality depends on a single factor or on a pair of factors (one pair, the models pair_filter.cu
+// serves for filtering; or several: chains, triangles, separate pairs).
 //
 // One CTA per agent; a unit of LPU lanes owns one time step (LPU = the largest state count rounded up
 // to a power of two, lane s owning state s of every factor), so the whole window iterates inside one
@@ -11,8 +11,10 @@
 //   * the two transition messages: dot products of the neighbours' beliefs with one row of a
 //     transposed transition matrix, read [summation index][own state] so that the unit's lanes read
 //     consecutive addresses (the matrices of a shared model stay in L1),
-//   * for the two factors of the pair, a matrix-vector product with the step's summed slice: its row
-//     in registers for the first factor, its column from a copy staged in shared memory for the second,
+//   * for every two-factor group the factor is in, a matrix-vector product with the step's summed
+//     slice, staged once per call in shared memory (row-major with a padded row: a lane reads its row
+//     for the group's first factor and its column for the second without bank conflicts; a model with
+//     a single such group and units below 32 lanes keeps the row in registers),
 // and takes the softmax over the unit's lanes (table-driven exponential, shift by the largest binary
 // exponent).  Float64 handles, plain (undamped) update, trivial B-dependencies.
 #include "bi_internal.h"
@@ -39,7 +41,10 @@ struct PairWinParams {
   int32_t r1_mod[BI_MAX_M], r1_m[BI_MAX_M], r1_P[BI_MAX_M];
   const R *r1_logA[BI_MAX_M];
   int64_t r1_gstride[BI_MAX_M];
-  int32_t fa, fb, na, nb, npb, n2;
+  // the groups over two factors (ng of them; fa[0] < 0 when ng == 0): factors, sizes, and their member
+  // modalities [g2_begin[j], g2_begin[j + 1]) of the r2 arrays; slices [m][na][npb]
+  int32_t ng, fa[BI_MAX_GROUPS], fb[BI_MAX_GROUPS], na[BI_MAX_GROUPS], nb[BI_MAX_GROUPS], npb[BI_MAX_GROUPS];
+  int32_t g2_begin[BI_MAX_GROUPS + 1];
   int32_t r2_mod[BI_MAX_M], r2_m[BI_MAX_M];
   const R *r2_logA[BI_MAX_M];
   int64_t r2_gstride[BI_MAX_M];
@@ -104,8 +109,8 @@ __global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams
   R *qb = exp_tab + EXP_TAB;                                    // [2][units + 2][F][LPU]; slot 0 and the last are never read as neighbours of a real edge
   const int slot_sz = p.F * LPU, buf_sz = (p.units + 2) * slot_sz;
   R *cst = qb + 2 * buf_sz;                                     // [units][F][LPU] constants of the logits
-  R *Ls = cst + p.units * slot_sz;                              // [units][LPU][LS] the pair's summed slice, row-major
-  int32_t *aoff = reinterpret_cast<int32_t *>(Ls + (p.fa >= 0 ? (size_t)p.units * LPU * LS : 0));   // [units][F][2] matrix offsets of the two edges
+  R *Ls = cst + p.units * slot_sz;                              // [units][ng][LPU][LS] the pair groups' summed slices, row-major
+  int32_t *aoff = reinterpret_cast<int32_t *>(Ls + (size_t)p.units * p.ng * LPU * LS);   // [units][F][2] matrix offsets of the two edges
   for (int j = threadIdx.x; j < EXP_TAB; j += blockDim.x) exp_tab[j] = exp2((double)j * (1.0 / EXP_TAB));
 
   const int agent = blockIdx.x, g = p.G == 1 ? 0 : agent;
@@ -114,8 +119,7 @@ __global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams
   const int t = live ? tl : p.T - 1;   // idle units shadow the last step; they store nothing
   const size_t ob = (size_t)agent * p.T + t;
   const int32_t *obs_t = p.obs + ob * p.M;
-  const bool pair = p.fa >= 0;
-  const bool a_ok = pair && s < p.na;
+  const int NG = p.ng;
 
   // ---- once per call: constants, matrix offsets, the pair's slice, the starting beliefs
   for (int f = 0; f < p.F; ++f) {
@@ -146,24 +150,29 @@ __global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams
       }
     }
   }
+  // the groups' summed slices: lane s forms row s; a single group's row also stays in registers
   R L[LPU];
 #pragma unroll
   for (int i = 0; i < LPU; ++i) L[i] = 0.0;
-  if (pair) {
-    for (int j = 0; j < p.n2; ++j) {
+  for (int gj = 0; gj < NG; ++gj) {
+    const bool a_ok = s < p.na[gj];
+#pragma unroll
+    for (int i = 0; i < LPU; ++i) L[i] = 0.0;
+    for (int j = p.g2_begin[gj]; j < p.g2_begin[gj + 1]; ++j) {
       const int o = clamp_flag(__ldg(obs_t + p.r2_mod[j]), p.r2_m[j], p.status, BI_FLAG_OBS_RANGE);
-      const R *row = p.r2_logA[j] + (size_t)g * p.r2_gstride[j] + ((size_t)o * p.na + (a_ok ? s : 0)) * p.npb;
+      const R *row = p.r2_logA[j] + (size_t)g * p.r2_gstride[j] + ((size_t)o * p.na[gj] + (a_ok ? s : 0)) * p.npb[gj];
 #pragma unroll
       for (int i = 0; i < LPU; i += 2) {
-        if (i < p.npb) {
+        if (i < p.npb[gj]) {
           const double2 x = __ldg(reinterpret_cast<const double2 *>(row + i));
           L[i] += x.x; L[i + 1] += x.y;
         }
       }
     }
-    {
 #pragma unroll
-      for (int i = 0; i < LPU; ++i) Ls[((size_t)tl * LPU + s) * LS + i] = a_ok ? L[i] : 0.0;
+    for (int i = 0; i < LPU; ++i) {
+      if (!a_ok) L[i] = 0.0;
+      Ls[(((size_t)tl * NG + gj) * LPU + s) * LS + i] = L[i];
     }
   }
   // slots 0 and units + 1 (the neighbours of the window's ends): zeros, never weighted
@@ -197,28 +206,32 @@ __global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams
         }
         x += (has_prev ? dp : 0.0) + (has_next ? df : 0.0);
       }
-      if (pair && f == p.fa) {        // row s of the slice with the other factor's belief
-        const R *qo = qc + p.fb * LPU;
-        const R *rowp = Ls + ((size_t)tl * LPU + s) * LS;   // (32-lane units read the row from the staged copy)
-        R v0 = 0.0, v1 = 0.0;
+      for (int gj = 0; gj < NG; ++gj) {
+        const R *Lg = Ls + ((size_t)tl * NG + gj) * LPU * LS;
+        if (f == p.fa[gj]) {          // row s of the group's slice with the other factor's belief
+          const R *qo = qc + p.fb[gj] * LPU;
+          const R *rowp = Lg + (size_t)s * LS;   // (several groups, or 32-lane units: the row from the staged copy)
+          const bool lreg = LREG && NG == 1;
+          R v0 = 0.0, v1 = 0.0;
 #pragma unroll
-        for (int i = 0; i < LPU; i += 2) {
-          R b0, b1;
-          lds2(qo + i, b0, b1);
-          v0 = fma(LREG ? L[i] : rowp[i], b0, v0); v1 = fma(LREG ? L[i + 1] : rowp[i + 1], b1, v1);
-        }
-        x += v0 + v1;
-      } else if (pair && f == p.fb) { // column s
-        const R *qo = qc + p.fa * LPU;
-        const R *col = Ls + (size_t)tl * LPU * LS + s;
-        R v0 = 0.0, v1 = 0.0;
+          for (int i = 0; i < LPU; i += 2) {
+            R b0, b1;
+            lds2(qo + i, b0, b1);
+            v0 = fma(lreg ? L[i] : rowp[i], b0, v0); v1 = fma(lreg ? L[i + 1] : rowp[i + 1], b1, v1);
+          }
+          x += v0 + v1;
+        } else if (f == p.fb[gj]) {   // column s
+          const R *qo = qc + p.fa[gj] * LPU;
+          const R *col = Lg + s;
+          R v0 = 0.0, v1 = 0.0;
 #pragma unroll
-        for (int i = 0; i < LPU; i += 2) {
-          R a0, a1;
-          lds2(qo + i, a0, a1);
-          v0 = fma(col[i * LS], a0, v0); v1 = fma(col[(i + 1) * LS], a1, v1);
+          for (int i = 0; i < LPU; i += 2) {
+            R a0, a1;
+            lds2(qo + i, a0, a1);
+            v0 = fma(col[i * LS], a0, v0); v1 = fma(col[(i + 1) * LS], a1, v1);
+          }
+          x += v0 + v1;
         }
-        x += v0 + v1;
       }
       int kk;
       const R mant = exp_mant(ok ? x : 0.0, exp_tab, kk);
@@ -251,7 +264,7 @@ int launch(PairWinParams &p, const bi_model *md, cudaStream_t stream) {
   if (threads > 512) return BI_ERR_UNSUPPORTED;   // (the kernel's register budget is set for this)
   p.units = threads / LPU;
   const size_t slot = (size_t)p.F * LPU;
-  size_t elems = EXP_TAB + 2 * (p.units + 2) * slot + p.units * slot + (p.fa >= 0 ? (size_t)p.units * LPU * (LPU + 1) : 0);
+  size_t elems = EXP_TAB + 2 * (p.units + 2) * slot + p.units * slot + (size_t)p.units * p.ng * LPU * (LPU + 1);
   const size_t bytes = elems * sizeof(R) + (size_t)p.units * p.F * 2 * sizeof(int32_t) + 16;
   if (bytes > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
   auto kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP> : bi_pair_window_kernel<LPU, BI_ALGO_MMP>;
@@ -266,13 +279,13 @@ int launch(PairWinParams &p, const bi_model *md, cudaStream_t stream) {
 }  // namespace
 
 // Applicable to float64 handles, the plain update, trivial B-dependencies, window calls (also warm
-// starts and continued windows) on models whose groups over more than one factor number at most one,
-// over exactly two factors, and to windows whose steps fit one CTA; BI_ERR_UNSUPPORTED otherwise.
+// starts and continued windows) on models with no group over more than two factors, and to windows
+// whose steps and staged slices fit one CTA; BI_ERR_UNSUPPORTED otherwise.
 int bi_launch_pair_window(const BiCall &c, bi_model *mut) {
   const bi_model *md = c.model;
   const BiDev &h = md->h;
   if (c.algo == BI_ALGO_FILTER || md->arith != BI_ARITH_F64 || c.lambda != 1.0 || h.has_bdep) return BI_ERR_UNSUPPORTED;
-  if (!md->pair_ok) return BI_ERR_UNSUPPORTED;
+  if (!md->rank2_ok) return BI_ERR_UNSUPPORTED;
   PairWinParams p;
   memset(&p, 0, sizeof(p));
   p.N = c.N; p.T = c.T; p.K = c.K; p.F = h.F; p.M = h.M; p.S = h.S; p.G = h.G; p.algo = c.algo;
@@ -285,7 +298,6 @@ int bi_launch_pair_window(const BiCall &c, bi_model *mut) {
     p.Bstride[f] = h.Bstride[f]; p.Dstride[f] = h.Dstride[f];
     nmax = h.n[f] > nmax ? h.n[f] : nmax;
   }
-  p.fa = p.fb = -1;
   int n1 = 0;
   for (int f = 0; f < h.F; ++f) {
     p.r1_begin[f] = n1;
@@ -301,20 +313,24 @@ int bi_launch_pair_window(const BiCall &c, bi_model *mut) {
     }
   }
   p.r1_begin[h.F] = n1;
+  int n2 = 0;
   for (int gi = 0; gi < h.ngroups; ++gi) {
     const BiGroup &gr = h.grp[gi];
     if (gr.rank != 2) continue;
-    p.fa = gr.axis[0]; p.fb = gr.axis[1];
-    p.na = gr.dim[0]; p.nb = gr.dim[1];
-    p.npb = bi_pad4(p.nb);
+    const int gj = p.ng++;
+    p.fa[gj] = gr.axis[0]; p.fb[gj] = gr.axis[1];
+    p.na[gj] = gr.dim[0]; p.nb[gj] = gr.dim[1];
+    p.npb[gj] = bi_pad4(gr.dim[1]);
+    p.g2_begin[gj] = n2;
     for (int mi = gr.mem_begin; mi < gr.mem_end; ++mi) {
       const BiMember &mm = h.mem[mi];
-      const int j = p.n2++;
-      p.r2_mod[j] = mm.modality; p.r2_m[j] = mm.m;
-      p.r2_logA[j] = (const R *)mm.logA;
-      p.r2_gstride[j] = mm.gstride;
+      p.r2_mod[n2] = mm.modality; p.r2_m[n2] = mm.m;
+      p.r2_logA[n2] = (const R *)mm.logA;
+      p.r2_gstride[n2] = mm.gstride;
+      ++n2;
     }
   }
+  p.g2_begin[p.ng] = n2;
   p.obs = c.obs; p.act = c.act; p.q_init = c.q_init; p.lnprior = (const R *)c.lnprior;
   p.q_out = c.q_out; p.logq_out = c.logq_out; p.argmax_out = c.argmax_out; p.status = h.status;
   int rc;

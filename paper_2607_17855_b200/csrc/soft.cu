@@ -187,7 +187,8 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
   }
   // (a group of one modality is its own pre-summed table: the shadow's T per-agent slices)
   sh.soft_shadow = 1;
-  sh.pair_ok = 0;   // (no transposed copy of the slices formed above: the pair kernel does not apply)
+  sh.pair_ok = 0;
+  sh.rank2_ok = 0;   // (no transposed copy of the slices formed above: the pair kernel does not apply)
   sh.tile_comb = tile ? w + off_tile : nullptr;
   sh.tile_ncomb = T;
   sh.tile_comb_mul[0] = 1;

@@ -1027,6 +1027,44 @@ def test_pair_window_kernel_on_sweep_structures(j, algo):
     assert res["kernel"] == f"pair_{algo}_f64", res
 
 
+RANK2_CASES = {
+    "chain": lambda: _custom(191, [6, 9, 5, 3], [4, 3, 5, 2], [[0, 1], [1, 2], [3], [2, 1]], [2, 1, 3, 2], N=9, T=6, K=6),
+    "triangle": lambda: _custom(192, [12, 16, 7], [3, 4, 2, 3], [[0, 1], [2, 0], [1, 2], [1]], [2, 2, 2], N=5, T=5, K=5,
+                                sparsity=0.5),
+    "two_pairs_32_lanes": lambda: _custom(193, [31, 32, 20, 6], [3, 2, 4], [[0, 1], [3, 2], [1, 0]], [1, 2, 2, 3],
+                                          N=3, T=4, K=4),
+    "per_agent": lambda: _custom(194, [5, 7, 4], [4, 3, 3], [[0, 1], [1, 2], [2]], [2, 2, 1], N=6, T=5, K=6, G=6, sparsity=0.5),
+}
+
+
+@pytest.mark.parametrize("algo", ["vmp", "mmp"])
+@pytest.mark.parametrize("case", sorted(RANK2_CASES))
+def test_pair_window_kernel_with_several_pairs(case, algo):
+    """Models whose groups all span at most two factors, several of them: the window kernel takes every
+    group's matrix-vector products from the staged slices."""
+    w = RANK2_CASES[case]()
+    res = check_workload(w, algo, conditioned=True)
+    print(case, algo, res)
+    assert res["kernel"] == f"pair_{algo}_f64", res
+
+
+@pytest.mark.parametrize("j", [1, 2, 4, 17, 30, 62, 78])
+def test_pair_window_kernel_on_sweep_structures_with_several_pairs(j):
+    w = make_sweep_config(j, N=11, T=6)
+    for algo in ("vmp", "mmp"):
+        res = check_workload(w, algo, conditioned=True)
+        assert res["kernel"] == f"pair_{algo}_f64", res
+
+
+@pytest.mark.parametrize("case", sorted(RANK2_CASES))
+def test_filtering_on_models_with_several_pairs(case):
+    """(the same models through bi_filter: the CTA-per-agent filtering kernel's rank-2 path)"""
+    w = RANK2_CASES[case]()
+    res = check_workload(w, "filter", conditioned=True)
+    print(case, res)
+    assert res["kernel"] == "cta_filter_f64", res
+
+
 def test_pair_window_kernel_limits():
     """A window whose steps do not fit one CTA goes to another kernel family; so does a damped call."""
     import torch
