@@ -56,12 +56,14 @@ struct BatchMember {
   int32_t ncp, rows;       // padded last axis; rows = product of the outer axes
   int64_t gstride;         // elements per agent's model (per-agent models), 0 when shared
   int32_t task0;           // first task slot of this member
+  int32_t split;           // unrolled forms: threads per unit (1, 2 or 4), each taking a range of the first axis
 };
 
 struct BatchParams {
   BatchMember mem[BI_MAX_M];
   int32_t nmem;            // members of rank >= 2
   int32_t NU, Sp, ntask, tu;   // tu: units per contraction CTA
+  int32_t sc_off;          // unrolled forms: element offset of the split tasks' scratch columns behind the slice
   int32_t lbuf, so_max;    // any-shape form: elements of the slice staging buffer; most outer states of a member
   const int32_t *perm;     // [nmem][NU] unit ids ordered by observed outcome
   const int4 *task;        // [ntask] (outcome, first position, count, unused)
@@ -77,6 +79,9 @@ struct BatchParams {
 // L: the slice in shared memory, rows of NCP; q / out: this unit's beliefs and
 // message area (padded layout); o0..: offsets of the axes' factors.
 
+// SPLIT > 1: the threads of `SPLIT` different warps share a unit, each taking a range of the first
+// axis (part = which); a thread writes the first axis' messages of its range, and its partial messages
+// of the other axes to the scratch columns sc[i * nt + tid], which the caller adds in a fixed order.
 template <typename R, int N1, int NC>
 __device__ __forceinline__ void contract2(const R *__restrict__ L, const R *__restrict__ q, R *__restrict__ out,
                                           const int32_t *o) {
@@ -100,16 +105,17 @@ __device__ __forceinline__ void contract2(const R *__restrict__ L, const R *__re
   for (int c = 0; c < NC; ++c) out[o[1] + c] = accc[c];
 }
 
-template <typename R, int N1, int N2, int NC>
+template <typename R, int N1, int N2, int NC, int SPLIT = 1>
 __device__ __forceinline__ void contract3(const R *__restrict__ L, const R *__restrict__ q, R *__restrict__ out,
-                                          const int32_t *o) {
+                                          const int32_t *o, int part = 0, bool wr = true, R *sc = nullptr, int nt = 0) {
+  const int sa = part * N1 / SPLIT, sb = (part + 1) * N1 / SPLIT;
   constexpr int NCP = (NC + 3) & ~3;
   R q2[N2], qc[NC], acc2[N2], accc[NC];
 #pragma unroll
   for (int i = 0; i < N2; ++i) { q2[i] = q[o[1] + i]; acc2[i] = (R)0; }
 #pragma unroll
   for (int c = 0; c < NC; ++c) { qc[c] = q[o[2] + c]; accc[c] = (R)0; }
-  for (int s1 = 0; s1 < N1; ++s1) {
+  for (int s1 = sa; s1 < sb; ++s1) {
     const R q1 = q[o[0] + s1];
     R a1 = (R)0;
 #pragma unroll
@@ -127,17 +133,24 @@ __device__ __forceinline__ void contract3(const R *__restrict__ L, const R *__re
       acc2[s2] = fma(q1, v, acc2[s2]);
       a1 = fma(q2[s2], v, a1);
     }
-    out[o[0] + s1] = a1;
+    if (wr) out[o[0] + s1] = a1;
   }
 #pragma unroll
-  for (int i = 0; i < N2; ++i) out[o[1] + i] = acc2[i];
+  for (int i = 0; i < N2; ++i) {
+    if (SPLIT > 1) sc[i * nt] = acc2[i];
+    else out[o[1] + i] = acc2[i];
+  }
 #pragma unroll
-  for (int c = 0; c < NC; ++c) out[o[2] + c] = accc[c];
+  for (int c = 0; c < NC; ++c) {
+    if (SPLIT > 1) sc[(N2 + c) * nt] = accc[c];
+    else out[o[2] + c] = accc[c];
+  }
 }
 
-template <typename R, int N1, int N2, int N3, int NC>
+template <typename R, int N1, int N2, int N3, int NC, int SPLIT = 1>
 __device__ __forceinline__ void contract4(const R *__restrict__ L, const R *__restrict__ q, R *__restrict__ out,
-                                          const int32_t *o) {
+                                          const int32_t *o, int part = 0, bool wr = true, R *sc = nullptr, int nt = 0) {
+  const int sa = part * N1 / SPLIT, sb = (part + 1) * N1 / SPLIT;
   constexpr int NCP = (NC + 3) & ~3;
   R q2[N2], q3[N3], qc[NC], acc2[N2], acc3[N3], accc[NC];
 #pragma unroll
@@ -146,7 +159,7 @@ __device__ __forceinline__ void contract4(const R *__restrict__ L, const R *__re
   for (int i = 0; i < N3; ++i) { q3[i] = q[o[2] + i]; acc3[i] = (R)0; }
 #pragma unroll
   for (int c = 0; c < NC; ++c) { qc[c] = q[o[3] + c]; accc[c] = (R)0; }
-  for (int s1 = 0; s1 < N1; ++s1) {
+  for (int s1 = sa; s1 < sb; ++s1) {
     const R q1 = q[o[0] + s1];
     R a1 = (R)0;
 #pragma unroll
@@ -171,21 +184,37 @@ __device__ __forceinline__ void contract4(const R *__restrict__ L, const R *__re
       acc2[s2] = fma(q1, v2, acc2[s2]);
       a1 = fma(q2[s2], v2, a1);
     }
-    out[o[0] + s1] = a1;
+    if (wr) out[o[0] + s1] = a1;
   }
 #pragma unroll
-  for (int i = 0; i < N2; ++i) out[o[1] + i] = acc2[i];
+  for (int i = 0; i < N2; ++i) {
+    if (SPLIT > 1) sc[i * nt] = acc2[i];
+    else out[o[1] + i] = acc2[i];
+  }
 #pragma unroll
-  for (int i = 0; i < N3; ++i) out[o[2] + i] = acc3[i];
+  for (int i = 0; i < N3; ++i) {
+    if (SPLIT > 1) sc[(N2 + i) * nt] = acc3[i];
+    else out[o[2] + i] = acc3[i];
+  }
 #pragma unroll
-  for (int c = 0; c < NC; ++c) out[o[3] + c] = accc[c];
+  for (int c = 0; c < NC; ++c) {
+    if (SPLIT > 1) sc[(N2 + N3 + c) * nt] = accc[c];
+    else out[o[3] + c] = accc[c];
+  }
 }
 
 template <typename R, int RANK, int D0, int D1, int D2, int D3>
-__device__ __forceinline__ void contract_shape(const R *L, const R *q, R *out, const int32_t *o) {
+__device__ __forceinline__ void contract_shape(const R *L, const R *q, R *out, const int32_t *o, int split, int part,
+                                               bool wr, R *sc, int nt) {
   if constexpr (RANK == 2) contract2<R, D0, D1>(L, q, out, o);
-  else if constexpr (RANK == 3) contract3<R, D0, D1, D2>(L, q, out, o);
-  else contract4<R, D0, D1, D2, D3>(L, q, out, o);
+  else if constexpr (RANK == 3) {
+    if (split == 1) contract3<R, D0, D1, D2>(L, q, out, o);
+    else contract3<R, D0, D1, D2, 2>(L, q, out, o, part, wr, sc, nt);
+  } else {
+    if (split == 1) contract4<R, D0, D1, D2, D3>(L, q, out, o);
+    else if (split == 2) contract4<R, D0, D1, D2, D3, 2>(L, q, out, o, part, wr, sc, nt);
+    else contract4<R, D0, D1, D2, D3, 4>(L, q, out, o, part, wr, sc, nt);
+  }
 }
 
 // ---- bucket the units of one modality by observed outcome (once per call) ----
@@ -207,7 +236,7 @@ bi_batch_bucket_kernel(BatchParams P, const int32_t *__restrict__ obs, int M, ui
   __syncthreads();
   if (threadIdx.x == 0) {
     int pos = 0, slot = mm.task0;
-    const int tu = P.tu;
+    const int tu = P.tu / mm.split;
     const int slot_end = mm.task0 + (NU + tu - 1) / tu + m;
     for (int o = 0; o < m; ++o) {
       cursor[o] = pos;
@@ -261,8 +290,12 @@ bi_batch_contract_kernel(BatchParams P, int cur, int first) {
     if (P.drop_copy) bi_mbar_expect(&bar, (uint32_t)(mm.P_pad * sizeof(R)));   // (testing aid: the copy never comes)
     else bi_bulk_load(L, (const R *)mm.logA + (size_t)tk.x * mm.P_pad, (uint32_t)(mm.P_pad * sizeof(R)), &bar);
   }
-  const bool has_unit = (int)threadIdx.x < tk.z;
-  const int unit = has_unit ? P.perm[(size_t)mi * P.NU + tk.y + threadIdx.x] : 0;
+  // (a heavy member's units are shared by `split` threads, one in each of `split` groups of warps: a
+  // warp's threads then still read the same slice row, a broadcast)
+  const int upt = (int)blockDim.x / mm.split;   // units per task of this member
+  const int ut = (int)threadIdx.x % upt, part = (int)threadIdx.x / upt;
+  const bool has_unit = ut < tk.z;
+  const int unit = has_unit ? P.perm[(size_t)mi * P.NU + tk.y + ut] : 0;
   const R *q = (const R *)P.qbuf + ((size_t)cur * P.NU + unit) * P.Sp;
   R *out = (R *)P.ellp + ((size_t)mi * P.NU + unit) * P.Sp;
   if (!first) {   // beliefs of the previous update, and the right to overwrite the messages it read
@@ -275,13 +308,29 @@ bi_batch_contract_kernel(BatchParams P, int cur, int first) {
     if (threadIdx.x == 0) atomicOr(P.status, BI_FLAG_COPY_TIMEOUT);
     return;
   }
-  if (!has_unit) return;
+  // (in a split task the threads without a unit stay for the barrier below; they contract unit 0's
+  // beliefs and write nothing)
+  if (!has_unit && mm.split == 1) return;
+  R *sc = L + P.sc_off + threadIdx.x;   // scratch columns behind the slice
   switch (mm.shape) {
 #define X(ID, RANK, D0, D1, D2, D3) \
-  case ID: contract_shape<R, RANK, D0, D1, D2, D3>(L, q, out, mm.offp); break;
+  case ID: contract_shape<R, RANK, D0, D1, D2, D3>(L, q, out, mm.offp, mm.split, part, has_unit, sc, (int)blockDim.x); break;
     BI_BATCH_SHAPES(X)
 #undef X
     default: break;
+  }
+  if (mm.split > 1) {   // add the parts' partial messages of the axes after the first, part 0 first
+    __syncthreads();
+    if (part == 0 && has_unit) {
+      const R *col = L + P.sc_off + ut;
+      int idx = 0;
+      for (int j = 1; j < mm.rank; ++j)
+        for (int i = 0; i < mm.dim[j]; ++i, ++idx) {
+          R sum = col[(size_t)idx * blockDim.x];
+          for (int pp = 1; pp < mm.split; ++pp) sum += col[(size_t)idx * blockDim.x + pp * upt];
+          out[mm.offp[j] + i] = sum;
+        }
+    }
   }
 }
 
@@ -719,6 +768,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     }
     bm.ncp = bi_pad4(g.dim[g.rank - 1]);
     bm.rows = rows;
+    bm.split = 1;
     if ((long long)rows * bm.ncp != mm.P_pad || bm.ncp > 32) return BI_ERR_UNSUPPORTED;
     so_max = std::max(so_max, so);
     max_slice = std::max(max_slice, (size_t)mm.P_pad * sizeof(R));
@@ -748,10 +798,33 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     P.tu = tu;
   }
   if (csmem > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
+  // Unrolled forms: a member whose contraction is several thousand multiply-adds per unit is shared by
+  // two threads per unit (halves of the first axis, in different warps), so that the schedulers that
+  // get one more of its warps than the rest do not set the time.  (Measured on a rank-4 group of 4800
+  // entries, 20 480 units: 1.32 ms per call unsplit, 1.23 ms in halves, 1.27 ms in quarters; lanes of one
+  // warp sharing a unit, which turns the slice rows' broadcast loads into four different rows, 2.3 ms.)
+  if (!any_shape)
+    for (int j = 0; j < cnt; ++j) {
+      BatchMember &bm = P.mem[j];
+      const long long fm = 2LL * bm.P_pad;
+      int sp = fm >= 4000 ? 2 : 1;
+      if (bm.rank == 3 && sp > 2) sp = 2;
+      if (bm.rank < 3) sp = 1;
+      while (sp > 1 && (bm.dim[0] < sp || (tu / sp) % 32 != 0)) sp >>= 1;   // (whole warps per part)
+      bm.split = sp;
+      if (sp > 1) {
+        int ns = 0;
+        for (int k = 1; k < bm.rank; ++k) ns += bm.dim[k];
+        P.sc_off = (int)((max_slice / sizeof(R) + 1) & ~(size_t)1);
+        csmem = std::max(csmem, ((size_t)P.sc_off + (size_t)ns * tu) * sizeof(R));
+      }
+    }
+  if (csmem > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
   int ntask = 0;
   for (int j = 0; j < cnt; ++j) {
     P.mem[j].task0 = ntask;
-    ntask += (NU + tu - 1) / tu + P.mem[j].m;
+    const int tum = tu / P.mem[j].split;
+    ntask += (NU + tum - 1) / tum + P.mem[j].m;
   }
   P.nmem = cnt; P.NU = NU; P.Sp = h.Sp; P.ntask = ntask;
 
