@@ -115,8 +115,10 @@ __device__ __forceinline__ void contract3(const R *__restrict__ L, const R *__re
   for (int i = 0; i < N2; ++i) { q2[i] = q[o[1] + i]; acc2[i] = (R)0; }
 #pragma unroll
   for (int c = 0; c < NC; ++c) { qc[c] = q[o[2] + c]; accc[c] = (R)0; }
+  R q1n = q[o[0] + sa];   // (the first axis' belief is read one index ahead: its latency hides under the rows)
   for (int s1 = sa; s1 < sb; ++s1) {
-    const R q1 = q[o[0] + s1];
+    const R q1 = q1n;
+    if (s1 + 1 < sb) q1n = q[o[0] + s1 + 1];
     R a1 = (R)0;
 #pragma unroll
     for (int s2 = 0; s2 < N2; ++s2) {
@@ -159,8 +161,10 @@ __device__ __forceinline__ void contract4(const R *__restrict__ L, const R *__re
   for (int i = 0; i < N3; ++i) { q3[i] = q[o[2] + i]; acc3[i] = (R)0; }
 #pragma unroll
   for (int c = 0; c < NC; ++c) { qc[c] = q[o[3] + c]; accc[c] = (R)0; }
+  R q1n = q[o[0] + sa];   // (read one index ahead, as above)
   for (int s1 = sa; s1 < sb; ++s1) {
-    const R q1 = q[o[0] + s1];
+    const R q1 = q1n;
+    if (s1 + 1 < sb) q1n = q[o[0] + s1 + 1];
     R a1 = (R)0;
 #pragma unroll
     for (int s2 = 0; s2 < N2; ++s2) {
