@@ -32,6 +32,7 @@ struct WarpSmem {       // element offsets (units of R) into dynamic shared memo
   int total_bytes;
   int W;                // warps per CTA
   int o_xp;             // filtering, damped calls: per-warp previous logits [Sp]; -1 otherwise
+  int o_Y;              // window, models with B-dependencies: per-warp [sum_h PB_h] next-belief-weighted tensors; -1 otherwise
   int xp;               // window, damped calls: [T][Sp] previous logits shared by the CTA; -1 otherwise
 };
 
@@ -238,59 +239,111 @@ __device__ __forceinline__ R col_dot_rt(const R *__restrict__ col, int npad, con
 }
 
 // Non-trivial B-dependencies (VMP only): the two transition messages of one state, summed by its lane.
+// The parents' state combinations are walked with an odometer (last parent fastest, the order the
+// tensor is stored in) and running prefix products of their beliefs, so a step costs one multiply
+// per digit that changed and no division.
 // Past: sum_{parents} ln B_f[s][parents] prod_j q_{t-1, parent_j}[s_j].
 template <typename R>
 __device__ R bdep_past_lane(const BiDev &md, int f, const R *__restrict__ Xrow, const R *qprev) {
   const int k = md.bdep_len[f], PB = md.PB[f];
+  int dig[BI_MAX_RANK], nj[BI_MAX_RANK], op[BI_MAX_RANK];
+  R wp[BI_MAX_RANK];   // wp[j] = prod_{i <= j} q_{parent_i}[dig_i]
+#pragma unroll
+  for (int j = 0; j < BI_MAX_RANK; ++j) {
+    dig[j] = 0;
+    nj[j] = j < k ? md.n[md.bdep[f][j]] : 1;
+    op[j] = j < k ? md.offp[md.bdep[f][j]] : 0;
+    wp[j] = (R)1;
+  }
+#pragma unroll
+  for (int j = 0; j < BI_MAX_RANK; ++j)
+    if (j < k) wp[j] = (j > 0 ? wp[j > 0 ? j - 1 : 0] : (R)1) * qprev[op[j]];
   R acc = (R)0;
   for (int e = 0; e < PB; ++e) {
-    int rem = e;
-    R w = (R)1;
-    for (int j = k - 1; j >= 0; --j) {
-      const int gq = md.bdep[f][j], nj = md.n[gq];
-      const int d = rem % nj;
-      rem /= nj;
-      w *= qprev[md.offp[gq] + d];
-    }
+    R w = wp[0];
+#pragma unroll
+    for (int j = 1; j < BI_MAX_RANK; ++j) w = j == k - 1 ? wp[j] : w;
     acc = fma(__ldg(Xrow + e), w, acc);
+    // next combination: increment from the last parent, carrying
+    int lo = k;   // lowest digit index that changed
+    bool carry = true;
+#pragma unroll
+    for (int j = BI_MAX_RANK - 1; j >= 0; --j) {
+      if (j < k && carry) {
+        dig[j] += 1;
+        if (dig[j] == nj[j]) dig[j] = 0; else carry = false;
+        lo = j;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < BI_MAX_RANK; ++j)
+      if (j < k && j >= lo) wp[j] = (j > 0 ? wp[j > 0 ? j - 1 : 0] : (R)1) * qprev[op[j] + dig[j]];
   }
   return acc;
 }
 // Future, to state s of factor f0: over every factor h whose transition reads f0,
 // sum_{s'} q_{t+1,h}[s'] sum_{parents with s_f0 = s} ln B_h[s'][parents] prod_{other parents} q_t[...];
-// act_t: the actions taken at this step.
+// act_t: the actions taken at this step.  The other parents' combinations are walked the same way.
+// Y: for every factor h in turn, Y_h[parents] = sum_{s'} q_{t+1,h}[s'] ln B_h[s'][parents], formed by the warp
+// before its lanes call this (bdep_weighted_tensors).
 template <typename R>
-__device__ R bdep_future_lane(const BiDev &md, int g, int f0, int s, const R *q, const R *qn,
-                              const int32_t *__restrict__ act_t) {
-  R acc = (R)0;
+__device__ void bdep_weighted_tensors(const BiDev &md, int g, const R *qn, const int32_t *__restrict__ act_t, R *Y,
+                                      int lane) {
+  int yo = 0;
   for (int h = 0; h < md.F; ++h) {
+    const int nh = md.n[h], PB = md.PB[h];
+    const int u = clamp_flag(act_t[h], md.U[h], md.status, BI_FLAG_ACT_RANGE);
+    const R *X = (const R *)md.logBfull[h] + (size_t)g * md.Bfull_stride[h] + (size_t)u * nh * PB;
+    for (int e = lane; e < PB; e += 32) {   // (consecutive lanes read consecutive entries of a tensor row)
+      R acc = (R)0;
+      for (int sn = 0; sn < nh; ++sn) acc = fma(qn[md.offp[h] + sn], __ldg(X + (size_t)sn * PB + e), acc);
+      Y[yo + e] = acc;
+    }
+    yo += PB;
+  }
+}
+template <typename R>
+__device__ R bdep_future_lane(const BiDev &md, int f0, int s, const R *q, const R *Y) {
+  R acc = (R)0;
+  int yo = 0;
+  for (int h = 0; h < md.F; yo += md.PB[h], ++h) {
     const int k = md.bdep_len[h];
     int pos = -1;
     for (int j = 0; j < k; ++j)
       if (md.bdep[h][j] == f0) pos = j;
     if (pos < 0) continue;
-    const int nh = md.n[h], PB = md.PB[h];
-    const int u = clamp_flag(act_t[h], md.U[h], md.status, BI_FLAG_ACT_RANGE);
-    const R *X = (const R *)md.logBfull[h] + (size_t)g * md.Bfull_stride[h] + (size_t)u * nh * PB;
+    const int PB = md.PB[h];
+    const R *Yh = Y + yo;
     const int others = PB / md.n[f0];
+    int dig[BI_MAX_RANK], nj[BI_MAX_RANK], op[BI_MAX_RANK], str[BI_MAX_RANK];
+    int stride = 1;
+#pragma unroll
+    for (int j = BI_MAX_RANK - 1; j >= 0; --j) {
+      dig[j] = 0;
+      nj[j] = j < k ? md.n[md.bdep[h][j]] : 1;
+      op[j] = j < k ? md.offp[md.bdep[h][j]] : 0;
+      str[j] = stride;           // element stride of parent j in the tensor's parent index
+      if (j < k) stride *= nj[j];
+    }
+    int e = 0;                   // parent index of the current combination (own digit fixed at s)
+#pragma unroll
+    for (int j = 0; j < BI_MAX_RANK; ++j)
+      if (j == pos) { dig[j] = s; e += s * str[j]; }
     for (int i = 0; i < others; ++i) {
-      int rem = i, e = 0, stride = 1;
       R w = (R)1;
-      for (int j = k - 1; j >= 0; --j) {
-        const int gq = md.bdep[h][j], nj = md.n[gq];
-        int d;
-        if (j == pos) d = s;
-        else {
-          d = rem % nj;
-          rem /= nj;
-          w *= q[md.offp[gq] + d];
+#pragma unroll
+      for (int j = 0; j < BI_MAX_RANK; ++j)
+        if (j < k && j != pos) w *= q[op[j] + dig[j]];
+      acc = fma(w, Yh[e], acc);
+      bool carry = true;
+#pragma unroll
+      for (int j = BI_MAX_RANK - 1; j >= 0; --j) {
+        if (j < k && j != pos && carry) {
+          dig[j] += 1;
+          e += str[j];
+          if (dig[j] == nj[j]) { dig[j] = 0; e -= nj[j] * str[j]; } else carry = false;
         }
-        e += d * stride;
-        stride *= nj;
       }
-      R inner = (R)0;
-      for (int sn = 0; sn < nh; ++sn) inner = fma(qn[md.offp[h] + sn], __ldg(X + (size_t)sn * PB + e), inner);
-      acc = fma(w, inner, acc);
     }
   }
   return acc;
@@ -432,6 +485,10 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
     for (int t = warp; t < T; t += W) {
       const R *qt = cur + (size_t)t * Sp;
       slice_table<R>(md, g, obs_s + t * M, false, sl, lane);
+      if (sm.o_Y >= 0 && t + 1 < T) {
+        bdep_weighted_tensors<R>(md, g, cur + (size_t)(t + 1) * Sp, act + ((size_t)a * (T - 1) + t) * F, wb + sm.o_Y, lane);
+        __syncwarp();
+      }
       // transition messages (Section IV): low-rank contractions of B with the
       // neighbouring steps' beliefs of the previous iterate; transposed layouts
       // so that consecutive lanes read consecutive addresses
@@ -456,7 +513,7 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
             msg = ALGO == BI_ALGO_VMP ? v : (R)0.5 * bi_log_inline(bi_max(v, (R)BI_EPS));
           }
           if (t + 1 < T && md.has_bdep) {
-            msg += bdep_future_lane<R>(md, g, f, s, qt, cur + (size_t)(t + 1) * Sp, act + ((size_t)a * (T - 1) + t) * F);
+            msg += bdep_future_lane<R>(md, f, s, qt, wb + sm.o_Y);
           } else if (t + 1 < T) {
             int u = clamp_flag(act[((size_t)a * (T - 1) + t) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *M1 = (const R *)(ALGO == BI_ALGO_VMP ? md.logB[f] : md.BdagT[f]);  // [next][previous]
@@ -504,6 +561,13 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
   const bool damped = c.lambda != 1.0;
   sm.o_xp = (!window && damped) ? o : -1;
   if (!window && damped) o += h.Sp;
+  sm.o_Y = -1;
+  if (window && h.has_bdep) {
+    int ysum = 0;
+    for (int f = 0; f < h.F; ++f) ysum += h.PB[f];
+    sm.o_Y = o;
+    o += bi_pad4(ysum);
+  }
   sm.per_warp = o;
   const size_t budget = 100 * 1024;  // at least two CTAs per SM
   size_t shared_elems = 0;
