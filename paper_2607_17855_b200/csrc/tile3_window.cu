@@ -295,7 +295,7 @@ bi_tile3_window_kernel(const Tile3Params p, const WindowGeom geo) {
   // iterations, and reading them from shared memory again every time was a third of the
   // kernel's shared-memory traffic.
   constexpr int NPA_ = (NA + 3) & ~3, NPB_ = (NB + 3) & ~3, NPC_ = (NC + 3) & ~3;
-  constexpr bool DUPA_ = SB >= 2, DUPB_ = !TT::TP && TT::SHB >= 1, DUPC_ = !TT::TP && TT::SHC >= 1;
+  constexpr bool DUPA_ = SB >= 2, DUPB_ = !TT::TP && TT::SHB >= 1;
   // (the a and b columns: with the c column as well the kernel spills at the 168 registers a
   // ten-warp CTA may use, and measured slower)
   constexpr bool BRA = !LREG && DUPA_, BRB = !LREG && DUPB_, BRC = false;
