@@ -375,11 +375,13 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
     qc[c] = (has_unit && c < NC) ? q[mm.offp[K1] + c] : (R)0;
     accc[c] = (R)0;
   }
+  // (the outer axes' beliefs once per unit: the splits of a unit read the same column)
   for (int j = 0; j < K1; ++j)
     for (int sj = 0; sj < mm.dim[j]; ++sj) {
-      qs[(mm.ooff[j] + sj) * nt + tid] = has_unit ? q[mm.offp[j] + sj] : (R)0;
+      if (r == 0) qs[(mm.ooff[j] + sj) * tu + u] = has_unit ? q[mm.offp[j] + sj] : (R)0;
       as[(mm.ooff[j] + sj) * nt + tid] = (R)0;
     }
+  __syncthreads();
   // this split's range of the first axis, and of rows
   const int d0 = mm.dim[0], rps = mm.rows / d0;
   const int s0a = (int)((long long)r * d0 / rs), s0b = (int)((long long)(r + 1) * d0 / rs);
@@ -389,7 +391,7 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
   R p[4] = {(R)0, (R)0, (R)0, (R)0}, Wp[4] = {(R)1, (R)1, (R)1, (R)1};
 #pragma unroll
   for (int lv = 0; lv < 4; ++lv)
-    if (lv < K1) Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * nt + tid];
+    if (lv < K1) Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * tu + u];
   const int lrows = PERUNIT ? most : lbuf / rs / NCP;   // rows of one split's staging area (PERUNIT: all at once)
   R *Lr = Lbuf + (size_t)r * (PERUNIT ? 0 : lrows) * NCP;
   __shared__ __align__(8) unsigned long long bar[8];   // one per split
@@ -442,7 +444,7 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
           const int idx = (mm.ooff[lv] + sj) * nt + tid;
           const R wprev = lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1;
           as[idx] = fma(wprev, val, as[idx]);
-          if (lv > 0) p[lv > 0 ? lv - 1 : 0] = fma(qs[idx], val, p[lv > 0 ? lv - 1 : 0]);
+          if (lv > 0) p[lv > 0 ? lv - 1 : 0] = fma(qs[(mm.ooff[lv] + sj) * tu + u], val, p[lv > 0 ? lv - 1 : 0]);
           if (sj + 1 == mm.dim[lv]) {
             dig[lv] = 0;
             if (lv > 0) {
@@ -460,33 +462,42 @@ __device__ __forceinline__ void contract_rt(const BatchMember &mm, const R *__re
 #pragma unroll
       for (int lv = 0; lv < 4; ++lv)
         if (lv < K1 && lv >= top)
-          Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * nt + tid];
+          Wp[lv] = (lv > 0 ? Wp[lv > 0 ? lv - 1 : 0] : (R)1) * qs[(mm.ooff[lv] + dig[lv]) * tu + u];
     }
   }
-  // ---- add the splits' partial messages and write them out
-  __syncthreads();
-#pragma unroll
-  for (int c = 0; c < NCP; ++c) qs[c * nt + tid] = accc[c];   // the belief columns are no longer needed
+  // ---- add the splits' partial messages and write them out: the outer axes' from the accumulator
+  // columns, then the last axis' through the same columns (they are free by then)
   __syncthreads();
   const int so = mm.ooff[K1];   // outer states of this member
-  for (int i = tid; i < (so + NC) * tu; i += nt) {
+  for (int i = tid; i < so * tu; i += nt) {
     const int uu = i % tu, st = i / tu;
     if (uu >= tk.z) continue;
-    const R *col = st < so ? as + (size_t)st * nt + uu : qs + (size_t)(st - so) * nt + uu;
+    const R *col = as + (size_t)st * nt + uu;
     R sum = col[0];
     for (int k = 1; k < rs; ++k) sum += col[k * tu];
-    int j = K1, base = so;   // st >= so: the last axis
-    if (st < so) {
-      j = 0;
-      while (j + 1 < K1 && st >= mm.ooff[j + 1]) ++j;
-      base = mm.ooff[j];
-    }
-    ((R *)P.ellp)[((size_t)mi * P.NU + unit_s[uu]) * P.Sp + mm.offp[j] + (st - base)] = sum;
+    int j = 0;
+    while (j + 1 < K1 && st >= mm.ooff[j + 1]) ++j;
+    ((R *)P.ellp)[((size_t)mi * P.NU + unit_s[uu]) * P.Sp + mm.offp[j] + (st - mm.ooff[j])] = sum;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int c = 0; c < NCP; ++c) as[c * nt + tid] = accc[c];
+  __syncthreads();
+  for (int i = tid; i < NC * tu; i += nt) {
+    const int uu = i % tu, st = i / tu;
+    if (uu >= tk.z) continue;
+    const R *col = as + (size_t)st * nt + uu;
+    R sum = col[0];
+    for (int k = 1; k < rs; ++k) sum += col[k * tu];
+    ((R *)P.ellp)[((size_t)mi * P.NU + unit_s[uu]) * P.Sp + mm.offp[K1] + st] = sum;
   }
 }
 
-template <typename R, bool PERUNIT>
-__global__ void __launch_bounds__(256)
+// NCPMAX: the largest padded last axis among the model's members.  The forms for longer last axes
+// hold that many beliefs and accumulators in registers; a model that needs none of them gets a kernel
+// with half the registers, two CTAs of which share an SM.
+template <typename R, bool PERUNIT, int NCPMAX>
+__global__ void __launch_bounds__(256, NCPMAX <= 16 ? 2 : 1)
 bi_batch_contract_rt_kernel(BatchParams P, int cur, int first) {
   // (this form reads beliefs from its first instruction on, so it waits at once)
   bi_grid_wait();
@@ -494,8 +505,8 @@ bi_batch_contract_rt_kernel(BatchParams P, int cur, int first) {
   (void)first;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *Lbuf = reinterpret_cast<R *>(smem_raw);
-  R *qs = Lbuf + P.lbuf;
-  R *as = qs + (size_t)P.so_max * blockDim.x;
+  R *qs = Lbuf + P.lbuf;                                   // [so_max][tu] beliefs of the outer axes, per unit
+  R *as = qs + (size_t)P.so_max * P.tu;                     // [so_max][threads] message accumulators, per thread
   int *unit_s = reinterpret_cast<int *>(as + (size_t)P.so_max * blockDim.x);
   int mi = 0;
   while (mi + 1 < P.nmem && (int)blockIdx.x >= P.mem[mi + 1].task0) ++mi;
@@ -508,10 +519,10 @@ bi_batch_contract_rt_kernel(BatchParams P, int cur, int first) {
     case 8: contract_rt<R, 8, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
     case 12: contract_rt<R, 12, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
     case 16: contract_rt<R, 16, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 20: contract_rt<R, 20, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 24: contract_rt<R, 24, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 28: contract_rt<R, 28, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
-    case 32: contract_rt<R, 32, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 20: if constexpr (NCPMAX > 16) contract_rt<R, 20, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 24: if constexpr (NCPMAX > 16) contract_rt<R, 24, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 28: if constexpr (NCPMAX > 16) contract_rt<R, 28, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
+    case 32: if constexpr (NCPMAX > 16) contract_rt<R, 32, PERUNIT>(mm, slice, Lbuf, P.lbuf, qs, as, unit_s, P, cur, tk, mi); break;
     default: break;
   }
 }
@@ -752,7 +763,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   // (cnt == 0: every modality depends on a single factor; the update kernel alone does the work)
   std::sort(order, order + cnt, [&](int x, int y) { return h.mem[x].P_pad > h.mem[y].P_pad; });
   size_t max_slice = 0;
-  int max_m = 1, so_max = 1;
+  int max_m = 1, so_max = 1, ncp_max = 4;
   for (int j = 0; j < cnt; ++j) {
     const BiMember &mm = h.mem[order[j]];
     int gi = 0;
@@ -775,6 +786,7 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     bm.split = 1;
     if ((long long)rows * bm.ncp != mm.P_pad || bm.ncp > 32) return BI_ERR_UNSUPPORTED;
     so_max = std::max(so_max, so);
+    ncp_max = std::max(ncp_max, (int)bm.ncp);
     max_slice = std::max(max_slice, (size_t)mm.P_pad * sizeof(R));
     max_m = std::max(max_m, mm.m);
   }
@@ -786,14 +798,20 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     // row splits: enough warps for about two per scheduler when the batch is small
     if (tu == 32) rs = NU <= 32 * 4 * md->sm_count ? 8 : 4;
     else if (tu == 64) rs = 2;
-    // two columns per thread and outer state (at least 32 rows: the columns also carry the last
-    // axis' partial messages to the final sum), and a staging area of whole rows per split
-    // (48 KB in all at most); fewer splits, then fewer units, when that does not fit
+    // a column per unit (beliefs) and one per thread (message accumulators; at least 32 rows: they also
+    // carry the last axis' partial messages to the final sum) for every outer state, and a staging area
+    // of whole rows per split: 48 KB at most, and less when that lets a second CTA share the SM (the
+    // kernel's loops are chains of shared-memory round trips: with one CTA of eight warps per SM it
+    // issued on 29 % of the cycles); fewer splits, then fewer units, when even that does not fit
     P.so_max = std::max(so_max, 32);
     for (;;) {
-      P.lbuf = (int)std::min<size_t>(max_slice / sizeof(R), 48 * 1024 / sizeof(R));
-      P.lbuf = (std::max(P.lbuf, 32 * rs) + 32 * rs - 1) / (32 * rs) * (32 * rs);
-      csmem = ((size_t)P.lbuf + 2 * (size_t)P.so_max * tu * rs) * sizeof(R) + (size_t)tu * sizeof(int);
+      const size_t cols = ((size_t)P.so_max * tu + (size_t)P.so_max * tu * rs) * sizeof(R) + (size_t)tu * sizeof(int);
+      size_t stage = std::min<size_t>(max_slice, 48 * 1024);
+      const size_t half_sm = ((size_t)md->max_smem_optin + 1024) / 2 - 1024 - 1024;   // two CTAs, their reserved 1 KB each
+      if (ncp_max <= 16 && cols + stage > half_sm && cols + 8 * 1024 <= half_sm) stage = half_sm - cols;
+      P.lbuf = (int)(stage / sizeof(R));
+      P.lbuf = std::max(P.lbuf / (32 * rs) * (32 * rs), 32 * rs);
+      csmem = cols + (size_t)P.lbuf * sizeof(R);
       if (csmem <= (size_t)md->max_smem_optin - 1024) break;
       if (rs > 1) rs >>= 1;
       else if (tu > 32) tu >>= 1;
@@ -877,9 +895,10 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     bi_batch_identity_tasks_kernel<<<dim3(64, cnt), 256, 0, c.stream>>>(P, perm, task);
   else if (cnt > 0)
     bi_batch_bucket_kernel<<<cnt, 1024, 2 * max_m * sizeof(int32_t), c.stream>>>(P, c.obs, h.M, h.status, perm, task);
-  void (*contract)(BatchParams, int, int) = per_unit    ? bi_batch_contract_rt_kernel<R, true>
-                                       : any_shape ? bi_batch_contract_rt_kernel<R, false>
-                                                   : bi_batch_contract_kernel<R>;
+  void (*contract)(BatchParams, int, int) =
+      per_unit    ? (ncp_max <= 16 ? bi_batch_contract_rt_kernel<R, true, 16> : bi_batch_contract_rt_kernel<R, true, 32>)
+      : any_shape ? (ncp_max <= 16 ? bi_batch_contract_rt_kernel<R, false, 16> : bi_batch_contract_rt_kernel<R, false, 32>)
+                  : bi_batch_contract_kernel<R>;
   if (cudaFuncSetAttribute((const void *)contract, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csmem) !=
       cudaSuccess)
     return BI_ERR_CUDA;
