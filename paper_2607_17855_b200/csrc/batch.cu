@@ -597,9 +597,13 @@ __device__ __forceinline__ R lane_group_max(R v) {
 // the unit's part of shared memory.  The per-factor pass then reads shared memory and the transition
 // matrices (L1) only.  (With the L2 reads inside the per-factor loop every factor paid several
 // dependent round trips: 35 us per launch on 20 480 units, `long_scoreboard` 8.9 stall cycles per issue.)
-template <typename R, int ALGO, int LW>
-__global__ void __launch_bounds__(128)
+// FW (small batches, 32 lanes per unit): a CTA is one unit and one warp per factor, so the factors are
+// updated side by side instead of one after the other: with a few thousand units the kernel is a chain
+// of latencies per unit, not a matter of throughput.
+template <typename R, int ALGO, int LW, bool FW>
+__global__ void __launch_bounds__(FW ? 32 * BI_MAX_F : 128)
 bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs A) {
+  static_assert(!FW || LW == 32, "a warp per factor needs a whole warp per unit");
   __shared__ FactorInfo fi[BI_MAX_F];
   __shared__ unsigned char pfac[BI_MAX_F * 32];   // factor of each padded state position
   extern __shared__ __align__(16) unsigned char upd_smem[];
@@ -621,8 +625,8 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
   __syncthreads();
   bi_grid_wait();   // the contraction's messages (and, for the beliefs, everything before it)
   bi_grid_launch_dependents();
-  const int sub = threadIdx.x / LW, s = threadIdx.x % LW;
-  int unit = blockIdx.x * UPB + sub;
+  const int sub = FW ? 0 : threadIdx.x / LW, s = threadIdx.x % LW;
+  int unit = FW ? (int)blockIdx.x : blockIdx.x * UPB + sub;
   const bool live = unit < NU;    // dead groups shadow the last unit so that whole warps reach the shuffles
   if (!live) unit = NU - 1;
   const int a = unit / T, t = unit - a * T;
@@ -634,7 +638,7 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
   const int32_t *acp = A.act + ((ptrdiff_t)a * (T - 1) + (t - 1)) * F;
   R *base = reinterpret_cast<R *>(upd_smem) + (size_t)sub * 3 * Sp;   // [Sp] logit constants, [Sp] q(t-1), [Sp] q(t+1)
   R *qprev = base + Sp, *qnext = base + 2 * Sp;
-  for (int p = s; p < Sp; p += LW) {
+  for (int p = FW ? (int)threadIdx.x : s; p < Sp; p += FW ? (int)blockDim.x : LW) {
     const int f = pfac[p];
     const FactorInfo I = fi[f];
     const int sl = p - I.op;
@@ -656,8 +660,9 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
     qprev[p] = t > 0 ? qc[(size_t)(unit - 1) * Sp + p] : (R)0;
     qnext[p] = t + 1 < T ? qc[(size_t)(unit + 1) * Sp + p] : (R)0;
   }
-  __syncwarp();
-  for (int f = 0; f < F; ++f) {
+  if (FW) __syncthreads();
+  else __syncwarp();
+  for (int f = FW ? (int)(threadIdx.x >> 5) : 0; f < F; f += FW ? BI_MAX_F : 1) {
     const FactorInfo I = fi[f];
     const int n = I.n, np = I.np, op = I.op;
     R x = -bi_inf<R>();
@@ -911,12 +916,17 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   for (int f = 0; f < h.F; ++f) nmax = std::max(nmax, (int)h.n[f]);
   const int lw = nmax <= 8 ? 8 : nmax <= 16 ? 16 : 32, upb = 128 / lw;
   void (*update)(const BiDev *, BatchParams, UpdateArgs);
+  const bool fw = lw == 32 && NU <= 64 * md->sm_count;   // a few thousand units: a warp per factor (see the kernel)
   if (c.algo == BI_ALGO_VMP)
-    update = lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 8>
-                     : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 16> : bi_batch_update_kernel<R, BI_ALGO_VMP, 32>;
+    update = fw ? bi_batch_update_kernel<R, BI_ALGO_VMP, 32, true>
+                : lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 8, false>
+                          : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 16, false>
+                                     : bi_batch_update_kernel<R, BI_ALGO_VMP, 32, false>;
   else
-    update = lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 8>
-                     : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 16> : bi_batch_update_kernel<R, BI_ALGO_MMP, 32>;
+    update = fw ? bi_batch_update_kernel<R, BI_ALGO_MMP, 32, true>
+                : lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 8, false>
+                          : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 16, false>
+                                     : bi_batch_update_kernel<R, BI_ALGO_MMP, 32, false>;
   // every launch of the loop may be scheduled while its predecessor drains (see bi_grid_wait)
   cudaLaunchAttribute pdl[1];
   pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -936,9 +946,9 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
       cfg.dynamicSmemBytes = csmem;
       if (cudaLaunchKernelEx(&cfg, contract, P, cur, (int)(k == 0)) != cudaSuccess) return BI_ERR_CUDA;
     }
-    cfg.gridDim = dim3((unsigned)((NU + upb - 1) / upb));
-    cfg.blockDim = dim3(128);
-    cfg.dynamicSmemBytes = (size_t)upb * 3 * h.Sp * sizeof(R);
+    cfg.gridDim = dim3((unsigned)(fw ? NU : (NU + upb - 1) / upb));
+    cfg.blockDim = dim3((unsigned)(fw ? 32 * h.F : 128));
+    cfg.dynamicSmemBytes = (size_t)(fw ? 1 : upb) * 3 * h.Sp * sizeof(R);
     if (cudaLaunchKernelEx(&cfg, update, (const BiDev *)md->d, P, A) != cudaSuccess) return BI_ERR_CUDA;
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
