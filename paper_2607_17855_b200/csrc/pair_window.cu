@@ -17,6 +17,8 @@
 //     a single such group and units below 32 lanes keeps the row in registers),
 // and takes the softmax over the unit's lanes (table-driven exponential, shift by the largest binary
 // exponent).  Float64 handles, plain (undamped) update, trivial B-dependencies.
+#include <algorithm>
+
 #include "bi_internal.h"
 #include "tile3_filter_f64.cuh"   // the table-driven exponential, the integer softmax shift, rcp_fast
 
@@ -55,6 +57,10 @@ struct PairWinParams {
   int32_t *argmax_out;
   uint32_t *status;
   int32_t units;   // step slots per CTA (whole warps)
+  // staged slices of the two-factor groups: `nar` rows of `ls` entries each (the groups' largest first
+  // axis; their largest padded second axis plus one: an odd stride, so rows and columns are both read
+  // without bank conflicts), sized by the model and not by the lane count so that two CTAs fit an SM
+  int32_t nar, ls;
 };
 
 template <int LPU>
@@ -100,9 +106,11 @@ __device__ __forceinline__ void edge_dots(const R *__restrict__ mp, const R *__r
   df = f0 + f1;
 }
 
-template <int LPU, int ALGO>
-__global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams p) {
-  constexpr int LS = LPU + 1;   // row stride of the staged pair slice
+// MAXT: the most threads a launch of this instantiation has; windows of up to 320 threads get a
+// register budget under which two CTAs share an SM.
+template <int LPU, int ALGO, int MAXT>
+__global__ void __launch_bounds__(MAXT, MAXT <= 320 ? 2 : 1) bi_pair_window_kernel(const PairWinParams p) {
+  const int LS = p.ls, NAR = p.nar;   // row stride and rows of a staged slice
   constexpr bool LREG = LPU < 32;   // the slice's row stays in registers for the iterations
   extern __shared__ __align__(16) unsigned char smem_raw[];
   R *exp_tab = reinterpret_cast<R *>(smem_raw);                 // [EXP_TAB]
@@ -110,7 +118,7 @@ __global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams
   const int slot_sz = p.F * LPU, buf_sz = (p.units + 2) * slot_sz;
   R *cst = qb + 2 * buf_sz;                                     // [units][F][LPU] constants of the logits
   R *Ls = cst + p.units * slot_sz;                              // [units][ng][LPU][LS] the pair groups' summed slices, row-major
-  int32_t *aoff = reinterpret_cast<int32_t *>(Ls + (size_t)p.units * p.ng * LPU * LS);   // [units][F][2] matrix offsets of the two edges
+  int32_t *aoff = reinterpret_cast<int32_t *>(Ls + (((size_t)p.units * p.ng * NAR * LS + 1) & ~(size_t)1));   // [units][F][2] matrix offsets of the two edges
   for (int j = threadIdx.x; j < EXP_TAB; j += blockDim.x) exp_tab[j] = exp2((double)j * (1.0 / EXP_TAB));
 
   const int agent = blockIdx.x, g = p.G == 1 ? 0 : agent;
@@ -172,7 +180,7 @@ __global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams
 #pragma unroll
     for (int i = 0; i < LPU; ++i) {
       if (!a_ok) L[i] = 0.0;
-      Ls[(((size_t)tl * NG + gj) * LPU + s) * LS + i] = L[i];
+      if (s < NAR && i < LS) Ls[(((size_t)tl * NG + gj) * NAR + s) * LS + i] = L[i];
     }
   }
   // slots 0 and units + 1 (the neighbours of the window's ends): zeros, never weighted
@@ -207,28 +215,32 @@ __global__ void __launch_bounds__(512) bi_pair_window_kernel(const PairWinParams
         x += (has_prev ? dp : 0.0) + (has_next ? df : 0.0);
       }
       for (int gj = 0; gj < NG; ++gj) {
-        const R *Lg = Ls + ((size_t)tl * NG + gj) * LPU * LS;
+        const R *Lg = Ls + ((size_t)tl * NG + gj) * NAR * LS;
         if (f == p.fa[gj]) {          // row s of the group's slice with the other factor's belief
           const R *qo = qc + p.fb[gj] * LPU;
-          const R *rowp = Lg + (size_t)s * LS;   // (several groups, or 32-lane units: the row from the staged copy)
+          const R *rowp = Lg + (size_t)(s < NAR ? s : 0) * LS;   // (several groups, or 32-lane units: the row from the staged copy)
           const bool lreg = LREG && NG == 1;
           R v0 = 0.0, v1 = 0.0;
 #pragma unroll
           for (int i = 0; i < LPU; i += 2) {
-            R b0, b1;
-            lds2(qo + i, b0, b1);
-            v0 = fma(lreg ? L[i] : rowp[i], b0, v0); v1 = fma(lreg ? L[i + 1] : rowp[i + 1], b1, v1);
+            if (i + 1 < LS) {   // (a row holds LS - 1 entries, an even count)
+              R b0, b1;
+              lds2(qo + i, b0, b1);
+              v0 = fma(lreg ? L[i] : rowp[i], b0, v0); v1 = fma(lreg ? L[i + 1] : rowp[i + 1], b1, v1);
+            }
           }
           x += v0 + v1;
         } else if (f == p.fb[gj]) {   // column s
           const R *qo = qc + p.fa[gj] * LPU;
-          const R *col = Lg + s;
+          const R *col = Lg + (s < LS - 1 ? s : 0);
           R v0 = 0.0, v1 = 0.0;
 #pragma unroll
           for (int i = 0; i < LPU; i += 2) {
-            R a0, a1;
-            lds2(qo + i, a0, a1);
-            v0 = fma(col[i * LS], a0, v0); v1 = fma(col[(i + 1) * LS], a1, v1);
+            if (i < NAR) {      // (NAR rows, an even count)
+              R a0, a1;
+              lds2(qo + i, a0, a1);
+              v0 = fma(col[i * LS], a0, v0); v1 = fma(col[(i + 1) * LS], a1, v1);
+            }
           }
           x += v0 + v1;
         }
@@ -264,10 +276,14 @@ int launch(PairWinParams &p, const bi_model *md, cudaStream_t stream) {
   if (threads > 512) return BI_ERR_UNSUPPORTED;   // (the kernel's register budget is set for this)
   p.units = threads / LPU;
   const size_t slot = (size_t)p.F * LPU;
-  size_t elems = EXP_TAB + 2 * (p.units + 2) * slot + p.units * slot + (size_t)p.units * p.ng * LPU * (LPU + 1);
+  size_t elems = EXP_TAB + 2 * (p.units + 2) * slot + p.units * slot + (((size_t)p.units * p.ng * p.nar * p.ls + 1) & ~(size_t)1);
   const size_t bytes = elems * sizeof(R) + (size_t)p.units * p.F * 2 * sizeof(int32_t) + 16;
   if (bytes > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
-  auto kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP> : bi_pair_window_kernel<LPU, BI_ALGO_MMP>;
+  void (*kern)(const PairWinParams);
+  if (threads <= 320)
+    kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 320> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 320>;
+  else
+    kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 512> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 512>;
   if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
     cudaGetLastError();
     return BI_ERR_CUDA;
@@ -331,6 +347,11 @@ int bi_launch_pair_window(const BiCall &c, bi_model *mut) {
     }
   }
   p.g2_begin[p.ng] = n2;
+  p.nar = 2; p.ls = 3;
+  for (int gj = 0; gj < p.ng; ++gj) {
+    p.nar = std::max(p.nar, (p.na[gj] + 1) & ~1);
+    p.ls = std::max(p.ls, p.npb[gj] + 1);
+  }
   p.obs = c.obs; p.act = c.act; p.q_init = c.q_init; p.lnprior = (const R *)c.lnprior;
   p.q_out = c.q_out; p.logq_out = c.logq_out; p.argmax_out = c.argmax_out; p.status = h.status;
   int rc;
