@@ -600,7 +600,10 @@ __device__ __forceinline__ R lane_group_max(R v) {
 // FW (small batches, 32 lanes per unit): a CTA is one unit and one warp per factor, so the factors are
 // updated side by side instead of one after the other: with a few thousand units the kernel is a chain
 // of latencies per unit, not a matter of throughput.
-template <typename R, int ALGO, int LW, bool FW>
+// FINAL: the call's last iteration (the only one that writes outputs); DAMPED: the damped update.  Both
+// are instantiations of their own: the plain iteration in between runs sixteen times a call and is
+// bound by instruction issue, so it carries none of their code.
+template <typename R, int ALGO, int LW, bool FW, bool FINAL, bool DAMPED>
 __global__ void __launch_bounds__(FW ? 32 * BI_MAX_F : 128)
 bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs A) {
   static_assert(!FW || LW == 32, "a warp per factor needs a whole warp per unit");
@@ -682,7 +685,7 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
       }
       x += (t > 0 ? dp : (R)0) + (t + 1 < T ? df : (R)0);
     }
-    if (A.xprev) {
+    if (DAMPED) {
       // damped step on the logits; the first one starts from ln q of the starting belief (uniform: a
       // constant, taken as 0)
       R *xp = (R *)A.xprev + (size_t)unit * Sp + op;
@@ -695,12 +698,12 @@ bi_batch_update_kernel(const BiDev *__restrict__ mdp, BatchParams P, UpdateArgs 
       }
     }
     // any shift near the maximum keeps the exponentials in range; the last iterate takes the exact one
-    const R mx = A.final ? lane_group_max<LW>(x) : (R)lane_group_max<LW>((float)x);
+    const R mx = FINAL ? lane_group_max<LW>(x) : (R)lane_group_max<LW>((float)x);
     const R e = s < n ? bi_exp_inline(x - mx) : (R)0;
     const R z = lane_group_sum<LW>(e);
     const R q = e * bi_rcp(z);
     if (live && s < np) qn[op + s] = q;
-    if (A.final) {
+    if (FINAL) {
       if (live && s < n) {
         A.q_out[(size_t)unit * S + I.off + s] = (float)q;
         if (A.logq_out) A.logq_out[(size_t)unit * S + I.off + s] = (float)(x - mx - bi_log(z));
@@ -915,18 +918,23 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
   int nmax = 1;
   for (int f = 0; f < h.F; ++f) nmax = std::max(nmax, (int)h.n[f]);
   const int lw = nmax <= 8 ? 8 : nmax <= 16 ? 16 : 32, upb = 128 / lw;
-  void (*update)(const BiDev *, BatchParams, UpdateArgs);
+  typedef void (*UpdateKernel)(const BiDev *, BatchParams, UpdateArgs);
   const bool fw = lw == 32 && NU <= 64 * md->sm_count;   // a few thousand units: a warp per factor (see the kernel)
-  if (c.algo == BI_ALGO_VMP)
-    update = fw ? bi_batch_update_kernel<R, BI_ALGO_VMP, 32, true>
-                : lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 8, false>
-                          : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_VMP, 16, false>
-                                     : bi_batch_update_kernel<R, BI_ALGO_VMP, 32, false>;
-  else
-    update = fw ? bi_batch_update_kernel<R, BI_ALGO_MMP, 32, true>
-                : lw == 8 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 8, false>
-                          : lw == 16 ? bi_batch_update_kernel<R, BI_ALGO_MMP, 16, false>
-                                     : bi_batch_update_kernel<R, BI_ALGO_MMP, 32, false>;
+  const bool damped = A.xprev != nullptr;
+  auto pick = [&](bool fin) -> UpdateKernel {
+#define BI_UPD(AL, LWV, FWV) \
+    (fin ? (damped ? (UpdateKernel)bi_batch_update_kernel<R, AL, LWV, FWV, true, true>   \
+                   : (UpdateKernel)bi_batch_update_kernel<R, AL, LWV, FWV, true, false>) \
+         : (damped ? (UpdateKernel)bi_batch_update_kernel<R, AL, LWV, FWV, false, true>  \
+                   : (UpdateKernel)bi_batch_update_kernel<R, AL, LWV, FWV, false, false>))
+    if (c.algo == BI_ALGO_VMP)
+      return fw ? BI_UPD(BI_ALGO_VMP, 32, true)
+                : lw == 8 ? BI_UPD(BI_ALGO_VMP, 8, false) : lw == 16 ? BI_UPD(BI_ALGO_VMP, 16, false) : BI_UPD(BI_ALGO_VMP, 32, false);
+    return fw ? BI_UPD(BI_ALGO_MMP, 32, true)
+              : lw == 8 ? BI_UPD(BI_ALGO_MMP, 8, false) : lw == 16 ? BI_UPD(BI_ALGO_MMP, 16, false) : BI_UPD(BI_ALGO_MMP, 32, false);
+#undef BI_UPD
+  };
+  const UpdateKernel update_mid = pick(false), update_last = pick(true);
   // every launch of the loop may be scheduled while its predecessor drains (see bi_grid_wait)
   cudaLaunchAttribute pdl[1];
   pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -949,7 +957,8 @@ int launch_batch_t(const BiCall &c, bi_model *mut) {
     cfg.gridDim = dim3((unsigned)(fw ? NU : (NU + upb - 1) / upb));
     cfg.blockDim = dim3((unsigned)(fw ? 32 * h.F : 128));
     cfg.dynamicSmemBytes = (size_t)(fw ? 1 : upb) * 3 * h.Sp * sizeof(R);
-    if (cudaLaunchKernelEx(&cfg, update, (const BiDev *)md->d, P, A) != cudaSuccess) return BI_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, A.final ? update_last : update_mid, (const BiDev *)md->d, P, A) != cudaSuccess)
+      return BI_ERR_CUDA;
   }
   if (cudaGetLastError() != cudaSuccess) return BI_ERR_CUDA;
   mut->launches += cnt > 0 ? 2 + 2 * c.K : 1 + c.K;
