@@ -20,7 +20,11 @@
 //      is left of them is a matrix of at most 32 x 32 over their first two
 //      axes: the factor's warp sums its rows or columns itself), rank-1 slices
 //      and phase B's rows, all in a fixed order; softmax, next beliefs (and the
-//      outputs after the last iteration).
+//      outputs after the last iteration).  What a factor adds up is a list of
+//      operations over shared memory, built once per launch, so that an iteration
+//      reads one 16-byte descriptor per operation instead of following the model's
+//      description; float64 calls take the softmax of every iteration but the last
+//      with the table-driven exponential and an integer reduction for the shift.
 // Models without a group of rank 3 or more skip phase A, models without one of rank 4 or
 // more phase B, each with its barrier.
 //
@@ -30,6 +34,7 @@
 
 #include "bi_internal.h"
 #include "tile3.cuh"
+#include "tile3_filter_f64.cuh"
 
 namespace {
 
@@ -53,6 +58,8 @@ struct CtaGeom {   // element offsets (units of R) into dynamic shared memory
   // rank-3 group's first partial tensor; its offset, row stride and the level that describes it
   int mat_off[BI_MAX_GROUPS], mat_ls[BI_MAX_GROUPS], mat_lev[BI_MAX_GROUPS];
   int deep;                       // any group of rank >= 4: phase B and its barrier are needed
+  int ops, maxops, nops, exptab;  // phase C's operation lists [F][maxops] (16 bytes each), their lengths, the exp table
+  int prior_tps;                  // threads that share one state when the prior is formed (1, 2 or 4)
   int total_bytes;
 };
 
@@ -175,29 +182,50 @@ __device__ __forceinline__ void last_level(const BiLevel &lv, const R *L, const 
   __syncwarp();
 }
 
-// rank-2 group, matrix L[r][c] at row stride ls: the messages to its first axis (this lane's row) and
-// to its second axis (this lane's column)
+// Phase C's operations.  ROW: this lane's row of a matrix against a belief vector, sum_c L[lane][c] q[c]
+// (count = padded columns / 4); COL: this lane's column, sum_r q[r] L[r][lane] (count = rows); ADD:
+// sum_i base[i * stride + lane] (count terms: per-warp partial sums, a rank-1 slice, phase B's row).
+enum { CTA_OP_ROW = 0, CTA_OP_COL = 1, CTA_OP_ADD = 2 };
+
 template <typename R>
-__device__ __forceinline__ R matrix_row_dot(const R *L, int ls, int row, const R *q1, int npad4) {
-  R v0 = (R)0, v1 = (R)0;
-  for (int c4 = 0; c4 < npad4; ++c4) {
-    const Vec4<R> x = lds4(L + row * ls + 4 * c4);
-    const Vec4<R> qq = lds4(q1 + 4 * c4);
-    v0 = fma(x.x, qq.x, v0); v1 = fma(x.y, qq.y, v1);
-    v0 = fma(x.z, qq.z, v0); v1 = fma(x.w, qq.w, v1);
+__device__ __forceinline__ R op_row_dot(const R *row, const R *q, int npad4) {
+  R v0 = (R)0, v1 = (R)0, v2 = (R)0, v3 = (R)0;
+  int c4 = 0;
+  for (; c4 + 1 < npad4; c4 += 2) {   // loads of two vectors first, then four independent chains
+    const Vec4<R> x = lds4(row + 4 * c4), y = lds4(row + 4 * c4 + 4);
+    const Vec4<R> qx = lds4(q + 4 * c4), qy = lds4(q + 4 * c4 + 4);
+    v0 = fma(x.x, qx.x, v0); v1 = fma(x.y, qx.y, v1); v2 = fma(x.z, qx.z, v2); v3 = fma(x.w, qx.w, v3);
+    v0 = fma(y.x, qy.x, v0); v1 = fma(y.y, qy.y, v1); v2 = fma(y.z, qy.z, v2); v3 = fma(y.w, qy.w, v3);
   }
-  return v0 + v1;
+  if (c4 < npad4) {
+    const Vec4<R> x = lds4(row + 4 * c4);
+    const Vec4<R> qx = lds4(q + 4 * c4);
+    v0 = fma(x.x, qx.x, v0); v1 = fma(x.y, qx.y, v1); v2 = fma(x.z, qx.z, v2); v3 = fma(x.w, qx.w, v3);
+  }
+  return (v0 + v1) + (v2 + v3);
 }
 template <typename R>
-__device__ __forceinline__ R matrix_col_dot(const R *L, int ls, int col, const R *q0, int nrows) {
-  R m0 = (R)0, m1 = (R)0;
+__device__ __forceinline__ R op_col_dot(const R *col, int ls, const R *q, int nrows) {
+  R m0 = (R)0, m1 = (R)0, m2 = (R)0, m3 = (R)0;
   int r = 0;
-  for (; r + 1 < nrows; r += 2) {
-    m0 = fma(q0[r], L[r * ls + col], m0);
-    m1 = fma(q0[r + 1], L[(r + 1) * ls + col], m1);
+  for (; r + 3 < nrows; r += 4) {
+    const Vec4<R> w = lds4(q + r);
+    const R a = col[r * ls], b = col[(r + 1) * ls], c = col[(r + 2) * ls], d = col[(r + 3) * ls];
+    m0 = fma(w.x, a, m0); m1 = fma(w.y, b, m1); m2 = fma(w.z, c, m2); m3 = fma(w.w, d, m3);
   }
-  if (r < nrows) m0 = fma(q0[r], L[r * ls + col], m0);
-  return m0 + m1;
+  for (; r < nrows; ++r) m0 = fma(q[r], col[r * ls], m0);
+  return (m0 + m1) + (m2 + m3);
+}
+
+// sum over the warp of values that are zero in lanes n and above
+template <typename R>
+__device__ __forceinline__ R warp_sum_first(R v, int n) {
+  if (n > 16) v += __shfl_xor_sync(0xffffffffu, v, 16);
+  if (n > 8) v += __shfl_xor_sync(0xffffffffu, v, 8);
+  if (n > 4) v += __shfl_xor_sync(0xffffffffu, v, 4);
+  v += __shfl_xor_sync(0xffffffffu, v, 2);
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  return v;
 }
 
 // Non-trivial B-dependencies (a transition that reads several factors' previous states): the prior of
@@ -253,6 +281,44 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
   for (int i = tid; i < 2 * Sp; i += NT) cur[i] = (R)0;   // q0 and q1 are adjacent
   for (int i = tid; i < NG * Sp; i += NT) ellg[i] = (R)0;  // entries of factors outside a group stay zero
   for (int i = sm.vtot_begin + tid; i < sm.vtot_end; i += NT) smem[i] = (R)0;
+  int4 *ops = reinterpret_cast<int4 *>(smem + sm.ops);     // [F][maxops]
+  int32_t *nops = reinterpret_cast<int32_t *>(smem + sm.nops);
+  if (tid < F) {   // what phase C adds up for factor tid, in the order it is added
+    const int f = tid;
+    int4 *o = ops + f * sm.maxops;
+    int c = 0;
+    for (unsigned mk = sm.f_cls[f]; mk; mk &= mk - 1) {   // per-warp partial sums: one operation per run of warps
+      const int cls = __ffs(mk) - 1;
+      const unsigned wm = (unsigned)sm.cls_wmask[cls];
+      for (int w = 0; w < NW;) {
+        if (!((wm >> w) & 1)) { ++w; continue; }
+        int e = w;
+        while (e < NW && ((wm >> e) & 1)) ++e;
+        o[c++] = make_int4(CTA_OP_ADD | ((e - w) << 8), sm.part + (cls * NW + w) * 32, 32, 0);
+        w = e;
+      }
+    }
+    for (unsigned mk = sm.f_m0[f]; mk; mk &= mk - 1) {   // groups of rank 2 or 3 with f as first axis
+      const int gi = __ffs(mk) - 1;
+      const BiLevel &lv = md.grp[gi].lev[sm.mat_lev[gi]];
+      o[c++] = make_int4(CTA_OP_ROW | (lv.last_npad4 << 8), sm.mat_off[gi], sm.mat_ls[gi], lv.last_qoff);
+    }
+    for (unsigned mk = sm.f_m1[f]; mk; mk &= mk - 1) {   // ... and as second axis
+      const int gi = __ffs(mk) - 1;
+      const BiLevel &lv = md.grp[gi].lev[sm.mat_lev[gi]];
+      o[c++] = make_int4(CTA_OP_COL | (lv.nrows << 8), sm.mat_off[gi], sm.mat_ls[gi], lv.qoff[0]);
+    }
+    for (unsigned mk = sm.f_r1[f]; mk; mk &= mk - 1) o[c++] = make_int4(CTA_OP_ADD | (1 << 8), sm.Lst[__ffs(mk) - 1], 0, 0);
+    for (unsigned mk = sm.f_deep[f]; mk; mk &= mk - 1)
+      o[c++] = make_int4(CTA_OP_ADD | (1 << 8), sm.ellg + (__ffs(mk) - 1) * Sp + md.offp[f], 0, 0);
+    nops[f] = c;
+  }
+  const double *exp_tab = nullptr;
+  if constexpr (sizeof(R) == 8) {
+    double *tab = reinterpret_cast<double *>(smem + sm.exptab);
+    for (int j = tid; j < tile3_f64::EXP_TAB; j += NT) tab[j] = exp2((double)j * (1.0 / tile3_f64::EXP_TAB));
+    exp_tab = tab;
+  }
   __syncthreads();
   const bool from_prev = q_prev != nullptr || carry_in != nullptr;
   if (from_prev) {  // continued filtering: the belief of the step before the first
@@ -283,32 +349,42 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
         }
         if (lane == 0) lpri[idx] = lp;
       }
-    } else
-    for (int idx = tid; idx < Sp; idx += NT) {
-      int f = 0;
-      while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
-      const int s = idx - md.offp[f], n = md.n[f];
-      R lp = (R)0;
-      if (s < n) {
-        if (t == 0 && !from_prev) {
-          lp = __ldg((const R *)md.logD[f] + (size_t)g * md.Dstride[f] + s);
-        } else {
+    } else if (t == 0 && !from_prev) {
+      for (int idx = tid; idx < Sp; idx += NT) {
+        int f = 0;
+        while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+        const int s = idx - md.offp[f];
+        lpri[idx] = s < md.n[f] ? __ldg((const R *)md.logD[f] + (size_t)g * md.Dstride[f] + s) : (R)0;
+      }
+    } else {
+      // tps threads of one warp share a state: each takes every tps-th term of the row's product with
+      // the previous belief (its loads are all in flight together), then the partial sums are added
+      const int tps = sm.prior_tps, per = NT / tps, sub = tid % tps;
+      for (int base = 0; base < Sp; base += per) {
+        const int idx = base + tid / tps;
+        int f = 0;
+        while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
+        const int s = idx - md.offp[f], n = md.n[f];
+        const bool live = idx < Sp && s < n;
+        R p0 = (R)0, p1 = (R)0;
+        if (live) {
           const int ur = t == 0 ? __ldg(act_prev + (size_t)a * F + f)
                                 : __ldg(act + ((size_t)a * (T - 1) + (t - 1)) * F + f);
           const int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
           const R *row = (const R *)md.Bf[f] + (size_t)g * md.Bstride[f] + ((size_t)u * n + s) * md.npad[f];
           const R *qf = cur + md.offp[f];
-          R p0 = (R)0, p1 = (R)0;
-          int r = 0;
-          for (; r + 1 < n; r += 2) {
+          int r = sub;
+#pragma unroll 4
+          for (; r + tps < n; r += 2 * tps) {
             p0 = fma(__ldg(row + r), qf[r], p0);
-            p1 = fma(__ldg(row + r + 1), qf[r + 1], p1);
+            p1 = fma(__ldg(row + r + tps), qf[r + tps], p1);
           }
           if (r < n) p0 = fma(__ldg(row + r), qf[r], p0);
-          lp = bi_log(bi_max(p0 + p1, (R)BI_EPS));
         }
+        R pr = p0 + p1;
+        for (int d = 1; d < tps; d <<= 1) pr += __shfl_xor_sync(0xffffffffu, pr, d);
+        if (idx < Sp && sub == 0) lpri[idx] = live ? bi_log(bi_max(pr, (R)BI_EPS)) : (R)0;
       }
-      lpri[idx] = lp;
     }
     // the step's summed slices, rows at their padded stride
     for (int gi = 0; gi < NG; ++gi) {
@@ -385,33 +461,49 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
         R x = -bi_inf<R>();
         if (lane < n) {
           R x0 = lpri[op + lane], x1 = (R)0;
-          for (unsigned mk = sm.f_cls[f]; mk; mk &= mk - 1) {
-            const int cls = __ffs(mk) - 1;
-            const R *pc = part + (size_t)cls * NW * 32 + lane;
-            for (unsigned wm = (unsigned)sm.cls_wmask[cls]; wm; wm &= wm - 1) x1 += pc[(__ffs(wm) - 1) * 32];
+          const int4 *o = ops + f * sm.maxops;
+          const int no = nops[f];
+          for (int j = 0; j < no; ++j) {
+            const int4 e = o[j];
+            const int cnt = e.x >> 8;
+            const R *base = smem + e.y;
+            switch (e.x & 255) {
+              case CTA_OP_ROW: x0 += op_row_dot<R>(base + lane * e.z, cur + e.w, cnt); break;
+              case CTA_OP_COL: x1 += op_col_dot<R>(base + lane, e.z, cur + e.w, cnt); break;
+              default: {
+                R s0 = base[lane];
+                for (int i = 1; i < cnt; ++i) s0 += base[i * e.z + lane];
+                x1 += s0;
+              }
+            }
           }
-          for (unsigned mk = sm.f_m0[f]; mk; mk &= mk - 1) {   // groups of rank 2 or 3 with f as first axis
-            const int gi = __ffs(mk) - 1;
-            const BiLevel &lv = md.grp[gi].lev[sm.mat_lev[gi]];
-            x0 += matrix_row_dot<R>(smem + sm.mat_off[gi], sm.mat_ls[gi], lane, cur + lv.last_qoff, lv.last_npad4);
-          }
-          for (unsigned mk = sm.f_m1[f]; mk; mk &= mk - 1) {   // ... and as second axis
-            const int gi = __ffs(mk) - 1;
-            const BiLevel &lv = md.grp[gi].lev[sm.mat_lev[gi]];
-            x1 += matrix_col_dot<R>(smem + sm.mat_off[gi], sm.mat_ls[gi], lane, cur + lv.qoff[0], lv.nrows);
-          }
-          for (unsigned mk = sm.f_r1[f]; mk; mk &= mk - 1) x0 += smem[sm.Lst[__ffs(mk) - 1] + lane];
-          for (unsigned mk = sm.f_deep[f]; mk; mk &= mk - 1) x1 += ellg[(size_t)(__ffs(mk) - 1) * Sp + op + lane];
           x = x0 + x1;
           if (xp) {   // damped step on the logits; xp: the previous iterate's
             x = fma(lam, x, ((R)1 - lam) * xp[op + lane]);
             xp[op + lane] = x;
           }
         }
-        const R mx = final ? warp_max(x) : (R)warp_max((float)x);
-        const R e = lane < n ? bi_exp_inline(x - mx) : (R)0;
-        const R z = warp_sum(e);
-        const R q = e * bi_rcp(z);
+        R mx, e, z, q;
+        bool fast = false;
+        if constexpr (sizeof(R) == 8) fast = !final;
+        if (fast) {
+          // every iteration but the last: exponentials relative to the largest binary exponent among the
+          // logits (one integer reduction; every e lies in [0, 2)) and a reciprocal good to 1e-13
+          if constexpr (sizeof(R) == 8) {
+            int kx;
+            const double mant = tile3_f64::exp_mant(lane < n ? x : 0.0, exp_tab, kx);
+            const int km = __reduce_max_sync(0xffffffffu, lane < n ? kx : INT_MIN);
+            e = lane < n ? tile3_f64::exp_scale(mant, (kx >> tile3_f64::EXP_BITS) - (km >> tile3_f64::EXP_BITS)) : 0.0;
+            z = warp_sum_first(e, n);
+            q = e * tile3_f64::rcp_fast(z);
+          }
+          mx = (R)0;
+        } else {
+          mx = warp_max(x);
+          e = lane < n ? bi_exp_inline(x - mx) : (R)0;
+          z = warp_sum(e);
+          q = e * bi_rcp(z);
+        }
         if (lane < md.npad[f]) nxt[op + lane] = lane < n ? q : (R)0;
         if (final) {
           const size_t ob = (size_t)a * T + t;
@@ -509,6 +601,24 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
     }
   }
   sm.part = o; o += std::max(1, sm.ncls) * NW * 32;
+  {  // phase C's operation lists: the longest decides the row length
+    sm.maxops = 1;
+    for (int f = 0; f < h.F; ++f) {
+      int c = __builtin_popcount(sm.f_m0[f]) + __builtin_popcount(sm.f_m1[f]) + __builtin_popcount(sm.f_r1[f]) +
+              __builtin_popcount(sm.f_deep[f]);
+      for (int cls = 0; cls < sm.ncls; ++cls) {
+        if (!((sm.f_cls[f] >> cls) & 1)) continue;
+        const unsigned wm = (unsigned)sm.cls_wmask[cls];
+        for (int w = 0; w < NW; ++w) c += ((wm >> w) & 1) && (w == 0 || !((wm >> (w - 1)) & 1));
+      }
+      sm.maxops = std::max(sm.maxops, c);
+    }
+    o = (o + 3) & ~3;
+    sm.ops = o; o += (int)((size_t)h.F * sm.maxops * 16 / sizeof(R));
+    sm.nops = o; o += bi_pad4(h.F);
+    sm.exptab = o;
+    if (sizeof(R) == 8) o += tile3_f64::EXP_TAB;
+  }
   sm.vtot_begin = o;
   for (int gi = 0; gi < BI_MAX_GROUPS; ++gi) sm.V[gi][0] = sm.V[gi][1] = o;
   for (int gi = 0; gi < h.ngroups; ++gi) {
@@ -544,6 +654,7 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
       sm.mat_lev[gi] = 1;
     }
   }
+  sm.prior_tps = 4 * h.Sp <= NT ? 4 : 2 * h.Sp <= NT ? 2 : 1;
   sm.total_bytes = (int)((size_t)o * sizeof(R));
   if ((size_t)o * sizeof(R) > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
 
