@@ -16,6 +16,7 @@
 namespace {
 
 constexpr int kTT = 16;   // steps accumulated per pass over a modality's outcomes
+constexpr int kTTP = kTT + 4;   // row stride of the staged vectors (an outcome's kTT weights; padded against bank conflicts when staging)
 
 struct SoftMember {
   const void *src;     // ln A of one modality in the layout being produced: [G][m][P]
@@ -32,56 +33,72 @@ struct SoftJob {
 
 // kEPT slice elements of one agent per thread; a modality's outcomes are read
 // once per block of kTT steps and weighted into kTT accumulators per element
-// (a step's weight is one broadcast shared-memory load for kEPT multiply-adds).
+// (four steps' weights are one broadcast shared-memory load for 4 kEPT multiply-adds).
 // The vectors are converted to the arithmetic type once, when they are staged.
-template <typename R, int kEPT>
-__global__ void __launch_bounds__(128) bi_soft_slices_kernel(const SoftJob J) {
-  extern __shared__ __align__(16) unsigned char w_raw[];
-  R *w_s = reinterpret_cast<R *>(w_raw);   // [kTT][Mtot] this agent's vectors for the current steps
-  const int a = blockIdx.y;
-  const int e0 = blockIdx.x * (kEPT * 128) + threadIdx.x;   // elements e0 + j * 128
-  R *dst = (R *)J.dst + (size_t)a * J.T * J.P;
-  for (int t0 = 0; t0 < J.T; t0 += kTT) {
-    const int nt = min(kTT, J.T - t0);
-    __syncthreads();
-    for (int i = threadIdx.x; i < nt * J.Mtot; i += blockDim.x)
-      w_s[i] = (R)J.soft[((size_t)a * J.T + t0) * J.Mtot + i];
-    for (int i = nt * J.Mtot + threadIdx.x; i < kTT * J.Mtot; i += blockDim.x) w_s[i] = (R)0;
-    __syncthreads();
-    R acc[kEPT][kTT];
+// One block of KT steps (nt of them real) starting at step t0.
+template <typename R, int kEPT, int KT>
+__device__ __forceinline__ void soft_block(const SoftJob &J, R *w_s, int a, int e0, R *dst, int t0, int nt) {
+  __syncthreads();
+  for (int i = threadIdx.x; i < KT * J.Mtot; i += blockDim.x) {   // (consecutive threads read consecutive floats)
+    const int tt = i / J.Mtot, o = i - tt * J.Mtot;
+    w_s[o * kTTP + tt] = tt < nt ? (R)J.soft[((size_t)a * J.T + t0) * J.Mtot + i] : (R)0;
+  }
+  __syncthreads();
+  R acc[kEPT][KT];
 #pragma unroll
-    for (int j = 0; j < kEPT; ++j)
+  for (int j = 0; j < kEPT; ++j)
 #pragma unroll
-      for (int tt = 0; tt < kTT; ++tt) acc[j][tt] = (R)0;
-    for (int mi = 0; mi < J.nmem; ++mi) {
-      const SoftMember &mm = J.mem[mi];
-      const R *src = (const R *)mm.src + (size_t)a * mm.gstride;
-      for (int o = 0; o < mm.m; ++o) {
-        R la[kEPT];
+    for (int tt = 0; tt < KT; ++tt) acc[j][tt] = (R)0;
+  for (int mi = 0; mi < J.nmem; ++mi) {
+    const SoftMember &mm = J.mem[mi];
+    const R *src = (const R *)mm.src + (size_t)a * mm.gstride;
+    for (int o = 0; o < mm.m; ++o) {
+      R la[kEPT];
+#pragma unroll
+      for (int j = 0; j < kEPT; ++j) {
+        const int e = e0 + j * 128;
+        la[j] = e < J.P ? __ldg(src + (size_t)o * J.P + e) : (R)0;
+      }
+      const Vec4<R> *wo = reinterpret_cast<const Vec4<R> *>(w_s + (size_t)(mm.moff + o) * kTTP);
+#pragma unroll
+      for (int t4 = 0; t4 < KT / 4; ++t4) {
+        const Vec4<R> wv = wo[t4];
 #pragma unroll
         for (int j = 0; j < kEPT; ++j) {
-          const int e = e0 + j * 128;
-          la[j] = e < J.P ? __ldg(src + (size_t)o * J.P + e) : (R)0;
+          acc[j][4 * t4 + 0] = fma(wv.x, la[j], acc[j][4 * t4 + 0]);
+          acc[j][4 * t4 + 1] = fma(wv.y, la[j], acc[j][4 * t4 + 1]);
+          acc[j][4 * t4 + 2] = fma(wv.z, la[j], acc[j][4 * t4 + 2]);
+          acc[j][4 * t4 + 3] = fma(wv.w, la[j], acc[j][4 * t4 + 3]);
         }
-        const R *wo = w_s + mm.moff + o;
-#pragma unroll
-        for (int tt = 0; tt < kTT; ++tt) {
-          const R wv = wo[tt * J.Mtot];
-#pragma unroll
-          for (int j = 0; j < kEPT; ++j) acc[j][tt] = fma(wv, la[j], acc[j][tt]);
-        }
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < kEPT; ++j) {
-      const int e = e0 + j * 128;
-      if (e < J.P) {
-#pragma unroll
-        for (int tt = 0; tt < kTT; ++tt)
-          if (tt < nt) dst[(size_t)(t0 + tt) * J.P + e] = acc[j][tt];
       }
     }
   }
+#pragma unroll
+  for (int j = 0; j < kEPT; ++j) {
+    const int e = e0 + j * 128;
+    if (e < J.P) {
+#pragma unroll
+      for (int tt = 0; tt < KT; ++tt)
+        if (tt < nt) dst[(size_t)(t0 + tt) * J.P + e] = acc[j][tt];
+    }
+  }
+}
+
+// Whole blocks of kTT steps, then the rest in the shortest block (a multiple of four steps) that holds it.
+template <typename R, int kEPT>
+__global__ void __launch_bounds__(128, kEPT * sizeof(R) <= 24 ? 4 : 3) bi_soft_slices_kernel(const SoftJob J) {
+  extern __shared__ __align__(16) unsigned char w_raw[];
+  R *w_s = reinterpret_cast<R *>(w_raw);   // [Mtot][kTTP] this agent's vectors for the current steps, outcome-major
+  const int a = blockIdx.y;
+  const int e0 = blockIdx.x * (kEPT * 128) + threadIdx.x;   // elements e0 + j * 128
+  R *dst = (R *)J.dst + (size_t)a * J.T * J.P;
+  int t0 = 0;
+  for (; t0 + kTT <= J.T; t0 += kTT) soft_block<R, kEPT, kTT>(J, w_s, a, e0, dst, t0, kTT);
+  const int rem = J.T - t0;
+  if (rem > 12) soft_block<R, kEPT, 16>(J, w_s, a, e0, dst, t0, rem);
+  else if (rem > 8) soft_block<R, kEPT, 12>(J, w_s, a, e0, dst, t0, rem);
+  else if (rem > 4) soft_block<R, kEPT, 8>(J, w_s, a, e0, dst, t0, rem);
+  else if (rem > 0) soft_block<R, kEPT, 4>(J, w_s, a, e0, dst, t0, rem);
 }
 
 __global__ void bi_soft_step_index_kernel(int32_t *obs, int N, int T, int M) {
@@ -99,7 +116,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
   const BiDev &h = model->h;
   int moff[BI_MAX_M], Mtot = 0;
   for (int i = 0; i < h.M; ++i) { moff[i] = Mtot; Mtot += h.m[i]; }
-  if ((size_t)kTT * Mtot * sizeof(R) > 96 * 1024) return BI_ERR_UNSUPPORTED;
+  if ((size_t)kTTP * Mtot * sizeof(R) > 96 * 1024) return BI_ERR_UNSUPPORTED;
   const bool tile = model->tile_sb > 0;
   const size_t NT = (size_t)N * T;
 
@@ -131,7 +148,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
 
   // ---- the slices.  A register-tile model's kernels read only the lane-interleaved layout, so
   // that one is formed first; the packed layout follows only if those kernels decline the call.
-  const size_t wsmem = (size_t)kTT * Mtot * sizeof(R);
+  const size_t wsmem = (size_t)kTTP * Mtot * sizeof(R);
   void (*kerns[4])(const SoftJob) = {bi_soft_slices_kernel<R, 1>, bi_soft_slices_kernel<R, 2>,
                                      bi_soft_slices_kernel<R, 3>, bi_soft_slices_kernel<R, 4>};
   for (auto kf : kerns)
