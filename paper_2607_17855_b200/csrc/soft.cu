@@ -6,7 +6,9 @@
 // group, the group's slice  sum_{i in group} sum_o o^i[o] ln A_i[o, .]  in the
 // layouts the inference kernels read, and then runs those kernels on a shadow
 // model in which every group has one modality with T "outcomes" per agent: the
-// slices just formed, selected by the step index.
+// slices just formed, selected by the step index.  Forming the slices is a
+// dense product (observation vectors times ln A): float64 handles take it on
+// the FP64 tensor instruction, float32 handles on scalar multiply-adds.
 #include <algorithm>
 #include <cstring>
 
@@ -101,6 +103,93 @@ __global__ void __launch_bounds__(128, kEPT * sizeof(R) <= 24 ? 4 : 3) bi_soft_s
   else if (rem > 0) soft_block<R, kEPT, 4>(J, w_s, a, e0, dst, t0, rem);
 }
 
+// ---- the same slices on the FP64 tensor path ----
+// Per agent the slices of a group are the product W S: W[t][k] the observation vectors' entries of
+// the group's modalities (T x K, K = the sum of their outcome counts), S[k][e] the rows ln A_i[o, .]
+// in the layout being produced (K x P).  A warp owns blocks of 32 columns and takes a block of up to
+// 32 steps at a time: 16 accumulator tiles of 8 x 8, each k-step of four outcomes one S fragment per
+// 8 columns (read once, used for every 8 steps) and one W fragment per 8 steps from shared memory.
+// The m8n8k4 instruction issues once per 16 cycles and scheduler for 256 multiply-adds, so the FP64
+// pipe is fed by a sixteenth of the issue slots the scalar form needs.
+__device__ __forceinline__ void bi_dmma(double &c0, double &c1, double a, double b) {
+  asm("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(c0), "+d"(c1)
+               : "d"(a), "d"(b));
+}
+
+constexpr int kMmaSteps = 32;   // steps per block (four tiles of 8)
+constexpr int kMmaCols = 384;   // columns per CTA (four warps, three blocks of 32 columns each)
+
+template <int MT>
+__device__ __forceinline__ void soft_mma_block(const SoftJob &J, const double *Ws, int KS, const double *const *srow,
+                                               int KP, double *dst, int t0, int nt, int c_begin, int c_end) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, gid = lane >> 2, tig = lane & 3;
+  for (int n0 = c_begin + 32 * warp; n0 < c_end; n0 += 32 * 4) {
+    double acc[MT][4][2];
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[m][j][0] = acc[m][j][1] = 0.0;
+#pragma unroll 2
+    for (int ks = 0; ks < KP; ks += 4) {
+      const double *rp = srow[ks + tig];
+      double b[4], av[MT];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int col = n0 + 8 * j + gid;
+        b[j] = col < J.P ? __ldg(rp + col) : 0.0;
+      }
+#pragma unroll
+      for (int m = 0; m < MT; ++m) av[m] = Ws[(8 * m + gid) * KS + ks + tig];
+#pragma unroll
+      for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) bi_dmma(acc[m][j][0], acc[m][j][1], av[m], b[j]);
+    }
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+      const int tt = 8 * m + gid;
+      if (tt >= nt) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int col = n0 + 8 * j + 2 * tig;   // (P is a multiple of 4: a pair never straddles its end)
+        if (col < J.P)
+          *reinterpret_cast<double2 *>(dst + (size_t)(t0 + tt) * J.P + col) = make_double2(acc[m][j][0], acc[m][j][1]);
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(128, 4) bi_soft_slices_mma_kernel(const SoftJob J, int Kg, int KP) {
+  extern __shared__ __align__(16) unsigned char w_raw[];
+  const int KS = KP + 2;                                        // row stride of the staged vectors
+  double *Ws = reinterpret_cast<double *>(w_raw);              // [kMmaSteps][KS]
+  const double **srow = reinterpret_cast<const double **>(Ws + kMmaSteps * KS);   // [KP] rows of S
+  int32_t *sidx = reinterpret_cast<int32_t *>(srow + KP);      // [KP] their entries in an observation vector
+  const int a = blockIdx.y;
+  const int c_begin = blockIdx.x * kMmaCols, c_end = min(J.P, c_begin + kMmaCols);
+  for (int k = threadIdx.x; k < KP; k += blockDim.x) {
+    int mi = 0, o = k < Kg ? k : 0;   // (the padding rows point at the first row; their weights are zero)
+    while (o >= J.mem[mi].m) { o -= J.mem[mi].m; ++mi; }
+    srow[k] = (const double *)J.mem[mi].src + (size_t)a * J.mem[mi].gstride + (size_t)o * J.P;
+    sidx[k] = J.mem[mi].moff + o;
+  }
+  double *dst = (double *)J.dst + (size_t)a * J.T * J.P;
+  for (int t0 = 0; t0 < J.T; t0 += kMmaSteps) {
+    const int nt = min(kMmaSteps, J.T - t0);
+    __syncthreads();   // (the table above; the previous block's readers)
+    for (int i = threadIdx.x; i < kMmaSteps * KP; i += blockDim.x) {
+      const int tt = i / KP, k = i - tt * KP;
+      Ws[tt * KS + k] = (tt < nt && k < Kg) ? (double)J.soft[((size_t)a * J.T + t0 + tt) * J.Mtot + sidx[k]] : 0.0;
+    }
+    __syncthreads();
+    if (nt > 24) soft_mma_block<4>(J, Ws, KS, srow, KP, dst, t0, nt, c_begin, c_end);
+    else if (nt > 16) soft_mma_block<3>(J, Ws, KS, srow, KP, dst, t0, nt, c_begin, c_end);
+    else if (nt > 8) soft_mma_block<2>(J, Ws, KS, srow, KP, dst, t0, nt, c_begin, c_end);
+    else soft_mma_block<1>(J, Ws, KS, srow, KP, dst, t0, nt, c_begin, c_end);
+  }
+}
+
 __global__ void bi_soft_step_index_kernel(int32_t *obs, int N, int T, int M) {
   const size_t total = (size_t)N * T * M;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
@@ -171,9 +260,17 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
         J.mem[i].m = mm.m;
         J.mem[i].moff = moff[mm.modality];
       }
-      // elements per thread: 4 for large slices, else just enough to cover the slice with one CTA
-      const int ept = J.P >= 512 ? 4 : (J.P + 127) / 128;
-      kerns[ept - 1]<<<dim3((J.P + ept * 128 - 1) / (ept * 128), N), 128, wsmem, stream>>>(J);
+      int Kg = 0;
+      for (int i = 0; i < J.nmem; ++i) Kg += J.mem[i].m;
+      const int KP = (Kg + 3) & ~3;
+      const size_t msmem = ((size_t)kMmaSteps * (KP + 2) + KP) * sizeof(double) + (size_t)KP * sizeof(int32_t);
+      if (sizeof(R) == 8 && msmem <= 48 * 1024) {   // float64: the tensor form
+        bi_soft_slices_mma_kernel<<<dim3((J.P + kMmaCols - 1) / kMmaCols, N), 128, msmem, stream>>>(J, Kg, KP);
+      } else {
+        // elements per thread: 4 for large slices, else just enough to cover the slice with one CTA
+        const int ept = J.P >= 512 ? 4 : (J.P + 127) / 128;
+        kerns[ept - 1]<<<dim3((J.P + ept * 128 - 1) / (ept * 128), N), 128, wsmem, stream>>>(J);
+      }
       ++launches;
     }
   };

@@ -462,6 +462,34 @@ def test_batched_window_of_a_single_step(algo):
     assert res["kernel"] == f"batch_{algo}_f64", res
 
 
+@pytest.mark.parametrize("arith", ["f64", "f32"])
+@pytest.mark.parametrize("T", [12, 20, 27, 43, 70])
+def test_soft_observations_long_trajectories(T, arith):
+    """The slice-forming kernels take the steps in blocks (of 32 on the float64 tensor path, of 16 on the
+    other) and the last steps in a shorter block: trajectories that end in every block length, on a
+    model whose groups have slices of 24, 15, 4 and 24 (padded: 24, 16, 4, 24) elements."""
+    import torch
+    import oracle
+    import paper_2607_17855_b200 as bi
+    w = _custom(53, [3, 4, 2, 5, 3], [3, 2, 4, 3], [[0, 1, 2], [3, 4], [1], [2, 0, 1]], [2, 1, 3, 2, 2],
+                N=5, T=T, K=3, sparsity=0.5)
+    md = bi.model_from_workload(w, arith=arith)
+    soft = _soft_vectors(w, 7)
+    q = md.run_soft("filter", torch.from_numpy(soft).cuda(), torch.from_numpy(w.act).cuda(), w.K).cpu().numpy()
+    assert md.status() == 0
+    ref = oracle.run("filter", w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, None, w.act, w.K, obs_soft=soft)[0]
+    assert np.abs(q - ref).max() <= (1e-5 if arith == "f64" else 2e-3), np.abs(q - ref).max()
+    # a register-tile model with per-agent slices of 384 elements: three blocks of 32 columns per warp
+    w = make_config(2, N=7, T=T, K=3)
+    md2 = bi.model_from_workload(w, arith=arith)
+    soft = _soft_vectors(w, 8)
+    q = md2.run_soft("filter", torch.from_numpy(soft).cuda(), torch.from_numpy(w.act).cuda(), w.K).cpu().numpy()
+    ref = oracle.run("filter", w.n, w.m, w.dep, w.U, w.G, w.A, w.B, w.D, None, w.act, w.K, obs_soft=soft)[0]
+    assert np.abs(q - ref).max() <= (1e-5 if arith == "f64" else 2e-3), np.abs(q - ref).max()
+    md.close()
+    md2.close()
+
+
 def test_soft_observations_single_step_and_empty_batch():
     import torch
     import oracle
