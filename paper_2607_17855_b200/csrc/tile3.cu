@@ -33,9 +33,10 @@ int bi_launch_tile3(const BiCall &c, bi_model *mut) {
   Tile3Params p;
   bi_tile3_fill_params(c, p);
   int rc;
-  if (p.lambda != 1.0)
-    rc = bi_tile3_filter_damped(p, md->arith, g.dim[0], g.dim[1], g.dim[2], c.stream);
-  else if (md->arith == BI_ARITH_F64) {
+  if (p.lambda != 1.0) {
+    rc = md->arith == BI_ARITH_F64 ? bi_tile3_filter_f64(p, g.dim[0], g.dim[1], g.dim[2], c.stream) : BI_ERR_UNSUPPORTED;
+    if (rc == BI_ERR_UNSUPPORTED) rc = bi_tile3_filter_damped(p, md->arith, g.dim[0], g.dim[1], g.dim[2], c.stream);
+  } else if (md->arith == BI_ARITH_F64) {
     rc = bi_tile3_filter_f64(p, g.dim[0], g.dim[1], g.dim[2], c.stream);
     if (rc == BI_ERR_UNSUPPORTED) rc = tile3_filter::dispatch_filter<double, false>(p, g.dim[0], g.dim[1], g.dim[2], c.stream);
   } else

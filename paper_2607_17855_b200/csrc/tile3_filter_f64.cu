@@ -12,7 +12,8 @@ int launch(const Tile3Params &p, cudaStream_t stream) {
   // common shift, and the product of its three normalisers must stay a normal number: with probabilities
   // in A a logit is at least (modalities + 1) ln 1e-16, i.e. 53.2 (modalities + 1) binary orders below
   // zero, and three times that must stay under 1022: the kernel shifts per agent beyond five modalities)
-  tile3_f64::bi_tile3_filter_f64_kernel<NA, NB, NC><<<grid, 32, 0, stream>>>(p);
+  if (p.lambda != 1.0) tile3_f64::bi_tile3_filter_f64_kernel<NA, NB, NC, true><<<grid, 32, 0, stream>>>(p);
+  else tile3_f64::bi_tile3_filter_f64_kernel<NA, NB, NC, false><<<grid, 32, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? BI_OK : BI_ERR_CUDA;
 }
 

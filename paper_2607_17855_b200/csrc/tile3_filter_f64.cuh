@@ -172,8 +172,12 @@ struct Sweep {
     Ma = Mb = Mc = 0;
   }
 
-  template <bool UNITMAX>
-  __device__ __forceinline__ void sweep() {
+  // DAMPED: the logits take a step of size lam from the previous iterate's (oml = 1 - lam; the
+  // uniform start's logits are a constant, taken as 0); a separate instantiation, so that the plain
+  // sweep carries none of it.
+  template <bool UNITMAX, bool DAMPED>
+  __device__ __forceinline__ void sweep(R lam, R oml) {
+    const R pxa = xa, pxb = xb, pxc = xc;
     R V[G::NP], W[G::NP];
 #pragma unroll
     for (int j = 0; j < G::NP; ++j) V[j] = W[j] = 0.0;
@@ -196,6 +200,7 @@ struct Sweep {
       else la0 = fma(V[b], eb[b], la0);
     }
     xa = fma(la0 + la1, sa, lpa);
+    if (DAMPED) xa = fma(lam, xa, oml * pxa);
     __syncwarp();
     R b0 = 0.0, b1 = 0.0, c0 = 0.0, c1 = 0.0;
 #pragma unroll
@@ -207,6 +212,10 @@ struct Sweep {
     }
     xb = fma(b0 + b1, sb, lpb);
     xc = fma(c0 + c1, sc, lpc);
+    if (DAMPED) {
+      xb = fma(lam, xb, oml * pxb);
+      xc = fma(lam, xc, oml * pxc);
+    }
     // ---- softmax numerators relative to the largest binary exponent
     int ka, kb, kc;
     const R ma = exp_mant(xa, tab, ka);
@@ -239,7 +248,7 @@ struct Sweep {
   }
 };
 
-template <int NA, int NB, int NC>
+template <int NA, int NB, int NC, bool DAMPED>
 __global__ void __launch_bounds__(32) bi_tile3_filter_f64_kernel(const Tile3Params p) {
   using R = double;
   using G = Geo<NA, NB, NC>;
@@ -387,8 +396,9 @@ __global__ void __launch_bounds__(32) bi_tile3_filter_f64_kernel(const Tile3Para
     sw.lpc = c_ok ? lpc : 0.0;
 
     sw.start();
-    if (unit_shift) for (int k = 0; k < p.K; ++k) sw.template sweep<true>();
-    else for (int k = 0; k < p.K; ++k) sw.template sweep<false>();
+    const R lam = (R)p.lambda, oml = 1.0 - lam;
+    if (unit_shift) for (int k = 0; k < p.K; ++k) sw.template sweep<true, DAMPED>(lam, oml);
+    else for (int k = 0; k < p.K; ++k) sw.template sweep<false, DAMPED>(lam, oml);
 
     // ---- final beliefs of the step: outputs, and the next step's prior input
     // (1/za = sc zb, 1/zb = sc za, 1/zc = sa zb)
