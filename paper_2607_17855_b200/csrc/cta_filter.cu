@@ -60,6 +60,7 @@ struct CtaGeom {   // element offsets (units of R) into dynamic shared memory
   int deep;                       // any group of rank >= 4: phase B and its barrier are needed
   int ops, maxops, nops, exptab;  // phase C's operation lists [F][maxops] (16 bytes each), their lengths, the exp table
   int prior_tps;                  // threads that share one state when the prior is formed (1, 2 or 4)
+  int wpar, wpar_cap;             // models with several parents per transition: the parents' outer product of one factor
   int total_bytes;
 };
 
@@ -334,20 +335,53 @@ bi_cta_filter_kernel(const BiDev *__restrict__ mdp, int T, const int32_t *__rest
 
   for (int t = 0; t < T; ++t) {
     // ln prior: D at the first step, else B_u q_{t-1} (cur still holds step t-1)
-    if (md.has_bdep && (t > 0 || from_prev)) {   // a warp per state: the expectation of the transition tensor
-      for (int idx = warp; idx < Sp; idx += NW) {
-        int f = 0;
-        while (f + 1 < F && idx >= md.offp[f + 1]) ++f;
-        const int s = idx - md.offp[f], n = md.n[f];
-        R lp = (R)0;
-        if (s < n) {
-          const int ur = t == 0 ? __ldg(act_prev + (size_t)a * F + f)
-                                : __ldg(act + ((size_t)a * (T - 1) + (t - 1)) * F + f);
-          const int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
-          const R *row = (const R *)md.Bfull[f] + (size_t)g * md.Bfull_stride[f] + ((size_t)u * n + s) * md.PB[f];
-          lp = bi_log(bi_max(cta_bdep_expect<R>(md, f, row, cur, lane), (R)BI_EPS));
+    if (md.has_bdep && (t > 0 || from_prev)) {
+      // The expectation of the transition tensor under the parents' beliefs.  The parents' outer product
+      // is the same for every next state of a factor: formed once per factor in shared memory (when it
+      // fits), then a warp per state sums its row against it, lane by lane in a fixed order.
+      R *wpar = smem + sm.wpar;
+      for (int f = 0; f < F; ++f) {
+        const int n = md.n[f], PB = md.PB[f], k = md.bdep_len[f];
+        const int ur = t == 0 ? __ldg(act_prev + (size_t)a * F + f) : __ldg(act + ((size_t)a * (T - 1) + (t - 1)) * F + f);
+        const int u = clamp_flag(ur, md.U[f], md.status, BI_FLAG_ACT_RANGE);
+        const R *Xu = (const R *)md.Bfull[f] + (size_t)g * md.Bfull_stride[f] + (size_t)u * n * PB;
+        const bool shared_w = PB <= sm.wpar_cap;
+        if (shared_w) {
+          for (int e = tid; e < PB; e += NT) {
+            int rem = e;
+            R w = (R)1;
+            for (int j = k - 1; j >= 0; --j) {
+              const int gq = md.bdep[f][j], nj = md.n[gq];
+              const int d = rem % nj;
+              rem /= nj;
+              w *= cur[md.offp[gq] + d];
+            }
+            wpar[e] = w;
+          }
+          __syncthreads();
         }
-        if (lane == 0) lpri[idx] = lp;
+        for (int s = warp; s < n; s += NW) {
+          const R *row = Xu + (size_t)s * PB;
+          R ex;
+          if (shared_w) {
+            R acc = (R)0;
+            int e = lane;
+            for (; e + 96 < PB; e += 128) {   // four loads in flight, one accumulator: the order of the plain loop
+              const R x0 = __ldg(row + e), x1 = __ldg(row + e + 32), x2 = __ldg(row + e + 64), x3 = __ldg(row + e + 96);
+              acc = fma(x0, wpar[e], acc);
+              acc = fma(x1, wpar[e + 32], acc);
+              acc = fma(x2, wpar[e + 64], acc);
+              acc = fma(x3, wpar[e + 96], acc);
+            }
+            for (; e < PB; e += 32) acc = fma(__ldg(row + e), wpar[e], acc);
+            ex = warp_sum(acc);
+          } else {
+            ex = cta_bdep_expect<R>(md, f, row, cur, lane);
+          }
+          if (lane == 0) lpri[md.offp[f] + s] = bi_log(bi_max(ex, (R)BI_EPS));
+        }
+        for (int s = n + tid; s < md.npad[f]; s += NT) lpri[md.offp[f] + s] = (R)0;
+        if (shared_w) __syncthreads();   // (the next factor overwrites the product)
       }
     } else if (t == 0 && !from_prev) {
       for (int idx = tid; idx < Sp; idx += NT) {
@@ -655,6 +689,13 @@ int launch_cta_filter_t(const BiCall &c, bi_model *mut) {
     }
   }
   sm.prior_tps = 4 * h.Sp <= NT ? 4 : 2 * h.Sp <= NT ? 2 : 1;
+  sm.wpar = o;
+  sm.wpar_cap = 0;
+  if (h.has_bdep) {
+    for (int f = 0; f < h.F; ++f) sm.wpar_cap = std::max(sm.wpar_cap, (int)h.PB[f]);
+    sm.wpar_cap = std::min(bi_pad4(sm.wpar_cap), 4096);
+    o += sm.wpar_cap;
+  }
   sm.total_bytes = (int)((size_t)o * sizeof(R));
   if ((size_t)o * sizeof(R) > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
 
