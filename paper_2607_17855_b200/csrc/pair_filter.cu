@@ -31,6 +31,7 @@ typedef double R;
 
 struct PairParams {
   int32_t N, T, K, F, M, S, G;
+  double lambda;   // damping step on the logits; 1 = the plain update
   int32_t n[BI_MAX_F], off[BI_MAX_F], npad[BI_MAX_F], U[BI_MAX_F];
   const R *Bf[BI_MAX_F], *logD[BI_MAX_F];   // forward matrices [u][next][previous (padded)], ln D
   int64_t Bstride[BI_MAX_F], Dstride[BI_MAX_F];
@@ -77,8 +78,11 @@ constexpr int WARPS = 4;
 // instruction) instead of the unit's (a shuffle per halving of the unit): every unit of the warp is then
 // scaled by the same power of two, which is exact, and safe while a logit cannot differ from another
 // agent's by more than the exponent range, which the caller checks from the number of modalities.
-template <int LPU, bool WARPMAX>
+// DAMPED: every iteration takes a step of size lambda on the logits from the previous iterate's (the
+// uniform start's logits are a constant, taken as 0); an instantiation of its own.
+template <int LPU, bool WARPMAX, bool DAMPED>
 __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairParams p) {
+  const R lam = p.lambda, oml = 1.0 - lam;
   // the normalisers come from the exchanged copies every lane reads anyway (additions in the shadow of the
   // products) instead of a shuffle sum at the end of the sweep's dependency chain (measured on the sweep's
   // 77 structures of this kind: 7.4 -> 7.0 ms with it for every unit size; config 1's call 65 -> 54 us)
@@ -143,6 +147,11 @@ __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairPa
       }
       if (pair && f == p.fa) { ca = c; continue; }
       if (pair && f == p.fb) { cb = c; continue; }
+      if (DAMPED) {   // a factor outside the pair: its message does not change, its logits approach it
+        R x = 0.0;
+        for (int k = 0; k < p.K; ++k) x = fma(lam, c, oml * x);
+        c = x;
+      }
       int k;
       const R mant = exp_mant(c, exp_tab, k);
       const int M = max_k<LPU, true>(ok ? k : INT_MIN) >> EXP_BITS;
@@ -208,8 +217,13 @@ __global__ void __launch_bounds__(WARPS * 32) bi_pair_filter_kernel(const PairPa
         za = sa0 + sa1; zb = sb0 + sb1;
         rza = rcp_fast(za); rzb = rcp_fast(zb);
       }
-      xa = fma(v0 + v1, rzb, ca);
-      xb = fma(w0 + w1, rza, cb);
+      if (DAMPED) {
+        xa = fma(lam, fma(v0 + v1, rzb, ca), oml * xa);
+        xb = fma(lam, fma(w0 + w1, rza, cb), oml * xb);
+      } else {
+        xa = fma(v0 + v1, rzb, ca);
+        xb = fma(w0 + w1, rza, cb);
+      }
       int ka, kb;
       const R ma = exp_mant(xa, exp_tab, ka);
       const R mb = exp_mant(xb, exp_tab, kb);
@@ -274,22 +288,26 @@ int launch(const PairParams &p, cudaStream_t stream) {
   const int grid = (p.N + per_cta - 1) / per_cta;
   // (logits are sums of at most M + 1 terms of magnitude below 37: with few modalities two agents'
   // logits are within a few hundred binary exponents of each other)
-  if (p.M <= 5) bi_pair_filter_kernel<LPU, true><<<grid, WARPS * 32, 0, stream>>>(p);
-  else bi_pair_filter_kernel<LPU, false><<<grid, WARPS * 32, 0, stream>>>(p);
+  if (p.lambda != 1.0) {
+    if (p.M <= 5) bi_pair_filter_kernel<LPU, true, true><<<grid, WARPS * 32, 0, stream>>>(p);
+    else bi_pair_filter_kernel<LPU, false, true><<<grid, WARPS * 32, 0, stream>>>(p);
+  } else if (p.M <= 5) bi_pair_filter_kernel<LPU, true, false><<<grid, WARPS * 32, 0, stream>>>(p);
+  else bi_pair_filter_kernel<LPU, false, false><<<grid, WARPS * 32, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? BI_OK : BI_ERR_CUDA;
 }
 
 }  // namespace
 
-// Applicable to float64 handles, the plain update, trivial B-dependencies and models whose groups
+// Applicable to float64 handles, plain and damped updates, trivial B-dependencies and models whose groups
 // over more than one factor number at most one, over exactly two factors; BI_ERR_UNSUPPORTED otherwise.
 int bi_launch_pair_filter(const BiCall &c, bi_model *mut) {
   const bi_model *md = c.model;
   const BiDev &h = md->h;
-  if (c.algo != BI_ALGO_FILTER || md->arith != BI_ARITH_F64 || c.lambda != 1.0 || h.has_bdep) return BI_ERR_UNSUPPORTED;
+  if (c.algo != BI_ALGO_FILTER || md->arith != BI_ARITH_F64 || h.has_bdep) return BI_ERR_UNSUPPORTED;
   if (!md->pair_ok) return BI_ERR_UNSUPPORTED;
   PairParams p;
   memset(&p, 0, sizeof(p));
+  p.lambda = c.lambda;
   p.N = c.N; p.T = c.T; p.K = c.K; p.F = h.F; p.M = h.M; p.S = h.S; p.G = h.G;
   int nmax = 1;
   for (int f = 0; f < h.F; ++f) {

@@ -551,7 +551,7 @@ def test_continued_windows(case, algo):
 # ---- damped updates (bi_model_set_damping)
 
 @pytest.mark.parametrize("algo", ALGOS)
-@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "cta", "per_agent"])
+@pytest.mark.parametrize("case", ["tile", "tile_cluster", "batch", "warp", "cta", "per_agent", "pair", "pair_and_others"])
 def test_damped_updates(case, algo):
     import torch
     import oracle
@@ -563,6 +563,10 @@ def test_damped_updates(case, algo):
         "warp": _custom(49, [5, 4, 3, 2], [3, 4], [[0, 1], [1, 2, 3]], [2, 2, 1, 2], N=10, T=7, K=6),
         "cta": make_config(3, N=10, T=7, K=6),
         "per_agent": _custom(8, [6, 5, 7], [4, 3], [[2, 0, 1], [1, 2]], [2, 2, 2], N=5, T=6, K=6, G=5),
+        "pair": make_config(1, N=11, T=9, K=6),
+        # two coupled factors, one with a modality of its own, and two factors outside the pair (one observed)
+        "pair_and_others": _custom(54, [5, 3, 7, 4], [3, 4, 2, 3], [[2, 0], [0], [1], [0, 2]], [2, 1, 3, 2],
+                                   N=37, T=8, K=5),
     }[case]
     lam = 0.45
     with (warp_filter_forced() if case == "warp" else contextlib.nullcontext()):
@@ -574,6 +578,8 @@ def test_damped_updates(case, algo):
     kernel = md.last_kernel
     if algo == "filter" and case in ("warp", "cta"):
         assert kernel == f"{case}_filter_f64", kernel
+    if algo == "filter" and case in ("pair", "pair_and_others"):
+        assert kernel == "pair_filter_f64", kernel
     assert md.status() == 0
     sel = list(range(0, w.N, max(1, w.N // 12)))
     sub = w.take_agents(sel)
@@ -1127,8 +1133,11 @@ def test_pair_filter_continued_calls():
                              act[:, 3].contiguous(), w.K).cpu().numpy()
     ref = oracle.run_workload(w, "filter")[0]
     assert np.abs(whole - ref).max() <= 1e-5 and np.abs(tail - ref[:, 4:]).max() <= 1e-5
-    # a damped call is not this kernel's
+    # a damped call is this kernel's too, block by block as well
     md.set_damping(0.5)
-    md.bi_filter(obs, act, w.K)
-    assert md.last_kernel == "cta_filter_f64" and md.status() == 0
+    damped = md.bi_filter(obs, act, w.K).cpu().numpy()
+    assert md.last_kernel == "pair_filter_f64" and md.status() == 0
+    q, names = _blockwise(md, w, [0, 2, 3, 7, w.T], w.K)
+    assert names == {"pair_filter_f64"} and np.array_equal(q, damped)
+    assert np.abs(damped - oracle.run_workload(w, "filter", damping=0.5)[0]).max() <= 1e-5
     md.close()
