@@ -35,6 +35,7 @@ typedef double R;
 
 struct PairWinParams {
   int32_t N, T, K, F, M, S, G, algo;
+  double lambda;   // damping step on the logits; 1 = the plain update
   int32_t n[BI_MAX_F], off[BI_MAX_F], npad[BI_MAX_F], U[BI_MAX_F];
   // transition matrices read [summation index][own state]: past edge and future edge
   const R *Mp[BI_MAX_F], *Mf[BI_MAX_F], *logD[BI_MAX_F];
@@ -107,8 +108,10 @@ __device__ __forceinline__ void edge_dots(const R *__restrict__ mp, const R *__r
 }
 
 // MAXT: the most threads a launch of this instantiation has; windows of up to 320 threads get a
-// register budget under which two CTAs share an SM.
-template <int LPU, int ALGO, int MAXT>
+// register budget under which two CTAs share an SM.  DAMPED: every iteration takes a step of size
+// lambda on the logits from the previous iterate's, kept in shared memory (the first from ln q of the
+// starting belief; the uniform start's is a constant, taken as 0); instantiations of their own.
+template <int LPU, int ALGO, int MAXT, bool DAMPED>
 __global__ void __launch_bounds__(MAXT, MAXT <= 320 ? 2 : 1) bi_pair_window_kernel(const PairWinParams p) {
   const int LS = p.ls, NAR = p.nar;   // row stride and rows of a staged slice
   constexpr bool LREG = LPU < 32;   // the slice's row stays in registers for the iterations
@@ -117,7 +120,9 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 320 ? 2 : 1) bi_pair_window_kern
   R *qb = exp_tab + EXP_TAB;                                    // [2][units + 2][F][LPU]; slot 0 and the last are never read as neighbours of a real edge
   const int slot_sz = p.F * LPU, buf_sz = (p.units + 2) * slot_sz;
   R *cst = qb + 2 * buf_sz;                                     // [units][F][LPU] constants of the logits
-  R *Ls = cst + p.units * slot_sz;                              // [units][ng][LPU][LS] the pair groups' summed slices, row-major
+  R *xpv = cst + p.units * slot_sz;                             // DAMPED: [units][F][LPU] the previous iterate's logits
+  R *Ls = xpv + (DAMPED ? p.units * slot_sz : 0);               // [units][ng][LPU][LS] the pair groups' summed slices, row-major
+  const R lam = p.lambda, oml = 1.0 - lam;
   int32_t *aoff = reinterpret_cast<int32_t *>(Ls + (((size_t)p.units * p.ng * NAR * LS + 1) & ~(size_t)1));   // [units][F][2] matrix offsets of the two edges
   for (int j = threadIdx.x; j < EXP_TAB; j += blockDim.x) exp_tab[j] = exp2((double)j * (1.0 / EXP_TAB));
 
@@ -146,6 +151,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 320 ? 2 : 1) bi_pair_window_kern
       cst[(tl * p.F + f) * LPU + s] = c;
       qb[(tl + 1) * slot_sz + f * LPU + s] = q0;
       qb[buf_sz + (tl + 1) * slot_sz + f * LPU + s] = 0.0;
+      if (DAMPED) xpv[(tl * p.F + f) * LPU + s] = (p.q_init && ok) ? bi_log(bi_max(q0, (R)BI_EPS)) : 0.0;
       if (s < 2) {
         int off = 0;
         const int tt = s == 0 ? t - 1 : t;   // the action that drives t-1 -> t, or t -> t+1
@@ -245,6 +251,11 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 320 ? 2 : 1) bi_pair_window_kern
           x += v0 + v1;
         }
       }
+      if (DAMPED) {
+        R *xq = xpv + (tl * p.F + f) * LPU + s;   // (this thread's own entry)
+        x = fma(lam, x, oml * *xq);
+        *xq = x;
+      }
       int kk;
       const R mant = exp_mant(ok ? x : 0.0, exp_tab, kk);
       const int Mx = max_k<LPU, true>(ok ? kk : INT_MIN) >> EXP_BITS;
@@ -276,14 +287,18 @@ int launch(PairWinParams &p, const bi_model *md, cudaStream_t stream) {
   if (threads > 512) return BI_ERR_UNSUPPORTED;   // (the kernel's register budget is set for this)
   p.units = threads / LPU;
   const size_t slot = (size_t)p.F * LPU;
-  size_t elems = EXP_TAB + 2 * (p.units + 2) * slot + p.units * slot + (((size_t)p.units * p.ng * p.nar * p.ls + 1) & ~(size_t)1);
+  const bool damped = p.lambda != 1.0;
+  size_t elems = EXP_TAB + 2 * (p.units + 2) * slot + (damped ? 2 : 1) * p.units * slot + (((size_t)p.units * p.ng * p.nar * p.ls + 1) & ~(size_t)1);
   const size_t bytes = elems * sizeof(R) + (size_t)p.units * p.F * 2 * sizeof(int32_t) + 16;
   if (bytes > (size_t)md->max_smem_optin - 1024) return BI_ERR_UNSUPPORTED;
   void (*kern)(const PairWinParams);
-  if (threads <= 320)
-    kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 320> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 320>;
-  else
-    kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 512> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 512>;
+  if (threads <= 320) {
+    if (damped) kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 320, true> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 320, true>;
+    else kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 320, false> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 320, false>;
+  } else {
+    if (damped) kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 512, true> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 512, true>;
+    else kern = p.algo == BI_ALGO_VMP ? bi_pair_window_kernel<LPU, BI_ALGO_VMP, 512, false> : bi_pair_window_kernel<LPU, BI_ALGO_MMP, 512, false>;
+  }
   if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
     cudaGetLastError();
     return BI_ERR_CUDA;
@@ -294,16 +309,17 @@ int launch(PairWinParams &p, const bi_model *md, cudaStream_t stream) {
 
 }  // namespace
 
-// Applicable to float64 handles, the plain update, trivial B-dependencies, window calls (also warm
+// Applicable to float64 handles, plain and damped updates, trivial B-dependencies, window calls (also warm
 // starts and continued windows) on models with no group over more than two factors, and to windows
 // whose steps and staged slices fit one CTA; BI_ERR_UNSUPPORTED otherwise.
 int bi_launch_pair_window(const BiCall &c, bi_model *mut) {
   const bi_model *md = c.model;
   const BiDev &h = md->h;
-  if (c.algo == BI_ALGO_FILTER || md->arith != BI_ARITH_F64 || c.lambda != 1.0 || h.has_bdep) return BI_ERR_UNSUPPORTED;
+  if (c.algo == BI_ALGO_FILTER || md->arith != BI_ARITH_F64 || h.has_bdep) return BI_ERR_UNSUPPORTED;
   if (!md->rank2_ok) return BI_ERR_UNSUPPORTED;
   PairWinParams p;
   memset(&p, 0, sizeof(p));
+  p.lambda = c.lambda;
   p.N = c.N; p.T = c.T; p.K = c.K; p.F = h.F; p.M = h.M; p.S = h.S; p.G = h.G; p.algo = c.algo;
   int nmax = 1;
   for (int f = 0; f < h.F; ++f) {

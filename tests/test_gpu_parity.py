@@ -578,8 +578,8 @@ def test_damped_updates(case, algo):
     kernel = md.last_kernel
     if algo == "filter" and case in ("warp", "cta"):
         assert kernel == f"{case}_filter_f64", kernel
-    if algo == "filter" and case in ("pair", "pair_and_others"):
-        assert kernel == "pair_filter_f64", kernel
+    if case in ("pair", "pair_and_others"):
+        assert kernel == f"pair_{algo}_f64", kernel
     assert md.status() == 0
     sel = list(range(0, w.N, max(1, w.N // 12)))
     sub = w.take_agents(sel)
@@ -1100,7 +1100,7 @@ def test_filtering_on_models_with_several_pairs(case):
 
 
 def test_pair_window_kernel_limits():
-    """A window whose steps do not fit one CTA goes to another kernel family; so does a damped call."""
+    """A window whose steps do not fit one CTA goes to another kernel family; a damped call does not."""
     import torch
     import paper_2607_17855_b200 as bi
     w = _custom(99, [32, 31], [3, 4], [[1, 0], [0]], [2, 2], N=40, T=20, K=3)   # 20 steps x 32 lanes > 512 threads
@@ -1111,9 +1111,12 @@ def test_pair_window_kernel_limits():
     obs, act = torch.from_numpy(w.obs).cuda(), torch.from_numpy(w.act).cuda()
     md.bi_vmp(obs, act, w.K)
     assert md.last_kernel == "pair_vmp_f64"
+    import oracle
     md.set_damping(0.5)
-    md.bi_vmp(obs, act, w.K)
-    assert not md.last_kernel.startswith("pair_") and md.status() == 0
+    for algo in ("vmp", "mmp"):
+        q = md.run(algo, obs, act, w.K).cpu().numpy()
+        assert md.last_kernel == f"pair_{algo}_f64" and md.status() == 0
+        assert np.abs(q - oracle.run_workload(w, algo, damping=0.5)[0]).max() <= 1e-5
     md.close()
 
 
