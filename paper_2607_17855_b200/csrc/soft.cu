@@ -217,6 +217,18 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     need += up256(NT * h.grp[k].P_pad * sizeof(R));
   }
   if (tile) { off_tile = need; need += up256(NT * model->tile_P * sizeof(R)); }
+  // a filtering call on a model the pair filtering kernel serves: that kernel also reads the pair's
+  // slices with the two axes exchanged, so those are formed too (from the handle's transposed copies)
+  int kpair = -1;
+  size_t off_packT = 0, PT = 0;
+  if (algo == BI_ALGO_FILTER && model->pair_ok && sizeof(R) == 8)
+    for (int k = 0; k < h.ngroups; ++k)
+      if (h.grp[k].rank == 2 && h.mem[h.grp[k].mem_begin].logA_T) kpair = k;
+  if (kpair >= 0) {
+    PT = (size_t)h.grp[kpair].dim[1] * bi_pad4(h.grp[kpair].dim[0]);
+    off_packT = need;
+    need += up256(NT * PT * sizeof(R));
+  }
   const size_t off_obs = need;
   need += up256(NT * h.ngroups * sizeof(int32_t));
   const size_t off_desc = need;
@@ -244,18 +256,20 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     if (cudaFuncSetAttribute((const void *)kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem) != cudaSuccess)
       return BI_ERR_CUDA;
   int launches = 0;
+  // layout 0: every group's packed slices; 1: the lane-interleaved slices of a tile model; 2: the
+  // pair's slices with the axes exchanged
   auto form = [&](int layout) {
-    for (int k = 0; k < (layout ? 1 : h.ngroups); ++k) {
+    for (int k = layout == 2 ? kpair : 0; k < (layout == 1 ? 1 : layout == 2 ? kpair + 1 : h.ngroups); ++k) {
       const BiGroup &g = h.grp[k];
       SoftJob J;
       memset(&J, 0, sizeof(J));
       J.nmem = g.mem_end - g.mem_begin;
-      J.P = layout ? model->tile_P : g.P_pad;
+      J.P = layout == 1 ? model->tile_P : layout == 2 ? (int)PT : g.P_pad;
       J.T = T; J.Mtot = Mtot; J.soft = obs_soft;
-      J.dst = w + (layout ? off_tile : off_pack[k]);
+      J.dst = w + (layout == 1 ? off_tile : layout == 2 ? off_packT : off_pack[k]);
       for (int i = 0; i < J.nmem; ++i) {
         const BiMember &mm = h.mem[g.mem_begin + i];
-        J.mem[i].src = layout ? mm.logA_tile : mm.logA;
+        J.mem[i].src = layout == 1 ? mm.logA_tile : layout == 2 ? mm.logA_T : mm.logA;
         J.mem[i].gstride = h.G == 1 ? 0 : (int64_t)mm.m * J.P;
         J.mem[i].m = mm.m;
         J.mem[i].moff = moff[mm.modality];
@@ -275,6 +289,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     }
   };
   form(tile ? 1 : 0);
+  if (kpair >= 0) form(2);
   int32_t *obs_idx = reinterpret_cast<int32_t *>(w + off_obs);
   bi_soft_step_index_kernel<<<256, 256, 0, stream>>>(obs_idx, N, T, h.ngroups);
   ++launches;
@@ -292,6 +307,7 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
     BiMember &mm = sh.h.mem[k];
     mm.logA = w + off_pack[k];
     mm.logA_tile = tile && k == 0 ? w + off_tile : nullptr;
+    mm.logA_T = k == kpair ? w + off_packT : nullptr;
     mm.cmask = nullptr; mm.cvals = nullptr; mm.coff = nullptr;   // (the slices formed above are dense)
     mm.gstride = (int64_t)T * g.P_pad;
     mm.m = T;
@@ -301,8 +317,9 @@ int run_soft_t(const bi_model *model, int algo, int N, int T, const float *obs_s
   }
   // (a group of one modality is its own pre-summed table: the shadow's T per-agent slices)
   sh.soft_shadow = 1;
-  sh.pair_ok = 0;
-  sh.rank2_ok = 0;   // (no transposed copy of the slices formed above: the pair kernel does not apply)
+  sh.pair_ok = kpair >= 0 || (model->pair_ok && sizeof(R) == 8 && algo == BI_ALGO_FILTER);
+  // (the pair filtering kernel needs the transposed slices formed above, or no pair at all; the pair
+  // window kernel reads rows only)
   sh.tile_comb = tile ? w + off_tile : nullptr;
   sh.tile_ncomb = T;
   sh.tile_comb_mul[0] = 1;
