@@ -34,6 +34,10 @@ struct WarpSmem {       // element offsets (units of R) into dynamic shared memo
   int o_xp;             // filtering, damped calls: per-warp previous logits [Sp]; -1 otherwise
   int o_Y;              // window, models with B-dependencies: per-warp [sum_h PB_h] next-belief-weighted tensors; -1 otherwise
   int xp;               // window, damped calls: [T][Sp] previous logits shared by the CTA; -1 otherwise
+  // window, models with B-dependencies of at most four parents: per-warp [sum_f PB_f] products of the
+  // parents' previous beliefs, and the CTA's table [sum_f PB_f] of the belief entries each product takes
+  // (one byte per parent: its padded belief offset); -1 otherwise
+  int o_W, dtab;
 };
 
 template <typename R>
@@ -281,6 +285,19 @@ __device__ R bdep_past_lane(const BiDev &md, int f, const R *__restrict__ Xrow, 
   }
   return acc;
 }
+// The same with the parents' products already formed (W: one entry per parent combination).
+template <typename R>
+__device__ __forceinline__ R bdep_past_dot(const R *__restrict__ Xrow, const R *W, int PB) {
+  R a0 = (R)0, a1 = (R)0;
+  int e = 0;
+#pragma unroll 2
+  for (; e + 1 < PB; e += 2) {
+    a0 = fma(__ldg(Xrow + e), W[e], a0);
+    a1 = fma(__ldg(Xrow + e + 1), W[e + 1], a1);
+  }
+  if (e < PB) a0 = fma(__ldg(Xrow + e), W[e], a0);
+  return a0 + a1;
+}
 // Future, to state s of factor f0: over every factor h whose transition reads f0,
 // sum_{s'} q_{t+1,h}[s'] sum_{parents with s_f0 = s} ln B_h[s'][parents] prod_{other parents} q_t[...];
 // act_t: the actions taken at this step.  The other parents' combinations are walked the same way.
@@ -463,6 +480,24 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
   for (int i = lane; i < sm.o_sl - sm.o_V0; i += 32) V0[i] = (R)0;  // V0 and V1 are adjacent
   for (int i = threadIdx.x; i < T * M; i += blockDim.x)
     obs_s[i] = clamp_flag(obs[(size_t)a * T * M + i], md.m[i % M], md.status, BI_FLAG_OBS_RANGE);
+  if (sm.dtab >= 0) {   // which belief entries the product of a parent combination takes (once per launch)
+    uint32_t *dt = reinterpret_cast<uint32_t *>(base + sm.dtab);
+    int yo = 0;
+    for (int f = 0; f < F; ++f) {
+      const int PB = md.PB[f], k = md.bdep_len[f];
+      for (int e = threadIdx.x; e < PB; e += blockDim.x) {
+        int rem = e;
+        uint32_t pack = 0;
+        for (int j = k - 1; j >= 0; --j) {
+          const int gq = md.bdep[f][j], nj = md.n[gq];
+          pack |= (uint32_t)(md.offp[gq] + rem % nj) << (8 * j);
+          rem /= nj;
+        }
+        dt[yo + e] = pack;
+      }
+      yo += PB;
+    }
+  }
   for (int i = threadIdx.x; i < 2 * T * Sp; i += blockDim.x) {
     const int pidx = i % Sp;
     int f = 0;
@@ -489,6 +524,25 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
         bdep_weighted_tensors<R>(md, g, cur + (size_t)(t + 1) * Sp, act + ((size_t)a * (T - 1) + t) * F, wb + sm.o_Y, lane);
         __syncwarp();
       }
+      if (sm.o_W >= 0 && t > 0) {   // the parents' products under the previous step's beliefs, for every factor
+        const R *qp = cur + (size_t)(t - 1) * Sp;
+        const uint32_t *dt = reinterpret_cast<const uint32_t *>(base + sm.dtab);
+        R *Wv = wb + sm.o_W;
+        int yo = 0;
+        for (int f = 0; f < F; ++f) {
+          const int PB = md.PB[f], k = md.bdep_len[f];
+          for (int e = lane; e < PB; e += 32) {
+            const uint32_t d = dt[yo + e];
+            R w = qp[d & 255u];
+            if (k > 1) w *= qp[(d >> 8) & 255u];
+            if (k > 2) w *= qp[(d >> 16) & 255u];
+            if (k > 3) w *= qp[d >> 24];
+            Wv[yo + e] = w;
+          }
+          yo += PB;
+        }
+        __syncwarp();
+      }
       // transition messages (Section IV): low-rank contractions of B with the
       // neighbouring steps' beliefs of the previous iterate; transposed layouts
       // so that consecutive lanes read consecutive addresses
@@ -504,7 +558,13 @@ bi_warp_window_kernel(const BiDev *__restrict__ mdp, int N, int T, const int32_t
           } else if (md.has_bdep) {
             const int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *row = (const R *)md.logBfull[f] + (size_t)g * md.Bfull_stride[f] + ((size_t)u * n + s) * md.PB[f];
-            msg = bdep_past_lane<R>(md, f, row, cur + (size_t)(t - 1) * Sp);
+            if (sm.o_W >= 0) {
+              int yo = 0;
+              for (int j = 0; j < f; ++j) yo += md.PB[j];
+              msg = bdep_past_dot<R>(row, wb + sm.o_W + yo, md.PB[f]);
+            } else {
+              msg = bdep_past_lane<R>(md, f, row, cur + (size_t)(t - 1) * Sp);
+            }
           } else {
             int u = clamp_flag(act[((size_t)a * (T - 1) + (t - 1)) * F + f], md.U[f], md.status, BI_FLAG_ACT_RANGE);
             const R *M0 = (const R *)(ALGO == BI_ALGO_VMP ? md.logBt[f] : md.BfT[f]);  // [previous][next]
@@ -562,11 +622,21 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
   sm.o_xp = (!window && damped) ? o : -1;
   if (!window && damped) o += h.Sp;
   sm.o_Y = -1;
+  sm.o_W = -1;
+  sm.dtab = -1;
+  int ysum = 0;
+  bool four = true;   // (a table entry holds four parents' offsets)
   if (window && h.has_bdep) {
-    int ysum = 0;
-    for (int f = 0; f < h.F; ++f) ysum += h.PB[f];
+    for (int f = 0; f < h.F; ++f) {
+      ysum += h.PB[f];
+      four = four && h.bdep_len[f] <= 4;
+    }
     sm.o_Y = o;
     o += bi_pad4(ysum);
+    if (four && ysum <= 4096) {
+      sm.o_W = o;
+      o += bi_pad4(ysum);
+    }
   }
   sm.per_warp = o;
   const size_t budget = 100 * 1024;  // at least two CTAs per SM
@@ -578,6 +648,10 @@ int launch_warp_t(const BiCall &c, bi_model *mut) {
     shared_elems += (size_t)bi_pad4((int)(((size_t)c.T * h.M * sizeof(int32_t) + sizeof(R) - 1) / sizeof(R)) + 1);
     sm.xp = damped ? (int)shared_elems : -1;
     if (damped) shared_elems += (size_t)c.T * h.Sp;
+    if (sm.o_W >= 0) {
+      sm.dtab = (int)shared_elems;
+      shared_elems += (size_t)bi_pad4((int)(((size_t)ysum * sizeof(uint32_t) + sizeof(R) - 1) / sizeof(R)));
+    }
   } else {
     sm.xp = -1;
     sm.q = 0;

@@ -871,6 +871,12 @@ BDEP_CASES = {
                  bdep=[[0, 1, 2, 3], [1], [3, 2], [0, 3]], N=5, T=4, K=4),
     "per_agent": dict(n=[3, 4], m=[3, 2], dep=[[0, 1], [1]], U=[2, 2], bdep=[[1, 0], [0]], N=4, T=5, K=4, G=4, sparsity=0.6),
     "ragged_edge": dict(n=[32, 2], m=[2], dep=[[0]], U=[1, 1], bdep=[[0, 1], [1, 0]], N=1, T=1, K=1),
+    # five parents: the window kernel's table of parent offsets holds four, so its lanes walk the combinations themselves
+    "five_parents": dict(n=[2, 3, 2, 2, 3], m=[3, 2], dep=[[0, 1], [4, 2, 3]], U=[2, 1, 1, 2, 1],
+                         bdep=[[4, 3, 2, 1, 0], [1], [2, 0], [3], [4, 1]], N=6, T=5, K=4),
+    # windows long enough that every warp takes several steps, parents' products of 96 and 120 entries
+    "long_window": dict(n=[8, 12, 10], m=[4, 3], dep=[[0, 1], [2]], U=[2, 2, 1], bdep=[[0, 1], [1, 2], [2, 0]],
+                        N=3, T=23, K=3),
 }
 
 
