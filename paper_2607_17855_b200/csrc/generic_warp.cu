@@ -331,6 +331,27 @@ __device__ R bdep_future_lane(const BiDev &md, int f0, int s, const R *q, const 
     if (pos < 0) continue;
     const int PB = md.PB[h];
     const R *Yh = Y + yo;
+    if (k == 1) {   // the factor's own previous state only: the weighted tensor's entry is the message
+      acc += Yh[s];
+      continue;
+    }
+    if (k == 2) {   // one other parent: a strided dot product with its belief, no odometer
+      const int go = md.bdep[h][1 - pos], no = md.n[go];
+      const R *qo = q + md.offp[go];
+      // parents in list order, last fastest: entry (d0, d1) sits at d0 * n1 + d1
+      const int n1 = md.n[md.bdep[h][1]];
+      const R *y = Yh + (pos == 0 ? s * n1 : s);
+      const int st = pos == 0 ? 1 : n1;
+      R a0 = (R)0, a1 = (R)0;
+      int i = 0;
+      for (; i + 1 < no; i += 2) {
+        a0 = fma(qo[i], y[i * st], a0);
+        a1 = fma(qo[i + 1], y[(i + 1) * st], a1);
+      }
+      if (i < no) a0 = fma(qo[i], y[i * st], a0);
+      acc += a0 + a1;
+      continue;
+    }
     const int others = PB / md.n[f0];
     int dig[BI_MAX_RANK], nj[BI_MAX_RANK], op[BI_MAX_RANK], str[BI_MAX_RANK];
     int stride = 1;
