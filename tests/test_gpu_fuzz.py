@@ -101,3 +101,32 @@ def test_random_models_with_observation_vectors(block):
         assert err <= (1e-5 if arith == "f64" else 5e-3), (case, algo, arith, md.last_kernel, err)
         md.close()
     print(kernels)
+
+
+@pytest.mark.parametrize("block", range(2))
+def test_random_models_with_several_parents_per_transition(block):
+    """Transitions that read up to four factors' previous states, on random structures: filtering (the
+    CTA kernel forms the parents' products once per factor and step) and VMP (the window kernel's table
+    of parent offsets, its one-, two- and many-parent forms of the future message)."""
+    kernels = {}
+    for case in range(block * 12, block * 12 + 12):
+        rng = np.random.default_rng(990000 + case)
+        F = int(rng.integers(1, 5))
+        n = [int(rng.integers(1, 9)) for _ in range(F)]
+        M = int(rng.integers(1, 4))
+        dep = [[int(x) for x in rng.choice(F, size=int(rng.integers(1, min(F, 3) + 1)), replace=False)] for _ in range(M)]
+        m = [int(rng.integers(1, 5)) for _ in range(M)]
+        U = [int(rng.integers(1, 3)) for _ in range(F)]
+        bdep = [[int(x) for x in rng.choice(F, size=int(rng.integers(1, min(F, 4) + 1)), replace=False)] for _ in range(F)]
+        N = int(rng.choice([1, 3, 8, 40]))
+        T = int(rng.choice([1, 2, 5, 9, 17]))
+        K = int(rng.integers(1, 5))
+        sparsity, b_sparsity = float(rng.choice([0.0, 0.5])), float(rng.choice([0.0, 0.5]))
+        A, B, D = make_model(rng, n, m, dep, U, 1, sparsity=sparsity, d_alpha=1.0, bdep=bdep, b_sparsity=b_sparsity)
+        obs, act = sample_streams(rng, n, m, dep, U, 1, A, B, D, N, T, bdep=bdep)
+        w = Workload(name=f"bdepfuzz{case}", algo="filter", n=np.asarray(n, np.int32), m=np.asarray(m, np.int32),
+                     dep=dep, U=np.asarray(U, np.int32), G=1, A=A, B=B, D=D, N=N, T=T, K=K, obs=obs, act=act, bdep=bdep)
+        for algo in ("filter", "vmp"):
+            res = check_workload(w, algo, agents=range(0, N, max(1, N // 8)))
+            kernels[res["kernel"]] = kernels.get(res["kernel"], 0) + 1
+    print(kernels)
